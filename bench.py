@@ -1,0 +1,386 @@
+#!/usr/bin/env python
+"""Benchmark of the PISA forward hot path (pyramid -> routing -> block-sparse attention).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl ours|reference]
+
+One "step" is one pass of the whole path over one batch of synthetic input.  Prints ONE JSON line
+(rank 0).  `value` is forward tokens/s with inputs resident in HBM; `e2e` is the same metric through
+pisa_forward_host (pinned host tensors in, host tensors out, copies inside the timed region).
+`--impl reference` times the CPU oracle, as it stands, on a bounded sample of the same workload.
+Multi-GPU: the path shards over independent (batch, KV head) units with no exchange step, so every
+rank runs its own replica of the workload (weak scaling) and no collective is on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import pisa_synth as S  # noqa: E402
+
+METRIC = "pisa_fwd_tokens_per_s_128k_ctx"
+UNIT = "tokens/s"
+
+
+def get_workload(name: str) -> S.Workload:
+    if name in S.WORKLOADS:
+        return S.WORKLOADS[name]
+    if name.startswith("cfg5_"):
+        return S.sweep_workload(int(name.split("_")[1]))
+    raise SystemExit(f"unknown workload {name}")
+
+
+def describe(w: S.Workload) -> str:
+    return (f"{w.name}: B={w.B} Hq={w.Hq} Hkv={w.Hkv} d={w.d} N={w.N} causal C={w.C} g={w.g} K={w.K} "
+            f"{w.dtype} {w.structure} seed={w.seed}")
+
+
+# ------------------------------------------------------------------ algorithmic work counts
+
+def work_counts(w: S.Workload) -> dict:
+    """Integer bookkeeping of what one forward pass must touch (depends on shapes only, not data):
+    scored (token, node) pairs per level and selected (token, block) pairs."""
+    M = [w.N, -(-w.N // w.C)]
+    while M[-1] > 1:
+        M.append(-(-M[-1] // w.g))
+    L = len(M) - 1
+    inter_pairs = 0      # (token, candidate) pairs scored from child summaries, summed over levels >= 2
+    leaf_pairs = 0       # (token, leaf) pairs scored from raw keys
+    sel_pairs = 0        # (token, selected leaf) pairs
+    for c in range(M[1]):
+        toks = min(w.C, w.N - c * w.C)
+        n_kept = 1
+        kept_has_anc = True
+        for l in range(L, 0, -1):
+            span = w.g ** (l - 1)
+            anc = c // span
+            if l == L:
+                nV = 1
+            else:
+                # children of the kept nodes; those of the current ancestor beyond anc are dropped
+                anc_up = c // (w.g ** l)
+                full = (n_kept - 1) * w.g
+                nV = full + (anc - anc_up * w.g + 1)
+            forced = len({0, anc, (c - 1) // span if c >= 1 else 0})
+            if nV > w.K:
+                if l >= 2:
+                    inter_pairs += toks * (nV - forced)
+                else:
+                    leaf_pairs += toks * (nV - forced)
+                n_kept = w.K
+            else:
+                n_kept = nV
+        sel_pairs += toks * n_kept
+    units = w.B * w.Hkv
+    G = w.Hq // w.Hkv
+    es = 2 if w.dtype == "bf16" else 4
+    return {
+        "inter_flops": 2.0 * inter_pairs * w.g * G * w.d * units,
+        "leaf_flops": 2.0 * leaf_pairs * w.C * G * w.d * units,
+        "attn_flops": 4.0 * sel_pairs * w.C * G * w.d * units,
+        "pyramid_bytes": float(w.B * w.N * w.Hkv * w.d * es + w.B * w.Hkv * sum(M[1:]) * w.d * es),
+        "hbm_min_bytes": float(w.B * w.N * ((2 * w.Hq + 2 * w.Hkv) * w.d * es + w.Hq * 4 + w.Hkv * w.K * 4)),
+        "sel_pairs": sel_pairs * units, "leaf_pairs": leaf_pairs * units, "inter_pairs": inter_pairs * units,
+    }
+
+
+# ------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.lines = []
+        self.proc = None
+        self.gpu_id = gpu_id
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------ CPU oracle legs
+
+def oracle_sample_rate(w: S.Workload, tensors: dict, n_queries: int, seed: int = 0):
+    """Times the oracle (as it stands) on one KV head's pyramid plus `n_queries` sampled queries of
+    that head (routing + attention for the G heads of the group); returns the whole-workload
+    tokens/s this extrapolates to, the seconds spent and a description of the sample."""
+    from oracle import pisa_oracle as O
+    try:
+        from threadpoolctl import threadpool_limits
+        ctx = threadpool_limits(limits=1)
+    except Exception:  # pragma: no cover
+        import contextlib
+        ctx = contextlib.nullcontext()
+    rng = np.random.default_rng(seed)
+    h = int(rng.integers(0, w.Hkv))
+    ps = np.sort(rng.integers(0, w.N, size=n_queries))
+    with ctx:
+        prob = O.Problem(tensors["q"], tensors["k"], tensors["v"], C=w.C, g=w.g, K=w.K, dtype=w.dtype)
+        t0 = time.perf_counter()
+        prob.head(0, h)                                   # converts the head's keys and pools its pyramid
+        t1 = time.perf_counter()
+        tri = np.stack([np.zeros_like(ps), np.full_like(ps, h), ps], axis=1)
+        idx, _ = prob.route_all(tri)
+        prob.attend_all(tri, idx)
+        t2 = time.perf_counter()
+    per_head = (t1 - t0) + (t2 - t1) / n_queries * w.N
+    total = per_head * w.B * w.Hkv
+    return (w.B * w.N) / total, (t2 - t0), (f"pyramid of 1 of {w.B * w.Hkv} (batch, KV head) units in full + {n_queries} "
+                                           f"uniformly sampled query positions of it (route + attention of its "
+                                           f"{w.Hq // w.Hkv} heads), scaled by N/{n_queries} and by the unit count")
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = get_workload(args.workload)
+    tensors = S.make_inputs(w)
+    nq = args.ref_queries
+    for _ in range(args.warmup):
+        oracle_sample_rate(w, tensors, max(4, nq // 8), seed=99)
+    t0 = time.perf_counter()
+    rates = []
+    for s in range(args.steps):
+        r, _, sample = oracle_sample_rate(w, tensors, nq, seed=s)
+        rates.append(r)
+    wall = time.perf_counter() - t0
+    value = float(len(rates) / sum(1.0 / r for r in rates))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": wall / max(1, args.steps) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": describe(w)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------ our arm
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2609_31093_b200 as P
+    from paper_2609_31093_b200 import binding as PB
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    w0 = get_workload(args.workload)
+    w = dataclasses.replace(w0, seed=w0.seed + 1000 * rank)       # every rank its own replica
+    impl = {"auto": PB.IMPL_AUTO, "simt": PB.IMPL_SIMT, "tensor": PB.IMPL_TENSOR}[args.path]
+    p = P.Params.from_workload(w, impl=impl)
+    tensors = S.make_inputs(w)
+    tdt = p.torch_dtype
+
+    def host(a):
+        t = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if w.dtype == "bf16" else torch.from_numpy(a)
+        return t.pin_memory()
+
+    qh, kh, vh = host(tensors["q"]), host(tensors["k"]), host(tensors["v"])
+    q, k, v = qh.cuda(non_blocking=True), kh.cuda(non_blocking=True), vh.cuda(non_blocking=True)
+    pyramid = PB.alloc_pyramid(p)
+    idx = torch.empty((w.B, w.Hkv, w.N, w.K), dtype=torch.int32, device="cuda")
+    out = torch.empty_like(q)
+    lse = torch.empty((w.B, w.Hq, w.N), dtype=torch.float32, device="cuda")
+    ws = PB.alloc_workspace(p, PB.OP_FORWARD)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    def step():
+        P.pisa_forward(p, q, k, v, pyramid, idx, out, lse, ws)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    st = P.read_status(ws)
+    if st != 0:
+        raise SystemExit(f"device status {st} after warm-up")
+
+    P.set_stage_timing(True)
+    sampler = ClockSampler(str(torch.cuda.get_device_properties(local).uuid) if hasattr(
+        torch.cuda.get_device_properties(local), "uuid") else str(local))
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    stage = np.zeros(3)
+    barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    l0 = P.launch_count()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+        stage += np.asarray(P.get_stage_ms())       # waits for this step's last stage event
+    ev1.record()
+    torch.cuda.synchronize()
+    launches = P.launch_count() - l0
+    clocks = sampler.stop()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    P.set_stage_timing(False)
+    stage /= args.steps
+
+    # end to end through the host-buffer entry point
+    arena = PB.alloc_workspace(p, PB.OP_FORWARD_HOST)
+    out_h = torch.empty(q.shape, dtype=tdt).pin_memory()
+    lse_h = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    for _ in range(2):
+        P.pisa_forward_host(p, qh, kh, vh, out_h, lse_h, None, arena)
+    barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        P.pisa_forward_host(p, qh, kh, vh, out_h, lse_h, None, arena)
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    if world > 1:
+        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = t.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    tokens = w.B * w.N
+    value = world * tokens * args.steps / (ms * 1e-3)
+    e2e_value = world * tokens * e2e_steps / (e2e_ms * 1e-3)
+    wc = work_counts(w)
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    hbm_peak = peaks.get("hbm_gbs", 6650.0)
+    tens_peak = peaks.get("bf16_tflops_sustained", 1400.0)
+    peak_src = "measured" if peaks else "fallback"
+    es = 2 if w.dtype == "bf16" else 4
+    # dominant stage -> roofline entry.  Attention and routing are contractions (tensor bound);
+    # the pyramid is one streaming pass over k (HBM bound).
+    names = ["pyramid", "route", "attn"]
+    dom = int(np.argmax(stage))
+    if dom == 0:
+        roof = {"kernel": "pyramid", "bound": "hbm", "achieved": wc["pyramid_bytes"] / (stage[0] * 1e-3) / 1e9,
+                "peak": hbm_peak, "unit": "GB/s"}
+    else:
+        flops = wc["attn_flops"] if dom == 2 else wc["leaf_flops"] + wc["inter_flops"]
+        roof = {"kernel": names[dom], "bound": "tensor", "achieved": flops / (stage[dom] * 1e-3) / 1e12,
+                "peak": tens_peak, "unit": "TFLOP/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["peak_source"] = peak_src
+    roof["traffic"] = None
+    stages = {
+        "pyramid_us": stage[0] * 1e3, "route_us": stage[1] * 1e3, "attn_us": stage[2] * 1e3,
+        "pyramid_gbs": wc["pyramid_bytes"] / (stage[0] * 1e-3) / 1e9,
+        "route_tflops": (wc["leaf_flops"] + wc["inter_flops"]) / (stage[1] * 1e-3) / 1e12,
+        "attn_tflops": wc["attn_flops"] / (stage[2] * 1e-3) / 1e12,
+        "whole_step_hbm_min_gbs": wc["hbm_min_bytes"] / (ms / args.steps * 1e-3) / 1e9,
+    }
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        val, secs, sample = oracle_sample_rate(w, tensors, args.ref_queries)
+        cpu = {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample, "seconds": secs}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": describe(w0), "path": args.path,
+                   "l2": f"inputs larger than L2 (q {q.numel() * es / 1e6:.0f} MB, k+v {2 * k.numel() * es / 1e6:.0f} MB)",
+                   "replicas": world},
+        "stages": stages, "roofline": roof, "cpu_baseline": cpu,
+        "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps,
+                "h2d_bytes_per_step": int((q.numel() + 2 * k.numel()) * es),
+                "d2h_bytes_per_step": int(out.numel() * es + lse.numel() * 4)},
+        "gpu_launches": int(launches), "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4")
+    ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--ref-queries", type=int, default=192)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,156 @@
+/*
+ * libpisa — forward hot path of Pyramid Sparse Attention (PISA) on NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every pointer is caller-owned.  "device" pointers are CUDA global memory of the
+ * current device, "host" pointers are ordinary host memory.  The library never allocates or
+ * frees device memory and, except where stated, never synchronises: all work is enqueued on
+ * `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream).  Scratch comes
+ * from a caller-provided workspace whose size is queried with pisa_workspace_bytes().
+ *
+ * Notation follows the paper (Sec. 3.1-3.2): N tokens, Hq query heads, Hkv KV heads
+ * (G = Hq/Hkv heads share KV head h: heads h*G .. h*G+G-1), head dim d, leaf block size C,
+ * pooling fan-in g above the leaves, block budget K, M_1 = ceil(N/C) leaf blocks,
+ * M_{l+1} = ceil(M_l/g), L = first level with M_L = 1.  Everything is 0-based.
+ *
+ * Tensor layouts (d contiguous, strides in elements, order (b, n, h)):
+ *   q, out : [B, N, Hq,  d]      k, v : [B, N, Hkv, d]
+ *   idx    : int32 [B, Hkv, N, K]   ascending leaf-block ids, padded with -1
+ *   lse    : float [B, Hq, N]       natural-log softmax denominator
+ *   pyramid: levels 1..L back to back, level l = [B, Hkv, M_l, d] in the input dtype,
+ *            at the element offsets pisa_pyramid_layout() reports.
+ *
+ * All functions return a pisa_status (0 = OK).  Nothing aborts, throws or traps the GPU.
+ */
+#ifndef PISA_H_
+#define PISA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PISA_VERSION 100
+
+typedef enum {
+  PISA_OK = 0,
+  PISA_ERR_INVALID_ARG = -1,         /* null pointer, non-positive size, Hq % Hkv != 0, K < 3, g < 2 */
+  PISA_ERR_UNSUPPORTED = -2,         /* causal = 0, d / G / g*K outside the built range, unknown dtype */
+  PISA_ERR_WORKSPACE_TOO_SMALL = -3,
+  PISA_ERR_CUDA = -4,                /* a launch or copy failed; pisa_last_cuda_error() has the text */
+  PISA_ERR_TIMEOUT = -5,             /* a bounded device-side wait gave up (read from the status word) */
+  PISA_ERR_BOUNDS = -6               /* a device-side index check failed (read from the status word) */
+} pisa_status;
+
+enum { PISA_BF16 = 0, PISA_FP32 = 1 };
+/* Block score (Sec. 4.3, App. A.2): PISA = log-sum-exp, PISA-1 = mean logit, PISA-2 = mean + var/2 */
+enum { PISA_SCORE_LSE = 0, PISA_SCORE_MEAN = 1, PISA_SCORE_MEAN_VAR = 2 };
+/* operations a workspace can be sized for */
+enum { PISA_OP_ROUTE = 0, PISA_OP_BSA = 1, PISA_OP_FORWARD = 2, PISA_OP_FLAT = 3, PISA_OP_FORWARD_HOST = 4 };
+/* implementation selector (params.impl): AUTO picks the tensor-core path where it applies */
+enum { PISA_IMPL_AUTO = 0, PISA_IMPL_SIMT = 1, PISA_IMPL_TENSOR = 2 };
+
+typedef struct {
+  int32_t B, N, Hq, Hkv, d, C, g, K; /* prefill self-attention: N queries = N keys            */
+  int32_t causal;                    /* must be 1: the paper defines only the causal LM case   */
+  int32_t dtype;                     /* PISA_BF16 | PISA_FP32: q, k, v, out, summaries share it */
+  int32_t score_mode;                /* PISA_SCORE_*                                            */
+  int32_t impl;                      /* PISA_IMPL_*                                             */
+  float   scale;                     /* logit scale; 0 => 1/sqrt(d)  (Eq. "block scores")       */
+  int32_t reserved;
+  int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3]; /* elements, (b, n, h); all 0 => dense */
+} pisa_params_t;
+
+int pisa_version(void);
+const char* pisa_status_string(int status);
+/* text of the last CUDA error seen by this thread's calls ("" if none) */
+const char* pisa_last_cuda_error(void);
+
+/*
+ * Hierarchy of Sec. 3.2 "Fine-to-coarse block aggregation".
+ * Host-only.  Writes L, M[0..L] (M[0] = N; caller provides >= 34 entries) and level_off[0..L]
+ * (element offset of level l inside the pyramid buffer; level_off[0] is unused), and the
+ * buffer size in bytes.  Any output pointer may be NULL.
+ */
+int pisa_pyramid_layout(const pisa_params_t* p, int32_t* L, int32_t* M, int64_t* level_off, size_t* bytes);
+
+/* Host-only.  Bytes of device workspace `op` needs for these parameters (256-byte aligned base). */
+int pisa_workspace_bytes(const pisa_params_t* p, int op, size_t* bytes);
+
+/*
+ * Eq. "mean pyramid": level 1 = mean of each leaf block's keys, level l+1 = unweighted mean of
+ * the valid level-l children (fp32 accumulation, each level rounded to the input dtype and pooled
+ * from the stored level below).  k: device [B,N,Hkv,d]; pyramid: device, pisa_pyramid_layout bytes.
+ */
+int pisa_build_pyramid(const pisa_params_t* p, const void* k, void* pyramid, void* stream);
+
+/*
+ * Coarse-to-fine Top-K block selection (Sec. 3.2 "Coarse-to-fine block selection", Eq. "direct
+ * child LSE", Eq. "grouped score", App. B "Causal masking"): per (b, KV head, query token) start
+ * from the root, drop candidates that do not exist or start after the query's leaf, keep all if
+ * at most K remain, else keep the forced nodes (ancestors of the first / previous / current leaf,
+ * never scored, counted inside K) plus the best of the rest by the group-summed score of their
+ * children (g child summaries above the leaves, the C raw keys at the leaves), ties to the smaller
+ * index; expand the kept nodes' children; the kept leaves are the result.
+ *   q, k, pyramid : device inputs            idx : device int32 [B,Hkv,N,K] output
+ *   margin        : device float [B,Hkv,N] or NULL — smallest relative gap between the last kept
+ *                   and the first dropped score over the scored levels (+inf if nothing was cut);
+ *                   gap = (u_kept - u_dropped) / max(|u_kept|, 1)
+ *   ws / ws_bytes : device workspace sized for PISA_OP_ROUTE
+ */
+int pisa_route(const pisa_params_t* p, const void* q, const void* k, const void* pyramid,
+               int32_t* idx, float* margin, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Eq. "selected sparse attention" with the causal mask inside selected blocks (App. B): for every
+ * query head, softmax over the tokens j <= t of the leaf blocks idx[b, h, t, :] (entries < 0 are
+ * skipped) with logits q.k*scale, fp32 accumulation.  out: device [B,N,Hq,d] in the input dtype;
+ * lse: device float [B,Hq,N].  Workspace sized for PISA_OP_BSA.
+ */
+int pisa_bsa_fwd(const pisa_params_t* p, const void* q, const void* k, const void* v, const int32_t* idx,
+                 void* out, float* lse, void* ws, size_t ws_bytes, void* stream);
+
+/* pyramid -> route -> attention in one call.  pyramid and idx are outputs too (kept for reuse). */
+int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const void* v, void* pyramid,
+                 int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The same forward pass for callers that hold HOST tensors: copies q, k, v to the device arena
+ * (`ws`, sized for PISA_OP_FORWARD_HOST), runs pisa_forward there, copies out, lse and (if not
+ * NULL) idx back to host memory, and waits for the stream.  Host buffers should be pinned for
+ * full copy bandwidth; strides must be dense.  This is the one entry point that synchronises.
+ */
+int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_host, const void* v_host,
+                      void* out_host, float* lse_host, int32_t* idx_host,
+                      void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Flat block selection (Sec. 3.1, the O(N^2/C) reference point): score every eligible leaf with
+ * q . level-1 summary * scale, softmax over the eligible leaves within each query head (App. C),
+ * sum over the group's heads, keep the forced leaves plus the best of the rest.
+ */
+int pisa_flat_select(const pisa_params_t* p, const void* q, const void* pyramid, int32_t* idx,
+                     void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Reads the device status word a workspace carries (written by bounded waits and index checks).
+ * Call after the stream has been synchronised.  *status receives a pisa_status.
+ */
+int pisa_read_status(const void* ws, int32_t* status);
+
+/*
+ * Device time of the stages of the last pisa_forward / pisa_forward_host issued by this thread,
+ * in milliseconds: pyramid, route, attention (measured with CUDA events on the call's stream).
+ * Recording is off unless pisa_set_stage_timing(1) was called; the getter waits for the events.
+ */
+int pisa_set_stage_timing(int enable);
+int pisa_get_stage_ms(float* pyramid_ms, float* route_ms, float* attn_ms);
+
+/* Number of kernels this process has launched through the library so far (host counter). */
+unsigned long long pisa_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PISA_H_ */

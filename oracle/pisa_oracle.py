@@ -304,51 +304,77 @@ def attend_query(q_vec: np.ndarray, k_bh: np.ndarray, v_bh: np.ndarray, p: int, 
 # --------------------------------------------------------------------------
 
 class Problem:
-    """Holds fp64 views of one problem's tensors and its pyramid."""
+    """One problem's tensors in storage form plus lazily built per-(b, KV head) fp64 views
+    (raw keys, values, pyramid levels), so that sampled queries of a long sequence stay cheap."""
 
     def __init__(self, q, k, v, *, C: int, g: int, K: int, dtype: str, scale: Optional[float] = None,
-                 mode: str = "lse", pyramid: Optional[List[Optional[np.ndarray]]] = None):
-        self.q = load_storage(q, dtype)   # [B, N, Hq, d]
-        self.k = load_storage(k, dtype)   # [B, N, Hkv, d]
-        self.v = load_storage(v, dtype) if v is not None else None
-        self.B, self.N, self.Hq, self.d = self.q.shape
-        self.Hkv = self.k.shape[2]
+                 mode: str = "lse"):
+        self.q_st, self.k_st, self.v_st = q, k, v      # [B,N,Hq,d], [B,N,Hkv,d] storage form
+        self.B, self.N, self.Hq, self.d = q.shape
+        self.Hkv = k.shape[2]
         assert self.Hq % self.Hkv == 0
         self.G = self.Hq // self.Hkv
         self.C, self.g, self.K, self.dtype, self.mode = C, g, K, dtype, mode
         self.scale = (1.0 / math.sqrt(self.d)) if scale is None else float(scale)
         self.M = hierarchy(self.N, C, g)
         self.L = len(self.M) - 1
-        self.levels = pyramid if pyramid is not None else build_pyramid(self.k, C, g, dtype)
+        self._cache_key = None
+        self._cache = None
 
-    def _bh(self, b: int, h: int):
-        lv = [None] + [self.levels[l][b, h] for l in range(1, self.L + 1)]
-        return lv, self.k[b, :, h, :]
+    # fp64 views -----------------------------------------------------------
+    def head(self, b: int, h: int):
+        """(k_bh [N,d], v_bh [N,d] or None, levels_bh[0..L] with levels_bh[l] [M_l,d])."""
+        if self._cache_key != (b, h):
+            k_bh = load_storage(np.ascontiguousarray(self.k_st[b, :, h, :]), self.dtype)
+            v_bh = None if self.v_st is None else load_storage(np.ascontiguousarray(self.v_st[b, :, h, :]), self.dtype)
+            lv = build_pyramid(k_bh[None, :, None, :], self.C, self.g, self.dtype)
+            levels = [None] + [lv[l][0, 0] for l in range(1, self.L + 1)]
+            self._cache_key, self._cache = (b, h), (k_bh, v_bh, levels)
+        return self._cache
 
+    def q_group(self, b: int, h: int, p: int) -> np.ndarray:
+        return load_storage(np.ascontiguousarray(self.q_st[b, p, h * self.G:(h + 1) * self.G, :]), self.dtype)
+
+    def pyramid(self) -> List[Optional[np.ndarray]]:
+        """All levels, fp64 stored values, levels[l] [B,Hkv,M_l,d]."""
+        out: List[Optional[np.ndarray]] = [None] + [np.empty((self.B, self.Hkv, self.M[l], self.d))
+                                                     for l in range(1, self.L + 1)]
+        for b in range(self.B):
+            for h in range(self.Hkv):
+                lv = self.head(b, h)[2]
+                for l in range(1, self.L + 1):
+                    out[l][b, h] = lv[l]
+        return out
+
+    # per-query ------------------------------------------------------------
     def route(self, b: int, h: int, p: int, trace: Optional[list] = None):
-        lv, k_bh = self._bh(b, h)
-        qh = self.q[b, p, h * self.G:(h + 1) * self.G, :]
-        return route_query(qh, lv, k_bh, p, self.C, self.g, self.K, self.scale, self.mode, trace)
+        k_bh, _, lv = self.head(b, h)
+        return route_query(self.q_group(b, h, p), lv, k_bh, p, self.C, self.g, self.K, self.scale, self.mode, trace)
 
     def flat_lse(self, b: int, h: int, p: int):
-        qh = self.q[b, p, h * self.G:(h + 1) * self.G, :]
-        return flat_lse_select(qh, self.k[b, :, h, :], p, self.C, self.K, self.scale, self.mode)
+        k_bh, _, _ = self.head(b, h)
+        return flat_lse_select(self.q_group(b, h, p), k_bh, p, self.C, self.K, self.scale, self.mode)
 
     def flat_mean(self, b: int, h: int, p: int):
-        qh = self.q[b, p, h * self.G:(h + 1) * self.G, :]
-        return flat_mean_select(qh, self.levels[1][b, h], p, self.C, self.K, self.scale)
+        _, _, lv = self.head(b, h)
+        return flat_mean_select(self.q_group(b, h, p), lv[1], p, self.C, self.K, self.scale)
 
     def attend(self, b: int, hq: int, p: int, blocks: Sequence[int]):
         h = hq // self.G
-        return attend_query(self.q[b, p, hq, :], self.k[b, :, h, :], self.v[b, :, h, :], p, blocks,
-                            self.C, self.scale)
+        k_bh, v_bh, _ = self.head(b, h)
+        qv = self.q_group(b, h, p)[hq - h * self.G]
+        return attend_query(qv, k_bh, v_bh, p, blocks, self.C, self.scale)
+
+    # drivers (loops over queries; use on small shapes or samples) -----------
+    def all_triples(self) -> np.ndarray:
+        return np.asarray([(b, h, p) for b in range(self.B) for h in range(self.Hkv)
+                           for p in range(self.N)], dtype=np.int64)
 
     def route_all(self, triples: Optional[np.ndarray] = None):
         """idx int32 [S, K], margin fp64 [S] for the given (b, h, p) triples
         (default: every query, in (b, h, p) order)."""
         if triples is None:
-            triples = np.asarray([(b, h, p) for b in range(self.B) for h in range(self.Hkv)
-                                  for p in range(self.N)], dtype=np.int64)
+            triples = self.all_triples()
         idx = np.empty((len(triples), self.K), dtype=np.int32)
         margin = np.empty((len(triples),), dtype=np.float64)
         for s, (b, h, p) in enumerate(triples):
@@ -357,14 +383,19 @@ class Problem:
             margin[s] = m
         return idx, margin
 
-    def forward_samples(self, triples: np.ndarray, idx: Optional[np.ndarray] = None):
-        """For each (b, h, p): route (unless idx is given), then attend for the G heads.
-        Returns idx [S,K], margin [S], out fp64 [S, G, d] (stored values), lse [S, G]."""
+    def flat_mean_all(self, triples: np.ndarray):
+        idx = np.empty((len(triples), self.K), dtype=np.int32)
+        margin = np.empty((len(triples),), dtype=np.float64)
+        for s, (b, h, p) in enumerate(triples):
+            I, m = self.flat_mean(int(b), int(h), int(p))
+            idx[s] = pad_indices(I, self.K)
+            margin[s] = m
+        return idx, margin
+
+    def attend_all(self, triples: np.ndarray, idx: np.ndarray):
+        """For each (b, h, p) and its block list idx[s]: the G heads' outputs (stored values,
+        fp64 [S, G, d]) and natural-log denominators [S, G]."""
         S = len(triples)
-        if idx is None:
-            idx, margin = self.route_all(triples)
-        else:
-            margin = np.full((S,), np.inf)
         out = np.empty((S, self.G, self.d), dtype=np.float64)
         lse = np.empty((S, self.G), dtype=np.float64)
         for s, (b, h, p) in enumerate(triples):
@@ -372,4 +403,4 @@ class Problem:
                 o, l = self.attend(int(b), int(h) * self.G + j, int(p), idx[s])
                 out[s, j] = o
                 lse[s, j] = l
-        return idx, margin, round_to_storage(out, self.dtype), lse
+        return round_to_storage(out, self.dtype), lse

@@ -1,0 +1,189 @@
+"""ctypes binding with the C ABI's names (include/pisa.h).  No arithmetic happens here."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libpisa.so")
+_lib = None
+
+BF16, FP32 = 0, 1
+SCORE_LSE, SCORE_MEAN, SCORE_MEAN_VAR = 0, 1, 2
+OP_ROUTE, OP_BSA, OP_FORWARD, OP_FLAT, OP_FORWARD_HOST = 0, 1, 2, 3, 4
+IMPL_AUTO, IMPL_SIMT, IMPL_TENSOR = 0, 1, 2
+_SCORE = {"lse": SCORE_LSE, "mean": SCORE_MEAN, "mean_var": SCORE_MEAN_VAR}
+
+
+class PisaError(RuntimeError):
+    pass
+
+
+class _CParams(C.Structure):
+    _fields_ = [
+        ("B", C.c_int32), ("N", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32),
+        ("d", C.c_int32), ("C", C.c_int32), ("g", C.c_int32), ("K", C.c_int32),
+        ("causal", C.c_int32), ("dtype", C.c_int32), ("score_mode", C.c_int32), ("impl", C.c_int32),
+        ("scale", C.c_float), ("reserved", C.c_int32),
+        ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 3),
+        ("v_stride", C.c_int64 * 3), ("o_stride", C.c_int64 * 3),
+    ]
+
+
+def lib():
+    """Loads libpisa.so (once).  There is no fallback: a missing library is an error."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise PisaError(f"{_LIB_PATH} is missing: build it with `python -m paper_2609_31093_b200.build`")
+    L = C.CDLL(_LIB_PATH)
+    vp, i32p, f32p, szp = C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_float), C.POINTER(C.c_size_t)
+    pp = C.POINTER(_CParams)
+    L.pisa_version.restype = C.c_int
+    L.pisa_status_string.restype = C.c_char_p
+    L.pisa_status_string.argtypes = [C.c_int]
+    L.pisa_last_cuda_error.restype = C.c_char_p
+    L.pisa_pyramid_layout.argtypes = [pp, i32p, i32p, C.POINTER(C.c_int64), szp]
+    L.pisa_workspace_bytes.argtypes = [pp, C.c_int, szp]
+    L.pisa_build_pyramid.argtypes = [pp, vp, vp, vp]
+    L.pisa_route.argtypes = [pp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+    L.pisa_bsa_fwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+    L.pisa_forward.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+    L.pisa_forward_host.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+    L.pisa_flat_select.argtypes = [pp, vp, vp, vp, vp, C.c_size_t, vp]
+    L.pisa_read_status.argtypes = [vp, i32p]
+    L.pisa_set_stage_timing.argtypes = [C.c_int]
+    L.pisa_get_stage_ms.argtypes = [f32p, f32p, f32p]
+    L.pisa_launch_count.restype = C.c_ulonglong
+    for name in ("pisa_pyramid_layout", "pisa_workspace_bytes", "pisa_build_pyramid", "pisa_route",
+                 "pisa_bsa_fwd", "pisa_forward", "pisa_forward_host", "pisa_flat_select", "pisa_read_status",
+                 "pisa_set_stage_timing", "pisa_get_stage_ms"):
+        getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def _check(st: int, what: str):
+    if st != 0:
+        L = lib()
+        msg = L.pisa_status_string(st).decode()
+        cuda = L.pisa_last_cuda_error().decode()
+        raise PisaError(f"{what}: {msg} ({st})" + (f" [{cuda}]" if cuda and st == -4 else ""))
+
+
+class Params:
+    """Problem description in the paper's notation; mirrors pisa_params_t."""
+
+    def __init__(self, B, N, Hq, Hkv, d, C, g, K, dtype="bf16", score_mode="lse", scale=0.0, impl=IMPL_AUTO):
+        self.c = _CParams()
+        self.c.B, self.c.N, self.c.Hq, self.c.Hkv = B, N, Hq, Hkv
+        self.c.d, self.c.C, self.c.g, self.c.K = d, C, g, K
+        self.c.causal = 1
+        self.c.dtype = BF16 if dtype == "bf16" else FP32
+        self.c.score_mode = _SCORE[score_mode] if isinstance(score_mode, str) else int(score_mode)
+        self.c.impl = impl
+        self.c.scale = float(scale)
+        self.dtype = dtype
+        self.B, self.N, self.Hq, self.Hkv, self.d, self.C, self.g, self.K = B, N, Hq, Hkv, d, C, g, K
+
+    @classmethod
+    def from_workload(cls, w, B=None, **kw):
+        return cls(w.B if B is None else B, w.N, w.Hq, w.Hkv, w.d, w.C, w.g, w.K, dtype=w.dtype, **kw)
+
+    @property
+    def torch_dtype(self):
+        return torch.bfloat16 if self.dtype == "bf16" else torch.float32
+
+    def ref(self):
+        return C.byref(self.c)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def pyramid_layout(p: Params) -> Tuple[int, list, list, int]:
+    """(L, M[0..L], level_off[0..L] in elements, bytes)."""
+    L = C.c_int32()
+    M = (C.c_int32 * 34)()
+    off = (C.c_int64 * 34)()
+    nbytes = C.c_size_t()
+    _check(lib().pisa_pyramid_layout(p.ref(), C.byref(L), M, off, C.byref(nbytes)), "pisa_pyramid_layout")
+    return L.value, list(M[:L.value + 1]), list(off[:L.value + 1]), nbytes.value
+
+
+def workspace_bytes(p: Params, op: int) -> int:
+    n = C.c_size_t()
+    _check(lib().pisa_workspace_bytes(p.ref(), op, C.byref(n)), "pisa_workspace_bytes")
+    return n.value
+
+
+def alloc_pyramid(p: Params, device="cuda") -> torch.Tensor:
+    nbytes = pyramid_layout(p)[3]
+    es = 2 if p.dtype == "bf16" else 4
+    return torch.empty(nbytes // es, dtype=p.torch_dtype, device=device)
+
+
+def alloc_workspace(p: Params, op: int, device="cuda") -> torch.Tensor:
+    return torch.zeros(max(workspace_bytes(p, op), 256), dtype=torch.uint8, device=device)
+
+
+def pisa_build_pyramid(p: Params, k: torch.Tensor, pyramid: torch.Tensor):
+    _check(lib().pisa_build_pyramid(p.ref(), _ptr(k), _ptr(pyramid), _stream()), "pisa_build_pyramid")
+
+
+def pisa_route(p: Params, q, k, pyramid, idx, margin, ws):
+    _check(lib().pisa_route(p.ref(), _ptr(q), _ptr(k), _ptr(pyramid), _ptr(idx), _ptr(margin), _ptr(ws),
+                            ws.numel(), _stream()), "pisa_route")
+
+
+def pisa_bsa_fwd(p: Params, q, k, v, idx, out, lse, ws):
+    _check(lib().pisa_bsa_fwd(p.ref(), _ptr(q), _ptr(k), _ptr(v), _ptr(idx), _ptr(out), _ptr(lse), _ptr(ws),
+                              ws.numel(), _stream()), "pisa_bsa_fwd")
+
+
+def pisa_forward(p: Params, q, k, v, pyramid, idx, out, lse, ws):
+    _check(lib().pisa_forward(p.ref(), _ptr(q), _ptr(k), _ptr(v), _ptr(pyramid), _ptr(idx), _ptr(out),
+                              _ptr(lse), _ptr(ws), ws.numel(), _stream()), "pisa_forward")
+
+
+def pisa_forward_host(p: Params, q_host, k_host, v_host, out_host, lse_host, idx_host, ws):
+    """Host tensors in, host tensors out; `ws` is a device arena sized for OP_FORWARD_HOST."""
+    for t in (q_host, k_host, v_host, out_host, lse_host):
+        assert not t.is_cuda and t.is_contiguous()
+    _check(lib().pisa_forward_host(p.ref(), _ptr(q_host), _ptr(k_host), _ptr(v_host), _ptr(out_host),
+                                   _ptr(lse_host), _ptr(idx_host), _ptr(ws), ws.numel(), _stream()),
+           "pisa_forward_host")
+
+
+def pisa_flat_select(p: Params, q, pyramid, idx, ws):
+    _check(lib().pisa_flat_select(p.ref(), _ptr(q), _ptr(pyramid), _ptr(idx), _ptr(ws), ws.numel(), _stream()),
+           "pisa_flat_select")
+
+
+def read_status(ws) -> int:
+    st = C.c_int32()
+    _check(lib().pisa_read_status(_ptr(ws), C.byref(st)), "pisa_read_status")
+    return st.value
+
+
+def set_stage_timing(enable: bool):
+    _check(lib().pisa_set_stage_timing(1 if enable else 0), "pisa_set_stage_timing")
+
+
+def get_stage_ms() -> Tuple[float, float, float]:
+    a, b, c = C.c_float(), C.c_float(), C.c_float()
+    _check(lib().pisa_get_stage_ms(C.byref(a), C.byref(b), C.byref(c)), "pisa_get_stage_ms")
+    return a.value, b.value, c.value
+
+
+def launch_count() -> int:
+    return int(lib().pisa_launch_count())

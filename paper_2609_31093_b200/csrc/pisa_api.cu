@@ -1,0 +1,366 @@
+// C-ABI entry points of libpisa: argument checks, hierarchy/workspace layout, stage sequencing.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "pisa_common.cuh"
+#include "pisa_tensor.cuh"
+
+namespace pisa {
+
+static thread_local char g_cuda_err[512] = "";
+static thread_local bool g_timing = false;
+static thread_local cudaEvent_t g_ev[4] = {nullptr, nullptr, nullptr, nullptr};
+static thread_local bool g_ev_valid = false;
+
+void record_cuda_error(const char* what, cudaError_t e) {
+  snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", what, cudaGetErrorString(e));
+}
+
+static unsigned long long g_launches = 0;   // kernels launched by this process (relaxed counter)
+
+int check_launch(const char* what) {
+  __atomic_fetch_add(&g_launches, 1ull, __ATOMIC_RELAXED);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    record_cuda_error(what, e);
+    return PISA_ERR_CUDA;
+  }
+  return PISA_OK;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static size_t elem_size(int dtype) { return dtype == PISA_BF16 ? 2 : 4; }
+
+int resolve(const pisa_params_t* p, Geometry* g) {
+  if (p == nullptr || g == nullptr) return PISA_ERR_INVALID_ARG;
+  if (p->B <= 0 || p->N <= 0 || p->Hq <= 0 || p->Hkv <= 0 || p->d <= 0 || p->C <= 0) return PISA_ERR_INVALID_ARG;
+  if (p->Hq % p->Hkv != 0 || p->K < 3 || p->g < 2) return PISA_ERR_INVALID_ARG;
+  if (p->dtype != PISA_BF16 && p->dtype != PISA_FP32) return PISA_ERR_UNSUPPORTED;
+  if (p->causal != 1) return PISA_ERR_UNSUPPORTED;
+  if (p->score_mode < PISA_SCORE_LSE || p->score_mode > PISA_SCORE_MEAN_VAR) return PISA_ERR_UNSUPPORTED;
+  if (p->impl < PISA_IMPL_AUTO || p->impl > PISA_IMPL_TENSOR) return PISA_ERR_INVALID_ARG;
+  if (p->d != 32 && p->d != 64 && p->d != 128) return PISA_ERR_UNSUPPORTED;
+  const int G = p->Hq / p->Hkv;
+  if (G != 1 && G != 2 && G != 4 && G != 8 && G != 16) return PISA_ERR_UNSUPPORTED;
+  if (p->K > kMaxK || (long long)p->g * p->K > kMaxCand) return PISA_ERR_UNSUPPORTED;
+  memset(g, 0, sizeof(*g));
+  g->B = p->B; g->N = p->N; g->Hq = p->Hq; g->Hkv = p->Hkv; g->G = G; g->d = p->d;
+  g->C = p->C; g->g = p->g; g->K = p->K;
+  g->score_mode = p->score_mode;
+  g->scale = (p->scale == 0.f) ? (float)(1.0 / sqrt((double)p->d)) : p->scale;
+  g->M[0] = p->N;
+  g->M[1] = (p->N + p->C - 1) / p->C;
+  int L = 1;
+  while (g->M[L] > 1) {
+    if (L + 1 >= kMaxLevels) return PISA_ERR_UNSUPPORTED;
+    g->M[L + 1] = (g->M[L] + p->g - 1) / p->g;
+    ++L;
+  }
+  g->L = L;
+  long long span = 1;
+  for (int l = 1; l < kMaxLevels; ++l) {
+    g->span[l] = span;
+    if (span < (1LL << 40)) span *= p->g;
+  }
+  // levels back to back, each starting on a 256-byte boundary
+  const size_t es = elem_size(p->dtype);
+  size_t off = 0;
+  for (int l = 1; l <= L; ++l) {
+    g->level_off[l] = (long long)(off / es);
+    off += align_up((size_t)p->B * p->Hkv * g->M[l] * p->d * es, 256);
+  }
+  auto strides = [&](const int64_t* in, long long* out, int H) {
+    if (in[0] == 0 && in[1] == 0 && in[2] == 0) {
+      out[2] = p->d; out[1] = (long long)H * p->d; out[0] = (long long)p->N * H * p->d;
+    } else {
+      out[0] = in[0]; out[1] = in[1]; out[2] = in[2];
+    }
+  };
+  strides(p->q_stride, g->qs, p->Hq);
+  strides(p->k_stride, g->ks, p->Hkv);
+  strides(p->v_stride, g->vs, p->Hkv);
+  strides(p->o_stride, g->os, p->Hq);
+  // 16-byte vector loads need every row to start on a 16-byte boundary
+  const long long vec = 16 / (long long)es;
+  for (int i = 0; i < 3; ++i)
+    if (g->qs[i] % vec || g->ks[i] % vec || g->vs[i] % vec || g->os[i] % vec) return PISA_ERR_INVALID_ARG;
+  return PISA_OK;
+}
+
+static size_t pyramid_bytes_dtype(const Geometry& g, int dtype) {
+  const size_t es = elem_size(dtype);
+  return (size_t)g.level_off[g.L] * es + align_up((size_t)g.B * g.Hkv * g.M[g.L] * g.d * es, 256);
+}
+
+static bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+static bool use_tensor(const pisa_params_t* p, const Geometry& g) {
+  if (p->impl == PISA_IMPL_SIMT) return false;
+  return tensor_path_supported(g, p->dtype);
+}
+
+static size_t route_ws_bytes(const pisa_params_t* p, const Geometry& g) {
+  size_t b = kStatusBytes;
+  if (use_tensor(p, g)) b += tensor_route_workspace_bytes(g);
+  return b;
+}
+static size_t bsa_ws_bytes(const pisa_params_t* p, const Geometry& g) {
+  size_t b = kStatusBytes;
+  if (use_tensor(p, g)) b += tensor_bsa_workspace_bytes(g);
+  return b;
+}
+
+static int clear_status(void* ws, cudaStream_t s) {
+  cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, s);
+  if (e != cudaSuccess) { record_cuda_error("status memset", e); return PISA_ERR_CUDA; }
+  return PISA_OK;
+}
+
+static int do_route(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* pyr,
+                    int32_t* idx, float* margin, void* ws, size_t ws_bytes, cudaStream_t s) {
+  if (ws_bytes < route_ws_bytes(p, g)) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  if (use_tensor(p, g))
+    return tensor_route(g, p->dtype, q, k, pyr, idx, margin, (char*)ws + kStatusBytes, (int32_t*)ws, s);
+  return launch_route_simt(g, p->dtype, q, k, pyr, idx, margin, s);
+}
+
+static int do_bsa(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v,
+                  const int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes, cudaStream_t s) {
+  if (ws_bytes < bsa_ws_bytes(p, g)) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  if (use_tensor(p, g))
+    return tensor_bsa(g, p->dtype, q, k, v, idx, out, lse, (char*)ws + kStatusBytes, (int32_t*)ws, s);
+  return launch_bsa_simt(g, p->dtype, q, k, v, idx, out, lse, s);
+}
+
+static void stage_mark(int i, cudaStream_t s) {
+  if (!g_timing) return;
+  if (!g_ev_valid) {
+    for (int j = 0; j < 4; ++j) cudaEventCreate(&g_ev[j]);
+    g_ev_valid = true;
+  }
+  cudaEventRecord(g_ev[i], s);
+}
+
+static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v,
+                      void* pyr, int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes,
+                      cudaStream_t s) {
+  size_t need = route_ws_bytes(p, g);
+  const size_t need_b = bsa_ws_bytes(p, g);
+  if (need_b > need) need = need_b;
+  if (ws_bytes < need) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  int st = clear_status(ws, s);
+  if (st != PISA_OK) return st;
+  stage_mark(0, s);
+  st = launch_pyramid(g, p->dtype, k, pyr, s);
+  if (st != PISA_OK) return st;
+  stage_mark(1, s);
+  st = do_route(p, g, q, k, pyr, idx, nullptr, ws, ws_bytes, s);
+  if (st != PISA_OK) return st;
+  stage_mark(2, s);
+  st = do_bsa(p, g, q, k, v, idx, out, lse, ws, ws_bytes, s);
+  stage_mark(3, s);
+  return st;
+}
+
+}  // namespace pisa
+
+using namespace pisa;
+
+extern "C" {
+
+int pisa_version(void) { return PISA_VERSION; }
+
+const char* pisa_status_string(int status) {
+  switch (status) {
+    case PISA_OK: return "ok";
+    case PISA_ERR_INVALID_ARG: return "invalid argument";
+    case PISA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case PISA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case PISA_ERR_CUDA: return "CUDA error";
+    case PISA_ERR_TIMEOUT: return "device-side wait timed out";
+    case PISA_ERR_BOUNDS: return "device-side index check failed";
+    default: return "unknown status";
+  }
+}
+
+const char* pisa_last_cuda_error(void) { return g_cuda_err; }
+
+int pisa_pyramid_layout(const pisa_params_t* p, int32_t* L, int32_t* M, int64_t* level_off, size_t* bytes) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (L) *L = g.L;
+  for (int l = 0; l <= g.L; ++l) {
+    if (M) M[l] = g.M[l];
+    if (level_off) level_off[l] = g.level_off[l];
+  }
+  if (bytes) *bytes = pyramid_bytes_dtype(g, p->dtype);
+  return PISA_OK;
+}
+
+int pisa_workspace_bytes(const pisa_params_t* p, int op, size_t* bytes) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (bytes == nullptr) return PISA_ERR_INVALID_ARG;
+  const size_t es = elem_size(p->dtype);
+  const size_t r = route_ws_bytes(p, g), a = bsa_ws_bytes(p, g);
+  const size_t f = r > a ? r : a;
+  switch (op) {
+    case PISA_OP_ROUTE: *bytes = r; break;
+    case PISA_OP_BSA: *bytes = a; break;
+    case PISA_OP_FORWARD: *bytes = f; break;
+    case PISA_OP_FLAT: *bytes = kStatusBytes; break;
+    case PISA_OP_FORWARD_HOST: {
+      size_t t = align_up(f, 256);
+      t += align_up((size_t)g.B * g.N * g.Hq * g.d * es, 256) * 2;      // q, out
+      t += align_up((size_t)g.B * g.N * g.Hkv * g.d * es, 256) * 2;     // k, v
+      t += align_up((size_t)g.B * g.Hq * g.N * sizeof(float), 256);      // lse
+      t += align_up((size_t)g.B * g.Hkv * g.N * g.K * sizeof(int32_t), 256);  // idx
+      t += align_up(pyramid_bytes_dtype(g, p->dtype), 256);
+      *bytes = t;
+      break;
+    }
+    default: return PISA_ERR_INVALID_ARG;
+  }
+  return PISA_OK;
+}
+
+int pisa_build_pyramid(const pisa_params_t* p, const void* k, void* pyramid, void* stream) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (k == nullptr || pyramid == nullptr || misaligned(k) || misaligned(pyramid)) return PISA_ERR_INVALID_ARG;
+  return launch_pyramid(g, p->dtype, k, pyramid, (cudaStream_t)stream);
+}
+
+int pisa_route(const pisa_params_t* p, const void* q, const void* k, const void* pyramid, int32_t* idx,
+               float* margin, void* ws, size_t ws_bytes, void* stream) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (!q || !k || !pyramid || !idx || !ws || misaligned(q) || misaligned(k) || misaligned(pyramid) ||
+      misaligned(ws))
+    return PISA_ERR_INVALID_ARG;
+  st = clear_status(ws, (cudaStream_t)stream);
+  if (st != PISA_OK) return st;
+  return do_route(p, g, q, k, pyramid, idx, margin, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+int pisa_bsa_fwd(const pisa_params_t* p, const void* q, const void* k, const void* v, const int32_t* idx,
+                 void* out, float* lse, void* ws, size_t ws_bytes, void* stream) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (!q || !k || !v || !idx || !out || !lse || !ws || misaligned(q) || misaligned(k) || misaligned(v) ||
+      misaligned(out) || misaligned(ws))
+    return PISA_ERR_INVALID_ARG;
+  st = clear_status(ws, (cudaStream_t)stream);
+  if (st != PISA_OK) return st;
+  return do_bsa(p, g, q, k, v, idx, out, lse, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const void* v, void* pyramid,
+                 int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes, void* stream) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (!q || !k || !v || !pyramid || !idx || !out || !lse || !ws || misaligned(q) || misaligned(k) ||
+      misaligned(v) || misaligned(pyramid) || misaligned(out) || misaligned(ws))
+    return PISA_ERR_INVALID_ARG;
+  return do_forward(p, g, q, k, v, pyramid, idx, out, lse, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_host, const void* v_host,
+                      void* out_host, float* lse_host, int32_t* idx_host, void* ws, size_t ws_bytes,
+                      void* stream) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (!q_host || !k_host || !v_host || !out_host || !lse_host || !ws || misaligned(ws)) return PISA_ERR_INVALID_ARG;
+  for (int i = 0; i < 3; ++i)
+    if (p->q_stride[i] || p->k_stride[i] || p->v_stride[i] || p->o_stride[i]) return PISA_ERR_INVALID_ARG;
+  size_t need = 0;
+  st = pisa_workspace_bytes(p, PISA_OP_FORWARD_HOST, &need);
+  if (st != PISA_OK) return st;
+  if (ws_bytes < need) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t es = elem_size(p->dtype);
+  size_t fwd = 0;
+  pisa_workspace_bytes(p, PISA_OP_FORWARD, &fwd);
+  const size_t qb = (size_t)g.B * g.N * g.Hq * g.d * es, kb = (size_t)g.B * g.N * g.Hkv * g.d * es;
+  const size_t lb = (size_t)g.B * g.Hq * g.N * sizeof(float);
+  const size_t ib = (size_t)g.B * g.Hkv * g.N * g.K * sizeof(int32_t);
+  char* base = (char*)ws;
+  size_t off = align_up(fwd, 256);
+  char* dq = base + off; off += align_up(qb, 256);
+  char* dout = base + off; off += align_up(qb, 256);
+  char* dk = base + off; off += align_up(kb, 256);
+  char* dv = base + off; off += align_up(kb, 256);
+  char* dl = base + off; off += align_up(lb, 256);
+  char* di = base + off; off += align_up(ib, 256);
+  char* dp = base + off;
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, s)) != cudaSuccess) {
+    record_cuda_error("h2d copy", e);
+    return PISA_ERR_CUDA;
+  }
+  st = do_forward(p, g, dq, dk, dv, dp, (int32_t*)di, dout, (float*)dl, ws, fwd, s);
+  if (st != PISA_OK) return st;
+  if ((e = cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, s)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(lse_host, dl, lb, cudaMemcpyDeviceToHost, s)) != cudaSuccess ||
+      (idx_host && (e = cudaMemcpyAsync(idx_host, di, ib, cudaMemcpyDeviceToHost, s)) != cudaSuccess) ||
+      (e = cudaStreamSynchronize(s)) != cudaSuccess) {
+    record_cuda_error("d2h copy", e);
+    return PISA_ERR_CUDA;
+  }
+  return PISA_OK;
+}
+
+int pisa_flat_select(const pisa_params_t* p, const void* q, const void* pyramid, int32_t* idx, void* ws,
+                     size_t ws_bytes, void* stream) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (!q || !pyramid || !idx || !ws || misaligned(q) || misaligned(pyramid)) return PISA_ERR_INVALID_ARG;
+  if (ws_bytes < kStatusBytes) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  st = clear_status(ws, (cudaStream_t)stream);
+  if (st != PISA_OK) return st;
+  return launch_flat_simt(g, p->dtype, q, pyramid, idx, (cudaStream_t)stream);
+}
+
+int pisa_read_status(const void* ws, int32_t* status) {
+  if (!ws || !status) return PISA_ERR_INVALID_ARG;
+  int32_t word = 0;
+  cudaError_t e = cudaMemcpy(&word, ws, sizeof(word), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) { record_cuda_error("status read", e); return PISA_ERR_CUDA; }
+  *status = word;
+  return PISA_OK;
+}
+
+unsigned long long pisa_launch_count(void) { return __atomic_load_n(&g_launches, __ATOMIC_RELAXED); }
+
+int pisa_set_stage_timing(int enable) {
+  g_timing = enable != 0;
+  return PISA_OK;
+}
+
+int pisa_get_stage_ms(float* pyramid_ms, float* route_ms, float* attn_ms) {
+  if (!g_timing || !g_ev_valid) return PISA_ERR_INVALID_ARG;
+  cudaError_t e = cudaEventSynchronize(g_ev[3]);
+  if (e != cudaSuccess) { record_cuda_error("stage events", e); return PISA_ERR_CUDA; }
+  float a = 0, b = 0, c = 0;
+  cudaEventElapsedTime(&a, g_ev[0], g_ev[1]);
+  cudaEventElapsedTime(&b, g_ev[1], g_ev[2]);
+  cudaEventElapsedTime(&c, g_ev[2], g_ev[3]);
+  if (pyramid_ms) *pyramid_ms = a;
+  if (route_ms) *route_ms = b;
+  if (attn_ms) *attn_ms = c;
+  return PISA_OK;
+}
+
+}  // extern "C"

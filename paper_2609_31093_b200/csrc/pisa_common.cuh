@@ -1,0 +1,89 @@
+// Internal declarations shared by the libpisa translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pisa.h"
+
+namespace pisa {
+
+constexpr int kMaxLevels = 34;     // ceil(log2(2^31)) + slack
+constexpr int kMaxK = 32;          // block budget (one kept node per lane)
+constexpr int kMaxCand = 128;      // g*K, candidates per level
+constexpr int kWarp = 32;
+
+// Resolved problem description handed to the kernels (by value).
+struct Geometry {
+  int B, N, Hq, Hkv, G, d, C, g, K, L;
+  int score_mode;
+  float scale;
+  int M[kMaxLevels];               // M[0] = N, M[l] = blocks at level l
+  long long span[kMaxLevels];      // span[l] = g^(l-1): leaves under one level-l node
+  long long level_off[kMaxLevels]; // element offset of level l in the pyramid buffer
+  long long qs[3], ks[3], vs[3], os[3];  // element strides (b, n, h)
+};
+
+// Status word at the start of every workspace (device int32[4]; [0] = pisa_status).
+constexpr size_t kStatusBytes = 256;
+
+int resolve(const pisa_params_t* p, Geometry* g);                // validates; returns pisa_status
+size_t align_up(size_t x, size_t a);
+
+// launchers (each returns a pisa_status; errors come from cudaGetLastError after the launch)
+int launch_pyramid(const Geometry& g, int dtype, const void* k, void* pyramid, cudaStream_t s);
+int launch_route_simt(const Geometry& g, int dtype, const void* q, const void* k, const void* pyramid,
+                      int32_t* idx, float* margin, cudaStream_t s);
+// stage 1 of the two-stage schedule: leaf candidates [B,Hkv,N,gK] (-1 padded), margin so far
+int launch_route_stage1_simt(const Geometry& g, int dtype, const void* q, const void* pyramid,
+                             int32_t* cand_out, float* margin, cudaStream_t s);
+int launch_route_final_topk(const Geometry& g, const int32_t* cand, const float* scores, int32_t* idx,
+                            float* margin, cudaStream_t s);
+int launch_bsa_simt(const Geometry& g, int dtype, const void* q, const void* k, const void* v,
+                    const int32_t* idx, void* out, float* lse, cudaStream_t s);
+int launch_flat_simt(const Geometry& g, int dtype, const void* q, const void* pyramid, int32_t* idx,
+                     cudaStream_t s);
+
+int check_launch(const char* what);   // cudaGetLastError -> pisa_status, records the text
+void record_cuda_error(const char* what, cudaError_t e);
+
+// ---------------------------------------------------------------- device helpers
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+  static constexpr int kVec = 4;                       // elements per 16-byte chunk
+  __device__ static inline void load_chunk(const float* p, float (&x)[4]) {
+    float4 v = *reinterpret_cast<const float4*>(p);
+    x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+  }
+  __device__ static inline float to_float(float v) { return v; }
+  __device__ static inline float from_float(float v) { return v; }
+};
+template <> struct Elem<__nv_bfloat16> {
+  static constexpr int kVec = 8;
+  __device__ static inline void load_chunk(const __nv_bfloat16* p, float (&x)[8]) {
+    uint4 v = *reinterpret_cast<const uint4*>(p);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      x[2 * i] = __uint_as_float(w[i] << 16);
+      x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+  __device__ static inline float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+  __device__ static inline __nv_bfloat16 from_float(float v) { return __float2bfloat16_rn(v); }
+};
+
+__device__ inline float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ inline float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+}  // namespace pisa

@@ -1,0 +1,17 @@
+// Tensor-core (tcgen05 / TMEM) path: key-block-major leaf scoring and block-sparse attention.
+#pragma once
+
+#include "pisa_common.cuh"
+
+namespace pisa {
+
+bool tensor_path_supported(const Geometry& g, int dtype);
+size_t tensor_route_workspace_bytes(const Geometry& g);
+size_t tensor_bsa_workspace_bytes(const Geometry& g);
+// ws points past the status word; status is the workspace's status word
+int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, const void* pyramid, int32_t* idx,
+                 float* margin, void* ws, int32_t* status, cudaStream_t s);
+int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const void* v, const int32_t* idx,
+               void* out, float* lse, void* ws, int32_t* status, cudaStream_t s);
+
+}  // namespace pisa

@@ -1,0 +1,134 @@
+"""Shared helpers for the GPU parity tests: move seeded inputs to the device, run the C-ABI entry
+points through the binding, and compare with the oracle under the stated tolerances."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import paper_2609_31093_b200 as P
+from paper_2609_31093_b200 import binding as PB
+from oracle import pisa_oracle as O
+import pisa_synth as S
+
+TIE_BAND = 1e-4          # relative tie band on the K-th score (index sets may differ inside it)
+BF16_MAX_ABS, BF16_MEAN_ABS = 2e-2, 2e-3
+FP32_TOL = 1e-4
+
+
+def to_torch(a: np.ndarray, dtype: str, device="cuda") -> torch.Tensor:
+    if dtype == "bf16":
+        return torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).to(device)
+    return torch.from_numpy(a).to(device)
+
+
+def from_torch(t: torch.Tensor, dtype: str) -> np.ndarray:
+    """Device tensor -> storage form (uint16 bits or float32)."""
+    if dtype == "bf16":
+        return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+    return t.detach().cpu().contiguous().numpy()
+
+
+class Device:
+    """q, k, v of one workload on the GPU plus every buffer the entry points need."""
+
+    def __init__(self, w: S.Workload, tensors: dict, impl=PB.IMPL_AUTO, score_mode="lse", B=None):
+        self.w = w
+        Bn = tensors["q"].shape[0]
+        self.p = P.Params(Bn, w.N, w.Hq, w.Hkv, w.d, w.C, w.g, w.K, dtype=w.dtype, impl=impl,
+                          score_mode=score_mode)
+        self.q = to_torch(tensors["q"], w.dtype)
+        self.k = to_torch(tensors["k"], w.dtype)
+        self.v = to_torch(tensors["v"], w.dtype)
+        self.L, self.M, self.level_off, self.pyr_bytes = P.pyramid_layout(self.p)
+        self.pyramid = PB.alloc_pyramid(self.p)
+        self.idx = torch.full((Bn, w.Hkv, w.N, w.K), -7, dtype=torch.int32, device="cuda")
+        self.margin = torch.zeros((Bn, w.Hkv, w.N), dtype=torch.float32, device="cuda")
+        self.out = torch.zeros_like(self.q)
+        self.lse = torch.zeros((Bn, w.Hq, w.N), dtype=torch.float32, device="cuda")
+        self.ws = PB.alloc_workspace(self.p, PB.OP_FORWARD)
+
+    def level(self, l: int) -> torch.Tensor:
+        n = self.p.B * self.w.Hkv * self.M[l] * self.w.d
+        return self.pyramid[self.level_off[l]:self.level_off[l] + n].view(self.p.B, self.w.Hkv, self.M[l], self.w.d)
+
+    def load_oracle_pyramid(self, levels):
+        """Copy the oracle's stored pyramid into the device buffer (isolates routing from pooling)."""
+        for l in range(1, self.L + 1):
+            st = O.f64_to_bf16_bits(levels[l]) if self.w.dtype == "bf16" else levels[l].astype(np.float32)
+            self.level(l).copy_(to_torch(st, self.w.dtype))
+
+    def build_pyramid(self):
+        P.pisa_build_pyramid(self.p, self.k, self.pyramid)
+
+    def route(self, with_margin=True):
+        P.pisa_route(self.p, self.q, self.k, self.pyramid, self.idx, self.margin if with_margin else None, self.ws)
+
+    def bsa(self, idx=None):
+        P.pisa_bsa_fwd(self.p, self.q, self.k, self.v, self.idx if idx is None else idx, self.out, self.lse, self.ws)
+
+    def forward(self):
+        P.pisa_forward(self.p, self.q, self.k, self.v, self.pyramid, self.idx, self.out, self.lse, self.ws)
+
+    def flat(self):
+        P.pisa_flat_select(self.p, self.q, self.pyramid, self.idx, self.ws)
+
+    def sync_status(self):
+        torch.cuda.synchronize()
+        return P.read_status(self.ws)
+
+
+def oracle_problem(w: S.Workload, tensors: dict, mode="lse") -> O.Problem:
+    return O.Problem(tensors["q"], tensors["k"], tensors["v"], C=w.C, g=w.g, K=w.K, dtype=w.dtype, mode=mode)
+
+
+def gather_idx(idx_dev: torch.Tensor, triples: np.ndarray) -> np.ndarray:
+    t = torch.from_numpy(triples).to(idx_dev.device)
+    return idx_dev[t[:, 0], t[:, 1], t[:, 2]].cpu().numpy()
+
+
+def compare_index_sets(idx_gpu: np.ndarray, idx_ref: np.ndarray, margin_ref: np.ndarray, band=TIE_BAND):
+    """Rows must be equal (both ascending, -1 padded) except where the oracle's cut margin lies in
+    the tie band.  Returns (rows differing, of those outside the band, rows inside the band)."""
+    diff = np.any(idx_gpu != idx_ref, axis=1)
+    in_band = margin_ref <= band
+    bad = diff & ~in_band
+    return int(diff.sum()), int(bad.sum()), int(in_band.sum())
+
+
+def check_index_rows_valid(idx_gpu: np.ndarray, triples: np.ndarray, w: S.Workload):
+    """What must hold for any correct answer, tie band or not: count = min(K, c+1), ascending,
+    distinct, causal, forced blocks present, -1 padding at the end."""
+    for row, (b, h, p) in zip(idx_gpu, triples):
+        c = int(p) // w.C
+        n = min(w.K, c + 1)
+        sel = row[:n]
+        assert np.all(row[n:] == -1), (p, row)
+        assert np.all(sel >= 0) and np.all(sel <= c), (p, row)
+        assert np.all(np.diff(sel) > 0), (p, row)
+        for f in (0, max(c - 1, 0), c):
+            assert f in sel, (p, row)
+
+
+def check_outputs(out_gpu: np.ndarray, lse_gpu: np.ndarray, out_ref: np.ndarray, lse_ref: np.ndarray, dtype: str):
+    """out_* are fp64 arrays of stored values; tolerances per dtype as stated for the path."""
+    err = np.abs(out_gpu - out_ref)
+    lerr = np.abs(lse_gpu - lse_ref)
+    if dtype == "bf16":
+        assert err.max() <= BF16_MAX_ABS, f"max abs {err.max()}"
+        assert err.mean() <= BF16_MEAN_ABS, f"mean abs {err.mean()}"
+        assert lerr.max() <= 1e-3 * max(1.0, np.abs(lse_ref).max()), f"lse {lerr.max()}"
+    else:
+        assert err.max() <= FP32_TOL, f"max abs {err.max()}"
+        assert lerr.max() <= FP32_TOL * max(1.0, np.abs(lse_ref).max()), f"lse {lerr.max()}"
+    return float(err.max()), float(err.mean()), float(lerr.max())
+
+
+def gather_out(dev: Device, triples: np.ndarray):
+    """GPU outputs for the sampled (b, h, p): fp64 [S, G, d] stored values and lse [S, G]."""
+    w = dev.w
+    G = w.Hq // w.Hkv
+    t = torch.from_numpy(triples).to("cuda")
+    heads = t[:, 1:2] * G + torch.arange(G, device="cuda")[None, :]           # [S, G]
+    o = dev.out[t[:, 0:1], t[:, 2:3], heads]                                   # [S, G, d]
+    l = dev.lse[t[:, 0:1], heads, t[:, 2:3]]                                   # [S, G]
+    return o.to(torch.float64).cpu().numpy(), l.to(torch.float64).cpu().numpy()

@@ -1,0 +1,84 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, validates its arguments, and lays out the hierarchy as the paper defines it."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2609_31093_b200 as P
+from paper_2609_31093_b200 import binding as PB
+from oracle import pisa_oracle as O
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    names = []
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if not fn.endswith(".h"):
+            continue
+        src = open(os.path.join(ROOT, "include", fn)).read()
+        src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+        names += re.findall(r"\b(pisa_[a-z_0-9]+)\s*\(", src)
+    return sorted(set(names))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = P.lib()
+    decl = _declared_functions()
+    assert len(decl) >= 12
+    for name in decl:
+        assert hasattr(lib, name), name
+    assert lib.pisa_version() == 100
+
+
+@pytest.mark.parametrize("N,C,g", [(1024, 64, 2), (32768, 64, 4), (131072, 128, 2), (1000, 24, 3), (50, 64, 2),
+                                   (524288, 64, 2)])
+def test_pyramid_layout_matches_paper_hierarchy(N, C, g):
+    p = P.Params(1, N, 4, 2, 64, C, g, 8)
+    L, M, off, nbytes = P.pyramid_layout(p)
+    assert M == O.hierarchy(N, C, g) and L == len(M) - 1
+    es = 2
+    for l in range(1, L):
+        assert off[l + 1] * es >= off[l] * es + 2 * M[l] * 64 * es      # levels do not overlap
+        assert (off[l] * es) % 256 == 0
+    assert nbytes >= off[L] * es + 2 * M[L] * 64 * es
+
+
+def test_argument_validation():
+    ok = P.Params(1, 1024, 4, 2, 64, 64, 2, 8)
+    assert P.workspace_bytes(ok, PB.OP_FORWARD) >= 256
+    bad = [
+        dict(Hq=3),            # Hq % Hkv != 0
+        dict(K=2),             # K < 3 (three forced blocks)
+        dict(g=1),
+        dict(N=0),
+    ]
+    for kw in bad:
+        args = dict(B=1, N=1024, Hq=4, Hkv=2, d=64, C=64, g=2, K=8)
+        args.update(kw)
+        with pytest.raises(P.PisaError, match="invalid argument"):
+            P.workspace_bytes(P.Params(**args), PB.OP_FORWARD)
+    for kw in [dict(d=48), dict(K=64), dict(g=8, K=32), dict(Hq=6, Hkv=2)]:
+        args = dict(B=1, N=1024, Hq=4, Hkv=2, d=64, C=64, g=2, K=8)
+        args.update(kw)
+        with pytest.raises(P.PisaError, match="unsupported"):
+            P.workspace_bytes(P.Params(**args), PB.OP_FORWARD)
+    nc = P.Params(1, 1024, 4, 2, 64, 64, 2, 8)
+    nc.c.causal = 0
+    with pytest.raises(P.PisaError, match="unsupported"):
+        P.workspace_bytes(nc, PB.OP_FORWARD)
+    # null pointers are rejected before anything is launched (no GPU needed to see that)
+    lib = P.lib()
+    assert lib.pisa_build_pyramid(ok.ref(), None, None, None) == -1
+    assert lib.pisa_route(ok.ref(), None, None, None, None, None, None, 0, None) == -1
+    assert lib.pisa_forward(ok.ref(), None, None, None, None, None, None, None, None, 0, None) == -1
+    assert lib.pisa_status_string(-3).decode() == "workspace too small"
+
+
+def test_host_arena_size_covers_all_tensors():
+    p = P.Params(1, 8192, 16, 16, 128, 64, 2, 16)
+    es = 2
+    need = 2 * 8192 * 16 * 128 * es * 2 + 16 * 8192 * 4 + 16 * 8192 * 16 * 4 + P.pyramid_layout(p)[3]
+    assert P.workspace_bytes(p, PB.OP_FORWARD_HOST) >= need

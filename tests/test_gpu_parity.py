@@ -1,0 +1,183 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Index sets: exact, except rows whose oracle cut margin lies inside the 1e-4 relative tie
+band (counted).  Outputs: max-abs 2e-2 / mean-abs 2e-3 for bf16 inputs, 1e-4 for fp32."""
+import numpy as np
+import pytest
+import torch
+
+import pisa_synth as S
+from oracle import pisa_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+import pisa_testlib as T  # noqa: E402
+from paper_2609_31093_b200 import binding as PB  # noqa: E402
+
+SMALL = {
+    # name: workload (sizes the oracle finishes in seconds; several tiles and ragged tails)
+    "tiny_fp32": S.WORKLOADS["cfg1"],
+    "gqa4_ragged": S.Workload("gqa4_ragged", 1, 2048 + 37, 8, 2, 128, 64, 2, 4, "bf16", 101, "iid"),
+    "fan4": S.Workload("fan4", 2, 4096, 4, 2, 64, 32, 4, 8, "bf16", 102, "walk"),
+    "mha_k3_fp32": S.Workload("mha_k3_fp32", 1, 1536, 2, 2, 128, 64, 2, 3, "fp32", 103, "iid"),
+    "g16": S.Workload("g16", 1, 3072, 16, 1, 64, 64, 2, 6, "bf16", 104, "iid"),
+    "c128_k32": S.Workload("c128_k32", 1, 16384, 4, 1, 128, 128, 2, 32, "bf16", 105, "needle64"),
+    "one_block": S.Workload("one_block", 1, 50, 2, 1, 32, 64, 2, 4, "fp32", 106, "iid"),
+    "g3_odd": S.Workload("g3_odd", 1, 1000, 2, 1, 32, 24, 3, 5, "fp32", 107, "iid"),
+}
+FULL = ["tiny_fp32", "gqa4_ragged", "mha_k3_fp32", "one_block", "g3_odd"]   # every query compared
+
+
+def _triples(name, w, Bn):
+    if name in FULL:
+        return np.asarray([(b, h, p) for b in range(Bn) for h in range(w.Hkv) for p in range(w.N)], dtype=np.int64)
+    return S.sample_queries(w, 160, B=Bn)
+
+
+@pytest.fixture(scope="module", params=list(SMALL))
+def case(request):
+    name = request.param
+    w = SMALL[name]
+    t = S.make_inputs(w)
+    prob = T.oracle_problem(w, t)
+    tri = _triples(name, w, t["q"].shape[0])
+    return name, w, t, prob, tri
+
+
+def _impls(w):
+    return [PB.IMPL_SIMT, PB.IMPL_AUTO]
+
+
+def test_pyramid_matches_oracle(case):
+    name, w, t, prob, tri = case
+    dev = T.Device(w, t)
+    dev.build_pyramid()
+    assert dev.sync_status() == 0
+    ref = prob.pyramid()
+    for l in range(1, dev.L + 1):
+        got = dev.level(l).to(torch.float64).cpu().numpy()
+        if w.dtype == "fp32":
+            np.testing.assert_allclose(got, ref[l], rtol=2e-6, atol=2e-6)
+        else:
+            # fp32 accumulation vs the oracle's fp64 can flip a bf16 rounding: rare, never more than 1 ulp
+            neq = got != ref[l]
+            assert neq.mean() <= 5e-3, (l, neq.mean())
+            ulp = np.maximum(np.abs(ref[l]), 1e-30) * 2.0 ** -7
+            assert np.all(np.abs(got - ref[l]) <= ulp * 1.001 + 1e-38), l
+
+
+@pytest.mark.parametrize("impl", [PB.IMPL_SIMT, PB.IMPL_AUTO])
+def test_route_matches_oracle(case, impl):
+    name, w, t, prob, tri = case
+    dev = T.Device(w, t, impl=impl)
+    dev.load_oracle_pyramid(prob.pyramid())
+    dev.route()
+    assert dev.sync_status() == 0
+    got = T.gather_idx(dev.idx, tri)
+    ref_idx, ref_margin = prob.route_all(tri)
+    T.check_index_rows_valid(got, tri, w)
+    n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin)
+    print(f"[{name} impl={impl}] rows={len(tri)} differ={n_diff} outside_band={n_bad} band={n_band}")
+    assert n_bad == 0
+    # the margin the library reports agrees with the oracle's where sets agree
+    mg = dev.margin[torch.from_numpy(tri[:, 0]).cuda(), torch.from_numpy(tri[:, 1]).cuda(),
+                    torch.from_numpy(tri[:, 2]).cuda()].cpu().numpy().astype(np.float64)
+    same = ~np.any(got != ref_idx, axis=1)
+    fin = same & np.isfinite(ref_margin)
+    assert np.array_equal(np.isinf(mg[same]), np.isinf(ref_margin[same]))
+    if fin.any():
+        np.testing.assert_allclose(mg[fin], ref_margin[fin], rtol=0, atol=2e-5)
+    # deterministic: a second run gives identical indices
+    first = dev.idx.clone()
+    dev.route()
+    torch.cuda.synchronize()
+    assert torch.equal(first, dev.idx)
+
+
+@pytest.mark.parametrize("impl", [PB.IMPL_SIMT, PB.IMPL_AUTO])
+def test_attention_matches_oracle_on_oracle_indices(case, impl):
+    name, w, t, prob, tri = case
+    if len(tri) > 1200:      # keep the oracle's share of the test to seconds
+        tri = tri[np.random.default_rng(0).choice(len(tri), 1200, replace=False)]
+    dev = T.Device(w, t, impl=impl)
+    ref_idx, _ = prob.route_all(tri)
+    # attention alone: feed the oracle's indices (rows outside the sample keep a valid default)
+    Bn = t["q"].shape[0]
+    idx = torch.full((Bn, w.Hkv, w.N, w.K), -1, dtype=torch.int32)
+    idx[:, :, :, 0] = 0
+    idx[torch.from_numpy(tri[:, 0]), torch.from_numpy(tri[:, 1]), torch.from_numpy(tri[:, 2])] = torch.from_numpy(ref_idx)
+    dev.idx.copy_(idx.cuda())
+    dev.bsa()
+    assert dev.sync_status() == 0
+    out_ref, lse_ref = prob.attend_all(tri, ref_idx)
+    out_gpu, lse_gpu = T.gather_out(dev, tri)
+    stats = T.check_outputs(out_gpu, lse_gpu, out_ref, lse_ref, w.dtype)
+    print(f"[{name} impl={impl}] attention max_abs={stats[0]:.3e} mean_abs={stats[1]:.3e} lse={stats[2]:.3e}")
+
+
+@pytest.mark.parametrize("impl", [PB.IMPL_SIMT, PB.IMPL_AUTO])
+def test_forward_matches_oracle(case, impl):
+    name, w, t, prob, tri = case
+    if len(tri) > 1200:
+        tri = tri[np.random.default_rng(1).choice(len(tri), 1200, replace=False)]
+    dev = T.Device(w, t, impl=impl)
+    dev.forward()
+    assert dev.sync_status() == 0
+    got = T.gather_idx(dev.idx, tri)
+    ref_idx, ref_margin = prob.route_all(tri)
+    T.check_index_rows_valid(got, tri, w)
+    n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin)
+    assert n_bad == 0
+    same = ~np.any(got != ref_idx, axis=1)
+    out_ref, lse_ref = prob.attend_all(tri[same], ref_idx[same])
+    out_gpu, lse_gpu = T.gather_out(dev, tri[same])
+    stats = T.check_outputs(out_gpu, lse_gpu, out_ref, lse_ref, w.dtype)
+    print(f"[{name} impl={impl}] forward rows={len(tri)} differ={n_diff} band={n_band} "
+          f"max_abs={stats[0]:.3e} mean_abs={stats[1]:.3e}")
+
+
+def test_flat_select_matches_oracle(case):
+    name, w, t, prob, tri = case
+    if len(tri) > 1500:
+        tri = tri[np.random.default_rng(2).choice(len(tri), 1500, replace=False)]
+    dev = T.Device(w, t)
+    dev.load_oracle_pyramid(prob.pyramid())
+    dev.flat()
+    assert dev.sync_status() == 0
+    got = T.gather_idx(dev.idx, tri)
+    ref_idx, ref_margin = prob.flat_mean_all(tri)
+    T.check_index_rows_valid(got, tri, w)
+    n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin)
+    print(f"[{name}] flat rows={len(tri)} differ={n_diff} outside_band={n_bad} band={n_band}")
+    assert n_bad == 0
+
+
+@pytest.mark.parametrize("mode", ["mean", "mean_var"])
+def test_score_modes_match_oracle(mode):
+    w = SMALL["gqa4_ragged"]
+    t = S.make_inputs(w)
+    prob = T.oracle_problem(w, t, mode=mode)
+    tri = S.sample_queries(w, 150)
+    dev = T.Device(w, t, impl=PB.IMPL_SIMT, score_mode=mode)
+    dev.load_oracle_pyramid(prob.pyramid())
+    dev.route()
+    assert dev.sync_status() == 0
+    got = T.gather_idx(dev.idx, tri)
+    ref_idx, ref_margin = prob.route_all(tri)
+    n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin)
+    assert n_bad == 0
+
+
+def test_dense_limit_equals_torch_causal_attention():
+    # K*C >= N: the path must reduce to dense causal attention (library routine on the GPU as a
+    # second witness next to the oracle)
+    w = S.Workload("dense", 1, 1024, 4, 2, 64, 64, 2, 16, "bf16", 108, "iid")
+    t = S.make_inputs(w)
+    dev = T.Device(w, t)
+    dev.forward()
+    assert dev.sync_status() == 0
+    q = dev.q.float().permute(0, 2, 1, 3)
+    k = dev.k.float().permute(0, 2, 1, 3).repeat_interleave(2, dim=1)
+    v = dev.v.float().permute(0, 2, 1, 3).repeat_interleave(2, dim=1)
+    ref = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True).permute(0, 2, 1, 3)
+    err = (dev.out.float() - ref).abs()
+    assert err.max().item() <= T.BF16_MAX_ABS and err.mean().item() <= T.BF16_MEAN_ABS

@@ -189,8 +189,8 @@ def _textbook_flat_topk(P, b, h, p):
     c = p // C
     if c + 1 <= K:
         return list(range(c + 1))
-    qh = torch.from_numpy(P.q[b, p, h * G:(h + 1) * G])              # [G, d]
-    kk = torch.from_numpy(P.k[b, :(c - 1) * C, h])                    # leaves 0..c-2, all in the past
+    qh = torch.from_numpy(P.q_group(b, h, p))                         # [G, d]
+    kk = torch.from_numpy(P.head(b, h)[0][:(c - 1) * C])              # leaves 0..c-2, all in the past
     z = (qh @ kk.T) * P.scale                                         # [G, (c-1)C]
     u = torch.logsumexp(z.reshape(G, c - 1, C), dim=2).sum(dim=0)     # [c-1]
     u[0] = -float("inf")                                              # leaf 0 is forced
@@ -331,9 +331,10 @@ def test_attention_equals_dense_causal_when_budget_covers_sequence():
     w = S.Workload("dense", 1, 256, 4, 2, 32, 16, 2, 16, "fp32", 31, "iid")
     P, t = _problem(w)
     assert w.K * w.C >= w.N
-    q = torch.from_numpy(P.q).permute(0, 2, 1, 3)                    # [B, Hq, N, d]
-    k = torch.from_numpy(P.k).permute(0, 2, 1, 3).repeat_interleave(P.G, dim=1)
-    v = torch.from_numpy(P.v).permute(0, 2, 1, 3).repeat_interleave(P.G, dim=1)
+    f64 = lambda a: torch.from_numpy(O.load_storage(a, w.dtype))
+    q = f64(t["q"]).permute(0, 2, 1, 3)                               # [B, Hq, N, d]
+    k = f64(t["k"]).permute(0, 2, 1, 3).repeat_interleave(P.G, dim=1)
+    v = f64(t["v"]).permute(0, 2, 1, 3).repeat_interleave(P.G, dim=1)
     ref = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True).numpy()
     z = (q @ k.transpose(-1, -2)) / math.sqrt(w.d)
     z = z.masked_fill(torch.triu(torch.ones(w.N, w.N, dtype=torch.bool), 1), -float("inf"))
@@ -361,13 +362,15 @@ def test_attention_block_decomposition():
     assert abs(lse - float(torch.logsumexp(lses, 0))) < 1e-12
     wts = torch.softmax(lses, 0).numpy()
     np.testing.assert_allclose(out, sum(wi * o for wi, (o, _) in zip(wts, parts)), atol=1e-12)
-    z = torch.from_numpy(P.k[0, 96:128, 0] @ P.q[0, p, 0]) * P.scale
-    ref = (torch.softmax(z, 0)[:, None] * torch.from_numpy(P.v[0, 96:128, 0])).sum(0).numpy()
+    kk, vv, _ = P.head(0, 0)
+    qv = P.q_group(0, 0, p)[0]
+    z = torch.from_numpy(kk[96:128] @ qv) * P.scale
+    ref = (torch.softmax(z, 0)[:, None] * torch.from_numpy(vv[96:128])).sum(0).numpy()
     np.testing.assert_allclose(parts[1][0], ref, atol=1e-12)
     # causal mask inside the current block: only tokens <= p
-    zc = torch.from_numpy(P.k[0, 480:p + 1, 0] @ P.q[0, p, 0]) * P.scale
+    zc = torch.from_numpy(kk[480:p + 1] @ qv) * P.scale
     assert abs(parts[3][1] - float(torch.logsumexp(zc, 0))) < 1e-12
-    vmin, vmax = P.v[0, :, 0].min(axis=0), P.v[0, :, 0].max(axis=0)
+    vmin, vmax = vv.min(axis=0), vv.max(axis=0)
     assert np.all(out >= vmin) and np.all(out <= vmax)
 
 
@@ -383,8 +386,8 @@ def test_flat_mean_bsa_matches_definition_and_g1_normalisation_invariance():
             if c + 1 <= w.K:
                 assert I == list(range(c + 1))
                 continue
-            qh = torch.from_numpy(P.q[0, p, h * 2:(h + 1) * 2])
-            s = (qh @ torch.from_numpy(P.levels[1][0, h][:c + 1]).T) * P.scale
+            qh = torch.from_numpy(P.q_group(0, h, p))
+            s = (qh @ torch.from_numpy(P.head(0, h)[2][1][:c + 1]).T) * P.scale
             u = torch.softmax(s, dim=1).sum(0)
             forced = sorted({0, c - 1, c})
             u[forced] = -1.0
@@ -396,7 +399,7 @@ def test_flat_mean_bsa_matches_definition_and_g1_normalisation_invariance():
     p = 2000
     c = p // 32
     I, _ = P1.flat_mean(0, 1, p)
-    s = (P1.levels[1][0, 1][:c + 1] @ P1.q[0, p, 1]) * P1.scale
+    s = (P1.head(0, 1)[2][1][:c + 1] @ P1.q_group(0, 1, p)[0]) * P1.scale
     s[[0, c - 1, c]] = -np.inf
     top = np.argsort(-s, kind="stable")[:8 - 3].tolist()
     assert I == sorted({0, c - 1, c} | set(top))
