@@ -119,18 +119,19 @@ static int clear_status(void* ws, cudaStream_t s) {
 }
 
 static int do_route(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* pyr,
-                    int32_t* idx, float* margin, void* ws, size_t ws_bytes, cudaStream_t s) {
+                    int32_t* idx, float* margin, float* lse_out, void* ws, size_t ws_bytes, cudaStream_t s) {
   if (ws_bytes < route_ws_bytes(p, g)) return PISA_ERR_WORKSPACE_TOO_SMALL;
   if (use_tensor(p, g))
-    return tensor_route(g, p->dtype, q, k, pyr, idx, margin, (char*)ws + kStatusBytes, (int32_t*)ws, s);
+    return tensor_route(g, p->dtype, q, k, pyr, idx, margin, lse_out, (char*)ws + kStatusBytes, (int32_t*)ws, s);
   return launch_route_simt(g, p->dtype, q, k, pyr, idx, margin, s);
 }
 
 static int do_bsa(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v,
-                  const int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes, cudaStream_t s) {
+                  const int32_t* idx, void* out, float* lse, bool lse_ready, void* ws, size_t ws_bytes,
+                  cudaStream_t s) {
   if (ws_bytes < bsa_ws_bytes(p, g)) return PISA_ERR_WORKSPACE_TOO_SMALL;
   if (use_tensor(p, g))
-    return tensor_bsa(g, p->dtype, q, k, v, idx, out, lse, (char*)ws + kStatusBytes, (int32_t*)ws, s);
+    return tensor_bsa(g, p->dtype, q, k, v, idx, out, lse, lse_ready, (char*)ws + kStatusBytes, (int32_t*)ws, s);
   return launch_bsa_simt(g, p->dtype, q, k, v, idx, out, lse, s);
 }
 
@@ -156,10 +157,12 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
   st = launch_pyramid(g, p->dtype, k, pyr, s);
   if (st != PISA_OK) return st;
   stage_mark(1, s);
-  st = do_route(p, g, q, k, pyr, idx, nullptr, ws, ws_bytes, s);
+  // the tensor-core routing already knows every kept leaf's per-head LSE, so it hands the rows'
+  // softmax denominators to the attention stage
+  st = do_route(p, g, q, k, pyr, idx, nullptr, lse, ws, ws_bytes, s);
   if (st != PISA_OK) return st;
   stage_mark(2, s);
-  st = do_bsa(p, g, q, k, v, idx, out, lse, ws, ws_bytes, s);
+  st = do_bsa(p, g, q, k, v, idx, out, lse, use_tensor(p, g), ws, ws_bytes, s);
   stage_mark(3, s);
   return st;
 }
@@ -246,7 +249,7 @@ int pisa_route(const pisa_params_t* p, const void* q, const void* k, const void*
     return PISA_ERR_INVALID_ARG;
   st = clear_status(ws, (cudaStream_t)stream);
   if (st != PISA_OK) return st;
-  return do_route(p, g, q, k, pyramid, idx, margin, ws, ws_bytes, (cudaStream_t)stream);
+  return do_route(p, g, q, k, pyramid, idx, margin, nullptr, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 int pisa_bsa_fwd(const pisa_params_t* p, const void* q, const void* k, const void* v, const int32_t* idx,
@@ -259,7 +262,7 @@ int pisa_bsa_fwd(const pisa_params_t* p, const void* q, const void* k, const voi
     return PISA_ERR_INVALID_ARG;
   st = clear_status(ws, (cudaStream_t)stream);
   if (st != PISA_OK) return st;
-  return do_bsa(p, g, q, k, v, idx, out, lse, ws, ws_bytes, (cudaStream_t)stream);
+  return do_bsa(p, g, q, k, v, idx, out, lse, false, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const void* v, void* pyramid,

@@ -35,11 +35,10 @@ size_t align_up(size_t x, size_t a);
 int launch_pyramid(const Geometry& g, int dtype, const void* k, void* pyramid, cudaStream_t s);
 int launch_route_simt(const Geometry& g, int dtype, const void* q, const void* k, const void* pyramid,
                       int32_t* idx, float* margin, cudaStream_t s);
-// stage 1 of the two-stage schedule: leaf candidates [B,Hkv,N,gK] (-1 padded), margin so far
+// stage 1 of the two-stage schedule (needs L >= 2): kept level-2 nodes [B,Hkv,N,K] (ascending,
+// -1 padded) and the cut margin of the intermediate levels
 int launch_route_stage1_simt(const Geometry& g, int dtype, const void* q, const void* pyramid,
                              int32_t* cand_out, float* margin, cudaStream_t s);
-int launch_route_final_topk(const Geometry& g, const int32_t* cand, const float* scores, int32_t* idx,
-                            float* margin, cudaStream_t s);
 int launch_bsa_simt(const Geometry& g, int dtype, const void* q, const void* k, const void* v,
                     const int32_t* idx, void* out, float* lse, cudaStream_t s);
 int launch_flat_simt(const Geometry& g, int dtype, const void* q, const void* pyramid, int32_t* idx,

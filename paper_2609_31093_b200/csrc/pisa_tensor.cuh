@@ -9,9 +9,11 @@ bool tensor_path_supported(const Geometry& g, int dtype);
 size_t tensor_route_workspace_bytes(const Geometry& g);
 size_t tensor_bsa_workspace_bytes(const Geometry& g);
 // ws points past the status word; status is the workspace's status word
+// lse_out (nullable): softmax denominators of the kept leaves, float [B,Hq,N]
 int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, const void* pyramid, int32_t* idx,
-                 float* margin, void* ws, int32_t* status, cudaStream_t s);
+                 float* margin, float* lse_out, void* ws, int32_t* status, cudaStream_t s);
+// lse_ready: `lse` already holds the denominators of exactly these idx (as tensor_route writes them)
 int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const void* v, const int32_t* idx,
-               void* out, float* lse, void* ws, int32_t* status, cudaStream_t s);
+               void* out, float* lse, bool lse_ready, void* ws, int32_t* status, cudaStream_t s);
 
 }  // namespace pisa

@@ -4,7 +4,7 @@
 // This is the exact-fp32 SIMT path: it serves the fp32 dtype, every shape the tensor-core path does
 // not cover, and the cross-check of that path.  The same kernel, stopped after the intermediate
 // levels (LEAF = false), is stage 1 of the two-stage schedule (Algorithm 1): it then stores the
-// leaf candidates instead of scoring them.
+// kept level-2 nodes, whose children are the leaf candidates, instead of scoring the leaves.
 //
 // Per warp state lives in shared memory: the G query vectors in fp32, the sorted candidate list
 // (at most g*K entries) and the candidates' grouped scores.  The query-summary score matrix is
@@ -213,7 +213,9 @@ route_simt_kernel(Geometry geo, const T* __restrict__ q, const T* __restrict__ k
         const int pos = base + __popc(bal & ((1u << lane) - 1u));
         if (keep) {
           const int i = cand[s];
-          if (l > 1) {
+          if (!LEAF && l == 2) {
+            cand_out[w * (long long)K + pos] = i;        // two-stage schedule: kept level-2 nodes
+          } else if (l > 1) {
             for (int r = 0; r < g; ++r) next[pos * g + r] = i * g + r;
           } else {
             next[pos] = i;
@@ -226,14 +228,15 @@ route_simt_kernel(Geometry geo, const T* __restrict__ q, const T* __restrict__ k
         const float a = s_cut[warp][0], bb = s_cut[warp][1];
         if (a < CUDART_INF_F) min_gap = fminf(min_gap, (a - bb) / fmaxf(fabsf(a), 1.f));
       }
+      if (!LEAF && l == 2) {
+        // stage 1 of the two-stage schedule ends here (Algorithm 1): the leaf level is scored
+        // key-block-major by the tensor-core stage
+        for (int s = base + lane; s < K; s += 32) cand_out[w * (long long)K + s] = -1;
+        if (margin != nullptr && lane == 0) margin[w] = min_gap;
+        return;
+      }
       n = (l > 1) ? base * g : base;
       cur ^= 1;
-    } else {
-      // two-stage schedule: hand the eligible leaf candidates to the leaf-scoring stage
-      int32_t* dst = cand_out + w * (long long)(g * K);
-      for (int s = lane; s < g * K; s += 32) dst[s] = (s < nV) ? cand[s] : -1;
-      if (margin != nullptr && lane == 0) margin[w] = min_gap;
-      return;
     }
   }
   // leaf level done: the kept leaves, ascending, padded with -1
@@ -241,67 +244,6 @@ route_simt_kernel(Geometry geo, const T* __restrict__ q, const T* __restrict__ k
   int32_t* dst = idx + w * (long long)K;
   for (int s = lane; s < K; s += 32) dst[s] = (s < n) ? fin[s] : -1;
   if (margin != nullptr && lane == 0) margin[w] = min_gap;
-}
-
-// Final Select_K of the two-stage schedule (Algorithm 1, "Final Top-K selection"): candidates and
-// their grouped leaf scores come from the workspace; forced leaves are kept unscored.
-__global__ void __launch_bounds__(kWarpsPerCta * 32)
-route_final_topk_kernel(Geometry geo, const int32_t* __restrict__ cand_in, const float* __restrict__ score_in,
-                        int32_t* __restrict__ idx, float* __restrict__ margin) {
-  __shared__ __align__(16) float s_u[kWarpsPerCta][kMaxCand];
-  __shared__ int s_out[kWarpsPerCta][kMaxK];
-  __shared__ float s_cut[kWarpsPerCta][2];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long w = (long long)blockIdx.x * kWarpsPerCta + warp;
-  const long long total = (long long)geo.B * geo.Hkv * geo.N;
-  if (w >= total) return;
-  const int t = (int)(w % geo.N);
-  const int K = geo.K, gK = geo.g * geo.K;
-  const int c = t / geo.C;
-  const int f1 = (c >= 1) ? c - 1 : 0;
-  const int32_t* cand = cand_in + w * (long long)gK;
-  const float* sc = score_in + w * (long long)gK;
-  float* u = s_u[warp];
-  int nV = 0;
-  for (int s0 = 0; s0 < gK; s0 += 32) {
-    const int s = s0 + lane;
-    const int i = (s < gK) ? cand[s] : -1;
-    if (s < gK) u[s] = (i == 0 || i == f1 || i == c) ? CUDART_INF_F : sc[s];
-    nV += __popc(__ballot_sync(0xffffffffu, i >= 0));
-  }
-  __syncwarp();
-  const bool prune = nV > K;
-  int base = 0;
-  for (int s0 = 0; s0 < nV; s0 += 32) {
-    const int s = s0 + lane;
-    bool keep = s < nV;
-    if (prune) {
-      int rank = 0;
-      const float ui = (s < nV) ? u[s] : 0.f;
-      for (int j = 0; j < nV; ++j) {
-        const float uj = u[j];
-        rank += (uj > ui) || (uj == ui && j < s);
-      }
-      keep = keep && (rank < K);
-      if (s < nV && rank == K - 1) s_cut[warp][0] = ui;
-      if (s < nV && rank == K) s_cut[warp][1] = ui;
-    }
-    const unsigned bal = __ballot_sync(0xffffffffu, keep);
-    const int pos = base + __popc(bal & ((1u << lane) - 1u));
-    if (keep) s_out[warp][pos] = cand[s];
-    base += __popc(bal);
-  }
-  __syncwarp();
-  int32_t* dst = idx + w * (long long)K;
-  for (int s = lane; s < K; s += 32) dst[s] = (s < base) ? s_out[warp][s] : -1;
-  if (margin != nullptr && lane == 0) {
-    float mg = margin[w];
-    if (prune) {
-      const float a = s_cut[warp][0], bb = s_cut[warp][1];
-      if (a < CUDART_INF_F) mg = fminf(mg, (a - bb) / fmaxf(fabsf(a), 1.f));
-    }
-    margin[w] = mg;
-  }
 }
 
 template <typename T, int D, int G>
@@ -351,17 +293,10 @@ int launch_route_simt(const Geometry& g, int dtype, const void* q, const void* k
 
 int launch_route_stage1_simt(const Geometry& g, int dtype, const void* q, const void* pyramid,
                              int32_t* cand_out, float* margin, cudaStream_t s) {
+  if (g.L < 2) return PISA_ERR_UNSUPPORTED;
   if (dtype == PISA_BF16)
     return launch_route_t<__nv_bfloat16>(g, q, nullptr, pyramid, nullptr, margin, cand_out, false, s);
   return launch_route_t<float>(g, q, nullptr, pyramid, nullptr, margin, cand_out, false, s);
-}
-
-int launch_route_final_topk(const Geometry& g, const int32_t* cand, const float* scores, int32_t* idx,
-                            float* margin, cudaStream_t s) {
-  const long long total = (long long)g.B * g.Hkv * g.N;
-  const long long ctas = (total + kWarpsPerCta - 1) / kWarpsPerCta;
-  route_final_topk_kernel<<<(unsigned)ctas, kWarpsPerCta * 32, 0, s>>>(g, cand, scores, idx, margin);
-  return check_launch("route_final_topk");
 }
 
 }  // namespace pisa

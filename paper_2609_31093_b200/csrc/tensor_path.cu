@@ -1,13 +1,831 @@
+// Tensor-core path (bf16, tcgen05 + TMEM): key-block-major leaf scoring and block-sparse attention.
+//
+// Every query token picks its own blocks, and only the G heads of a group share them, so a
+// query-major tile would have G useful rows out of 128.  Both dense contractions of the path are
+// therefore run key-block-major (the two-stage idea of Algorithm 1, applied to the leaf scores and
+// to the attention alike): the per-token lists are inverted into per-block lists of (token, slot)
+// references, 128/G tokens x G heads are gathered into a 128-row A operand, and the block's keys
+// (and values) stay resident in shared memory as the B operand while the list is walked.
+//
+//   routing   : stage 1 (levels L..2, SIMT) -> kept level-2 nodes
+//               invert by level-2 node      -> lists of (token, slot)
+//               tile_lse_kernel             -> per-head LSE of every child leaf (g*C keys per tile),
+//                                              causal mask inside the query's own leaf
+//               final_topk_kernel           -> grouped score = sum over heads, forced leaves, Top-K;
+//                                              also the softmax denominator of the kept leaves
+//   attention : invert idx by leaf          -> lists of (token, slot)
+//               [tile_lse + row_lse only when the denominators are not already known]
+//               tile_pv_kernel              -> S = Q K^T, P = exp(S - lse_row) (already normalised),
+//                                              O_partial = P V, added into an fp32 accumulator with
+//                                              bulk reductions (one 256-byte row segment per thread)
+//               convert                     -> out in the storage dtype
+#include <math_constants.h>
+
 #include "pisa_tensor.cuh"
+#include "tc_utils.cuh"
 
 namespace pisa {
 
-bool tensor_path_supported(const Geometry&, int) { return false; }
-size_t tensor_route_workspace_bytes(const Geometry&) { return 0; }
-size_t tensor_bsa_workspace_bytes(const Geometry&) { return 0; }
-int tensor_route(const Geometry&, int, const void*, const void*, const void*, int32_t*, float*, void*, int32_t*,
-                 cudaStream_t) { return PISA_ERR_UNSUPPORTED; }
-int tensor_bsa(const Geometry&, int, const void*, const void*, const void*, const int32_t*, void*, float*, void*,
-               int32_t*, cudaStream_t) { return PISA_ERR_UNSUPPORTED; }
+using namespace tc;
+
+namespace {
+
+constexpr int kInvTok = 1024;          // tokens per CTA in the inversion kernels
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// ------------------------------------------------------------------ list inversion
+
+struct InvArgs {
+  const int32_t* nodes;   // [BH, N, K] node ids (ascending, -1 padded)
+  int K, fan, Mk, N, C, BH, tpt;
+  int32_t* count;         // [BH*Mk]
+  int32_t* entry_off;     // [BH*Mk + 1]
+  int32_t* tile_off;      // [BH*Mk + 1]
+  int32_t* cursor;        // [BH*Mk]
+  int32_t* entries;       // [<= BH*N*K]  token | slot << 24
+};
+
+__device__ __forceinline__ bool inv_valid(const InvArgs& a, int node, int t) {
+  return node >= 0 && node < a.Mk && (long long)node * a.fan <= (long long)(t / a.C);
+}
+
+__global__ void __launch_bounds__(256) inv_count_kernel(InvArgs a, int use_smem) {
+  extern __shared__ int s_hist[];
+  const int bh = blockIdx.y;
+  const int t0 = blockIdx.x * kInvTok, t1 = min(t0 + kInvTok, a.N);
+  if (use_smem) {
+    for (int j = threadIdx.x; j < a.Mk; j += blockDim.x) s_hist[j] = 0;
+    __syncthreads();
+  }
+  const int n = (t1 - t0) * a.K;
+  for (int e = threadIdx.x; e < n; e += blockDim.x) {
+    const int t = t0 + e / a.K;
+    const int node = a.nodes[((long long)bh * a.N + t0) * a.K + e];
+    if (inv_valid(a, node, t)) {
+      if (use_smem) atomicAdd(&s_hist[node], 1);
+      else atomicAdd(&a.count[(long long)bh * a.Mk + node], 1);
+    }
+  }
+  if (use_smem) {
+    __syncthreads();
+    for (int j = threadIdx.x; j < a.Mk; j += blockDim.x)
+      if (s_hist[j]) atomicAdd(&a.count[(long long)bh * a.Mk + j], s_hist[j]);
+  }
+}
+
+// exclusive scans of the list lengths (entries) and of their tile counts; one CTA
+__global__ void __launch_bounds__(1024) inv_scan_kernel(InvArgs a) {
+  __shared__ int s_e[1024], s_t[1024];
+  const int nkeys = a.BH * a.Mk;
+  const int per = (nkeys + 1023) / 1024;
+  const int lo = min(nkeys, (int)threadIdx.x * per), hi = min(nkeys, lo + per);
+  int se = 0, st = 0;
+  for (int i = lo; i < hi; ++i) {
+    const int c = a.count[i];
+    se += c;
+    st += (c + a.tpt - 1) / a.tpt;
+  }
+  s_e[threadIdx.x] = se; s_t[threadIdx.x] = st;
+  __syncthreads();
+  for (int o = 1; o < 1024; o <<= 1) {
+    int ve = 0, vt = 0;
+    if ((int)threadIdx.x >= o) { ve = s_e[threadIdx.x - o]; vt = s_t[threadIdx.x - o]; }
+    __syncthreads();
+    s_e[threadIdx.x] += ve; s_t[threadIdx.x] += vt;
+    __syncthreads();
+  }
+  int be = s_e[threadIdx.x] - se, bt = s_t[threadIdx.x] - st;
+  for (int i = lo; i < hi; ++i) {
+    const int c = a.count[i];
+    a.entry_off[i] = be; a.tile_off[i] = bt; a.cursor[i] = be;
+    be += c;
+    bt += (c + a.tpt - 1) / a.tpt;
+  }
+  if (threadIdx.x == 1023) { a.entry_off[nkeys] = s_e[1023]; a.tile_off[nkeys] = s_t[1023]; }
+}
+
+__global__ void __launch_bounds__(256) inv_fill_kernel(InvArgs a, int use_smem) {
+  extern __shared__ int s_mem[];
+  int* s_hist = s_mem;
+  int* s_base = s_mem + a.Mk;
+  const int bh = blockIdx.y;
+  const int t0 = blockIdx.x * kInvTok, t1 = min(t0 + kInvTok, a.N);
+  const int n = (t1 - t0) * a.K;
+  const int32_t* nodes = a.nodes + ((long long)bh * a.N + t0) * a.K;
+  if (!use_smem) {
+    for (int e = threadIdx.x; e < n; e += blockDim.x) {
+      const int t = t0 + e / a.K, slot = e % a.K, node = nodes[e];
+      if (inv_valid(a, node, t)) {
+        const int pos = atomicAdd(&a.cursor[(long long)bh * a.Mk + node], 1);
+        a.entries[pos] = t | (slot << 24);
+      }
+    }
+    return;
+  }
+  for (int j = threadIdx.x; j < a.Mk; j += blockDim.x) s_hist[j] = 0;
+  __syncthreads();
+  for (int e = threadIdx.x; e < n; e += blockDim.x) {
+    const int node = nodes[e];
+    if (inv_valid(a, node, t0 + e / a.K)) atomicAdd(&s_hist[node], 1);
+  }
+  __syncthreads();
+  for (int j = threadIdx.x; j < a.Mk; j += blockDim.x) {
+    const int c = s_hist[j];
+    if (c) s_base[j] = atomicAdd(&a.cursor[(long long)bh * a.Mk + j], c);
+    s_hist[j] = 0;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < n; e += blockDim.x) {
+    const int t = t0 + e / a.K, slot = e % a.K, node = nodes[e];
+    if (inv_valid(a, node, t)) {
+      const int r = atomicAdd(&s_hist[node], 1);
+      a.entries[s_base[node] + r] = t | (slot << 24);
+    }
+  }
+}
+
+// ------------------------------------------------------------------ tile kernels
+
+struct TileArgs {
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k;
+  const __nv_bfloat16* v;
+  const int32_t* entry_off;
+  const int32_t* tile_off;
+  const int32_t* entries;
+  int nkeys, Mk, fan, slots;
+  float* blk_lse;          // [BH, N, slots*fan, G]   (tile_lse)
+  const float* row_lse;    // [B, Hq, N]              (tile_pv)
+  float* o_acc;            // [B, N, Hq, D] fp32      (tile_pv)
+  int32_t* status;
+};
+
+__device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
+  return reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~(uintptr_t)1023);
+}
+
+// last key whose first tile is <= tile (lists without tiles share their successor's offset)
+__device__ __forceinline__ int find_key(const int32_t* tile_off, int nkeys, int tile) {
+  int lo = 0, hi = nkeys;            // invariant: tile_off[lo] <= tile < tile_off[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (tile_off[mid] <= tile) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// rows [row0, row0 + nrows) of a [tokens][D] bf16 matrix -> 128B-swizzled K-major slabs
+// (slab s holds elements [64 s, 64 s + 64) of every row); rows at or past `limit` become zeros
+template <int D>
+__device__ __forceinline__ void load_rows_swizzled(uint8_t* dst, int slab_bytes, const __nv_bfloat16* base,
+                                                   long long row_stride, int row0, int nrows, int limit, int tid) {
+  constexpr int CH = D / 8;
+  for (int idx = tid; idx < nrows * CH; idx += 128) {
+    const int row = idx / CH, ck = idx % CH;
+    const uint32_t d = smem_u32(dst + (ck >> 3) * slab_bytes) + swz128(row, ck & 7);
+    if (row0 + row < limit) cp_async16(d, base + (long long)(row0 + row) * row_stride + ck * 8);
+    else st_shared_zero16(d);
+  }
+}
+
+// gathered query rows: row r = (entry r / G, head r % G)
+template <int D>
+__device__ __forceinline__ void gather_q_swizzled(uint8_t* dst, const Geometry& geo, const __nv_bfloat16* q,
+                                                  int b, int h, const int* s_ent, int tid) {
+  constexpr int CH = D / 8;
+  const int G = geo.G;
+  for (int idx = tid; idx < 128 * CH; idx += 128) {
+    const int row = idx / CH, ck = idx % CH;
+    const uint32_t d = smem_u32(dst + (ck >> 3) * (128 * 128)) + swz128(row, ck & 7);
+    const int ent = s_ent[row / G];
+    if (ent >= 0) {
+      const int t = ent & 0xFFFFFF;
+      cp_async16(d, q + (long long)b * geo.qs[0] + (long long)t * geo.qs[1] +
+                        (long long)(h * G + row % G) * geo.qs[2] + ck * 8);
+    } else {
+      st_shared_zero16(d);
+    }
+  }
+}
+
+// Per-head log-sum-exp of the scaled logits of every (gathered query row, child leaf) pair of a
+// key group: the B operand is NB = fan*C consecutive keys, so one UMMA chain of D/16 steps gives a
+// 128 x NB logit tile in TMEM; each thread then owns one row and reduces C columns per child.
+template <int D, int NB>
+__global__ void __launch_bounds__(128) tile_lse_kernel(Geometry geo, TileArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  constexpr int KS = D / 64;
+  constexpr int A_SLAB = 128 * 128, B_SLAB = NB * 128;
+  constexpr uint32_t TM_COLS = NB < 32 ? 32 : NB;
+  uint8_t* smem = align1024(smem_raw);
+  uint8_t* sA = smem;
+  uint8_t* sB = smem + KS * A_SLAB;
+  __shared__ uint64_t bar;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int s_ent[128];
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if (tid == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
+  if (warp == 0) { tmem_alloc(&tmem_slot, TM_COLS); tmem_relinquish(); }
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  tcgen05_fence_after_sync();
+  const uint32_t tmem = tmem_slot;
+
+  const int G = geo.G, tpt = 128 / G, C = geo.C;
+  const int T = a.tile_off[a.nkeys];
+  const int per = (T + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int tile_begin = min(T, (int)blockIdx.x * per), tile_end = min(T, tile_begin + per);
+  const float sl2 = geo.scale * kLog2e;
+  const uint32_t idesc = make_idesc_bf16(128, NB, 0, 0);
+  uint32_t phase = 0;
+  int key = (tile_begin < tile_end) ? find_key(a.tile_off, a.nkeys, tile_begin) : 0;
+  int loaded_key = -1;
+
+  for (int tile = tile_begin; tile < tile_end; ++tile) {
+    while (tile >= a.tile_off[key + 1]) ++key;
+    const int bh = key / a.Mk, j = key % a.Mk;
+    const int b = bh / geo.Hkv, h = bh % geo.Hkv;
+    const int e0 = a.entry_off[key] + (tile - a.tile_off[key]) * tpt;
+    const int n_e = min(tpt, a.entry_off[key + 1] - e0);
+    if (tid < tpt) s_ent[tid] = (tid < n_e) ? a.entries[e0 + tid] : -1;
+    __syncthreads();      // entries visible; the previous tile's TMEM reads and smem reads are done
+    if (key != loaded_key) {
+      load_rows_swizzled<D>(sB, B_SLAB, a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2], geo.ks[1],
+                            j * NB, NB, geo.N, tid);
+      loaded_key = key;
+    }
+    gather_q_swizzled<D>(sA, geo, a.q, b, h, s_ent, tid);
+    const int ent = s_ent[tid / G];     // read before the barrier: the next iteration rewrites s_ent
+    cp_async_wait_all();
+    fence_proxy_async_smem();
+    __syncthreads();
+    if (tid == 0) {
+      tcgen05_fence_after_sync();
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const uint64_t da = make_smem_desc(smem_u32(sA) + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
+        const uint64_t db = make_smem_desc(smem_u32(sB) + (kk >> 2) * B_SLAB + (kk & 3) * 32, 0, 1024);
+        umma_bf16(tmem, da, db, idesc, kk > 0);
+      }
+      umma_commit(&bar);
+    }
+    const bool ok = mbar_wait_bounded(&bar, phase);
+    phase ^= 1u;
+    if (__syncthreads_or(!ok)) {
+      if (tid == 0) atomicExch(a.status, (int)PISA_ERR_TIMEOUT);
+      break;
+    }
+    tcgen05_fence_after_sync();
+
+    const int head = tid % G;
+    const bool valid = ent >= 0;
+    const int t = ent & 0xFFFFFF, slot = valid ? (ent >> 24) : 0;
+    const int c_t = t / C;
+    const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+    for (int r = 0; r < a.fan; ++r) {
+      const int leaf = j * a.fan + r;
+      int ncols = 0;
+      if (valid && leaf <= c_t && leaf < geo.M[1])
+        ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
+      float m = -CUDART_INF_F, ssum = 0.f;
+      for (int c0 = 0; c0 < C; c0 += 32) {
+        uint32_t rr[32];
+        tmem_ld_32x32(lane_base + (uint32_t)(r * C + c0), rr);
+        tmem_ld_wait();
+        float x[32];
+        float cm = -CUDART_INF_F;
+#pragma unroll
+        for (int jx = 0; jx < 32; ++jx) {
+          x[jx] = (c0 + jx < ncols) ? __uint_as_float(rr[jx]) * sl2 : -CUDART_INF_F;
+          cm = fmaxf(cm, x[jx]);
+        }
+        if (cm > -CUDART_INF_F) {
+          const float mn = fmaxf(m, cm);
+          float acc = 0.f;
+#pragma unroll
+          for (int jx = 0; jx < 32; ++jx) acc += exp2f(x[jx] - mn);
+          ssum = ssum * exp2f(m - mn) + acc;
+          m = mn;
+        }
+      }
+      if (valid) {
+        const float lse = (ssum > 0.f) ? (m + log2f(ssum)) * kLn2 : -CUDART_INF_F;
+        a.blk_lse[(((long long)bh * geo.N + t) * (a.slots * a.fan) + slot * a.fan + r) * G + head] = lse;
+      }
+    }
+    tcgen05_fence_before_sync();
+  }
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, TM_COLS);
+}
+
+// One (leaf block, tile of gathered query rows): S = Q K^T in TMEM, P = exp(S*scale - lse_row)
+// written back to shared memory as the bf16 A operand of O_partial = P V, and the fp32 partial
+// rows added into the accumulator by bulk reductions.  lse_row is the row's final softmax
+// denominator, so partials from different blocks simply add up.
+template <int D, int C>
+__global__ void __launch_bounds__(128) tile_pv_kernel(Geometry geo, TileArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  constexpr int KS = D / 64;                 // 64-wide slabs of d
+  constexpr int PS = C / 64;                 // 64-wide slabs of keys (P operand)
+  constexpr int A_SLAB = 128 * 128, KV_SLAB = C * 128;
+  constexpr int STAGE_ROW = 256 + 16;        // 64 fp32 + pad: conflict-free 16-byte row writes
+  constexpr int QP_BYTES = (KS * A_SLAB > 128 * STAGE_ROW) ? KS * A_SLAB : 128 * STAGE_ROW;
+  constexpr int QP_ALIGNED = (QP_BYTES + 1023) / 1024 * 1024;
+  constexpr uint32_t TM_COLS = 256;          // S at column 0 (C columns), O at column 128 (D columns)
+  uint8_t* smem = align1024(smem_raw);
+  uint8_t* sQ = smem;                        // Q tile, then P tile, then the O staging rows
+  uint8_t* sK = smem + QP_ALIGNED;
+  uint8_t* sV = sK + KS * KV_SLAB;
+  __shared__ uint64_t bar;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int s_ent[128];
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if (tid == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
+  if (warp == 0) { tmem_alloc(&tmem_slot, TM_COLS); tmem_relinquish(); }
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  tcgen05_fence_after_sync();
+  const uint32_t tmem = tmem_slot;
+  const uint32_t tmem_s = tmem, tmem_o = tmem + 128;
+
+  const int G = geo.G, tpt = 128 / G;
+  const int T = a.tile_off[a.nkeys];
+  const int per = (T + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int tile_begin = min(T, (int)blockIdx.x * per), tile_end = min(T, tile_begin + per);
+  const float sl2 = geo.scale * kLog2e;
+  const uint32_t idesc_s = make_idesc_bf16(128, C, 0, 0);
+  const uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
+  uint32_t phase = 0;
+  int key = (tile_begin < tile_end) ? find_key(a.tile_off, a.nkeys, tile_begin) : 0;
+  int loaded_key = -1;
+  bool failed = false;
+
+  for (int tile = tile_begin; tile < tile_end; ++tile) {
+    while (tile >= a.tile_off[key + 1]) ++key;
+    const int bh = key / a.Mk, leaf = key % a.Mk;
+    const int b = bh / geo.Hkv, h = bh % geo.Hkv;
+    const int e0 = a.entry_off[key] + (tile - a.tile_off[key]) * tpt;
+    const int n_e = min(tpt, a.entry_off[key + 1] - e0);
+    if (tid < tpt) s_ent[tid] = (tid < n_e) ? a.entries[e0 + tid] : -1;
+    bulk_wait_read_all();    // this thread's staging rows of the previous tile have been read
+    __syncthreads();
+    if (key != loaded_key) {
+      load_rows_swizzled<D>(sK, KV_SLAB, a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2], geo.ks[1],
+                            leaf * C, C, geo.N, tid);
+      load_rows_swizzled<D>(sV, KV_SLAB, a.v + (long long)b * geo.vs[0] + (long long)h * geo.vs[2], geo.vs[1],
+                            leaf * C, C, geo.N, tid);
+      loaded_key = key;
+    }
+    gather_q_swizzled<D>(sQ, geo, a.q, b, h, s_ent, tid);
+
+    const int ent = s_ent[tid / G];
+    const int head = tid % G;
+    const bool valid = ent >= 0;
+    const int t = ent & 0xFFFFFF;
+    const int hq = h * G + head;
+    float lse2 = 0.f;                  // row denominator in log2 units
+    int ncols = 0;
+    if (valid) {
+      lse2 = a.row_lse[((long long)b * geo.Hq + hq) * geo.N + t] * kLog2e;
+      const int c_t = t / C;
+      if (leaf <= c_t && lse2 > -CUDART_INF_F) ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
+    }
+    cp_async_wait_all();
+    fence_proxy_async_smem();
+    __syncthreads();
+    if (tid == 0) {
+      tcgen05_fence_after_sync();
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const uint64_t da = make_smem_desc(smem_u32(sQ) + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
+        const uint64_t db = make_smem_desc(smem_u32(sK) + (kk >> 2) * KV_SLAB + (kk & 3) * 32, 0, 1024);
+        umma_bf16(tmem_s, da, db, idesc_s, kk > 0);
+      }
+      umma_commit(&bar);
+    }
+    bool ok = mbar_wait_bounded(&bar, phase);
+    phase ^= 1u;
+    if (__syncthreads_or(!ok)) { failed = true; break; }
+    tcgen05_fence_after_sync();
+
+    // P = exp2(S*scale*log2e - lse2), masked, as the bf16 K-major A operand (overwrites the Q tile:
+    // the S chain that read it has completed)
+    const uint32_t lane_base = tmem_s + ((uint32_t)(warp * 32) << 16);
+#pragma unroll
+    for (int c0 = 0; c0 < C; c0 += 32) {
+      uint32_t rr[32];
+      tmem_ld_32x32(lane_base + (uint32_t)c0, rr);
+      tmem_ld_wait();
+      uint32_t pk[16];
+#pragma unroll
+      for (int jx = 0; jx < 16; ++jx) {
+        const float p0 = (c0 + 2 * jx < ncols) ? exp2f(__uint_as_float(rr[2 * jx]) * sl2 - lse2) : 0.f;
+        const float p1 = (c0 + 2 * jx + 1 < ncols) ? exp2f(__uint_as_float(rr[2 * jx + 1]) * sl2 - lse2) : 0.f;
+        const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
+        pk[jx] = *reinterpret_cast<const uint32_t*>(&pp);
+      }
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        const int ck = c0 / 8 + q4;                       // 16-byte chunk (8 keys) of this row
+        const uint32_t d = smem_u32(sQ + (ck >> 3) * A_SLAB) + swz128(tid, ck & 7);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d), "r"(pk[4 * q4]), "r"(pk[4 * q4 + 1]),
+                     "r"(pk[4 * q4 + 2]), "r"(pk[4 * q4 + 3])
+                     : "memory");
+      }
+    }
+    fence_proxy_async_smem();
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {
+      tcgen05_fence_after_sync();
+#pragma unroll
+      for (int kk = 0; kk < C / 16; ++kk) {
+        const uint64_t da = make_smem_desc(smem_u32(sQ) + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
+        const uint64_t db = make_smem_desc(smem_u32(sV) + kk * (16 * 128), KV_SLAB, 1024);
+        umma_bf16(tmem_o, da, db, idesc_o, kk > 0);
+      }
+      umma_commit(&bar);
+    }
+    ok = mbar_wait_bounded(&bar, phase);
+    phase ^= 1u;
+    if (__syncthreads_or(!ok)) { failed = true; break; }
+    tcgen05_fence_after_sync();
+
+    // O partial: 64 columns at a time through this thread's private staging row, then one bulk
+    // reduction (256 bytes) into the fp32 accumulator row of (b, t, hq)
+    const uint32_t o_base = tmem_o + ((uint32_t)(warp * 32) << 16);
+    uint8_t* stage = sQ + tid * STAGE_ROW;
+    float* orow = a.o_acc + (((long long)b * geo.N + t) * geo.Hq + hq) * D;
+#pragma unroll
+    for (int half = 0; half < KS; ++half) {
+      if (half > 0) bulk_wait_read_all();
+#pragma unroll
+      for (int c0 = 0; c0 < 64; c0 += 32) {
+        uint32_t rr[32];
+        tmem_ld_32x32(o_base + (uint32_t)(half * 64 + c0), rr);
+        tmem_ld_wait();
+#pragma unroll
+        for (int q4 = 0; q4 < 8; ++q4)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(stage) + (c0 + 4 * q4) * 4),
+                       "r"(rr[4 * q4]), "r"(rr[4 * q4 + 1]), "r"(rr[4 * q4 + 2]), "r"(rr[4 * q4 + 3])
+                       : "memory");
+      }
+      fence_proxy_async_smem();
+      if (valid) {
+        bulk_reduce_add_f32(orow + half * 64, smem_u32(stage), 256);
+        bulk_commit();
+      }
+    }
+    tcgen05_fence_before_sync();
+  }
+  (void)PS;
+  if (failed && tid == 0) atomicExch(a.status, (int)PISA_ERR_TIMEOUT);
+  bulk_wait_all();
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, TM_COLS);
+}
+
+// ------------------------------------------------------------------ small SIMT stages
+
+// Final Select_K of the two-stage schedule (Algorithm 1): the candidates are the children of the
+// kept level-2 nodes; grouped score = sum of the per-head leaf LSEs; forced leaves kept unscored.
+// Also emits the softmax denominator of the kept leaves per query head (their LSEs are known).
+__global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int32_t* __restrict__ par,
+                                                          const float* __restrict__ blk_lse,
+                                                          int32_t* __restrict__ idx, float* __restrict__ margin,
+                                                          float* __restrict__ lse_out) {
+  __shared__ __align__(16) float s_u[4][kMaxCand];
+  __shared__ int s_sel[4][kMaxK];
+  __shared__ float s_cut[4][2];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long w = (long long)blockIdx.x * 4 + warp;
+  const long long total = (long long)geo.B * geo.Hkv * geo.N;
+  if (w >= total) return;
+  const int t = (int)(w % geo.N);
+  const int bh = (int)(w / geo.N);
+  const int K = geo.K, g = geo.g, gK = g * K, G = geo.G;
+  const int c = t / geo.C;
+  const int f1 = (c >= 1) ? c - 1 : 0;
+  const int32_t* pr = par + w * (long long)K;
+  const float* bl = blk_lse + w * (long long)gK * G;
+  float* u = s_u[warp];
+  // candidate ci = slot*g + r  <->  leaf par[slot]*g + r; valid ones form a prefix
+  int nV = 0;
+  for (int c0 = 0; c0 < gK; c0 += 32) {
+    const int ci = c0 + lane;
+    bool ok = false;
+    if (ci < gK) {
+      const int p = pr[ci / g];
+      const int leaf = p * g + ci % g;
+      ok = (p >= 0) && (leaf <= c);
+      float sc = -CUDART_INF_F;
+      if (ok) {
+        if (leaf == 0 || leaf == f1 || leaf == c) sc = CUDART_INF_F;
+        else {
+          sc = 0.f;
+          for (int hh = 0; hh < G; ++hh) sc += bl[ci * G + hh];
+        }
+      }
+      u[ci] = sc;
+    }
+    nV += __popc(__ballot_sync(0xffffffffu, ok));
+  }
+  __syncwarp();
+  const bool prune = nV > K;
+  int base = 0;
+  unsigned kept_mask[kMaxCand / 32];
+  for (int s0 = 0, ch = 0; s0 < gK; s0 += 32, ++ch) {
+    const int s = s0 + lane;
+    bool keep = s < nV;
+    if (prune && s0 < nV) {
+      int rank = 0;
+      const float ui = (s < nV) ? u[s] : 0.f;
+      for (int j = 0; j < nV; ++j) {
+        const float uj = u[j];
+        rank += (uj > ui) || (uj == ui && j < s);
+      }
+      keep = keep && (rank < K);
+      if (s < nV && rank == K - 1) s_cut[warp][0] = ui;
+      if (s < nV && rank == K) s_cut[warp][1] = ui;
+    }
+    const unsigned bal = __ballot_sync(0xffffffffu, keep);
+    kept_mask[ch] = bal;
+    const int pos = base + __popc(bal & ((1u << lane) - 1u));
+    if (keep) s_sel[warp][pos] = pr[s / g] * g + s % g;
+    base += __popc(bal);
+  }
+  __syncwarp();
+  int32_t* dst = idx + w * (long long)K;
+  for (int s = lane; s < K; s += 32) dst[s] = (s < base) ? s_sel[warp][s] : -1;
+  if (margin != nullptr && lane == 0) {
+    float mg = margin[w];
+    if (prune) {
+      const float a = s_cut[warp][0], bb = s_cut[warp][1];
+      if (a < CUDART_INF_F) mg = fminf(mg, (a - bb) / fmaxf(fabsf(a), 1.f));
+    }
+    margin[w] = mg;
+  }
+  if (lse_out != nullptr) {
+    const int b = bh / geo.Hkv, h = bh % geo.Hkv;
+    for (int hh = 0; hh < G; ++hh) {
+      float m = -CUDART_INF_F;
+      for (int s0 = 0, ch = 0; s0 < gK; s0 += 32, ++ch)
+        if ((kept_mask[ch] >> lane) & 1u) m = fmaxf(m, bl[(s0 + lane) * G + hh]);
+      m = warp_max(m);
+      float ssum = 0.f;
+      for (int s0 = 0, ch = 0; s0 < gK; s0 += 32, ++ch)
+        if ((kept_mask[ch] >> lane) & 1u) ssum += expf(bl[(s0 + lane) * G + hh] - m);
+      ssum = warp_sum(ssum);
+      if (lane == 0) lse_out[((long long)b * geo.Hq + h * G + hh) * geo.N + t] = m + logf(ssum);
+    }
+  }
+}
+
+// softmax denominator of a row from the per-block LSEs of its selected leaves (stand-alone attention)
+__global__ void __launch_bounds__(256) row_lse_kernel(Geometry geo, const int32_t* __restrict__ idx,
+                                                       const float* __restrict__ blk_lse, float* __restrict__ lse_out) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long total = (long long)geo.B * geo.Hkv * geo.N * geo.G;
+  if (i >= total) return;
+  const int head = (int)(i % geo.G);
+  const long long w = i / geo.G;
+  const int t = (int)(w % geo.N);
+  const int bh = (int)(w / geo.N);
+  const int c = t / geo.C;
+  float m = -CUDART_INF_F;
+  for (int s = 0; s < geo.K; ++s) {
+    const int leaf = idx[w * geo.K + s];
+    if (leaf >= 0 && leaf <= c && leaf < geo.M[1]) m = fmaxf(m, blk_lse[(w * geo.K + s) * geo.G + head]);
+  }
+  float ssum = 0.f;
+  for (int s = 0; s < geo.K; ++s) {
+    const int leaf = idx[w * geo.K + s];
+    if (leaf >= 0 && leaf <= c && leaf < geo.M[1]) ssum += expf(blk_lse[(w * geo.K + s) * geo.G + head] - m);
+  }
+  const int b = bh / geo.Hkv, h = bh % geo.Hkv;
+  lse_out[((long long)b * geo.Hq + h * geo.G + head) * geo.N + t] = (ssum > 0.f) ? m + logf(ssum) : -CUDART_INF_F;
+}
+
+// fp32 accumulator [B,N,Hq,D] -> out in bf16 (strided)
+__global__ void __launch_bounds__(256) convert_out_kernel(Geometry geo, const float* __restrict__ acc,
+                                                           __nv_bfloat16* __restrict__ out) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;     // one 8-element chunk
+  const int ch = geo.d / 8;
+  const long long total = (long long)geo.B * geo.N * geo.Hq * ch;
+  if (i >= total) return;
+  const int ck = (int)(i % ch);
+  const long long row = i / ch;
+  const int hq = (int)(row % geo.Hq);
+  const long long bt = row / geo.Hq;
+  const int t = (int)(bt % geo.N), b = (int)(bt / geo.N);
+  const float4 x0 = *reinterpret_cast<const float4*>(acc + row * geo.d + ck * 8);
+  const float4 x1 = *reinterpret_cast<const float4*>(acc + row * geo.d + ck * 8 + 4);
+  __nv_bfloat162 p0 = __floats2bfloat162_rn(x0.x, x0.y), p1 = __floats2bfloat162_rn(x0.z, x0.w);
+  __nv_bfloat162 p2 = __floats2bfloat162_rn(x1.x, x1.y), p3 = __floats2bfloat162_rn(x1.z, x1.w);
+  uint4 o;
+  o.x = *reinterpret_cast<uint32_t*>(&p0); o.y = *reinterpret_cast<uint32_t*>(&p1);
+  o.z = *reinterpret_cast<uint32_t*>(&p2); o.w = *reinterpret_cast<uint32_t*>(&p3);
+  *reinterpret_cast<uint4*>(out + (long long)b * geo.os[0] + (long long)t * geo.os[1] + (long long)hq * geo.os[2] + ck * 8) = o;
+}
+
+// ------------------------------------------------------------------ host side
+
+struct InvLayout {
+  size_t count, entry_off, tile_off, cursor, entries, end;
+};
+
+InvLayout inv_layout(size_t base, const Geometry& g, int Mk) {
+  const size_t nkeys = (size_t)g.B * g.Hkv * Mk;
+  InvLayout l;
+  size_t o = base;
+  l.count = o; o += align_up(nkeys * 4, 256);
+  l.entry_off = o; o += align_up((nkeys + 1) * 4, 256);
+  l.tile_off = o; o += align_up((nkeys + 1) * 4, 256);
+  l.cursor = o; o += align_up(nkeys * 4, 256);
+  l.entries = o; o += align_up((size_t)g.B * g.Hkv * g.N * g.K * 4, 256);
+  l.end = o;
+  return l;
+}
+
+struct RouteLayout { size_t par, blk, total; InvLayout inv; };
+RouteLayout route_layout(const Geometry& g) {
+  RouteLayout r;
+  size_t o = 0;
+  r.par = o; o += align_up((size_t)g.B * g.Hkv * g.N * g.K * 4, 256);
+  r.blk = o; o += align_up((size_t)g.B * g.Hkv * g.N * g.g * g.K * g.G * 4, 256);
+  r.inv = inv_layout(o, g, g.M[2]);
+  r.total = r.inv.end;
+  return r;
+}
+struct BsaLayout { size_t blk, acc, total; InvLayout inv; };
+BsaLayout bsa_layout(const Geometry& g) {
+  BsaLayout r;
+  size_t o = 0;
+  r.blk = o; o += align_up((size_t)g.B * g.Hkv * g.N * g.K * g.G * 4, 256);
+  r.acc = o; o += align_up((size_t)g.B * g.N * g.Hq * g.d * 4, 256);
+  r.inv = inv_layout(o, g, g.M[1]);
+  r.total = r.inv.end;
+  return r;
+}
+
+int num_sms() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char* ws, const InvLayout& l,
+                  InvArgs* out, cudaStream_t s) {
+  InvArgs a;
+  a.nodes = nodes; a.K = g.K; a.fan = fan; a.Mk = Mk; a.N = g.N; a.C = g.C; a.BH = g.B * g.Hkv;
+  a.tpt = 128 / g.G;
+  a.count = (int32_t*)(ws + l.count); a.entry_off = (int32_t*)(ws + l.entry_off);
+  a.tile_off = (int32_t*)(ws + l.tile_off); a.cursor = (int32_t*)(ws + l.cursor);
+  a.entries = (int32_t*)(ws + l.entries);
+  const size_t nkeys = (size_t)a.BH * Mk;
+  cudaError_t e = cudaMemsetAsync(a.count, 0, nkeys * 4, s);
+  if (e != cudaSuccess) { record_cuda_error("inversion memset", e); return PISA_ERR_CUDA; }
+  const int use_smem = (2 * (size_t)Mk * 4 <= 96 * 1024) ? 1 : 0;
+  const size_t sm_count = use_smem ? (size_t)Mk * 4 : 0, sm_fill = use_smem ? 2 * (size_t)Mk * 4 : 0;
+  dim3 grid((g.N + kInvTok - 1) / kInvTok, a.BH);
+  if (sm_fill > 48 * 1024) {
+    cudaFuncSetAttribute(inv_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_count);
+    cudaFuncSetAttribute(inv_fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_fill);
+  }
+  inv_count_kernel<<<grid, 256, sm_count, s>>>(a, use_smem);
+  int st = check_launch("inv_count");
+  if (st != PISA_OK) return st;
+  inv_scan_kernel<<<1, 1024, 0, s>>>(a);
+  st = check_launch("inv_scan");
+  if (st != PISA_OK) return st;
+  inv_fill_kernel<<<grid, 256, sm_fill, s>>>(a, use_smem);
+  st = check_launch("inv_fill");
+  *out = a;
+  return st;
+}
+
+template <int D, int NB>
+int launch_tile_lse(const Geometry& g, const TileArgs& a, cudaStream_t s) {
+  const size_t smem = (size_t)(D / 64) * (128 * 128 + NB * 128) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(tile_lse_kernel<D, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) { record_cuda_error("tile_lse attr", e); return PISA_ERR_CUDA; }
+  const int ctas_per_sm = (smem <= 100 * 1024 && NB <= 256) ? 2 : 1;
+  tile_lse_kernel<D, NB><<<num_sms() * ctas_per_sm, 128, smem, s>>>(g, a);
+  return check_launch("tile_lse");
+}
+
+int dispatch_tile_lse(const Geometry& g, int nb, const TileArgs& a, cudaStream_t s) {
+  if (g.d == 128) {
+    if (nb == 64) return launch_tile_lse<128, 64>(g, a, s);
+    if (nb == 128) return launch_tile_lse<128, 128>(g, a, s);
+    if (nb == 256) return launch_tile_lse<128, 256>(g, a, s);
+  } else if (g.d == 64) {
+    if (nb == 64) return launch_tile_lse<64, 64>(g, a, s);
+    if (nb == 128) return launch_tile_lse<64, 128>(g, a, s);
+    if (nb == 256) return launch_tile_lse<64, 256>(g, a, s);
+  }
+  return PISA_ERR_UNSUPPORTED;
+}
+
+template <int D, int C>
+int launch_tile_pv(const Geometry& g, const TileArgs& a, cudaStream_t s) {
+  constexpr int KS = D / 64;
+  constexpr int QP = (KS * 128 * 128 > 128 * 272) ? KS * 128 * 128 : 128 * 272;
+  const size_t smem = (size_t)((QP + 1023) / 1024 * 1024) + 2 * (size_t)KS * C * 128 + 1024;
+  cudaError_t e = cudaFuncSetAttribute(tile_pv_kernel<D, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) { record_cuda_error("tile_pv attr", e); return PISA_ERR_CUDA; }
+  tile_pv_kernel<D, C><<<num_sms() * 2, 128, smem, s>>>(g, a);
+  return check_launch("tile_pv");
+}
+
+int dispatch_tile_pv(const Geometry& g, const TileArgs& a, cudaStream_t s) {
+  if (g.d == 128 && g.C == 128) return launch_tile_pv<128, 128>(g, a, s);
+  if (g.d == 128 && g.C == 64) return launch_tile_pv<128, 64>(g, a, s);
+  if (g.d == 64 && g.C == 128) return launch_tile_pv<64, 128>(g, a, s);
+  if (g.d == 64 && g.C == 64) return launch_tile_pv<64, 64>(g, a, s);
+  return PISA_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+bool tensor_path_supported(const Geometry& g, int dtype) {
+  if (dtype != PISA_BF16 || g.score_mode != PISA_SCORE_LSE) return false;
+  if (g.d != 64 && g.d != 128) return false;
+  if (g.C != 64 && g.C != 128) return false;
+  const int nb = g.g * g.C;
+  if (nb != 128 && nb != 256) return false;
+  if (g.L < 2 || g.N >= (1 << 24)) return false;
+  if ((long long)g.B * g.Hkv * g.N * g.K >= (1LL << 31)) return false;   // entry offsets are int32
+  return true;
+}
+
+size_t tensor_route_workspace_bytes(const Geometry& g) { return route_layout(g).total; }
+size_t tensor_bsa_workspace_bytes(const Geometry& g) { return bsa_layout(g).total; }
+
+int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, const void* pyramid, int32_t* idx,
+                 float* margin, float* lse_out, void* ws_, int32_t* status, cudaStream_t s) {
+  char* ws = (char*)ws_;
+  const RouteLayout L = route_layout(g);
+  int32_t* par = (int32_t*)(ws + L.par);
+  float* blk = (float*)(ws + L.blk);
+  int st = launch_route_stage1_simt(g, dtype, q, pyramid, par, margin, s);
+  if (st != PISA_OK) return st;
+  InvArgs inv;
+  st = run_inversion(g, par, g.g, g.M[2], ws, L.inv, &inv, s);
+  if (st != PISA_OK) return st;
+  TileArgs a = {};
+  a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = nullptr;
+  a.entry_off = inv.entry_off; a.tile_off = inv.tile_off; a.entries = inv.entries;
+  a.nkeys = g.B * g.Hkv * g.M[2]; a.Mk = g.M[2]; a.fan = g.g; a.slots = g.K;
+  a.blk_lse = blk; a.status = status;
+  st = dispatch_tile_lse(g, g.g * g.C, a, s);
+  if (st != PISA_OK) return st;
+  const long long total = (long long)g.B * g.Hkv * g.N;
+  final_topk_kernel<<<(unsigned)((total + 3) / 4), 128, 0, s>>>(g, par, blk, idx, margin, lse_out);
+  return check_launch("final_topk");
+}
+
+int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const void* v, const int32_t* idx,
+               void* out, float* lse, bool lse_ready, void* ws_, int32_t* status, cudaStream_t s) {
+  (void)dtype;
+  char* ws = (char*)ws_;
+  const BsaLayout L = bsa_layout(g);
+  float* blk = (float*)(ws + L.blk);
+  float* acc = (float*)(ws + L.acc);
+  InvArgs inv;
+  int st = run_inversion(g, idx, 1, g.M[1], ws, L.inv, &inv, s);
+  if (st != PISA_OK) return st;
+  TileArgs a = {};
+  a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
+  a.entry_off = inv.entry_off; a.tile_off = inv.tile_off; a.entries = inv.entries;
+  a.nkeys = g.B * g.Hkv * g.M[1]; a.Mk = g.M[1]; a.fan = 1; a.slots = g.K;
+  a.blk_lse = blk; a.row_lse = lse; a.o_acc = acc; a.status = status;
+  if (!lse_ready) {
+    st = dispatch_tile_lse(g, g.C, a, s);
+    if (st != PISA_OK) return st;
+    const long long rows = (long long)g.B * g.Hkv * g.N * g.G;
+    row_lse_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, s>>>(g, idx, blk, lse);
+    st = check_launch("row_lse");
+    if (st != PISA_OK) return st;
+  }
+  cudaError_t e = cudaMemsetAsync(acc, 0, (size_t)g.B * g.N * g.Hq * g.d * 4, s);
+  if (e != cudaSuccess) { record_cuda_error("accumulator memset", e); return PISA_ERR_CUDA; }
+  st = dispatch_tile_pv(g, a, s);
+  if (st != PISA_OK) return st;
+  const long long chunks = (long long)g.B * g.N * g.Hq * (g.d / 8);
+  convert_out_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, s>>>(g, acc, (__nv_bfloat16*)out);
+  return check_launch("convert_out");
+}
 
 }  // namespace pisa
