@@ -38,6 +38,9 @@ def get_workload(name: str) -> S.Workload:
         return S.WORKLOADS[name]
     if name.startswith("cfg5_"):
         return S.sweep_workload(int(name.split("_")[1]))
+    if name.startswith("custom:"):       # custom:B,N,Hq,Hkv,d,C,g,K  (bf16, i.i.d., for profiling captures)
+        B, N, Hq, Hkv, d, C, g, K = (int(x) for x in name.split(":")[1].split(","))
+        return S.Workload(name, B, N, Hq, Hkv, d, C, g, K, "bf16", 9, "iid")
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -181,8 +184,8 @@ def oracle_sample_rate(w: S.Workload, tensors: dict, n_queries: int, seed: int =
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    rank = rank_env()[0]
+    if rank != 0:             # under torchrun only rank 0 runs the CPU reference
         return
     w = get_workload(args.workload)
     tensors = S.make_inputs(w)
@@ -207,6 +210,35 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------ multi-rank plumbing
+
+def rank_env():
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def replica_workload(w: S.Workload, rank: int) -> S.Workload:
+    """The path shards over independent (batch, KV head) units without any exchange step, so rank r
+    simply owns its own replica of the workload (same shape, its own seed): weak scaling."""
+    return dataclasses.replace(w, seed=w.seed + 1000 * rank)
+
+
+def max_over_ranks(values, world: int, device=None):
+    """Element-wise max of a list of floats over all ranks (identity for one rank)."""
+    if world <= 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_tokens_per_s(w: S.Workload, world: int, steps: int, ms: float) -> float:
+    """Whole-job throughput: every rank processed B*N tokens per step in `ms` (max over ranks)."""
+    return world * w.B * w.N * steps / (ms * 1e-3)
+
+
 # ------------------------------------------------------------------ our arm
 
 def run_ours(args):
@@ -216,9 +248,7 @@ def run_ours(args):
     import paper_2609_31093_b200 as P
     from paper_2609_31093_b200 import binding as PB
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
     torch.cuda.set_device(local)
@@ -226,7 +256,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     w0 = get_workload(args.workload)
-    w = dataclasses.replace(w0, seed=w0.seed + 1000 * rank)       # every rank its own replica
+    w = replica_workload(w0, rank)
     impl = {"auto": PB.IMPL_AUTO, "simt": PB.IMPL_SIMT, "tensor": PB.IMPL_TENSOR}[args.path]
     p = P.Params.from_workload(w, impl=impl)
     tensors = S.make_inputs(w)
@@ -260,8 +290,12 @@ def run_ours(args):
         raise SystemExit(f"device status {st} after warm-up")
 
     P.set_stage_timing(True)
-    sampler = ClockSampler(str(torch.cuda.get_device_properties(local).uuid) if hasattr(
-        torch.cuda.get_device_properties(local), "uuid") else str(local))
+    props = torch.cuda.get_device_properties(local)
+    gpu_id = str(local)
+    if hasattr(props, "uuid"):
+        u = str(props.uuid)
+        gpu_id = u if u.startswith("GPU-") else "GPU-" + u
+    sampler = ClockSampler(gpu_id)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     stage = np.zeros(3)
     barrier()
@@ -285,32 +319,30 @@ def run_ours(args):
     arena = PB.alloc_workspace(p, PB.OP_FORWARD_HOST)
     out_h = torch.empty(q.shape, dtype=tdt).pin_memory()
     lse_h = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
-    e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    for _ in range(2):
-        P.pisa_forward_host(p, qh, kh, vh, out_h, lse_h, None, arena)
-    barrier()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(e2e_steps):
-        P.pisa_forward_host(p, qh, kh, vh, out_h, lse_h, None, arena)
-    e1.record()
-    torch.cuda.synchronize()
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
+    e2e_steps = max(0, min(args.steps, args.e2e_steps))
+    e2e_ms = float("nan")
+    if e2e_steps > 0:
+        for _ in range(2):
+            P.pisa_forward_host(p, qh, kh, vh, out_h, lse_h, None, arena)
+        barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(e2e_steps):
+            P.pisa_forward_host(p, qh, kh, vh, out_h, lse_h, None, arena)
+        e1.record()
+        torch.cuda.synchronize()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
 
-    if world > 1:
-        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = t.tolist()
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], world, device="cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    tokens = w.B * w.N
-    value = world * tokens * args.steps / (ms * 1e-3)
-    e2e_value = world * tokens * e2e_steps / (e2e_ms * 1e-3)
+    value = job_tokens_per_s(w, world, args.steps, ms)
+    e2e_value = job_tokens_per_s(w, world, e2e_steps, e2e_ms) if e2e_steps > 0 else None
     wc = work_counts(w)
     peaks = {}
     try:

@@ -39,6 +39,10 @@ int launch_route_simt(const Geometry& g, int dtype, const void* q, const void* k
 // -1 padded) and the cut margin of the intermediate levels
 int launch_route_stage1_simt(const Geometry& g, int dtype, const void* q, const void* pyramid,
                              int32_t* cand_out, float* margin, cudaStream_t s);
+// the same stage on warp-level tensor-core MMAs (bf16, LSE score)
+bool route_stage1_mma_supported(const Geometry& g, int dtype);
+int launch_route_stage1_mma(const Geometry& g, const void* q, const void* pyramid, int32_t* par, float* margin,
+                            cudaStream_t s);
 int launch_bsa_simt(const Geometry& g, int dtype, const void* q, const void* k, const void* v,
                     const int32_t* idx, void* out, float* lse, cudaStream_t s);
 int launch_flat_simt(const Geometry& g, int dtype, const void* q, const void* pyramid, int32_t* idx,

@@ -1,0 +1,210 @@
+// Stage 1 of the two-stage routing schedule (Algorithm 1, levels L..2) for bf16 inputs, one warp per
+// (b, KV head, query token), with the candidate scoring on warp-level tensor-core MMAs.
+//
+// At one level a token scores at most g*K candidates, each from g child summaries, against its own G
+// query vectors: a gathered [g*K*g rows] x [d] by [d] x [G] product, far too small and too irregular
+// for a CTA-wide UMMA tile but a natural fit for m16n8k16 fragments held in registers.  The child
+// summaries are the A operand, loaded straight from global/L2 into fragment registers with 16-byte
+// loads (the k index of both operands is permuted identically so that a lane's fragment pieces are
+// contiguous in memory); the G query vectors, padded to 8 columns, are the B operand and stay in
+// registers for all levels.  A candidate's g children occupy rows (r, r+8) of consecutive tiles, so
+// their logits meet in one lane and the child LSE needs no shuffles; the head sum takes two.
+// The selection logic (eligibility, forced nodes, Select_K, expansion) is the SIMT kernel's.
+#include <math_constants.h>
+
+#include "pisa_common.cuh"
+
+namespace pisa {
+
+namespace {
+
+constexpr int kWarpsPerCta = 4;
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint4 ldg128(const void* p) { return *reinterpret_cast<const uint4*>(p); }
+
+// running (max, sum exp) of one head's child logits
+__device__ __forceinline__ void lse_add(float& m, float& s, float z) {
+  const float mn = fmaxf(m, z);
+  s = s * __expf(m - mn) + __expf(z - mn);
+  m = mn;
+}
+
+}  // namespace
+
+template <int D, int NT>
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ pyr,
+                        int32_t* __restrict__ par_out, float* __restrict__ margin) {
+  constexpr int C4 = D / 32;              // groups of four 16-byte chunks per row (one chunk per tig)
+  __shared__ int s_cand[kWarpsPerCta][2][kMaxCand];
+  __shared__ __align__(16) float s_u[kWarpsPerCta][kMaxCand];
+  __shared__ float s_cut[kWarpsPerCta][2];
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gid = lane >> 2, tig = lane & 3;
+  const long long w = (long long)blockIdx.x * kWarpsPerCta + warp;
+  const long long total = (long long)geo.B * geo.Hkv * geo.N;
+  if (w >= total) return;
+  const int t = (int)(w % geo.N);
+  const int h = (int)((w / geo.N) % geo.Hkv);
+  const int b = (int)(w / ((long long)geo.N * geo.Hkv));
+  const int K = geo.K, g = geo.g, G = geo.G;
+  const int c = t / geo.C;
+  float* u = s_u[warp];
+
+  // B fragments: column n = gid is query head nt*8 + gid (zero beyond G); k permuted as the A loads
+  uint32_t bq[NT][C4][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    const int head = nt * 8 + gid;
+    const __nv_bfloat16* row = q + (long long)b * geo.qs[0] + (long long)t * geo.qs[1] +
+                               (long long)(h * G + head) * geo.qs[2];
+#pragma unroll
+    for (int c4 = 0; c4 < C4; ++c4) {
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (head < G) v = ldg128(row + (c4 * 4 + tig) * 8);
+      bq[nt][c4][0] = v.x; bq[nt][c4][1] = v.y; bq[nt][c4][2] = v.z; bq[nt][c4][3] = v.w;
+    }
+  }
+
+  int cur = 0;
+  int n = 1;
+  if (lane == 0) s_cand[warp][0][0] = 0;
+  float min_gap = CUDART_INF_F;
+  __syncwarp();
+
+  for (int l = geo.L; l >= 2; --l) {
+    int* cand = s_cand[warp][cur];
+    int* next = s_cand[warp][cur ^ 1];
+    const long long span = geo.span[l];
+    const int anc_c = (int)(c / span);
+    const int f1 = (c >= 1) ? (int)((c - 1) / span) : 0;
+    int nV = 0;
+    for (int s0 = 0; s0 < n; s0 += 32) {
+      const int s = s0 + lane;
+      const bool ok = (s < n) && (cand[s] <= anc_c);
+      nV += __popc(__ballot_sync(0xffffffffu, ok));
+    }
+    const bool prune = nV > K;
+    if (prune) {
+      const int Mb = geo.M[l - 1];
+      const __nv_bfloat16* below = pyr + geo.level_off[l - 1] + ((long long)b * geo.Hkv + h) * Mb * D;
+      for (int k0 = 0; k0 < nV; k0 += 8) {
+        const int kap = k0 + gid;
+        const bool has = kap < nV;
+        const int node = has ? cand[kap] : 0;
+        float m[NT][2], ssum[NT][2];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { m[nt][0] = m[nt][1] = -CUDART_INF_F; ssum[nt][0] = ssum[nt][1] = 0.f; }
+        for (int r0 = 0; r0 < g; r0 += 2) {
+          const int ch_lo = node * g + r0, ch_hi = ch_lo + 1;
+          const bool ok_lo = has && ch_lo < Mb, ok_hi = has && (r0 + 1 < g) && ch_hi < Mb;
+          uint4 lo[C4], hi[C4];
+#pragma unroll
+          for (int c4 = 0; c4 < C4; ++c4) {
+            lo[c4] = ok_lo ? ldg128(below + (long long)ch_lo * D + (c4 * 4 + tig) * 8) : make_uint4(0u, 0u, 0u, 0u);
+            hi[c4] = ok_hi ? ldg128(below + (long long)ch_hi * D + (c4 * 4 + tig) * 8) : make_uint4(0u, 0u, 0u, 0u);
+          }
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int c4 = 0; c4 < C4; ++c4) {
+              mma_bf16_16816(acc, lo[c4].x, hi[c4].x, lo[c4].y, hi[c4].y, bq[nt][c4][0], bq[nt][c4][1]);
+              mma_bf16_16816(acc, lo[c4].z, hi[c4].z, lo[c4].w, hi[c4].w, bq[nt][c4][2], bq[nt][c4][3]);
+            }
+            // acc[0..1]: child lo, heads nt*8 + 2*tig + {0,1};  acc[2..3]: child hi, same heads
+#pragma unroll
+            for (int jh = 0; jh < 2; ++jh) {
+              if (ok_lo) lse_add(m[nt][jh], ssum[nt][jh], acc[jh] * geo.scale);
+              if (ok_hi) lse_add(m[nt][jh], ssum[nt][jh], acc[2 + jh] * geo.scale);
+            }
+          }
+        }
+        float usum = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int jh = 0; jh < 2; ++jh)
+            if (nt * 8 + 2 * tig + jh < G && has) usum += m[nt][jh] + __logf(ssum[nt][jh]);
+        usum += __shfl_xor_sync(0xffffffffu, usum, 1);
+        usum += __shfl_xor_sync(0xffffffffu, usum, 2);
+        if (has && tig == 0) u[kap] = (node == 0 || node == f1 || node == anc_c) ? CUDART_INF_F : usum;
+      }
+      __syncwarp();
+    }
+    // Select_K: rank by (score desc, position asc); keep rank < K.  Without pruning keep all.
+    int base = 0;
+    for (int s0 = 0; s0 < nV; s0 += 32) {
+      const int s = s0 + lane;
+      bool keep = s < nV;
+      if (prune) {
+        int rank = 0;
+        const float ui = (s < nV) ? u[s] : 0.f;
+        for (int j = 0; j < nV; ++j) {
+          const float uj = u[j];
+          rank += (uj > ui) || (uj == ui && j < s);
+        }
+        keep = keep && (rank < K);
+        if (s < nV && rank == K - 1) s_cut[warp][0] = ui;
+        if (s < nV && rank == K) s_cut[warp][1] = ui;
+      }
+      const unsigned bal = __ballot_sync(0xffffffffu, keep);
+      const int pos = base + __popc(bal & ((1u << lane) - 1u));
+      if (keep) {
+        const int i = cand[s];
+        if (l == 2) {
+          par_out[w * (long long)K + pos] = i;
+        } else {
+          for (int r = 0; r < g; ++r) next[pos * g + r] = i * g + r;
+        }
+      }
+      base += __popc(bal);
+    }
+    __syncwarp();
+    if (prune) {
+      const float a = s_cut[warp][0], bb = s_cut[warp][1];
+      if (a < CUDART_INF_F) min_gap = fminf(min_gap, (a - bb) / fmaxf(fabsf(a), 1.f));
+    }
+    if (l == 2) {
+      for (int s = base + lane; s < K; s += 32) par_out[w * (long long)K + s] = -1;
+      if (margin != nullptr && lane == 0) margin[w] = min_gap;
+      return;
+    }
+    n = base * g;
+    cur ^= 1;
+  }
+}
+
+template <int D, int NT>
+static int launch_dn(const Geometry& g, const void* q, const void* pyr, int32_t* par, float* margin, cudaStream_t s) {
+  const long long total = (long long)g.B * g.Hkv * g.N;
+  const long long ctas = (total + kWarpsPerCta - 1) / kWarpsPerCta;
+  if (ctas > 0x7fffffffLL) return PISA_ERR_UNSUPPORTED;
+  route_stage1_mma_kernel<D, NT><<<(unsigned)ctas, kWarpsPerCta * 32, 0, s>>>(
+      g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pyr, par, margin);
+  return check_launch("route_stage1_mma");
+}
+
+bool route_stage1_mma_supported(const Geometry& g, int dtype) {
+  return dtype == PISA_BF16 && g.score_mode == PISA_SCORE_LSE && (g.d == 64 || g.d == 128) && g.L >= 2 &&
+         g.G <= 16;
+}
+
+int launch_route_stage1_mma(const Geometry& g, const void* q, const void* pyramid, int32_t* par, float* margin,
+                            cudaStream_t s) {
+  const bool wide = g.G > 8;
+  if (g.d == 128) return wide ? launch_dn<128, 2>(g, q, pyramid, par, margin, s) : launch_dn<128, 1>(g, q, pyramid, par, margin, s);
+  if (g.d == 64) return wide ? launch_dn<64, 2>(g, q, pyramid, par, margin, s) : launch_dn<64, 1>(g, q, pyramid, par, margin, s);
+  return PISA_ERR_UNSUPPORTED;
+}
+
+}  // namespace pisa

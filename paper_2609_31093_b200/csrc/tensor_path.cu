@@ -31,14 +31,20 @@ using namespace tc;
 namespace {
 
 constexpr int kInvTok = 1024;          // tokens per CTA in the inversion kernels
+constexpr int kWindowTok = 8192;       // tokens per window of the inverted lists
+constexpr int kRunTiles = 8;           // consecutive tiles a CTA takes at a time (round-robin over CTAs)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
 // ------------------------------------------------------------------ list inversion
 
+// A list is keyed by (b*Hkv + h, token window, node): window-major inside a head, so that the tiles
+// being worked on at any moment gather queries from (and, in the attention stage, accumulate into)
+// a slice of the sequence small enough to stay in L2.
 struct InvArgs {
   const int32_t* nodes;   // [BH, N, K] node ids (ascending, -1 padded)
   int K, fan, Mk, N, C, BH, tpt;
+  int W, NW;              // tokens per window (a multiple of kInvTok), windows per sequence
   int32_t* count;         // [BH*Mk]
   int32_t* entry_off;     // [BH*Mk + 1]
   int32_t* tile_off;      // [BH*Mk + 1]
@@ -54,6 +60,7 @@ __global__ void __launch_bounds__(256) inv_count_kernel(InvArgs a, int use_smem)
   extern __shared__ int s_hist[];
   const int bh = blockIdx.y;
   const int t0 = blockIdx.x * kInvTok, t1 = min(t0 + kInvTok, a.N);
+  const long long kbase = ((long long)bh * a.NW + t0 / a.W) * a.Mk;
   if (use_smem) {
     for (int j = threadIdx.x; j < a.Mk; j += blockDim.x) s_hist[j] = 0;
     __syncthreads();
@@ -64,20 +71,20 @@ __global__ void __launch_bounds__(256) inv_count_kernel(InvArgs a, int use_smem)
     const int node = a.nodes[((long long)bh * a.N + t0) * a.K + e];
     if (inv_valid(a, node, t)) {
       if (use_smem) atomicAdd(&s_hist[node], 1);
-      else atomicAdd(&a.count[(long long)bh * a.Mk + node], 1);
+      else atomicAdd(&a.count[kbase + node], 1);
     }
   }
   if (use_smem) {
     __syncthreads();
     for (int j = threadIdx.x; j < a.Mk; j += blockDim.x)
-      if (s_hist[j]) atomicAdd(&a.count[(long long)bh * a.Mk + j], s_hist[j]);
+      if (s_hist[j]) atomicAdd(&a.count[kbase + j], s_hist[j]);
   }
 }
 
 // exclusive scans of the list lengths (entries) and of their tile counts; one CTA
 __global__ void __launch_bounds__(1024) inv_scan_kernel(InvArgs a) {
   __shared__ int s_e[1024], s_t[1024];
-  const int nkeys = a.BH * a.Mk;
+  const int nkeys = a.BH * a.NW * a.Mk;
   const int per = (nkeys + 1023) / 1024;
   const int lo = min(nkeys, (int)threadIdx.x * per), hi = min(nkeys, lo + per);
   int se = 0, st = 0;
@@ -111,13 +118,14 @@ __global__ void __launch_bounds__(256) inv_fill_kernel(InvArgs a, int use_smem) 
   int* s_base = s_mem + a.Mk;
   const int bh = blockIdx.y;
   const int t0 = blockIdx.x * kInvTok, t1 = min(t0 + kInvTok, a.N);
+  const long long kbase = ((long long)bh * a.NW + t0 / a.W) * a.Mk;
   const int n = (t1 - t0) * a.K;
   const int32_t* nodes = a.nodes + ((long long)bh * a.N + t0) * a.K;
   if (!use_smem) {
     for (int e = threadIdx.x; e < n; e += blockDim.x) {
       const int t = t0 + e / a.K, slot = e % a.K, node = nodes[e];
       if (inv_valid(a, node, t)) {
-        const int pos = atomicAdd(&a.cursor[(long long)bh * a.Mk + node], 1);
+        const int pos = atomicAdd(&a.cursor[kbase + node], 1);
         a.entries[pos] = t | (slot << 24);
       }
     }
@@ -132,7 +140,7 @@ __global__ void __launch_bounds__(256) inv_fill_kernel(InvArgs a, int use_smem) 
   __syncthreads();
   for (int j = threadIdx.x; j < a.Mk; j += blockDim.x) {
     const int c = s_hist[j];
-    if (c) s_base[j] = atomicAdd(&a.cursor[(long long)bh * a.Mk + j], c);
+    if (c) s_base[j] = atomicAdd(&a.cursor[kbase + j], c);
     s_hist[j] = 0;
   }
   __syncthreads();
@@ -154,7 +162,7 @@ struct TileArgs {
   const int32_t* entry_off;
   const int32_t* tile_off;
   const int32_t* entries;
-  int nkeys, Mk, fan, slots;
+  int nkeys, Mk, NW, fan, slots;
   float* blk_lse;          // [BH, N, slots*fan, G]   (tile_lse)
   const float* row_lse;    // [B, Hq, N]              (tile_pv)
   float* o_acc;            // [B, N, Hq, D] fp32      (tile_pv)
@@ -175,38 +183,92 @@ __device__ __forceinline__ int find_key(const int32_t* tile_off, int nkeys, int 
   return lo;
 }
 
+// Thread `tid` of 128 always moves 16-byte chunk (tid % (D/8)) of rows (tid / (D/8)) + i * (1024/D):
+// the row index modulo 8 -- hence the swizzle -- is the same for every i, so the destination advances
+// by a constant and the loop body is one address computation and one copy.
+//
 // rows [row0, row0 + nrows) of a [tokens][D] bf16 matrix -> 128B-swizzled K-major slabs
 // (slab s holds elements [64 s, 64 s + 64) of every row); rows at or past `limit` become zeros
 template <int D>
 __device__ __forceinline__ void load_rows_swizzled(uint8_t* dst, int slab_bytes, const __nv_bfloat16* base,
                                                    long long row_stride, int row0, int nrows, int limit, int tid) {
-  constexpr int CH = D / 8;
-  for (int idx = tid; idx < nrows * CH; idx += 128) {
-    const int row = idx / CH, ck = idx % CH;
-    const uint32_t d = smem_u32(dst + (ck >> 3) * slab_bytes) + swz128(row, ck & 7);
-    if (row0 + row < limit) cp_async16(d, base + (long long)(row0 + row) * row_stride + ck * 8);
+  constexpr int CH = D / 8, RPP = 128 / CH;
+  const int ck = tid % CH, rb = tid / CH;
+  uint32_t d = smem_u32(dst + (ck >> 3) * slab_bytes) + swz128(rb, ck & 7);
+  const __nv_bfloat16* src = base + (long long)(row0 + rb) * row_stride + ck * 8;
+  for (int row = rb; row < nrows; row += RPP) {
+    if (row0 + row < limit) cp_async16(d, src);
     else st_shared_zero16(d);
+    d += RPP * 128;
+    src += (long long)RPP * row_stride;
   }
 }
 
-// gathered query rows: row r = (entry r / G, head r % G)
+// gathered query rows: row r = (entry r >> lgG, head r & (G-1))
 template <int D>
 __device__ __forceinline__ void gather_q_swizzled(uint8_t* dst, const Geometry& geo, const __nv_bfloat16* q,
                                                   int b, int h, const int* s_ent, int tid) {
-  constexpr int CH = D / 8;
-  const int G = geo.G;
-  for (int idx = tid; idx < 128 * CH; idx += 128) {
-    const int row = idx / CH, ck = idx % CH;
-    const uint32_t d = smem_u32(dst + (ck >> 3) * (128 * 128)) + swz128(row, ck & 7);
-    const int ent = s_ent[row / G];
-    if (ent >= 0) {
-      const int t = ent & 0xFFFFFF;
-      cp_async16(d, q + (long long)b * geo.qs[0] + (long long)t * geo.qs[1] +
-                        (long long)(h * G + row % G) * geo.qs[2] + ck * 8);
-    } else {
-      st_shared_zero16(d);
-    }
+  constexpr int CH = D / 8, RPP = 128 / CH;
+  const int ck = tid % CH, rb = tid / CH;
+  const int G = geo.G, lgG = 31 - __clz(G);
+  uint32_t d = smem_u32(dst + (ck >> 3) * (128 * 128)) + swz128(rb, ck & 7);
+  const __nv_bfloat16* qb = q + (long long)b * geo.qs[0] + (long long)(h * G) * geo.qs[2] + ck * 8;
+  const long long s1 = geo.qs[1], s2 = geo.qs[2];
+#pragma unroll 4
+  for (int row = rb; row < 128; row += RPP) {
+    const int ent = s_ent[row >> lgG];
+    if (ent >= 0) cp_async16(d, qb + (long long)(ent & 0xFFFFFF) * s1 + (long long)(row & (G - 1)) * s2);
+    else st_shared_zero16(d);
+    d += RPP * 128;
   }
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Online log-sum-exp (base 2) over one 32-column chunk of raw fp32 logits; (m, ssum) is the running
+// (max, sum of 2^(x - max)) with x = raw * sl2.  sl2 > 0, so the max commutes with the scaling.
+__device__ __forceinline__ void lse_chunk(const uint32_t (&rr)[32], float sl2, float& m, float& ssum) {
+  float c0 = __uint_as_float(rr[0]), c1 = __uint_as_float(rr[1]);
+  float c2 = __uint_as_float(rr[2]), c3 = __uint_as_float(rr[3]);
+#pragma unroll
+  for (int j = 4; j < 32; j += 4) {
+    c0 = fmaxf(c0, __uint_as_float(rr[j]));
+    c1 = fmaxf(c1, __uint_as_float(rr[j + 1]));
+    c2 = fmaxf(c2, __uint_as_float(rr[j + 2]));
+    c3 = fmaxf(c3, __uint_as_float(rr[j + 3]));
+  }
+  const float mn = fmaxf(m, fmaxf(fmaxf(c0, c1), fmaxf(c2, c3)) * sl2);
+  const float neg = -mn;
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+  for (int j = 0; j < 32; j += 4) {
+    a0 += ex2_approx(fmaf(__uint_as_float(rr[j]), sl2, neg));
+    a1 += ex2_approx(fmaf(__uint_as_float(rr[j + 1]), sl2, neg));
+    a2 += ex2_approx(fmaf(__uint_as_float(rr[j + 2]), sl2, neg));
+    a3 += ex2_approx(fmaf(__uint_as_float(rr[j + 3]), sl2, neg));
+  }
+  ssum = ssum * ex2_approx(m - mn) + ((a0 + a1) + (a2 + a3));
+  m = mn;
+}
+// the same with only the first `nvalid` (>= 1) columns of the chunk taking part
+__device__ __forceinline__ void lse_chunk_masked(const uint32_t (&rr)[32], int nvalid, float sl2, float& m,
+                                                 float& ssum) {
+  float cm = -CUDART_INF_F;
+#pragma unroll
+  for (int j = 0; j < 32; ++j)
+    if (j < nvalid) cm = fmaxf(cm, __uint_as_float(rr[j]));
+  const float mn = fmaxf(m, cm * sl2);
+  const float neg = -mn;
+  float acc = 0.f;
+#pragma unroll
+  for (int j = 0; j < 32; ++j)
+    if (j < nvalid) acc += ex2_approx(fmaf(__uint_as_float(rr[j]), sl2, neg));
+  ssum = ssum * ex2_approx(m - mn) + acc;
+  m = mn;
 }
 
 // Per-head log-sum-exp of the scaled logits of every (gathered query row, child leaf) pair of a
@@ -235,88 +297,83 @@ __global__ void __launch_bounds__(128) tile_lse_kernel(Geometry geo, TileArgs a)
 
   const int G = geo.G, tpt = 128 / G, C = geo.C;
   const int T = a.tile_off[a.nkeys];
-  const int per = (T + (int)gridDim.x - 1) / (int)gridDim.x;
-  const int tile_begin = min(T, (int)blockIdx.x * per), tile_end = min(T, tile_begin + per);
   const float sl2 = geo.scale * kLog2e;
   const uint32_t idesc = make_idesc_bf16(128, NB, 0, 0);
+  const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
   uint32_t phase = 0;
-  int key = (tile_begin < tile_end) ? find_key(a.tile_off, a.nkeys, tile_begin) : 0;
   int loaded_key = -1;
+  bool failed = false;
 
-  for (int tile = tile_begin; tile < tile_end; ++tile) {
-    while (tile >= a.tile_off[key + 1]) ++key;
-    const int bh = key / a.Mk, j = key % a.Mk;
-    const int b = bh / geo.Hkv, h = bh % geo.Hkv;
-    const int e0 = a.entry_off[key] + (tile - a.tile_off[key]) * tpt;
-    const int n_e = min(tpt, a.entry_off[key + 1] - e0);
-    if (tid < tpt) s_ent[tid] = (tid < n_e) ? a.entries[e0 + tid] : -1;
-    __syncthreads();      // entries visible; the previous tile's TMEM reads and smem reads are done
-    if (key != loaded_key) {
-      load_rows_swizzled<D>(sB, B_SLAB, a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2], geo.ks[1],
-                            j * NB, NB, geo.N, tid);
-      loaded_key = key;
-    }
-    gather_q_swizzled<D>(sA, geo, a.q, b, h, s_ent, tid);
-    const int ent = s_ent[tid / G];     // read before the barrier: the next iteration rewrites s_ent
-    cp_async_wait_all();
-    fence_proxy_async_smem();
-    __syncthreads();
-    if (tid == 0) {
+  for (int run = blockIdx.x; run * kRunTiles < T && !failed; run += gridDim.x) {
+    const int tile0 = run * kRunTiles, tile1 = min(T, tile0 + kRunTiles);
+    int key = find_key(a.tile_off, a.nkeys, tile0);
+    for (int tile = tile0; tile < tile1; ++tile) {
+      while (tile >= a.tile_off[key + 1]) ++key;
+      const int bh = key / (a.NW * a.Mk), j = key % a.Mk;
+      const int b = bh / geo.Hkv, h = bh % geo.Hkv;
+      const int e0 = a.entry_off[key] + (tile - a.tile_off[key]) * tpt;
+      const int n_e = min(tpt, a.entry_off[key + 1] - e0);
+      if (tid < tpt) s_ent[tid] = (tid < n_e) ? a.entries[e0 + tid] : -1;
+      __syncthreads();      // entries visible; the previous tile's TMEM reads and smem reads are done
+      if (key != loaded_key) {
+        load_rows_swizzled<D>(sB, B_SLAB, a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2], geo.ks[1],
+                              j * NB, NB, geo.N, tid);
+        loaded_key = key;
+      }
+      gather_q_swizzled<D>(sA, geo, a.q, b, h, s_ent, tid);
+      const int ent = s_ent[tid >> (31 - __clz(G))];     // read before the barrier: the next iteration rewrites s_ent
+      cp_async_wait_all();
+      fence_proxy_async_smem();
+      __syncthreads();
+      if (tid == 0) {
+        tcgen05_fence_after_sync();
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint64_t da = make_smem_desc(smem_u32(sA) + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
+          const uint64_t db = make_smem_desc(smem_u32(sB) + (kk >> 2) * B_SLAB + (kk & 3) * 32, 0, 1024);
+          umma_bf16(tmem, da, db, idesc, kk > 0);
+        }
+        umma_commit(&bar);
+      }
+      const bool ok = mbar_wait_bounded(&bar, phase);
+      phase ^= 1u;
+      if (__syncthreads_or(!ok)) { failed = true; break; }
       tcgen05_fence_after_sync();
-#pragma unroll
-      for (int kk = 0; kk < D / 16; ++kk) {
-        const uint64_t da = make_smem_desc(smem_u32(sA) + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
-        const uint64_t db = make_smem_desc(smem_u32(sB) + (kk >> 2) * B_SLAB + (kk & 3) * 32, 0, 1024);
-        umma_bf16(tmem, da, db, idesc, kk > 0);
-      }
-      umma_commit(&bar);
-    }
-    const bool ok = mbar_wait_bounded(&bar, phase);
-    phase ^= 1u;
-    if (__syncthreads_or(!ok)) {
-      if (tid == 0) atomicExch(a.status, (int)PISA_ERR_TIMEOUT);
-      break;
-    }
-    tcgen05_fence_after_sync();
 
-    const int head = tid % G;
-    const bool valid = ent >= 0;
-    const int t = ent & 0xFFFFFF, slot = valid ? (ent >> 24) : 0;
-    const int c_t = t / C;
-    const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-    for (int r = 0; r < a.fan; ++r) {
-      const int leaf = j * a.fan + r;
-      int ncols = 0;
-      if (valid && leaf <= c_t && leaf < geo.M[1])
-        ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
-      float m = -CUDART_INF_F, ssum = 0.f;
-      for (int c0 = 0; c0 < C; c0 += 32) {
-        uint32_t rr[32];
-        tmem_ld_32x32(lane_base + (uint32_t)(r * C + c0), rr);
-        tmem_ld_wait();
-        float x[32];
-        float cm = -CUDART_INF_F;
-#pragma unroll
-        for (int jx = 0; jx < 32; ++jx) {
-          x[jx] = (c0 + jx < ncols) ? __uint_as_float(rr[jx]) * sl2 : -CUDART_INF_F;
-          cm = fmaxf(cm, x[jx]);
+      const int head = tid & (G - 1);
+      const bool valid = ent >= 0;
+      const int t = ent & 0xFFFFFF, slot = valid ? (ent >> 24) : 0;
+      const int c_t = t / C;
+      for (int r = 0; r < a.fan; ++r) {
+        const int leaf = j * a.fan + r;
+        int ncols = 0;
+        if (valid && leaf <= c_t && leaf < geo.M[1])
+          ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
+        // whole-warp fast path: every row either takes all C columns or does not need a result
+        const bool fast = __all_sync(0xffffffffu, ncols == C || ncols == 0);
+        float m = -CUDART_INF_F, ssum = 0.f;
+        uint32_t ra[32], rb[32];
+        const uint32_t col0 = lane_base + (uint32_t)(r * C);
+        tmem_ld_32x32(col0, ra);
+        for (int c0 = 0; c0 < C; c0 += 64) {
+          tmem_ld_wait();
+          tmem_ld_32x32(col0 + (uint32_t)(c0 + 32), rb);
+          if (fast) lse_chunk(ra, sl2, m, ssum);
+          else if (c0 < ncols) lse_chunk_masked(ra, ncols - c0, sl2, m, ssum);
+          tmem_ld_wait();
+          if (c0 + 64 < C) tmem_ld_32x32(col0 + (uint32_t)(c0 + 64), ra);
+          if (fast) lse_chunk(rb, sl2, m, ssum);
+          else if (c0 + 32 < ncols) lse_chunk_masked(rb, ncols - c0 - 32, sl2, m, ssum);
         }
-        if (cm > -CUDART_INF_F) {
-          const float mn = fmaxf(m, cm);
-          float acc = 0.f;
-#pragma unroll
-          for (int jx = 0; jx < 32; ++jx) acc += exp2f(x[jx] - mn);
-          ssum = ssum * exp2f(m - mn) + acc;
-          m = mn;
+        if (valid) {
+          const float lse = (ncols > 0) ? (m + log2f(ssum)) * kLn2 : -CUDART_INF_F;
+          a.blk_lse[(((long long)bh * geo.N + t) * (a.slots * a.fan) + slot * a.fan + r) * G + head] = lse;
         }
       }
-      if (valid) {
-        const float lse = (ssum > 0.f) ? (m + log2f(ssum)) * kLn2 : -CUDART_INF_F;
-        a.blk_lse[(((long long)bh * geo.N + t) * (a.slots * a.fan) + slot * a.fan + r) * G + head] = lse;
-      }
+      tcgen05_fence_before_sync();
     }
-    tcgen05_fence_before_sync();
   }
+  if (failed && tid == 0) atomicExch(a.status, (int)PISA_ERR_TIMEOUT);
   tcgen05_fence_before_sync();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, TM_COLS);
@@ -330,7 +387,6 @@ template <int D, int C>
 __global__ void __launch_bounds__(128) tile_pv_kernel(Geometry geo, TileArgs a) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int KS = D / 64;                 // 64-wide slabs of d
-  constexpr int PS = C / 64;                 // 64-wide slabs of keys (P operand)
   constexpr int A_SLAB = 128 * 128, KV_SLAB = C * 128;
   constexpr int STAGE_ROW = 256 + 16;        // 64 fp32 + pad: conflict-free 16-byte row writes
   constexpr int QP_BYTES = (KS * A_SLAB > 128 * STAGE_ROW) ? KS * A_SLAB : 128 * STAGE_ROW;
@@ -355,135 +411,149 @@ __global__ void __launch_bounds__(128) tile_pv_kernel(Geometry geo, TileArgs a) 
 
   const int G = geo.G, tpt = 128 / G;
   const int T = a.tile_off[a.nkeys];
-  const int per = (T + (int)gridDim.x - 1) / (int)gridDim.x;
-  const int tile_begin = min(T, (int)blockIdx.x * per), tile_end = min(T, tile_begin + per);
   const float sl2 = geo.scale * kLog2e;
   const uint32_t idesc_s = make_idesc_bf16(128, C, 0, 0);
   const uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
+  const uint32_t s_base = tmem_s + ((uint32_t)(warp * 32) << 16);
+  const uint32_t o_base = tmem_o + ((uint32_t)(warp * 32) << 16);
+  uint8_t* stage = sQ + tid * STAGE_ROW;
   uint32_t phase = 0;
-  int key = (tile_begin < tile_end) ? find_key(a.tile_off, a.nkeys, tile_begin) : 0;
   int loaded_key = -1;
   bool failed = false;
 
-  for (int tile = tile_begin; tile < tile_end; ++tile) {
-    while (tile >= a.tile_off[key + 1]) ++key;
-    const int bh = key / a.Mk, leaf = key % a.Mk;
-    const int b = bh / geo.Hkv, h = bh % geo.Hkv;
-    const int e0 = a.entry_off[key] + (tile - a.tile_off[key]) * tpt;
-    const int n_e = min(tpt, a.entry_off[key + 1] - e0);
-    if (tid < tpt) s_ent[tid] = (tid < n_e) ? a.entries[e0 + tid] : -1;
-    bulk_wait_read_all();    // this thread's staging rows of the previous tile have been read
-    __syncthreads();
-    if (key != loaded_key) {
-      load_rows_swizzled<D>(sK, KV_SLAB, a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2], geo.ks[1],
-                            leaf * C, C, geo.N, tid);
-      load_rows_swizzled<D>(sV, KV_SLAB, a.v + (long long)b * geo.vs[0] + (long long)h * geo.vs[2], geo.vs[1],
-                            leaf * C, C, geo.N, tid);
-      loaded_key = key;
-    }
-    gather_q_swizzled<D>(sQ, geo, a.q, b, h, s_ent, tid);
+  for (int run = blockIdx.x; run * kRunTiles < T && !failed; run += gridDim.x) {
+    const int tile0 = run * kRunTiles, tile1 = min(T, tile0 + kRunTiles);
+    int key = find_key(a.tile_off, a.nkeys, tile0);
+    for (int tile = tile0; tile < tile1; ++tile) {
+      while (tile >= a.tile_off[key + 1]) ++key;
+      const int bh = key / (a.NW * a.Mk), leaf = key % a.Mk;
+      const int b = bh / geo.Hkv, h = bh % geo.Hkv;
+      const int e0 = a.entry_off[key] + (tile - a.tile_off[key]) * tpt;
+      const int n_e = min(tpt, a.entry_off[key + 1] - e0);
+      if (tid < tpt) s_ent[tid] = (tid < n_e) ? a.entries[e0 + tid] : -1;
+      bulk_wait_read_all();    // this thread's staging rows of the previous tile have been read
+      __syncthreads();
+      if (key != loaded_key) {
+        load_rows_swizzled<D>(sK, KV_SLAB, a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2], geo.ks[1],
+                              leaf * C, C, geo.N, tid);
+        load_rows_swizzled<D>(sV, KV_SLAB, a.v + (long long)b * geo.vs[0] + (long long)h * geo.vs[2], geo.vs[1],
+                              leaf * C, C, geo.N, tid);
+        loaded_key = key;
+      }
+      gather_q_swizzled<D>(sQ, geo, a.q, b, h, s_ent, tid);
 
-    const int ent = s_ent[tid / G];
-    const int head = tid % G;
-    const bool valid = ent >= 0;
-    const int t = ent & 0xFFFFFF;
-    const int hq = h * G + head;
-    float lse2 = 0.f;                  // row denominator in log2 units
-    int ncols = 0;
-    if (valid) {
-      lse2 = a.row_lse[((long long)b * geo.Hq + hq) * geo.N + t] * kLog2e;
-      const int c_t = t / C;
-      if (leaf <= c_t && lse2 > -CUDART_INF_F) ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
-    }
-    cp_async_wait_all();
-    fence_proxy_async_smem();
-    __syncthreads();
-    if (tid == 0) {
+      const int ent = s_ent[tid >> (31 - __clz(G))];
+      const int head = tid & (G - 1);
+      const bool valid = ent >= 0;
+      const int t = ent & 0xFFFFFF;
+      const int hq = h * G + head;
+      float neg_lse2 = 0.f;              // minus the row denominator, in log2 units
+      int ncols = 0;
+      if (valid) {
+        const float l2 = a.row_lse[((long long)b * geo.Hq + hq) * geo.N + t] * kLog2e;
+        const int c_t = t / C;
+        if (leaf <= c_t && l2 > -CUDART_INF_F) ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
+        neg_lse2 = -l2;
+      }
+      cp_async_wait_all();
+      fence_proxy_async_smem();
+      __syncthreads();
+      if (tid == 0) {
+        tcgen05_fence_after_sync();
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint64_t da = make_smem_desc(smem_u32(sQ) + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
+          const uint64_t db = make_smem_desc(smem_u32(sK) + (kk >> 2) * KV_SLAB + (kk & 3) * 32, 0, 1024);
+          umma_bf16(tmem_s, da, db, idesc_s, kk > 0);
+        }
+        umma_commit(&bar);
+      }
+      bool ok = mbar_wait_bounded(&bar, phase);
+      phase ^= 1u;
+      if (__syncthreads_or(!ok)) { failed = true; break; }
       tcgen05_fence_after_sync();
-#pragma unroll
-      for (int kk = 0; kk < D / 16; ++kk) {
-        const uint64_t da = make_smem_desc(smem_u32(sQ) + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
-        const uint64_t db = make_smem_desc(smem_u32(sK) + (kk >> 2) * KV_SLAB + (kk & 3) * 32, 0, 1024);
-        umma_bf16(tmem_s, da, db, idesc_s, kk > 0);
-      }
-      umma_commit(&bar);
-    }
-    bool ok = mbar_wait_bounded(&bar, phase);
-    phase ^= 1u;
-    if (__syncthreads_or(!ok)) { failed = true; break; }
-    tcgen05_fence_after_sync();
 
-    // P = exp2(S*scale*log2e - lse2), masked, as the bf16 K-major A operand (overwrites the Q tile:
-    // the S chain that read it has completed)
-    const uint32_t lane_base = tmem_s + ((uint32_t)(warp * 32) << 16);
+      // P = 2^(S*scale*log2e - lse2), masked, as the bf16 K-major A operand (overwrites the Q tile:
+      // the S chain that read it has completed)
+      {
+        const bool fast = __all_sync(0xffffffffu, ncols == C);
+        uint32_t ra[32], rb[32];
+        tmem_ld_32x32(s_base, ra);
 #pragma unroll
-    for (int c0 = 0; c0 < C; c0 += 32) {
-      uint32_t rr[32];
-      tmem_ld_32x32(lane_base + (uint32_t)c0, rr);
-      tmem_ld_wait();
-      uint32_t pk[16];
+        for (int c0 = 0; c0 < C; c0 += 32) {
+          uint32_t (&cur)[32] = ((c0 >> 5) & 1) ? rb : ra;
+          uint32_t (&nxt)[32] = ((c0 >> 5) & 1) ? ra : rb;
+          tmem_ld_wait();
+          if (c0 + 32 < C) tmem_ld_32x32(s_base + (uint32_t)(c0 + 32), nxt);
+          uint32_t pk[16];
 #pragma unroll
-      for (int jx = 0; jx < 16; ++jx) {
-        const float p0 = (c0 + 2 * jx < ncols) ? exp2f(__uint_as_float(rr[2 * jx]) * sl2 - lse2) : 0.f;
-        const float p1 = (c0 + 2 * jx + 1 < ncols) ? exp2f(__uint_as_float(rr[2 * jx + 1]) * sl2 - lse2) : 0.f;
-        const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
-        pk[jx] = *reinterpret_cast<const uint32_t*>(&pp);
+          for (int jx = 0; jx < 16; ++jx) {
+            float p0 = ex2_approx(fmaf(__uint_as_float(cur[2 * jx]), sl2, neg_lse2));
+            float p1 = ex2_approx(fmaf(__uint_as_float(cur[2 * jx + 1]), sl2, neg_lse2));
+            if (!fast) {
+              if (c0 + 2 * jx >= ncols) p0 = 0.f;
+              if (c0 + 2 * jx + 1 >= ncols) p1 = 0.f;
+            }
+            const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
+            pk[jx] = *reinterpret_cast<const uint32_t*>(&pp);
+          }
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const int ck = c0 / 8 + q4;                       // 16-byte chunk (8 keys) of this row
+            const uint32_t d = smem_u32(sQ + (ck >> 3) * A_SLAB) + swz128(tid, ck & 7);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d), "r"(pk[4 * q4]),
+                         "r"(pk[4 * q4 + 1]), "r"(pk[4 * q4 + 2]), "r"(pk[4 * q4 + 3])
+                         : "memory");
+          }
+        }
       }
+      fence_proxy_async_smem();
+      tcgen05_fence_before_sync();
+      __syncthreads();
+      if (tid == 0) {
+        tcgen05_fence_after_sync();
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        const int ck = c0 / 8 + q4;                       // 16-byte chunk (8 keys) of this row
-        const uint32_t d = smem_u32(sQ + (ck >> 3) * A_SLAB) + swz128(tid, ck & 7);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d), "r"(pk[4 * q4]), "r"(pk[4 * q4 + 1]),
-                     "r"(pk[4 * q4 + 2]), "r"(pk[4 * q4 + 3])
-                     : "memory");
+        for (int kk = 0; kk < C / 16; ++kk) {
+          const uint64_t da = make_smem_desc(smem_u32(sQ) + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
+          const uint64_t db = make_smem_desc(smem_u32(sV) + kk * (16 * 128), KV_SLAB, 1024);
+          umma_bf16(tmem_o, da, db, idesc_o, kk > 0);
+        }
+        umma_commit(&bar);
       }
-    }
-    fence_proxy_async_smem();
-    tcgen05_fence_before_sync();
-    __syncthreads();
-    if (tid == 0) {
+      ok = mbar_wait_bounded(&bar, phase);
+      phase ^= 1u;
+      if (__syncthreads_or(!ok)) { failed = true; break; }
       tcgen05_fence_after_sync();
-#pragma unroll
-      for (int kk = 0; kk < C / 16; ++kk) {
-        const uint64_t da = make_smem_desc(smem_u32(sQ) + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
-        const uint64_t db = make_smem_desc(smem_u32(sV) + kk * (16 * 128), KV_SLAB, 1024);
-        umma_bf16(tmem_o, da, db, idesc_o, kk > 0);
-      }
-      umma_commit(&bar);
-    }
-    ok = mbar_wait_bounded(&bar, phase);
-    phase ^= 1u;
-    if (__syncthreads_or(!ok)) { failed = true; break; }
-    tcgen05_fence_after_sync();
 
-    // O partial: 64 columns at a time through this thread's private staging row, then one bulk
-    // reduction (256 bytes) into the fp32 accumulator row of (b, t, hq)
-    const uint32_t o_base = tmem_o + ((uint32_t)(warp * 32) << 16);
-    uint8_t* stage = sQ + tid * STAGE_ROW;
-    float* orow = a.o_acc + (((long long)b * geo.N + t) * geo.Hq + hq) * D;
+      // O partial: 64 columns at a time through this thread's private staging row, then one bulk
+      // reduction (256 bytes) into the fp32 accumulator row of (b, t, hq)
+      float* orow = a.o_acc + (((long long)b * geo.N + t) * geo.Hq + hq) * D;
 #pragma unroll
-    for (int half = 0; half < KS; ++half) {
-      if (half > 0) bulk_wait_read_all();
-#pragma unroll
-      for (int c0 = 0; c0 < 64; c0 += 32) {
-        uint32_t rr[32];
-        tmem_ld_32x32(o_base + (uint32_t)(half * 64 + c0), rr);
+      for (int half = 0; half < KS; ++half) {
+        uint32_t ra[32], rb[32];
+        tmem_ld_32x32(o_base + (uint32_t)(half * 64), ra);
+        tmem_ld_32x32(o_base + (uint32_t)(half * 64 + 32), rb);
+        if (half > 0) bulk_wait_read_all();
         tmem_ld_wait();
 #pragma unroll
         for (int q4 = 0; q4 < 8; ++q4)
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(stage) + (c0 + 4 * q4) * 4),
-                       "r"(rr[4 * q4]), "r"(rr[4 * q4 + 1]), "r"(rr[4 * q4 + 2]), "r"(rr[4 * q4 + 3])
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(stage) + q4 * 16), "r"(ra[4 * q4]),
+                       "r"(ra[4 * q4 + 1]), "r"(ra[4 * q4 + 2]), "r"(ra[4 * q4 + 3])
                        : "memory");
+#pragma unroll
+        for (int q4 = 0; q4 < 8; ++q4)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(stage) + 128 + q4 * 16),
+                       "r"(rb[4 * q4]), "r"(rb[4 * q4 + 1]), "r"(rb[4 * q4 + 2]), "r"(rb[4 * q4 + 3])
+                       : "memory");
+        fence_proxy_async_smem();
+        if (valid) {
+          bulk_reduce_add_f32(orow + half * 64, smem_u32(stage), 256);
+          bulk_commit();
+        }
       }
-      fence_proxy_async_smem();
-      if (valid) {
-        bulk_reduce_add_f32(orow + half * 64, smem_u32(stage), 256);
-        bulk_commit();
-      }
+      tcgen05_fence_before_sync();
     }
-    tcgen05_fence_before_sync();
   }
-  (void)PS;
   if (failed && tid == 0) atomicExch(a.status, (int)PISA_ERR_TIMEOUT);
   bulk_wait_all();
   tcgen05_fence_before_sync();
@@ -640,8 +710,11 @@ struct InvLayout {
   size_t count, entry_off, tile_off, cursor, entries, end;
 };
 
+int window_tokens(const Geometry& g) { return g.N < kWindowTok ? ((g.N + kInvTok - 1) / kInvTok) * kInvTok : kWindowTok; }
+int num_windows(const Geometry& g) { return (g.N + window_tokens(g) - 1) / window_tokens(g); }
+
 InvLayout inv_layout(size_t base, const Geometry& g, int Mk) {
-  const size_t nkeys = (size_t)g.B * g.Hkv * Mk;
+  const size_t nkeys = (size_t)g.B * g.Hkv * num_windows(g) * Mk;
   InvLayout l;
   size_t o = base;
   l.count = o; o += align_up(nkeys * 4, 256);
@@ -690,10 +763,11 @@ int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char
   InvArgs a;
   a.nodes = nodes; a.K = g.K; a.fan = fan; a.Mk = Mk; a.N = g.N; a.C = g.C; a.BH = g.B * g.Hkv;
   a.tpt = 128 / g.G;
+  a.W = window_tokens(g); a.NW = num_windows(g);
   a.count = (int32_t*)(ws + l.count); a.entry_off = (int32_t*)(ws + l.entry_off);
   a.tile_off = (int32_t*)(ws + l.tile_off); a.cursor = (int32_t*)(ws + l.cursor);
   a.entries = (int32_t*)(ws + l.entries);
-  const size_t nkeys = (size_t)a.BH * Mk;
+  const size_t nkeys = (size_t)a.BH * a.NW * Mk;
   cudaError_t e = cudaMemsetAsync(a.count, 0, nkeys * 4, s);
   if (e != cudaSuccess) { record_cuda_error("inversion memset", e); return PISA_ERR_CUDA; }
   const int use_smem = (2 * (size_t)Mk * 4 <= 96 * 1024) ? 1 : 0;
@@ -779,7 +853,8 @@ int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, con
   const RouteLayout L = route_layout(g);
   int32_t* par = (int32_t*)(ws + L.par);
   float* blk = (float*)(ws + L.blk);
-  int st = launch_route_stage1_simt(g, dtype, q, pyramid, par, margin, s);
+  int st = route_stage1_mma_supported(g, dtype) ? launch_route_stage1_mma(g, q, pyramid, par, margin, s)
+                                                : launch_route_stage1_simt(g, dtype, q, pyramid, par, margin, s);
   if (st != PISA_OK) return st;
   InvArgs inv;
   st = run_inversion(g, par, g.g, g.M[2], ws, L.inv, &inv, s);
@@ -787,7 +862,7 @@ int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, con
   TileArgs a = {};
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = nullptr;
   a.entry_off = inv.entry_off; a.tile_off = inv.tile_off; a.entries = inv.entries;
-  a.nkeys = g.B * g.Hkv * g.M[2]; a.Mk = g.M[2]; a.fan = g.g; a.slots = g.K;
+  a.nkeys = g.B * g.Hkv * inv.NW * g.M[2]; a.Mk = g.M[2]; a.NW = inv.NW; a.fan = g.g; a.slots = g.K;
   a.blk_lse = blk; a.status = status;
   st = dispatch_tile_lse(g, g.g * g.C, a, s);
   if (st != PISA_OK) return st;
@@ -809,7 +884,7 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
   TileArgs a = {};
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
   a.entry_off = inv.entry_off; a.tile_off = inv.tile_off; a.entries = inv.entries;
-  a.nkeys = g.B * g.Hkv * g.M[1]; a.Mk = g.M[1]; a.fan = 1; a.slots = g.K;
+  a.nkeys = g.B * g.Hkv * inv.NW * g.M[1]; a.Mk = g.M[1]; a.NW = inv.NW; a.fan = 1; a.slots = g.K;
   a.blk_lse = blk; a.row_lse = lse; a.o_acc = acc; a.status = status;
   if (!lse_ready) {
     st = dispatch_tile_lse(g, g.C, a, s);
