@@ -9,13 +9,13 @@
 //
 //   routing   : stage 1 (levels L..2, SIMT) -> kept level-2 nodes
 //               invert by level-2 node      -> lists of (token, slot)
-//               tile_lse_kernel             -> per-head LSE of every child leaf (g*C keys per tile),
+//               lse_ws_kernel               -> per-head LSE of every child leaf (g*C keys per tile),
 //                                              causal mask inside the query's own leaf
 //               final_topk_kernel           -> grouped score = sum over heads, forced leaves, Top-K;
 //                                              also the softmax denominator of the kept leaves
 //   attention : invert idx by leaf          -> lists of (token, slot)
-//               [tile_lse + row_lse only when the denominators are not already known]
-//               tile_pv_kernel              -> S = Q K^T, P = exp(S - lse_row) (already normalised),
+//               [lse_ws + row_lse only when the denominators are not already known]
+//               pv_ws_kernel                -> S = Q K^T, P = exp(S - lse_row) (already normalised),
 //                                              O_partial = P V, added into an fp32 accumulator with
 //                                              bulk reductions (one 256-byte row segment per thread)
 //               convert                     -> out in the storage dtype
@@ -32,7 +32,7 @@ namespace {
 
 constexpr int kInvTok = 1024;          // tokens per CTA in the inversion kernels
 constexpr int kWindowTok = 8192;       // tokens per window of the inverted lists
-constexpr int kRunTiles = 8;           // consecutive tiles a CTA takes at a time (round-robin over CTAs)
+constexpr int kItemTiles = 16;         // a work item: at most this many consecutive tiles of one list
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -47,8 +47,10 @@ struct InvArgs {
   int W, NW;              // tokens per window (a multiple of kInvTok), windows per sequence
   int32_t* count;         // [BH*Mk]
   int32_t* entry_off;     // [BH*Mk + 1]
-  int32_t* tile_off;      // [BH*Mk + 1]
-  int32_t* cursor;        // [BH*Mk]
+  int32_t* tile_off;      // [nkeys + 1]  tiles of tpt tokens
+  int32_t* item_off;      // [nkeys + 1]  work items: runs of at most kItemTiles tiles of one list
+  int32_t* item_key;      // [items]      the list each work item belongs to
+  int32_t* cursor;        // [nkeys]
   int32_t* entries;       // [<= BH*N*K]  token | slot << 24
 };
 
@@ -81,35 +83,40 @@ __global__ void __launch_bounds__(256) inv_count_kernel(InvArgs a, int use_smem)
   }
 }
 
-// exclusive scans of the list lengths (entries) and of their tile counts; one CTA
+// exclusive scans of the list lengths (entries), of their tile counts and of their work-item
+// counts; one CTA
 __global__ void __launch_bounds__(1024) inv_scan_kernel(InvArgs a) {
-  __shared__ int s_e[1024], s_t[1024];
+  __shared__ int s_e[1024], s_t[1024], s_i[1024];
   const int nkeys = a.BH * a.NW * a.Mk;
   const int per = (nkeys + 1023) / 1024;
   const int lo = min(nkeys, (int)threadIdx.x * per), hi = min(nkeys, lo + per);
-  int se = 0, st = 0;
+  int se = 0, st = 0, si = 0;
   for (int i = lo; i < hi; ++i) {
     const int c = a.count[i];
-    se += c;
-    st += (c + a.tpt - 1) / a.tpt;
+    const int tl = (c + a.tpt - 1) / a.tpt;
+    se += c; st += tl; si += (tl + kItemTiles - 1) / kItemTiles;
   }
-  s_e[threadIdx.x] = se; s_t[threadIdx.x] = st;
+  s_e[threadIdx.x] = se; s_t[threadIdx.x] = st; s_i[threadIdx.x] = si;
   __syncthreads();
   for (int o = 1; o < 1024; o <<= 1) {
-    int ve = 0, vt = 0;
-    if ((int)threadIdx.x >= o) { ve = s_e[threadIdx.x - o]; vt = s_t[threadIdx.x - o]; }
+    int ve = 0, vt = 0, vi = 0;
+    if ((int)threadIdx.x >= o) { ve = s_e[threadIdx.x - o]; vt = s_t[threadIdx.x - o]; vi = s_i[threadIdx.x - o]; }
     __syncthreads();
-    s_e[threadIdx.x] += ve; s_t[threadIdx.x] += vt;
+    s_e[threadIdx.x] += ve; s_t[threadIdx.x] += vt; s_i[threadIdx.x] += vi;
     __syncthreads();
   }
-  int be = s_e[threadIdx.x] - se, bt = s_t[threadIdx.x] - st;
+  int be = s_e[threadIdx.x] - se, bt = s_t[threadIdx.x] - st, bi = s_i[threadIdx.x] - si;
   for (int i = lo; i < hi; ++i) {
     const int c = a.count[i];
-    a.entry_off[i] = be; a.tile_off[i] = bt; a.cursor[i] = be;
-    be += c;
-    bt += (c + a.tpt - 1) / a.tpt;
+    const int tl = (c + a.tpt - 1) / a.tpt;
+    a.entry_off[i] = be; a.tile_off[i] = bt; a.item_off[i] = bi; a.cursor[i] = be;
+    const int ni = (tl + kItemTiles - 1) / kItemTiles;
+    for (int x = 0; x < ni; ++x) a.item_key[bi + x] = i;
+    be += c; bt += tl; bi += ni;
   }
-  if (threadIdx.x == 1023) { a.entry_off[nkeys] = s_e[1023]; a.tile_off[nkeys] = s_t[1023]; }
+  if (threadIdx.x == 1023) {
+    a.entry_off[nkeys] = s_e[1023]; a.tile_off[nkeys] = s_t[1023]; a.item_off[nkeys] = s_i[1023];
+  }
 }
 
 __global__ void __launch_bounds__(256) inv_fill_kernel(InvArgs a, int use_smem) {
@@ -161,6 +168,8 @@ struct TileArgs {
   const __nv_bfloat16* v;
   const int32_t* entry_off;
   const int32_t* tile_off;
+  const int32_t* item_off;
+  const int32_t* item_key;
   const int32_t* entries;
   int nkeys, Mk, NW, fan, slots;
   float* blk_lse;          // [BH, N, slots*fan, G]   (tile_lse)
@@ -181,46 +190,6 @@ __device__ __forceinline__ int find_key(const int32_t* tile_off, int nkeys, int 
     if (tile_off[mid] <= tile) lo = mid; else hi = mid;
   }
   return lo;
-}
-
-// Thread `tid` of 128 always moves 16-byte chunk (tid % (D/8)) of rows (tid / (D/8)) + i * (1024/D):
-// the row index modulo 8 -- hence the swizzle -- is the same for every i, so the destination advances
-// by a constant and the loop body is one address computation and one copy.
-//
-// rows [row0, row0 + nrows) of a [tokens][D] bf16 matrix -> 128B-swizzled K-major slabs
-// (slab s holds elements [64 s, 64 s + 64) of every row); rows at or past `limit` become zeros
-template <int D>
-__device__ __forceinline__ void load_rows_swizzled(uint8_t* dst, int slab_bytes, const __nv_bfloat16* base,
-                                                   long long row_stride, int row0, int nrows, int limit, int tid) {
-  constexpr int CH = D / 8, RPP = 128 / CH;
-  const int ck = tid % CH, rb = tid / CH;
-  uint32_t d = smem_u32(dst + (ck >> 3) * slab_bytes) + swz128(rb, ck & 7);
-  const __nv_bfloat16* src = base + (long long)(row0 + rb) * row_stride + ck * 8;
-  for (int row = rb; row < nrows; row += RPP) {
-    if (row0 + row < limit) cp_async16(d, src);
-    else st_shared_zero16(d);
-    d += RPP * 128;
-    src += (long long)RPP * row_stride;
-  }
-}
-
-// gathered query rows: row r = (entry r >> lgG, head r & (G-1))
-template <int D>
-__device__ __forceinline__ void gather_q_swizzled(uint8_t* dst, const Geometry& geo, const __nv_bfloat16* q,
-                                                  int b, int h, const int* s_ent, int tid) {
-  constexpr int CH = D / 8, RPP = 128 / CH;
-  const int ck = tid % CH, rb = tid / CH;
-  const int G = geo.G, lgG = 31 - __clz(G);
-  uint32_t d = smem_u32(dst + (ck >> 3) * (128 * 128)) + swz128(rb, ck & 7);
-  const __nv_bfloat16* qb = q + (long long)b * geo.qs[0] + (long long)(h * G) * geo.qs[2] + ck * 8;
-  const long long s1 = geo.qs[1], s2 = geo.qs[2];
-#pragma unroll 4
-  for (int row = rb; row < 128; row += RPP) {
-    const int ent = s_ent[row >> lgG];
-    if (ent >= 0) cp_async16(d, qb + (long long)(ent & 0xFFFFFF) * s1 + (long long)(row & (G - 1)) * s2);
-    else st_shared_zero16(d);
-    d += RPP * 128;
-  }
 }
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -271,293 +240,536 @@ __device__ __forceinline__ void lse_chunk_masked(const uint32_t (&rr)[32], int n
   m = mn;
 }
 
-// Per-head log-sum-exp of the scaled logits of every (gathered query row, child leaf) pair of a
-// key group: the B operand is NB = fan*C consecutive keys, so one UMMA chain of D/16 steps gives a
-// 128 x NB logit tile in TMEM; each thread then owns one row and reduces C columns per child.
+// ------------------------------------------------------------------ warp-specialised tile kernels
+//
+// One CTA per SM, thirteen warps: warps 0-3 stage operands (16-byte cp.async into the swizzled
+// layouts, a ring of NS query tiles; the block's keys/values ride with the first tile of a work item),
+// warp 4 issues the UMMA chains, warps 5-8 and 9-12 are two epilogue groups that take alternate tiles, each
+// on its own TMEM accumulator, so that the exponentials of one tile overlap the gathers and the MMAs
+// of the next.  Every role walks the same deterministic sequence of (work item, tile) and derives
+// ring slots and mbarrier parities from its own tile counter; all waits are time-bounded.
+
+constexpr int kWsThreads = 416;        // 4 producer warps, 1 MMA warp, 2 x 4 epilogue warps
+constexpr int kProdThreads = 128;
+
+struct ItemInfo {
+  int key, ntiles, e_begin, e_end;
+};
+__device__ __forceinline__ ItemInfo item_info(const TileArgs& a, int item, int tpt) {
+  ItemInfo r;
+  r.key = a.item_key[item];
+  const int local = item - a.item_off[r.key];
+  const int list0 = a.entry_off[r.key], cnt = a.entry_off[r.key + 1] - list0;
+  const int tiles = (cnt + tpt - 1) / tpt;
+  const int first = local * kItemTiles;
+  r.ntiles = min(kItemTiles, tiles - first);
+  r.e_begin = list0 + first * tpt;
+  r.e_end = list0 + cnt;
+  return r;
+}
+
+// The 128 producer threads copy rows [row0, row0+nrows) of a [tokens][D] matrix into swizzled K-major
+// slabs.  Thread p always moves 16-byte chunk (p % (D/8)) of rows (p / (D/8)) + i * (1024/D): the row
+// index modulo 8 -- hence the swizzle -- is the same for every i, so the destination just advances.
+template <int D>
+__device__ __forceinline__ void prod_load_rows(uint8_t* dst, int slab_bytes, const __nv_bfloat16* base,
+                                               long long row_stride, int row0, int nrows, int limit, int p) {
+  constexpr int CH = D / 8, RPP = kProdThreads / CH;
+  const int ck = p % CH, rb = p / CH;
+  uint32_t d = smem_u32(dst + (ck >> 3) * slab_bytes) + swz128(rb, ck & 7);
+  const __nv_bfloat16* src = base + (long long)(row0 + rb) * row_stride + ck * 8;
+  for (int row = rb; row < nrows; row += RPP) {
+    if (row0 + row < limit) cp_async16(d, src);
+    else st_shared_zero16(d);
+    d += RPP * 128;
+    src += (long long)RPP * row_stride;
+  }
+}
+// ... and gather the 128 query rows of a tile: row r = (entry r >> lgG, head r & (G-1)); the tile's
+// entries sit in shared memory (-1 = no entry)
+template <int D>
+__device__ __forceinline__ void prod_gather_q(uint8_t* dst, const Geometry& geo, const __nv_bfloat16* qb,
+                                              const int* s_ent, int p) {
+  constexpr int CH = D / 8, RPP = kProdThreads / CH;
+  const int ck = p % CH, rb = p / CH;
+  const int G = geo.G, lgG = 31 - __clz(G);
+  uint32_t d = smem_u32(dst + (ck >> 3) * (128 * 128)) + swz128(rb, ck & 7);
+  const __nv_bfloat16* src0 = qb + ck * 8;
+  const long long s1 = geo.qs[1], s2 = geo.qs[2];
+#pragma unroll 4
+  for (int row = rb; row < 128; row += RPP) {
+    const int ent = s_ent[row >> lgG];
+    if (ent >= 0) cp_async16(d, src0 + (long long)(ent & 0xFFFFFF) * s1 + (long long)(row & (G - 1)) * s2);
+    else st_shared_zero16(d);
+    d += RPP * 128;
+  }
+}
+// barrier among the 128 producer threads that also ORs a flag, so that they leave their loops together
+__device__ __forceinline__ bool prod_sync_or(bool flag) {
+  uint32_t any;
+  asm volatile(
+      "{\n"
+      ".reg .pred p, q;\n"
+      "setp.ne.b32 q, %1, 0;\n"
+      "bar.red.or.pred p, 1, 128, q;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(any)
+      : "r"(flag ? 1u : 0u)
+      : "memory");
+  return any != 0;
+}
+
 template <int D, int NB>
-__global__ void __launch_bounds__(128) tile_lse_kernel(Geometry geo, TileArgs a) {
+__global__ void __launch_bounds__(kWsThreads, 1) lse_ws_kernel(Geometry geo, TileArgs a) {
   extern __shared__ uint8_t smem_raw[];
+  constexpr int NS = 3;
   constexpr int KS = D / 64;
   constexpr int A_SLAB = 128 * 128, B_SLAB = NB * 128;
-  constexpr uint32_t TM_COLS = NB < 32 ? 32 : NB;
+  constexpr int A_STAGE = KS * A_SLAB;
+  constexpr uint32_t TM_COLS = (2 * NB < 32) ? 32 : 2 * NB;
   uint8_t* smem = align1024(smem_raw);
   uint8_t* sA = smem;
-  uint8_t* sB = smem + KS * A_SLAB;
-  __shared__ uint64_t bar;
+  uint8_t* sB = smem + NS * A_STAGE;
+  __shared__ uint64_t a_full[NS], a_empty[NS], b_empty, t_full[2], t_empty[2];
   __shared__ uint32_t tmem_slot;
-  __shared__ int s_ent[128];
+  __shared__ volatile int s_fail;
+  __shared__ int s_ent[2][128];          // the producers' copy of the current / next tile's entries
 
-  const int tid = threadIdx.x, warp = tid >> 5;
-  if (tid == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    for (int i = 0; i < NS; ++i) { mbar_init(&a_full[i], kProdThreads); mbar_init(&a_empty[i], 1); }
+    mbar_init(&b_empty, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 128); }
+    s_fail = 0;
+    mbar_fence_init();
+  }
   if (warp == 0) { tmem_alloc(&tmem_slot, TM_COLS); tmem_relinquish(); }
   tcgen05_fence_before_sync();
   __syncthreads();
   tcgen05_fence_after_sync();
   const uint32_t tmem = tmem_slot;
 
-  const int G = geo.G, tpt = 128 / G, C = geo.C;
-  const int T = a.tile_off[a.nkeys];
+  const int G = geo.G, lgG = 31 - __clz(G), tpt = 128 >> lgG, C = geo.C;
+  const int n_items = a.item_off[a.nkeys];
   const float sl2 = geo.scale * kLog2e;
-  const uint32_t idesc = make_idesc_bf16(128, NB, 0, 0);
-  const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-  uint32_t phase = 0;
-  int loaded_key = -1;
-  bool failed = false;
 
-  for (int run = blockIdx.x; run * kRunTiles < T && !failed; run += gridDim.x) {
-    const int tile0 = run * kRunTiles, tile1 = min(T, tile0 + kRunTiles);
-    int key = find_key(a.tile_off, a.nkeys, tile0);
-    for (int tile = tile0; tile < tile1; ++tile) {
-      while (tile >= a.tile_off[key + 1]) ++key;
-      const int bh = key / (a.NW * a.Mk), j = key % a.Mk;
+  if (warp < 4) {
+    // ------------------------------------------------ producers
+    int it = 0, signalled = 0, kiter = 0;
+    bool stop = false;
+    for (int item = blockIdx.x; item < n_items && !stop; item += gridDim.x, ++kiter) {
+      const ItemInfo inf = item_info(a, item, tpt);
+      const int bh = inf.key / (a.NW * a.Mk), j = inf.key % a.Mk;
       const int b = bh / geo.Hkv, h = bh % geo.Hkv;
-      const int e0 = a.entry_off[key] + (tile - a.tile_off[key]) * tpt;
-      const int n_e = min(tpt, a.entry_off[key + 1] - e0);
-      if (tid < tpt) s_ent[tid] = (tid < n_e) ? a.entries[e0 + tid] : -1;
-      __syncthreads();      // entries visible; the previous tile's TMEM reads and smem reads are done
-      if (key != loaded_key) {
-        load_rows_swizzled<D>(sB, B_SLAB, a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2], geo.ks[1],
-                              j * NB, NB, geo.N, tid);
-        loaded_key = key;
-      }
-      gather_q_swizzled<D>(sA, geo, a.q, b, h, s_ent, tid);
-      const int ent = s_ent[tid >> (31 - __clz(G))];     // read before the barrier: the next iteration rewrites s_ent
+      // hand over everything issued so far, then wait until the previous item's MMAs released B
       cp_async_wait_all();
       fence_proxy_async_smem();
-      __syncthreads();
-      if (tid == 0) {
-        tcgen05_fence_after_sync();
+      for (; signalled < it; ++signalled) mbar_arrive(&a_full[signalled % NS]);
+      bool bad = s_fail != 0;
+      if (!bad && kiter > 0) bad = !mbar_wait_bounded(&b_empty, (uint32_t)((kiter - 1) & 1));
+      if (prod_sync_or(bad)) { s_fail = 1; stop = true; break; }
+      prod_load_rows<D>(sB, B_SLAB, a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2], geo.ks[1], j * NB,
+                        NB, geo.N, tid);
+      const __nv_bfloat16* qb = a.q + (long long)b * geo.qs[0] + (long long)(h * G) * geo.qs[2];
+      for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
+        const int s = it % NS;
+        bool bad_t = false;
+        if (it >= NS) {
+          // ring slot still busy: first hand over every tile already issued (their arrival is what
+          // lets the consumers make the progress that frees the slot), then wait for it
+          const uint32_t par = (uint32_t)((it / NS - 1) & 1);
+          if (prod_sync_or(!mbar_test(&a_empty[s], par))) {
+            cp_async_wait_all();
+            fence_proxy_async_smem();
+            for (; signalled < it; ++signalled) mbar_arrive(&a_full[signalled % NS]);
+            bad_t = !mbar_wait_bounded(&a_empty[s], par);
+          }
+        }
+        const int e0 = inf.e_begin + jt * tpt;
+        s_ent[it & 1][tid] = (tid < tpt && e0 + tid < inf.e_end) ? a.entries[e0 + tid] : -1;
+        if (prod_sync_or(bad_t)) { s_fail = 1; stop = true; break; }
+        prod_gather_q<D>(sA + s * A_STAGE, geo, qb, s_ent[it & 1], tid);
+        cp_async_commit();
+        if (it + 1 - signalled >= NS) {          // the oldest outstanding tile has landed
+          cp_async_wait_group<NS - 1>();
+          fence_proxy_async_smem();
+          mbar_arrive(&a_full[signalled % NS]);
+          ++signalled;
+        }
+      }
+    }
+    cp_async_wait_all();
+    fence_proxy_async_smem();
+    for (; signalled < it; ++signalled) mbar_arrive(&a_full[signalled % NS]);
+  } else if (warp == 4) {
+    // ------------------------------------------------ MMA issuer (the warp walks the loop, lane 0 issues)
+    const uint32_t idesc = make_idesc_bf16(128, NB, 0, 0);
+    int it = 0;
+    for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x) {
+      const ItemInfo inf = item_info(a, item, tpt);
+      bool ok = true;
+      for (int jt = 0; jt < inf.ntiles && ok; ++jt, ++it) {
+        const int s = it % NS, buf = it & 1;
+        ok = mbar_wait_bounded(&a_full[s], (uint32_t)((it / NS) & 1));
+        if (ok && it >= 2) ok = mbar_wait_bounded(&t_empty[buf], (uint32_t)(((it >> 1) - 1) & 1));
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (lane == 0) {
+          tcgen05_fence_after_sync();
+          const uint32_t a0 = smem_u32(sA + s * A_STAGE), b0 = smem_u32(sB);
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint64_t da = make_smem_desc(smem_u32(sA) + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
-          const uint64_t db = make_smem_desc(smem_u32(sB) + (kk >> 2) * B_SLAB + (kk & 3) * 32, 0, 1024);
-          umma_bf16(tmem, da, db, idesc, kk > 0);
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint64_t da = make_smem_desc(a0 + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
+            const uint64_t db = make_smem_desc(b0 + (kk >> 2) * B_SLAB + (kk & 3) * 32, 0, 1024);
+            umma_bf16(tmem + (uint32_t)(buf * NB), da, db, idesc, kk > 0);
+          }
+          umma_commit(&a_empty[s]);
+          umma_commit(&t_full[buf]);
         }
-        umma_commit(&bar);
+        __syncwarp();
       }
-      const bool ok = mbar_wait_bounded(&bar, phase);
-      phase ^= 1u;
-      if (__syncthreads_or(!ok)) { failed = true; break; }
-      tcgen05_fence_after_sync();
-
-      const int head = tid & (G - 1);
-      const bool valid = ent >= 0;
-      const int t = ent & 0xFFFFFF, slot = valid ? (ent >> 24) : 0;
-      const int c_t = t / C;
-      for (int r = 0; r < a.fan; ++r) {
-        const int leaf = j * a.fan + r;
-        int ncols = 0;
-        if (valid && leaf <= c_t && leaf < geo.M[1])
-          ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
-        // whole-warp fast path: every row either takes all C columns or does not need a result
-        const bool fast = __all_sync(0xffffffffu, ncols == C || ncols == 0);
-        float m = -CUDART_INF_F, ssum = 0.f;
-        uint32_t ra[32], rb[32];
-        const uint32_t col0 = lane_base + (uint32_t)(r * C);
-        tmem_ld_32x32(col0, ra);
-        for (int c0 = 0; c0 < C; c0 += 64) {
-          tmem_ld_wait();
-          tmem_ld_32x32(col0 + (uint32_t)(c0 + 32), rb);
-          if (fast) lse_chunk(ra, sl2, m, ssum);
-          else if (c0 < ncols) lse_chunk_masked(ra, ncols - c0, sl2, m, ssum);
-          tmem_ld_wait();
-          if (c0 + 64 < C) tmem_ld_32x32(col0 + (uint32_t)(c0 + 64), ra);
-          if (fast) lse_chunk(rb, sl2, m, ssum);
-          else if (c0 + 32 < ncols) lse_chunk_masked(rb, ncols - c0 - 32, sl2, m, ssum);
+      if (!ok) { s_fail = 1; break; }
+      if (lane == 0) umma_commit(&b_empty);
+      __syncwarp();
+    }
+  } else {
+    // ------------------------------------------------ epilogue groups
+    const int grp = (warp - 5) >> 2;                    // 0: even tiles, 1: odd tiles
+    const int row = (warp & 3) * 32 + lane;             // TMEM lane quarter of this warp = warp % 4
+    const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(grp * NB);
+    const int head = row & (G - 1);
+    int it = 0;
+    for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x) {
+      const ItemInfo inf = item_info(a, item, tpt);
+      const int bh = inf.key / (a.NW * a.Mk), j = inf.key % a.Mk;
+      for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
+        if ((it & 1) != grp) continue;
+        const int e0 = inf.e_begin + jt * tpt;
+        const int e = row >> lgG;
+        const int ent = (e0 + e < inf.e_end && e < tpt) ? a.entries[e0 + e] : -1;
+        if (!mbar_wait_bounded(&t_full[grp], (uint32_t)((it >> 1) & 1))) { s_fail = 1; break; }
+        tcgen05_fence_after_sync();
+        const bool valid = ent >= 0;
+        const int t = ent & 0xFFFFFF, slot = valid ? (ent >> 24) : 0;
+        const int c_t = t / C;
+        for (int r = 0; r < a.fan; ++r) {
+          const int leaf = j * a.fan + r;
+          int ncols = 0;
+          if (valid && leaf <= c_t && leaf < geo.M[1])
+            ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
+          const bool fast = __all_sync(0xffffffffu, ncols == C || ncols == 0);
+          float m = -CUDART_INF_F, ssum = 0.f;
+          uint32_t ra[32], rb[32];
+          const uint32_t col0 = lane_base + (uint32_t)(r * C);
+          tmem_ld_32x32(col0, ra);
+          for (int c0 = 0; c0 < C; c0 += 64) {
+            tmem_ld_wait();
+            tmem_ld_32x32(col0 + (uint32_t)(c0 + 32), rb);
+            if (fast) lse_chunk(ra, sl2, m, ssum);
+            else if (c0 < ncols) lse_chunk_masked(ra, ncols - c0, sl2, m, ssum);
+            tmem_ld_wait();
+            if (c0 + 64 < C) tmem_ld_32x32(col0 + (uint32_t)(c0 + 64), ra);
+            if (fast) lse_chunk(rb, sl2, m, ssum);
+            else if (c0 + 32 < ncols) lse_chunk_masked(rb, ncols - c0 - 32, sl2, m, ssum);
+          }
+          if (valid) {
+            const float lse = (ncols > 0) ? (m + log2f(ssum)) * kLn2 : -CUDART_INF_F;
+            a.blk_lse[(((long long)bh * geo.N + t) * (a.slots * a.fan) + slot * a.fan + r) * G + head] = lse;
+          }
         }
-        if (valid) {
-          const float lse = (ncols > 0) ? (m + log2f(ssum)) * kLn2 : -CUDART_INF_F;
-          a.blk_lse[(((long long)bh * geo.N + t) * (a.slots * a.fan) + slot * a.fan + r) * G + head] = lse;
-        }
+        tcgen05_fence_before_sync();
+        mbar_arrive(&t_empty[grp]);
       }
-      tcgen05_fence_before_sync();
     }
   }
-  if (failed && tid == 0) atomicExch(a.status, (int)PISA_ERR_TIMEOUT);
   tcgen05_fence_before_sync();
   __syncthreads();
+  if (s_fail && tid == 0) atomicExch(a.status, (int)PISA_ERR_TIMEOUT);
   if (warp == 0) tmem_dealloc(tmem, TM_COLS);
 }
 
-// One (leaf block, tile of gathered query rows): S = Q K^T in TMEM, P = exp(S*scale - lse_row)
-// written back to shared memory as the bf16 A operand of O_partial = P V, and the fp32 partial
-// rows added into the accumulator by bulk reductions.  lse_row is the row's final softmax
-// denominator, so partials from different blocks simply add up.
+// Attention tiles, same role layout.  Per tile: S = Q K^T (UMMA) -> an epilogue group turns S into
+// P = 2^(S*scale*log2e - lse2) in bf16, overwriting the query tile's ring slot -> O_partial = P V
+// (UMMA, V as the MN-major operand) -> the same group moves O through its ring slot (now free) into
+// the fp32 accumulator with bulk reductions, then releases the slot and the TMEM buffers.
 template <int D, int C>
-__global__ void __launch_bounds__(128) tile_pv_kernel(Geometry geo, TileArgs a) {
+__global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, TileArgs a) {
   extern __shared__ uint8_t smem_raw[];
-  constexpr int KS = D / 64;                 // 64-wide slabs of d
+  constexpr int NS = 3;
+  constexpr int KS = D / 64;
   constexpr int A_SLAB = 128 * 128, KV_SLAB = C * 128;
   constexpr int STAGE_ROW = 256 + 16;        // 64 fp32 + pad: conflict-free 16-byte row writes
   constexpr int QP_BYTES = (KS * A_SLAB > 128 * STAGE_ROW) ? KS * A_SLAB : 128 * STAGE_ROW;
-  constexpr int QP_ALIGNED = (QP_BYTES + 1023) / 1024 * 1024;
-  constexpr uint32_t TM_COLS = 256;          // S at column 0 (C columns), O at column 128 (D columns)
+  constexpr int Q_STAGE = (QP_BYTES + 1023) / 1024 * 1024;
+  constexpr uint32_t TM_COLS = 512;          // S buffers at columns 0 / 128, O buffers at 256 / 384
   uint8_t* smem = align1024(smem_raw);
-  uint8_t* sQ = smem;                        // Q tile, then P tile, then the O staging rows
-  uint8_t* sK = smem + QP_ALIGNED;
+  uint8_t* sQ = smem;
+  uint8_t* sK = smem + NS * Q_STAGE;
   uint8_t* sV = sK + KS * KV_SLAB;
-  __shared__ uint64_t bar;
+  __shared__ uint64_t q_full[NS], q_empty[NS], kv_empty, s_full[2], p_ready[2], o_full[2], t_empty[2];
   __shared__ uint32_t tmem_slot;
-  __shared__ int s_ent[128];
+  __shared__ volatile int s_fail;
+  __shared__ int s_ent[2][128];          // the producers' copy of the current / next tile's entries
 
-  const int tid = threadIdx.x, warp = tid >> 5;
-  if (tid == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    for (int i = 0; i < NS; ++i) { mbar_init(&q_full[i], kProdThreads); mbar_init(&q_empty[i], 128); }
+    mbar_init(&kv_empty, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&s_full[i], 1); mbar_init(&p_ready[i], 128); mbar_init(&o_full[i], 1); mbar_init(&t_empty[i], 128);
+    }
+    s_fail = 0;
+    mbar_fence_init();
+  }
   if (warp == 0) { tmem_alloc(&tmem_slot, TM_COLS); tmem_relinquish(); }
   tcgen05_fence_before_sync();
   __syncthreads();
   tcgen05_fence_after_sync();
   const uint32_t tmem = tmem_slot;
-  const uint32_t tmem_s = tmem, tmem_o = tmem + 128;
 
-  const int G = geo.G, tpt = 128 / G;
-  const int T = a.tile_off[a.nkeys];
+  const int G = geo.G, lgG = 31 - __clz(G), tpt = 128 >> lgG;
+  const int n_items = a.item_off[a.nkeys];
   const float sl2 = geo.scale * kLog2e;
-  const uint32_t idesc_s = make_idesc_bf16(128, C, 0, 0);
-  const uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
-  const uint32_t s_base = tmem_s + ((uint32_t)(warp * 32) << 16);
-  const uint32_t o_base = tmem_o + ((uint32_t)(warp * 32) << 16);
-  uint8_t* stage = sQ + tid * STAGE_ROW;
-  uint32_t phase = 0;
-  int loaded_key = -1;
-  bool failed = false;
 
-  for (int run = blockIdx.x; run * kRunTiles < T && !failed; run += gridDim.x) {
-    const int tile0 = run * kRunTiles, tile1 = min(T, tile0 + kRunTiles);
-    int key = find_key(a.tile_off, a.nkeys, tile0);
-    for (int tile = tile0; tile < tile1; ++tile) {
-      while (tile >= a.tile_off[key + 1]) ++key;
-      const int bh = key / (a.NW * a.Mk), leaf = key % a.Mk;
+  if (warp < 4) {
+    // ------------------------------------------------ producers
+    int it = 0, signalled = 0, kiter = 0;
+    bool stop = false;
+    for (int item = blockIdx.x; item < n_items && !stop; item += gridDim.x, ++kiter) {
+      const ItemInfo inf = item_info(a, item, tpt);
+      const int bh = inf.key / (a.NW * a.Mk), leaf = inf.key % a.Mk;
       const int b = bh / geo.Hkv, h = bh % geo.Hkv;
-      const int e0 = a.entry_off[key] + (tile - a.tile_off[key]) * tpt;
-      const int n_e = min(tpt, a.entry_off[key + 1] - e0);
-      if (tid < tpt) s_ent[tid] = (tid < n_e) ? a.entries[e0 + tid] : -1;
-      bulk_wait_read_all();    // this thread's staging rows of the previous tile have been read
-      __syncthreads();
-      if (key != loaded_key) {
-        load_rows_swizzled<D>(sK, KV_SLAB, a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2], geo.ks[1],
-                              leaf * C, C, geo.N, tid);
-        load_rows_swizzled<D>(sV, KV_SLAB, a.v + (long long)b * geo.vs[0] + (long long)h * geo.vs[2], geo.vs[1],
-                              leaf * C, C, geo.N, tid);
-        loaded_key = key;
-      }
-      gather_q_swizzled<D>(sQ, geo, a.q, b, h, s_ent, tid);
-
-      const int ent = s_ent[tid >> (31 - __clz(G))];
-      const int head = tid & (G - 1);
-      const bool valid = ent >= 0;
-      const int t = ent & 0xFFFFFF;
-      const int hq = h * G + head;
-      float neg_lse2 = 0.f;              // minus the row denominator, in log2 units
-      int ncols = 0;
-      if (valid) {
-        const float l2 = a.row_lse[((long long)b * geo.Hq + hq) * geo.N + t] * kLog2e;
-        const int c_t = t / C;
-        if (leaf <= c_t && l2 > -CUDART_INF_F) ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
-        neg_lse2 = -l2;
-      }
       cp_async_wait_all();
       fence_proxy_async_smem();
-      __syncthreads();
-      if (tid == 0) {
-        tcgen05_fence_after_sync();
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint64_t da = make_smem_desc(smem_u32(sQ) + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
-          const uint64_t db = make_smem_desc(smem_u32(sK) + (kk >> 2) * KV_SLAB + (kk & 3) * 32, 0, 1024);
-          umma_bf16(tmem_s, da, db, idesc_s, kk > 0);
-        }
-        umma_commit(&bar);
-      }
-      bool ok = mbar_wait_bounded(&bar, phase);
-      phase ^= 1u;
-      if (__syncthreads_or(!ok)) { failed = true; break; }
-      tcgen05_fence_after_sync();
-
-      // P = 2^(S*scale*log2e - lse2), masked, as the bf16 K-major A operand (overwrites the Q tile:
-      // the S chain that read it has completed)
-      {
-        const bool fast = __all_sync(0xffffffffu, ncols == C);
-        uint32_t ra[32], rb[32];
-        tmem_ld_32x32(s_base, ra);
-#pragma unroll
-        for (int c0 = 0; c0 < C; c0 += 32) {
-          uint32_t (&cur)[32] = ((c0 >> 5) & 1) ? rb : ra;
-          uint32_t (&nxt)[32] = ((c0 >> 5) & 1) ? ra : rb;
-          tmem_ld_wait();
-          if (c0 + 32 < C) tmem_ld_32x32(s_base + (uint32_t)(c0 + 32), nxt);
-          uint32_t pk[16];
-#pragma unroll
-          for (int jx = 0; jx < 16; ++jx) {
-            float p0 = ex2_approx(fmaf(__uint_as_float(cur[2 * jx]), sl2, neg_lse2));
-            float p1 = ex2_approx(fmaf(__uint_as_float(cur[2 * jx + 1]), sl2, neg_lse2));
-            if (!fast) {
-              if (c0 + 2 * jx >= ncols) p0 = 0.f;
-              if (c0 + 2 * jx + 1 >= ncols) p1 = 0.f;
-            }
-            const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
-            pk[jx] = *reinterpret_cast<const uint32_t*>(&pp);
-          }
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            const int ck = c0 / 8 + q4;                       // 16-byte chunk (8 keys) of this row
-            const uint32_t d = smem_u32(sQ + (ck >> 3) * A_SLAB) + swz128(tid, ck & 7);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d), "r"(pk[4 * q4]),
-                         "r"(pk[4 * q4 + 1]), "r"(pk[4 * q4 + 2]), "r"(pk[4 * q4 + 3])
-                         : "memory");
+      for (; signalled < it; ++signalled) mbar_arrive(&q_full[signalled % NS]);
+      bool bad = s_fail != 0;
+      if (!bad && kiter > 0) bad = !mbar_wait_bounded(&kv_empty, (uint32_t)((kiter - 1) & 1));
+      if (prod_sync_or(bad)) { s_fail = 1; stop = true; break; }
+      prod_load_rows<D>(sK, KV_SLAB, a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2], geo.ks[1], leaf * C,
+                        C, geo.N, tid);
+      prod_load_rows<D>(sV, KV_SLAB, a.v + (long long)b * geo.vs[0] + (long long)h * geo.vs[2], geo.vs[1], leaf * C,
+                        C, geo.N, tid);
+      const __nv_bfloat16* qb = a.q + (long long)b * geo.qs[0] + (long long)(h * G) * geo.qs[2];
+      for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
+        const int s = it % NS;
+        bool bad_t = false;
+        if (it >= NS) {
+          // ring slot still busy: first hand over every tile already issued (their arrival is what
+          // lets the consumers make the progress that frees the slot), then wait for it
+          const uint32_t par = (uint32_t)((it / NS - 1) & 1);
+          if (prod_sync_or(!mbar_test(&q_empty[s], par))) {
+            cp_async_wait_all();
+            fence_proxy_async_smem();
+            for (; signalled < it; ++signalled) mbar_arrive(&q_full[signalled % NS]);
+            bad_t = !mbar_wait_bounded(&q_empty[s], par);
           }
         }
-      }
-      fence_proxy_async_smem();
-      tcgen05_fence_before_sync();
-      __syncthreads();
-      if (tid == 0) {
-        tcgen05_fence_after_sync();
-#pragma unroll
-        for (int kk = 0; kk < C / 16; ++kk) {
-          const uint64_t da = make_smem_desc(smem_u32(sQ) + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
-          const uint64_t db = make_smem_desc(smem_u32(sV) + kk * (16 * 128), KV_SLAB, 1024);
-          umma_bf16(tmem_o, da, db, idesc_o, kk > 0);
-        }
-        umma_commit(&bar);
-      }
-      ok = mbar_wait_bounded(&bar, phase);
-      phase ^= 1u;
-      if (__syncthreads_or(!ok)) { failed = true; break; }
-      tcgen05_fence_after_sync();
-
-      // O partial: 64 columns at a time through this thread's private staging row, then one bulk
-      // reduction (256 bytes) into the fp32 accumulator row of (b, t, hq)
-      float* orow = a.o_acc + (((long long)b * geo.N + t) * geo.Hq + hq) * D;
-#pragma unroll
-      for (int half = 0; half < KS; ++half) {
-        uint32_t ra[32], rb[32];
-        tmem_ld_32x32(o_base + (uint32_t)(half * 64), ra);
-        tmem_ld_32x32(o_base + (uint32_t)(half * 64 + 32), rb);
-        if (half > 0) bulk_wait_read_all();
-        tmem_ld_wait();
-#pragma unroll
-        for (int q4 = 0; q4 < 8; ++q4)
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(stage) + q4 * 16), "r"(ra[4 * q4]),
-                       "r"(ra[4 * q4 + 1]), "r"(ra[4 * q4 + 2]), "r"(ra[4 * q4 + 3])
-                       : "memory");
-#pragma unroll
-        for (int q4 = 0; q4 < 8; ++q4)
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(stage) + 128 + q4 * 16),
-                       "r"(rb[4 * q4]), "r"(rb[4 * q4 + 1]), "r"(rb[4 * q4 + 2]), "r"(rb[4 * q4 + 3])
-                       : "memory");
-        fence_proxy_async_smem();
-        if (valid) {
-          bulk_reduce_add_f32(orow + half * 64, smem_u32(stage), 256);
-          bulk_commit();
+        const int e0 = inf.e_begin + jt * tpt;
+        s_ent[it & 1][tid] = (tid < tpt && e0 + tid < inf.e_end) ? a.entries[e0 + tid] : -1;
+        if (prod_sync_or(bad_t)) { s_fail = 1; stop = true; break; }
+        prod_gather_q<D>(sQ + s * Q_STAGE, geo, qb, s_ent[it & 1], tid);
+        cp_async_commit();
+        if (it + 1 - signalled >= NS) {
+          cp_async_wait_group<NS - 1>();
+          fence_proxy_async_smem();
+          mbar_arrive(&q_full[signalled % NS]);
+          ++signalled;
         }
       }
-      tcgen05_fence_before_sync();
     }
+    cp_async_wait_all();
+    fence_proxy_async_smem();
+    for (; signalled < it; ++signalled) mbar_arrive(&q_full[signalled % NS]);
+  } else if (warp == 4) {
+    // ------------------------------------------------ MMA issuer
+    // Event driven: S(it) goes out as soon as its query tile has landed and its TMEM buffers are
+    // free, P V(it) as soon as the epilogue group has written P(it); neither waits for the other, so
+    // a late query tile cannot hold back the P V that frees the ring slot the producer is waiting
+    // for.  Lane 0 probes and issues; the warp stays converged on its decisions.
+    const uint32_t idesc_s = make_idesc_bf16(128, C, 0, 0);
+    const uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
+    int s_it = 0, pv_it = 0;              // next tile whose S / whose P V is to be issued
+    unsigned last_bits = 0;               // bit (it & 31): tile `it` closes its work item
+    int item = blockIdx.x, jt = 0;
+    ItemInfo inf = {0, 0, 0, 0};
+    if (item < n_items) inf = item_info(a, item, tpt);
+    uint64_t t_idle = 0;
+    bool ok = true;
+    while (ok && !s_fail) {
+      const bool more_s = item < n_items;
+      if (!more_s && pv_it == s_it) break;
+      int do_s = 0, do_pv = 0;
+      if (lane == 0) {
+        if (more_s && s_it - pv_it < 2) {
+          const int s = s_it % NS, buf = s_it & 1;
+          do_s = mbar_test(&q_full[s], (uint32_t)((s_it / NS) & 1)) &&
+                 (s_it < 2 || mbar_test(&t_empty[buf], (uint32_t)(((s_it >> 1) - 1) & 1)));
+        }
+        if (pv_it < s_it) do_pv = mbar_test(&p_ready[pv_it & 1], (uint32_t)((pv_it >> 1) & 1));
+      }
+      do_s = __shfl_sync(0xffffffffu, do_s, 0);
+      do_pv = __shfl_sync(0xffffffffu, do_pv, 0);
+      if (do_pv) {
+        const int ps = pv_it % NS, pb = pv_it & 1;
+        if (lane == 0) {
+          tcgen05_fence_after_sync();
+          const uint32_t p0 = smem_u32(sQ + ps * Q_STAGE), v0 = smem_u32(sV);
+#pragma unroll
+          for (int kk = 0; kk < C / 16; ++kk) {
+            const uint64_t da = make_smem_desc(p0 + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
+            const uint64_t db = make_smem_desc(v0 + kk * (16 * 128), KV_SLAB, 1024);
+            umma_bf16(tmem + 256u + (uint32_t)(pb * 128), da, db, idesc_o, kk > 0);
+          }
+          umma_commit(&o_full[pb]);
+          if ((last_bits >> (pv_it & 31)) & 1u) umma_commit(&kv_empty);   // K/V of that item are free
+        }
+        ++pv_it;
+      }
+      if (do_s) {
+        const int s = s_it % NS, buf = s_it & 1;
+        if (lane == 0) {
+          tcgen05_fence_after_sync();
+          const uint32_t q0 = smem_u32(sQ + s * Q_STAGE), k0 = smem_u32(sK);
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint64_t da = make_smem_desc(q0 + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
+            const uint64_t db = make_smem_desc(k0 + (kk >> 2) * KV_SLAB + (kk & 3) * 32, 0, 1024);
+            umma_bf16(tmem + (uint32_t)(buf * 128), da, db, idesc_s, kk > 0);
+          }
+          umma_commit(&s_full[buf]);
+        }
+        const bool last = (jt == inf.ntiles - 1);
+        last_bits = (last_bits & ~(1u << (s_it & 31))) | ((last ? 1u : 0u) << (s_it & 31));
+        ++s_it;
+        if (last) {
+          item += gridDim.x;
+          jt = 0;
+          if (item < n_items) inf = item_info(a, item, tpt);
+        } else {
+          ++jt;
+        }
+      }
+      __syncwarp();
+      if (do_s || do_pv) {
+        t_idle = 0;
+      } else {
+        const uint64_t now = global_timer_ns();
+        if (t_idle == 0) t_idle = now;
+        else if (now - t_idle > 2000000000ull) ok = false;
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      }
+    }
+    if (!ok) s_fail = 1;
+  } else {
+    // ------------------------------------------------ epilogue groups
+    const int grp = (warp - 5) >> 2;
+    const int row = (warp & 3) * 32 + lane;
+    const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t s_base = tmem + lane_sel + (uint32_t)(grp * 128);
+    const uint32_t o_base = tmem + lane_sel + 256u + (uint32_t)(grp * 128);
+    const int head = row & (G - 1);
+    int it = 0;
+    for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x) {
+      const ItemInfo inf = item_info(a, item, tpt);
+      const int bh = inf.key / (a.NW * a.Mk), leaf = inf.key % a.Mk;
+      const int b = bh / geo.Hkv, h = bh % geo.Hkv;
+      const int hq = h * G + head;
+      for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
+        if ((it & 1) != grp) continue;
+        const int s = it % NS;
+        uint8_t* slot_base = sQ + s * Q_STAGE;
+        const int e0 = inf.e_begin + jt * tpt;
+        const int e = row >> lgG;
+        const int ent = (e0 + e < inf.e_end && e < tpt) ? a.entries[e0 + e] : -1;
+        const bool valid = ent >= 0;
+        const int t = ent & 0xFFFFFF;
+        float neg_lse2 = 0.f;
+        int ncols = 0;
+        if (valid) {
+          const float l2 = a.row_lse[((long long)b * geo.Hq + hq) * geo.N + t] * kLog2e;
+          const int c_t = t / C;
+          if (leaf <= c_t && l2 > -CUDART_INF_F)
+            ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
+          neg_lse2 = -l2;
+        }
+        const uint32_t par = (uint32_t)((it >> 1) & 1);
+        if (!mbar_wait_bounded(&s_full[grp], par)) { s_fail = 1; break; }
+        tcgen05_fence_after_sync();
+        {
+          const bool fast = __all_sync(0xffffffffu, ncols == C);
+          uint32_t ra[32], rb[32];
+          tmem_ld_32x32(s_base, ra);
+#pragma unroll
+          for (int c0 = 0; c0 < C; c0 += 32) {
+            uint32_t (&cur)[32] = ((c0 >> 5) & 1) ? rb : ra;
+            uint32_t (&nxt)[32] = ((c0 >> 5) & 1) ? ra : rb;
+            tmem_ld_wait();
+            if (c0 + 32 < C) tmem_ld_32x32(s_base + (uint32_t)(c0 + 32), nxt);
+            uint32_t pk[16];
+#pragma unroll
+            for (int jx = 0; jx < 16; ++jx) {
+              float p0 = ex2_approx(fmaf(__uint_as_float(cur[2 * jx]), sl2, neg_lse2));
+              float p1 = ex2_approx(fmaf(__uint_as_float(cur[2 * jx + 1]), sl2, neg_lse2));
+              if (!fast) {
+                if (c0 + 2 * jx >= ncols) p0 = 0.f;
+                if (c0 + 2 * jx + 1 >= ncols) p1 = 0.f;
+              }
+              const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
+              pk[jx] = *reinterpret_cast<const uint32_t*>(&pp);
+            }
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+              const int ck = c0 / 8 + q4;
+              const uint32_t d = smem_u32(slot_base + (ck >> 3) * A_SLAB) + swz128(row, ck & 7);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d), "r"(pk[4 * q4]),
+                           "r"(pk[4 * q4 + 1]), "r"(pk[4 * q4 + 2]), "r"(pk[4 * q4 + 3])
+                           : "memory");
+            }
+          }
+        }
+        fence_proxy_async_smem();
+        tcgen05_fence_before_sync();
+        mbar_arrive(&p_ready[grp]);
+        if (!mbar_wait_bounded(&o_full[grp], par)) { s_fail = 1; break; }
+        tcgen05_fence_after_sync();
+        // O partial through this thread's private row of the (now free) ring slot
+        uint8_t* stage = slot_base + row * STAGE_ROW;
+        float* orow = a.o_acc + (((long long)b * geo.N + t) * geo.Hq + hq) * D;
+#pragma unroll
+        for (int half = 0; half < KS; ++half) {
+          uint32_t ra[32], rb[32];
+          tmem_ld_32x32(o_base + (uint32_t)(half * 64), ra);
+          tmem_ld_32x32(o_base + (uint32_t)(half * 64 + 32), rb);
+          if (half > 0) bulk_wait_read_all();
+          tmem_ld_wait();
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(stage) + q4 * 16), "r"(ra[4 * q4]),
+                         "r"(ra[4 * q4 + 1]), "r"(ra[4 * q4 + 2]), "r"(ra[4 * q4 + 3])
+                         : "memory");
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(stage) + 128 + q4 * 16),
+                         "r"(rb[4 * q4]), "r"(rb[4 * q4 + 1]), "r"(rb[4 * q4 + 2]), "r"(rb[4 * q4 + 3])
+                         : "memory");
+          fence_proxy_async_smem();
+          if (valid) {
+            bulk_reduce_add_f32(orow + half * 64, smem_u32(stage), 256);
+            bulk_commit();
+          }
+        }
+        tcgen05_fence_before_sync();
+        mbar_arrive(&t_empty[grp]);        // S and O accumulators of this parity are free
+        bulk_wait_read_all();               // the ring slot has been read out
+        mbar_arrive(&q_empty[s]);
+      }
+    }
+    bulk_wait_all();
   }
-  if (failed && tid == 0) atomicExch(a.status, (int)PISA_ERR_TIMEOUT);
-  bulk_wait_all();
   tcgen05_fence_before_sync();
   __syncthreads();
+  if (s_fail && tid == 0) atomicExch(a.status, (int)PISA_ERR_TIMEOUT);
   if (warp == 0) tmem_dealloc(tmem, TM_COLS);
 }
 
@@ -707,7 +919,7 @@ __global__ void __launch_bounds__(256) convert_out_kernel(Geometry geo, const fl
 // ------------------------------------------------------------------ host side
 
 struct InvLayout {
-  size_t count, entry_off, tile_off, cursor, entries, end;
+  size_t count, entry_off, tile_off, item_off, item_key, cursor, entries, end;
 };
 
 int window_tokens(const Geometry& g) { return g.N < kWindowTok ? ((g.N + kInvTok - 1) / kInvTok) * kInvTok : kWindowTok; }
@@ -720,6 +932,10 @@ InvLayout inv_layout(size_t base, const Geometry& g, int Mk) {
   l.count = o; o += align_up(nkeys * 4, 256);
   l.entry_off = o; o += align_up((nkeys + 1) * 4, 256);
   l.tile_off = o; o += align_up((nkeys + 1) * 4, 256);
+  l.item_off = o; o += align_up((nkeys + 1) * 4, 256);
+  // every list adds at most one partial item on top of (all tiles) / kItemTiles
+  const size_t max_tiles = (size_t)g.B * g.Hkv * g.N * g.K / (128 / g.G) + nkeys;
+  l.item_key = o; o += align_up((max_tiles / kItemTiles + nkeys + 1) * 4, 256);
   l.cursor = o; o += align_up(nkeys * 4, 256);
   l.entries = o; o += align_up((size_t)g.B * g.Hkv * g.N * g.K * 4, 256);
   l.end = o;
@@ -765,7 +981,9 @@ int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char
   a.tpt = 128 / g.G;
   a.W = window_tokens(g); a.NW = num_windows(g);
   a.count = (int32_t*)(ws + l.count); a.entry_off = (int32_t*)(ws + l.entry_off);
-  a.tile_off = (int32_t*)(ws + l.tile_off); a.cursor = (int32_t*)(ws + l.cursor);
+  a.tile_off = (int32_t*)(ws + l.tile_off); a.item_off = (int32_t*)(ws + l.item_off);
+  a.item_key = (int32_t*)(ws + l.item_key);
+  a.cursor = (int32_t*)(ws + l.cursor);
   a.entries = (int32_t*)(ws + l.entries);
   const size_t nkeys = (size_t)a.BH * a.NW * Mk;
   cudaError_t e = cudaMemsetAsync(a.count, 0, nkeys * 4, s);
@@ -791,12 +1009,11 @@ int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char
 
 template <int D, int NB>
 int launch_tile_lse(const Geometry& g, const TileArgs& a, cudaStream_t s) {
-  const size_t smem = (size_t)(D / 64) * (128 * 128 + NB * 128) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(tile_lse_kernel<D, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) { record_cuda_error("tile_lse attr", e); return PISA_ERR_CUDA; }
-  const int ctas_per_sm = (smem <= 100 * 1024 && NB <= 256) ? 2 : 1;
-  tile_lse_kernel<D, NB><<<num_sms() * ctas_per_sm, 128, smem, s>>>(g, a);
-  return check_launch("tile_lse");
+  const size_t smem = (size_t)(D / 64) * (3 * 128 * 128 + NB * 128) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(lse_ws_kernel<D, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) { record_cuda_error("lse_ws attr", e); return PISA_ERR_CUDA; }
+  lse_ws_kernel<D, NB><<<num_sms(), kWsThreads, smem, s>>>(g, a);
+  return check_launch("lse_ws");
 }
 
 int dispatch_tile_lse(const Geometry& g, int nb, const TileArgs& a, cudaStream_t s) {
@@ -816,11 +1033,11 @@ template <int D, int C>
 int launch_tile_pv(const Geometry& g, const TileArgs& a, cudaStream_t s) {
   constexpr int KS = D / 64;
   constexpr int QP = (KS * 128 * 128 > 128 * 272) ? KS * 128 * 128 : 128 * 272;
-  const size_t smem = (size_t)((QP + 1023) / 1024 * 1024) + 2 * (size_t)KS * C * 128 + 1024;
-  cudaError_t e = cudaFuncSetAttribute(tile_pv_kernel<D, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) { record_cuda_error("tile_pv attr", e); return PISA_ERR_CUDA; }
-  tile_pv_kernel<D, C><<<num_sms() * 2, 128, smem, s>>>(g, a);
-  return check_launch("tile_pv");
+  const size_t smem = 3 * (size_t)((QP + 1023) / 1024 * 1024) + 2 * (size_t)KS * C * 128 + 1024;
+  cudaError_t e = cudaFuncSetAttribute(pv_ws_kernel<D, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) { record_cuda_error("pv_ws attr", e); return PISA_ERR_CUDA; }
+  pv_ws_kernel<D, C><<<num_sms(), kWsThreads, smem, s>>>(g, a);
+  return check_launch("pv_ws");
 }
 
 int dispatch_tile_pv(const Geometry& g, const TileArgs& a, cudaStream_t s) {
@@ -861,7 +1078,7 @@ int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, con
   if (st != PISA_OK) return st;
   TileArgs a = {};
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = nullptr;
-  a.entry_off = inv.entry_off; a.tile_off = inv.tile_off; a.entries = inv.entries;
+  a.entry_off = inv.entry_off; a.tile_off = inv.tile_off; a.item_off = inv.item_off; a.item_key = inv.item_key; a.entries = inv.entries;
   a.nkeys = g.B * g.Hkv * inv.NW * g.M[2]; a.Mk = g.M[2]; a.NW = inv.NW; a.fan = g.g; a.slots = g.K;
   a.blk_lse = blk; a.status = status;
   st = dispatch_tile_lse(g, g.g * g.C, a, s);
@@ -883,7 +1100,7 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
   if (st != PISA_OK) return st;
   TileArgs a = {};
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
-  a.entry_off = inv.entry_off; a.tile_off = inv.tile_off; a.entries = inv.entries;
+  a.entry_off = inv.entry_off; a.tile_off = inv.tile_off; a.item_off = inv.item_off; a.item_key = inv.item_key; a.entries = inv.entries;
   a.nkeys = g.B * g.Hkv * inv.NW * g.M[1]; a.Mk = g.M[1]; a.NW = inv.NW; a.fan = 1; a.slots = g.K;
   a.blk_lse = blk; a.row_lse = lse; a.o_acc = acc; a.status = status;
   if (!lse_ready) {
