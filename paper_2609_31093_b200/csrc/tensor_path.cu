@@ -250,11 +250,16 @@ __device__ __forceinline__ void lse_chunk_masked(const uint32_t (&rr)[32], int n
 // ring slots and mbarrier parities from its own tile counter; all waits are time-bounded.
 
 constexpr int kWsThreads = 416;        // 4 producer warps, 1 MMA warp, 2 x 4 epilogue warps
+constexpr int kLseThreads = 672;       // 4 producer warps, 1 MMA warp, 2 x 8 epilogue warps
 constexpr int kProdThreads = 128;
+constexpr int kMetaRing = 8;           // ring of per-tile metadata; deeper than any role can run ahead
 
 struct ItemInfo {
   int key, ntiles, e_begin, e_end;
 };
+__device__ __forceinline__ int fetch_entry(const int32_t* entries, int e0, int e_end, int tpt, int p) {
+  return (p < tpt && e0 + p < e_end) ? entries[e0 + p] : -1;
+}
 __device__ __forceinline__ ItemInfo item_info(const TileArgs& a, int item, int tpt) {
   ItemInfo r;
   r.key = a.item_key[item];
@@ -321,9 +326,9 @@ __device__ __forceinline__ bool prod_sync_or(bool flag) {
 }
 
 template <int D, int NB>
-__global__ void __launch_bounds__(kWsThreads, 1) lse_ws_kernel(Geometry geo, TileArgs a) {
+__global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, TileArgs a) {
   extern __shared__ uint8_t smem_raw[];
-  constexpr int NS = 3;
+  constexpr int NS = 4;
   constexpr int KS = D / 64;
   constexpr int A_SLAB = 128 * 128, B_SLAB = NB * 128;
   constexpr int A_STAGE = KS * A_SLAB;
@@ -334,13 +339,14 @@ __global__ void __launch_bounds__(kWsThreads, 1) lse_ws_kernel(Geometry geo, Til
   __shared__ uint64_t a_full[NS], a_empty[NS], b_empty, t_full[2], t_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_fail;
-  __shared__ int s_ent[2][128];          // the producers' copy of the current / next tile's entries
+  __shared__ int s_ent[kMetaRing][128];  // per-tile entries, written by the producers, read by all roles
+  __shared__ float s_lse[kMetaRing][128]; // per-row softmax denominators (attention kernel only)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) { mbar_init(&a_full[i], kProdThreads); mbar_init(&a_empty[i], 1); }
     mbar_init(&b_empty, 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 128); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 256); }
     s_fail = 0;
     mbar_fence_init();
   }
@@ -356,16 +362,13 @@ __global__ void __launch_bounds__(kWsThreads, 1) lse_ws_kernel(Geometry geo, Til
 
   if (warp < 4) {
     // ------------------------------------------------ producers
-    int it = 0, signalled = 0, kiter = 0;
+    int it = 0, kiter = 0, ent_next = -1;
     bool stop = false;
     for (int item = blockIdx.x; item < n_items && !stop; item += gridDim.x, ++kiter) {
       const ItemInfo inf = item_info(a, item, tpt);
       const int bh = inf.key / (a.NW * a.Mk), j = inf.key % a.Mk;
       const int b = bh / geo.Hkv, h = bh % geo.Hkv;
-      // hand over everything issued so far, then wait until the previous item's MMAs released B
-      cp_async_wait_all();
-      fence_proxy_async_smem();
-      for (; signalled < it; ++signalled) mbar_arrive(&a_full[signalled % NS]);
+      // the previous item's MMAs must have released the key tile
       bool bad = s_fail != 0;
       if (!bad && kiter > 0) bad = !mbar_wait_bounded(&b_empty, (uint32_t)((kiter - 1) & 1));
       if (prod_sync_or(bad)) { s_fail = 1; stop = true; break; }
@@ -374,34 +377,19 @@ __global__ void __launch_bounds__(kWsThreads, 1) lse_ws_kernel(Geometry geo, Til
       const __nv_bfloat16* qb = a.q + (long long)b * geo.qs[0] + (long long)(h * G) * geo.qs[2];
       for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
         const int s = it % NS;
-        bool bad_t = false;
-        if (it >= NS) {
-          // ring slot still busy: first hand over every tile already issued (their arrival is what
-          // lets the consumers make the progress that frees the slot), then wait for it
-          const uint32_t par = (uint32_t)((it / NS - 1) & 1);
-          if (prod_sync_or(!mbar_test(&a_empty[s], par))) {
-            cp_async_wait_all();
-            fence_proxy_async_smem();
-            for (; signalled < it; ++signalled) mbar_arrive(&a_full[signalled % NS]);
-            bad_t = !mbar_wait_bounded(&a_empty[s], par);
-          }
-        }
+        const bool bad_t = it >= NS && !mbar_wait_bounded(&a_empty[s], (uint32_t)((it / NS - 1) & 1));
         const int e0 = inf.e_begin + jt * tpt;
-        s_ent[it & 1][tid] = (tid < tpt && e0 + tid < inf.e_end) ? a.entries[e0 + tid] : -1;
+        // this tile's entries were fetched one tile ahead; fetch the next tile's now
+        const int ent_now = (jt == 0) ? fetch_entry(a.entries, e0, inf.e_end, tpt, tid) : ent_next;
+        ent_next = (jt + 1 < inf.ntiles) ? fetch_entry(a.entries, e0 + tpt, inf.e_end, tpt, tid) : -1;
+        s_ent[it % kMetaRing][tid] = ent_now;
         if (prod_sync_or(bad_t)) { s_fail = 1; stop = true; break; }
-        prod_gather_q<D>(sA + s * A_STAGE, geo, qb, s_ent[it & 1], tid);
-        cp_async_commit();
-        if (it + 1 - signalled >= NS) {          // the oldest outstanding tile has landed
-          cp_async_wait_group<NS - 1>();
-          fence_proxy_async_smem();
-          mbar_arrive(&a_full[signalled % NS]);
-          ++signalled;
-        }
+        prod_gather_q<D>(sA + s * A_STAGE, geo, qb, s_ent[it % kMetaRing], tid);
+        fence_proxy_async_smem();                 // zero-filled rows (plain stores) -> async proxy
+        cp_async_arrive_noinc(&a_full[s]);        // fires when this thread's copies have landed
       }
     }
     cp_async_wait_all();
-    fence_proxy_async_smem();
-    for (; signalled < it; ++signalled) mbar_arrive(&a_full[signalled % NS]);
   } else if (warp == 4) {
     // ------------------------------------------------ MMA issuer (the warp walks the loop, lane 0 issues)
     const uint32_t idesc = make_idesc_bf16(128, NB, 0, 0);
@@ -416,6 +404,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) lse_ws_kernel(Geometry geo, Til
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         if (lane == 0) {
+          fence_proxy_async_smem();
           tcgen05_fence_after_sync();
           const uint32_t a0 = smem_u32(sA + s * A_STAGE), b0 = smem_u32(sB);
 #pragma unroll
@@ -435,25 +424,28 @@ __global__ void __launch_bounds__(kWsThreads, 1) lse_ws_kernel(Geometry geo, Til
     }
   } else {
     // ------------------------------------------------ epilogue groups
-    const int grp = (warp - 5) >> 2;                    // 0: even tiles, 1: odd tiles
+    // eight warps per group: two warps share each TMEM lane quarter and split the tile's children
+    const int ew = warp - 5;
+    const int grp = ew >> 3;                            // 0: even tiles, 1: odd tiles
+    const int half = (ew >> 2) & 1;
     const int row = (warp & 3) * 32 + lane;             // TMEM lane quarter of this warp = warp % 4
     const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(grp * NB);
     const int head = row & (G - 1);
+    const int r_lo = (a.fan >= 2) ? half * (a.fan / 2) : 0;
+    const int r_hi = (a.fan >= 2) ? ((half == 1) ? a.fan : a.fan / 2) : (half == 0 ? 1 : 0);
     int it = 0;
     for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x) {
       const ItemInfo inf = item_info(a, item, tpt);
       const int bh = inf.key / (a.NW * a.Mk), j = inf.key % a.Mk;
       for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
         if ((it & 1) != grp) continue;
-        const int e0 = inf.e_begin + jt * tpt;
-        const int e = row >> lgG;
-        const int ent = (e0 + e < inf.e_end && e < tpt) ? a.entries[e0 + e] : -1;
         if (!mbar_wait_bounded(&t_full[grp], (uint32_t)((it >> 1) & 1))) { s_fail = 1; break; }
         tcgen05_fence_after_sync();
+        const int ent = s_ent[it % kMetaRing][row >> lgG];
         const bool valid = ent >= 0;
         const int t = ent & 0xFFFFFF, slot = valid ? (ent >> 24) : 0;
         const int c_t = t / C;
-        for (int r = 0; r < a.fan; ++r) {
+        for (int r = r_lo; r < r_hi; ++r) {
           const int leaf = j * a.fan + r;
           int ncols = 0;
           if (valid && leaf <= c_t && leaf < geo.M[1])
@@ -496,7 +488,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) lse_ws_kernel(Geometry geo, Til
 template <int D, int C>
 __global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, TileArgs a) {
   extern __shared__ uint8_t smem_raw[];
-  constexpr int NS = 3;
+  constexpr int NS = 4;
   constexpr int KS = D / 64;
   constexpr int A_SLAB = 128 * 128, KV_SLAB = C * 128;
   constexpr int STAGE_ROW = 256 + 16;        // 64 fp32 + pad: conflict-free 16-byte row writes
@@ -510,7 +502,8 @@ __global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, Tile
   __shared__ uint64_t q_full[NS], q_empty[NS], kv_empty, s_full[2], p_ready[2], o_full[2], t_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_fail;
-  __shared__ int s_ent[2][128];          // the producers' copy of the current / next tile's entries
+  __shared__ int s_ent[kMetaRing][128];  // per-tile entries, written by the producers, read by all roles
+  __shared__ float s_lse[kMetaRing][128]; // per-row softmax denominators (attention kernel only)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
@@ -534,15 +527,12 @@ __global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, Tile
 
   if (warp < 4) {
     // ------------------------------------------------ producers
-    int it = 0, signalled = 0, kiter = 0;
+    int it = 0, kiter = 0, ent_next = -1;
     bool stop = false;
     for (int item = blockIdx.x; item < n_items && !stop; item += gridDim.x, ++kiter) {
       const ItemInfo inf = item_info(a, item, tpt);
       const int bh = inf.key / (a.NW * a.Mk), leaf = inf.key % a.Mk;
       const int b = bh / geo.Hkv, h = bh % geo.Hkv;
-      cp_async_wait_all();
-      fence_proxy_async_smem();
-      for (; signalled < it; ++signalled) mbar_arrive(&q_full[signalled % NS]);
       bool bad = s_fail != 0;
       if (!bad && kiter > 0) bad = !mbar_wait_bounded(&kv_empty, (uint32_t)((kiter - 1) & 1));
       if (prod_sync_or(bad)) { s_fail = 1; stop = true; break; }
@@ -553,34 +543,24 @@ __global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, Tile
       const __nv_bfloat16* qb = a.q + (long long)b * geo.qs[0] + (long long)(h * G) * geo.qs[2];
       for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
         const int s = it % NS;
-        bool bad_t = false;
-        if (it >= NS) {
-          // ring slot still busy: first hand over every tile already issued (their arrival is what
-          // lets the consumers make the progress that frees the slot), then wait for it
-          const uint32_t par = (uint32_t)((it / NS - 1) & 1);
-          if (prod_sync_or(!mbar_test(&q_empty[s], par))) {
-            cp_async_wait_all();
-            fence_proxy_async_smem();
-            for (; signalled < it; ++signalled) mbar_arrive(&q_full[signalled % NS]);
-            bad_t = !mbar_wait_bounded(&q_empty[s], par);
-          }
-        }
+        const bool bad_t = it >= NS && !mbar_wait_bounded(&q_empty[s], (uint32_t)((it / NS - 1) & 1));
         const int e0 = inf.e_begin + jt * tpt;
-        s_ent[it & 1][tid] = (tid < tpt && e0 + tid < inf.e_end) ? a.entries[e0 + tid] : -1;
+        const int ent_now = (jt == 0) ? fetch_entry(a.entries, e0, inf.e_end, tpt, tid) : ent_next;
+        ent_next = (jt + 1 < inf.ntiles) ? fetch_entry(a.entries, e0 + tpt, inf.e_end, tpt, tid) : -1;
+        s_ent[it % kMetaRing][tid] = ent_now;
         if (prod_sync_or(bad_t)) { s_fail = 1; stop = true; break; }
-        prod_gather_q<D>(sQ + s * Q_STAGE, geo, qb, s_ent[it & 1], tid);
-        cp_async_commit();
-        if (it + 1 - signalled >= NS) {
-          cp_async_wait_group<NS - 1>();
-          fence_proxy_async_smem();
-          mbar_arrive(&q_full[signalled % NS]);
-          ++signalled;
+        prod_gather_q<D>(sQ + s * Q_STAGE, geo, qb, s_ent[it % kMetaRing], tid);
+        {  // the row's softmax denominator rides along (4-byte copy per row)
+          const int ent_r = s_ent[it % kMetaRing][tid >> lgG];
+          if (ent_r >= 0)
+            cp_async4(smem_u32(&s_lse[it % kMetaRing][tid]),
+                      a.row_lse + ((long long)b * geo.Hq + h * G + (tid & (G - 1))) * geo.N + (ent_r & 0xFFFFFF));
         }
+        fence_proxy_async_smem();                 // zero-filled rows (plain stores) -> async proxy
+        cp_async_arrive_noinc(&q_full[s]);        // fires when this thread's copies have landed
       }
     }
     cp_async_wait_all();
-    fence_proxy_async_smem();
-    for (; signalled < it; ++signalled) mbar_arrive(&q_full[signalled % NS]);
   } else if (warp == 4) {
     // ------------------------------------------------ MMA issuer
     // Event driven: S(it) goes out as soon as its query tile has landed and its TMEM buffers are
@@ -629,6 +609,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, Tile
       if (do_s) {
         const int s = s_it % NS, buf = s_it & 1;
         if (lane == 0) {
+          fence_proxy_async_smem();
           tcgen05_fence_after_sync();
           const uint32_t q0 = smem_u32(sQ + s * Q_STAGE), k0 = smem_u32(sK);
 #pragma unroll
@@ -679,23 +660,21 @@ __global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, Tile
         if ((it & 1) != grp) continue;
         const int s = it % NS;
         uint8_t* slot_base = sQ + s * Q_STAGE;
-        const int e0 = inf.e_begin + jt * tpt;
-        const int e = row >> lgG;
-        const int ent = (e0 + e < inf.e_end && e < tpt) ? a.entries[e0 + e] : -1;
+        const uint32_t par = (uint32_t)((it >> 1) & 1);
+        if (!mbar_wait_bounded(&s_full[grp], par)) { s_fail = 1; break; }
+        tcgen05_fence_after_sync();
+        const int ent = s_ent[it % kMetaRing][row >> lgG];
         const bool valid = ent >= 0;
         const int t = ent & 0xFFFFFF;
         float neg_lse2 = 0.f;
         int ncols = 0;
         if (valid) {
-          const float l2 = a.row_lse[((long long)b * geo.Hq + hq) * geo.N + t] * kLog2e;
+          const float l2 = s_lse[it % kMetaRing][row] * kLog2e;
           const int c_t = t / C;
           if (leaf <= c_t && l2 > -CUDART_INF_F)
             ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
           neg_lse2 = -l2;
         }
-        const uint32_t par = (uint32_t)((it >> 1) & 1);
-        if (!mbar_wait_bounded(&s_full[grp], par)) { s_fail = 1; break; }
-        tcgen05_fence_after_sync();
         {
           const bool fast = __all_sync(0xffffffffu, ncols == C);
           uint32_t ra[32], rb[32];
@@ -1009,10 +988,10 @@ int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char
 
 template <int D, int NB>
 int launch_tile_lse(const Geometry& g, const TileArgs& a, cudaStream_t s) {
-  const size_t smem = (size_t)(D / 64) * (3 * 128 * 128 + NB * 128) + 1024;
+  const size_t smem = (size_t)(D / 64) * (4 * 128 * 128 + NB * 128) + 1024;
   cudaError_t e = cudaFuncSetAttribute(lse_ws_kernel<D, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("lse_ws attr", e); return PISA_ERR_CUDA; }
-  lse_ws_kernel<D, NB><<<num_sms(), kWsThreads, smem, s>>>(g, a);
+  lse_ws_kernel<D, NB><<<num_sms(), kLseThreads, smem, s>>>(g, a);
   return check_launch("lse_ws");
 }
 
@@ -1033,7 +1012,7 @@ template <int D, int C>
 int launch_tile_pv(const Geometry& g, const TileArgs& a, cudaStream_t s) {
   constexpr int KS = D / 64;
   constexpr int QP = (KS * 128 * 128 > 128 * 272) ? KS * 128 * 128 : 128 * 272;
-  const size_t smem = 3 * (size_t)((QP + 1023) / 1024 * 1024) + 2 * (size_t)KS * C * 128 + 1024;
+  const size_t smem = 4 * (size_t)((QP + 1023) / 1024 * 1024) + 2 * (size_t)KS * C * 128 + 1024;
   cudaError_t e = cudaFuncSetAttribute(pv_ws_kernel<D, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("pv_ws attr", e); return PISA_ERR_CUDA; }
   pv_ws_kernel<D, C><<<num_sms(), kWsThreads, smem, s>>>(g, a);
