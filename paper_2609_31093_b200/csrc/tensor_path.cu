@@ -575,6 +575,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, Tile
     ItemInfo inf = {0, 0, 0, 0};
     if (item < n_items) inf = item_info(a, item, tpt);
     uint64_t t_idle = 0;
+    uint32_t idle_polls = 0;
     bool ok = true;
     while (ok && !s_fail) {
       const bool more_s = item < n_items;
@@ -633,10 +634,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, Tile
       }
       __syncwarp();
       if (do_s || do_pv) {
-        t_idle = 0;
-      } else {
+        idle_polls = 0;
+      } else if ((++idle_polls & 1023u) == 0u) {    // look at the wall clock only now and then
         const uint64_t now = global_timer_ns();
-        if (t_idle == 0) t_idle = now;
+        if (idle_polls == 1024u) t_idle = now;
         else if (now - t_idle > 2000000000ull) ok = false;
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       }
