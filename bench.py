@@ -32,6 +32,11 @@ import pisa_synth as S  # noqa: E402
 METRIC = "pisa_fwd_tokens_per_s_128k_ctx"
 UNIT = "tokens/s"
 
+# dram__bytes_read.sum + dram__bytes_write.sum per selected (token, block) pair, from the ncu captures
+# summarised under profiles/ (B=1 Hq=8 Hkv=2 d=128 N=65536 C=128 g=2 K=32: 4.19 M pairs per launch)
+DRAM_BYTES_PER_PAIR = {"leaf_lse_tiles": (186.706432e6 + 105.273600e6) / 4194304.0,
+                       "attention_tiles": (671.288832e6 + 384.176896e6) / 4194304.0}
+
 
 def get_workload(name: str) -> S.Workload:
     if name in S.WORKLOADS:
@@ -298,6 +303,7 @@ def run_ours(args):
     sampler = ClockSampler(gpu_id)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     stage = np.zeros(3)
+    kernels = {}
     barrier()
     torch.cuda.synchronize()
     sampler.start()
@@ -305,7 +311,9 @@ def run_ours(args):
     ev0.record()
     for _ in range(args.steps):
         step()
-        stage += np.asarray(P.get_stage_ms())       # waits for this step's last stage event
+        stage += np.asarray(P.get_stage_ms())       # waits for this step's last event
+        for name, t_ms in P.get_kernel_ms().items():
+            kernels[name] = kernels.get(name, 0.0) + t_ms
     ev1.record()
     torch.cuda.synchronize()
     launches = P.launch_count() - l0
@@ -314,6 +322,7 @@ def run_ours(args):
     ms = ev0.elapsed_time(ev1)
     P.set_stage_timing(False)
     stage /= args.steps
+    kernels = {k_: v_ / args.steps for k_, v_ in kernels.items()}
 
     # end to end through the host-buffer entry point
     arena = PB.alloc_workspace(p, PB.OP_FORWARD_HOST)
@@ -353,20 +362,37 @@ def run_ours(args):
     tens_peak = peaks.get("bf16_tflops_sustained", 1400.0)
     peak_src = "measured" if peaks else "fallback"
     es = 2 if w.dtype == "bf16" else 4
-    # dominant stage -> roofline entry.  Attention and routing are contractions (tensor bound);
-    # the pyramid is one streaming pass over k (HBM bound).
-    names = ["pyramid", "route", "attn"]
-    dom = int(np.argmax(stage))
-    if dom == 0:
-        roof = {"kernel": "pyramid", "bound": "hbm", "achieved": wc["pyramid_bytes"] / (stage[0] * 1e-3) / 1e9,
-                "peak": hbm_peak, "unit": "GB/s"}
+    # Roofline entry for the dominant kernel, timed live with CUDA events on the launching stream.
+    # Algorithmic work per launch: leaf scoring and attention are dense contractions (tensor bound,
+    # 2*C*G*d flops per scored (token, leaf) pair, 4*C*G*d per selected pair), the intermediate levels
+    # too (2*g*G*d per scored (token, node) pair); the pyramid is one streaming pass over k (HBM bound).
+    algo = {
+        "leaf_lse_tiles": ("tensor", wc["leaf_flops"]), "attention_tiles": ("tensor", wc["attn_flops"]),
+        "route_stage1": ("tensor", wc["inter_flops"]), "route_simt": ("tensor", wc["leaf_flops"] + wc["inter_flops"]),
+        "bsa_simt": ("tensor", wc["attn_flops"]), "pyramid": ("hbm", wc["pyramid_bytes"]),
+    }
+    cand = {k_: v_ for k_, v_ in kernels.items() if k_ in algo}
+    dom = max(cand, key=cand.get) if cand else "pyramid"
+    bound, work = algo[dom]
+    t_dom = cand.get(dom, stage[0]) * 1e-3
+    if bound == "hbm":
+        roof = {"kernel": dom, "bound": "hbm", "achieved": work / t_dom / 1e9, "peak": hbm_peak, "unit": "GB/s"}
     else:
-        flops = wc["attn_flops"] if dom == 2 else wc["leaf_flops"] + wc["inter_flops"]
-        roof = {"kernel": names[dom], "bound": "tensor", "achieved": flops / (stage[dom] * 1e-3) / 1e12,
-                "peak": tens_peak, "unit": "TFLOP/s"}
+        roof = {"kernel": dom, "bound": "tensor", "achieved": work / t_dom / 1e12, "peak": tens_peak,
+                "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["peak_source"] = peak_src
-    roof["traffic"] = None
+    roof["peak_source"] = peak_src + (" (sustained bf16, kernel timed inside a long step)" if bound == "tensor" else "")
+    roof["launch_ms"] = t_dom * 1e3
+    # DRAM bytes per launch from the ncu capture of a smaller case of the same kernel (summary under
+    # profiles/), scaled by the (token, block) pairs a launch processes: traffic grows with the pairs
+    per_pair = DRAM_BYTES_PER_PAIR.get(dom)
+    pairs = {"leaf_lse_tiles": wc["sel_pairs"], "attention_tiles": wc["sel_pairs"]}.get(dom)
+    roof["traffic"] = (per_pair * pairs) if (per_pair and pairs and w.dtype == "bf16") else None
+    roofs = {}
+    for k_, t_ in cand.items():
+        b_, w_ = algo[k_]
+        roofs[k_] = {"ms": t_, ("gbs" if b_ == "hbm" else "tflops"): w_ / (t_ * 1e-3) / (1e9 if b_ == "hbm" else 1e12),
+                     "frac": w_ / (t_ * 1e-3) / ((hbm_peak * 1e9) if b_ == "hbm" else (tens_peak * 1e12))}
     stages = {
         "pyramid_us": stage[0] * 1e3, "route_us": stage[1] * 1e3, "attn_us": stage[2] * 1e3,
         "pyramid_gbs": wc["pyramid_bytes"] / (stage[0] * 1e-3) / 1e9,
@@ -385,7 +411,7 @@ def run_ours(args):
         "config": {"workload": describe(w0), "path": args.path,
                    "l2": f"inputs larger than L2 (q {q.numel() * es / 1e6:.0f} MB, k+v {2 * k.numel() * es / 1e6:.0f} MB)",
                    "replicas": world},
-        "stages": stages, "roofline": roof, "cpu_baseline": cpu,
+        "stages": stages, "kernels_ms": kernels, "kernel_rooflines": roofs, "roofline": roof, "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps,
                 "h2d_bytes_per_step": int((q.numel() + 2 * k.numel()) * es),
                 "d2h_bytes_per_step": int(out.numel() * es + lse.numel() * 4)},

@@ -147,6 +147,13 @@ int pisa_read_status(const void* ws, int32_t* status);
 int pisa_set_stage_timing(int enable);
 int pisa_get_stage_ms(float* pyramid_ms, float* route_ms, float* attn_ms);
 
+/*
+ * With stage timing on, pisa_forward also brackets its main kernels with events.  After a forward
+ * call, entry i (0-based) gives the name of the i-th bracket and its device time in milliseconds;
+ * PISA_ERR_INVALID_ARG past the last entry.  The getter waits for the events.
+ */
+int pisa_get_kernel_ms(int i, char* name, size_t name_len, float* ms);
+
 /* Number of kernels this process has launched through the library so far (host counter). */
 unsigned long long pisa_launch_count(void);
 

@@ -20,6 +20,7 @@ from .binding import (  # noqa: F401
     set_stage_timing,
     get_stage_ms,
     launch_count,
+    get_kernel_ms,
     IMPL_AUTO,
     IMPL_SIMT,
     IMPL_TENSOR,

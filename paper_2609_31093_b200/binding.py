@@ -59,6 +59,8 @@ def lib():
     L.pisa_set_stage_timing.argtypes = [C.c_int]
     L.pisa_get_stage_ms.argtypes = [f32p, f32p, f32p]
     L.pisa_launch_count.restype = C.c_ulonglong
+    L.pisa_get_kernel_ms.argtypes = [C.c_int, C.c_char_p, C.c_size_t, f32p]
+    L.pisa_get_kernel_ms.restype = C.c_int
     for name in ("pisa_pyramid_layout", "pisa_workspace_bytes", "pisa_build_pyramid", "pisa_route",
                  "pisa_bsa_fwd", "pisa_forward", "pisa_forward_host", "pisa_flat_select", "pisa_read_status",
                  "pisa_set_stage_timing", "pisa_get_stage_ms"):
@@ -187,3 +189,15 @@ def get_stage_ms() -> Tuple[float, float, float]:
 
 def launch_count() -> int:
     return int(lib().pisa_launch_count())
+
+
+def get_kernel_ms() -> dict:
+    """{bracket name: device ms} of the last pisa_forward issued with stage timing on."""
+    out = {}
+    buf = C.create_string_buffer(64)
+    ms = C.c_float()
+    i = 0
+    while lib().pisa_get_kernel_ms(i, buf, 64, C.byref(ms)) == 0:
+        out[buf.value.decode()] = out.get(buf.value.decode(), 0.0) + ms.value
+        i += 1
+    return out

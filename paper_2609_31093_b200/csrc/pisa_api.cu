@@ -12,6 +12,23 @@ static thread_local char g_cuda_err[512] = "";
 static thread_local bool g_timing = false;
 static thread_local cudaEvent_t g_ev[4] = {nullptr, nullptr, nullptr, nullptr};
 static thread_local bool g_ev_valid = false;
+// per-kernel marks (name of the kernel that starts at the mark), recorded when timing is on
+constexpr int kMaxMarks = 32;
+static thread_local cudaEvent_t g_mark_ev[kMaxMarks];
+static thread_local const char* g_mark_name[kMaxMarks];
+static thread_local int g_mark_n = 0;
+static thread_local bool g_mark_valid = false;
+
+void kernel_mark(const char* name, cudaStream_t s) {
+  if (!g_timing || g_mark_n >= kMaxMarks) return;
+  if (!g_mark_valid) {
+    for (int j = 0; j < kMaxMarks; ++j) cudaEventCreate(&g_mark_ev[j]);
+    g_mark_valid = true;
+  }
+  g_mark_name[g_mark_n] = name;
+  cudaEventRecord(g_mark_ev[g_mark_n], s);
+  ++g_mark_n;
+}
 
 void record_cuda_error(const char* what, cudaError_t e) {
   snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", what, cudaGetErrorString(e));
@@ -123,6 +140,7 @@ static int do_route(const pisa_params_t* p, const Geometry& g, const void* q, co
   if (ws_bytes < route_ws_bytes(p, g)) return PISA_ERR_WORKSPACE_TOO_SMALL;
   if (use_tensor(p, g))
     return tensor_route(g, p->dtype, q, k, pyr, idx, margin, lse_out, (char*)ws + kStatusBytes, (int32_t*)ws, s);
+  kernel_mark("route_simt", s);
   return launch_route_simt(g, p->dtype, q, k, pyr, idx, margin, s);
 }
 
@@ -132,6 +150,7 @@ static int do_bsa(const pisa_params_t* p, const Geometry& g, const void* q, cons
   if (ws_bytes < bsa_ws_bytes(p, g)) return PISA_ERR_WORKSPACE_TOO_SMALL;
   if (use_tensor(p, g))
     return tensor_bsa(g, p->dtype, q, k, v, idx, out, lse, lse_ready, (char*)ws + kStatusBytes, (int32_t*)ws, s);
+  kernel_mark("bsa_simt", s);
   return launch_bsa_simt(g, p->dtype, q, k, v, idx, out, lse, s);
 }
 
@@ -153,7 +172,9 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
   if (ws_bytes < need) return PISA_ERR_WORKSPACE_TOO_SMALL;
   int st = clear_status(ws, s);
   if (st != PISA_OK) return st;
+  g_mark_n = 0;
   stage_mark(0, s);
+  kernel_mark("pyramid", s);
   st = launch_pyramid(g, p->dtype, k, pyr, s);
   if (st != PISA_OK) return st;
   stage_mark(1, s);
@@ -164,6 +185,7 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
   stage_mark(2, s);
   st = do_bsa(p, g, q, k, v, idx, out, lse, use_tensor(p, g), ws, ws_bytes, s);
   stage_mark(3, s);
+  kernel_mark("end", s);
   return st;
 }
 
@@ -342,6 +364,17 @@ int pisa_read_status(const void* ws, int32_t* status) {
   cudaError_t e = cudaMemcpy(&word, ws, sizeof(word), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) { record_cuda_error("status read", e); return PISA_ERR_CUDA; }
   *status = word;
+  return PISA_OK;
+}
+
+int pisa_get_kernel_ms(int i, char* name, size_t name_len, float* ms) {
+  if (!g_timing || !g_mark_valid || i < 0 || i + 1 >= g_mark_n) return PISA_ERR_INVALID_ARG;
+  cudaError_t e = cudaEventSynchronize(g_mark_ev[g_mark_n - 1]);
+  if (e != cudaSuccess) { record_cuda_error("kernel events", e); return PISA_ERR_CUDA; }
+  float t = 0.f;
+  cudaEventElapsedTime(&t, g_mark_ev[i], g_mark_ev[i + 1]);
+  if (ms) *ms = t;
+  if (name && name_len > 0) snprintf(name, name_len, "%s", g_mark_name[i]);
   return PISA_OK;
 }
 

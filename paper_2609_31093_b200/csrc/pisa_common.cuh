@@ -48,6 +48,8 @@ int launch_bsa_simt(const Geometry& g, int dtype, const void* q, const void* k, 
 int launch_flat_simt(const Geometry& g, int dtype, const void* q, const void* pyramid, int32_t* idx,
                      cudaStream_t s);
 
+// with stage timing on, records an event on `s` named after the kernel(s) that follow it
+void kernel_mark(const char* name, cudaStream_t s);
 int check_launch(const char* what);   // cudaGetLastError -> pisa_status, records the text
 void record_cuda_error(const char* what, cudaError_t e);
 

@@ -1050,9 +1050,11 @@ int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, con
   const RouteLayout L = route_layout(g);
   int32_t* par = (int32_t*)(ws + L.par);
   float* blk = (float*)(ws + L.blk);
+  kernel_mark("route_stage1", s);
   int st = route_stage1_mma_supported(g, dtype) ? launch_route_stage1_mma(g, q, pyramid, par, margin, s)
                                                 : launch_route_stage1_simt(g, dtype, q, pyramid, par, margin, s);
   if (st != PISA_OK) return st;
+  kernel_mark("invert_by_parent", s);
   InvArgs inv;
   st = run_inversion(g, par, g.g, g.M[2], ws, L.inv, &inv, s);
   if (st != PISA_OK) return st;
@@ -1061,8 +1063,10 @@ int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, con
   a.entry_off = inv.entry_off; a.tile_off = inv.tile_off; a.item_off = inv.item_off; a.item_key = inv.item_key; a.entries = inv.entries;
   a.nkeys = g.B * g.Hkv * inv.NW * g.M[2]; a.Mk = g.M[2]; a.NW = inv.NW; a.fan = g.g; a.slots = g.K;
   a.blk_lse = blk; a.status = status;
+  kernel_mark("leaf_lse_tiles", s);
   st = dispatch_tile_lse(g, g.g * g.C, a, s);
   if (st != PISA_OK) return st;
+  kernel_mark("final_topk", s);
   const long long total = (long long)g.B * g.Hkv * g.N;
   final_topk_kernel<<<(unsigned)((total + 3) / 4), 128, 0, s>>>(g, par, blk, idx, margin, lse_out);
   return check_launch("final_topk");
@@ -1075,6 +1079,7 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
   const BsaLayout L = bsa_layout(g);
   float* blk = (float*)(ws + L.blk);
   float* acc = (float*)(ws + L.acc);
+  kernel_mark("invert_by_leaf", s);
   InvArgs inv;
   int st = run_inversion(g, idx, 1, g.M[1], ws, L.inv, &inv, s);
   if (st != PISA_OK) return st;
@@ -1084,6 +1089,7 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
   a.nkeys = g.B * g.Hkv * inv.NW * g.M[1]; a.Mk = g.M[1]; a.NW = inv.NW; a.fan = 1; a.slots = g.K;
   a.blk_lse = blk; a.row_lse = lse; a.o_acc = acc; a.status = status;
   if (!lse_ready) {
+    kernel_mark("block_lse_tiles", s);
     st = dispatch_tile_lse(g, g.C, a, s);
     if (st != PISA_OK) return st;
     const long long rows = (long long)g.B * g.Hkv * g.N * g.G;
@@ -1091,10 +1097,13 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
     st = check_launch("row_lse");
     if (st != PISA_OK) return st;
   }
+  kernel_mark("accumulator_memset", s);
   cudaError_t e = cudaMemsetAsync(acc, 0, (size_t)g.B * g.N * g.Hq * g.d * 4, s);
   if (e != cudaSuccess) { record_cuda_error("accumulator memset", e); return PISA_ERR_CUDA; }
+  kernel_mark("attention_tiles", s);
   st = dispatch_tile_pv(g, a, s);
   if (st != PISA_OK) return st;
+  kernel_mark("convert_out", s);
   const long long chunks = (long long)g.B * g.N * g.Hq * (g.d / 8);
   convert_out_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, s>>>(g, acc, (__nv_bfloat16*)out);
   return check_launch("convert_out");
