@@ -40,7 +40,9 @@ typedef enum {
   PISA_ERR_WORKSPACE_TOO_SMALL = -3,
   PISA_ERR_CUDA = -4,                /* a launch or copy failed; pisa_last_cuda_error() has the text */
   PISA_ERR_TIMEOUT = -5,             /* a bounded device-side wait gave up (read from the status word) */
-  PISA_ERR_BOUNDS = -6               /* a device-side index check failed (read from the status word) */
+  PISA_ERR_BOUNDS = -6,              /* a device-side index check failed (read from the status word) */
+  PISA_ERR_STATIC_SCRATCH_TOO_SMALL = -7  /* pisa_route_static: the problem needs more scratch than the
+                                             library's built-in device array holds */
 } pisa_status;
 
 enum { PISA_BF16 = 0, PISA_FP32 = 1 };
@@ -110,6 +112,29 @@ int pisa_route(const pisa_params_t* p, const void* q, const void* k, const void*
  */
 int pisa_bsa_fwd(const pisa_params_t* p, const void* q, const void* k, const void* v, const int32_t* idx,
                  void* out, float* lse, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * pisa_route for callers that cannot provide a workspace because they are not allowed to allocate
+ * device memory where they run (a memory pool that is fully assigned, a serving plugin that forbids
+ * allocation after start-up, a loop that cannot afford cudaMalloc's implicit synchronisation).
+ * (No counterpart in the paper: this is a property of the library, not of the method.)
+ *
+ * Same arguments and results as pisa_route, without ws / ws_bytes: the scratch is a 32 MiB device
+ * array built into the library (pisa_route_static_capacity()), present on every GPU that loads the
+ * library until the process exits.  The call allocates nothing, on the host or on the device.
+ *  - Problems whose PISA_OP_ROUTE workspace exceeds the capacity are refused with
+ *    PISA_ERR_STATIC_SCRATCH_TOO_SMALL before anything is launched.
+ *  - The first call on each device looks up the array's device address (the device that is current
+ *    at the call); make that first call outside any stream capture.
+ *  - All calls on one device share the array, which keeps whatever the last call left in it; each
+ *    call zeroes what it needs zeroed, on `stream`, before use.  Two calls that can overlap on the
+ *    GPU (different streams, or different host threads without ordering) race on it: serialise them.
+ *  - The device status word of this variant is not exposed; use pisa_route with your own workspace
+ *    where you need pisa_read_status.  Keep stage timing off (the default) for an allocation-free call.
+ */
+int pisa_route_static(const pisa_params_t* p, const void* q, const void* k, const void* pyramid,
+                      int32_t* idx, float* margin, void* stream);
+size_t pisa_route_static_capacity(void);
 
 /* pyramid -> route -> attention in one call.  pyramid and idx are outputs too (kept for reuse). */
 int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const void* v, void* pyramid,

@@ -12,6 +12,8 @@ from .binding import (  # noqa: F401
     workspace_bytes,
     pisa_build_pyramid,
     pisa_route,
+    pisa_route_static,
+    route_static_capacity,
     pisa_bsa_fwd,
     pisa_forward,
     pisa_forward_host,

@@ -56,6 +56,9 @@ def lib():
     L.pisa_forward_host.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
     L.pisa_flat_select.argtypes = [pp, vp, vp, vp, vp, C.c_size_t, vp]
     L.pisa_read_status.argtypes = [vp, i32p]
+    L.pisa_route_static.argtypes = [pp, vp, vp, vp, vp, vp, vp]
+    L.pisa_route_static.restype = C.c_int
+    L.pisa_route_static_capacity.restype = C.c_size_t
     L.pisa_set_stage_timing.argtypes = [C.c_int]
     L.pisa_get_stage_ms.argtypes = [f32p, f32p, f32p]
     L.pisa_launch_count.restype = C.c_ulonglong
@@ -145,6 +148,18 @@ def pisa_build_pyramid(p: Params, k: torch.Tensor, pyramid: torch.Tensor):
 def pisa_route(p: Params, q, k, pyramid, idx, margin, ws):
     _check(lib().pisa_route(p.ref(), _ptr(q), _ptr(k), _ptr(pyramid), _ptr(idx), _ptr(margin), _ptr(ws),
                             ws.numel(), _stream()), "pisa_route")
+
+
+def pisa_route_static(p: Params, q, k, pyramid, idx, margin):
+    """pisa_route without a workspace argument: scratch lives in a device array inside the library.
+    For callers that may not allocate device memory; refuses problems above
+    pisa_route_static_capacity() and must not overlap with another such call on the same GPU."""
+    _check(lib().pisa_route_static(p.ref(), _ptr(q), _ptr(k), _ptr(pyramid), _ptr(idx), _ptr(margin), _stream()),
+           "pisa_route_static")
+
+
+def route_static_capacity() -> int:
+    return int(lib().pisa_route_static_capacity())
 
 
 def pisa_bsa_fwd(p: Params, q, k, v, idx, out, lse, ws):

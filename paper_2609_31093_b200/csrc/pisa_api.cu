@@ -206,6 +206,8 @@ const char* pisa_status_string(int status) {
     case PISA_ERR_CUDA: return "CUDA error";
     case PISA_ERR_TIMEOUT: return "device-side wait timed out";
     case PISA_ERR_BOUNDS: return "device-side index check failed";
+    case PISA_ERR_STATIC_SCRATCH_TOO_SMALL:
+      return "problem needs more scratch than the library's built-in device array holds";
     default: return "unknown status";
   }
 }
