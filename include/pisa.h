@@ -59,7 +59,7 @@ typedef struct {
   int32_t dtype;                     /* PISA_BF16 | PISA_FP32: q, k, v, out, summaries share it */
   int32_t score_mode;                /* PISA_SCORE_*                                            */
   int32_t impl;                      /* PISA_IMPL_*                                             */
-  float   scale;                     /* logit scale; 0 => 1/sqrt(d)  (Eq. "block scores")       */
+  float   scale;                     /* logit scale, > 0; 0 => 1/sqrt(d)  (Eq. "block scores")  */
   int32_t reserved;
   int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3]; /* elements, (b, n, h); all 0 => dense */
 } pisa_params_t;

@@ -53,7 +53,7 @@ static size_t elem_size(int dtype) { return dtype == PISA_BF16 ? 2 : 4; }
 int resolve(const pisa_params_t* p, Geometry* g) {
   if (p == nullptr || g == nullptr) return PISA_ERR_INVALID_ARG;
   if (p->B <= 0 || p->N <= 0 || p->Hq <= 0 || p->Hkv <= 0 || p->d <= 0 || p->C <= 0) return PISA_ERR_INVALID_ARG;
-  if (p->Hq % p->Hkv != 0 || p->K < 3 || p->g < 2) return PISA_ERR_INVALID_ARG;
+  if (p->Hq % p->Hkv != 0 || p->K < 3 || p->g < 2 || !(p->scale >= 0.f)) return PISA_ERR_INVALID_ARG;
   if (p->dtype != PISA_BF16 && p->dtype != PISA_FP32) return PISA_ERR_UNSUPPORTED;
   if (p->causal != 1) return PISA_ERR_UNSUPPORTED;
   if (p->score_mode < PISA_SCORE_LSE || p->score_mode > PISA_SCORE_MEAN_VAR) return PISA_ERR_UNSUPPORTED;

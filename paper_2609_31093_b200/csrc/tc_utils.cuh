@@ -193,6 +193,22 @@ __device__ __forceinline__ void st_shared_zero16(uint32_t saddr) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(saddr), "r"(0u) : "memory");
 }
 
+// ---------------------------------------------------------------- TMA (tiled tensor copies)
+
+// 4-D tiled load global -> shared memory of this CTA; completes `bytes` of transaction on `bar`.
+// `tmap` points at a CUtensorMap (kernel parameter / constant / global memory, 64-byte aligned).
+__device__ __forceinline__ void tma_load_4d(uint32_t sdst, const void* tmap, uint64_t* bar, int c0, int c1, int c2,
+                                            int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(sdst), "l"(tmap), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+// announce `bytes` of pending transaction on `bar` without arriving
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+
 // ---------------------------------------------------------------- bulk reduction to global
 
 // global[dst .. dst+bytes) += shared[src .. src+bytes) as fp32 adds, performed by the copy engine

@@ -17,7 +17,7 @@
 //               [lse_ws + row_lse only when the denominators are not already known]
 //               pv_ws_kernel                -> S = Q K^T, P = exp(S - lse_row) (already normalised),
 //                                              O_partial = P V, added into an fp32 accumulator with
-//                                              bulk reductions (one 256-byte row segment per thread)
+//                                              vector reductions (two 256-byte row segments per instruction)
 //               convert                     -> out in the storage dtype
 #include <math_constants.h>
 
@@ -481,12 +481,17 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
   if (warp == 0) tmem_dealloc(tmem, TM_COLS);
 }
 
-// Attention tiles, same role layout.  Per tile: S = Q K^T (UMMA) -> an epilogue group turns S into
-// P = 2^(S*scale*log2e - lse2) in bf16, overwriting the query tile's ring slot -> O_partial = P V
-// (UMMA, V as the MN-major operand) -> the same group moves O through its ring slot (now free) into
-// the fp32 accumulator with bulk reductions, then releases the slot and the TMEM buffers.
+// Attention tiles.  Roles: warps 0-3 producers, warp 4 UMMA issuer, warps 5-8 / 9-12 two softmax groups
+// taking alternate tiles, warps 13-16 the reducer.  Per tile: S = Q K^T (UMMA) -> a softmax group
+// turns S into P = 2^(S*scale*log2e - lse2) in bf16, overwriting the query tile's ring slot ->
+// O_partial = P V (UMMA, V as the MN-major operand) -> the reducer moves O out of TMEM through the
+// (now free) ring slot and adds it into the fp32 accumulator with coalesced vector reductions, then
+// releases the slot.  The reduction stream into L2 is the floor of this kernel (64 KB of fp32 adds
+// per tile), so it gets warps of its own and is never stalled by the exponentials.
+constexpr int kPvThreads = 544;
+
 template <int D, int C>
-__global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, TileArgs a) {
+__global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, TileArgs a) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int NS = 4;
   constexpr int KS = D / 64;
@@ -499,18 +504,19 @@ __global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, Tile
   uint8_t* sQ = smem;
   uint8_t* sK = smem + NS * Q_STAGE;
   uint8_t* sV = sK + KS * KV_SLAB;
-  __shared__ uint64_t q_full[NS], q_empty[NS], kv_empty, s_full[2], p_ready[2], o_full[2], t_empty[2];
+  __shared__ uint64_t q_full[NS], q_empty[NS], kv_empty, s_full[2], s_empty[2], p_ready[2], o_full[2], o_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_fail;
-  __shared__ int s_ent[kMetaRing][128];  // per-tile entries, written by the producers, read by all roles
-  __shared__ float s_lse[kMetaRing][128]; // per-row softmax denominators (attention kernel only)
+  __shared__ int s_ent[kMetaRing][128];   // per-tile entries, written by the producers, read by all roles
+  __shared__ float s_lse[kMetaRing][128]; // per-row softmax denominators
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) { mbar_init(&q_full[i], kProdThreads); mbar_init(&q_empty[i], 128); }
     mbar_init(&kv_empty, 1);
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&s_full[i], 1); mbar_init(&p_ready[i], 128); mbar_init(&o_full[i], 1); mbar_init(&t_empty[i], 128);
+      mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 128); mbar_init(&p_ready[i], 128);
+      mbar_init(&o_full[i], 1); mbar_init(&o_empty[i], 128);
     }
     s_fail = 0;
     mbar_fence_init();
@@ -563,10 +569,9 @@ __global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, Tile
     cp_async_wait_all();
   } else if (warp == 4) {
     // ------------------------------------------------ MMA issuer
-    // Event driven: S(it) goes out as soon as its query tile has landed and its TMEM buffers are
-    // free, P V(it) as soon as the epilogue group has written P(it); neither waits for the other, so
-    // a late query tile cannot hold back the P V that frees the ring slot the producer is waiting
-    // for.  Lane 0 probes and issues; the warp stays converged on its decisions.
+    // Event driven: S(it) goes out as soon as its query tile has landed and its S buffer has been
+    // read out, P V(it) as soon as P(it) is written and its O buffer has been read out; neither
+    // waits for the other.  Lane 0 probes and issues; the warp stays converged on its decisions.
     const uint32_t idesc_s = make_idesc_bf16(128, C, 0, 0);
     const uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
     int s_it = 0, pv_it = 0;              // next tile whose S / whose P V is to be issued
@@ -585,9 +590,13 @@ __global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, Tile
         if (more_s && s_it - pv_it < 2) {
           const int s = s_it % NS, buf = s_it & 1;
           do_s = mbar_test(&q_full[s], (uint32_t)((s_it / NS) & 1)) &&
-                 (s_it < 2 || mbar_test(&t_empty[buf], (uint32_t)(((s_it >> 1) - 1) & 1)));
+                 (s_it < 2 || mbar_test(&s_empty[buf], (uint32_t)(((s_it >> 1) - 1) & 1)));
         }
-        if (pv_it < s_it) do_pv = mbar_test(&p_ready[pv_it & 1], (uint32_t)((pv_it >> 1) & 1));
+        if (pv_it < s_it) {
+          const int pb = pv_it & 1;
+          do_pv = mbar_test(&p_ready[pb], (uint32_t)((pv_it >> 1) & 1)) &&
+                  (pv_it < 2 || mbar_test(&o_empty[pb], (uint32_t)(((pv_it >> 1) - 1) & 1)));
+        }
       }
       do_s = __shfl_sync(0xffffffffu, do_s, 0);
       do_pv = __shfl_sync(0xffffffffu, do_pv, 0);
@@ -643,86 +652,103 @@ __global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, Tile
       }
     }
     if (!ok) s_fail = 1;
-  } else {
-    // ------------------------------------------------ epilogue groups
+  } else if (warp < 13) {
+    // ------------------------------------------------ softmax groups: S -> P
     const int grp = (warp - 5) >> 2;
     const int row = (warp & 3) * 32 + lane;
-    const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t s_base = tmem + lane_sel + (uint32_t)(grp * 128);
-    const uint32_t o_base = tmem + lane_sel + 256u + (uint32_t)(grp * 128);
-    const int head = row & (G - 1);
+    const uint32_t s_base = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(grp * 128);
     int it = 0;
     for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x) {
       const ItemInfo inf = item_info(a, item, tpt);
-      const int bh = inf.key / (a.NW * a.Mk), leaf = inf.key % a.Mk;
-      const int b = bh / geo.Hkv, h = bh % geo.Hkv;
-      const int hq = h * G + head;
+      const int leaf = inf.key % a.Mk;
       for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
         if ((it & 1) != grp) continue;
         const int s = it % NS;
         uint8_t* slot_base = sQ + s * Q_STAGE;
-        const uint32_t par = (uint32_t)((it >> 1) & 1);
-        if (!mbar_wait_bounded(&s_full[grp], par)) { s_fail = 1; break; }
+        if (!mbar_wait_bounded(&s_full[grp], (uint32_t)((it >> 1) & 1))) { s_fail = 1; break; }
         tcgen05_fence_after_sync();
         const int ent = s_ent[it % kMetaRing][row >> lgG];
-        const bool valid = ent >= 0;
         const int t = ent & 0xFFFFFF;
         float neg_lse2 = 0.f;
         int ncols = 0;
-        if (valid) {
+        if (ent >= 0) {
           const float l2 = s_lse[it % kMetaRing][row] * kLog2e;
           const int c_t = t / C;
           if (leaf <= c_t && l2 > -CUDART_INF_F)
             ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
           neg_lse2 = -l2;
         }
-        {
-          const bool fast = __all_sync(0xffffffffu, ncols == C);
-          uint32_t ra[32], rb[32];
-          tmem_ld_32x32(s_base, ra);
+        const bool fast = __all_sync(0xffffffffu, ncols == C);
+        uint32_t ra[32], rb[32];
+        tmem_ld_32x32(s_base, ra);
 #pragma unroll
-          for (int c0 = 0; c0 < C; c0 += 32) {
-            uint32_t (&cur)[32] = ((c0 >> 5) & 1) ? rb : ra;
-            uint32_t (&nxt)[32] = ((c0 >> 5) & 1) ? ra : rb;
-            tmem_ld_wait();
-            if (c0 + 32 < C) tmem_ld_32x32(s_base + (uint32_t)(c0 + 32), nxt);
-            uint32_t pk[16];
+        for (int c0 = 0; c0 < C; c0 += 32) {
+          uint32_t (&cur)[32] = ((c0 >> 5) & 1) ? rb : ra;
+          uint32_t (&nxt)[32] = ((c0 >> 5) & 1) ? ra : rb;
+          tmem_ld_wait();
+          if (c0 + 32 < C) {
+            tmem_ld_32x32(s_base + (uint32_t)(c0 + 32), nxt);
+          } else {
+            tcgen05_fence_before_sync();
+            mbar_arrive(&s_empty[grp]);         // S has been read out: the next S chain may overwrite it
+          }
+          uint32_t pk[16];
 #pragma unroll
-            for (int jx = 0; jx < 16; ++jx) {
-              float p0 = ex2_approx(fmaf(__uint_as_float(cur[2 * jx]), sl2, neg_lse2));
-              float p1 = ex2_approx(fmaf(__uint_as_float(cur[2 * jx + 1]), sl2, neg_lse2));
-              if (!fast) {
-                if (c0 + 2 * jx >= ncols) p0 = 0.f;
-                if (c0 + 2 * jx + 1 >= ncols) p1 = 0.f;
-              }
-              const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
-              pk[jx] = *reinterpret_cast<const uint32_t*>(&pp);
+          for (int jx = 0; jx < 16; ++jx) {
+            float p0 = ex2_approx(fmaf(__uint_as_float(cur[2 * jx]), sl2, neg_lse2));
+            float p1 = ex2_approx(fmaf(__uint_as_float(cur[2 * jx + 1]), sl2, neg_lse2));
+            if (!fast) {
+              if (c0 + 2 * jx >= ncols) p0 = 0.f;
+              if (c0 + 2 * jx + 1 >= ncols) p1 = 0.f;
             }
+            const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
+            pk[jx] = *reinterpret_cast<const uint32_t*>(&pp);
+          }
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-              const int ck = c0 / 8 + q4;
-              const uint32_t d = smem_u32(slot_base + (ck >> 3) * A_SLAB) + swz128(row, ck & 7);
-              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d), "r"(pk[4 * q4]),
-                           "r"(pk[4 * q4 + 1]), "r"(pk[4 * q4 + 2]), "r"(pk[4 * q4 + 3])
-                           : "memory");
-            }
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const int ck = c0 / 8 + q4;
+            const uint32_t d = smem_u32(slot_base + (ck >> 3) * A_SLAB) + swz128(row, ck & 7);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d), "r"(pk[4 * q4]),
+                         "r"(pk[4 * q4 + 1]), "r"(pk[4 * q4 + 2]), "r"(pk[4 * q4 + 3])
+                         : "memory");
           }
         }
         fence_proxy_async_smem();
-        tcgen05_fence_before_sync();
         mbar_arrive(&p_ready[grp]);
-        if (!mbar_wait_bounded(&o_full[grp], par)) { s_fail = 1; break; }
-        tcgen05_fence_after_sync();
-        // O partial through this thread's private row of the (now free) ring slot
+      }
+    }
+  } else {
+    // ------------------------------------------------ reducer: O partials -> fp32 accumulator
+    // Every thread parks 64 columns of its row in its padded row of the tile's ring slot (free once
+    // P V has completed); the warp then re-reads its own 32 rows two at a time, so that each vector
+    // reduction instruction adds two full 256-byte row segments.
+    const int row = (warp & 3) * 32 + lane;
+    const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+    const int sub = lane >> 4, ch = lane & 15;
+    int it = 0;
+    for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x) {
+      const ItemInfo inf = item_info(a, item, tpt);
+      const int bh = inf.key / (a.NW * a.Mk);
+      const int b = bh / geo.Hkv, h = bh % geo.Hkv;
+      float* acc_bh = a.o_acc + ((long long)b * geo.N * geo.Hq + h * G) * D;
+      for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
+        const int s = it % NS, ob = it & 1;
+        uint8_t* slot_base = sQ + s * Q_STAGE;
         uint8_t* stage = slot_base + row * STAGE_ROW;
-        float* orow = a.o_acc + (((long long)b * geo.N + t) * geo.Hq + hq) * D;
+        const int* ents = s_ent[it % kMetaRing];
+        const uint32_t o_base = tmem + lane_sel + 256u + (uint32_t)(ob * 128);
+        if (!mbar_wait_bounded(&o_full[ob], (uint32_t)((it >> 1) & 1))) { s_fail = 1; break; }
+        tcgen05_fence_after_sync();
 #pragma unroll
         for (int half = 0; half < KS; ++half) {
           uint32_t ra[32], rb[32];
           tmem_ld_32x32(o_base + (uint32_t)(half * 64), ra);
           tmem_ld_32x32(o_base + (uint32_t)(half * 64 + 32), rb);
-          if (half > 0) bulk_wait_read_all();
           tmem_ld_wait();
+          if (half == KS - 1) {
+            tcgen05_fence_before_sync();
+            mbar_arrive(&o_empty[ob]);          // O has been read out of TMEM
+          }
 #pragma unroll
           for (int q4 = 0; q4 < 8; ++q4)
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(stage) + q4 * 16), "r"(ra[4 * q4]),
@@ -733,19 +759,27 @@ __global__ void __launch_bounds__(kWsThreads, 1) pv_ws_kernel(Geometry geo, Tile
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(stage) + 128 + q4 * 16),
                          "r"(rb[4 * q4]), "r"(rb[4 * q4 + 1]), "r"(rb[4 * q4 + 2]), "r"(rb[4 * q4 + 3])
                          : "memory");
-          fence_proxy_async_smem();
-          if (valid) {
-            bulk_reduce_add_f32(orow + half * 64, smem_u32(stage), 256);
-            bulk_commit();
+          __syncwarp();
+#pragma unroll 4
+          for (int i = 0; i < 16; ++i) {
+            const int R = (warp & 3) * 32 + 2 * i + sub;           // tile row served by this half-warp
+            const int ent_r = ents[R >> lgG];
+            if (ent_r >= 0) {
+              float4 x;
+              asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                           : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w)
+                           : "r"(smem_u32(slot_base + R * STAGE_ROW) + ch * 16));
+              float* dst = acc_bh + ((long long)(ent_r & 0xFFFFFF) * geo.Hq + (R & (G - 1))) * D + half * 64 + ch * 4;
+              asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(x.x), "f"(x.y),
+                           "f"(x.z), "f"(x.w)
+                           : "memory");
+            }
           }
+          __syncwarp();
         }
-        tcgen05_fence_before_sync();
-        mbar_arrive(&t_empty[grp]);        // S and O accumulators of this parity are free
-        bulk_wait_read_all();               // the ring slot has been read out
-        mbar_arrive(&q_empty[s]);
+        mbar_arrive(&q_empty[s]);          // the ring slot is free again
       }
     }
-    bulk_wait_all();
   }
   tcgen05_fence_before_sync();
   __syncthreads();
@@ -1016,7 +1050,7 @@ int launch_tile_pv(const Geometry& g, const TileArgs& a, cudaStream_t s) {
   const size_t smem = 4 * (size_t)((QP + 1023) / 1024 * 1024) + 2 * (size_t)KS * C * 128 + 1024;
   cudaError_t e = cudaFuncSetAttribute(pv_ws_kernel<D, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("pv_ws attr", e); return PISA_ERR_CUDA; }
-  pv_ws_kernel<D, C><<<num_sms(), kWsThreads, smem, s>>>(g, a);
+  pv_ws_kernel<D, C><<<num_sms(), kPvThreads, smem, s>>>(g, a);
   return check_launch("pv_ws");
 }
 

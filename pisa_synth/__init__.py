@@ -3,9 +3,8 @@
 This module serves both the CPU oracle's tests and the CUDA path's tests and
 benchmark.  It holds none of the method's arithmetic (no pooling, scoring,
 selection or attention): it only draws random tensors with the structure of
-the paper's own selection benchmark (random queries and keys with a fixed
-seed, App. B "Block-selection benchmarks") plus the planted structure the
-workload table asks for, and converts fp32 values to bf16 bit patterns.
+the paper's own selection benchmark (seeded random tensors, App. B) plus the
+planted structure the workload table asks for, and converts fp32 values to bf16 bit patterns.
 
 Layouts: q is [B, N, Hq, d]; k and v are [B, N, Hkv, d]; d contiguous.
 bf16 tensors are returned as numpy uint16 bit patterns (numpy has no bf16).
