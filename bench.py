@@ -422,6 +422,61 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Routing latency vs N (BASELINE configs[4]) next to the flat O(N^2/C) selector built in the same
+    library, plus the paper's own benchmark shape; one JSON line per (workload, N).  Not the bench line."""
+    import torch
+
+    import paper_2609_31093_b200 as P
+    from paper_2609_31093_b200 import binding as PB
+
+    torch.cuda.set_device(0)
+    rows = []
+    plans = [("cfg5", [8192, 32768, 131072, 524288], lambda n: S.sweep_workload(n)),
+             ("paper_shape", [4096, 8192, 16384, 32768, 65536, 131072, 262144],
+              lambda n: S.Workload(f"paper_{n}", 1, n, 32, 2, 64, 64, 2, 8, "bf16", 5, "iid"))]
+    for tag, ns, mk in plans:
+        for n in ns:
+            w = mk(n)
+            t = S.make_inputs(w)
+            p = P.Params.from_workload(w)
+            dev = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda()
+            q, k, v = dev(t["q"]), dev(t["k"]), dev(t["v"])
+            pyramid = PB.alloc_pyramid(p)
+            idx = torch.empty((w.B, w.Hkv, w.N, w.K), dtype=torch.int32, device="cuda")
+            out = torch.empty_like(q)
+            lse = torch.empty((w.B, w.Hq, w.N), dtype=torch.float32, device="cuda")
+            ws = PB.alloc_workspace(p, PB.OP_FORWARD)
+
+            def timed(fn, reps):
+                for _ in range(2):
+                    fn()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(reps):
+                    fn()
+                e1.record()
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) / reps
+
+            reps = 5 if n <= 131072 else 2
+            t_pyr = timed(lambda: P.pisa_build_pyramid(p, k, pyramid), reps)
+            t_route = timed(lambda: P.pisa_route(p, q, k, pyramid, idx, None, ws), reps)
+            t_flat = timed(lambda: P.pisa_flat_select(p, q, pyramid, idx, ws), 1 if n > 131072 else reps)
+            t_fwd = timed(lambda: P.pisa_forward(p, q, k, v, pyramid, idx, out, lse, ws), reps)
+            st = P.read_status(ws)
+            row = {"sweep": tag, "workload": describe(w), "N": n, "pyramid_ms": t_pyr, "route_ms": t_route,
+                   "selection_ms": t_pyr + t_route, "flat_select_ms": t_flat, "flat_selection_ms": t_pyr + t_flat,
+                   "forward_ms": t_fwd, "forward_tokens_per_s": w.B * n / (t_fwd * 1e-3), "status": st,
+                   "route_us_per_token": t_route * 1e3 / n}
+            rows.append(row)
+            print(json.dumps(row), flush=True)
+            del q, k, v, pyramid, idx, out, lse, ws
+            torch.cuda.empty_cache()
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -433,7 +488,11 @@ def main():
     ap.add_argument("--ref-queries", type=int, default=192)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="routing latency vs N and the flat selector (not the bench line)")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

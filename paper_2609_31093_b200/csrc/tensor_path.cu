@@ -31,8 +31,8 @@ using namespace tc;
 namespace {
 
 constexpr int kInvTok = 1024;          // tokens per CTA in the inversion kernels
-constexpr int kWindowTok = 8192;       // tokens per window of the inverted lists
-constexpr int kItemTiles = 16;         // a work item: at most this many consecutive tiles of one list
+constexpr int kWindowTok = 16384;      // tokens per window of the inverted lists
+constexpr int kItemTiles = 32;         // a work item: at most this many consecutive tiles of one list
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -500,11 +500,17 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
   constexpr int QP_BYTES = (KS * A_SLAB > 128 * STAGE_ROW) ? KS * A_SLAB : 128 * STAGE_ROW;
   constexpr int Q_STAGE = (QP_BYTES + 1023) / 1024 * 1024;
   constexpr uint32_t TM_COLS = 512;          // S buffers at columns 0 / 128, O buffers at 256 / 384
+  // d = 128: the second product is issued transposed, O^T = V^T P^T (A = V, MN-major; B = P): a TMEM lane
+  // is then one output column d and consecutive TMEM columns are the G heads of one token.  With the
+  // accumulator laid out [B, N, Hkv, d, G] (heads innermost) a thread adds its G values with one vector
+  // reduction and a warp covers 32*G consecutive floats: fully coalesced, no staging in shared memory.
+  constexpr bool kTransO = (D == 128);
   uint8_t* smem = align1024(smem_raw);
   uint8_t* sQ = smem;
   uint8_t* sK = smem + NS * Q_STAGE;
   uint8_t* sV = sK + KS * KV_SLAB;
   __shared__ uint64_t q_full[NS], q_empty[NS], kv_empty, s_full[2], s_empty[2], p_ready[2], o_full[2], o_empty[2];
+  __shared__ __align__(16) int s_rowidx[kMetaRing][128];  // accumulator row (t*Hq + head) of every tile row, -1 = none
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_fail;
   __shared__ int s_ent[kMetaRing][128];   // per-tile entries, written by the producers, read by all roles
@@ -512,7 +518,7 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
-    for (int i = 0; i < NS; ++i) { mbar_init(&q_full[i], kProdThreads); mbar_init(&q_empty[i], 128); }
+    for (int i = 0; i < NS; ++i) { mbar_init(&q_full[i], kProdThreads); mbar_init(&q_empty[i], kTransO ? 1 : 128); }
     mbar_init(&kv_empty, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 128); mbar_init(&p_ready[i], 128);
@@ -574,6 +580,7 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
     // waits for the other.  Lane 0 probes and issues; the warp stays converged on its decisions.
     const uint32_t idesc_s = make_idesc_bf16(128, C, 0, 0);
     const uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
+    const uint32_t idesc_ot = make_idesc_bf16(128, 128, 1, 0);   // O^T: M = d (V, MN-major), N = tile rows (P)
     int s_it = 0, pv_it = 0;              // next tile whose S / whose P V is to be issued
     unsigned last_bits = 0;               // bit (it & 31): tile `it` closes its work item
     int item = blockIdx.x, jt = 0;
@@ -607,11 +614,13 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
           const uint32_t p0 = smem_u32(sQ + ps * Q_STAGE), v0 = smem_u32(sV);
 #pragma unroll
           for (int kk = 0; kk < C / 16; ++kk) {
-            const uint64_t da = make_smem_desc(p0 + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
-            const uint64_t db = make_smem_desc(v0 + kk * (16 * 128), KV_SLAB, 1024);
-            umma_bf16(tmem + 256u + (uint32_t)(pb * 128), da, db, idesc_o, kk > 0);
+            const uint64_t dp = make_smem_desc(p0 + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
+            const uint64_t dv = make_smem_desc(v0 + kk * (16 * 128), KV_SLAB, 1024);
+            if (kTransO) umma_bf16(tmem + 256u + (uint32_t)(pb * 128), dv, dp, idesc_ot, kk > 0);
+            else umma_bf16(tmem + 256u + (uint32_t)(pb * 128), dp, dv, idesc_o, kk > 0);
           }
           umma_commit(&o_full[pb]);
+          if (kTransO) umma_commit(&q_empty[ps]);     // P has been consumed: the ring slot is free
           if ((last_bits >> (pv_it & 31)) & 1u) umma_commit(&kv_empty);   // K/V of that item are free
         }
         ++pv_it;
@@ -739,6 +748,58 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
         const uint32_t o_base = tmem + lane_sel + 256u + (uint32_t)(ob * 128);
         if (!mbar_wait_bounded(&o_full[ob], (uint32_t)((it >> 1) & 1))) { s_fail = 1; break; }
         tcgen05_fence_after_sync();
+        if (kTransO) {
+          // lane = output column d (= `row` of this thread), TMEM column = tile row = entry*G + head
+          const int* ents = s_ent[it % kMetaRing];
+          float* acc_d = a.o_acc + (((long long)b * geo.N) * geo.Hkv + h) * (long long)(D * G) + (long long)row * G;
+          const long long tok_stride = (long long)geo.Hkv * D * G;
+          uint32_t ra[32], rb[32];
+          tmem_ld_32x32(o_base, ra);
+#pragma unroll
+          for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t (&cur)[32] = ((c0 >> 5) & 1) ? rb : ra;
+            uint32_t (&nxt)[32] = ((c0 >> 5) & 1) ? ra : rb;
+            tmem_ld_wait();
+            if (c0 + 32 < 128) {
+              tmem_ld_32x32(o_base + (uint32_t)(c0 + 32), nxt);
+            } else {
+              tcgen05_fence_before_sync();
+              mbar_arrive(&o_empty[ob]);          // O has been read out of TMEM
+            }
+            if (G >= 4) {
+#pragma unroll
+              for (int q4 = 0; q4 < 8; ++q4) {
+                const int col = c0 + 4 * q4;
+                const int ent_c = ents[col >> lgG];
+                if (ent_c >= 0) {
+                  float* dst = acc_d + (long long)(ent_c & 0xFFFFFF) * tok_stride + (col & (G - 1));
+                  asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst),
+                               "f"(__uint_as_float(cur[4 * q4])), "f"(__uint_as_float(cur[4 * q4 + 1])),
+                               "f"(__uint_as_float(cur[4 * q4 + 2])), "f"(__uint_as_float(cur[4 * q4 + 3]))
+                               : "memory");
+                }
+              }
+            } else if (G == 2) {
+#pragma unroll
+              for (int q2 = 0; q2 < 16; ++q2) {
+                const int ent_c = ents[(c0 + 2 * q2) >> 1];
+                if (ent_c >= 0) {
+                  float* dst = acc_d + (long long)(ent_c & 0xFFFFFF) * tok_stride;
+                  asm volatile("red.relaxed.gpu.global.add.v2.f32 [%0], {%1, %2};" ::"l"(dst),
+                               "f"(__uint_as_float(cur[2 * q2])), "f"(__uint_as_float(cur[2 * q2 + 1]))
+                               : "memory");
+                }
+              }
+            } else {
+#pragma unroll
+              for (int q1 = 0; q1 < 32; ++q1) {
+                const int ent_c = ents[c0 + q1];
+                if (ent_c >= 0) atomicAdd(acc_d + (long long)(ent_c & 0xFFFFFF) * tok_stride, __uint_as_float(cur[q1]));
+              }
+            }
+          }
+          continue;
+        }
 #pragma unroll
         for (int half = 0; half < KS; ++half) {
           uint32_t ra[32], rb[32];
@@ -908,7 +969,7 @@ __global__ void __launch_bounds__(256) row_lse_kernel(Geometry geo, const int32_
   lse_out[((long long)b * geo.Hq + h * geo.G + head) * geo.N + t] = (ssum > 0.f) ? m + logf(ssum) : -CUDART_INF_F;
 }
 
-// fp32 accumulator [B,N,Hq,D] -> out in bf16 (strided)
+// fp32 accumulator [B,N,Hq,d] -> out in bf16 (strided)
 __global__ void __launch_bounds__(256) convert_out_kernel(Geometry geo, const float* __restrict__ acc,
                                                            __nv_bfloat16* __restrict__ out) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;     // one 8-element chunk
@@ -928,6 +989,28 @@ __global__ void __launch_bounds__(256) convert_out_kernel(Geometry geo, const fl
   o.x = *reinterpret_cast<uint32_t*>(&p0); o.y = *reinterpret_cast<uint32_t*>(&p1);
   o.z = *reinterpret_cast<uint32_t*>(&p2); o.w = *reinterpret_cast<uint32_t*>(&p3);
   *reinterpret_cast<uint4*>(out + (long long)b * geo.os[0] + (long long)t * geo.os[1] + (long long)hq * geo.os[2] + ck * 8) = o;
+}
+
+// fp32 accumulator [B,N,Hkv,d,G] (heads innermost, the transposed-product layout) -> out in bf16.
+// One thread takes two consecutive d of one (b, t, KV head): 2*G contiguous floats in, one bf16x2 per
+// head out; a warp reads 64*G contiguous floats and writes 128 contiguous bytes per head row.
+__global__ void __launch_bounds__(256) convert_out_heads_inner_kernel(Geometry geo, const float* __restrict__ acc,
+                                                                       __nv_bfloat16* __restrict__ out) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;     // one pair of d
+  const int pairs = geo.d / 2, G = geo.G;
+  const long long total = (long long)geo.B * geo.N * geo.Hkv * pairs;
+  if (i >= total) return;
+  const int dp = (int)(i % pairs);
+  const long long row = i / pairs;                    // (b*N + t)*Hkv + h
+  const int h = (int)(row % geo.Hkv);
+  const long long bt = row / geo.Hkv;
+  const int t = (int)(bt % geo.N), b = (int)(bt / geo.N);
+  const float* src = acc + (row * geo.d + dp * 2) * G;
+  __nv_bfloat16* dst = out + (long long)b * geo.os[0] + (long long)t * geo.os[1] + (long long)(h * G) * geo.os[2] + dp * 2;
+  for (int hd = 0; hd < G; ++hd) {
+    const __nv_bfloat162 p = __floats2bfloat162_rn(src[hd], src[G + hd]);
+    *reinterpret_cast<__nv_bfloat162*>(dst + (long long)hd * geo.os[2]) = p;
+  }
 }
 
 // ------------------------------------------------------------------ host side
@@ -1138,8 +1221,13 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
   st = dispatch_tile_pv(g, a, s);
   if (st != PISA_OK) return st;
   kernel_mark("convert_out", s);
-  const long long chunks = (long long)g.B * g.N * g.Hq * (g.d / 8);
-  convert_out_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, s>>>(g, acc, (__nv_bfloat16*)out);
+  if (g.d == 128) {
+    const long long n = (long long)g.B * g.N * g.Hkv * (g.d / 2);
+    convert_out_heads_inner_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(g, acc, (__nv_bfloat16*)out);
+  } else {
+    const long long n = (long long)g.B * g.N * g.Hq * (g.d / 8);
+    convert_out_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(g, acc, (__nv_bfloat16*)out);
+  }
   return check_launch("convert_out");
 }
 
