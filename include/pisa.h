@@ -141,10 +141,16 @@ int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const voi
                  int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes, void* stream);
 
 /*
- * The same forward pass for callers that hold HOST tensors: copies q, k, v to the device arena
- * (`ws`, sized for PISA_OP_FORWARD_HOST), runs pisa_forward there, copies out, lse and (if not
- * NULL) idx back to host memory, and waits for the stream.  Host buffers should be pinned for
- * full copy bandwidth; strides must be dense.  This is the one entry point that synchronises.
+ * The same forward pass for callers that hold HOST tensors.  KV heads are independent units of the
+ * path (Sec. 3.3: one selected set per KV head), so the call walks them one at a time: the strided
+ * slice of q, k, v that belongs to head h is copied into one of two slots of the device arena
+ * (`ws`, sized for PISA_OP_FORWARD_HOST: two slots of per-head tensors, one per-head pyramid and
+ * one per-head forward workspace), pisa_forward runs on it, and out, lse and (if not NULL) idx of
+ * that head are copied back into their places in the host tensors.  The copies run on two internal
+ * streams, so the upload of head h+1 and the download of head h-1 overlap the kernels of head h.
+ * Host buffers should be pinned (pageable memory makes the copies synchronous); strides must be
+ * dense.  Work already queued on `stream` is ordered before the call; the call returns after
+ * everything it queued has finished.  This is the one entry point that synchronises.
  */
 int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_host, const void* v_host,
                       void* out_host, float* lse_host, int32_t* idx_host,

@@ -129,6 +129,36 @@ static size_t bsa_ws_bytes(const pisa_params_t* p, const Geometry& g) {
   return b;
 }
 
+// Device arena of pisa_forward_host.  The call walks the KV heads one at a time (they are independent
+// units of the path): unit u's tensors live in slot u % 2 so that the host->device copy of the next
+// unit and the device->host copy of the previous one overlap the kernels of the current one.
+struct HostArena {
+  pisa_params_t unit;          // the per-unit problem: Hkv = 1, Hq = G, dense strides
+  Geometry ug;
+  size_t fwd, qb, kb, lb, ib, pb;   // bytes: forward workspace, q/out, k/v, lse, idx, pyramid (one unit)
+  size_t slot, total;
+};
+static int host_arena(const pisa_params_t* p, HostArena* a) {
+  a->unit = *p;
+  a->unit.Hq = p->Hq / p->Hkv;
+  a->unit.Hkv = 1;
+  for (int i = 0; i < 3; ++i) a->unit.q_stride[i] = a->unit.k_stride[i] = a->unit.v_stride[i] = a->unit.o_stride[i] = 0;
+  int st = resolve(&a->unit, &a->ug);
+  if (st != PISA_OK) return st;
+  const Geometry& g = a->ug;
+  const size_t es = elem_size(p->dtype);
+  const size_t r = route_ws_bytes(&a->unit, g), b = bsa_ws_bytes(&a->unit, g);
+  a->fwd = align_up(r > b ? r : b, 256);
+  a->qb = align_up((size_t)g.B * g.N * g.Hq * g.d * es, 256);
+  a->kb = align_up((size_t)g.B * g.N * g.d * es, 256);
+  a->lb = align_up((size_t)g.B * g.Hq * g.N * sizeof(float), 256);
+  a->ib = align_up((size_t)g.B * g.N * g.K * sizeof(int32_t), 256);
+  a->pb = align_up(pyramid_bytes_dtype(g, p->dtype), 256);
+  a->slot = 2 * a->qb + 2 * a->kb + a->lb + a->ib;
+  a->total = a->fwd + a->pb + 2 * a->slot;
+  return PISA_OK;
+}
+
 static int clear_status(void* ws, cudaStream_t s) {
   cudaError_t e = cudaMemsetAsync(ws, 0, kStatusBytes, s);
   if (e != cudaSuccess) { record_cuda_error("status memset", e); return PISA_ERR_CUDA; }
@@ -165,12 +195,12 @@ static void stage_mark(int i, cudaStream_t s) {
 
 static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v,
                       void* pyr, int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes,
-                      cudaStream_t s) {
+                      cudaStream_t s, bool clear = true) {
   size_t need = route_ws_bytes(p, g);
   const size_t need_b = bsa_ws_bytes(p, g);
   if (need_b > need) need = need_b;
   if (ws_bytes < need) return PISA_ERR_WORKSPACE_TOO_SMALL;
-  int st = clear_status(ws, s);
+  int st = clear ? clear_status(ws, s) : PISA_OK;
   if (st != PISA_OK) return st;
   g_mark_n = 0;
   stage_mark(0, s);
@@ -232,7 +262,6 @@ int pisa_workspace_bytes(const pisa_params_t* p, int op, size_t* bytes) {
   int st = resolve(p, &g);
   if (st != PISA_OK) return st;
   if (bytes == nullptr) return PISA_ERR_INVALID_ARG;
-  const size_t es = elem_size(p->dtype);
   const size_t r = route_ws_bytes(p, g), a = bsa_ws_bytes(p, g);
   const size_t f = r > a ? r : a;
   switch (op) {
@@ -241,13 +270,10 @@ int pisa_workspace_bytes(const pisa_params_t* p, int op, size_t* bytes) {
     case PISA_OP_FORWARD: *bytes = f; break;
     case PISA_OP_FLAT: *bytes = kStatusBytes; break;
     case PISA_OP_FORWARD_HOST: {
-      size_t t = align_up(f, 256);
-      t += align_up((size_t)g.B * g.N * g.Hq * g.d * es, 256) * 2;      // q, out
-      t += align_up((size_t)g.B * g.N * g.Hkv * g.d * es, 256) * 2;     // k, v
-      t += align_up((size_t)g.B * g.Hq * g.N * sizeof(float), 256);      // lse
-      t += align_up((size_t)g.B * g.Hkv * g.N * g.K * sizeof(int32_t), 256);  // idx
-      t += align_up(pyramid_bytes_dtype(g, p->dtype), 256);
-      *bytes = t;
+      HostArena a;
+      st = host_arena(p, &a);
+      if (st != PISA_OK) return st;
+      *bytes = a.total;
       break;
     }
     default: return PISA_ERR_INVALID_ARG;
@@ -309,43 +335,87 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
   if (!q_host || !k_host || !v_host || !out_host || !lse_host || !ws || misaligned(ws)) return PISA_ERR_INVALID_ARG;
   for (int i = 0; i < 3; ++i)
     if (p->q_stride[i] || p->k_stride[i] || p->v_stride[i] || p->o_stride[i]) return PISA_ERR_INVALID_ARG;
-  size_t need = 0;
-  st = pisa_workspace_bytes(p, PISA_OP_FORWARD_HOST, &need);
+  HostArena A;
+  st = host_arena(p, &A);
   if (st != PISA_OK) return st;
-  if (ws_bytes < need) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  if (ws_bytes < A.total) return PISA_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t s = (cudaStream_t)stream;
   const size_t es = elem_size(p->dtype);
-  size_t fwd = 0;
-  pisa_workspace_bytes(p, PISA_OP_FORWARD, &fwd);
-  const size_t qb = (size_t)g.B * g.N * g.Hq * g.d * es, kb = (size_t)g.B * g.N * g.Hkv * g.d * es;
-  const size_t lb = (size_t)g.B * g.Hq * g.N * sizeof(float);
-  const size_t ib = (size_t)g.B * g.Hkv * g.N * g.K * sizeof(int32_t);
   char* base = (char*)ws;
-  size_t off = align_up(fwd, 256);
-  char* dq = base + off; off += align_up(qb, 256);
-  char* dout = base + off; off += align_up(qb, 256);
-  char* dk = base + off; off += align_up(kb, 256);
-  char* dv = base + off; off += align_up(kb, 256);
-  char* dl = base + off; off += align_up(lb, 256);
-  char* di = base + off; off += align_up(ib, 256);
-  char* dp = base + off;
-  cudaError_t e;
-  if ((e = cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, s)) != cudaSuccess) {
-    record_cuda_error("h2d copy", e);
-    return PISA_ERR_CUDA;
+  char* dpyr = base + A.fwd;
+  char* slot0 = dpyr + A.pb;
+  const int U = g.Hkv, G = g.G;
+  const size_t rows = (size_t)g.B * g.N;                         // tokens of all batches
+  const size_t q_w = (size_t)G * g.d * es, q_pitch = (size_t)g.Hq * g.d * es;
+  const size_t k_w = (size_t)g.d * es, k_pitch = (size_t)g.Hkv * g.d * es;
+  const size_t l_w = (size_t)G * g.N * sizeof(float), l_pitch = (size_t)g.Hq * g.N * sizeof(float);
+  const size_t i_w = (size_t)g.N * g.K * sizeof(int32_t), i_pitch = (size_t)g.Hkv * i_w;
+
+  // copy streams and the events that order the three stages of every unit
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  cudaEvent_t ev_begin = nullptr, ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr},
+              ev_out[2] = {nullptr, nullptr};
+  cudaError_t e = cudaSuccess;
+  const char* what = "copy streams";
+  auto ok = [&](cudaError_t r, const char* w) { if (e == cudaSuccess && r != cudaSuccess) { e = r; what = w; } return e == cudaSuccess; };
+  ok(cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking), "stream create");
+  ok(cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking), "stream create");
+  ok(cudaEventCreateWithFlags(&ev_begin, cudaEventDisableTiming), "event create");
+  for (int i = 0; i < 2; ++i) {
+    ok(cudaEventCreateWithFlags(&ev_in[i], cudaEventDisableTiming), "event create");
+    ok(cudaEventCreateWithFlags(&ev_done[i], cudaEventDisableTiming), "event create");
+    ok(cudaEventCreateWithFlags(&ev_out[i], cudaEventDisableTiming), "event create");
   }
-  st = do_forward(p, g, dq, dk, dv, dp, (int32_t*)di, dout, (float*)dl, ws, fwd, s);
-  if (st != PISA_OK) return st;
-  if ((e = cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, s)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(lse_host, dl, lb, cudaMemcpyDeviceToHost, s)) != cudaSuccess ||
-      (idx_host && (e = cudaMemcpyAsync(idx_host, di, ib, cudaMemcpyDeviceToHost, s)) != cudaSuccess) ||
-      (e = cudaStreamSynchronize(s)) != cudaSuccess) {
-    record_cuda_error("d2h copy", e);
-    return PISA_ERR_CUDA;
+  // work already queued on the caller's stream comes first
+  if (e == cudaSuccess) {
+    ok(cudaEventRecord(ev_begin, s), "event record");
+    ok(cudaStreamWaitEvent(s_in, ev_begin, 0), "stream wait");
+    ok(cudaStreamWaitEvent(s_out, ev_begin, 0), "stream wait");
   }
-  return PISA_OK;
+  st = (e == cudaSuccess) ? clear_status(ws, s) : PISA_OK;
+  for (int u = 0; u < U && e == cudaSuccess && st == PISA_OK; ++u) {
+    const int sl = u & 1;
+    char* dq = slot0 + sl * A.slot;
+    char* dout = dq + A.qb;
+    char* dk = dout + A.qb;
+    char* dv = dk + A.kb;
+    char* dl = dv + A.kb;
+    char* di = dl + A.lb;
+    // stage 1: inputs of unit u (its slot was last read by the kernels of unit u-2)
+    if (u >= 2) ok(cudaStreamWaitEvent(s_in, ev_done[sl], 0), "stream wait");
+    ok(cudaMemcpy2DAsync(dq, q_w, (const char*)q_host + (size_t)u * q_w, q_pitch, q_w, rows, cudaMemcpyHostToDevice, s_in), "h2d copy");
+    ok(cudaMemcpy2DAsync(dk, k_w, (const char*)k_host + (size_t)u * k_w, k_pitch, k_w, rows, cudaMemcpyHostToDevice, s_in), "h2d copy");
+    ok(cudaMemcpy2DAsync(dv, k_w, (const char*)v_host + (size_t)u * k_w, k_pitch, k_w, rows, cudaMemcpyHostToDevice, s_in), "h2d copy");
+    ok(cudaEventRecord(ev_in[sl], s_in), "event record");
+    // stage 2: the kernels (the slot's outputs were last read by the copies of unit u-2)
+    ok(cudaStreamWaitEvent(s, ev_in[sl], 0), "stream wait");
+    if (u >= 2) ok(cudaStreamWaitEvent(s, ev_out[sl], 0), "stream wait");
+    if (e != cudaSuccess) break;
+    st = do_forward(&A.unit, A.ug, dq, dk, dv, dpyr, (int32_t*)di, dout, (float*)dl, ws, A.fwd, s, /*clear=*/false);
+    if (st != PISA_OK) break;
+    ok(cudaEventRecord(ev_done[sl], s), "event record");
+    // stage 3: results of unit u
+    ok(cudaStreamWaitEvent(s_out, ev_done[sl], 0), "stream wait");
+    ok(cudaMemcpy2DAsync((char*)out_host + (size_t)u * q_w, q_pitch, dout, q_w, q_w, rows, cudaMemcpyDeviceToHost, s_out), "d2h copy");
+    ok(cudaMemcpy2DAsync((char*)lse_host + (size_t)u * l_w, l_pitch, dl, l_w, l_w, (size_t)g.B, cudaMemcpyDeviceToHost, s_out), "d2h copy");
+    if (idx_host)
+      ok(cudaMemcpy2DAsync((char*)idx_host + (size_t)u * i_w, i_pitch, di, i_w, i_w, (size_t)g.B, cudaMemcpyDeviceToHost, s_out), "d2h copy");
+    ok(cudaEventRecord(ev_out[sl], s_out), "event record");
+  }
+  // everything this call queued must be finished before its streams and events go away
+  if (s_in) ok(cudaStreamSynchronize(s_in), "stream sync");
+  ok(cudaStreamSynchronize(s), "stream sync");
+  if (s_out) ok(cudaStreamSynchronize(s_out), "stream sync");
+  for (int i = 0; i < 2; ++i) {
+    if (ev_in[i]) cudaEventDestroy(ev_in[i]);
+    if (ev_done[i]) cudaEventDestroy(ev_done[i]);
+    if (ev_out[i]) cudaEventDestroy(ev_out[i]);
+  }
+  if (ev_begin) cudaEventDestroy(ev_begin);
+  if (s_in) cudaStreamDestroy(s_in);
+  if (s_out) cudaStreamDestroy(s_out);
+  if (e != cudaSuccess) { record_cuda_error(what, e); return PISA_ERR_CUDA; }
+  return st;
 }
 
 int pisa_flat_select(const pisa_params_t* p, const void* q, const void* pyramid, int32_t* idx, void* ws,
