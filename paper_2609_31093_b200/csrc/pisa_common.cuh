@@ -91,4 +91,56 @@ __device__ inline float warp_sum(float v) {
   return v;
 }
 
+// ---------------------------------------------------------------- Select_K ranks (Algorithm 1)
+//
+// Forced candidates are never scored: they take distinct scores above every real one, ordered by
+// position, so that they rank first.  A real score never comes near kForcedFloor.
+constexpr float kForcedFloor = 1.0e38f;
+__device__ __forceinline__ float forced_score(int pos) { return 3.0e38f - (float)pos * 1.0e34f; }
+
+// Rank of each candidate under (score descending, position ascending), for the candidates
+// s = lane + 32*k this lane owns.  `u` is the warp's score array in shared memory, 16-byte aligned,
+// n <= kMaxCand scores followed by -inf up to the next multiple of four.  The common case, all
+// scores distinct, only counts the strictly larger ones (four per 16-byte load); whether a tie
+// exists shows in the sum of the counts (every unordered pair of distinct scores is counted exactly
+// once), and only then the exact order with positions is evaluated.
+__device__ __forceinline__ void warp_select_ranks(const float* u, int n, int lane, int (&rank)[kMaxCand / 32]) {
+  constexpr int SLOTS = kMaxCand / 32;
+  float ui[SLOTS];
+#pragma unroll
+  for (int k = 0; k < SLOTS; ++k) {
+    const int s = lane + 32 * k;
+    ui[k] = (s < n) ? u[s] : 0.f;
+    rank[k] = 0;
+  }
+  const float4* u4 = reinterpret_cast<const float4*>(u);
+  const int n4 = (n + 3) >> 2;
+  for (int j4 = 0; j4 < n4; ++j4) {
+    const float4 v = u4[j4];
+#pragma unroll
+    for (int k = 0; k < SLOTS; ++k)
+      if (32 * k < n) rank[k] += (int)(v.x > ui[k]) + (int)(v.y > ui[k]) + (int)(v.z > ui[k]) + (int)(v.w > ui[k]);
+  }
+  int tot = 0;
+#pragma unroll
+  for (int k = 0; k < SLOTS; ++k)
+    if (lane + 32 * k < n) tot += rank[k];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+  if (tot != n * (n - 1) / 2) {
+#pragma unroll
+    for (int k = 0; k < SLOTS; ++k) {
+      const int s = lane + 32 * k;
+      if (s < n) {
+        int r = 0;
+        for (int j = 0; j < n; ++j) {
+          const float uj = u[j];
+          r += (uj > ui[k]) || (uj == ui[k] && j < s);
+        }
+        rank[k] = r;
+      }
+    }
+  }
+}
+
 }  // namespace pisa

@@ -39,7 +39,7 @@ __device__ __forceinline__ void lse_add(float& m, float& s, float z) {
 
 }  // namespace
 
-template <int D, int NT>
+template <int D, int NT, bool G2>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ pyr,
                         int32_t* __restrict__ par_out, float* __restrict__ margin) {
@@ -101,16 +101,15 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
         const int kap = k0 + gid;
         const bool has = kap < nV;
         const int node = has ? cand[kap] : 0;
-        float m[NT][2], ssum[NT][2];
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) { m[nt][0] = m[nt][1] = -CUDART_INF_F; ssum[nt][0] = ssum[nt][1] = 0.f; }
-        for (int r0 = 0; r0 < g; r0 += 2) {
-          const int ch_lo = node * g + r0, ch_hi = ch_lo + 1;
-          const bool ok_lo = has && ch_lo < Mb, ok_hi = has && (r0 + 1 < g) && ch_hi < Mb;
+        float usum = 0.f;
+        if (G2) {
+          // fan-in 2: both children of a candidate meet in one lane; LSE(a, b) = max + log(1 + e^-|a-b|)
+          const int ch_lo = node * 2, ch_hi = ch_lo + 1;
+          const bool ok_hi = has && ch_hi < Mb;
           uint4 lo[C4], hi[C4];
 #pragma unroll
           for (int c4 = 0; c4 < C4; ++c4) {
-            lo[c4] = ok_lo ? ldg128(below + (long long)ch_lo * D + (c4 * 4 + tig) * 8) : make_uint4(0u, 0u, 0u, 0u);
+            lo[c4] = has ? ldg128(below + (long long)ch_lo * D + (c4 * 4 + tig) * 8) : make_uint4(0u, 0u, 0u, 0u);
             hi[c4] = ok_hi ? ldg128(below + (long long)ch_hi * D + (c4 * 4 + tig) * 8) : make_uint4(0u, 0u, 0u, 0u);
           }
 #pragma unroll
@@ -121,41 +120,70 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
               mma_bf16_16816(acc, lo[c4].x, hi[c4].x, lo[c4].y, hi[c4].y, bq[nt][c4][0], bq[nt][c4][1]);
               mma_bf16_16816(acc, lo[c4].z, hi[c4].z, lo[c4].w, hi[c4].w, bq[nt][c4][2], bq[nt][c4][3]);
             }
-            // acc[0..1]: child lo, heads nt*8 + 2*tig + {0,1};  acc[2..3]: child hi, same heads
 #pragma unroll
             for (int jh = 0; jh < 2; ++jh) {
-              if (ok_lo) lse_add(m[nt][jh], ssum[nt][jh], acc[jh] * geo.scale);
-              if (ok_hi) lse_add(m[nt][jh], ssum[nt][jh], acc[2 + jh] * geo.scale);
+              const float za = acc[jh] * geo.scale, zb = acc[2 + jh] * geo.scale;
+              const float lse2 = fmaxf(za, zb) + __logf(1.f + __expf(-fabsf(za - zb)));
+              if (nt * 8 + 2 * tig + jh < G) usum += ok_hi ? lse2 : za;
             }
           }
+          if (!has) usum = 0.f;
+        } else {
+          float m[NT][2], ssum[NT][2];
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) { m[nt][0] = m[nt][1] = -CUDART_INF_F; ssum[nt][0] = ssum[nt][1] = 0.f; }
+          for (int r0 = 0; r0 < g; r0 += 2) {
+            const int ch_lo = node * g + r0, ch_hi = ch_lo + 1;
+            const bool ok_lo = has && ch_lo < Mb, ok_hi = has && (r0 + 1 < g) && ch_hi < Mb;
+            uint4 lo[C4], hi[C4];
+#pragma unroll
+            for (int c4 = 0; c4 < C4; ++c4) {
+              lo[c4] = ok_lo ? ldg128(below + (long long)ch_lo * D + (c4 * 4 + tig) * 8) : make_uint4(0u, 0u, 0u, 0u);
+              hi[c4] = ok_hi ? ldg128(below + (long long)ch_hi * D + (c4 * 4 + tig) * 8) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+              for (int c4 = 0; c4 < C4; ++c4) {
+                mma_bf16_16816(acc, lo[c4].x, hi[c4].x, lo[c4].y, hi[c4].y, bq[nt][c4][0], bq[nt][c4][1]);
+                mma_bf16_16816(acc, lo[c4].z, hi[c4].z, lo[c4].w, hi[c4].w, bq[nt][c4][2], bq[nt][c4][3]);
+              }
+              // acc[0..1]: child lo, heads nt*8 + 2*tig + {0,1};  acc[2..3]: child hi, same heads
+#pragma unroll
+              for (int jh = 0; jh < 2; ++jh) {
+                if (ok_lo) lse_add(m[nt][jh], ssum[nt][jh], acc[jh] * geo.scale);
+                if (ok_hi) lse_add(m[nt][jh], ssum[nt][jh], acc[2 + jh] * geo.scale);
+              }
+            }
+          }
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int jh = 0; jh < 2; ++jh)
+              if (nt * 8 + 2 * tig + jh < G && has) usum += m[nt][jh] + __logf(ssum[nt][jh]);
         }
-        float usum = 0.f;
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-          for (int jh = 0; jh < 2; ++jh)
-            if (nt * 8 + 2 * tig + jh < G && has) usum += m[nt][jh] + __logf(ssum[nt][jh]);
         usum += __shfl_xor_sync(0xffffffffu, usum, 1);
         usum += __shfl_xor_sync(0xffffffffu, usum, 2);
-        if (has && tig == 0) u[kap] = (node == 0 || node == f1 || node == anc_c) ? CUDART_INF_F : usum;
+        if (has && tig == 0) u[kap] = (node == 0 || node == f1 || node == anc_c) ? forced_score(kap) : usum;
       }
+      if (lane < 4 && nV + lane < kMaxCand) u[nV + lane] = -CUDART_INF_F;     // padding read by the 16-byte loads
       __syncwarp();
     }
     // Select_K: rank by (score desc, position asc); keep rank < K.  Without pruning keep all.
+    int rank[kMaxCand / 32];
+    if (prune) warp_select_ranks(u, nV, lane, rank);
     int base = 0;
-    for (int s0 = 0; s0 < nV; s0 += 32) {
+#pragma unroll
+    for (int ch = 0; ch < kMaxCand / 32; ++ch) {
+      const int s0 = ch * 32;
+      if (s0 >= nV) break;
       const int s = s0 + lane;
       bool keep = s < nV;
       if (prune) {
-        int rank = 0;
-        const float ui = (s < nV) ? u[s] : 0.f;
-        for (int j = 0; j < nV; ++j) {
-          const float uj = u[j];
-          rank += (uj > ui) || (uj == ui && j < s);
-        }
-        keep = keep && (rank < K);
-        if (s < nV && rank == K - 1) s_cut[warp][0] = ui;
-        if (s < nV && rank == K) s_cut[warp][1] = ui;
+        keep = keep && (rank[ch] < K);
+        if (s < nV && rank[ch] == K - 1) s_cut[warp][0] = u[s];
+        if (s < nV && rank[ch] == K) s_cut[warp][1] = u[s];
       }
       const unsigned bal = __ballot_sync(0xffffffffu, keep);
       const int pos = base + __popc(bal & ((1u << lane) - 1u));
@@ -172,7 +200,7 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
     __syncwarp();
     if (prune) {
       const float a = s_cut[warp][0], bb = s_cut[warp][1];
-      if (a < CUDART_INF_F) min_gap = fminf(min_gap, (a - bb) / fmaxf(fabsf(a), 1.f));
+      if (a < kForcedFloor) min_gap = fminf(min_gap, (a - bb) / fmaxf(fabsf(a), 1.f));
     }
     if (l == 2) {
       for (int s = base + lane; s < K; s += 32) par_out[w * (long long)K + s] = -1;
@@ -189,8 +217,12 @@ static int launch_dn(const Geometry& g, const void* q, const void* pyr, int32_t*
   const long long total = (long long)g.B * g.Hkv * g.N;
   const long long ctas = (total + kWarpsPerCta - 1) / kWarpsPerCta;
   if (ctas > 0x7fffffffLL) return PISA_ERR_UNSUPPORTED;
-  route_stage1_mma_kernel<D, NT><<<(unsigned)ctas, kWarpsPerCta * 32, 0, s>>>(
-      g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pyr, par, margin);
+  if (g.g == 2)
+    route_stage1_mma_kernel<D, NT, true><<<(unsigned)ctas, kWarpsPerCta * 32, 0, s>>>(
+        g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pyr, par, margin);
+  else
+    route_stage1_mma_kernel<D, NT, false><<<(unsigned)ctas, kWarpsPerCta * 32, 0, s>>>(
+        g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pyr, par, margin);
   return check_launch("route_stage1_mma");
 }
 

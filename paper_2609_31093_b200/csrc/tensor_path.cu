@@ -883,7 +883,7 @@ __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int
       ok = (p >= 0) && (leaf <= c);
       float sc = -CUDART_INF_F;
       if (ok) {
-        if (leaf == 0 || leaf == f1 || leaf == c) sc = CUDART_INF_F;
+        if (leaf == 0 || leaf == f1 || leaf == c) sc = forced_score(ci);
         else {
           sc = 0.f;
           for (int hh = 0; hh < G; ++hh) sc += bl[ci * G + hh];
@@ -894,22 +894,22 @@ __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int
     nV += __popc(__ballot_sync(0xffffffffu, ok));
   }
   __syncwarp();
+  if (lane < 4 && nV + lane < kMaxCand) u[nV + lane] = -CUDART_INF_F;     // padding read by the 16-byte loads
+  __syncwarp();
   const bool prune = nV > K;
+  int rank[kMaxCand / 32];
+  if (prune) warp_select_ranks(u, nV, lane, rank);
   int base = 0;
   unsigned kept_mask[kMaxCand / 32];
-  for (int s0 = 0, ch = 0; s0 < gK; s0 += 32, ++ch) {
+#pragma unroll
+  for (int ch = 0; ch < kMaxCand / 32; ++ch) {
+    const int s0 = ch * 32;
     const int s = s0 + lane;
     bool keep = s < nV;
     if (prune && s0 < nV) {
-      int rank = 0;
-      const float ui = (s < nV) ? u[s] : 0.f;
-      for (int j = 0; j < nV; ++j) {
-        const float uj = u[j];
-        rank += (uj > ui) || (uj == ui && j < s);
-      }
-      keep = keep && (rank < K);
-      if (s < nV && rank == K - 1) s_cut[warp][0] = ui;
-      if (s < nV && rank == K) s_cut[warp][1] = ui;
+      keep = keep && (rank[ch] < K);
+      if (s < nV && rank[ch] == K - 1) s_cut[warp][0] = u[s];
+      if (s < nV && rank[ch] == K) s_cut[warp][1] = u[s];
     }
     const unsigned bal = __ballot_sync(0xffffffffu, keep);
     kept_mask[ch] = bal;
@@ -924,7 +924,7 @@ __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int
     float mg = margin[w];
     if (prune) {
       const float a = s_cut[warp][0], bb = s_cut[warp][1];
-      if (a < CUDART_INF_F) mg = fminf(mg, (a - bb) / fmaxf(fabsf(a), 1.f));
+      if (a < kForcedFloor) mg = fminf(mg, (a - bb) / fmaxf(fabsf(a), 1.f));
     }
     margin[w] = mg;
   }
