@@ -362,12 +362,18 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
 
   if (warp < 4) {
     // ------------------------------------------------ producers
-    int it = 0, kiter = 0, ent_next = -1;
+    int it = 0, kiter = 0;
     bool stop = false;
     for (int item = blockIdx.x; item < n_items && !stop; item += gridDim.x, ++kiter) {
       const ItemInfo inf = item_info(a, item, tpt);
       const int bh = inf.key / (a.NW * a.Mk), j = inf.key % a.Mk;
       const int b = bh / geo.Hkv, h = bh % geo.Hkv;
+      // Entries are fetched two tiles ahead from a clamped (always readable) address and their
+      // validity is decided only when the tile comes up, so that nothing waits on the load.
+      const int e_last = inf.e_end - 1;
+      const int my = (tid < tpt) ? tid : 0;
+      int raw0 = a.entries[min(inf.e_begin + my, e_last)];
+      int raw1 = a.entries[min(inf.e_begin + tpt + my, e_last)];
       // the previous item's MMAs must have released the key tile
       bool bad = s_fail != 0;
       if (!bad && kiter > 0) bad = !mbar_wait_bounded(&b_empty, (uint32_t)((kiter - 1) & 1));
@@ -379,10 +385,9 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
         const int s = it % NS;
         const bool bad_t = it >= NS && !mbar_wait_bounded(&a_empty[s], (uint32_t)((it / NS - 1) & 1));
         const int e0 = inf.e_begin + jt * tpt;
-        // this tile's entries were fetched one tile ahead; fetch the next tile's now
-        const int ent_now = (jt == 0) ? fetch_entry(a.entries, e0, inf.e_end, tpt, tid) : ent_next;
-        ent_next = (jt + 1 < inf.ntiles) ? fetch_entry(a.entries, e0 + tpt, inf.e_end, tpt, tid) : -1;
-        s_ent[it % kMetaRing][tid] = ent_now;
+        const int raw2 = a.entries[min(e0 + 2 * tpt + my, e_last)];
+        s_ent[it % kMetaRing][tid] = (tid < tpt && e0 + tid < inf.e_end) ? raw0 : -1;
+        raw0 = raw1; raw1 = raw2;
         if (prod_sync_or(bad_t)) { s_fail = 1; stop = true; break; }
         prod_gather_q<D>(sA + s * A_STAGE, geo, qb, s_ent[it % kMetaRing], tid);
         fence_proxy_async_smem();                 // zero-filled rows (plain stores) -> async proxy
@@ -462,6 +467,12 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
             else if (c0 < ncols) lse_chunk_masked(ra, ncols - c0, sl2, m, ssum);
             tmem_ld_wait();
             if (c0 + 64 < C) tmem_ld_32x32(col0 + (uint32_t)(c0 + 64), ra);
+            else if (r + 1 == r_hi) {
+              // the last chunk of this warp's share is in registers: the accumulator can be refilled
+              // while it is being reduced
+              tcgen05_fence_before_sync();
+              mbar_arrive(&t_empty[grp]);
+            }
             if (fast) lse_chunk(rb, sl2, m, ssum);
             else if (c0 + 32 < ncols) lse_chunk_masked(rb, ncols - c0 - 32, sl2, m, ssum);
           }
@@ -470,8 +481,10 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
             a.blk_lse[(((long long)bh * geo.N + t) * (a.slots * a.fan) + slot * a.fan + r) * G + head] = lse;
           }
         }
-        tcgen05_fence_before_sync();
-        mbar_arrive(&t_empty[grp]);
+        if (r_lo >= r_hi) {              // a warp without a share of this tile still counts as an arrival
+          tcgen05_fence_before_sync();
+          mbar_arrive(&t_empty[grp]);
+        }
       }
     }
   }
