@@ -309,6 +309,25 @@ __device__ __forceinline__ void prod_gather_q(uint8_t* dst, const Geometry& geo,
     d += RPP * 128;
   }
 }
+// ... the same gather with the tile's entries already in the thread's registers (ent[i] belongs to row
+// rb + i * RPP; -1 = no entry): no shared-memory round trip and no barrier among the producer warps
+template <int D>
+__device__ __forceinline__ void prod_gather_q_regs(uint8_t* dst, const Geometry& geo, const __nv_bfloat16* qb,
+                                                   const int (&ent)[128 / (kProdThreads / (D / 8))], int p) {
+  constexpr int CH = D / 8, RPP = kProdThreads / CH, RPT = 128 / RPP;
+  const int ck = p % CH, rb = p / CH;
+  const int G = geo.G;
+  uint32_t d = smem_u32(dst + (ck >> 3) * (128 * 128)) + swz128(rb, ck & 7);
+  const __nv_bfloat16* src0 = qb + ck * 8;
+  const long long s1 = geo.qs[1], s2 = geo.qs[2];
+#pragma unroll
+  for (int i = 0; i < RPT; ++i) {
+    const int row = rb + i * RPP;
+    if (ent[i] >= 0) cp_async16(d, src0 + (long long)(ent[i] & 0xFFFFFF) * s1 + (long long)(row & (G - 1)) * s2);
+    else st_shared_zero16(d);
+    d += RPP * 128;
+  }
+}
 // barrier among the 128 producer threads that also ORs a flag, so that they leave their loops together
 __device__ __forceinline__ bool prod_sync_or(bool flag) {
   uint32_t any;
@@ -339,8 +358,6 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
   __shared__ uint64_t a_full[NS], a_empty[NS], b_empty, t_full[2], t_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_fail;
-  __shared__ int s_ent[kMetaRing][128];  // per-tile entries, written by the producers, read by all roles
-  __shared__ float s_lse[kMetaRing][128]; // per-row softmax denominators (attention kernel only)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
@@ -362,34 +379,41 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
 
   if (warp < 4) {
     // ------------------------------------------------ producers
+    // The four producer warps run independently of one another: a thread reads the entries of the
+    // rows it copies straight from the list (one tile ahead, from a clamped -- always readable --
+    // address; validity is decided when the tile comes up, so nothing waits on the loads).
+    constexpr int CH = D / 8, RPP = kProdThreads / CH, RPT = 128 / RPP;
+    const int rb = tid / CH;
     int it = 0, kiter = 0;
     bool stop = false;
     for (int item = blockIdx.x; item < n_items && !stop; item += gridDim.x, ++kiter) {
       const ItemInfo inf = item_info(a, item, tpt);
       const int bh = inf.key / (a.NW * a.Mk), j = inf.key % a.Mk;
       const int b = bh / geo.Hkv, h = bh % geo.Hkv;
-      // Entries are fetched two tiles ahead from a clamped (always readable) address and their
-      // validity is decided only when the tile comes up, so that nothing waits on the load.
       const int e_last = inf.e_end - 1;
-      const int my = (tid < tpt) ? tid : 0;
-      int raw0 = a.entries[min(inf.e_begin + my, e_last)];
-      int raw1 = a.entries[min(inf.e_begin + tpt + my, e_last)];
+      int nxt[RPT];
+#pragma unroll
+      for (int i = 0; i < RPT; ++i) nxt[i] = a.entries[min(inf.e_begin + ((rb + i * RPP) >> lgG), e_last)];
       // the previous item's MMAs must have released the key tile
-      bool bad = s_fail != 0;
-      if (!bad && kiter > 0) bad = !mbar_wait_bounded(&b_empty, (uint32_t)((kiter - 1) & 1));
-      if (prod_sync_or(bad)) { s_fail = 1; stop = true; break; }
+      bool ok = s_fail == 0;
+      if (ok && kiter > 0) ok = mbar_wait_bounded(&b_empty, (uint32_t)((kiter - 1) & 1));
+      if (!__all_sync(0xffffffffu, ok)) { s_fail = 1; stop = true; break; }
       prod_load_rows<D>(sB, B_SLAB, a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2], geo.ks[1], j * NB,
                         NB, geo.N, tid);
       const __nv_bfloat16* qb = a.q + (long long)b * geo.qs[0] + (long long)(h * G) * geo.qs[2];
       for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
         const int s = it % NS;
-        const bool bad_t = it >= NS && !mbar_wait_bounded(&a_empty[s], (uint32_t)((it / NS - 1) & 1));
+        ok = it < NS || mbar_wait_bounded(&a_empty[s], (uint32_t)((it / NS - 1) & 1));
+        if (!__all_sync(0xffffffffu, ok)) { s_fail = 1; stop = true; break; }
         const int e0 = inf.e_begin + jt * tpt;
-        const int raw2 = a.entries[min(e0 + 2 * tpt + my, e_last)];
-        s_ent[it % kMetaRing][tid] = (tid < tpt && e0 + tid < inf.e_end) ? raw0 : -1;
-        raw0 = raw1; raw1 = raw2;
-        if (prod_sync_or(bad_t)) { s_fail = 1; stop = true; break; }
-        prod_gather_q<D>(sA + s * A_STAGE, geo, qb, s_ent[it % kMetaRing], tid);
+        int cur[RPT];
+#pragma unroll
+        for (int i = 0; i < RPT; ++i) {
+          const int slot_i = (rb + i * RPP) >> lgG;
+          cur[i] = (e0 + slot_i < inf.e_end) ? nxt[i] : -1;
+          nxt[i] = a.entries[min(e0 + tpt + slot_i, e_last)];
+        }
+        prod_gather_q_regs<D>(sA + s * A_STAGE, geo, qb, cur, tid);
         fence_proxy_async_smem();                 // zero-filled rows (plain stores) -> async proxy
         cp_async_arrive_noinc(&a_full[s]);        // fires when this thread's copies have landed
       }
@@ -444,9 +468,11 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
       const int bh = inf.key / (a.NW * a.Mk), j = inf.key % a.Mk;
       for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
         if ((it & 1) != grp) continue;
+        const int e_row = inf.e_begin + jt * tpt + (row >> lgG);
+        const int ent_raw = a.entries[min(e_row, inf.e_end - 1)];
         if (!mbar_wait_bounded(&t_full[grp], (uint32_t)((it >> 1) & 1))) { s_fail = 1; break; }
         tcgen05_fence_after_sync();
-        const int ent = s_ent[it % kMetaRing][row >> lgG];
+        const int ent = (e_row < inf.e_end) ? ent_raw : -1;
         const bool valid = ent >= 0;
         const int t = ent & 0xFFFFFF, slot = valid ? (ent >> 24) : 0;
         const int c_t = t / C;
