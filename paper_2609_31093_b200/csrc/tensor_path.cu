@@ -174,7 +174,7 @@ struct TileArgs {
   int nkeys, Mk, NW, fan, slots;
   float* blk_lse;          // [BH, N, slots*fan, G]   (tile_lse)
   const float* row_lse;    // [B, Hq, N]              (tile_pv)
-  float* o_acc;            // [B, N, Hq, D] fp32      (tile_pv)
+  float* o_acc;            // fp32 accumulator: [B, Hkv, N, D, G] when the second product is transposed, else [B, N, Hq, D]
   int32_t* status;
 };
 
@@ -541,7 +541,7 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
   constexpr uint32_t TM_COLS = 512;          // S buffers at columns 0 / 128, O buffers at 256 / 384
   // d = 128: the second product is issued transposed, O^T = V^T P^T (A = V, MN-major; B = P): a TMEM lane
   // is then one output column d and consecutive TMEM columns are the G heads of one token.  With the
-  // accumulator laid out [B, N, Hkv, d, G] (heads innermost) a thread adds its G values with one vector
+  // accumulator laid out [B, Hkv, N, d, G] (heads innermost) a thread adds its G values with one vector
   // reduction and a warp covers 32*G consecutive floats: fully coalesced, no staging in shared memory.
   constexpr bool kTransO = (D == 128);
   uint8_t* smem = align1024(smem_raw);
@@ -790,8 +790,8 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
         if (kTransO) {
           // lane = output column d (= `row` of this thread), TMEM column = tile row = entry*G + head
           const int* ents = s_ent[it % kMetaRing];
-          float* acc_d = a.o_acc + (((long long)b * geo.N) * geo.Hkv + h) * (long long)(D * G) + (long long)row * G;
-          const long long tok_stride = (long long)geo.Hkv * D * G;
+          float* acc_d = a.o_acc + (((long long)b * geo.Hkv + h) * geo.N) * (long long)(D * G) + (long long)row * G;
+          const long long tok_stride = (long long)D * G;
           uint32_t ra[32], rb[32];
           tmem_ld_32x32(o_base, ra);
 #pragma unroll
@@ -1030,7 +1030,7 @@ __global__ void __launch_bounds__(256) convert_out_kernel(Geometry geo, const fl
   *reinterpret_cast<uint4*>(out + (long long)b * geo.os[0] + (long long)t * geo.os[1] + (long long)hq * geo.os[2] + ck * 8) = o;
 }
 
-// fp32 accumulator [B,N,Hkv,d,G] (heads innermost, the transposed-product layout) -> out in bf16.
+// fp32 accumulator [B,Hkv,N,d,G] (heads innermost, the transposed-product layout) -> out in bf16.
 // One thread takes two consecutive d of one (b, t, KV head): 2*G contiguous floats in, one bf16x2 per
 // head out; a warp reads 64*G contiguous floats and writes 128 contiguous bytes per head row.
 __global__ void __launch_bounds__(256) convert_out_heads_inner_kernel(Geometry geo, const float* __restrict__ acc,
@@ -1044,7 +1044,7 @@ __global__ void __launch_bounds__(256) convert_out_heads_inner_kernel(Geometry g
   const int h = (int)(row % geo.Hkv);
   const long long bt = row / geo.Hkv;
   const int t = (int)(bt % geo.N), b = (int)(bt / geo.N);
-  const float* src = acc + (row * geo.d + dp * 2) * G;
+  const float* src = acc + ((((long long)b * geo.Hkv + h) * geo.N + t) * geo.d + dp * 2) * G;
   __nv_bfloat16* dst = out + (long long)b * geo.os[0] + (long long)t * geo.os[1] + (long long)(h * G) * geo.os[2] + dp * 2;
   for (int hd = 0; hd < G; ++hd) {
     const __nv_bfloat162 p = __floats2bfloat162_rn(src[hd], src[G + hd]);
