@@ -27,6 +27,12 @@ What follows which passage of the paper:
                          (App. C), Top-K.
 * `score_mode`           Sec. 4.3 / App. A.2: "lse" (PISA), "mean" (PISA-1),
                          "mean_var" (PISA-2).
+* `decode_pyramid`,      Sec. 3.3 "Decoding" and App. B "Decode cache": when the
+  `decode_step`          token at position p is generated the cached pyramid
+                         holds the means of the keys seen so far, i.e. it is the
+                         pyramid of the (p+1)-token sequence; selection walks
+                         all levels down to the raw key blocks for that one
+                         query and attention runs over the selected blocks.
 
 Readings taken where the paper is silent (all 0-based here):
   - summaries are stored in the input dtype (bf16 or fp32, round to nearest
@@ -43,7 +49,11 @@ Taylor identity for the intermediate score, a textbook flat Top-K built from
 torch.logsumexp/topk in the unpruned regime, torch's dense causal attention
 when K*C >= N, a hand-derived pruned example (tests/golden), and structural
 invariants.  The pruned regime has no external numeric anchor beyond the
-hand-derived example and the invariants.
+hand-derived example and the invariants.  Decoding is pinned by what the
+definitions imply: the step at position p selects what the prefill of any
+longer sequence selects for row p (every scored node lies strictly in the past),
+equals torch's dense causal attention when K*C > p, and the cached pyramid's
+completed nodes equal those of the longer sequence's pyramid.
 """
 from __future__ import annotations
 
@@ -404,3 +414,42 @@ class Problem:
                 out[s, j] = o
                 lse[s, j] = l
         return round_to_storage(out, self.dtype), lse
+
+
+# --------------------------------------------------------------------------
+# decoding (Sec. 3.3 "Decoding", App. B "Decode cache")
+# --------------------------------------------------------------------------
+
+def decode_pyramid(k_cache, pos: int, C: int, g: int, dtype: str) -> List[Optional[np.ndarray]]:
+    """The cached pyramid after the token at `pos` has been appended: the mean pyramid of keys
+    0..pos (each summary the mean of its valid children, the last leaf the mean of the keys it
+    holds so far).  k_cache: [B, Ncap, Hkv, d] in storage form; returns levels[l] [B,Hkv,M_l(pos+1),d]."""
+    k = load_storage(np.ascontiguousarray(k_cache[:, :pos + 1]), dtype)
+    return build_pyramid(k, C, g, dtype)
+
+
+def decode_step(q_new, k_cache, v_cache, pos: int, *, C: int, g: int, K: int, dtype: str,
+                scale: Optional[float] = None, mode: str = "lse"):
+    """One decoding step for the token at position `pos` (its key and value already in the caches).
+
+    q_new: [B, Hq, d] storage form; k_cache, v_cache: [B, Ncap, Hkv, d] storage form, rows 0..pos valid.
+    Returns idx int32 [B, Hkv, K] (ascending, -1 padded), margin [B, Hkv], out fp64 [B, Hq, d]
+    (stored values) and lse [B, Hq]."""
+    B, Hq, d = q_new.shape
+    n = pos + 1
+    q_seq = np.zeros((B, n, Hq, d), dtype=q_new.dtype)
+    q_seq[:, pos] = q_new
+    prob = Problem(q_seq, np.ascontiguousarray(k_cache[:, :n]), np.ascontiguousarray(v_cache[:, :n]),
+                   C=C, g=g, K=K, dtype=dtype, scale=scale, mode=mode)
+    idx = np.empty((B, prob.Hkv, K), dtype=np.int32)
+    margin = np.empty((B, prob.Hkv), dtype=np.float64)
+    out = np.empty((B, Hq, d), dtype=np.float64)
+    lse = np.empty((B, Hq), dtype=np.float64)
+    for b in range(B):
+        for h in range(prob.Hkv):
+            I, m = prob.route(b, h, pos)
+            idx[b, h] = pad_indices(I, K)
+            margin[b, h] = m
+            for hq in range(h * prob.G, (h + 1) * prob.G):
+                out[b, hq], lse[b, hq] = prob.attend(b, hq, pos, I)
+    return idx, margin, round_to_storage(out, dtype), lse
