@@ -49,7 +49,8 @@ enum { PISA_BF16 = 0, PISA_FP32 = 1 };
 /* Block score (Sec. 4.3, App. A.2): PISA = log-sum-exp, PISA-1 = mean logit, PISA-2 = mean + var/2 */
 enum { PISA_SCORE_LSE = 0, PISA_SCORE_MEAN = 1, PISA_SCORE_MEAN_VAR = 2 };
 /* operations a workspace can be sized for */
-enum { PISA_OP_ROUTE = 0, PISA_OP_BSA = 1, PISA_OP_FORWARD = 2, PISA_OP_FLAT = 3, PISA_OP_FORWARD_HOST = 4 };
+enum { PISA_OP_ROUTE = 0, PISA_OP_BSA = 1, PISA_OP_FORWARD = 2, PISA_OP_FLAT = 3, PISA_OP_FORWARD_HOST = 4,
+       PISA_OP_DECODE = 5 };
 /* implementation selector (params.impl): AUTO picks the tensor-core path where it applies */
 enum { PISA_IMPL_AUTO = 0, PISA_IMPL_SIMT = 1, PISA_IMPL_TENSOR = 2 };
 
@@ -155,6 +156,46 @@ int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const voi
 int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_host, const void* v_host,
                       void* out_host, float* lse_host, int32_t* idx_host,
                       void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Decoding (Sec. 3.3 "Decoding", App. B "Decode cache"): one new token per sequence, one kernel launch.
+ *
+ *   p->N             : CAPACITY of the caches in tokens (the pyramid layout is that of
+ *                      pisa_pyramid_layout for this N); B, Hq, Hkv, d, C, g, K, scale as usual
+ *   pos              : 0-based position of the new token, pos < p->N
+ *   q                : device [B, Hq, d], dense (q_stride is ignored)
+ *   k_cache, v_cache : device [B, N, Hkv, d] (k_stride / v_stride honoured); rows 0..pos hold the
+ *                      sequence, the new token's key and value already written at row pos; rows
+ *                      after pos are never read
+ *   pyramid          : the cached pyramid, updated in place: the summary of the leaf that holds pos
+ *                      becomes the mean of the keys it holds so far and each of its ancestors the mean
+ *                      of its children up to the path (every other node is left as it is).  Nodes
+ *                      that lie entirely after pos are never read, so the buffer needs no
+ *                      initialisation: a cache built by calling this for pos = 0, 1, 2, ... , or by
+ *                      pisa_build_pyramid over the first tokens followed by steps from there on,
+ *                      holds the pyramid of keys 0..pos after every step
+ *   idx              : device int32 [B, Hkv, K], ascending, -1 padded
+ *   out, lse         : device [B, Hq, d] (input dtype), float [B, Hq]
+ *   ws               : device workspace sized for PISA_OP_DECODE
+ *
+ * The step selects exactly what the prefill path selects for row pos of the same sequence (every
+ * scored node lies strictly in the past of the query) and attends over keys <= pos of the selected
+ * blocks.  bf16, LSE score mode, d in {64, 128}, C in {32, 64, 128}, group size <= 16; other
+ * configurations return PISA_ERR_UNSUPPORTED.  Asynchronous on `stream`; allocates nothing.
+ */
+int pisa_decode_step(const pisa_params_t* p, int32_t pos, const void* q, const void* k_cache,
+                     const void* v_cache, void* pyramid, int32_t* idx, void* out, float* lse,
+                     void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Capacity growth of a cached pyramid (App. B "Decode cache": every level's buffer grows when more
+ * space is needed): copies every level of `pyramid_old` (layout of p_old, capacity p_old->N) into
+ * the layout of p_new (same shape parameters, p_new->N >= p_old->N) in `pyramid_new`.  The two
+ * buffers must not overlap.  Levels that only the larger hierarchy has are rebuilt by the next
+ * decoding steps along the path, as any other ancestor.
+ */
+int pisa_pyramid_regrow(const pisa_params_t* p_old, const pisa_params_t* p_new, const void* pyramid_old,
+                        void* pyramid_new, void* stream);
 
 /*
  * Flat block selection (Sec. 3.1, the O(N^2/C) reference point): score every eligible leaf with

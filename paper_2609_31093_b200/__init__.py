@@ -18,6 +18,8 @@ from .binding import (  # noqa: F401
     pisa_forward,
     pisa_forward_host,
     pisa_flat_select,
+    pisa_decode_step,
+    pisa_pyramid_regrow,
     read_status,
     set_stage_timing,
     get_stage_ms,

@@ -269,6 +269,10 @@ int pisa_workspace_bytes(const pisa_params_t* p, int op, size_t* bytes) {
     case PISA_OP_BSA: *bytes = a; break;
     case PISA_OP_FORWARD: *bytes = f; break;
     case PISA_OP_FLAT: *bytes = kStatusBytes; break;
+    case PISA_OP_DECODE:
+      if (!decode_supported(g, p->dtype)) return PISA_ERR_UNSUPPORTED;
+      *bytes = kStatusBytes + decode_workspace_bytes(g);
+      break;
     case PISA_OP_FORWARD_HOST: {
       HostArena a;
       st = host_arena(p, &a);
@@ -416,6 +420,47 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
   if (s_out) cudaStreamDestroy(s_out);
   if (e != cudaSuccess) { record_cuda_error(what, e); return PISA_ERR_CUDA; }
   return st;
+}
+
+int pisa_decode_step(const pisa_params_t* p, int32_t pos, const void* q, const void* k_cache,
+                     const void* v_cache, void* pyramid, int32_t* idx, void* out, float* lse,
+                     void* ws, size_t ws_bytes, void* stream) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (!q || !k_cache || !v_cache || !pyramid || !idx || !out || !lse || !ws) return PISA_ERR_INVALID_ARG;
+  if (misaligned(q) || misaligned(k_cache) || misaligned(v_cache) || misaligned(pyramid) || misaligned(ws))
+    return PISA_ERR_INVALID_ARG;
+  if (pos < 0 || pos >= g.N) return PISA_ERR_INVALID_ARG;
+  if (!decode_supported(g, p->dtype)) return PISA_ERR_UNSUPPORTED;
+  if (ws_bytes < kStatusBytes + decode_workspace_bytes(g)) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t s = (cudaStream_t)stream;
+  kernel_mark("decode_step", s);
+  st = launch_decode_step(g, pos, q, k_cache, v_cache, pyramid, idx, out, lse, (char*)ws + kStatusBytes, s);
+  kernel_mark("end", s);
+  return st;
+}
+
+int pisa_pyramid_regrow(const pisa_params_t* p_old, const pisa_params_t* p_new, const void* pyramid_old,
+                        void* pyramid_new, void* stream) {
+  Geometry go, gn;
+  int st = resolve(p_old, &go);
+  if (st != PISA_OK) return st;
+  st = resolve(p_new, &gn);
+  if (st != PISA_OK) return st;
+  if (!pyramid_old || !pyramid_new) return PISA_ERR_INVALID_ARG;
+  if (go.B != gn.B || go.Hkv != gn.Hkv || go.d != gn.d || go.C != gn.C || go.g != gn.g ||
+      p_old->dtype != p_new->dtype || gn.N < go.N)
+    return PISA_ERR_INVALID_ARG;
+  const size_t es = elem_size(p_old->dtype);
+  for (int l = 1; l <= go.L; ++l) {
+    const size_t w = (size_t)go.M[l] * go.d * es;           // one (b, KV head) of the old level
+    cudaError_t e = cudaMemcpy2DAsync((char*)pyramid_new + (size_t)gn.level_off[l] * es, (size_t)gn.M[l] * gn.d * es,
+                                      (const char*)pyramid_old + (size_t)go.level_off[l] * es, w, w,
+                                      (size_t)go.B * go.Hkv, cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
+    if (e != cudaSuccess) { record_cuda_error("pyramid regrow", e); return PISA_ERR_CUDA; }
+  }
+  return PISA_OK;
 }
 
 int pisa_flat_select(const pisa_params_t* p, const void* q, const void* pyramid, int32_t* idx, void* ws,

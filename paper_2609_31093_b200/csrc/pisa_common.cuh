@@ -48,6 +48,12 @@ int launch_bsa_simt(const Geometry& g, int dtype, const void* q, const void* k, 
 int launch_flat_simt(const Geometry& g, int dtype, const void* q, const void* pyramid, int32_t* idx,
                      cudaStream_t s);
 
+// decoding step (one token per sequence); ws points past the status word
+bool decode_supported(const Geometry& g, int dtype);
+size_t decode_workspace_bytes(const Geometry& g);
+int launch_decode_step(const Geometry& g, int pos, const void* q, const void* k, const void* v, void* pyramid,
+                       int32_t* idx, void* out, float* lse, void* ws, cudaStream_t s);
+
 // with stage timing on, records an event on `s` named after the kernel(s) that follow it
 void kernel_mark(const char* name, cudaStream_t s);
 int check_launch(const char* what);   // cudaGetLastError -> pisa_status, records the text

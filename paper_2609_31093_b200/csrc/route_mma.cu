@@ -12,30 +12,16 @@
 // The selection logic (eligibility, forced nodes, Select_K, expansion) is the SIMT kernel's.
 #include <math_constants.h>
 
+#include "mma_frag.cuh"
 #include "pisa_common.cuh"
 
 namespace pisa {
 
+using namespace frag;
+
 namespace {
 
 constexpr int kWarpsPerCta = 4;
-
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                               uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ uint4 ldg128(const void* p) { return *reinterpret_cast<const uint4*>(p); }
-
-// running (max, sum exp) of one head's child logits
-__device__ __forceinline__ void lse_add(float& m, float& s, float z) {
-  const float mn = fmaxf(m, z);
-  s = s * __expf(m - mn) + __expf(z - mn);
-  m = mn;
-}
 
 }  // namespace
 
