@@ -477,6 +477,103 @@ def run_sweep(args):
     return rows
 
 
+def decode_bytes_per_step(w, pos):
+    """Algorithmic bytes one decoding step must read for a late token (per the method, Sec. 3.3
+    "Decoding"): child summaries of the scored candidates at every pruned intermediate level, the raw
+    keys of the scored leaf candidates, keys and values of the selected blocks."""
+    es, c = 2, pos // w.C
+    M = [w.N, -(-w.N // w.C)]
+    while M[-1] > 1:
+        M.append(-(-M[-1] // w.g))
+    L = len(M) - 1
+    per_head = 0
+    n = 1
+    for l in range(L, 1, -1):
+        anc = c // (w.g ** (l - 1))
+        nV = min(n, anc + 1)
+        if nV > w.K:
+            per_head += nV * w.g * w.d * es
+            nV = w.K
+        n = nV * w.g
+    nV1 = min(n, c + 1)
+    if nV1 > w.K:
+        per_head += (nV1 - 3) * w.C * w.d * es
+    per_head += min(nV1, w.K) * w.C * w.d * es * 2
+    return per_head * w.B * w.Hkv
+
+
+def run_decode(args):
+    """Decoding latency vs context length: one pisa_decode_step launch per token over a cache whose
+    pyramid was built by the prefill kernels.  One JSON line per (shape, N).  Not the bench line."""
+    import torch
+
+    import paper_2609_31093_b200 as P
+    from paper_2609_31093_b200 import binding as PB
+
+    torch.cuda.set_device(0)
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        peaks = {}
+    hbm_peak = peaks.get("hbm_gbs", 6650.0)
+    shapes = [("cfg4_shape", dict(B=1, Hq=32, Hkv=8, d=128, C=128, g=2, K=32)),
+              ("cfg5_shape", dict(B=1, Hq=16, Hkv=4, d=128, C=64, g=2, K=16)),
+              ("paper_shape", dict(B=1, Hq=32, Hkv=2, d=64, C=64, g=2, K=8)),
+              ("cfg4_shape_b8", dict(B=8, Hq=32, Hkv=8, d=128, C=128, g=2, K=32))]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for tag, sh in shapes:
+        for n in [8192, 32768, 131072, 524288]:
+            if sh["B"] * n * sh["Hkv"] * sh["d"] * 2 * 2 > 40e9:
+                continue
+            w = S.Workload(f"{tag}_{n}", sh["B"], n, sh["Hq"], sh["Hkv"], sh["d"], sh["C"], sh["g"], sh["K"],
+                           "bf16", 6, "iid")
+            p = P.Params.from_workload(w)
+            gen = torch.Generator(device="cuda").manual_seed(1000 + n)
+            k = torch.randn((w.B, n, w.Hkv, w.d), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+            v = torch.randn((w.B, n, w.Hkv, w.d), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+            steps = 32
+            qs = torch.randn((steps, w.B, w.Hq, w.d), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+            pyramid = PB.alloc_pyramid(p)
+            P.pisa_build_pyramid(p, k, pyramid)
+            idx = torch.empty((w.B, w.Hkv, w.K), dtype=torch.int32, device="cuda")
+            out = torch.empty((w.B, w.Hq, w.d), dtype=torch.bfloat16, device="cuda")
+            lse = torch.empty((w.B, w.Hq), dtype=torch.float32, device="cuda")
+            ws = PB.alloc_workspace(p, PB.OP_DECODE)
+            pos0 = n - steps
+            for i in range(3):
+                P.pisa_decode_step(p, pos0 + i, qs[i], k, v, pyramid, idx, out, lse, ws)
+            torch.cuda.synchronize()
+            # cold: L2 flushed before every step
+            cold = 0.0
+            evs = []
+            for i in range(steps):
+                flush.fill_(i & 0xFF)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                P.pisa_decode_step(p, pos0 + i, qs[i], k, v, pyramid, idx, out, lse, ws)
+                e1.record()
+                evs.append((e0, e1))
+            torch.cuda.synchronize()
+            cold = sum(a.elapsed_time(b) for a, b in evs) / steps * 1e3
+            # warm: steps back to back
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(steps):
+                P.pisa_decode_step(p, pos0 + i, qs[i], k, v, pyramid, idx, out, lse, ws)
+            e1.record()
+            torch.cuda.synchronize()
+            warm = e0.elapsed_time(e1) / steps * 1e3
+            nbytes = decode_bytes_per_step(w, n - 1)
+            row = {"decode": tag, "workload": describe(w), "N": n, "us_per_step_cold_l2": cold,
+                   "us_per_step_back_to_back": warm, "algorithmic_bytes_per_step": nbytes,
+                   "gbs_cold": nbytes / (cold * 1e-6) / 1e9, "hbm_peak_gbs": hbm_peak,
+                   "frac_hbm_cold": nbytes / (cold * 1e-6) / 1e9 / hbm_peak, "status": P.read_status(ws),
+                   "tokens_per_s_back_to_back": w.B / (warm * 1e-6)}
+            print(json.dumps(row), flush=True)
+            del k, v, qs, pyramid
+            torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -489,9 +586,13 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="routing latency vs N and the flat selector (not the bench line)")
+    ap.add_argument("--decode", action="store_true", help="decoding latency vs context length (not the bench line)")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
+        return
+    if args.decode:
+        run_decode(args)
         return
     if args.impl == "reference":
         run_reference(args)

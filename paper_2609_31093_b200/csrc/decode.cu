@@ -81,8 +81,10 @@ __device__ void refresh_path(const Geometry& geo, const DecArgs& a, int b, int h
   }
 }
 
-template <int D, int NT>
-__global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kDecThreads, 1)
+// MINB = 1: all registers to one CTA per SM (lowest latency, small batches); MINB = 2: two CTAs per SM so
+// that the latency-bound phases of different clusters overlap once the grid exceeds the SM count.
+template <int D, int NT, int MINB>
+__global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kDecThreads, MINB)
 decode_step_kernel(Geometry geo, DecArgs a) {
   extern __shared__ float s_part[];                       // [kDecWarps][G*D + 2*G] attention partials
   __shared__ int s_cand[2][kMaxCand];
@@ -204,10 +206,21 @@ decode_step_kernel(Geometry geo, DecArgs a) {
       float m[NT][2], ssum[NT][2];
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) { m[nt][0] = m[nt][1] = -CUDART_INF_F; ssum[nt][0] = ssum[nt][1] = 0.f; }
-      for (int kt = 0; kt < C; kt += 16) {
+      for (int kt = 0; kt < C; kt += 32) {                       // two key tiles in flight per round
         const long long t_lo = (long long)leaf * C + kt + gid;
+        RowPair<D> r0, r1;
+        r0.load(kbh + t_lo * geo.ks[1], kbh + (t_lo + 8) * geo.ks[1], lane);
+        r1.load(kbh + (t_lo + 16) * geo.ks[1], kbh + (t_lo + 24) * geo.ks[1], lane);
         float z[NT][4];
-        rows2_dot<D, NT>(qf, kbh + t_lo * geo.ks[1], kbh + (t_lo + 8) * geo.ks[1], lane, z);
+        rows2_dot<D, NT>(qf, r0, z);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int jh = 0; jh < 2; ++jh) {
+            lse_add(m[nt][jh], ssum[nt][jh], z[nt][jh] * geo.scale);
+            lse_add(m[nt][jh], ssum[nt][jh], z[nt][2 + jh] * geo.scale);
+          }
+        rows2_dot<D, NT>(qf, r1, z);
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -288,9 +301,24 @@ decode_step_kernel(Geometry geo, DecArgs a) {
     for (int kt = 0; kt < C / 2; kt += 16) {
       const int t_lo = key0 + kt + gid, t_hi = t_lo + 8;
       if (key0 + kt > pos) break;                          // the rest of the block lies in the future
+      RowPair<D> kr;
+      kr.load((t_lo <= pos) ? kbh + (long long)t_lo * geo.ks[1] : nullptr,
+              (t_hi <= pos) ? kbh + (long long)t_hi * geo.ks[1] : nullptr, lane);
+      // the tile's sixteen value rows (this lane's DV columns of each), in flight during the softmax
+      uint32_t vraw[16][DV / 2];
+#pragma unroll
+      for (int kk = 0; kk < 16; ++kk) {
+        const int t = key0 + kt + kk;
+#pragma unroll
+        for (int j = 0; j < DV / 2; ++j) vraw[kk][j] = 0u;
+        if (t <= pos) {
+          const uint32_t* vr = reinterpret_cast<const uint32_t*>(vbh + (long long)t * geo.vs[1] + lane * DV);
+#pragma unroll
+          for (int j = 0; j < DV / 2; ++j) vraw[kk][j] = vr[j];
+        }
+      }
       float z[NT][4];
-      rows2_dot<D, NT>(qf, (t_lo <= pos) ? kbh + (long long)t_lo * geo.ks[1] : nullptr,
-                       (t_hi <= pos) ? kbh + (long long)t_hi * geo.ks[1] : nullptr, lane, z);
+      rows2_dot<D, NT>(qf, kr, z);
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -327,13 +355,14 @@ decode_step_kernel(Geometry geo, DecArgs a) {
 #pragma unroll
           for (int j = 0; j < DV; ++j) o_acc[hh][j] *= al;
         }
-      for (int kk = 0; kk < 16; ++kk) {
-        const int t = key0 + kt + kk;
-        if (t > pos) break;
-        float vv[DV];
-        const __nv_bfloat16* vr = vbh + (long long)t * geo.vs[1] + lane * DV;
 #pragma unroll
-        for (int j = 0; j < DV; ++j) vv[j] = __bfloat162float(vr[j]);
+      for (int kk = 0; kk < 16; ++kk) {                    // rows after pos hold zeros and weight 0
+        float vv[DV];
+#pragma unroll
+        for (int j = 0; j < DV / 2; ++j) {
+          vv[2 * j] = __uint_as_float(vraw[kk][j] << 16);
+          vv[2 * j + 1] = __uint_as_float(vraw[kk][j] & 0xFFFF0000u);
+        }
 #pragma unroll
         for (int hh = 0; hh < 16; ++hh)
           if (hh < G) {
@@ -392,13 +421,24 @@ decode_step_kernel(Geometry geo, DecArgs a) {
   }
 }
 
+template <int D, int NT, int MINB>
+int launch_dnb(const Geometry& g, const DecArgs& a, cudaStream_t s) {
+  const size_t smem = (size_t)kDecWarps * (g.G * D + 2 * g.G) * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(decode_step_kernel<D, NT, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)smem);
+  if (e != cudaSuccess) { record_cuda_error("decode_step attr", e); return PISA_ERR_CUDA; }
+  decode_step_kernel<D, NT, MINB><<<dim3(kClu, (unsigned)(g.B * g.Hkv)), kDecThreads, smem, s>>>(g, a);
+  return check_launch("decode_step");
+}
 template <int D, int NT>
 int launch_dn(const Geometry& g, const DecArgs& a, cudaStream_t s) {
-  const size_t smem = (size_t)kDecWarps * (g.G * D + 2 * g.G) * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(decode_step_kernel<D, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) { record_cuda_error("decode_step attr", e); return PISA_ERR_CUDA; }
-  decode_step_kernel<D, NT><<<dim3(kClu, (unsigned)(g.B * g.Hkv)), kDecThreads, smem, s>>>(g, a);
-  return check_launch("decode_step");
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  }
+  return ((long long)g.B * g.Hkv * kClu > sms) ? launch_dnb<D, NT, 2>(g, a, s) : launch_dnb<D, NT, 1>(g, a, s);
 }
 
 }  // namespace

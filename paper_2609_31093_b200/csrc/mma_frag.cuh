@@ -81,5 +81,32 @@ __device__ __forceinline__ void rows2_dot(const QFrag<D, NT>& q, const __nv_bflo
   }
 }
 
+// The same dot products with the loads split from the arithmetic, so that a caller can put the loads
+// of several row pairs in flight before the first MMA waits on any of them.
+template <int D>
+struct RowPair {
+  uint4 a[D / 32], b[D / 32];
+  __device__ __forceinline__ void load(const __nv_bfloat16* lo, const __nv_bfloat16* hi, int lane) {
+    const int tig = lane & 3;
+#pragma unroll
+    for (int c4 = 0; c4 < D / 32; ++c4) {
+      a[c4] = lo ? ldg128(lo + (c4 * 4 + tig) * 8) : make_uint4(0u, 0u, 0u, 0u);
+      b[c4] = hi ? ldg128(hi + (c4 * 4 + tig) * 8) : make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+};
+template <int D, int NT>
+__device__ __forceinline__ void rows2_dot(const QFrag<D, NT>& q, const RowPair<D>& r, float (&z)[NT][4]) {
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    z[nt][0] = z[nt][1] = z[nt][2] = z[nt][3] = 0.f;
+#pragma unroll
+    for (int c4 = 0; c4 < D / 32; ++c4) {
+      mma_bf16_16816(z[nt], r.a[c4].x, r.b[c4].x, r.a[c4].y, r.b[c4].y, q.r[nt][c4][0], q.r[nt][c4][1]);
+      mma_bf16_16816(z[nt], r.a[c4].z, r.b[c4].z, r.a[c4].w, r.b[c4].w, q.r[nt][c4][2], q.r[nt][c4][3]);
+    }
+  }
+}
+
 }  // namespace frag
 }  // namespace pisa
