@@ -117,9 +117,10 @@ decode_step_kernel(Geometry geo, DecArgs a) {
     const int* cand = s_cand[cur];
     int* next = s_cand[cur ^ 1];
     const int n = s_n;
-    const long long span = geo.span[l];
-    const int anc_c = (int)(c / span);
-    const int f1l = (c >= 1) ? (int)((c - 1) / span) : 0;
+    // leaves under a level-l node; c < 2^31, so a span beyond that just means ancestor 0 (32-bit division)
+    const unsigned span = (unsigned)min(geo.span[l], (long long)0x7fffffff);
+    const int anc_c = (int)((unsigned)c / span);
+    const int f1l = (c >= 1) ? (int)((unsigned)(c - 1) / span) : 0;
     int nV = 0;                                           // eligible candidates form a prefix
     for (int s0 = 0; s0 < n; s0 += 32) {
       const int s = s0 + lane;

@@ -70,9 +70,10 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
   for (int l = geo.L; l >= 2; --l) {
     int* cand = s_cand[warp][cur];
     int* next = s_cand[warp][cur ^ 1];
-    const long long span = geo.span[l];
-    const int anc_c = (int)(c / span);
-    const int f1 = (c >= 1) ? (int)((c - 1) / span) : 0;
+    // leaves under a level-l node; c < 2^31, so a span beyond that just means ancestor 0 (32-bit division)
+    const unsigned span = (unsigned)min(geo.span[l], (long long)0x7fffffff);
+    const int anc_c = (int)((unsigned)c / span);
+    const int f1 = (c >= 1) ? (int)((unsigned)(c - 1) / span) : 0;
     int nV = 0;
     for (int s0 = 0; s0 < n; s0 += 32) {
       const int s = s0 + lane;
