@@ -574,6 +574,86 @@ def run_decode(args):
             torch.cuda.empty_cache()
 
 
+def selection_quality(idx_sparse, mass):
+    """Recall@K and MassRatio (Sec. 5 "Block-selection quality") of selected block sets against the
+    reference sets built from full-attention block masses.
+
+    idx_sparse: int array [S, K] (-1 padded); mass: float array [S, M] = full-attention mass of every
+    block for the same S queries (already averaged over the group's heads, zero for future blocks).
+    The reference set of a query is its K blocks of largest mass (among blocks with non-zero mass when
+    fewer than K exist).  Returns (recall [S], mass_ratio [S])."""
+    idx_sparse = np.asarray(idx_sparse)
+    mass = np.asarray(mass, dtype=np.float64)
+    S_, K = idx_sparse.shape
+    recall = np.empty(S_)
+    ratio = np.empty(S_)
+    for s in range(S_):
+        live = int((mass[s] > 0).sum())
+        k_ref = min(K, live)
+        ref = np.argsort(-mass[s], kind="stable")[:k_ref]
+        sel = idx_sparse[s][idx_sparse[s] >= 0]
+        recall[s] = len(set(ref.tolist()) & set(sel.tolist())) / float(max(k_ref, 1))
+        ratio[s] = mass[s][sel].sum() / max(mass[s][ref].sum(), 1e-300)
+    return recall, ratio
+
+
+def run_quality(args):
+    """Selection quality of the score modes (LSE = PISA, mean = PISA-1, mean + variance/2 = PISA-2) and of
+    the flat mean selector against full attention, on synthetic tensors with a drifting mean (the
+    paper measures this on a trained model's queries and keys, which are not available here; the
+    numbers say how the selectors differ on this synthetic structure, nothing about a model).
+    One JSON line per selector.  Not the bench line."""
+    import torch
+
+    import paper_2609_31093_b200 as P
+    from paper_2609_31093_b200 import binding as PB
+
+    torch.cuda.set_device(0)
+    w = S.Workload("quality_walk", 1, 16384, 8, 2, 128, 64, 2, 8, "bf16", 7, "walk")
+    t = S.make_inputs(w)
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda()
+    q, k = dev(t["q"]), dev(t["k"])
+    rng = np.random.default_rng(11)
+    pos = np.sort(rng.choice(np.arange(w.K * w.C, w.N), size=512, replace=False))
+    # full-attention block masses of the sampled queries, averaged over the group's heads
+    G, M1 = w.G, w.M1
+    mass = np.zeros((w.Hkv, len(pos), M1))
+    scale = 1.0 / np.sqrt(w.d)
+    for h in range(w.Hkv):
+        kf = k[0, :, h].float()                                            # [N, d]
+        for j, p_ in enumerate(pos.tolist()):
+            qf = q[0, p_, h * G:(h + 1) * G].float()                       # [G, d]
+            z = (qf @ kf[:p_ + 1].T) * scale
+            pr = torch.softmax(z.double(), dim=-1).mean(dim=0)              # [p+1]
+            pad = torch.zeros(M1 * w.C, dtype=torch.float64, device="cuda")
+            pad[:p_ + 1] = pr
+            mass[h, j] = pad.view(M1, w.C).sum(dim=1).cpu().numpy()
+    rows = []
+    for name, mode, impl, flat in (("pisa_lse", "lse", PB.IMPL_AUTO, False), ("pisa1_mean", "mean", PB.IMPL_SIMT, False),
+                                   ("pisa2_mean_var", "mean_var", PB.IMPL_SIMT, False), ("flat_mean", "lse", PB.IMPL_AUTO, True)):
+        p = P.Params.from_workload(w, score_mode=mode, impl=impl)
+        pyramid = PB.alloc_pyramid(p)
+        idx = torch.empty((w.B, w.Hkv, w.N, w.K), dtype=torch.int32, device="cuda")
+        ws = PB.alloc_workspace(p, PB.OP_FORWARD)
+        P.pisa_build_pyramid(p, k, pyramid)
+        if flat:
+            P.pisa_flat_select(p, q, pyramid, idx, ws)
+        else:
+            P.pisa_route(p, q, k, pyramid, idx, None, ws)
+        torch.cuda.synchronize()
+        sel = idx[0][:, torch.from_numpy(pos).cuda()].cpu().numpy()         # [Hkv, S, K]
+        rec, rat = [], []
+        for h in range(w.Hkv):
+            r_, m_ = selection_quality(sel[h], mass[h])
+            rec.append(r_)
+            rat.append(m_)
+        row = {"quality": name, "workload": describe(w), "queries": int(len(pos) * w.Hkv), "K": w.K,
+               "recall_at_k": float(np.mean(rec)), "mass_ratio": float(np.mean(rat)), "status": P.read_status(ws)}
+        rows.append(row)
+        print(json.dumps(row), flush=True)
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -586,6 +666,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="routing latency vs N and the flat selector (not the bench line)")
+    ap.add_argument("--quality", action="store_true", help="Recall@K / MassRatio of the score modes vs full attention (not the bench line)")
     ap.add_argument("--decode", action="store_true", help="decoding latency vs context length (not the bench line)")
     args = ap.parse_args()
     if args.sweep:
@@ -593,6 +674,9 @@ def main():
         return
     if args.decode:
         run_decode(args)
+        return
+    if args.quality:
+        run_quality(args)
         return
     if args.impl == "reference":
         run_reference(args)

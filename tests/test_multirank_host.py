@@ -59,3 +59,19 @@ def test_reference_arm_runs_on_rank0_only():
     line = json.loads(r.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["value"] > 0 and line["unit"] == "tokens/s"
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_selection_quality_metrics_on_a_hand_case():
+    """Recall@K and MassRatio as the paper defines them (Sec. 5 "Block-selection quality")."""
+    import numpy as np
+
+    import bench
+    mass = np.array([[0.5, 0.1, 0.3, 0.1, 0.0, 0.0],        # reference top-2: blocks 0, 2
+                     [0.2, 0.2, 0.6, 0.0, 0.0, 0.0]])       # reference top-2: 2 and 0 (tie -> smaller index)
+    idx = np.array([[0, 3], [1, 2]], dtype=np.int32)
+    rec, rat = bench.selection_quality(idx, mass)
+    assert np.allclose(rec, [0.5, 0.5])
+    assert np.allclose(rat, [0.6 / 0.8, 0.8 / 0.8])
+    # fewer live blocks than K: the reference set shrinks, padding is ignored
+    rec, rat = bench.selection_quality(np.array([[0, -1, -1]], dtype=np.int32), np.array([[1.0, 0.0, 0.0]]))
+    assert np.allclose(rec, [1.0]) and np.allclose(rat, [1.0])
