@@ -27,6 +27,9 @@ What follows which passage of the paper:
                          (App. C), Top-K.
 * `score_mode`           Sec. 4.3 / App. A.2: "lse" (PISA), "mean" (PISA-1),
                          "mean_var" (PISA-2).
+* `attend_backward`      App. B: backward of the selected sparse attention with the
+                         selected indices held fixed (softmax-attention gradients
+                         restricted to the selected, visible keys).
 * `decode_pyramid`,      Sec. 3.3 "Decoding" and App. B "Decode cache": when the
   `decode_step`          token at position p is generated the cached pyramid
                          holds the means of the keys seen so far, i.e. it is the
@@ -53,7 +56,9 @@ hand-derived example and the invariants.  Decoding is pinned by what the
 definitions imply: the step at position p selects what the prefill of any
 longer sequence selects for row p (every scored node lies strictly in the past),
 equals torch's dense causal attention when K*C > p, and the cached pyramid's
-completed nodes equal those of the longer sequence's pyramid.
+completed nodes equal those of the longer sequence's pyramid.  The backward is
+pinned by torch autograd on a dense masked attention built from the same index
+sets and by finite differences of the forward (tests/test_oracle_backward_pins.py).
 """
 from __future__ import annotations
 
@@ -453,3 +458,48 @@ def decode_step(q_new, k_cache, v_cache, pos: int, *, C: int, g: int, K: int, dt
             for hq in range(h * prob.G, (h + 1) * prob.G):
                 out[b, hq], lse[b, hq] = prob.attend(b, hq, pos, I)
     return idx, margin, round_to_storage(out, dtype), lse
+
+
+# --------------------------------------------------------------------------
+# backward of the selected sparse attention with frozen indices (App. B)
+# --------------------------------------------------------------------------
+
+def attend_backward(q, k, v, idx, dout, *, C: int, dtype: str, scale: Optional[float] = None):
+    """Gradients of Eq. "selected sparse attention" with the selected block indices held fixed
+    (App. B: gradients flow through attention on the selected entries, not through the selection).
+
+    q, dout: [B, N, Hq, d]; k, v: [B, N, Hkv, d] storage form; idx: int [B, Hkv, N, K] (-1 padded).
+    For one query row with probabilities p_j over its visible selected keys, o = sum_j p_j v_j:
+        dv_j += p_j do,   dp_j = do . v_j,   ds_j = p_j (dp_j - sum_i p_i dp_i),
+        dq   += scale * sum_j ds_j k_j,      dk_j += scale * ds_j q.
+    Returns dq [B,N,Hq,d], dk, dv [B,N,Hkv,d] in fp64 (not rounded to the storage dtype)."""
+    B, N, Hq, d = q.shape
+    Hkv = k.shape[2]
+    G = Hq // Hkv
+    sc = (1.0 / math.sqrt(d)) if scale is None else float(scale)
+    qf, kf, vf, dof = (load_storage(np.ascontiguousarray(x), dtype) for x in (q, k, v, dout))
+    dq = np.zeros((B, N, Hq, d))
+    dk = np.zeros((B, N, Hkv, d))
+    dv = np.zeros((B, N, Hkv, d))
+    for b in range(B):
+        for h in range(Hkv):
+            k_bh, v_bh = kf[b, :, h], vf[b, :, h]
+            for p in range(N):
+                toks: List[int] = []
+                for i in idx[b, h, p]:
+                    if i >= 0:
+                        toks.extend(j for j in range(int(i) * C, min((int(i) + 1) * C, N)) if j <= p)
+                if not toks:
+                    continue
+                ta = np.asarray(toks, dtype=np.int64)
+                for hq in range(h * G, (h + 1) * G):
+                    z = (k_bh[ta] @ qf[b, p, hq]) * sc
+                    e = np.exp(z - z.max())
+                    pr = e / e.sum()
+                    do = dof[b, p, hq]
+                    dp = v_bh[ta] @ do
+                    ds = pr * (dp - float(pr @ dp))
+                    dq[b, p, hq] += sc * (ds @ k_bh[ta])
+                    dk[b, ta, h] += sc * ds[:, None] * qf[b, p, hq][None, :]
+                    dv[b, ta, h] += pr[:, None] * do[None, :]
+    return dq, dk, dv
