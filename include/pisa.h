@@ -50,7 +50,7 @@ enum { PISA_BF16 = 0, PISA_FP32 = 1 };
 enum { PISA_SCORE_LSE = 0, PISA_SCORE_MEAN = 1, PISA_SCORE_MEAN_VAR = 2 };
 /* operations a workspace can be sized for */
 enum { PISA_OP_ROUTE = 0, PISA_OP_BSA = 1, PISA_OP_FORWARD = 2, PISA_OP_FLAT = 3, PISA_OP_FORWARD_HOST = 4,
-       PISA_OP_DECODE = 5 };
+       PISA_OP_DECODE = 5, PISA_OP_BSA_BWD = 6 };
 /* implementation selector (params.impl): AUTO picks the tensor-core path where it applies */
 enum { PISA_IMPL_AUTO = 0, PISA_IMPL_SIMT = 1, PISA_IMPL_TENSOR = 2 };
 
@@ -156,6 +156,26 @@ int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const voi
 int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_host, const void* v_host,
                       void* out_host, float* lse_host, int32_t* idx_host,
                       void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Backward of the block-sparse attention with the selected indices held fixed (App. B: gradients
+ * flow through attention on the selected entries, not through the selection).
+ *
+ *   q, k, v, idx   : as for pisa_bsa_fwd
+ *   out, lse       : what pisa_bsa_fwd / pisa_forward produced for these idx (out with o_stride)
+ *   dout           : gradient of the loss w.r.t. out, device, same dtype and strides as out
+ *   dq             : device [B, N, Hq, d], dense, input dtype
+ *   dk, dv         : device [B, N, Hkv, d], dense, input dtype; keys no query selected get zeros
+ *   ws             : device workspace sized for PISA_OP_BSA_BWD (holds fp32 accumulators of all
+ *                    three gradients; partial sums are added with fp32 reductions, so results are
+ *                    reproducible to fp32 rounding, not bitwise)
+ *
+ * bf16, d = 128, C in {64, 128}, g*C in {128, 256}; other configurations return
+ * PISA_ERR_UNSUPPORTED.  Asynchronous on `stream`.
+ */
+int pisa_bsa_bwd(const pisa_params_t* p, const void* q, const void* k, const void* v, const int32_t* idx,
+                 const void* out, const float* lse, const void* dout, void* dq, void* dk, void* dv,
+                 void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Decoding (Sec. 3.3 "Decoding", App. B "Decode cache"): one new token per sequence, one kernel launch.

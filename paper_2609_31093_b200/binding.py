@@ -13,7 +13,7 @@ _lib = None
 
 BF16, FP32 = 0, 1
 SCORE_LSE, SCORE_MEAN, SCORE_MEAN_VAR = 0, 1, 2
-OP_ROUTE, OP_BSA, OP_FORWARD, OP_FLAT, OP_FORWARD_HOST, OP_DECODE = 0, 1, 2, 3, 4, 5
+OP_ROUTE, OP_BSA, OP_FORWARD, OP_FLAT, OP_FORWARD_HOST, OP_DECODE, OP_BSA_BWD = 0, 1, 2, 3, 4, 5, 6
 IMPL_AUTO, IMPL_SIMT, IMPL_TENSOR = 0, 1, 2
 _SCORE = {"lse": SCORE_LSE, "mean": SCORE_MEAN, "mean_var": SCORE_MEAN_VAR}
 
@@ -57,6 +57,7 @@ def lib():
     L.pisa_flat_select.argtypes = [pp, vp, vp, vp, vp, C.c_size_t, vp]
     L.pisa_decode_step.argtypes = [pp, C.c_int32, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
     L.pisa_pyramid_regrow.argtypes = [pp, pp, vp, vp, vp]
+    L.pisa_bsa_bwd.argtypes = [pp] + [vp] * 11 + [C.c_size_t, vp]
     L.pisa_read_status.argtypes = [vp, i32p]
     L.pisa_route_static.argtypes = [pp, vp, vp, vp, vp, vp, vp]
     L.pisa_route_static.restype = C.c_int
@@ -68,7 +69,7 @@ def lib():
     L.pisa_get_kernel_ms.restype = C.c_int
     for name in ("pisa_pyramid_layout", "pisa_workspace_bytes", "pisa_build_pyramid", "pisa_route",
                  "pisa_bsa_fwd", "pisa_forward", "pisa_forward_host", "pisa_flat_select", "pisa_read_status",
-                 "pisa_decode_step", "pisa_pyramid_regrow",
+                 "pisa_decode_step", "pisa_pyramid_regrow", "pisa_bsa_bwd",
                  "pisa_set_stage_timing", "pisa_get_stage_ms"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -182,6 +183,12 @@ def pisa_forward_host(p: Params, q_host, k_host, v_host, out_host, lse_host, idx
     _check(lib().pisa_forward_host(p.ref(), _ptr(q_host), _ptr(k_host), _ptr(v_host), _ptr(out_host),
                                    _ptr(lse_host), _ptr(idx_host), _ptr(ws), ws.numel(), _stream()),
            "pisa_forward_host")
+
+
+def pisa_bsa_bwd(p: Params, q, k, v, idx, out, lse, dout, dq, dk, dv, ws):
+    """Gradients of the block-sparse attention for fixed idx; dq, dk, dv are dense outputs."""
+    _check(lib().pisa_bsa_bwd(p.ref(), _ptr(q), _ptr(k), _ptr(v), _ptr(idx), _ptr(out), _ptr(lse), _ptr(dout),
+                              _ptr(dq), _ptr(dk), _ptr(dv), _ptr(ws), ws.numel(), _stream()), "pisa_bsa_bwd")
 
 
 def pisa_decode_step(p: Params, pos: int, q, k_cache, v_cache, pyramid, idx, out, lse, ws):

@@ -269,6 +269,10 @@ int pisa_workspace_bytes(const pisa_params_t* p, int op, size_t* bytes) {
     case PISA_OP_BSA: *bytes = a; break;
     case PISA_OP_FORWARD: *bytes = f; break;
     case PISA_OP_FLAT: *bytes = kStatusBytes; break;
+    case PISA_OP_BSA_BWD:
+      if (!tensor_bwd_supported(g, p->dtype) || p->impl == PISA_IMPL_SIMT) return PISA_ERR_UNSUPPORTED;
+      *bytes = kStatusBytes + tensor_bwd_workspace_bytes(g);
+      break;
     case PISA_OP_DECODE:
       if (!decode_supported(g, p->dtype)) return PISA_ERR_UNSUPPORTED;
       *bytes = kStatusBytes + decode_workspace_bytes(g);
@@ -419,6 +423,27 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
   if (s_in) cudaStreamDestroy(s_in);
   if (s_out) cudaStreamDestroy(s_out);
   if (e != cudaSuccess) { record_cuda_error(what, e); return PISA_ERR_CUDA; }
+  return st;
+}
+
+int pisa_bsa_bwd(const pisa_params_t* p, const void* q, const void* k, const void* v, const int32_t* idx,
+                 const void* out, const float* lse, const void* dout, void* dq, void* dk, void* dv,
+                 void* ws, size_t ws_bytes, void* stream) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (!q || !k || !v || !idx || !out || !lse || !dout || !dq || !dk || !dv || !ws) return PISA_ERR_INVALID_ARG;
+  if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(out) || misaligned(dout) || misaligned(dq) ||
+      misaligned(dk) || misaligned(dv) || misaligned(ws))
+    return PISA_ERR_INVALID_ARG;
+  if (!tensor_bwd_supported(g, p->dtype) || p->impl == PISA_IMPL_SIMT) return PISA_ERR_UNSUPPORTED;
+  if (ws_bytes < kStatusBytes + tensor_bwd_workspace_bytes(g)) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t s = (cudaStream_t)stream;
+  st = clear_status(ws, s);
+  if (st != PISA_OK) return st;
+  g_mark_n = 0;
+  st = tensor_bsa_bwd(g, q, k, v, idx, out, lse, dout, dq, dk, dv, (char*)ws + kStatusBytes, (int32_t*)ws, s);
+  kernel_mark("end", s);
   return st;
 }
 

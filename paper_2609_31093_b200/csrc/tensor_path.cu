@@ -1184,6 +1184,30 @@ int dispatch_tile_pv(const Geometry& g, const TileArgs& a, cudaStream_t s) {
   return PISA_ERR_UNSUPPORTED;
 }
 
+#include "bsa_bwd_kernel.cuh"
+
+struct BwdLayout { size_t delta, dq, dk, dv, total; InvLayout inv; };
+BwdLayout bwd_layout(const Geometry& g) {
+  BwdLayout r;
+  size_t o = 0;
+  r.delta = o; o += align_up((size_t)g.B * g.Hq * g.N * 4, 256);
+  r.dq = o; o += align_up((size_t)g.B * g.N * g.Hq * g.d * 4, 256);
+  r.dk = o; o += align_up((size_t)g.B * g.N * g.Hkv * g.d * 4, 256);
+  r.dv = o; o += align_up((size_t)g.B * g.N * g.Hkv * g.d * 4, 256);
+  r.inv = inv_layout(o, g, g.M[1]);
+  r.total = r.inv.end;
+  return r;
+}
+
+template <int C>
+int launch_bwd(const Geometry& g, const BwdArgs& a, cudaStream_t s) {
+  const size_t smem = 4 * (size_t)(128 * 128) + 2 * (size_t)(C / 64) * (128 * 128) + 4 * (size_t)(C * 128) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(bsa_bwd_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) { record_cuda_error("bsa_bwd attr", e); return PISA_ERR_CUDA; }
+  bsa_bwd_kernel<C><<<num_sms(), kBwdThreads, smem, s>>>(g, a);
+  return check_launch("bsa_bwd");
+}
+
 }  // namespace
 
 bool tensor_path_supported(const Geometry& g, int dtype) {
@@ -1268,6 +1292,59 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
     convert_out_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(g, acc, (__nv_bfloat16*)out);
   }
   return check_launch("convert_out");
+}
+
+bool tensor_bwd_supported(const Geometry& g, int dtype) {
+  return tensor_path_supported(g, dtype) && g.d == 128;
+}
+size_t tensor_bwd_workspace_bytes(const Geometry& g) { return bwd_layout(g).total; }
+
+int tensor_bsa_bwd(const Geometry& g, const void* q, const void* k, const void* v, const int32_t* idx,
+                   const void* out, const float* lse, const void* dout, void* dq, void* dk, void* dv, void* ws_,
+                   int32_t* status, cudaStream_t s) {
+  char* ws = (char*)ws_;
+  const BwdLayout L = bwd_layout(g);
+  kernel_mark("invert_by_leaf", s);
+  InvArgs inv;
+  int st = run_inversion(g, idx, 1, g.M[1], ws, L.inv, &inv, s);
+  if (st != PISA_OK) return st;
+  BwdArgs a = {};
+  a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
+  a.dout = (const __nv_bfloat16*)dout; a.lse = lse;
+  float* delta = (float*)(ws + L.delta);
+  a.delta = delta;
+  a.entry_off = inv.entry_off; a.item_off = inv.item_off; a.item_key = inv.item_key; a.entries = inv.entries;
+  a.nkeys = g.B * g.Hkv * inv.NW * g.M[1]; a.Mk = g.M[1]; a.NW = inv.NW;
+  a.dq_acc = (float*)(ws + L.dq); a.dk_acc = (float*)(ws + L.dk); a.dv_acc = (float*)(ws + L.dv);
+  a.status = status;
+  kernel_mark("gradient_memset", s);
+  cudaError_t e = cudaMemsetAsync(ws + L.dq, 0, L.inv.count - L.dq, s);     // dq, dk, dv accumulators are adjacent
+  if (e != cudaSuccess) { record_cuda_error("gradient memset", e); return PISA_ERR_CUDA; }
+  kernel_mark("delta", s);
+  {
+    const long long rows = (long long)g.B * g.N * g.Hq;
+    bwd_delta_kernel<<<(unsigned)((rows * 32 + 255) / 256), 256, 0, s>>>(g, (const __nv_bfloat16*)out,
+                                                                        (const __nv_bfloat16*)dout, delta);
+    st = check_launch("bwd_delta");
+    if (st != PISA_OK) return st;
+  }
+  kernel_mark("backward_tiles", s);
+  st = (g.C == 128) ? launch_bwd<128>(g, a, s) : launch_bwd<64>(g, a, s);
+  if (st != PISA_OK) return st;
+  kernel_mark("convert_gradients", s);
+  {
+    Geometry gd = g;                                   // dq is dense [B, N, Hq, d]
+    gd.os[2] = g.d; gd.os[1] = (long long)g.Hq * g.d; gd.os[0] = (long long)g.N * g.Hq * g.d;
+    const long long n = (long long)g.B * g.N * g.Hkv * (g.d / 2);
+    convert_out_heads_inner_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(gd, a.dq_acc, (__nv_bfloat16*)dq);
+    st = check_launch("convert_dq");
+    if (st != PISA_OK) return st;
+    const long long n2 = (long long)g.B * g.N * g.Hkv * g.d / 2;
+    bwd_convert_kernel<<<(unsigned)((n2 + 255) / 256), 256, 0, s>>>(a.dk_acc, (__nv_bfloat16*)dk, n2);
+    bwd_convert_kernel<<<(unsigned)((n2 + 255) / 256), 256, 0, s>>>(a.dv_acc, (__nv_bfloat16*)dv, n2);
+    st = check_launch("convert_dkv");
+  }
+  return st;
 }
 
 }  // namespace pisa
