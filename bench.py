@@ -654,6 +654,60 @@ def run_quality(args):
     return rows
 
 
+def run_backward(args):
+    """Backward of the block-sparse attention (frozen indices) at the requested workload: forward once for
+    idx / out / lse, then timed pisa_bsa_bwd calls.  One JSON line.  Not the bench line."""
+    import torch
+
+    import paper_2609_31093_b200 as P
+    from paper_2609_31093_b200 import binding as PB
+
+    torch.cuda.set_device(0)
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        peaks = {}
+    tens_peak = peaks.get("bf16_tflops_sustained", 1400.0)
+    w = get_workload(args.workload)
+    t = S.make_inputs(w)
+    p = P.Params.from_workload(w)
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda()
+    q, k, v = dev(t["q"]), dev(t["k"]), dev(t["v"])
+    pyramid = PB.alloc_pyramid(p)
+    idx = torch.empty((w.B, w.Hkv, w.N, w.K), dtype=torch.int32, device="cuda")
+    out = torch.empty_like(q)
+    lse = torch.empty((w.B, w.Hq, w.N), dtype=torch.float32, device="cuda")
+    ws = PB.alloc_workspace(p, PB.OP_FORWARD)
+    P.pisa_forward(p, q, k, v, pyramid, idx, out, lse, ws)
+    torch.cuda.synchronize()
+    del ws
+    gen = torch.Generator(device="cuda").manual_seed(77)
+    dout = torch.randn(q.shape, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    wsb = PB.alloc_workspace(p, PB.OP_BSA_BWD)
+    P.set_stage_timing(True)
+    for _ in range(max(1, args.warmup)):
+        P.pisa_bsa_bwd(p, q, k, v, idx, out, lse, dout, dq, dk, dv, wsb)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        P.pisa_bsa_bwd(p, q, k, v, idx, out, lse, dout, dq, dk, dv, wsb)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    kern = P.get_kernel_ms()
+    wc = work_counts(w)
+    flops = 2.5 * wc["attn_flops"]                     # five products of the forward's two shapes
+    t_tiles = kern.get("backward_tiles", ms)
+    row = {"backward": describe(w), "ms_per_call": ms, "tokens_per_s": w.B * w.N / (ms * 1e-3), "kernels_ms": kern,
+           "algorithmic_tflop": flops / 1e12,
+           "roofline": {"kernel": "backward_tiles", "bound": "tensor", "achieved": flops / (t_tiles * 1e-3) / 1e12,
+                        "peak": tens_peak, "unit": "TFLOP/s", "frac": flops / (t_tiles * 1e-3) / 1e12 / tens_peak},
+           "status": P.read_status(wsb)}
+    print(json.dumps(row), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -666,6 +720,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="routing latency vs N and the flat selector (not the bench line)")
+    ap.add_argument("--backward", action="store_true", help="attention backward with frozen indices (not the bench line)")
     ap.add_argument("--quality", action="store_true", help="Recall@K / MassRatio of the score modes vs full attention (not the bench line)")
     ap.add_argument("--decode", action="store_true", help="decoding latency vs context length (not the bench line)")
     args = ap.parse_args()
@@ -677,6 +732,9 @@ def main():
         return
     if args.quality:
         run_quality(args)
+        return
+    if args.backward:
+        run_backward(args)
         return
     if args.impl == "reference":
         run_reference(args)

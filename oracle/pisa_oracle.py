@@ -464,6 +464,33 @@ def decode_step(q_new, k_cache, v_cache, pos: int, *, C: int, g: int, K: int, dt
 # backward of the selected sparse attention with frozen indices (App. B)
 # --------------------------------------------------------------------------
 
+def _backward_row(q_heads, k_bh, v_bh, do_heads, toks, sc):
+    """One (b, KV head, position): q_heads, do_heads [G, d]; toks = its visible selected keys.
+    Returns dq [G, d] and this row's contributions dk, dv [len(toks), d]."""
+    G, d = q_heads.shape
+    dq = np.zeros((G, d))
+    dk = np.zeros((len(toks), d))
+    dv = np.zeros((len(toks), d))
+    for j in range(G):
+        z = (k_bh[toks] @ q_heads[j]) * sc
+        e = np.exp(z - z.max())
+        pr = e / e.sum()
+        dp = v_bh[toks] @ do_heads[j]
+        ds = pr * (dp - float(pr @ dp))
+        dq[j] = sc * (ds @ k_bh[toks])
+        dk += sc * ds[:, None] * q_heads[j][None, :]
+        dv += pr[:, None] * do_heads[j][None, :]
+    return dq, dk, dv
+
+
+def _visible_tokens(blocks, p: int, C: int, N: int) -> np.ndarray:
+    toks: List[int] = []
+    for i in blocks:
+        if i >= 0:
+            toks.extend(j for j in range(int(i) * C, min((int(i) + 1) * C, N)) if j <= p)
+    return np.asarray(toks, dtype=np.int64)
+
+
 def attend_backward(q, k, v, idx, dout, *, C: int, dtype: str, scale: Optional[float] = None):
     """Gradients of Eq. "selected sparse attention" with the selected block indices held fixed
     (App. B: gradients flow through attention on the selected entries, not through the selection).
@@ -485,21 +512,23 @@ def attend_backward(q, k, v, idx, dout, *, C: int, dtype: str, scale: Optional[f
         for h in range(Hkv):
             k_bh, v_bh = kf[b, :, h], vf[b, :, h]
             for p in range(N):
-                toks: List[int] = []
-                for i in idx[b, h, p]:
-                    if i >= 0:
-                        toks.extend(j for j in range(int(i) * C, min((int(i) + 1) * C, N)) if j <= p)
-                if not toks:
+                ta = _visible_tokens(idx[b, h, p], p, C, N)
+                if len(ta) == 0:
                     continue
-                ta = np.asarray(toks, dtype=np.int64)
-                for hq in range(h * G, (h + 1) * G):
-                    z = (k_bh[ta] @ qf[b, p, hq]) * sc
-                    e = np.exp(z - z.max())
-                    pr = e / e.sum()
-                    do = dof[b, p, hq]
-                    dp = v_bh[ta] @ do
-                    ds = pr * (dp - float(pr @ dp))
-                    dq[b, p, hq] += sc * (ds @ k_bh[ta])
-                    dk[b, ta, h] += sc * ds[:, None] * qf[b, p, hq][None, :]
-                    dv[b, ta, h] += pr[:, None] * do[None, :]
+                rq, rk, rv = _backward_row(qf[b, p, h * G:(h + 1) * G], k_bh, v_bh, dof[b, p, h * G:(h + 1) * G], ta, sc)
+                dq[b, p, h * G:(h + 1) * G] = rq
+                dk[b, ta, h] += rk
+                dv[b, ta, h] += rv
     return dq, dk, dv
+
+
+def attend_backward_dq_rows(prob: "Problem", triples, idx_rows, dout_rows):
+    """dq of sampled queries of a long sequence: triples [S, 3] (b, KV head, position), idx_rows [S, K],
+    dout_rows [S, G, d] storage form.  Returns fp64 [S, G, d]."""
+    out = np.empty((len(triples), prob.G, prob.d))
+    for s, (b, h, p) in enumerate(triples):
+        k_bh, v_bh, _ = prob.head(int(b), int(h))
+        ta = _visible_tokens(idx_rows[s], int(p), prob.C, prob.N)
+        do = load_storage(np.ascontiguousarray(dout_rows[s]), prob.dtype)
+        out[s] = _backward_row(prob.q_group(int(b), int(h), int(p)), k_bh, v_bh, do, ta, prob.scale)[0]
+    return out

@@ -76,3 +76,44 @@ def test_backward_rejects_unsupported_head_dim():
     p = P.Params(1, 1024, 4, 2, 64, 64, 2, 4)
     with pytest.raises(P.PisaError, match="unsupported"):
         P.workspace_bytes(p, PB.OP_BSA_BWD)
+
+
+def test_backward_at_the_headline_size_sampled_rows_and_identities():
+    """cfg4 in the launch configuration bench.py --backward times: sampled dq rows against the oracle and two
+    identities that hold at any size: sum over keys of dv = sum over the group's rows of dO (probabilities of a
+    row add up to one) and sum over keys of dk = 0 (the dS of a row add up to zero)."""
+    w = S.WORKLOADS["cfg4"]
+    t = S.make_inputs(w)
+    dev = T.Device(w, t)
+    dev.forward()
+    assert dev.sync_status() == 0
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    dout = torch.randn(dev.q.shape, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    dq, dk, dv = torch.empty_like(dev.q), torch.empty_like(dev.k), torch.empty_like(dev.v)
+    del dev.ws
+    ws = PB.alloc_workspace(dev.p, PB.OP_BSA_BWD)
+    P.pisa_bsa_bwd(dev.p, dev.q, dev.k, dev.v, dev.idx, dev.out, dev.lse, dout, dq, dk, dv, ws)
+    torch.cuda.synchronize()
+    assert P.read_status(ws) == 0
+    G = w.G
+    # identities, per (b, KV head), in fp64 on the device
+    dv_sum = dv.double().sum(dim=1)                                              # [B, Hkv, d]
+    do_sum = dout.double().view(w.B, w.N, w.Hkv, G, w.d).sum(dim=(1, 3))         # [B, Hkv, d]
+    scale_v = dout.double().abs().view(w.B, w.N, w.Hkv, G, w.d).sum(dim=(1, 3))
+    assert bool(((dv_sum - do_sum).abs() <= 2.0 ** -8 * scale_v).all())
+    dk_sum = dk.double().sum(dim=1)
+    assert bool((dk_sum.abs() <= 2.0 ** -8 * dk.double().abs().sum(dim=1)).all())
+    # sampled rows
+    tri = S.sample_queries(w, 10)
+    prob = T.oracle_problem(w, t)
+    ti = torch.from_numpy(tri).cuda()
+    idx_rows = dev.idx[ti[:, 0], ti[:, 1], ti[:, 2]].cpu().numpy()
+    heads = ti[:, 1:2] * G + torch.arange(G, device="cuda")[None, :]
+    do_rows = T.from_torch(dout[ti[:, 0:1], ti[:, 2:3], heads], "bf16")
+    ref = O.attend_backward_dq_rows(prob, tri, idx_rows, do_rows)               # [S, G, d]
+    got = dq[ti[:, 0:1], ti[:, 2:3], heads].double().cpu().numpy()
+    o64 = dev.out[ti[:, 0:1], ti[:, 2:3], heads].double().cpu().numpy()
+    do64 = O.load_storage(do_rows, "bf16")
+    kmax = float(dev.k.abs().max())
+    d_delta = 2.0 ** -9 * np.abs(o64 * do64).sum(axis=-1, keepdims=True) / np.sqrt(w.d) * kmax
+    _close("dq rows", got, ref, d_delta)
