@@ -108,8 +108,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
   __shared__ uint64_t bar_mma;
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_fail;
-  __shared__ int s_ent[128];
-  __shared__ float s_nlse2[128], s_delta[128];
+  __shared__ int s_ent2[2][128];                            // per-tile metadata, two tiles (current, next)
+  __shared__ float s_nlse22[2][128], s_delta2[2][128];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
@@ -155,29 +155,46 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
     });
     const __nv_bfloat16* qb = a.q + (long long)b * geo.qs[0] + (long long)(h * G) * geo.qs[2];
     const __nv_bfloat16* dob = a.dout + (long long)b * geo.os[0] + (long long)(h * G) * geo.os[2];
-    for (int jt = 0; jt < inf.ntiles && !dead; ++jt) {
-      // ---- rows of this tile: entry, -lse*log2e and delta per row
-      if (tid < 128) {
-        const int e = inf.e_begin + jt * tpt + (tid >> lgG);
-        const int ent = (e < inf.e_end) ? a.entries[e] : -1;
-        s_ent[tid] = ent;
-        if (ent >= 0) {
-          const long long li = ((long long)b * geo.Hq + h * G + (tid & (G - 1))) * geo.N + (ent & 0xFFFFFF);
-          s_nlse2[tid] = -a.lse[li] * kLog2e;
-          s_delta[tid] = a.delta[li];
-        }
+    // rows of a tile: entry, -lse*log2e and delta per row (threads 0..127, one row each)
+    auto load_meta = [&](int jt_, int& ent, float& nl, float& dl) {
+      const int e = inf.e_begin + jt_ * tpt + (tid >> lgG);
+      ent = (jt_ < inf.ntiles && e < inf.e_end) ? a.entries[e] : -1;
+      nl = 0.f; dl = 0.f;
+      if (ent >= 0) {
+        const long long li = ((long long)b * geo.Hq + h * G + (tid & (G - 1))) * geo.N + (ent & 0xFFFFFF);
+        nl = -a.lse[li] * kLog2e;
+        dl = a.delta[li];
       }
-      __syncthreads();
+    };
+    auto gather_tile = [&](const int* ents) {
       bwd_load_rows(sQ, A_SLAB, 128, tid, [&](int r) {
-        const int ent = s_ent[r];
+        const int ent = ents[r];
         return (ent >= 0) ? qb + (long long)(ent & 0xFFFFFF) * geo.qs[1] + (long long)(r & (G - 1)) * geo.qs[2]
                           : (const __nv_bfloat16*)nullptr;
       });
       bwd_load_rows(sdO, A_SLAB, 128, tid, [&](int r) {
-        const int ent = s_ent[r];
+        const int ent = ents[r];
         return (ent >= 0) ? dob + (long long)(ent & 0xFFFFFF) * geo.os[1] + (long long)(r & (G - 1)) * geo.os[2]
                           : (const __nv_bfloat16*)nullptr;
       });
+    };
+    // first tile of the item: metadata and gathers up front; later tiles are fetched while the previous
+    // tile's dQ^T is being reduced
+    if (tid < 128) {
+      int ent; float nl, dl;
+      load_meta(0, ent, nl, dl);
+      s_ent2[0][tid] = ent; s_nlse22[0][tid] = nl; s_delta2[0][tid] = dl;
+    }
+    __syncthreads();
+    gather_tile(s_ent2[0]);
+    for (int jt = 0; jt < inf.ntiles && !dead; ++jt) {
+      const int cb = jt & 1;
+      const int* s_ent = s_ent2[cb];
+      const float* s_nlse2 = s_nlse22[cb];
+      const float* s_delta = s_delta2[cb];
+      // next tile's metadata: loads issued now, stored once this tile's products are under way
+      int n_ent = -1; float n_nl = 0.f, n_dl = 0.f;
+      if (tid < 128) load_meta(jt + 1, n_ent, n_nl, n_dl);
       cp_async_wait_all();
       fence_proxy_async_smem();
       __syncthreads();
@@ -282,6 +299,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
         if (__syncthreads_or(!ok)) { s_fail = 1; dead = true; break; }
       }
       tcgen05_fence_after_sync();
+      // Q, dO, P, dS tiles are free: bring in the next tile while this one's dQ^T is reduced
+      if (tid < 128) { s_ent2[cb ^ 1][tid] = n_ent; s_nlse22[cb ^ 1][tid] = n_nl; s_delta2[cb ^ 1][tid] = n_dl; }
+      __syncthreads();
+      if (jt + 1 < inf.ntiles) gather_tile(s_ent2[cb ^ 1]);
       // ---- dQ^T out of TMEM: lane = column d, TMEM column = tile row (entry*G + head); this warp's 64 rows
       {
         float* acc_d = a.dq_acc + (((long long)b * geo.Hkv + h) * geo.N) * (long long)(D * G) + (long long)row * G;
@@ -344,6 +365,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
       __syncthreads();                                       // K, V tiles and the accumulators are free again
     }
   }
+  cp_async_wait_all();                                      // nothing of this CTA's copies may outlive it
   tcgen05_fence_before_sync();
   __syncthreads();
   if (s_fail && tid == 0) atomicExch(a.status, (int)PISA_ERR_TIMEOUT);
