@@ -1,8 +1,6 @@
 // Decoding step (Sec. 3.3 "Decoding", App. B "Decode cache"): one new token per sequence, one launch.
 //
 // A thread-block cluster of eight CTAs serves one (batch, KV head):
-//   0. the first CTA refreshes the cached pyramid along the new token's path: the current leaf's mean
-//      over the keys it holds so far, then each ancestor from its stored children;
 //   1. every CTA walks the intermediate levels L..2 redundantly (identical arithmetic, identical
 //      result; the summaries are a few KB): eight warps score eight candidates each per round on
 //      m16n8k16 fragments, warp 0 applies Select_K and expands;
@@ -11,7 +9,10 @@
 //   3. after a cluster barrier every CTA applies the final Select_K to the same scores;
 //   4. attention over the selected blocks: two warps per block (halves of its keys), scores on the
 //      same fragments, online softmax, P*V on the FMA pipe; partial (max, sum, output) are merged
-//      first inside a CTA through shared memory, then across the cluster through global scratch.
+//      first inside a CTA through shared memory, then across the cluster through global scratch;
+//   5. while the first CTA does the last merge, the last CTA refreshes the cached pyramid along the new
+//      token's path: the current leaf's mean over the keys it holds so far, then each ancestor from its
+//      stored children (nothing in the same step reads these nodes: the path is forced, never scored).
 // Cluster barriers are hardware barriers among co-scheduled CTAs: there is no software spin anywhere.
 // Decoding is bound by the key/value bytes it must read (about (g*K + 2*K)*C*d*2 bytes per KV head),
 // not by arithmetic, which is why nothing here is a CTA-wide tensor-core tile.
@@ -55,29 +56,66 @@ __device__ __forceinline__ float ex2f(float x) {
   return y;
 }
 
-// Step 0: the new token's path.  Thread dd owns output column dd at every level, so the value it
-// reads back from the level below is the one it has just written.
-__device__ void refresh_path(const Geometry& geo, const DecArgs& a, int b, int h) {
-  const int dd = threadIdx.x;
-  if (dd >= geo.d) return;
-  const int c = a.pos / geo.C;
-  const __nv_bfloat16* kb = a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2] + dd;
+// The new token's path in the cached pyramid, by one whole CTA.  Nothing in the same step reads these
+// nodes (the path is forced, never scored), so this runs off the critical path, after the CTA's share
+// of the attention.  The current leaf's mean takes every loaded key in one round (eight warps, sixteen
+// keys each at most per round, a lane owning d/32 columns); the ancestors need one sibling load per
+// level and child, all issued before the dependent chain of means starts.
+__device__ void refresh_path(const Geometry& geo, const DecArgs& a, int b, int h, float* scratch /* [8][128] */) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int d = geo.d, dv = d / 32;
+  const int c = a.pos / geo.C, t0 = c * geo.C, cnt = a.pos - t0 + 1;
+  const __nv_bfloat16* kb = a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2] + lane * dv;
+  float part[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int r0 = warp; r0 < cnt; r0 += kDecWarps * 4) {
+    uint2 raw[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int r = r0 + u * kDecWarps;
+      raw[u] = make_uint2(0u, 0u);
+      if (r < cnt) {
+        const __nv_bfloat16* src = kb + (long long)(t0 + r) * geo.ks[1];
+        if (dv == 4) raw[u] = *reinterpret_cast<const uint2*>(src);
+        else raw[u].x = *reinterpret_cast<const uint32_t*>(src);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      part[0] += __uint_as_float(raw[u].x << 16);
+      part[1] += __uint_as_float(raw[u].x & 0xFFFF0000u);
+      part[2] += __uint_as_float(raw[u].y << 16);
+      part[3] += __uint_as_float(raw[u].y & 0xFFFF0000u);
+    }
+  }
+  for (int j = 0; j < dv; ++j) scratch[warp * 128 + lane * dv + j] = part[j];
+  __syncthreads();
+  const int dd = tid;
+  if (dd >= d) return;
   float s = 0.f;
-  const int t0 = c * geo.C;
-  for (int t = t0; t <= a.pos; ++t) s += __bfloat162float(kb[(long long)t * geo.ks[1]]);
+  for (int w = 0; w < kDecWarps; ++w) s += scratch[w * 128 + dd];
   const long long bh = (long long)b * geo.Hkv + h;
-  __nv_bfloat16* lv = a.pyr + geo.level_off[1] + bh * geo.M[1] * geo.d;
-  lv[(long long)c * geo.d + dd] = __float2bfloat16_rn(s / (float)(a.pos - t0 + 1));
-  int below_last = c;                   // last valid node of the level below (the path's node there)
+  // siblings of the path at every level (stored values of completed nodes), all loads first
+  float sib[kMaxLevels];
+  int nch[kMaxLevels];
+  int below = c;
   for (int l = 2; l <= geo.L; ++l) {
-    const int node = below_last / geo.g;
-    const int lo = node * geo.g, hi = min(lo + geo.g - 1, below_last);
+    const int node = below / geo.g;
+    const int lo = node * geo.g, hi = below;                // valid children: lo .. the path's node
     const __nv_bfloat16* bl = a.pyr + geo.level_off[l - 1] + bh * geo.M[l - 1] * geo.d;
     float acc = 0.f;
-    for (int r = lo; r <= hi; ++r) acc += __bfloat162float(bl[(long long)r * geo.d + dd]);
-    __nv_bfloat16* cur = a.pyr + geo.level_off[l] + bh * geo.M[l] * geo.d;
-    cur[(long long)node * geo.d + dd] = __float2bfloat16_rn(acc / (float)(hi - lo + 1));
-    below_last = node;
+    for (int r = lo; r < hi; ++r) acc += __bfloat162float(bl[(long long)r * geo.d + dd]);
+    sib[l] = acc;
+    nch[l] = hi - lo + 1;
+    below = node;
+  }
+  __nv_bfloat16 cur = __float2bfloat16_rn(s / (float)cnt);
+  a.pyr[geo.level_off[1] + (bh * geo.M[1] + c) * geo.d + dd] = cur;
+  below = c;
+  for (int l = 2; l <= geo.L; ++l) {
+    const int node = below / geo.g;
+    cur = __float2bfloat16_rn((sib[l] + __bfloat162float(cur)) / (float)nch[l]);
+    a.pyr[geo.level_off[l] + (bh * geo.M[l] + node) * geo.d + dd] = cur;
+    below = node;
   }
 }
 
@@ -104,16 +142,30 @@ decode_step_kernel(Geometry geo, DecArgs a) {
   const int c = pos / C;
   const int f1 = (c >= 1) ? c - 1 : 0;
 
-  if (rank == 0) refresh_path(geo, a, b, h);
-
   QFrag<D, NT> qf;
   qf.load(a.q + ((long long)b * geo.Hq + (long long)h * G) * D, D, G, lane);
 
   // ---------------------------------------------------------------- 1. levels L..2
-  if (tid == 0) { s_cand[0][0] = 0; s_n = 1; }
+  // Levels whose live nodes (those that do not start after the query's leaf) number at most K keep
+  // everything, so the walk starts at the highest level that has more, with every child of the live
+  // nodes of the level above as its candidates.
+  int l_top = 1;                                            // level of the first candidate list
+  for (int l = geo.L; l >= 2; --l) {
+    const unsigned sp = (unsigned)min(geo.span[l], (long long)0x7fffffff);
+    if ((int)((unsigned)c / sp) + 1 > K) { l_top = l; break; }
+  }
+  {
+    int n_init = 1;                                         // the root, when the walk starts there
+    if (l_top < geo.L) {
+      const unsigned sp = (unsigned)min(geo.span[l_top + 1], (long long)0x7fffffff);
+      n_init = min(((int)((unsigned)c / sp) + 1) * g, geo.M[l_top]);
+    }
+    for (int s = tid; s < n_init; s += kDecThreads) s_cand[0][s] = s;
+    if (tid == 0) s_n = n_init;
+  }
   __syncthreads();
   int cur = 0;
-  for (int l = geo.L; l >= 2; --l) {
+  for (int l = l_top; l >= 2; --l) {
     const int* cand = s_cand[cur];
     int* next = s_cand[cur ^ 1];
     const int n = s_n;
@@ -400,6 +452,8 @@ decode_step_kernel(Geometry geo, DecArgs a) {
     else { cta_out[G * D + hh] = M; cta_out[G * D + G + hh] = acc; }
   }
   cluster_barrier();
+  // the last CTA refreshes the cached pyramid while the first one merges the partials
+  if (rank == kClu - 1) refresh_path(geo, a, b, h, &s_z[0][0][0]);
   // the first CTA merges the cluster's partials and writes the token's output
   if (rank == 0) {
     const float* parts = a.ws_part + (long long)bh * kClu * W;
