@@ -423,7 +423,7 @@ def run_ours(args):
 
 
 def run_sweep(args):
-    """Routing latency vs N (BASELINE configs[4]) next to the flat O(N^2/C) selector built in the same
+    """Routing latency vs N (the scaling-sweep workload) next to the flat O(N^2/C) selector built in the same
     library, plus the paper's own benchmark shape; one JSON line per (workload, N).  Not the bench line."""
     import torch
 

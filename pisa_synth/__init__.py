@@ -56,14 +56,14 @@ class Workload:
 
 
 WORKLOADS: Dict[str, Workload] = {
-    # configs[0]: tiny fp32 case
+    # tiny fp32 case
     "cfg1": Workload("cfg1", 1, 1024, 1, 1, 64, 64, 2, 4, "fp32", 0, "iid"),
-    # configs[1]: MHA, one planted needle block per head, q scaled by 1/sqrt(d)
+    # MHA, one planted needle block per head, q scaled by 1/sqrt(d)
     "cfg2": Workload("cfg2", 1, 8192, 16, 16, 128, 64, 2, 16, "bf16", 1, "needle1",
                      q_scale=1.0 / math.sqrt(128.0)),
-    # configs[2]: GQA, fan-in 4, random-walk mean
+    # GQA, fan-in 4, random-walk mean
     "cfg3": Workload("cfg3", 2, 32768, 32, 8, 128, 64, 4, 16, "bf16", 2, "walk"),
-    # configs[3]: headline
+    # headline workload
     "cfg4": Workload("cfg4", 1, 131072, 32, 8, 128, 128, 2, 32, "bf16", 3, "needle64"),
     # the paper's own benchmark shape (App. B), for a like-for-like row
     "paper128k": Workload("paper128k", 1, 131072, 32, 2, 64, 64, 2, 8, "bf16", 5, "iid"),
@@ -71,7 +71,7 @@ WORKLOADS: Dict[str, Workload] = {
 
 
 def sweep_workload(N: int) -> Workload:
-    """configs[4]: the scaling sweep, one instance per N."""
+    """The scaling sweep, one instance per N."""
     return Workload(f"cfg5_{N}", 1, N, 16, 4, 128, 64, 2, 16, "bf16", 4, "iid")
 
 
