@@ -636,11 +636,16 @@ def run_quality(args):
         idx = torch.empty((w.B, w.Hkv, w.N, w.K), dtype=torch.int32, device="cuda")
         ws = PB.alloc_workspace(p, PB.OP_FORWARD)
         P.pisa_build_pyramid(p, k, pyramid)
-        if flat:
-            P.pisa_flat_select(p, q, pyramid, idx, ws)
-        else:
-            P.pisa_route(p, q, k, pyramid, idx, None, ws)
+        run = (lambda: P.pisa_flat_select(p, q, pyramid, idx, ws)) if flat else \
+              (lambda: P.pisa_route(p, q, k, pyramid, idx, None, ws))
+        run()
         torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        run()
+        e1.record()
+        torch.cuda.synchronize()
+        select_ms = e0.elapsed_time(e1)
         sel = idx[0][:, torch.from_numpy(pos).cuda()].cpu().numpy()         # [Hkv, S, K]
         rec, rat = [], []
         for h in range(w.Hkv):
@@ -648,7 +653,9 @@ def run_quality(args):
             rec.append(r_)
             rat.append(m_)
         row = {"quality": name, "workload": describe(w), "queries": int(len(pos) * w.Hkv), "K": w.K,
-               "recall_at_k": float(np.mean(rec)), "mass_ratio": float(np.mean(rat)), "status": P.read_status(ws)}
+               "recall_at_k": float(np.mean(rec)), "mass_ratio": float(np.mean(rat)), "select_ms": select_ms,
+               "path": "flat SIMT" if flat else ("tcgen05 + mma.sync" if impl == PB.IMPL_AUTO else "SIMT fp32"),
+               "status": P.read_status(ws)}
         rows.append(row)
         print(json.dumps(row), flush=True)
     return rows
