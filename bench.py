@@ -388,6 +388,13 @@ def run_ours(args):
     per_pair = DRAM_BYTES_PER_PAIR.get(dom)
     pairs = {"leaf_lse_tiles": wc["sel_pairs"], "attention_tiles": wc["sel_pairs"]}.get(dom)
     roof["traffic"] = (per_pair * pairs) if (per_pair and pairs and w.dtype == "bf16") else None
+    # The two tile kernels are limited by what L2 can gather and reduce, not by the tensor pipe: report
+    # that stream too (per selected pair: G*d*2 bytes of query rows L2->SM, and in the attention
+    # kernel G*d*4 bytes of fp32 reductions SM->L2).  Context for `frac`, not a substitute for it.
+    if dom in ("leaf_lse_tiles", "attention_tiles") and w.dtype == "bf16":
+        per_pair_l2 = w.G * w.d * 2 + (w.G * w.d * 4 if dom == "attention_tiles" else 0)
+        roof["l2_stream_bytes"] = per_pair_l2 * wc["sel_pairs"]
+        roof["l2_stream_tbs"] = per_pair_l2 * wc["sel_pairs"] / t_dom / 1e12
     roofs = {}
     for k_, t_ in cand.items():
         b_, w_ = algo[k_]
@@ -629,8 +636,8 @@ def run_quality(args):
             pad[:p_ + 1] = pr
             mass[h, j] = pad.view(M1, w.C).sum(dim=1).cpu().numpy()
     rows = []
-    for name, mode, impl, flat in (("pisa_lse", "lse", PB.IMPL_AUTO, False), ("pisa1_mean", "mean", PB.IMPL_SIMT, False),
-                                   ("pisa2_mean_var", "mean_var", PB.IMPL_SIMT, False), ("flat_mean", "lse", PB.IMPL_AUTO, True)):
+    for name, mode, impl, flat in (("pisa_lse", "lse", PB.IMPL_AUTO, False), ("pisa1_mean", "mean", PB.IMPL_AUTO, False),
+                                   ("pisa2_mean_var", "mean_var", PB.IMPL_AUTO, False), ("flat_mean", "lse", PB.IMPL_AUTO, True)):
         p = P.Params.from_workload(w, score_mode=mode, impl=impl)
         pyramid = PB.alloc_pyramid(p)
         idx = torch.empty((w.B, w.Hkv, w.N, w.K), dtype=torch.int32, device="cuda")

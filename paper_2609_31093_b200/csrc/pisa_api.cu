@@ -213,7 +213,7 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
   st = do_route(p, g, q, k, pyr, idx, nullptr, lse, ws, ws_bytes, s);
   if (st != PISA_OK) return st;
   stage_mark(2, s);
-  st = do_bsa(p, g, q, k, v, idx, out, lse, use_tensor(p, g), ws, ws_bytes, s);
+  st = do_bsa(p, g, q, k, v, idx, out, lse, use_tensor(p, g) && g.score_mode == PISA_SCORE_LSE, ws, ws_bytes, s);
   stage_mark(3, s);
   kernel_mark("end", s);
   return st;

@@ -25,7 +25,8 @@ constexpr int kWarpsPerCta = 4;
 
 }  // namespace
 
-template <int D, int NT, bool G2>
+// MODE: PISA_SCORE_LSE, _MEAN (mean of the children's logits) or _MEAN_VAR (mean + variance / 2), Sec. 4.3
+template <int D, int NT, bool G2, int MODE>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ pyr,
                         int32_t* __restrict__ par_out, float* __restrict__ margin) {
@@ -110,15 +111,20 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
 #pragma unroll
             for (int jh = 0; jh < 2; ++jh) {
               const float za = acc[jh] * geo.scale, zb = acc[2 + jh] * geo.scale;
-              const float lse2 = fmaxf(za, zb) + __logf(1.f + __expf(-fabsf(za - zb)));
-              if (nt * 8 + 2 * tig + jh < G) usum += ok_hi ? lse2 : za;
+              float sc2;
+              if (MODE == PISA_SCORE_LSE) sc2 = fmaxf(za, zb) + __logf(1.f + __expf(-fabsf(za - zb)));
+              else sc2 = 0.5f * (za + zb) + ((MODE == PISA_SCORE_MEAN_VAR) ? 0.125f * (za - zb) * (za - zb) : 0.f);
+              if (nt * 8 + 2 * tig + jh < G) usum += ok_hi ? sc2 : za;
             }
           }
           if (!has) usum = 0.f;
         } else {
-          float m[NT][2], ssum[NT][2];
+          float m[NT][2], ssum[NT][2], sq[NT][2];
 #pragma unroll
-          for (int nt = 0; nt < NT; ++nt) { m[nt][0] = m[nt][1] = -CUDART_INF_F; ssum[nt][0] = ssum[nt][1] = 0.f; }
+          for (int nt = 0; nt < NT; ++nt) {
+            m[nt][0] = m[nt][1] = -CUDART_INF_F; ssum[nt][0] = ssum[nt][1] = 0.f; sq[nt][0] = sq[nt][1] = 0.f;
+          }
+          const int nch = has ? min(g, Mb - node * g) : 1;                 // valid children of the candidate
           for (int r0 = 0; r0 < g; r0 += 2) {
             const int ch_lo = node * g + r0, ch_hi = ch_lo + 1;
             const bool ok_lo = has && ch_lo < Mb, ok_hi = has && (r0 + 1 < g) && ch_hi < Mb;
@@ -139,8 +145,15 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
               // acc[0..1]: child lo, heads nt*8 + 2*tig + {0,1};  acc[2..3]: child hi, same heads
 #pragma unroll
               for (int jh = 0; jh < 2; ++jh) {
-                if (ok_lo) lse_add(m[nt][jh], ssum[nt][jh], acc[jh] * geo.scale);
-                if (ok_hi) lse_add(m[nt][jh], ssum[nt][jh], acc[2 + jh] * geo.scale);
+                if (MODE == PISA_SCORE_LSE) {
+                  if (ok_lo) lse_add(m[nt][jh], ssum[nt][jh], acc[jh] * geo.scale);
+                  if (ok_hi) lse_add(m[nt][jh], ssum[nt][jh], acc[2 + jh] * geo.scale);
+                } else {
+                  // m: the first child's logit (shift); ssum, sq: first and second moments about it
+                  if (r0 == 0) m[nt][jh] = acc[jh] * geo.scale;
+                  if (ok_lo) { const float dl = acc[jh] * geo.scale - m[nt][jh]; ssum[nt][jh] += dl; sq[nt][jh] += dl * dl; }
+                  if (ok_hi) { const float dl = acc[2 + jh] * geo.scale - m[nt][jh]; ssum[nt][jh] += dl; sq[nt][jh] += dl * dl; }
+                }
               }
             }
           }
@@ -148,7 +161,14 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
           for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int jh = 0; jh < 2; ++jh)
-              if (nt * 8 + 2 * tig + jh < G && has) usum += m[nt][jh] + __logf(ssum[nt][jh]);
+              if (nt * 8 + 2 * tig + jh < G && has) {
+                if (MODE == PISA_SCORE_LSE) usum += m[nt][jh] + __logf(ssum[nt][jh]);
+                else {
+                  const float mu = ssum[nt][jh] / (float)nch;
+                  usum += m[nt][jh] + mu +
+                          ((MODE == PISA_SCORE_MEAN_VAR) ? 0.5f * fmaxf(sq[nt][jh] / (float)nch - mu * mu, 0.f) : 0.f);
+                }
+              }
         }
         usum += __shfl_xor_sync(0xffffffffu, usum, 1);
         usum += __shfl_xor_sync(0xffffffffu, usum, 2);
@@ -204,17 +224,29 @@ static int launch_dn(const Geometry& g, const void* q, const void* pyr, int32_t*
   const long long total = (long long)g.B * g.Hkv * g.N;
   const long long ctas = (total + kWarpsPerCta - 1) / kWarpsPerCta;
   if (ctas > 0x7fffffffLL) return PISA_ERR_UNSUPPORTED;
-  if (g.g == 2)
-    route_stage1_mma_kernel<D, NT, true><<<(unsigned)ctas, kWarpsPerCta * 32, 0, s>>>(
-        g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pyr, par, margin);
-  else
-    route_stage1_mma_kernel<D, NT, false><<<(unsigned)ctas, kWarpsPerCta * 32, 0, s>>>(
-        g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pyr, par, margin);
+  auto go = [&](auto kern) {
+    kern<<<(unsigned)ctas, kWarpsPerCta * 32, 0, s>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pyr, par, margin);
+  };
+  const bool g2 = g.g == 2;
+  switch (g.score_mode) {
+    case PISA_SCORE_LSE:
+      if (g2) go(route_stage1_mma_kernel<D, NT, true, PISA_SCORE_LSE>);
+      else go(route_stage1_mma_kernel<D, NT, false, PISA_SCORE_LSE>);
+      break;
+    case PISA_SCORE_MEAN:
+      if (g2) go(route_stage1_mma_kernel<D, NT, true, PISA_SCORE_MEAN>);
+      else go(route_stage1_mma_kernel<D, NT, false, PISA_SCORE_MEAN>);
+      break;
+    default:
+      if (g2) go(route_stage1_mma_kernel<D, NT, true, PISA_SCORE_MEAN_VAR>);
+      else go(route_stage1_mma_kernel<D, NT, false, PISA_SCORE_MEAN_VAR>);
+      break;
+  }
   return check_launch("route_stage1_mma");
 }
 
 bool route_stage1_mma_supported(const Geometry& g, int dtype) {
-  return dtype == PISA_BF16 && g.score_mode == PISA_SCORE_LSE && (g.d == 64 || g.d == 128) && g.L >= 2 &&
+  return dtype == PISA_BF16 && (g.d == 64 || g.d == 128) && g.L >= 2 &&
          g.G <= 16;
 }
 

@@ -172,6 +172,7 @@ struct TileArgs {
   const int32_t* item_key;
   const int32_t* entries;
   int nkeys, Mk, NW, fan, slots;
+  int mode;                // score written per (leaf, head): PISA_SCORE_LSE (also what attention needs), MEAN, MEAN_VAR
   float* blk_lse;          // [BH, N, slots*fan, G]   (tile_lse)
   const float* row_lse;    // [B, Hq, N]              (tile_pv)
   float* o_acc;            // fp32 accumulator: [B, Hkv, N, D, G] when the second product is transposed, else [B, N, Hq, D]
@@ -238,6 +239,18 @@ __device__ __forceinline__ void lse_chunk_masked(const uint32_t (&rr)[32], int n
     if (j < nvalid) acc += ex2_approx(fmaf(__uint_as_float(rr[j]), sl2, neg));
   ssum = ssum * ex2_approx(m - mn) + acc;
   m = mn;
+}
+// first and second moments of the first `nvalid` of 32 logits about `shift` (score modes "mean" and
+// "mean + variance/2", Sec. 4.3)
+__device__ __forceinline__ void stat_chunk(const uint32_t (&rr)[32], int nvalid, float scale, float shift, float& s1,
+                                           float& s2) {
+#pragma unroll
+  for (int j = 0; j < 32; ++j)
+    if (j < nvalid) {
+      const float dlt = fmaf(__uint_as_float(rr[j]), scale, -shift);
+      s1 += dlt;
+      s2 = fmaf(dlt, dlt, s2);
+    }
 }
 
 // ------------------------------------------------------------------ warp-specialised tile kernels
@@ -462,6 +475,7 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
     const int head = row & (G - 1);
     const int r_lo = (a.fan >= 2) ? half * (a.fan / 2) : 0;
     const int r_hi = (a.fan >= 2) ? ((half == 1) ? a.fan : a.fan / 2) : (half == 0 ? 1 : 0);
+    const bool lse_mode = a.mode == PISA_SCORE_LSE;
     int it = 0;
     for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x) {
       const ItemInfo inf = item_info(a, item, tpt);
@@ -483,13 +497,17 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
             ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
           const bool fast = __all_sync(0xffffffffu, ncols == C || ncols == 0);
           float m = -CUDART_INF_F, ssum = 0.f;
+          float shift = 0.f, s1 = 0.f, s2 = 0.f;          // moment modes: logits about the first one
           uint32_t ra[32], rb[32];
           const uint32_t col0 = lane_base + (uint32_t)(r * C);
           tmem_ld_32x32(col0, ra);
           for (int c0 = 0; c0 < C; c0 += 64) {
             tmem_ld_wait();
             tmem_ld_32x32(col0 + (uint32_t)(c0 + 32), rb);
-            if (fast) lse_chunk(ra, sl2, m, ssum);
+            if (!lse_mode) {
+              if (c0 == 0) shift = __uint_as_float(ra[0]) * geo.scale;
+              if (c0 < ncols) stat_chunk(ra, ncols - c0, geo.scale, shift, s1, s2);
+            } else if (fast) lse_chunk(ra, sl2, m, ssum);
             else if (c0 < ncols) lse_chunk_masked(ra, ncols - c0, sl2, m, ssum);
             tmem_ld_wait();
             if (c0 + 64 < C) tmem_ld_32x32(col0 + (uint32_t)(c0 + 64), ra);
@@ -499,11 +517,17 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
               tcgen05_fence_before_sync();
               mbar_arrive(&t_empty[grp]);
             }
-            if (fast) lse_chunk(rb, sl2, m, ssum);
+            if (!lse_mode) {
+              if (c0 + 32 < ncols) stat_chunk(rb, ncols - c0 - 32, geo.scale, shift, s1, s2);
+            } else if (fast) lse_chunk(rb, sl2, m, ssum);
             else if (c0 + 32 < ncols) lse_chunk_masked(rb, ncols - c0 - 32, sl2, m, ssum);
           }
           if (valid) {
-            const float lse = (ncols > 0) ? (m + log2f(ssum)) * kLn2 : -CUDART_INF_F;
+            float lse = (ncols > 0) ? (m + log2f(ssum)) * kLn2 : -CUDART_INF_F;
+            if (!lse_mode && ncols > 0) {
+              const float inv_n = 1.f / (float)ncols, mu = s1 * inv_n;
+              lse = shift + mu + ((a.mode == PISA_SCORE_MEAN_VAR) ? 0.5f * fmaxf(s2 * inv_n - mu * mu, 0.f) : 0.f);
+            }
             a.blk_lse[(((long long)bh * geo.N + t) * (a.slots * a.fan) + slot * a.fan + r) * G + head] = lse;
           }
         }
@@ -1211,7 +1235,7 @@ int launch_bwd(const Geometry& g, const BwdArgs& a, cudaStream_t s) {
 }  // namespace
 
 bool tensor_path_supported(const Geometry& g, int dtype) {
-  if (dtype != PISA_BF16 || g.score_mode != PISA_SCORE_LSE) return false;
+  if (dtype != PISA_BF16) return false;
   if (g.d != 64 && g.d != 128) return false;
   if (g.C != 64 && g.C != 128) return false;
   const int nb = g.g * g.C;
@@ -1242,13 +1266,15 @@ int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, con
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = nullptr;
   a.entry_off = inv.entry_off; a.tile_off = inv.tile_off; a.item_off = inv.item_off; a.item_key = inv.item_key; a.entries = inv.entries;
   a.nkeys = g.B * g.Hkv * inv.NW * g.M[2]; a.Mk = g.M[2]; a.NW = inv.NW; a.fan = g.g; a.slots = g.K;
-  a.blk_lse = blk; a.status = status;
+  a.blk_lse = blk; a.status = status; a.mode = g.score_mode;
   kernel_mark("leaf_lse_tiles", s);
   st = dispatch_tile_lse(g, g.g * g.C, a, s);
   if (st != PISA_OK) return st;
   kernel_mark("final_topk", s);
   const long long total = (long long)g.B * g.Hkv * g.N;
-  final_topk_kernel<<<(unsigned)((total + 3) / 4), 128, 0, s>>>(g, par, blk, idx, margin, lse_out);
+  // only the LSE scores are also the per-leaf softmax denominators the attention stage can reuse
+  final_topk_kernel<<<(unsigned)((total + 3) / 4), 128, 0, s>>>(g, par, blk, idx, margin,
+                                                                (g.score_mode == PISA_SCORE_LSE) ? lse_out : nullptr);
   return check_launch("final_topk");
 }
 

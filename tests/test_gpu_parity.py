@@ -151,20 +151,32 @@ def test_flat_select_matches_oracle(case):
     assert n_bad == 0
 
 
+@pytest.mark.parametrize("impl", [PB.IMPL_SIMT, PB.IMPL_AUTO])
 @pytest.mark.parametrize("mode", ["mean", "mean_var"])
-def test_score_modes_match_oracle(mode):
-    w = SMALL["gqa4_ragged"]
+@pytest.mark.parametrize("name", ["gqa4_ragged", "fan4", "c128_k32"])
+def test_score_modes_match_oracle(name, mode, impl):
+    """PISA-1 / PISA-2 scores (Sec. 4.3) on the exact-fp32 path and on the tensor-core path; the forward
+    with these modes must also attend correctly (no LSE hand-over from routing in these modes)."""
+    w = SMALL[name]
     t = S.make_inputs(w)
     prob = T.oracle_problem(w, t, mode=mode)
-    tri = S.sample_queries(w, 150)
-    dev = T.Device(w, t, impl=PB.IMPL_SIMT, score_mode=mode)
+    tri = S.sample_queries(w, 150 if w.N < 8192 else 40)
+    dev = T.Device(w, t, impl=impl, score_mode=mode)
     dev.load_oracle_pyramid(prob.pyramid())
     dev.route()
     assert dev.sync_status() == 0
     got = T.gather_idx(dev.idx, tri)
+    T.check_index_rows_valid(got, tri, w)
     ref_idx, ref_margin = prob.route_all(tri)
     n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin)
-    assert n_bad == 0
+    assert n_bad == 0, f"{n_bad} rows differ outside the tie band"
+    dev.forward()
+    assert dev.sync_status() == 0
+    got = T.gather_idx(dev.idx, tri)
+    same = ~np.any(got != ref_idx, axis=1)
+    out_ref, lse_ref = prob.attend_all(tri[same], ref_idx[same])
+    out_gpu, lse_gpu = T.gather_out(dev, tri[same])
+    T.check_outputs(out_gpu, lse_gpu, out_ref, lse_ref, w.dtype)
 
 
 def test_dense_limit_equals_torch_causal_attention():
