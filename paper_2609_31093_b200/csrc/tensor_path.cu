@@ -357,7 +357,9 @@ __device__ __forceinline__ bool prod_sync_or(bool flag) {
   return any != 0;
 }
 
-template <int D, int NB>
+// MOM: false = per-head LSE of every leaf; true = first / second moments of the logits (score modes
+// "mean" and "mean + variance/2"), a separate instantiation so that the LSE one keeps its registers.
+template <int D, int NB, bool MOM>
 __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, TileArgs a) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int NS = 4;
@@ -475,7 +477,7 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
     const int head = row & (G - 1);
     const int r_lo = (a.fan >= 2) ? half * (a.fan / 2) : 0;
     const int r_hi = (a.fan >= 2) ? ((half == 1) ? a.fan : a.fan / 2) : (half == 0 ? 1 : 0);
-    const bool lse_mode = a.mode == PISA_SCORE_LSE;
+    constexpr bool lse_mode = !MOM;
     int it = 0;
     for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x) {
       const ItemInfo inf = item_info(a, item, tpt);
@@ -1167,13 +1169,17 @@ int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char
   return st;
 }
 
+template <int D, int NB, bool MOM>
+int launch_tile_lse_m(const Geometry& g, const TileArgs& a, cudaStream_t s) {
+  const size_t smem = (size_t)(D / 64) * (4 * 128 * 128 + NB * 128) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(lse_ws_kernel<D, NB, MOM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) { record_cuda_error("lse_ws attr", e); return PISA_ERR_CUDA; }
+  lse_ws_kernel<D, NB, MOM><<<num_sms(), kLseThreads, smem, s>>>(g, a);
+  return check_launch("lse_ws");
+}
 template <int D, int NB>
 int launch_tile_lse(const Geometry& g, const TileArgs& a, cudaStream_t s) {
-  const size_t smem = (size_t)(D / 64) * (4 * 128 * 128 + NB * 128) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(lse_ws_kernel<D, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) { record_cuda_error("lse_ws attr", e); return PISA_ERR_CUDA; }
-  lse_ws_kernel<D, NB><<<num_sms(), kLseThreads, smem, s>>>(g, a);
-  return check_launch("lse_ws");
+  return (a.mode == PISA_SCORE_LSE) ? launch_tile_lse_m<D, NB, false>(g, a, s) : launch_tile_lse_m<D, NB, true>(g, a, s);
 }
 
 int dispatch_tile_lse(const Geometry& g, int nb, const TileArgs& a, cudaStream_t s) {
