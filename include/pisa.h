@@ -142,6 +142,27 @@ int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const voi
                  int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Packed variable-length batches: `nseq` sequences laid back to back along the token axis.
+ * Boundary rule (the paper leaves packed inputs open): every sequence has its own block grid that
+ * starts at its first token, its own hierarchy and its own causal order; nothing is shared across
+ * sequences, i.e. the result is what pisa_forward gives on each sequence alone.
+ *
+ *   p           : B must be 1 and strides dense; p->N is the LONGEST sequence (it sizes the pyramid
+ *                 scratch and the workspace)
+ *   cu_seqlens  : HOST int32 [nseq + 1], cu[0] = 0, non-decreasing; sequence i is tokens cu[i]..cu[i+1]-1
+ *                 (empty sequences are skipped)
+ *   q, out      : device [total, Hq, d];  k, v : device [total, Hkv, d]   (total = cu[nseq])
+ *   pyramid     : device scratch sized by pisa_pyramid_layout for p (overwritten per sequence)
+ *   idx         : device int32, sequence-major: sequence i's [Hkv, len_i, K] block starts at element
+ *                 Hkv * K * cu[i]; block ids are relative to the sequence
+ *   lse         : device float, sequence-major: sequence i's [Hq, len_i] block starts at Hq * cu[i]
+ *   ws          : device workspace sized for PISA_OP_FORWARD with p (N = the longest sequence)
+ */
+int pisa_forward_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32_t nseq, const void* q,
+                        const void* k, const void* v, void* pyramid, int32_t* idx, void* out, float* lse,
+                        void* ws, size_t ws_bytes, void* stream);
+
+/*
  * The same forward pass for callers that hold HOST tensors.  KV heads are independent units of the
  * path (Sec. 3.3: one selected set per KV head), so the call walks them one at a time: the strided
  * slice of q, k, v that belongs to head h is copied into one of two slots of the device arena

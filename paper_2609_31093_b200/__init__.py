@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     pisa_bsa_fwd,
     pisa_forward,
     pisa_forward_host,
+    pisa_forward_packed,
     pisa_flat_select,
     pisa_bsa_bwd,
     pisa_decode_step,

@@ -58,6 +58,7 @@ def lib():
     L.pisa_decode_step.argtypes = [pp, C.c_int32, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
     L.pisa_pyramid_regrow.argtypes = [pp, pp, vp, vp, vp]
     L.pisa_bsa_bwd.argtypes = [pp] + [vp] * 11 + [C.c_size_t, vp]
+    L.pisa_forward_packed.argtypes = [pp, i32p, C.c_int32] + [vp] * 8 + [C.c_size_t, vp]
     L.pisa_read_status.argtypes = [vp, i32p]
     L.pisa_route_static.argtypes = [pp, vp, vp, vp, vp, vp, vp]
     L.pisa_route_static.restype = C.c_int
@@ -69,7 +70,7 @@ def lib():
     L.pisa_get_kernel_ms.restype = C.c_int
     for name in ("pisa_pyramid_layout", "pisa_workspace_bytes", "pisa_build_pyramid", "pisa_route",
                  "pisa_bsa_fwd", "pisa_forward", "pisa_forward_host", "pisa_flat_select", "pisa_read_status",
-                 "pisa_decode_step", "pisa_pyramid_regrow", "pisa_bsa_bwd",
+                 "pisa_decode_step", "pisa_pyramid_regrow", "pisa_bsa_bwd", "pisa_forward_packed",
                  "pisa_set_stage_timing", "pisa_get_stage_ms"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -174,6 +175,14 @@ def pisa_bsa_fwd(p: Params, q, k, v, idx, out, lse, ws):
 def pisa_forward(p: Params, q, k, v, pyramid, idx, out, lse, ws):
     _check(lib().pisa_forward(p.ref(), _ptr(q), _ptr(k), _ptr(v), _ptr(pyramid), _ptr(idx), _ptr(out),
                               _ptr(lse), _ptr(ws), ws.numel(), _stream()), "pisa_forward")
+
+
+def pisa_forward_packed(p: Params, cu_seqlens, q, k, v, pyramid, idx, out, lse, ws):
+    """Packed variable-length batch; cu_seqlens is a host sequence of nseq + 1 offsets, p.N the longest length."""
+    cu = (C.c_int32 * len(cu_seqlens))(*[int(x) for x in cu_seqlens])
+    _check(lib().pisa_forward_packed(p.ref(), cu, len(cu_seqlens) - 1, _ptr(q), _ptr(k), _ptr(v), _ptr(pyramid),
+                                     _ptr(idx), _ptr(out), _ptr(lse), _ptr(ws), ws.numel(), _stream()),
+           "pisa_forward_packed")
 
 
 def pisa_forward_host(p: Params, q_host, k_host, v_host, out_host, lse_host, idx_host, ws):

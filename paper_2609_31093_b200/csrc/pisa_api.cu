@@ -334,6 +334,43 @@ int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const voi
   return do_forward(p, g, q, k, v, pyramid, idx, out, lse, ws, ws_bytes, (cudaStream_t)stream);
 }
 
+int pisa_forward_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32_t nseq, const void* q,
+                        const void* k, const void* v, void* pyramid, int32_t* idx, void* out, float* lse,
+                        void* ws, size_t ws_bytes, void* stream) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (!cu_seqlens || nseq < 0 || !q || !k || !v || !pyramid || !idx || !out || !lse || !ws || misaligned(q) ||
+      misaligned(k) || misaligned(v) || misaligned(pyramid) || misaligned(out) || misaligned(ws))
+    return PISA_ERR_INVALID_ARG;
+  if (p->B != 1 || cu_seqlens[0] != 0) return PISA_ERR_INVALID_ARG;
+  for (int i = 0; i < 3; ++i)
+    if (p->q_stride[i] || p->k_stride[i] || p->v_stride[i] || p->o_stride[i]) return PISA_ERR_INVALID_ARG;
+  for (int i = 0; i < nseq; ++i) {
+    const int len = cu_seqlens[i + 1] - cu_seqlens[i];
+    if (len < 0 || len > p->N) return PISA_ERR_INVALID_ARG;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  st = clear_status(ws, s);
+  if (st != PISA_OK) return st;
+  const size_t es = elem_size(p->dtype);
+  for (int i = 0; i < nseq; ++i) {
+    const size_t t0 = (size_t)cu_seqlens[i];
+    const int len = cu_seqlens[i + 1] - cu_seqlens[i];
+    if (len == 0) continue;
+    pisa_params_t pi = *p;
+    pi.N = len;
+    Geometry gi;
+    st = resolve(&pi, &gi);
+    if (st != PISA_OK) return st;
+    st = do_forward(&pi, gi, (const char*)q + t0 * g.Hq * g.d * es, (const char*)k + t0 * g.Hkv * g.d * es,
+                    (const char*)v + t0 * g.Hkv * g.d * es, pyramid, idx + t0 * g.Hkv * g.K,
+                    (char*)out + t0 * g.Hq * g.d * es, lse + t0 * g.Hq, ws, ws_bytes, s, /*clear=*/false);
+    if (st != PISA_OK) return st;
+  }
+  return PISA_OK;
+}
+
 int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_host, const void* v_host,
                       void* out_host, float* lse_host, int32_t* idx_host, void* ws, size_t ws_bytes,
                       void* stream) {

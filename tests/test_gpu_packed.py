@@ -1,0 +1,57 @@
+"""Packed variable-length batches: every sequence of the pack must come out exactly as pisa_forward gives it
+alone (own block grid, own hierarchy), and sampled rows must match the oracle run on that sequence."""
+import numpy as np
+import pytest
+import torch
+
+import pisa_synth as S
+
+pytestmark = pytest.mark.gpu
+
+import pisa_testlib as T  # noqa: E402
+import paper_2609_31093_b200 as P  # noqa: E402
+from paper_2609_31093_b200 import binding as PB  # noqa: E402
+
+
+def test_packed_sequences_equal_the_sequences_alone_and_the_oracle():
+    lens = [700, 64, 1, 2085, 0, 130, 4096]
+    Hq, Hkv, d, C, g, K = 8, 2, 128, 64, 2, 4
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    total = int(cu[-1])
+    parts = []
+    for i, n in enumerate(lens):
+        parts.append(S.make_inputs(S.Workload(f"pk{i}", 1, max(n, 1), Hq, Hkv, d, C, g, K, "bf16", 700 + i, "iid")))
+    cat = lambda key: np.concatenate([p_[key][0, :n] for p_, n in zip(parts, lens)], axis=0)
+    q, k, v = (T.to_torch(cat(x), "bf16") for x in ("q", "k", "v"))          # [total, H, d]
+    p = P.Params(1, max(lens), Hq, Hkv, d, C, g, K, dtype="bf16")
+    pyramid = PB.alloc_pyramid(p)
+    ws = PB.alloc_workspace(p, PB.OP_FORWARD)
+    idx = torch.full((Hkv * K * total,), -7, dtype=torch.int32, device="cuda")
+    out = torch.zeros_like(q)
+    lse = torch.zeros((Hq * total,), dtype=torch.float32, device="cuda")
+    P.pisa_forward_packed(p, cu.tolist(), q, k, v, pyramid, idx, out, lse, ws)
+    torch.cuda.synchronize()
+    assert P.read_status(ws) == 0
+    for i, n in enumerate(lens):
+        if n == 0:
+            continue
+        t0 = int(cu[i])
+        w = S.Workload(f"pk{i}", 1, n, Hq, Hkv, d, C, g, K, "bf16", 700 + i, "iid")
+        t = {key: parts[i][key][:, :n] for key in ("q", "k", "v")}
+        alone = T.Device(w, t)
+        alone.forward()
+        assert alone.sync_status() == 0
+        got_idx = idx[Hkv * K * t0:Hkv * K * (t0 + n)].view(Hkv, n, K)
+        got_lse = lse[Hq * t0:Hq * (t0 + n)].view(Hq, n)
+        assert torch.equal(got_idx, alone.idx[0]), i
+        assert torch.allclose(got_lse, alone.lse[0], rtol=1e-5, atol=1e-5), i
+        a, b = out[t0:t0 + n].double(), alone.out[0].double()
+        assert bool(((a - b).abs() <= 2.0 ** -7 * b.abs() + 1e-3).all()), i
+        # sampled rows of this sequence against the oracle
+        tri = S.sample_queries(w, 12)
+        prob = T.oracle_problem(w, t)
+        ref_idx, ref_margin = prob.route_all(tri)
+        ti = torch.from_numpy(tri)
+        gi = got_idx.cpu()[ti[:, 1], ti[:, 2]].numpy()
+        n_diff, n_bad, n_band = T.compare_index_sets(gi, ref_idx, ref_margin)
+        assert n_bad == 0, i
