@@ -730,7 +730,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
-    ap.add_argument("--ref-queries", type=int, default=192)
+    ap.add_argument("--ref-queries", type=int, default=1024)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="routing latency vs N and the flat selector (not the bench line)")
