@@ -23,6 +23,10 @@ SMALL = {
     "c128_k32": S.Workload("c128_k32", 1, 16384, 4, 1, 128, 128, 2, 32, "bf16", 105, "needle64"),
     "one_block": S.Workload("one_block", 1, 50, 2, 1, 32, 64, 2, 4, "fp32", 106, "iid"),
     "g3_odd": S.Workload("g3_odd", 1, 1000, 2, 1, 32, 24, 3, 5, "fp32", 107, "iid"),
+    # two token windows with a ragged second one, the largest candidate count the kernels take (g*K = 128)
+    "two_windows_gk128": S.Workload("two_windows_gk128", 1, 16384 + 1024 + 77, 4, 1, 64, 64, 4, 32, "bf16", 109, "iid"),
+    # eight heads per group, batch 2, C = 128
+    "g8_b2": S.Workload("g8_b2", 2, 5000, 8, 1, 128, 128, 2, 8, "bf16", 110, "walk"),
 }
 FULL = ["tiny_fp32", "gqa4_ragged", "mha_k3_fp32", "one_block", "g3_odd"]   # every query compared
 
