@@ -132,3 +132,19 @@ def test_decode_rejects_what_it_does_not_support():
     p = P.Params(1, 1024, 2, 2, 64, 64, 2, 4, dtype="fp32")
     with pytest.raises(P.PisaError, match="unsupported"):
         P.workspace_bytes(p, PB.OP_DECODE)
+
+
+def test_decode_long_context_uses_both_parts_of_the_walk():
+    """More than 1024 past nodes at the lower levels: the upper levels are walked from the cluster-wide
+    dense scores, the lower ones candidate by candidate."""
+    w = S.Workload("dec_long_c32", 1, 72000, 2, 1, 64, 32, 2, 4, "bf16", 405, "iid")
+    t = S.make_inputs(w)
+    n0 = w.N - 40
+    cache = Cache(w, t, cap=w.N, filled=n0)
+    P.pisa_build_pyramid(cache.p, cache.k, cache.pyr)
+    in_band = 0
+    for pos in range(n0, w.N):
+        cache.step(pos)
+        if pos % 4 == 0 or pos == w.N - 1:
+            in_band += _check_step(cache, t, pos)
+    print(f"[long] rows inside the tie band: {in_band}")
