@@ -134,9 +134,8 @@ def test_decode_rejects_what_it_does_not_support():
         P.workspace_bytes(p, PB.OP_DECODE)
 
 
-def test_decode_long_context_uses_both_parts_of_the_walk():
-    """More than 1024 past nodes at the lower levels: the upper levels are walked from the cluster-wide
-    dense scores, the lower ones candidate by candidate."""
+def test_decode_long_context():
+    """A deep hierarchy (2250 leaves, twelve levels, ten of them pruning) continued from a prefill-built cache."""
     w = S.Workload("dec_long_c32", 1, 72000, 2, 1, 64, 32, 2, 4, "bf16", 405, "iid")
     t = S.make_inputs(w)
     n0 = w.N - 40
