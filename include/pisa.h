@@ -191,7 +191,7 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
  *                    three gradients; partial sums are added with fp32 reductions, so results are
  *                    reproducible to fp32 rounding, not bitwise)
  *
- * bf16, d = 128, C in {64, 128}, g*C in {128, 256}; other configurations return
+ * bf16, d in {64, 128}, C in {64, 128}, g*C in {128, 256}; other configurations return
  * PISA_ERR_UNSUPPORTED.  Asynchronous on `stream`.
  */
 int pisa_bsa_bwd(const pisa_params_t* p, const void* q, const void* k, const void* v, const int32_t* idx,

@@ -1,4 +1,4 @@
-// Backward of the block-sparse attention with the selected indices held fixed (App. B), d = 128.
+// Backward of the block-sparse attention with the selected indices held fixed (App. B), d = 128 or 64.
 // Included by tensor_path.cu inside its unnamed namespace: it works on the same inverted
 // (key block -> tokens) lists, work items and operand layouts as the forward attention kernel.
 //
@@ -14,6 +14,9 @@
 // read-out has d along the TMEM lanes: a warp's reduction covers 32 consecutive floats.
 // TMEM: S / dQ^T at columns 0..127 (dQ^T reuses S once P and dS are in shared memory), dP at
 // 128.., dV^T at 256.., dK^T at 384...  delta = rowsum(dO o O) comes from a small kernel of its own.
+// d = 64 runs on the same M = 128 shapes: rows are staged as 128 columns with the upper 64 zero, and only
+// the first 64 TMEM lanes of the gradients are read out (half of the tensor work is padding; the kernel is
+// bound by its gathers and reductions, not by the tensor pipe).
 #pragma once
 
 constexpr int kBwdThreads = 256;
@@ -65,12 +68,12 @@ __global__ void __launch_bounds__(256) bwd_convert_kernel(const float* __restric
 
 // 256 threads copy `nrows` rows of 256 bytes ([row][128 bf16]) into two swizzled K-major slabs of
 // `slab_bytes` each; src_of(row) returns the row's address or nullptr (zero fill).
-template <typename F>
+template <int CHV, typename F>                              // CHV: 16-byte chunks a source row really has (d / 8)
 __device__ __forceinline__ void bwd_load_rows(uint8_t* dst, int slab_bytes, int nrows, int p, F src_of) {
   const int ck = p & 15, rb = p >> 4;                       // 16-byte chunk of the row, first row
   uint32_t d = smem_u32(dst + (ck >> 3) * slab_bytes) + swz128(rb, ck & 7);
   for (int row = rb; row < nrows; row += 16) {              // row % 8 is the same for all of a thread's rows
-    const __nv_bfloat16* src = src_of(row);
+    const __nv_bfloat16* src = (ck < CHV) ? src_of(row) : nullptr;
     if (src != nullptr) cp_async16(d, src + ck * 8);
     else st_shared_zero16(d);
     d += 16 * 128;
@@ -91,10 +94,11 @@ __device__ __forceinline__ ItemInfo item_info_keys(const int32_t* item_key, cons
   return r;
 }
 
-template <int C>
+template <int C, int DIN>
 __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, BwdArgs a) {
   extern __shared__ uint8_t smem_raw[];
-  constexpr int D = 128;
+  constexpr int D = 128;                                    // staged (padded) head dimension
+  constexpr int CHV = DIN / 8;
   constexpr int A_SLAB = 128 * 128;                         // one 64-column slab of a 128-row tile
   constexpr int KV_SLAB = C * 128;
   constexpr int P_BYTES = (C / 64) * A_SLAB;
@@ -145,11 +149,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
     const int b = bh / geo.Hkv, h = bh % geo.Hkv;
     const __nv_bfloat16* kb = a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2];
     const __nv_bfloat16* vb = a.v + (long long)b * geo.vs[0] + (long long)h * geo.vs[2];
-    bwd_load_rows(sK, KV_SLAB, C, tid, [&](int r) {
+    bwd_load_rows<CHV>(sK, KV_SLAB, C, tid, [&](int r) {
       const int t = leaf * C + r;
       return (t < geo.N) ? kb + (long long)t * geo.ks[1] : (const __nv_bfloat16*)nullptr;
     });
-    bwd_load_rows(sV, KV_SLAB, C, tid, [&](int r) {
+    bwd_load_rows<CHV>(sV, KV_SLAB, C, tid, [&](int r) {
       const int t = leaf * C + r;
       return (t < geo.N) ? vb + (long long)t * geo.vs[1] : (const __nv_bfloat16*)nullptr;
     });
@@ -167,12 +171,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
       }
     };
     auto gather_tile = [&](const int* ents) {
-      bwd_load_rows(sQ, A_SLAB, 128, tid, [&](int r) {
+      bwd_load_rows<CHV>(sQ, A_SLAB, 128, tid, [&](int r) {
         const int ent = ents[r];
         return (ent >= 0) ? qb + (long long)(ent & 0xFFFFFF) * geo.qs[1] + (long long)(r & (G - 1)) * geo.qs[2]
                           : (const __nv_bfloat16*)nullptr;
       });
-      bwd_load_rows(sdO, A_SLAB, 128, tid, [&](int r) {
+      bwd_load_rows<CHV>(sdO, A_SLAB, 128, tid, [&](int r) {
         const int ent = ents[r];
         return (ent >= 0) ? dob + (long long)(ent & 0xFFFFFF) * geo.os[1] + (long long)(r & (G - 1)) * geo.os[2]
                           : (const __nv_bfloat16*)nullptr;
@@ -305,8 +309,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
       if (jt + 1 < inf.ntiles) gather_tile(s_ent2[cb ^ 1]);
       // ---- dQ^T out of TMEM: lane = column d, TMEM column = tile row (entry*G + head); this warp's 64 rows
       {
-        float* acc_d = a.dq_acc + (((long long)b * geo.Hkv + h) * geo.N) * (long long)(D * G) + (long long)row * G;
-        const long long tok_stride = (long long)D * G;
+        float* acc_d = a.dq_acc + (((long long)b * geo.Hkv + h) * geo.N) * (long long)(DIN * G) + (long long)row * G;
+        const long long tok_stride = (long long)DIN * G;
+        const bool live = row < DIN;                          // lanes beyond d hold padding
 #pragma unroll
         for (int cc = 0; cc < 64; cc += 32) {
           const int c0 = chalf * 64 + cc;
@@ -318,7 +323,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
             for (int q4 = 0; q4 < 8; ++q4) {
               const int col = c0 + 4 * q4;
               const int ent_c = s_ent[col];
-              if (ent_c >= 0) {
+              if (ent_c >= 0 && live) {
                 float* dst = acc_d + (long long)(ent_c & 0xFFFFFF) * tok_stride + (col & (G - 1));
                 asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst),
                              "f"(__uint_as_float(r[4 * q4])), "f"(__uint_as_float(r[4 * q4 + 1])),
@@ -331,7 +336,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
             for (int q1 = 0; q1 < 32; ++q1) {
               const int col = c0 + q1;
               const int ent_c = s_ent[col];
-              if (ent_c >= 0)
+              if (ent_c >= 0 && live)
                 atomicAdd(acc_d + (long long)(ent_c & 0xFFFFFF) * tok_stride + (col & (G - 1)), __uint_as_float(r[q1]));
             }
           }
@@ -354,8 +359,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const int t = leaf * C + c0 + j;
-          if (t < geo.N) {
-            const long long o = (((long long)b * geo.N + t) * geo.Hkv + h) * D + row;
+          if (t < geo.N && row < DIN) {
+            const long long o = (((long long)b * geo.N + t) * geo.Hkv + h) * DIN + row;
             atomicAdd(a.dv_acc + o, __uint_as_float(rv[j]));
             atomicAdd(a.dk_acc + o, __uint_as_float(rk[j]));
           }

@@ -16,7 +16,7 @@ int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, con
 int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const void* v, const int32_t* idx,
                void* out, float* lse, bool lse_ready, void* ws, int32_t* status, cudaStream_t s);
 
-// backward of the block-sparse attention with frozen indices (d = 128); dq [B,N,Hq,d], dk, dv [B,N,Hkv,d] dense
+// backward of the block-sparse attention with frozen indices; dq [B,N,Hq,d], dk, dv [B,N,Hkv,d] dense
 bool tensor_bwd_supported(const Geometry& g, int dtype);
 size_t tensor_bwd_workspace_bytes(const Geometry& g);
 int tensor_bsa_bwd(const Geometry& g, const void* q, const void* k, const void* v, const int32_t* idx,

@@ -1229,12 +1229,12 @@ BwdLayout bwd_layout(const Geometry& g) {
   return r;
 }
 
-template <int C>
+template <int C, int DIN>
 int launch_bwd(const Geometry& g, const BwdArgs& a, cudaStream_t s) {
   const size_t smem = 4 * (size_t)(128 * 128) + 2 * (size_t)(C / 64) * (128 * 128) + 4 * (size_t)(C * 128) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(bsa_bwd_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(bsa_bwd_kernel<C, DIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("bsa_bwd attr", e); return PISA_ERR_CUDA; }
-  bsa_bwd_kernel<C><<<num_sms(), kBwdThreads, smem, s>>>(g, a);
+  bsa_bwd_kernel<C, DIN><<<num_sms(), kBwdThreads, smem, s>>>(g, a);
   return check_launch("bsa_bwd");
 }
 
@@ -1327,7 +1327,7 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
 }
 
 bool tensor_bwd_supported(const Geometry& g, int dtype) {
-  return tensor_path_supported(g, dtype) && g.d == 128;
+  return tensor_path_supported(g, dtype);                  // d in {64, 128}
 }
 size_t tensor_bwd_workspace_bytes(const Geometry& g) { return bwd_layout(g).total; }
 
@@ -1361,7 +1361,8 @@ int tensor_bsa_bwd(const Geometry& g, const void* q, const void* k, const void* 
     if (st != PISA_OK) return st;
   }
   kernel_mark("backward_tiles", s);
-  st = (g.C == 128) ? launch_bwd<128>(g, a, s) : launch_bwd<64>(g, a, s);
+  if (g.d == 128) st = (g.C == 128) ? launch_bwd<128, 128>(g, a, s) : launch_bwd<64, 128>(g, a, s);
+  else st = (g.C == 128) ? launch_bwd<128, 64>(g, a, s) : launch_bwd<64, 64>(g, a, s);
   if (st != PISA_OK) return st;
   kernel_mark("convert_gradients", s);
   {

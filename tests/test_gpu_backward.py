@@ -27,6 +27,8 @@ CASES = {
     "gqa4_c128": S.Workload("bwd_gqa4_c128", 1, 1536, 4, 1, 128, 128, 2, 3, "bf16", 602, "iid"),
     "mha_c64_fan4_b2": S.Workload("bwd_mha_c64", 2, 640, 2, 2, 128, 64, 4, 5, "bf16", 603, "walk"),
     "g16_c128": S.Workload("bwd_g16_c128", 1, 768, 16, 1, 128, 128, 2, 4, "bf16", 604, "iid"),
+    "d64_c64_g16": S.Workload("bwd_d64_c64", 1, 1100, 16, 1, 64, 64, 2, 4, "bf16", 605, "iid"),
+    "d64_c128_gqa2": S.Workload("bwd_d64_c128", 1, 900, 4, 2, 64, 128, 2, 3, "bf16", 606, "walk"),
 }
 
 
@@ -73,7 +75,7 @@ def test_backward_matches_oracle(name):
 
 
 def test_backward_rejects_unsupported_head_dim():
-    p = P.Params(1, 1024, 4, 2, 64, 64, 2, 4)
+    p = P.Params(1, 1024, 4, 2, 32, 64, 2, 4)
     with pytest.raises(P.PisaError, match="unsupported"):
         P.workspace_bytes(p, PB.OP_BSA_BWD)
 
