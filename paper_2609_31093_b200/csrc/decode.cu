@@ -364,10 +364,14 @@ decode_step_kernel(Geometry geo, DecArgs a) {
         const int t = key0 + kt + kk;
 #pragma unroll
         for (int j = 0; j < DV / 2; ++j) vraw[kk][j] = 0u;
-        if (t <= pos) {
-          const uint32_t* vr = reinterpret_cast<const uint32_t*>(vbh + (long long)t * geo.vs[1] + lane * DV);
-#pragma unroll
-          for (int j = 0; j < DV / 2; ++j) vraw[kk][j] = vr[j];
+        if (t <= pos) {                                    // one 8-byte (d = 128) or 4-byte (d = 64) load per row
+          const __nv_bfloat16* vr = vbh + (long long)t * geo.vs[1] + lane * DV;
+          if (DV == 4) {
+            const uint2 x = *reinterpret_cast<const uint2*>(vr);
+            vraw[kk][0] = x.x; vraw[kk][DV / 2 - 1] = x.y;
+          } else {
+            vraw[kk][0] = *reinterpret_cast<const uint32_t*>(vr);
+          }
         }
       }
       float z[NT][4];
