@@ -21,7 +21,7 @@ using namespace frag;
 
 namespace {
 
-constexpr int kWarpsPerCta = 4;
+constexpr int kWarpsPerCta = 8;
 
 }  // namespace
 
