@@ -950,8 +950,13 @@ __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int
       if (ok) {
         if (leaf == 0 || leaf == f1 || leaf == c) sc = forced_score(ci);
         else {
-          sc = 0.f;
-          for (int hh = 0; hh < G; ++hh) sc += bl[ci * G + hh];
+          if (G == 4) {                        // the group's four per-head scores in one 16-byte load
+            const float4 x = *reinterpret_cast<const float4*>(bl + ci * 4);
+            sc = (x.x + x.y) + (x.z + x.w);
+          } else {
+            sc = 0.f;
+            for (int hh = 0; hh < G; ++hh) sc += bl[ci * G + hh];
+          }
         }
       }
       u[ci] = sc;
@@ -1002,9 +1007,9 @@ __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int
       m = warp_max(m);
       float ssum = 0.f;
       for (int s0 = 0, ch = 0; s0 < gK; s0 += 32, ++ch)
-        if ((kept_mask[ch] >> lane) & 1u) ssum += expf(bl[(s0 + lane) * G + hh] - m);
+        if ((kept_mask[ch] >> lane) & 1u) ssum += __expf(bl[(s0 + lane) * G + hh] - m);
       ssum = warp_sum(ssum);
-      if (lane == 0) lse_out[((long long)b * geo.Hq + h * G + hh) * geo.N + t] = m + logf(ssum);
+      if (lane == 0) lse_out[((long long)b * geo.Hq + h * G + hh) * geo.N + t] = m + __logf(ssum);
     }
   }
 }
