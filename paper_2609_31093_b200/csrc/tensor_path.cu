@@ -51,6 +51,7 @@ struct InvArgs {
   int32_t* item_off;      // [nkeys + 1]  work items: runs of at most kItemTiles tiles of one list
   int32_t* item_key;      // [items]      the list each work item belongs to
   int32_t* cursor;        // [nkeys]
+  int32_t* blk_tot;       // [3][ceil(nkeys / 1024) + 1] scan scratch: per-block totals, then block offsets
   int32_t* entries;       // [<= BH*N*K]  token | slot << 24
 };
 
@@ -83,39 +84,92 @@ __global__ void __launch_bounds__(256) inv_count_kernel(InvArgs a, int use_smem)
   }
 }
 
-// exclusive scans of the list lengths (entries), of their tile counts and of their work-item
-// counts; one CTA
-__global__ void __launch_bounds__(1024) inv_scan_kernel(InvArgs a) {
-  __shared__ int s_e[1024], s_t[1024], s_i[1024];
-  const int nkeys = a.BH * a.NW * a.Mk;
-  const int per = (nkeys + 1023) / 1024;
-  const int lo = min(nkeys, (int)threadIdx.x * per), hi = min(nkeys, lo + per);
-  int se = 0, st = 0, si = 0;
-  for (int i = lo; i < hi; ++i) {
-    const int c = a.count[i];
-    const int tl = (c + a.tpt - 1) / a.tpt;
-    se += c; st += tl; si += (tl + kItemTiles - 1) / kItemTiles;
+// Exclusive scans of the list lengths (entries), of their tile counts and of their work-item counts,
+// in three launches: per-block scans of 1024 lists each, a scan of the block totals, the fix-up.
+__device__ __forceinline__ int3 inv_key_counts(const InvArgs& a, int i, int nkeys) {
+  if (i >= nkeys) return make_int3(0, 0, 0);
+  const int c = a.count[i];
+  const int tl = (c + a.tpt - 1) / a.tpt;
+  return make_int3(c, tl, (tl + kItemTiles - 1) / kItemTiles);
+}
+// inclusive scan of three ints over the 1024 threads of a CTA (warp shuffles, then the warp totals)
+__device__ __forceinline__ int3 block_scan3(int3 v, int3* s_w /* [32] */) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int x = __shfl_up_sync(0xffffffffu, v.x, o), y = __shfl_up_sync(0xffffffffu, v.y, o),
+              z = __shfl_up_sync(0xffffffffu, v.z, o);
+    if (lane >= o) { v.x += x; v.y += y; v.z += z; }
   }
-  s_e[threadIdx.x] = se; s_t[threadIdx.x] = st; s_i[threadIdx.x] = si;
+  if (lane == 31) s_w[warp] = v;
   __syncthreads();
-  for (int o = 1; o < 1024; o <<= 1) {
-    int ve = 0, vt = 0, vi = 0;
-    if ((int)threadIdx.x >= o) { ve = s_e[threadIdx.x - o]; vt = s_t[threadIdx.x - o]; vi = s_i[threadIdx.x - o]; }
-    __syncthreads();
-    s_e[threadIdx.x] += ve; s_t[threadIdx.x] += vt; s_i[threadIdx.x] += vi;
-    __syncthreads();
+  if (warp == 0) {
+    int3 w = s_w[lane];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int x = __shfl_up_sync(0xffffffffu, w.x, o), y = __shfl_up_sync(0xffffffffu, w.y, o),
+                z = __shfl_up_sync(0xffffffffu, w.z, o);
+      if (lane >= o) { w.x += x; w.y += y; w.z += z; }
+    }
+    s_w[lane] = w;
   }
-  int be = s_e[threadIdx.x] - se, bt = s_t[threadIdx.x] - st, bi = s_i[threadIdx.x] - si;
-  for (int i = lo; i < hi; ++i) {
-    const int c = a.count[i];
-    const int tl = (c + a.tpt - 1) / a.tpt;
-    a.entry_off[i] = be; a.tile_off[i] = bt; a.item_off[i] = bi; a.cursor[i] = be;
-    const int ni = (tl + kItemTiles - 1) / kItemTiles;
-    for (int x = 0; x < ni; ++x) a.item_key[bi + x] = i;
-    be += c; bt += tl; bi += ni;
+  __syncthreads();
+  if (warp > 0) { const int3 p = s_w[warp - 1]; v.x += p.x; v.y += p.y; v.z += p.z; }
+  return v;
+}
+__global__ void __launch_bounds__(1024) inv_scan_blocks_kernel(InvArgs a) {
+  __shared__ int3 s_w[32];
+  const int nkeys = a.BH * a.NW * a.Mk;
+  const int nblk = (nkeys + 1023) / 1024;
+  const int i = blockIdx.x * 1024 + threadIdx.x;
+  const int3 own = inv_key_counts(a, i, nkeys);
+  const int3 inc = block_scan3(own, s_w);
+  if (i < nkeys) {                                         // exclusive prefix inside the block, for now
+    a.entry_off[i] = inc.x - own.x; a.tile_off[i] = inc.y - own.y; a.item_off[i] = inc.z - own.z;
   }
   if (threadIdx.x == 1023) {
-    a.entry_off[nkeys] = s_e[1023]; a.tile_off[nkeys] = s_t[1023]; a.item_off[nkeys] = s_i[1023];
+    a.blk_tot[blockIdx.x] = inc.x; a.blk_tot[(nblk + 1) + blockIdx.x] = inc.y;
+    a.blk_tot[2 * (nblk + 1) + blockIdx.x] = inc.z;
+  }
+}
+// block totals -> exclusive block offsets (entry [nblk] = grand total); one CTA walks them 1024 at a time
+__global__ void __launch_bounds__(1024) inv_scan_totals_kernel(InvArgs a) {
+  __shared__ int3 s_w[32];
+  const int nkeys = a.BH * a.NW * a.Mk;
+  const int nblk = (nkeys + 1023) / 1024;
+  int3 carry = make_int3(0, 0, 0);
+  for (int b0 = 0; b0 < nblk; b0 += 1024) {
+    const int j = b0 + threadIdx.x;
+    int3 own = make_int3(0, 0, 0);
+    if (j < nblk) own = make_int3(a.blk_tot[j], a.blk_tot[(nblk + 1) + j], a.blk_tot[2 * (nblk + 1) + j]);
+    __syncthreads();                                       // s_w of the previous round has been read
+    const int3 inc = block_scan3(own, s_w);
+    if (j < nblk) {
+      a.blk_tot[j] = carry.x + inc.x - own.x; a.blk_tot[(nblk + 1) + j] = carry.y + inc.y - own.y;
+      a.blk_tot[2 * (nblk + 1) + j] = carry.z + inc.z - own.z;
+    }
+    const int3 tot = s_w[31];
+    carry.x += tot.x; carry.y += tot.y; carry.z += tot.z;
+  }
+  if (threadIdx.x == 0) {
+    a.blk_tot[nblk] = carry.x; a.blk_tot[(nblk + 1) + nblk] = carry.y; a.blk_tot[2 * (nblk + 1) + nblk] = carry.z;
+  }
+}
+__global__ void __launch_bounds__(1024) inv_scan_fix_kernel(InvArgs a) {
+  const int nkeys = a.BH * a.NW * a.Mk;
+  const int nblk = (nkeys + 1023) / 1024;
+  const int i = blockIdx.x * 1024 + threadIdx.x;
+  if (i < nkeys) {
+    const int be = a.entry_off[i] + a.blk_tot[blockIdx.x];
+    const int bt = a.tile_off[i] + a.blk_tot[(nblk + 1) + blockIdx.x];
+    const int bi = a.item_off[i] + a.blk_tot[2 * (nblk + 1) + blockIdx.x];
+    a.entry_off[i] = be; a.tile_off[i] = bt; a.item_off[i] = bi; a.cursor[i] = be;
+    const int ni = inv_key_counts(a, i, nkeys).z;
+    for (int x = 0; x < ni; ++x) a.item_key[bi + x] = i;
+  }
+  if (i == 0) {
+    a.entry_off[nkeys] = a.blk_tot[nblk]; a.tile_off[nkeys] = a.blk_tot[(nblk + 1) + nblk];
+    a.item_off[nkeys] = a.blk_tot[2 * (nblk + 1) + nblk];
   }
 }
 
@@ -1086,7 +1140,7 @@ __global__ void __launch_bounds__(256) convert_out_heads_inner_kernel(Geometry g
 // ------------------------------------------------------------------ host side
 
 struct InvLayout {
-  size_t count, entry_off, tile_off, item_off, item_key, cursor, entries, end;
+  size_t count, entry_off, tile_off, item_off, item_key, cursor, blk_tot, entries, end;
 };
 
 int window_tokens(const Geometry& g) { return g.N < kWindowTok ? ((g.N + kInvTok - 1) / kInvTok) * kInvTok : kWindowTok; }
@@ -1104,6 +1158,7 @@ InvLayout inv_layout(size_t base, const Geometry& g, int Mk) {
   const size_t max_tiles = (size_t)g.B * g.Hkv * g.N * g.K / (128 / g.G) + nkeys;
   l.item_key = o; o += align_up((max_tiles / kItemTiles + nkeys + 1) * 4, 256);
   l.cursor = o; o += align_up(nkeys * 4, 256);
+  l.blk_tot = o; o += align_up(3 * ((nkeys + 1023) / 1024 + 1) * 4, 256);
   l.entries = o; o += align_up((size_t)g.B * g.Hkv * g.N * g.K * 4, 256);
   l.end = o;
   return l;
@@ -1151,6 +1206,7 @@ int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char
   a.tile_off = (int32_t*)(ws + l.tile_off); a.item_off = (int32_t*)(ws + l.item_off);
   a.item_key = (int32_t*)(ws + l.item_key);
   a.cursor = (int32_t*)(ws + l.cursor);
+  a.blk_tot = (int32_t*)(ws + l.blk_tot);
   a.entries = (int32_t*)(ws + l.entries);
   const size_t nkeys = (size_t)a.BH * a.NW * Mk;
   cudaError_t e = cudaMemsetAsync(a.count, 0, nkeys * 4, s);
@@ -1165,8 +1221,15 @@ int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char
   inv_count_kernel<<<grid, 256, sm_count, s>>>(a, use_smem);
   int st = check_launch("inv_count");
   if (st != PISA_OK) return st;
-  inv_scan_kernel<<<1, 1024, 0, s>>>(a);
-  st = check_launch("inv_scan");
+  const unsigned nblk = (unsigned)((nkeys + 1023) / 1024);
+  inv_scan_blocks_kernel<<<nblk, 1024, 0, s>>>(a);
+  st = check_launch("inv_scan_blocks");
+  if (st != PISA_OK) return st;
+  inv_scan_totals_kernel<<<1, 1024, 0, s>>>(a);
+  st = check_launch("inv_scan_totals");
+  if (st != PISA_OK) return st;
+  inv_scan_fix_kernel<<<nblk, 1024, 0, s>>>(a);
+  st = check_launch("inv_scan_fix");
   if (st != PISA_OK) return st;
   inv_fill_kernel<<<grid, 256, sm_fill, s>>>(a, use_smem);
   st = check_launch("inv_fill");
