@@ -1,5 +1,6 @@
 /*
- * libpisa — forward hot path of Pyramid Sparse Attention (PISA) on NVIDIA B200 (sm_100a).
+ * libpisa — Pyramid Sparse Attention (PISA) on NVIDIA B200 (sm_100a): the forward hot path (pyramid,
+ * routing, block-sparse attention), the decoding step and the attention backward.
  *
  * C ABI.  Every pointer is caller-owned.  "device" pointers are CUDA global memory of the
  * current device, "host" pointers are ordinary host memory.  The library never allocates or
