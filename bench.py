@@ -34,8 +34,8 @@ UNIT = "tokens/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per selected (token, block) pair, from the ncu captures
 # summarised under profiles/ (B=1 Hq=8 Hkv=2 d=128 N=65536 C=128 g=2 K=32: 4.19 M pairs per launch)
-DRAM_BYTES_PER_PAIR = {"leaf_lse_tiles": (208.961536e6 + 106.553600e6) / 4194304.0,
-                       "attention_tiles": (1226.759e6 + 939.463936e6) / 4194304.0}
+DRAM_BYTES_PER_PAIR = {"leaf_lse_tiles": (209.686784e6 + 108.383232e6) / 4194304.0,
+                       "attention_tiles": (1216.039e6 + 934.548736e6) / 4194304.0}
 
 
 def get_workload(name: str) -> S.Workload:
