@@ -15,6 +15,8 @@ CASES = {
     "cfg3": (S.WORKLOADS["cfg3"], 20),
     "cfg4": (S.WORKLOADS["cfg4"], 40),
     "cfg5_32768": (S.sweep_workload(32768), 40),
+    # the longest context of the paper's scaling experiment: 64 inversion windows, 8192 leaves
+    "cfg5_1048576": (S.sweep_workload(1048576), 6),
 }
 
 
