@@ -1,11 +1,12 @@
 // Decoding step (Sec. 3.3 "Decoding", App. B "Decode cache"): one new token per sequence, one launch.
 //
-// A thread-block cluster of eight CTAs serves one (batch, KV head):
+// A thread-block cluster of eight CTAs (four or two once the batch alone fills the GPU, so that every
+// cluster is resident at once) serves one (batch, KV head):
 //   1. every CTA walks the intermediate levels L..2 redundantly (identical arithmetic, identical
 //      result; the summaries are a few KB): eight warps score eight candidates each per round on
 //      m16n8k16 fragments, warp 0 applies Select_K and expands;
 //   2. the leaf candidates (at most g*K blocks of C raw keys, the only large read of the selection) are
-//      spread over the cluster's 64 warps, one block per warp and round; scores meet in global scratch;
+//      spread over the cluster's warps, one block per warp and round; scores meet in global scratch;
 //   3. after a cluster barrier every CTA applies the final Select_K to the same scores;
 //   4. attention over the selected blocks: two warps per block (halves of its keys), scores on the
 //      same fragments, online softmax, P*V on the FMA pipe; partial (max, sum, output) are merged
@@ -27,7 +28,7 @@ using namespace frag;
 
 namespace {
 
-constexpr int kClu = 8;                 // CTAs per cluster
+constexpr int kCluMax = 8;              // CTAs per cluster, at most (scratch is laid out for this many)
 constexpr int kDecWarps = 8;
 constexpr int kDecThreads = kDecWarps * 32;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -43,7 +44,7 @@ struct DecArgs {
   __nv_bfloat16* out;                   // [B, Hq, d]
   float* lse;                           // [B, Hq]
   float* ws_u;                          // [B*Hkv][kMaxCand] leaf scores
-  float* ws_part;                       // [B*Hkv][kClu][G*d + 2*G] attention partials
+  float* ws_part;                       // [B*Hkv][kCluMax][G*d + 2*G] attention partials
 };
 
 __device__ __forceinline__ void cluster_barrier() {
@@ -121,8 +122,9 @@ __device__ void refresh_path(const Geometry& geo, const DecArgs& a, int b, int h
 
 // MINB = 1: all registers to one CTA per SM (lowest latency, small batches); MINB = 2: two CTAs per SM so
 // that the latency-bound phases of different clusters overlap once the grid exceeds the SM count.
-template <int D, int NT, int MINB>
-__global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kDecThreads, MINB)
+// CLU: CTAs per cluster.
+template <int D, int NT, int MINB, int CLU>
+__global__ void __cluster_dims__(CLU, 1, 1) __launch_bounds__(kDecThreads, MINB)
 decode_step_kernel(Geometry geo, DecArgs a) {
   extern __shared__ float s_part[];                       // [kDecWarps][G*D + 2*G] attention partials
   __shared__ int s_cand[2][kMaxCand];
@@ -252,7 +254,7 @@ decode_step_kernel(Geometry geo, DecArgs a) {
   const __nv_bfloat16* kbh = a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2];
   const __nv_bfloat16* vbh = a.v + (long long)b * geo.vs[0] + (long long)h * geo.vs[2];
   if (prune1) {
-    for (int ci = rank * kDecWarps + warp; ci < nV1; ci += kClu * kDecWarps) {
+    for (int ci = rank * kDecWarps + warp; ci < nV1; ci += CLU * kDecWarps) {
       const int leaf = cand1[ci];
       if (leaf == 0 || leaf == f1 || leaf == c) continue;        // forced: never scored
       // a scored leaf lies strictly before the current one: all C keys exist and are visible
@@ -335,9 +337,9 @@ decode_step_kernel(Geometry geo, DecArgs a) {
   __syncthreads();
 
   // ---------------------------------------------------------------- 4. attention
-  // warp gw of the cluster takes block gw/2, keys [half*C/2, (half+1)*C/2) of it
+  // warp gw of the cluster takes the half blocks gw, gw + (warps in the cluster), ...: half block sh is
+  // keys [half*C/2, (half+1)*C/2) of selected block sh/2; the online softmax state runs across them
   const int gw = rank * kDecWarps + warp;
-  const int slot = gw >> 1, half = gw & 1;
   const int nsel = s_nsel;
   constexpr int DV = D / 32;                               // output columns per lane
   const int W = G * D + 2 * G;                             // floats per partial: o[G][D], m[G], l[G]
@@ -348,7 +350,8 @@ decode_step_kernel(Geometry geo, DecArgs a) {
     for (int j = 0; j < DV; ++j) o_acc[hh][j] = 0.f;
   float m_run = -CUDART_INF_F, l_run = 0.f;                // lanes 0..G-1: running max (base 2) / sum of head `lane`
   const float sl2 = geo.scale * kLog2e;
-  if (slot < nsel) {
+  for (int sh = gw; sh < 2 * nsel; sh += CLU * kDecWarps) {
+    const int slot = sh >> 1, half = sh & 1;
     const int leaf = s_sel[slot];
     const int key0 = leaf * C + half * (C / 2);
     for (int kt = 0; kt < C / 2; kt += 16) {
@@ -441,7 +444,7 @@ decode_step_kernel(Geometry geo, DecArgs a) {
   if (lane < G) { mine[G * D + lane] = m_run; mine[G * D + G + lane] = l_run; }
   __syncthreads();
   // CTA partial: merge the eight warps
-  float* cta_out = a.ws_part + ((long long)bh * kClu + rank) * W;
+  float* cta_out = a.ws_part + ((long long)bh * kCluMax + rank) * W;
   for (int e = tid; e < G * D + G; e += kDecThreads) {
     const bool is_o = e < G * D;
     const int hh = is_o ? e / D : e - G * D;
@@ -457,16 +460,16 @@ decode_step_kernel(Geometry geo, DecArgs a) {
   }
   cluster_barrier();
   // the last CTA refreshes the cached pyramid while the first one merges the partials
-  if (rank == kClu - 1) refresh_path(geo, a, b, h, &s_z[0][0][0]);
+  if (rank == CLU - 1) refresh_path(geo, a, b, h, &s_z[0][0][0]);
   // the first CTA merges the cluster's partials and writes the token's output
   if (rank == 0) {
-    const float* parts = a.ws_part + (long long)bh * kClu * W;
+    const float* parts = a.ws_part + (long long)bh * kCluMax * W;
     for (int e = tid; e < G * D; e += kDecThreads) {
       const int hh = e / D;
       float M = -CUDART_INF_F;
-      for (int r = 0; r < kClu; ++r) M = fmaxf(M, __ldcg(parts + r * W + G * D + hh));
+      for (int r = 0; r < CLU; ++r) M = fmaxf(M, __ldcg(parts + r * W + G * D + hh));
       float acc = 0.f, den = 0.f;
-      for (int r = 0; r < kClu; ++r) {
+      for (int r = 0; r < CLU; ++r) {
         const float mr = __ldcg(parts + r * W + G * D + hh);
         if (mr > -CUDART_INF_F) {
           const float f = ex2f(mr - M);
@@ -480,15 +483,17 @@ decode_step_kernel(Geometry geo, DecArgs a) {
   }
 }
 
-template <int D, int NT, int MINB>
+template <int D, int NT, int MINB, int CLU>
 int launch_dnb(const Geometry& g, const DecArgs& a, cudaStream_t s) {
   const size_t smem = (size_t)kDecWarps * (g.G * D + 2 * g.G) * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(decode_step_kernel<D, NT, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(decode_step_kernel<D, NT, MINB, CLU>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("decode_step attr", e); return PISA_ERR_CUDA; }
-  decode_step_kernel<D, NT, MINB><<<dim3(kClu, (unsigned)(g.B * g.Hkv)), kDecThreads, smem, s>>>(g, a);
+  decode_step_kernel<D, NT, MINB, CLU><<<dim3(CLU, (unsigned)(g.B * g.Hkv)), kDecThreads, smem, s>>>(g, a);
   return check_launch("decode_step");
 }
+// Eight CTAs per (batch, KV head) while all clusters fit the GPU at once (one, then two CTAs per SM);
+// beyond that narrower clusters, so that a large batch still runs as a single wave.
 template <int D, int NT>
 int launch_dn(const Geometry& g, const DecArgs& a, cudaStream_t s) {
   static int sms = 0;
@@ -497,7 +502,11 @@ int launch_dn(const Geometry& g, const DecArgs& a, cudaStream_t s) {
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   }
-  return ((long long)g.B * g.Hkv * kClu > sms) ? launch_dnb<D, NT, 2>(g, a, s) : launch_dnb<D, NT, 1>(g, a, s);
+  const long long units = (long long)g.B * g.Hkv;
+  if (units * 8 <= sms) return launch_dnb<D, NT, 1, 8>(g, a, s);
+  if (units * 8 <= 2LL * sms) return launch_dnb<D, NT, 2, 8>(g, a, s);
+  if (units * 4 <= 2LL * sms) return launch_dnb<D, NT, 2, 4>(g, a, s);
+  return launch_dnb<D, NT, 2, 2>(g, a, s);
 }
 
 }  // namespace
@@ -510,7 +519,7 @@ bool decode_supported(const Geometry& g, int dtype) {
 size_t decode_workspace_bytes(const Geometry& g) {
   const size_t bh = (size_t)g.B * g.Hkv;
   return align_up(bh * kMaxCand * sizeof(float), 256) +
-         align_up(bh * kClu * (size_t)(g.G * g.d + 2 * g.G) * sizeof(float), 256);
+         align_up(bh * kCluMax * (size_t)(g.G * g.d + 2 * g.G) * sizeof(float), 256);
 }
 
 int launch_decode_step(const Geometry& g, int pos, const void* q, const void* k, const void* v, void* pyramid,

@@ -147,3 +147,20 @@ def test_decode_long_context():
         if pos % 4 == 0 or pos == w.N - 1:
             in_band += _check_step(cache, t, pos)
     print(f"[long] rows inside the tie band: {in_band}")
+
+
+@pytest.mark.parametrize("B,Hkv", [(5, 4), (10, 4), (20, 4)])
+def test_decode_large_batches_use_narrower_clusters(B, Hkv):
+    """20, 40 and 80 (batch, KV head) units: eight CTAs per unit at two per SM, then four, then two, where a
+    warp runs its online softmax across several half blocks (2 K = 40 of them per unit)."""
+    w = S.Workload(f"dec_batch{B}", B, 2000, 2 * Hkv, Hkv, 64, 32, 2, 20, "bf16", 406 + B, "iid")
+    t = S.make_inputs(w)
+    n0 = w.N - 12
+    cache = Cache(w, t, cap=w.N, filled=n0)
+    P.pisa_build_pyramid(cache.p, cache.k, cache.pyr)
+    in_band = 0
+    for pos in range(n0, w.N):
+        cache.step(pos)
+        if pos % 4 == 0 or pos == w.N - 1:
+            in_band += _check_step(cache, t, pos)
+    print(f"[batch {B}] rows inside the tie band: {in_band}")
