@@ -192,12 +192,27 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
  *                    three gradients; partial sums are added with fp32 reductions, so results are
  *                    reproducible to fp32 rounding, not bitwise)
  *
- * bf16, d in {64, 128}, C in {64, 128}, g*C in {128, 256}; other configurations return
- * PISA_ERR_UNSUPPORTED.  Asynchronous on `stream`.
+ * bf16, d in {64, 128}, C in {64, 128}; other configurations return PISA_ERR_UNSUPPORTED.
+ * Asynchronous on `stream`.
  */
 int pisa_bsa_bwd(const pisa_params_t* p, const void* q, const void* k, const void* v, const int32_t* idx,
                  const void* out, const float* lse, const void* dout, void* dq, void* dk, void* dv,
                  void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * pisa_bsa_bwd for a packed variable-length batch laid out as for pisa_forward_packed (same boundary
+ * rule: nothing is shared across sequences).
+ *
+ *   p, cu_seqlens, nseq : as for pisa_forward_packed (B = 1, dense strides, p->N the longest sequence)
+ *   q, out, dout, dq    : device [total, Hq, d];  k, v, dk, dv : device [total, Hkv, d]
+ *   idx, lse            : sequence-major, as pisa_forward_packed wrote them
+ *   ws                  : device workspace sized for PISA_OP_BSA_BWD with p
+ *
+ * All sequences are validated before anything is queued; one unsupported sequence fails the call.
+ */
+int pisa_bsa_bwd_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32_t nseq, const void* q,
+                        const void* k, const void* v, const int32_t* idx, const void* out, const float* lse,
+                        const void* dout, void* dq, void* dk, void* dv, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Decoding (Sec. 3.3 "Decoding", App. B "Decode cache"): one new token per sequence, one kernel launch.

@@ -20,6 +20,7 @@ from .binding import (  # noqa: F401
     pisa_forward_packed,
     pisa_flat_select,
     pisa_bsa_bwd,
+    pisa_bsa_bwd_packed,
     pisa_decode_step,
     pisa_pyramid_regrow,
     read_status,

@@ -59,6 +59,7 @@ def lib():
     L.pisa_pyramid_regrow.argtypes = [pp, pp, vp, vp, vp]
     L.pisa_bsa_bwd.argtypes = [pp] + [vp] * 11 + [C.c_size_t, vp]
     L.pisa_forward_packed.argtypes = [pp, i32p, C.c_int32] + [vp] * 8 + [C.c_size_t, vp]
+    L.pisa_bsa_bwd_packed.argtypes = [pp, i32p, C.c_int32] + [vp] * 11 + [C.c_size_t, vp]
     L.pisa_read_status.argtypes = [vp, i32p]
     L.pisa_route_static.argtypes = [pp, vp, vp, vp, vp, vp, vp]
     L.pisa_route_static.restype = C.c_int
@@ -70,7 +71,7 @@ def lib():
     L.pisa_get_kernel_ms.restype = C.c_int
     for name in ("pisa_pyramid_layout", "pisa_workspace_bytes", "pisa_build_pyramid", "pisa_route",
                  "pisa_bsa_fwd", "pisa_forward", "pisa_forward_host", "pisa_flat_select", "pisa_read_status",
-                 "pisa_decode_step", "pisa_pyramid_regrow", "pisa_bsa_bwd", "pisa_forward_packed",
+                 "pisa_decode_step", "pisa_pyramid_regrow", "pisa_bsa_bwd", "pisa_forward_packed", "pisa_bsa_bwd_packed",
                  "pisa_set_stage_timing", "pisa_get_stage_ms"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -198,6 +199,14 @@ def pisa_bsa_bwd(p: Params, q, k, v, idx, out, lse, dout, dq, dk, dv, ws):
     """Gradients of the block-sparse attention for fixed idx; dq, dk, dv are dense outputs."""
     _check(lib().pisa_bsa_bwd(p.ref(), _ptr(q), _ptr(k), _ptr(v), _ptr(idx), _ptr(out), _ptr(lse), _ptr(dout),
                               _ptr(dq), _ptr(dk), _ptr(dv), _ptr(ws), ws.numel(), _stream()), "pisa_bsa_bwd")
+
+
+def pisa_bsa_bwd_packed(p: Params, cu_seqlens, q, k, v, idx, out, lse, dout, dq, dk, dv, ws):
+    """pisa_bsa_bwd over a packed variable-length batch laid out as for pisa_forward_packed."""
+    cu = (C.c_int32 * len(cu_seqlens))(*[int(x) for x in cu_seqlens])
+    _check(lib().pisa_bsa_bwd_packed(p.ref(), cu, len(cu_seqlens) - 1, _ptr(q), _ptr(k), _ptr(v), _ptr(idx),
+                                     _ptr(out), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(ws),
+                                     ws.numel(), _stream()), "pisa_bsa_bwd_packed")
 
 
 def pisa_decode_step(p: Params, pos: int, q, k_cache, v_cache, pyramid, idx, out, lse, ws):

@@ -484,6 +484,58 @@ int pisa_bsa_bwd(const pisa_params_t* p, const void* q, const void* k, const voi
   return st;
 }
 
+int pisa_bsa_bwd_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32_t nseq, const void* q,
+                        const void* k, const void* v, const int32_t* idx, const void* out, const float* lse,
+                        const void* dout, void* dq, void* dk, void* dv, void* ws, size_t ws_bytes, void* stream) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (!cu_seqlens || nseq < 0 || !q || !k || !v || !idx || !out || !lse || !dout || !dq || !dk || !dv || !ws)
+    return PISA_ERR_INVALID_ARG;
+  if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(out) || misaligned(dout) || misaligned(dq) ||
+      misaligned(dk) || misaligned(dv) || misaligned(ws))
+    return PISA_ERR_INVALID_ARG;
+  if (p->B != 1 || cu_seqlens[0] != 0) return PISA_ERR_INVALID_ARG;
+  for (int i = 0; i < 3; ++i)
+    if (p->q_stride[i] || p->k_stride[i] || p->v_stride[i] || p->o_stride[i]) return PISA_ERR_INVALID_ARG;
+  if (p->impl == PISA_IMPL_SIMT) return PISA_ERR_UNSUPPORTED;
+  // everything is checked before anything is queued
+  for (int i = 0; i < nseq; ++i) {
+    const int len = cu_seqlens[i + 1] - cu_seqlens[i];
+    if (len < 0 || len > p->N) return PISA_ERR_INVALID_ARG;
+    if (len == 0) continue;
+    pisa_params_t pi = *p;
+    pi.N = len;
+    Geometry gi;
+    st = resolve(&pi, &gi);
+    if (st != PISA_OK) return st;
+    if (!tensor_bwd_supported(gi, p->dtype)) return PISA_ERR_UNSUPPORTED;
+    if (ws_bytes < kStatusBytes + tensor_bwd_workspace_bytes(gi)) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  st = clear_status(ws, s);
+  if (st != PISA_OK) return st;
+  g_mark_n = 0;
+  const size_t es = elem_size(p->dtype);
+  for (int i = 0; i < nseq; ++i) {
+    const size_t t0 = (size_t)cu_seqlens[i];
+    const int len = cu_seqlens[i + 1] - cu_seqlens[i];
+    if (len == 0) continue;
+    pisa_params_t pi = *p;
+    pi.N = len;
+    Geometry gi;
+    st = resolve(&pi, &gi);
+    if (st != PISA_OK) return st;
+    const size_t oq = t0 * g.Hq * g.d * es, ok = t0 * g.Hkv * g.d * es;
+    st = tensor_bsa_bwd(gi, (const char*)q + oq, (const char*)k + ok, (const char*)v + ok, idx + t0 * g.Hkv * g.K,
+                        (const char*)out + oq, lse + t0 * g.Hq, (const char*)dout + oq, (char*)dq + oq,
+                        (char*)dk + ok, (char*)dv + ok, (char*)ws + kStatusBytes, (int32_t*)ws, s);
+    if (st != PISA_OK) return st;
+  }
+  kernel_mark("end", s);
+  return PISA_OK;
+}
+
 int pisa_decode_step(const pisa_params_t* p, int32_t pos, const void* q, const void* k_cache,
                      const void* v_cache, void* pyramid, int32_t* idx, void* out, float* lse,
                      void* ws, size_t ws_bytes, void* stream) {

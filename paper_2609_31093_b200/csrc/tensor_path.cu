@@ -1443,8 +1443,14 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
   return check_launch("convert_out");
 }
 
+// the backward reads only leaf-level lists: the routing's conditions on g*C and on the depth do not apply
 bool tensor_bwd_supported(const Geometry& g, int dtype) {
-  return tensor_path_supported(g, dtype);                  // d in {64, 128}
+  if (dtype != PISA_BF16) return false;
+  if (g.d != 64 && g.d != 128) return false;
+  if (g.C != 64 && g.C != 128) return false;
+  if (g.N >= (1 << 24)) return false;
+  if ((long long)g.B * g.Hkv * g.N * g.K >= (1LL << 31)) return false;   // entry offsets are int32
+  return true;
 }
 size_t tensor_bwd_workspace_bytes(const Geometry& g) { return bwd_layout(g).total; }
 

@@ -138,3 +138,14 @@ def gather_out(dev: Device, triples: np.ndarray):
     o = dev.out[t[:, 0:1], t[:, 2:3], heads]                                   # [S, G, d]
     l = dev.lse[t[:, 0:1], heads, t[:, 2:3]]                                   # [S, G]
     return o.to(torch.float64).cpu().numpy(), l.to(torch.float64).cpu().numpy()
+
+
+def check_gradient_rows(name, got, ref, extra=0.0):
+    """Per-row bound for a bf16 attention gradient (see tests/test_gpu_backward.py for its derivation):
+    |err| <= 2^-5 max|ref_row| + 1e-2 rms(ref) + extra, mean error <= 4e-3 rms(ref) + mean(extra) (the
+    second term matters only where the reference vanishes, e.g. dq of a one-token sequence)."""
+    rms = float(np.sqrt(np.mean(ref * ref)))
+    err = np.abs(got - ref)
+    bound = 2.0 ** -5 * np.abs(ref).max(axis=-1, keepdims=True) + 1e-2 * rms + extra
+    assert np.all(err <= bound), f"{name}: max excess {(err - bound).max():.3e} (rms {rms:.3e})"
+    assert err.mean() <= 4e-3 * rms + float(np.mean(extra)), f"{name}: mean err {err.mean():.3e} vs rms {rms:.3e}"

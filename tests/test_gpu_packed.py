@@ -55,3 +55,51 @@ def test_packed_sequences_equal_the_sequences_alone_and_the_oracle():
         gi = got_idx.cpu()[ti[:, 1], ti[:, 2]].numpy()
         n_diff, n_bad, n_band = T.compare_index_sets(gi, ref_idx, ref_margin)
         assert n_bad == 0, i
+
+
+def test_packed_backward_matches_the_oracle_per_sequence():
+    """Forward then backward over a pack; every sequence's gradients against the oracle run on that sequence
+    alone with the indices the forward selected (one sequence is a single partial block, one a single token)."""
+    from oracle import pisa_oracle as O
+    lens = [700, 64, 1, 1500, 0, 130, 37]
+    Hq, Hkv, d, C, g, K = 8, 2, 128, 64, 2, 4
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    total = int(cu[-1])
+    parts = [S.make_inputs(S.Workload(f"pb{i}", 1, max(n, 1), Hq, Hkv, d, C, g, K, "bf16", 720 + i, "iid"))
+             for i, n in enumerate(lens)]
+    cat = lambda key: np.concatenate([p_[key][0, :n] for p_, n in zip(parts, lens)], axis=0)
+    q, k, v = (T.to_torch(cat(x), "bf16") for x in ("q", "k", "v"))
+    p = P.Params(1, max(lens), Hq, Hkv, d, C, g, K, dtype="bf16")
+    pyramid = PB.alloc_pyramid(p)
+    ws = PB.alloc_workspace(p, PB.OP_FORWARD)
+    idx = torch.full((Hkv * K * total,), -7, dtype=torch.int32, device="cuda")
+    out = torch.zeros_like(q)
+    lse = torch.zeros((Hq * total,), dtype=torch.float32, device="cuda")
+    P.pisa_forward_packed(p, cu.tolist(), q, k, v, pyramid, idx, out, lse, ws)
+    rng = np.random.default_rng(77)
+    dout_bits = S.f32_to_bf16_bits(rng.standard_normal((total, Hq, d)).astype(np.float32))
+    dout = T.to_torch(dout_bits, "bf16")
+    dq, dk, dv = (torch.full_like(x, float("nan")) for x in (q, k, v))
+    wsb = PB.alloc_workspace(p, PB.OP_BSA_BWD)
+    P.pisa_bsa_bwd_packed(p, cu.tolist(), q, k, v, idx, out, lse, dout, dq, dk, dv, wsb)
+    torch.cuda.synchronize()
+    assert P.read_status(ws) == 0 and P.read_status(wsb) == 0
+    for i, n in enumerate(lens):
+        if n == 0:
+            continue
+        t0 = int(cu[i])
+        t = {key: parts[i][key][:, :n] for key in ("q", "k", "v")}
+        idx_i = idx[Hkv * K * t0:Hkv * K * (t0 + n)].view(1, Hkv, n, K).cpu().numpy()
+        do_i = dout_bits[None, t0:t0 + n]
+        rq, rk, rv = O.attend_backward(t["q"], t["k"], t["v"], idx_i, do_i, C=C, dtype="bf16")
+        o64 = out[t0:t0 + n].to(torch.float64).cpu().numpy()[None]
+        do64 = O.load_storage(do_i, "bf16")
+        kmax = float(np.abs(O.load_storage(t["k"], "bf16")).max())
+        d_delta = 2.0 ** -9 * np.abs(o64 * do64).sum(axis=-1, keepdims=True) / np.sqrt(d) * kmax
+        # a one-token sequence has dS = 0 exactly, so the rounding of delta is all there is in dk too
+        qmax = float(np.abs(O.load_storage(t["q"], "bf16")).max())
+        dk_extra = float(d_delta.sum()) / kmax * qmax if n == 1 else 0.0
+        for nm, got, ref, extra in (("dq", dq, rq, d_delta), ("dk", dk, rk, dk_extra), ("dv", dv, rv, 0.0)):
+            g64 = got[t0:t0 + n].to(torch.float64).cpu().numpy()[None]
+            assert np.isfinite(g64).all(), (i, nm)
+            T.check_gradient_rows(f"seq{i}.{nm}", g64, ref, extra)
