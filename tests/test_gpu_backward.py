@@ -29,6 +29,10 @@ CASES = {
     "g16_c128": S.Workload("bwd_g16_c128", 1, 768, 16, 1, 128, 128, 2, 4, "bf16", 604, "iid"),
     "d64_c64_g16": S.Workload("bwd_d64_c64", 1, 1100, 16, 1, 64, 64, 2, 4, "bf16", 605, "iid"),
     "d64_c128_gqa2": S.Workload("bwd_d64_c128", 1, 900, 4, 2, 64, 128, 2, 3, "bf16", 606, "walk"),
+    # shapes whose forward runs on the SIMT kernels (g*C = 512; a single partial leaf): the backward only
+    # needs the leaf-level lists
+    "fan4_c128": S.Workload("bwd_fan4_c128", 1, 1100, 4, 2, 128, 128, 4, 4, "bf16", 607, "iid"),
+    "single_leaf": S.Workload("bwd_single_leaf", 2, 50, 8, 2, 128, 64, 2, 4, "bf16", 608, "iid"),
 }
 
 
