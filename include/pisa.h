@@ -138,7 +138,15 @@ int pisa_route_static(const pisa_params_t* p, const void* q, const void* k, cons
                       int32_t* idx, float* margin, void* stream);
 size_t pisa_route_static_capacity(void);
 
-/* pyramid -> route -> attention in one call.  pyramid and idx are outputs too (kept for reuse). */
+/*
+ * pyramid -> route -> attention in one call.  pyramid and idx are outputs too (kept for reuse).
+ * A large tensor-path problem is cut into up to four chunks of (batch, KV head) units that alternate
+ * between `stream` and one stream the library owns (created on the first such call, per host
+ * thread): the chunks' kernels stress different parts of the GPU and fill each other's tails.  The
+ * internal stream forks from `stream` after the pyramid and joins it before the call's last
+ * operation, so the call still behaves as ordered work on `stream` (and can be captured into a CUDA
+ * graph).  The workspace query for PISA_OP_FORWARD covers both streams' scratch.
+ */
 int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const void* v, void* pyramid,
                  int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes, void* stream);
 
@@ -278,10 +286,19 @@ int pisa_get_stage_ms(float* pyramid_ms, float* route_ms, float* attn_ms);
 
 /*
  * With stage timing on, pisa_forward also brackets its main kernels with events.  After a forward
- * call, entry i (0-based) gives the name of the i-th bracket and its device time in milliseconds;
- * PISA_ERR_INVALID_ARG past the last entry.  The getter waits for the events.
+ * call, entry i (0-based) gives the name of the i-th bracket and its device time in milliseconds
+ * (from its event to the next one on the same stream; a name occurs once per chunk; the last bracket
+ * of a stream is named "end" and has no time); PISA_ERR_INVALID_ARG past the last entry.  The getter
+ * waits for the events.
  */
 int pisa_get_kernel_ms(int i, char* name, size_t name_len, float* ms);
+
+/*
+ * Upper limit on the chunks pisa_forward cuts a problem into, for the calling host thread:
+ * 0 = automatic (the default), 1 = never split (every kernel runs alone on `stream`, which is what a
+ * per-kernel measurement wants).  Workspace sizes queried before stay sufficient.
+ */
+int pisa_set_forward_chunks(int max_chunks);
 
 /* Number of kernels this process has launched through the library so far (host counter). */
 unsigned long long pisa_launch_count(void);

@@ -28,6 +28,8 @@ from .binding import (  # noqa: F401
     get_stage_ms,
     launch_count,
     get_kernel_ms,
+    get_kernel_brackets,
+    set_forward_chunks,
     IMPL_AUTO,
     IMPL_SIMT,
     IMPL_TENSOR,

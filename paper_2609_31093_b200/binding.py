@@ -65,6 +65,7 @@ def lib():
     L.pisa_route_static.restype = C.c_int
     L.pisa_route_static_capacity.restype = C.c_size_t
     L.pisa_set_stage_timing.argtypes = [C.c_int]
+    L.pisa_set_forward_chunks.argtypes = [C.c_int]
     L.pisa_get_stage_ms.argtypes = [f32p, f32p, f32p]
     L.pisa_launch_count.restype = C.c_ulonglong
     L.pisa_get_kernel_ms.argtypes = [C.c_int, C.c_char_p, C.c_size_t, f32p]
@@ -72,7 +73,7 @@ def lib():
     for name in ("pisa_pyramid_layout", "pisa_workspace_bytes", "pisa_build_pyramid", "pisa_route",
                  "pisa_bsa_fwd", "pisa_forward", "pisa_forward_host", "pisa_flat_select", "pisa_read_status",
                  "pisa_decode_step", "pisa_pyramid_regrow", "pisa_bsa_bwd", "pisa_forward_packed", "pisa_bsa_bwd_packed",
-                 "pisa_set_stage_timing", "pisa_get_stage_ms"):
+                 "pisa_set_stage_timing", "pisa_get_stage_ms", "pisa_set_forward_chunks"):
         getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -246,13 +247,29 @@ def launch_count() -> int:
     return int(lib().pisa_launch_count())
 
 
-def get_kernel_ms() -> dict:
-    """{bracket name: device ms} of the last pisa_forward issued with stage timing on."""
-    out = {}
+def set_forward_chunks(max_chunks: int):
+    """0 = automatic chunking of pisa_forward over two streams, 1 = never split."""
+    _check(lib().pisa_set_forward_chunks(int(max_chunks)), "pisa_set_forward_chunks")
+
+
+def get_kernel_brackets() -> list:
+    """[(bracket name, device ms)] of the last pisa_forward issued with stage timing on, one entry per
+    launch bracket (a name occurs once per chunk); the closing brackets of the streams are left out."""
+    out = []
     buf = C.create_string_buffer(64)
     ms = C.c_float()
     i = 0
     while lib().pisa_get_kernel_ms(i, buf, 64, C.byref(ms)) == 0:
-        out[buf.value.decode()] = out.get(buf.value.decode(), 0.0) + ms.value
+        name = buf.value.decode()
+        if name != "end":
+            out.append((name, ms.value))
         i += 1
+    return out
+
+
+def get_kernel_ms() -> dict:
+    """{bracket name: device ms summed over its launches} of the last pisa_forward with stage timing on."""
+    out = {}
+    for name, t in get_kernel_brackets():
+        out[name] = out.get(name, 0.0) + t
     return out

@@ -12,10 +12,12 @@ static thread_local char g_cuda_err[512] = "";
 static thread_local bool g_timing = false;
 static thread_local cudaEvent_t g_ev[4] = {nullptr, nullptr, nullptr, nullptr};
 static thread_local bool g_ev_valid = false;
-// per-kernel marks (name of the kernel that starts at the mark), recorded when timing is on
-constexpr int kMaxMarks = 32;
+// per-kernel marks (name of the kernel that starts at the mark, and the stream it was recorded on),
+// recorded when timing is on; a kernel's time runs to the next mark on the same stream
+constexpr int kMaxMarks = 192;
 static thread_local cudaEvent_t g_mark_ev[kMaxMarks];
 static thread_local const char* g_mark_name[kMaxMarks];
+static thread_local cudaStream_t g_mark_stream[kMaxMarks];
 static thread_local int g_mark_n = 0;
 static thread_local bool g_mark_valid = false;
 
@@ -26,6 +28,7 @@ void kernel_mark(const char* name, cudaStream_t s) {
     g_mark_valid = true;
   }
   g_mark_name[g_mark_n] = name;
+  g_mark_stream[g_mark_n] = s;
   cudaEventRecord(g_mark_ev[g_mark_n], s);
   ++g_mark_n;
 }
@@ -193,14 +196,123 @@ static void stage_mark(int i, cudaStream_t s) {
   cudaEventRecord(g_ev[i], s);
 }
 
+// ---------------------------------------------------------------- forward in chunks on two streams
+//
+// The (batch, KV head) units of a forward are independent, and its kernels load different parts of
+// the machine (stage 1 of the routing: instruction issue; the two tile kernels: L2 and tensor cores).
+// A large tensor-path forward is therefore cut into chunks of units that alternate between the
+// caller's stream and one internal stream: while a persistent tile kernel of one chunk drains, the
+// next kernels of the other chunk fill the SMs it frees.  A chunk is a rectangular sub-problem that
+// is contiguous in idx and lse: whole batches, or a range of KV heads of one batch.  The pyramid is
+// built once for the whole problem; a chunk's geometry points at its units inside it.
+constexpr int kMaxChunks = 4;                     // measured at B=1, Hkv=8, N=128K: 2 / 4 / 8 chunks -> 46.4 / 45.2 / 46.4 ms
+constexpr int kStreams = 2;                       // the caller's stream + one internal (3 or 4 streams: no gain)
+constexpr int kMaxStreams = kStreams;
+static thread_local int g_chunk_limit = 0;        // pisa_set_forward_chunks: 0 = automatic, 1 = never split
+constexpr long long kMinChunkTokens = 65536;      // units * N per chunk below which splitting does not pay
+
+struct Chunk { int b0, nb, h0, nh; };
+struct ForwardPlan {
+  int n;                        // 1 = not split
+  Chunk c[kMaxChunks];
+  int streams;                  // streams the chunks alternate on (the caller's + internal ones)
+  size_t region;                // workspace bytes of one stream's region (largest chunk), 256-aligned
+  size_t total;                 // status word + regions
+};
+
+static int chunk_problem(const pisa_params_t* p, const Geometry& g, const Chunk& c, pisa_params_t* pc, Geometry* gc) {
+  *pc = *p;
+  pc->B = c.nb;
+  pc->Hkv = c.nh;
+  pc->Hq = c.nh * g.G;
+  for (int i = 0; i < 3; ++i) {
+    pc->q_stride[i] = g.qs[i]; pc->k_stride[i] = g.ks[i]; pc->v_stride[i] = g.vs[i]; pc->o_stride[i] = g.os[i];
+  }
+  const int st = resolve(pc, gc);
+  if (st != PISA_OK) return st;
+  const long long unit0 = (long long)c.b0 * g.Hkv + c.h0;
+  for (int l = 1; l <= g.L; ++l) gc->level_off[l] = g.level_off[l] + unit0 * g.M[l] * g.d;
+  return PISA_OK;
+}
+
+static int forward_plan(const pisa_params_t* p, const Geometry& g, ForwardPlan* pl) {
+  pl->n = 1;
+  pl->c[0] = {0, g.B, 0, g.Hkv};
+  const long long units = (long long)g.B * g.Hkv;
+  long long parts = units * g.N / kMinChunkTokens;
+  if (parts > kMaxChunks) parts = kMaxChunks;
+  if (g_chunk_limit > 0 && parts > g_chunk_limit) parts = g_chunk_limit;
+  if (parts > units) parts = units;
+  if (use_tensor(p, g) && parts >= 2) {
+    int n = 0;
+    if (g.B >= parts) {                       // whole batches
+      for (int i = 0; i < parts; ++i) {
+        const int b0 = (int)((long long)g.B * i / parts), b1 = (int)((long long)g.B * (i + 1) / parts);
+        pl->c[n++] = {b0, b1 - b0, 0, g.Hkv};
+      }
+    } else {                                  // head ranges inside every batch
+      int per = (int)(parts / g.B);
+      if (per > g.Hkv) per = g.Hkv;
+      for (int b = 0; b < g.B; ++b)
+        for (int i = 0; i < per; ++i) {
+          const int h0 = g.Hkv * i / per, h1 = g.Hkv * (i + 1) / per;
+          pl->c[n++] = {b, 1, h0, h1 - h0};
+        }
+    }
+    pl->n = n;
+  }
+  size_t region = 0;
+  for (int i = 0; i < pl->n; ++i) {
+    pisa_params_t pc;
+    Geometry gc;
+    const int st = chunk_problem(p, g, pl->c[i], &pc, &gc);
+    if (st != PISA_OK) return st;
+    if (pl->n > 1 && !use_tensor(&pc, gc)) {   // a chunk the tensor path does not take: run unsplit
+      pl->n = 1;
+      pl->c[0] = {0, g.B, 0, g.Hkv};
+      i = -1;
+      region = 0;
+      continue;
+    }
+    const size_t r = route_ws_bytes(&pc, gc) - kStatusBytes, b = bsa_ws_bytes(&pc, gc) - kStatusBytes;
+    const size_t m = align_up(r > b ? r : b, 256);
+    if (m > region) region = m;
+  }
+  pl->region = region;
+  pl->streams = (pl->n > 1) ? (pl->n < kStreams ? pl->n : kStreams) : 1;
+  pl->total = kStatusBytes + pl->streams * region;
+  return PISA_OK;
+}
+
+static thread_local cudaStream_t g_side[kMaxStreams] = {};  // internal streams ([0] unused) and fork / join events
+static thread_local cudaEvent_t g_fork = nullptr, g_join[kMaxStreams] = {};
+
+static int side_streams() {
+  if (g_fork != nullptr) return PISA_OK;
+  cudaError_t e = cudaSuccess;
+  for (int i = 1; i < kMaxStreams && e == cudaSuccess; ++i) {
+    e = cudaStreamCreateWithFlags(&g_side[i], cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_join[i], cudaEventDisableTiming);
+  }
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_fork, cudaEventDisableTiming);
+  if (e != cudaSuccess) { record_cuda_error("internal streams", e); g_fork = nullptr; return PISA_ERR_CUDA; }
+  return PISA_OK;
+}
+
 static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v,
                       void* pyr, int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes,
                       cudaStream_t s, bool clear = true) {
-  size_t need = route_ws_bytes(p, g);
-  const size_t need_b = bsa_ws_bytes(p, g);
-  if (need_b > need) need = need_b;
-  if (ws_bytes < need) return PISA_ERR_WORKSPACE_TOO_SMALL;
-  int st = clear ? clear_status(ws, s) : PISA_OK;
+  ForwardPlan pl;
+  int st = forward_plan(p, g, &pl);
+  if (st != PISA_OK) return st;
+  if (pl.n > 1 && ws_bytes < pl.total) {     // a workspace sized for another length of the same problem: unsplit
+    const size_t r = route_ws_bytes(p, g), b = bsa_ws_bytes(p, g);
+    pl.n = 1;
+    pl.total = r > b ? r : b;
+  }
+  if (ws_bytes < pl.total) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  if (pl.n > 1 && (st = side_streams()) != PISA_OK) return st;
+  st = clear ? clear_status(ws, s) : PISA_OK;
   if (st != PISA_OK) return st;
   g_mark_n = 0;
   stage_mark(0, s);
@@ -208,12 +320,53 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
   st = launch_pyramid(g, p->dtype, k, pyr, s);
   if (st != PISA_OK) return st;
   stage_mark(1, s);
-  // the tensor-core routing already knows every kept leaf's per-head LSE, so it hands the rows'
-  // softmax denominators to the attention stage
-  st = do_route(p, g, q, k, pyr, idx, nullptr, lse, ws, ws_bytes, s);
-  if (st != PISA_OK) return st;
-  stage_mark(2, s);
-  st = do_bsa(p, g, q, k, v, idx, out, lse, use_tensor(p, g) && g.score_mode == PISA_SCORE_LSE, ws, ws_bytes, s);
+  if (pl.n == 1) {
+    // the tensor-core routing already knows every kept leaf's per-head LSE, so it hands the rows'
+    // softmax denominators to the attention stage
+    st = do_route(p, g, q, k, pyr, idx, nullptr, lse, ws, ws_bytes, s);
+    if (st != PISA_OK) return st;
+    stage_mark(2, s);
+    st = do_bsa(p, g, q, k, v, idx, out, lse, use_tensor(p, g) && g.score_mode == PISA_SCORE_LSE, ws, ws_bytes, s);
+    stage_mark(3, s);
+    kernel_mark("end", s);
+    return st;
+  }
+  // fork: the internal stream starts after the pyramid (and after whatever the caller queued before)
+  cudaError_t e = cudaEventRecord(g_fork, s);
+  for (int i = 1; i < pl.streams && e == cudaSuccess; ++i) e = cudaStreamWaitEvent(g_side[i], g_fork, 0);
+  if (e != cudaSuccess) { record_cuda_error("fork", e); return PISA_ERR_CUDA; }
+  const size_t es = elem_size(p->dtype);
+  int32_t* status = (int32_t*)ws;
+  st = PISA_OK;
+  for (int i = 0; i < pl.n && st == PISA_OK; ++i) {
+    const Chunk& c = pl.c[i];
+    pisa_params_t pc;
+    Geometry gc;
+    st = chunk_problem(p, g, c, &pc, &gc);
+    if (st != PISA_OK) break;
+    const int si = i % pl.streams;
+    cudaStream_t cs = si ? g_side[si] : s;
+    char* region = (char*)ws + kStatusBytes + (size_t)si * pl.region;
+    const long long unit0 = (long long)c.b0 * g.Hkv + c.h0;
+    const char* qc = (const char*)q + ((long long)c.b0 * g.qs[0] + (long long)c.h0 * g.G * g.qs[2]) * es;
+    const char* kc = (const char*)k + ((long long)c.b0 * g.ks[0] + (long long)c.h0 * g.ks[2]) * es;
+    const char* vc = (const char*)v + ((long long)c.b0 * g.vs[0] + (long long)c.h0 * g.vs[2]) * es;
+    char* oc = (char*)out + ((long long)c.b0 * g.os[0] + (long long)c.h0 * g.G * g.os[2]) * es;
+    int32_t* ic = idx + unit0 * g.N * g.K;
+    float* lc = lse + unit0 * g.G * g.N;
+    st = tensor_route(gc, p->dtype, qc, kc, pyr, ic, nullptr, lc, region, status, cs);
+    if (st != PISA_OK) break;
+    if (i == 0) stage_mark(2, s);
+    st = tensor_bsa(gc, p->dtype, qc, kc, vc, ic, oc, lc, g.score_mode == PISA_SCORE_LSE, region, status, cs);
+  }
+  // join, also after a failed launch: the caller's stream must not run ahead of the internal one
+  e = cudaSuccess;
+  for (int i = 1; i < pl.streams; ++i) {
+    kernel_mark("end", g_side[i]);
+    if (e == cudaSuccess) e = cudaEventRecord(g_join[i], g_side[i]);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s, g_join[i], 0);
+  }
+  if (e != cudaSuccess && st == PISA_OK) { record_cuda_error("join", e); st = PISA_ERR_CUDA; }
   stage_mark(3, s);
   kernel_mark("end", s);
   return st;
@@ -263,7 +416,13 @@ int pisa_workspace_bytes(const pisa_params_t* p, int op, size_t* bytes) {
   if (st != PISA_OK) return st;
   if (bytes == nullptr) return PISA_ERR_INVALID_ARG;
   const size_t r = route_ws_bytes(p, g), a = bsa_ws_bytes(p, g);
-  const size_t f = r > a ? r : a;
+  size_t f = r > a ? r : a;                  // also lets one buffer serve pisa_route and pisa_bsa_fwd
+  {
+    ForwardPlan pl;
+    st = forward_plan(p, g, &pl);
+    if (st != PISA_OK) return st;
+    if (pl.total > f) f = pl.total;
+  }
   switch (op) {
     case PISA_OP_ROUTE: *bytes = r; break;
     case PISA_OP_BSA: *bytes = a; break;
@@ -599,13 +758,23 @@ int pisa_read_status(const void* ws, int32_t* status) {
 }
 
 int pisa_get_kernel_ms(int i, char* name, size_t name_len, float* ms) {
-  if (!g_timing || !g_mark_valid || i < 0 || i + 1 >= g_mark_n) return PISA_ERR_INVALID_ARG;
-  cudaError_t e = cudaEventSynchronize(g_mark_ev[g_mark_n - 1]);
-  if (e != cudaSuccess) { record_cuda_error("kernel events", e); return PISA_ERR_CUDA; }
+  if (!g_timing || !g_mark_valid || i < 0 || i >= g_mark_n) return PISA_ERR_INVALID_ARG;
+  int j = i + 1;
+  while (j < g_mark_n && g_mark_stream[j] != g_mark_stream[i]) ++j;
   float t = 0.f;
-  cudaEventElapsedTime(&t, g_mark_ev[i], g_mark_ev[i + 1]);
+  if (j < g_mark_n) {
+    cudaError_t e = cudaEventSynchronize(g_mark_ev[j]);
+    if (e != cudaSuccess) { record_cuda_error("kernel events", e); return PISA_ERR_CUDA; }
+    cudaEventElapsedTime(&t, g_mark_ev[i], g_mark_ev[j]);
+  }
   if (ms) *ms = t;
-  if (name && name_len > 0) snprintf(name, name_len, "%s", g_mark_name[i]);
+  if (name && name_len > 0) snprintf(name, name_len, "%s", (j < g_mark_n) ? g_mark_name[i] : "end");
+  return PISA_OK;
+}
+
+int pisa_set_forward_chunks(int max_chunks) {
+  if (max_chunks < 0) return PISA_ERR_INVALID_ARG;
+  g_chunk_limit = max_chunks;
   return PISA_OK;
 }
 

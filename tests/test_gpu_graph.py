@@ -1,6 +1,9 @@
 """The asynchronous entry points are plain stream work: no allocation, no synchronisation, no host
 read-back.  So a call can be captured into a CUDA graph and replayed, and the replay gives what the
-eager call gives (indices exactly; outputs up to the order of the fp32 accumulator additions)."""
+eager call gives (indices exactly; outputs up to the order of the fp32 accumulator additions).
+The forward here is large enough to run as chunks on the caller's stream and the library's internal
+one (fork after the pyramid, join before the end), which the capture must follow; and chunked and
+unsplit forwards must agree."""
 import pytest
 import torch
 
@@ -12,7 +15,7 @@ import pisa_testlib as T  # noqa: E402
 import paper_2609_31093_b200 as P  # noqa: E402
 from paper_2609_31093_b200 import binding as PB  # noqa: E402
 
-W = S.Workload("graph_gqa4", 2, 3000, 8, 2, 128, 128, 2, 6, "bf16", 501, "iid")
+W = S.Workload("graph_gqa4", 2, 40000, 8, 2, 128, 128, 2, 6, "bf16", 501, "iid")     # 2 chunks (one batch each)
 
 
 def _capture(fn):
@@ -71,3 +74,28 @@ def test_backward_replays_from_a_cuda_graph():
     assert P.read_status(ws) == 0
     for got, want in zip((dq, dk, dv), ref):
         assert torch.allclose(got.float(), want, rtol=0, atol=2.0 ** -6 * float(want.abs().max()))
+
+
+@pytest.mark.parametrize("B,Hkv,N", [(3, 2, 50000), (4, 1, 70000), (1, 4, 66000)])
+def test_chunked_forward_equals_the_unsplit_one(B, Hkv, N):
+    """Chunks of whole batches, of one batch each, and of head ranges of a single batch."""
+    w = S.Workload(f"chunks_b{B}", B, N, 4 * Hkv, Hkv, 64, 64, 2, 5, "bf16", 510 + B, "iid")
+    t = S.make_inputs(w)
+    dev = T.Device(w, t)
+    P.set_forward_chunks(1)
+    try:
+        dev.forward()
+        assert dev.sync_status() == 0
+    finally:
+        P.set_forward_chunks(0)
+    idx, out, lse, pyr = dev.idx.clone(), dev.out.clone(), dev.lse.clone(), dev.pyramid.clone()
+    dev.idx.fill_(-7)
+    dev.out.zero_()
+    dev.lse.zero_()
+    dev.pyramid.zero_()
+    dev.forward()
+    assert dev.sync_status() == 0
+    assert torch.equal(dev.pyramid, pyr)
+    assert torch.equal(dev.idx, idx)
+    assert torch.allclose(dev.lse, lse, rtol=1e-5, atol=1e-5)
+    assert torch.allclose(dev.out.float(), out.float(), rtol=0, atol=2.0 ** -7 * float(out.float().abs().max()))
