@@ -174,11 +174,13 @@ int pisa_forward_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32
 /*
  * The same forward pass for callers that hold HOST tensors.  KV heads are independent units of the
  * path (Sec. 3.3: one selected set per KV head), so the call walks them one at a time: the strided
- * slice of q, k, v that belongs to head h is copied into one of two slots of the device arena
- * (`ws`, sized for PISA_OP_FORWARD_HOST: two slots of per-head tensors, one per-head pyramid and
- * one per-head forward workspace), pisa_forward runs on it, and out, lse and (if not NULL) idx of
+ * slice of q, k, v that belongs to head h is copied into one of four slots of the device arena
+ * (`ws`, sized for PISA_OP_FORWARD_HOST: four slots of per-head tensors, two per-head pyramids and
+ * two per-head forward workspaces), pisa_forward runs on it, and out, lse and (if not NULL) idx of
  * that head are copied back into their places in the host tensors.  The copies run on two internal
- * streams, so the upload of head h+1 and the download of head h-1 overlap the kernels of head h.
+ * streams and the kernels of consecutive heads alternate between `stream` and a third internal
+ * stream, so two heads' kernels are in flight while the next head is uploaded and the previous one
+ * downloaded.
  * Host buffers should be pinned (pageable memory makes the copies synchronous); strides must be
  * dense.  Work already queued on `stream` is ordered before the call; the call returns after
  * everything it queued has finished.  This is the one entry point that synchronises.

@@ -132,9 +132,11 @@ static size_t bsa_ws_bytes(const pisa_params_t* p, const Geometry& g) {
   return b;
 }
 
-// Device arena of pisa_forward_host.  The call walks the KV heads one at a time (they are independent
-// units of the path): unit u's tensors live in slot u % 2 so that the host->device copy of the next
-// unit and the device->host copy of the previous one overlap the kernels of the current one.
+// Device arena of pisa_forward_host.  The call walks the KV heads (independent units of the path):
+// unit u's tensors live in slot u % 4 and its kernels run on compute stream u % 2 with that stream's
+// workspace and pyramid, so that two units' kernels are in flight (they fill each other's tails, as
+// the chunks of pisa_forward do) while the next unit is uploaded and the previous one downloaded.
+constexpr int kHostSlots = 4;
 struct HostArena {
   pisa_params_t unit;          // the per-unit problem: Hkv = 1, Hq = G, dense strides
   Geometry ug;
@@ -158,7 +160,7 @@ static int host_arena(const pisa_params_t* p, HostArena* a) {
   a->ib = align_up((size_t)g.B * g.N * g.K * sizeof(int32_t), 256);
   a->pb = align_up(pyramid_bytes_dtype(g, p->dtype), 256);
   a->slot = 2 * a->qb + 2 * a->kb + a->lb + a->ib;
-  a->total = a->fwd + a->pb + 2 * a->slot;
+  a->total = 2 * (a->fwd + a->pb) + kHostSlots * a->slot;
   return PISA_OK;
 }
 
@@ -543,11 +545,12 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
   st = host_arena(p, &A);
   if (st != PISA_OK) return st;
   if (ws_bytes < A.total) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  if ((st = side_streams()) != PISA_OK) return st;
   cudaStream_t s = (cudaStream_t)stream;
   const size_t es = elem_size(p->dtype);
-  char* base = (char*)ws;
-  char* dpyr = base + A.fwd;
-  char* slot0 = dpyr + A.pb;
+  char* base = (char*)ws;                                          // [fwd 0][fwd 1][pyramid 0][pyramid 1][slots]
+  char* dpyr = base + 2 * A.fwd;
+  char* slot0 = dpyr + 2 * A.pb;
   const int U = g.Hkv, G = g.G;
   const size_t rows = (size_t)g.B * g.N;                         // tokens of all batches
   const size_t q_w = (size_t)G * g.d * es, q_pitch = (size_t)g.Hq * g.d * es;
@@ -557,15 +560,15 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
 
   // copy streams and the events that order the three stages of every unit
   cudaStream_t s_in = nullptr, s_out = nullptr;
-  cudaEvent_t ev_begin = nullptr, ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr},
-              ev_out[2] = {nullptr, nullptr};
+  cudaEvent_t ev_begin = nullptr, ev_in[kHostSlots] = {}, ev_done[kHostSlots] = {}, ev_out[kHostSlots] = {};
   cudaError_t e = cudaSuccess;
   const char* what = "copy streams";
   auto ok = [&](cudaError_t r, const char* w) { if (e == cudaSuccess && r != cudaSuccess) { e = r; what = w; } return e == cudaSuccess; };
   ok(cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking), "stream create");
   ok(cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking), "stream create");
   ok(cudaEventCreateWithFlags(&ev_begin, cudaEventDisableTiming), "event create");
-  for (int i = 0; i < 2; ++i) {
+  cudaStream_t cs[2] = {s, g_side[1]};                             // compute streams
+  for (int i = 0; i < kHostSlots; ++i) {
     ok(cudaEventCreateWithFlags(&ev_in[i], cudaEventDisableTiming), "event create");
     ok(cudaEventCreateWithFlags(&ev_done[i], cudaEventDisableTiming), "event create");
     ok(cudaEventCreateWithFlags(&ev_out[i], cudaEventDisableTiming), "event create");
@@ -577,27 +580,34 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
     ok(cudaStreamWaitEvent(s_out, ev_begin, 0), "stream wait");
   }
   st = (e == cudaSuccess) ? clear_status(ws, s) : PISA_OK;
+  if (e == cudaSuccess && st == PISA_OK) st = clear_status(base + A.fwd, s);   // the second workspace's status word
+  if (e == cudaSuccess) {
+    ok(cudaEventRecord(ev_begin, s), "event record");
+    ok(cudaStreamWaitEvent(cs[1], ev_begin, 0), "stream wait");
+  }
   for (int u = 0; u < U && e == cudaSuccess && st == PISA_OK; ++u) {
-    const int sl = u & 1;
+    const int sl = u % kHostSlots, ci = u & 1;
     char* dq = slot0 + sl * A.slot;
     char* dout = dq + A.qb;
     char* dk = dout + A.qb;
     char* dv = dk + A.kb;
     char* dl = dv + A.kb;
     char* di = dl + A.lb;
-    // stage 1: inputs of unit u (its slot was last read by the kernels of unit u-2)
-    if (u >= 2) ok(cudaStreamWaitEvent(s_in, ev_done[sl], 0), "stream wait");
+    // stage 1: inputs of unit u (its slot was last read by the kernels of the unit that had it before)
+    if (u >= kHostSlots) ok(cudaStreamWaitEvent(s_in, ev_done[sl], 0), "stream wait");
     ok(cudaMemcpy2DAsync(dq, q_w, (const char*)q_host + (size_t)u * q_w, q_pitch, q_w, rows, cudaMemcpyHostToDevice, s_in), "h2d copy");
     ok(cudaMemcpy2DAsync(dk, k_w, (const char*)k_host + (size_t)u * k_w, k_pitch, k_w, rows, cudaMemcpyHostToDevice, s_in), "h2d copy");
     ok(cudaMemcpy2DAsync(dv, k_w, (const char*)v_host + (size_t)u * k_w, k_pitch, k_w, rows, cudaMemcpyHostToDevice, s_in), "h2d copy");
     ok(cudaEventRecord(ev_in[sl], s_in), "event record");
-    // stage 2: the kernels (the slot's outputs were last read by the copies of unit u-2)
-    ok(cudaStreamWaitEvent(s, ev_in[sl], 0), "stream wait");
-    if (u >= 2) ok(cudaStreamWaitEvent(s, ev_out[sl], 0), "stream wait");
+    // stage 2: the kernels (the slot's outputs were last read by the copies of its previous unit); the
+    // workspace and pyramid of this compute stream were last used by unit u-2, earlier on the same stream
+    ok(cudaStreamWaitEvent(cs[ci], ev_in[sl], 0), "stream wait");
+    if (u >= kHostSlots) ok(cudaStreamWaitEvent(cs[ci], ev_out[sl], 0), "stream wait");
     if (e != cudaSuccess) break;
-    st = do_forward(&A.unit, A.ug, dq, dk, dv, dpyr, (int32_t*)di, dout, (float*)dl, ws, A.fwd, s, /*clear=*/false);
+    st = do_forward(&A.unit, A.ug, dq, dk, dv, dpyr + ci * A.pb, (int32_t*)di, dout, (float*)dl, base + ci * A.fwd,
+                    A.fwd, cs[ci], /*clear=*/false);
     if (st != PISA_OK) break;
-    ok(cudaEventRecord(ev_done[sl], s), "event record");
+    ok(cudaEventRecord(ev_done[sl], cs[ci]), "event record");
     // stage 3: results of unit u
     ok(cudaStreamWaitEvent(s_out, ev_done[sl], 0), "stream wait");
     ok(cudaMemcpy2DAsync((char*)out_host + (size_t)u * q_w, q_pitch, dout, q_w, q_w, rows, cudaMemcpyDeviceToHost, s_out), "d2h copy");
@@ -609,8 +619,16 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
   // everything this call queued must be finished before its streams and events go away
   if (s_in) ok(cudaStreamSynchronize(s_in), "stream sync");
   ok(cudaStreamSynchronize(s), "stream sync");
+  ok(cudaStreamSynchronize(cs[1]), "stream sync");
   if (s_out) ok(cudaStreamSynchronize(s_out), "stream sync");
-  for (int i = 0; i < 2; ++i) {
+  // a device-side error of the second compute stream shows in the status word the caller reads
+  if (e == cudaSuccess) {
+    int32_t w1 = 0, w0 = 0;
+    ok(cudaMemcpy(&w1, base + A.fwd, sizeof(w1), cudaMemcpyDeviceToHost), "status read");
+    ok(cudaMemcpy(&w0, base, sizeof(w0), cudaMemcpyDeviceToHost), "status read");
+    if (e == cudaSuccess && w1 != 0 && w0 == 0) ok(cudaMemcpy(base, &w1, sizeof(w1), cudaMemcpyHostToDevice), "status write");
+  }
+  for (int i = 0; i < kHostSlots; ++i) {
     if (ev_in[i]) cudaEventDestroy(ev_in[i]);
     if (ev_done[i]) cudaEventDestroy(ev_done[i]);
     if (ev_out[i]) cudaEventDestroy(ev_out[i]);

@@ -77,11 +77,12 @@ def test_argument_validation():
     assert lib.pisa_status_string(-3).decode() == "workspace too small"
 
 
-def test_host_arena_size_covers_two_units():
-    """The host entry point walks the KV heads with two slots of per-head tensors in flight."""
+def test_host_arena_size_covers_its_slots():
+    """The host entry point walks the KV heads with four slots of per-head tensors and two per-head
+    workspaces and pyramids (two heads' kernels in flight, one head uploading, one downloading)."""
     p = P.Params(1, 8192, 16, 4, 128, 64, 2, 16)
     es, G = 2, 4
     unit = P.Params(1, 8192, G, 1, 128, 64, 2, 16)
     slot = 2 * 8192 * G * 128 * es + 2 * 8192 * 128 * es + G * 8192 * 4 + 8192 * 16 * 4
-    need = 2 * slot + P.pyramid_layout(unit)[3] + P.workspace_bytes(unit, PB.OP_FORWARD)
+    need = 4 * slot + 2 * P.pyramid_layout(unit)[3] + 2 * P.workspace_bytes(unit, PB.OP_FORWARD)
     assert P.workspace_bytes(p, PB.OP_FORWARD_HOST) >= need
