@@ -34,8 +34,8 @@ UNIT = "tokens/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per selected (token, block) pair, from the ncu captures
 # summarised under profiles/ (B=1 Hq=8 Hkv=2 d=128 N=65536 C=128 g=2 K=32: 4.19 M pairs per launch)
-DRAM_BYTES_PER_PAIR = {"leaf_lse_tiles": (209.686784e6 + 108.383232e6) / 4194304.0,
-                       "attention_tiles": (1216.039e6 + 934.548736e6) / 4194304.0}
+DRAM_BYTES_PER_PAIR = {"leaf_lse_tiles": (207.892736e6 + 106.752e6) / 4194304.0,
+                       "attention_tiles": (1222.929e6 + 940.475136e6) / 4194304.0}
 
 
 def get_workload(name: str) -> S.Workload:
@@ -284,6 +284,8 @@ def run_ours(args):
         if world > 1:
             dist.barrier()
 
+    P.set_forward_chunks(args.forward_chunks)
+
     def step():
         P.pisa_forward(p, q, k, v, pyramid, idx, out, lse, ws)
 
@@ -336,7 +338,7 @@ def run_ours(args):
         P.get_stage_ms()
         for name, t_ms in P.get_kernel_ms().items():
             kernels[name] = kernels.get(name, 0.0) + t_ms / n_serial
-    P.set_forward_chunks(0)
+    P.set_forward_chunks(args.forward_chunks)
     P.set_stage_timing(False)
 
     # end to end through the host-buffer entry point
@@ -398,21 +400,22 @@ def run_ours(args):
                 "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["peak_source"] = peak_src + (" (sustained bf16, kernel timed inside a long step)" if bound == "tensor" else "")
-    roof["launch_ms"] = t_dom * 1e3
-    roof["launches_per_step"] = launches_of.get(dom, 1)
-    roof["alone_ms"] = t_alone * 1e3
+    n_launch = max(1, launches_of.get(dom, 1))                    # one launch per chunk
+    roof["launch_ms"] = t_dom * 1e3 / n_launch                    # average launch; achieved = (work / n) / this
+    roof["launches_per_step"] = n_launch
+    roof["alone_ms"] = t_alone * 1e3                               # the whole problem as one launch, GPU to itself
     roof["alone_frac"] = work / t_alone / ((hbm_peak * 1e9) if bound == "hbm" else (tens_peak * 1e12))
     # DRAM bytes per launch from the ncu capture of a smaller case of the same kernel (summary under
     # profiles/), scaled by the (token, block) pairs a launch processes: traffic grows with the pairs
     per_pair = DRAM_BYTES_PER_PAIR.get(dom)
     pairs = {"leaf_lse_tiles": wc["sel_pairs"], "attention_tiles": wc["sel_pairs"]}.get(dom)
-    roof["traffic"] = (per_pair * pairs) if (per_pair and pairs and w.dtype == "bf16") else None
+    roof["traffic"] = (per_pair * pairs / n_launch) if (per_pair and pairs and w.dtype == "bf16") else None
     # The two tile kernels are limited by what L2 can gather and reduce, not by the tensor pipe: report
     # that stream too (per selected pair: G*d*2 bytes of query rows L2->SM, and in the attention
     # kernel G*d*4 bytes of fp32 reductions SM->L2).  Context for `frac`, not a substitute for it.
     if dom in ("leaf_lse_tiles", "attention_tiles") and w.dtype == "bf16":
         per_pair_l2 = w.G * w.d * 2 + (w.G * w.d * 4 if dom == "attention_tiles" else 0)
-        roof["l2_stream_bytes"] = per_pair_l2 * wc["sel_pairs"]
+        roof["l2_stream_bytes"] = per_pair_l2 * wc["sel_pairs"] / n_launch
         roof["l2_stream_tbs"] = per_pair_l2 * wc["sel_pairs"] / t_dom / 1e12
     roofs = {}
     for k_, t_ in cand.items():
@@ -758,6 +761,9 @@ def main():
     ap.add_argument("--ref-queries", type=int, default=1024)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--forward-chunks", type=int, default=0,
+                    help="upper limit on the chunks pisa_forward runs on two streams (0 = automatic, 1 = never split; "
+                         "1 is what a per-kernel ncu capture wants)")
     ap.add_argument("--sweep", action="store_true", help="routing latency vs N and the flat selector (not the bench line)")
     ap.add_argument("--backward", action="store_true", help="attention backward with frozen indices (not the bench line)")
     ap.add_argument("--quality", action="store_true", help="Recall@K / MassRatio of the score modes vs full attention (not the bench line)")
