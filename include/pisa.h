@@ -145,7 +145,8 @@ size_t pisa_route_static_capacity(void);
  * thread): the chunks' kernels stress different parts of the GPU and fill each other's tails.  The
  * internal stream forks from `stream` after the pyramid and joins it before the call's last
  * operation, so the call still behaves as ordered work on `stream` (and can be captured into a CUDA
- * graph).  The workspace query for PISA_OP_FORWARD covers both streams' scratch.
+ * graph).  The workspace query for PISA_OP_FORWARD covers both streams' scratch.  pisa_route and
+ * pisa_bsa_fwd split large problems the same way.
  */
 int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const void* v, void* pyramid,
                  int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes, void* stream);
@@ -296,7 +297,8 @@ int pisa_get_stage_ms(float* pyramid_ms, float* route_ms, float* attn_ms);
 int pisa_get_kernel_ms(int i, char* name, size_t name_len, float* ms);
 
 /*
- * Upper limit on the chunks pisa_forward cuts a problem into, for the calling host thread:
+ * Upper limit on the chunks pisa_forward, pisa_route and pisa_bsa_fwd cut a problem into, for the
+ * calling host thread:
  * 0 = automatic (the default), 1 = never split (every kernel runs alone on `stream`, which is what a
  * per-kernel measurement wants).  Workspace sizes queried before stay sufficient.
  */

@@ -237,7 +237,9 @@ static int chunk_problem(const pisa_params_t* p, const Geometry& g, const Chunk&
   return PISA_OK;
 }
 
-static int forward_plan(const pisa_params_t* p, const Geometry& g, ForwardPlan* pl) {
+constexpr int kOpRoute = 1, kOpBsa = 2;
+
+static int forward_plan(const pisa_params_t* p, const Geometry& g, int ops, ForwardPlan* pl) {
   pl->n = 1;
   pl->c[0] = {0, g.B, 0, g.Hkv};
   const long long units = (long long)g.B * g.Hkv;
@@ -276,7 +278,8 @@ static int forward_plan(const pisa_params_t* p, const Geometry& g, ForwardPlan* 
       region = 0;
       continue;
     }
-    const size_t r = route_ws_bytes(&pc, gc) - kStatusBytes, b = bsa_ws_bytes(&pc, gc) - kStatusBytes;
+    const size_t r = (ops & kOpRoute) ? route_ws_bytes(&pc, gc) - kStatusBytes : 0;
+    const size_t b = (ops & kOpBsa) ? bsa_ws_bytes(&pc, gc) - kStatusBytes : 0;
     const size_t m = align_up(r > b ? r : b, 256);
     if (m > region) region = m;
   }
@@ -301,19 +304,112 @@ static int side_streams() {
   return PISA_OK;
 }
 
-static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v,
+// A chunk's view of the caller's tensors.
+struct ChunkView {
+  pisa_params_t p;
+  Geometry g;
+  long long unit0;              // first (batch, KV head) unit, flattened
+  size_t q_off, k_off, v_off, o_off;   // byte offsets into q / k / v / out
+  char* region;                 // this chunk's scratch (past any status word)
+  cudaStream_t stream;
+};
+
+// Plans `ops` for (p, g), falls back to the unsplit plan when `ws_bytes` only covers that one, and
+// returns the bytes the plan needs.
+static int plan_for(const pisa_params_t* p, const Geometry& g, int ops, size_t ws_bytes, ForwardPlan* pl) {
+  int st = forward_plan(p, g, ops, pl);
+  if (st != PISA_OK) return st;
+  if (pl->n > 1 && ws_bytes < pl->total) {   // a workspace sized for another length of the same problem: unsplit
+    const size_t r = (ops & kOpRoute) ? route_ws_bytes(p, g) : 0, b = (ops & kOpBsa) ? bsa_ws_bytes(p, g) : 0;
+    pl->n = 1;
+    pl->streams = 1;
+    pl->total = r > b ? r : b;
+  }
+  if (ws_bytes < pl->total) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  if (pl->n > 1) return side_streams();
+  return PISA_OK;
+}
+
+// Runs fn(view) for every chunk of a split plan: chunk i on stream i % streams (the caller's, then the
+// internal ones, forked here and joined before returning -- also after a failed launch, so that the
+// caller's stream never runs ahead of the internal one).
+template <typename F>
+static int run_chunks(const pisa_params_t* p, const Geometry& g, const ForwardPlan& pl, void* ws, cudaStream_t s,
+                      F&& fn) {
+  cudaError_t e = cudaEventRecord(g_fork, s);
+  for (int i = 1; i < pl.streams && e == cudaSuccess; ++i) e = cudaStreamWaitEvent(g_side[i], g_fork, 0);
+  if (e != cudaSuccess) { record_cuda_error("fork", e); return PISA_ERR_CUDA; }
+  const size_t es = elem_size(p->dtype);
+  int st = PISA_OK;
+  for (int i = 0; i < pl.n && st == PISA_OK; ++i) {
+    const Chunk& c = pl.c[i];
+    ChunkView v;
+    st = chunk_problem(p, g, c, &v.p, &v.g);
+    if (st != PISA_OK) break;
+    const int si = i % pl.streams;
+    v.stream = si ? g_side[si] : s;
+    v.region = (char*)ws + kStatusBytes + (size_t)si * pl.region;
+    v.unit0 = (long long)c.b0 * g.Hkv + c.h0;
+    v.q_off = (size_t)((long long)c.b0 * g.qs[0] + (long long)c.h0 * g.G * g.qs[2]) * es;
+    v.k_off = (size_t)((long long)c.b0 * g.ks[0] + (long long)c.h0 * g.ks[2]) * es;
+    v.v_off = (size_t)((long long)c.b0 * g.vs[0] + (long long)c.h0 * g.vs[2]) * es;
+    v.o_off = (size_t)((long long)c.b0 * g.os[0] + (long long)c.h0 * g.G * g.os[2]) * es;
+    st = fn(v, i);
+  }
+  e = cudaSuccess;
+  for (int i = 1; i < pl.streams; ++i) {
+    kernel_mark("end", g_side[i]);
+    if (e == cudaSuccess) e = cudaEventRecord(g_join[i], g_side[i]);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s, g_join[i], 0);
+  }
+  if (e != cudaSuccess && st == PISA_OK) { record_cuda_error("join", e); st = PISA_ERR_CUDA; }
+  return st;
+}
+
+static int do_route_chunked(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* pyr,
+                            int32_t* idx, float* margin, void* ws, size_t ws_bytes, cudaStream_t s) {
+  ForwardPlan pl;
+  int st = plan_for(p, g, kOpRoute, ws_bytes, &pl);
+  if (st != PISA_OK) return st;
+  st = clear_status(ws, s);
+  if (st != PISA_OK) return st;
+  g_mark_n = 0;
+  if (pl.n == 1) st = do_route(p, g, q, k, pyr, idx, margin, nullptr, ws, ws_bytes, s);
+  else
+    st = run_chunks(p, g, pl, ws, s, [&](const ChunkView& v, int) {
+      return tensor_route(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, pyr,
+                          idx + v.unit0 * g.N * g.K, margin ? margin + v.unit0 * g.N : nullptr, nullptr, v.region,
+                          (int32_t*)ws, v.stream);
+    });
+  kernel_mark("end", s);
+  return st;
+}
+
+static int do_bsa_chunked(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v_,
+                          const int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes, cudaStream_t s) {
+  ForwardPlan pl;
+  int st = plan_for(p, g, kOpBsa, ws_bytes, &pl);
+  if (st != PISA_OK) return st;
+  st = clear_status(ws, s);
+  if (st != PISA_OK) return st;
+  g_mark_n = 0;
+  if (pl.n == 1) st = do_bsa(p, g, q, k, v_, idx, out, lse, false, ws, ws_bytes, s);
+  else
+    st = run_chunks(p, g, pl, ws, s, [&](const ChunkView& v, int) {
+      return tensor_bsa(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, (const char*)v_ + v.v_off,
+                        idx + v.unit0 * g.N * g.K, (char*)out + v.o_off, lse + v.unit0 * g.G * g.N, false, v.region,
+                        (int32_t*)ws, v.stream);
+    });
+  kernel_mark("end", s);
+  return st;
+}
+
+static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v_,
                       void* pyr, int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes,
                       cudaStream_t s, bool clear = true) {
   ForwardPlan pl;
-  int st = forward_plan(p, g, &pl);
+  int st = plan_for(p, g, kOpRoute | kOpBsa, ws_bytes, &pl);
   if (st != PISA_OK) return st;
-  if (pl.n > 1 && ws_bytes < pl.total) {     // a workspace sized for another length of the same problem: unsplit
-    const size_t r = route_ws_bytes(p, g), b = bsa_ws_bytes(p, g);
-    pl.n = 1;
-    pl.total = r > b ? r : b;
-  }
-  if (ws_bytes < pl.total) return PISA_ERR_WORKSPACE_TOO_SMALL;
-  if (pl.n > 1 && (st = side_streams()) != PISA_OK) return st;
   st = clear ? clear_status(ws, s) : PISA_OK;
   if (st != PISA_OK) return st;
   g_mark_n = 0;
@@ -328,47 +424,19 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
     st = do_route(p, g, q, k, pyr, idx, nullptr, lse, ws, ws_bytes, s);
     if (st != PISA_OK) return st;
     stage_mark(2, s);
-    st = do_bsa(p, g, q, k, v, idx, out, lse, use_tensor(p, g) && g.score_mode == PISA_SCORE_LSE, ws, ws_bytes, s);
-    stage_mark(3, s);
-    kernel_mark("end", s);
-    return st;
+    st = do_bsa(p, g, q, k, v_, idx, out, lse, use_tensor(p, g) && g.score_mode == PISA_SCORE_LSE, ws, ws_bytes, s);
+  } else {
+    st = run_chunks(p, g, pl, ws, s, [&](const ChunkView& v, int i) {
+      int32_t* ic = idx + v.unit0 * g.N * g.K;
+      float* lc = lse + v.unit0 * g.G * g.N;
+      int r = tensor_route(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, pyr, ic, nullptr, lc,
+                           v.region, (int32_t*)ws, v.stream);
+      if (r != PISA_OK) return r;
+      if (i == 0) stage_mark(2, s);
+      return tensor_bsa(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, (const char*)v_ + v.v_off,
+                        ic, (char*)out + v.o_off, lc, g.score_mode == PISA_SCORE_LSE, v.region, (int32_t*)ws, v.stream);
+    });
   }
-  // fork: the internal stream starts after the pyramid (and after whatever the caller queued before)
-  cudaError_t e = cudaEventRecord(g_fork, s);
-  for (int i = 1; i < pl.streams && e == cudaSuccess; ++i) e = cudaStreamWaitEvent(g_side[i], g_fork, 0);
-  if (e != cudaSuccess) { record_cuda_error("fork", e); return PISA_ERR_CUDA; }
-  const size_t es = elem_size(p->dtype);
-  int32_t* status = (int32_t*)ws;
-  st = PISA_OK;
-  for (int i = 0; i < pl.n && st == PISA_OK; ++i) {
-    const Chunk& c = pl.c[i];
-    pisa_params_t pc;
-    Geometry gc;
-    st = chunk_problem(p, g, c, &pc, &gc);
-    if (st != PISA_OK) break;
-    const int si = i % pl.streams;
-    cudaStream_t cs = si ? g_side[si] : s;
-    char* region = (char*)ws + kStatusBytes + (size_t)si * pl.region;
-    const long long unit0 = (long long)c.b0 * g.Hkv + c.h0;
-    const char* qc = (const char*)q + ((long long)c.b0 * g.qs[0] + (long long)c.h0 * g.G * g.qs[2]) * es;
-    const char* kc = (const char*)k + ((long long)c.b0 * g.ks[0] + (long long)c.h0 * g.ks[2]) * es;
-    const char* vc = (const char*)v + ((long long)c.b0 * g.vs[0] + (long long)c.h0 * g.vs[2]) * es;
-    char* oc = (char*)out + ((long long)c.b0 * g.os[0] + (long long)c.h0 * g.G * g.os[2]) * es;
-    int32_t* ic = idx + unit0 * g.N * g.K;
-    float* lc = lse + unit0 * g.G * g.N;
-    st = tensor_route(gc, p->dtype, qc, kc, pyr, ic, nullptr, lc, region, status, cs);
-    if (st != PISA_OK) break;
-    if (i == 0) stage_mark(2, s);
-    st = tensor_bsa(gc, p->dtype, qc, kc, vc, ic, oc, lc, g.score_mode == PISA_SCORE_LSE, region, status, cs);
-  }
-  // join, also after a failed launch: the caller's stream must not run ahead of the internal one
-  e = cudaSuccess;
-  for (int i = 1; i < pl.streams; ++i) {
-    kernel_mark("end", g_side[i]);
-    if (e == cudaSuccess) e = cudaEventRecord(g_join[i], g_side[i]);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(s, g_join[i], 0);
-  }
-  if (e != cudaSuccess && st == PISA_OK) { record_cuda_error("join", e); st = PISA_ERR_CUDA; }
   stage_mark(3, s);
   kernel_mark("end", s);
   return st;
@@ -417,12 +485,18 @@ int pisa_workspace_bytes(const pisa_params_t* p, int op, size_t* bytes) {
   int st = resolve(p, &g);
   if (st != PISA_OK) return st;
   if (bytes == nullptr) return PISA_ERR_INVALID_ARG;
-  const size_t r = route_ws_bytes(p, g), a = bsa_ws_bytes(p, g);
-  size_t f = r > a ? r : a;                  // also lets one buffer serve pisa_route and pisa_bsa_fwd
+  size_t r = route_ws_bytes(p, g), a = bsa_ws_bytes(p, g);
+  {                                          // the chunked plans of the three calls
+    ForwardPlan pl;
+    if ((st = forward_plan(p, g, kOpRoute, &pl)) != PISA_OK) return st;
+    if (pl.total > r) r = pl.total;
+    if ((st = forward_plan(p, g, kOpBsa, &pl)) != PISA_OK) return st;
+    if (pl.total > a) a = pl.total;
+  }
+  size_t f = r > a ? r : a;                  // one buffer sized for the forward also serves pisa_route and pisa_bsa_fwd
   {
     ForwardPlan pl;
-    st = forward_plan(p, g, &pl);
-    if (st != PISA_OK) return st;
+    if ((st = forward_plan(p, g, kOpRoute | kOpBsa, &pl)) != PISA_OK) return st;
     if (pl.total > f) f = pl.total;
   }
   switch (op) {
@@ -466,9 +540,7 @@ int pisa_route(const pisa_params_t* p, const void* q, const void* k, const void*
   if (!q || !k || !pyramid || !idx || !ws || misaligned(q) || misaligned(k) || misaligned(pyramid) ||
       misaligned(ws))
     return PISA_ERR_INVALID_ARG;
-  st = clear_status(ws, (cudaStream_t)stream);
-  if (st != PISA_OK) return st;
-  return do_route(p, g, q, k, pyramid, idx, margin, nullptr, ws, ws_bytes, (cudaStream_t)stream);
+  return do_route_chunked(p, g, q, k, pyramid, idx, margin, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 int pisa_bsa_fwd(const pisa_params_t* p, const void* q, const void* k, const void* v, const int32_t* idx,
@@ -479,9 +551,7 @@ int pisa_bsa_fwd(const pisa_params_t* p, const void* q, const void* k, const voi
   if (!q || !k || !v || !idx || !out || !lse || !ws || misaligned(q) || misaligned(k) || misaligned(v) ||
       misaligned(out) || misaligned(ws))
     return PISA_ERR_INVALID_ARG;
-  st = clear_status(ws, (cudaStream_t)stream);
-  if (st != PISA_OK) return st;
-  return do_bsa(p, g, q, k, v, idx, out, lse, false, ws, ws_bytes, (cudaStream_t)stream);
+  return do_bsa_chunked(p, g, q, k, v, idx, out, lse, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const void* v, void* pyramid,
