@@ -14,7 +14,7 @@ from paper_2609_31093_b200 import binding as PB  # noqa: E402
 
 
 def test_packed_sequences_equal_the_sequences_alone_and_the_oracle():
-    lens = [700, 64, 1, 2085, 0, 130, 4096]
+    lens = [700, 64, 1, 2085, 0, 130, 70000]          # the last one is long enough to run as two chunks
     Hq, Hkv, d, C, g, K = 8, 2, 128, 64, 2, 4
     cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
     total = int(cu[-1])
