@@ -727,7 +727,7 @@ def run_backward(args):
     dout = torch.randn(q.shape, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
     dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
     wsb = PB.alloc_workspace(p, PB.OP_BSA_BWD)
-    P.set_stage_timing(True)
+    P.set_forward_chunks(args.forward_chunks)
     for _ in range(max(1, args.warmup)):
         P.pisa_bsa_bwd(p, q, k, v, idx, out, lse, dout, dq, dk, dv, wsb)
     torch.cuda.synchronize()
@@ -738,11 +738,19 @@ def run_backward(args):
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / args.steps
+    # per-kernel times: one more call with every kernel alone on the GPU (a large backward runs as
+    # chunks on two streams, as the forward does)
+    P.set_forward_chunks(1)
+    P.set_stage_timing(True)
+    P.pisa_bsa_bwd(p, q, k, v, idx, out, lse, dout, dq, dk, dv, wsb)
     kern = P.get_kernel_ms()
+    P.set_stage_timing(False)
+    P.set_forward_chunks(args.forward_chunks)
     wc = work_counts(w)
     flops = 2.5 * wc["attn_flops"]                     # five products of the forward's two shapes
     t_tiles = kern.get("backward_tiles", ms)
     row = {"backward": describe(w), "ms_per_call": ms, "tokens_per_s": w.B * w.N / (ms * 1e-3), "kernels_ms": kern,
+           "kernels_ms_note": "each kernel alone (chunking off); ms_per_call is the chunked call",
            "algorithmic_tflop": flops / 1e12,
            "roofline": {"kernel": "backward_tiles", "bound": "tensor", "achieved": flops / (t_tiles * 1e-3) / 1e12,
                         "peak": tens_peak, "unit": "TFLOP/s", "frac": flops / (t_tiles * 1e-3) / 1e12 / tens_peak},

@@ -58,12 +58,15 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(Geometry geo, const __nv
 }
 
 // fp32 -> bf16, contiguous
+// fp32 accumulator rows of `row2` element pairs, dense -> bf16 rows `dst_pitch2` pairs apart (a chunk of
+// KV heads writes its columns of the caller's [B, N, Hkv, d] tensor)
 __global__ void __launch_bounds__(256) bwd_convert_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst,
-                                                          long long n2) {
+                                                          long long n2, int row2, long long dst_pitch2) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n2) return;
   const float2 x = reinterpret_cast<const float2*>(src)[i];
-  reinterpret_cast<__nv_bfloat162*>(dst)[i] = __floats2bfloat162_rn(x.x, x.y);
+  const long long row = i / row2;
+  reinterpret_cast<__nv_bfloat162*>(dst)[row * dst_pitch2 + (i - row * row2)] = __floats2bfloat162_rn(x.x, x.y);
 }
 
 // 256 threads copy `nrows` rows of 256 bytes ([row][128 bf16]) into two swizzled K-major slabs of

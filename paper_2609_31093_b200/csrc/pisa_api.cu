@@ -237,7 +237,19 @@ static int chunk_problem(const pisa_params_t* p, const Geometry& g, const Chunk&
   return PISA_OK;
 }
 
-constexpr int kOpRoute = 1, kOpBsa = 2;
+constexpr int kOpRoute = 1, kOpBsa = 2, kOpBwd = 4;
+
+static bool ops_supported(const pisa_params_t* p, const Geometry& g, int ops) {
+  if (ops == kOpBwd) return p->impl != PISA_IMPL_SIMT && tensor_bwd_supported(g, p->dtype);
+  return use_tensor(p, g);
+}
+static size_t ops_ws_bytes(const pisa_params_t* p, const Geometry& g, int ops) {     // with the status word
+  size_t m = kStatusBytes;
+  if (ops & kOpRoute) { const size_t r = route_ws_bytes(p, g); if (r > m) m = r; }
+  if (ops & kOpBsa) { const size_t b = bsa_ws_bytes(p, g); if (b > m) m = b; }
+  if (ops & kOpBwd) { const size_t b = kStatusBytes + tensor_bwd_workspace_bytes(g); if (b > m) m = b; }
+  return m;
+}
 
 static int forward_plan(const pisa_params_t* p, const Geometry& g, int ops, ForwardPlan* pl) {
   pl->n = 1;
@@ -247,7 +259,7 @@ static int forward_plan(const pisa_params_t* p, const Geometry& g, int ops, Forw
   if (parts > kMaxChunks) parts = kMaxChunks;
   if (g_chunk_limit > 0 && parts > g_chunk_limit) parts = g_chunk_limit;
   if (parts > units) parts = units;
-  if (use_tensor(p, g) && parts >= 2) {
+  if (ops_supported(p, g, ops) && parts >= 2) {
     int n = 0;
     if (g.B >= parts) {                       // whole batches
       for (int i = 0; i < parts; ++i) {
@@ -271,16 +283,14 @@ static int forward_plan(const pisa_params_t* p, const Geometry& g, int ops, Forw
     Geometry gc;
     const int st = chunk_problem(p, g, pl->c[i], &pc, &gc);
     if (st != PISA_OK) return st;
-    if (pl->n > 1 && !use_tensor(&pc, gc)) {   // a chunk the tensor path does not take: run unsplit
+    if (pl->n > 1 && !ops_supported(&pc, gc, ops)) {   // a chunk the tensor path does not take: run unsplit
       pl->n = 1;
       pl->c[0] = {0, g.B, 0, g.Hkv};
       i = -1;
       region = 0;
       continue;
     }
-    const size_t r = (ops & kOpRoute) ? route_ws_bytes(&pc, gc) - kStatusBytes : 0;
-    const size_t b = (ops & kOpBsa) ? bsa_ws_bytes(&pc, gc) - kStatusBytes : 0;
-    const size_t m = align_up(r > b ? r : b, 256);
+    const size_t m = align_up(ops_ws_bytes(&pc, gc, ops) - kStatusBytes, 256);
     if (m > region) region = m;
   }
   pl->region = region;
@@ -308,6 +318,7 @@ static int side_streams() {
 struct ChunkView {
   pisa_params_t p;
   Geometry g;
+  Chunk c;
   long long unit0;              // first (batch, KV head) unit, flattened
   size_t q_off, k_off, v_off, o_off;   // byte offsets into q / k / v / out
   char* region;                 // this chunk's scratch (past any status word)
@@ -320,10 +331,9 @@ static int plan_for(const pisa_params_t* p, const Geometry& g, int ops, size_t w
   int st = forward_plan(p, g, ops, pl);
   if (st != PISA_OK) return st;
   if (pl->n > 1 && ws_bytes < pl->total) {   // a workspace sized for another length of the same problem: unsplit
-    const size_t r = (ops & kOpRoute) ? route_ws_bytes(p, g) : 0, b = (ops & kOpBsa) ? bsa_ws_bytes(p, g) : 0;
     pl->n = 1;
     pl->streams = 1;
-    pl->total = r > b ? r : b;
+    pl->total = ops_ws_bytes(p, g, ops);
   }
   if (ws_bytes < pl->total) return PISA_ERR_WORKSPACE_TOO_SMALL;
   if (pl->n > 1) return side_streams();
@@ -347,6 +357,7 @@ static int run_chunks(const pisa_params_t* p, const Geometry& g, const ForwardPl
     st = chunk_problem(p, g, c, &v.p, &v.g);
     if (st != PISA_OK) break;
     const int si = i % pl.streams;
+    v.c = c;
     v.stream = si ? g_side[si] : s;
     v.region = (char*)ws + kStatusBytes + (size_t)si * pl.region;
     v.unit0 = (long long)c.b0 * g.Hkv + c.h0;
@@ -402,6 +413,29 @@ static int do_bsa_chunked(const pisa_params_t* p, const Geometry& g, const void*
     });
   kernel_mark("end", s);
   return st;
+}
+
+// Attention backward of one dense problem (dq, dk, dv dense like q, k, v), in chunks when it is large.
+static int do_bwd(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v_,
+                  const int32_t* idx, const void* out, const float* lse, const void* dout, void* dq, void* dk,
+                  void* dv, void* ws, size_t ws_bytes, cudaStream_t s) {
+  ForwardPlan pl;
+  int st = plan_for(p, g, kOpBwd, ws_bytes, &pl);
+  if (st != PISA_OK) return st;
+  const size_t es = elem_size(p->dtype);
+  const long long dqs[3] = {(long long)g.N * g.Hq * g.d, (long long)g.Hq * g.d, g.d};
+  const long long pitch = (long long)g.Hkv * g.d;
+  if (pl.n == 1)
+    return tensor_bsa_bwd(g, q, k, v_, idx, out, lse, dout, dq, dk, dv, dqs, pitch, (char*)ws + kStatusBytes,
+                          (int32_t*)ws, s);
+  return run_chunks(p, g, pl, ws, s, [&](const ChunkView& v, int) {
+    const size_t dq_off = (size_t)((long long)v.c.b0 * dqs[0] + (long long)v.c.h0 * g.G * dqs[2]) * es;
+    const size_t dkv_off = (size_t)((long long)v.c.b0 * g.N * pitch + (long long)v.c.h0 * g.d) * es;
+    return tensor_bsa_bwd(v.g, (const char*)q + v.q_off, (const char*)k + v.k_off, (const char*)v_ + v.v_off,
+                          idx + v.unit0 * g.N * g.K, (const char*)out + v.o_off, lse + v.unit0 * g.G * g.N,
+                          (const char*)dout + v.o_off, (char*)dq + dq_off, (char*)dk + dkv_off, (char*)dv + dkv_off, dqs,
+                          pitch, v.region, (int32_t*)ws, v.stream);
+  });
 }
 
 static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v_,
@@ -507,6 +541,11 @@ int pisa_workspace_bytes(const pisa_params_t* p, int op, size_t* bytes) {
     case PISA_OP_BSA_BWD:
       if (!tensor_bwd_supported(g, p->dtype) || p->impl == PISA_IMPL_SIMT) return PISA_ERR_UNSUPPORTED;
       *bytes = kStatusBytes + tensor_bwd_workspace_bytes(g);
+      {
+        ForwardPlan pl;
+        if ((st = forward_plan(p, g, kOpBwd, &pl)) != PISA_OK) return st;
+        if (pl.total > *bytes) *bytes = pl.total;
+      }
       break;
     case PISA_OP_DECODE:
       if (!decode_supported(g, p->dtype)) return PISA_ERR_UNSUPPORTED;
@@ -721,12 +760,15 @@ int pisa_bsa_bwd(const pisa_params_t* p, const void* q, const void* k, const voi
       misaligned(dk) || misaligned(dv) || misaligned(ws))
     return PISA_ERR_INVALID_ARG;
   if (!tensor_bwd_supported(g, p->dtype) || p->impl == PISA_IMPL_SIMT) return PISA_ERR_UNSUPPORTED;
-  if (ws_bytes < kStatusBytes + tensor_bwd_workspace_bytes(g)) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  {
+    ForwardPlan pl;                            // sizes are checked before anything is queued
+    if ((st = plan_for(p, g, kOpBwd, ws_bytes, &pl)) != PISA_OK) return st;
+  }
   cudaStream_t s = (cudaStream_t)stream;
   st = clear_status(ws, s);
   if (st != PISA_OK) return st;
   g_mark_n = 0;
-  st = tensor_bsa_bwd(g, q, k, v, idx, out, lse, dout, dq, dk, dv, (char*)ws + kStatusBytes, (int32_t*)ws, s);
+  st = do_bwd(p, g, q, k, v, idx, out, lse, dout, dq, dk, dv, ws, ws_bytes, s);
   kernel_mark("end", s);
   return st;
 }
@@ -774,9 +816,9 @@ int pisa_bsa_bwd_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32
     st = resolve(&pi, &gi);
     if (st != PISA_OK) return st;
     const size_t oq = t0 * g.Hq * g.d * es, ok = t0 * g.Hkv * g.d * es;
-    st = tensor_bsa_bwd(gi, (const char*)q + oq, (const char*)k + ok, (const char*)v + ok, idx + t0 * g.Hkv * g.K,
-                        (const char*)out + oq, lse + t0 * g.Hq, (const char*)dout + oq, (char*)dq + oq,
-                        (char*)dk + ok, (char*)dv + ok, (char*)ws + kStatusBytes, (int32_t*)ws, s);
+    st = do_bwd(&pi, gi, (const char*)q + oq, (const char*)k + ok, (const char*)v + ok, idx + t0 * g.Hkv * g.K,
+                (const char*)out + oq, lse + t0 * g.Hq, (const char*)dout + oq, (char*)dq + oq, (char*)dk + ok,
+                (char*)dv + ok, ws, ws_bytes, s);
     if (st != PISA_OK) return st;
   }
   kernel_mark("end", s);

@@ -19,8 +19,10 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
 // backward of the block-sparse attention with frozen indices; dq [B,N,Hq,d], dk, dv [B,N,Hkv,d] dense
 bool tensor_bwd_supported(const Geometry& g, int dtype);
 size_t tensor_bwd_workspace_bytes(const Geometry& g);
+// dq_strides: element strides (b, n, h) of dq; dkv_pitch: elements between consecutive tokens of dk / dv
+// (both describe the caller's dense tensors, of which a chunk of units writes its part)
 int tensor_bsa_bwd(const Geometry& g, const void* q, const void* k, const void* v, const int32_t* idx,
-                   const void* out, const float* lse, const void* dout, void* dq, void* dk, void* dv, void* ws,
-                   int32_t* status, cudaStream_t s);
+                   const void* out, const float* lse, const void* dout, void* dq, void* dk, void* dv,
+                   const long long* dq_strides, long long dkv_pitch, void* ws, int32_t* status, cudaStream_t s);
 
 }  // namespace pisa

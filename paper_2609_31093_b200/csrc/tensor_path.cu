@@ -1455,8 +1455,8 @@ bool tensor_bwd_supported(const Geometry& g, int dtype) {
 size_t tensor_bwd_workspace_bytes(const Geometry& g) { return bwd_layout(g).total; }
 
 int tensor_bsa_bwd(const Geometry& g, const void* q, const void* k, const void* v, const int32_t* idx,
-                   const void* out, const float* lse, const void* dout, void* dq, void* dk, void* dv, void* ws_,
-                   int32_t* status, cudaStream_t s) {
+                   const void* out, const float* lse, const void* dout, void* dq, void* dk, void* dv,
+                   const long long* dq_strides, long long dkv_pitch, void* ws_, int32_t* status, cudaStream_t s) {
   char* ws = (char*)ws_;
   const BwdLayout L = bwd_layout(g);
   kernel_mark("invert_by_leaf", s);
@@ -1489,15 +1489,16 @@ int tensor_bsa_bwd(const Geometry& g, const void* q, const void* k, const void* 
   if (st != PISA_OK) return st;
   kernel_mark("convert_gradients", s);
   {
-    Geometry gd = g;                                   // dq is dense [B, N, Hq, d]
-    gd.os[2] = g.d; gd.os[1] = (long long)g.Hq * g.d; gd.os[0] = (long long)g.N * g.Hq * g.d;
+    Geometry gd = g;                                   // dq: the caller's dense [B, N, Hq, d] (this chunk's heads of it)
+    gd.os[0] = dq_strides[0]; gd.os[1] = dq_strides[1]; gd.os[2] = dq_strides[2];
     const long long n = (long long)g.B * g.N * g.Hkv * (g.d / 2);
     convert_out_heads_inner_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(gd, a.dq_acc, (__nv_bfloat16*)dq);
     st = check_launch("convert_dq");
     if (st != PISA_OK) return st;
     const long long n2 = (long long)g.B * g.N * g.Hkv * g.d / 2;
-    bwd_convert_kernel<<<(unsigned)((n2 + 255) / 256), 256, 0, s>>>(a.dk_acc, (__nv_bfloat16*)dk, n2);
-    bwd_convert_kernel<<<(unsigned)((n2 + 255) / 256), 256, 0, s>>>(a.dv_acc, (__nv_bfloat16*)dv, n2);
+    const int row2 = g.Hkv * g.d / 2;                 // one token's pairs in the accumulator; dkv_pitch in the output
+    bwd_convert_kernel<<<(unsigned)((n2 + 255) / 256), 256, 0, s>>>(a.dk_acc, (__nv_bfloat16*)dk, n2, row2, dkv_pitch / 2);
+    bwd_convert_kernel<<<(unsigned)((n2 + 255) / 256), 256, 0, s>>>(a.dv_acc, (__nv_bfloat16*)dv, n2, row2, dkv_pitch / 2);
     st = check_launch("convert_dkv");
   }
   return st;
