@@ -248,7 +248,7 @@ int pisa_bsa_bwd_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32
  *
  * The step selects exactly what the prefill path selects for row pos of the same sequence (every
  * scored node lies strictly in the past of the query) and attends over keys <= pos of the selected
- * blocks.  bf16, LSE score mode, d in {64, 128}, C in {32, 64, 128}, group size <= 16; other
+ * blocks.  bf16, every score mode, d in {64, 128}, C in {32, 64, 128}, group size <= 16; other
  * configurations return PISA_ERR_UNSUPPORTED.  Asynchronous on `stream`; allocates nothing.
  */
 int pisa_decode_step(const pisa_params_t* p, int32_t pos, const void* q, const void* k_cache,

@@ -57,6 +57,19 @@ __device__ __forceinline__ float ex2f(float x) {
   return y;
 }
 
+// One logit into a candidate's running score state (Sec. 4.3).  LSE score: (m, acc) = running max and sum
+// of exponentials.  Moment scores: m = the shift (the candidate's first logit, set by the caller), acc and
+// sq = first and second moments about it.
+__device__ __forceinline__ void score_add(int mode, float& m, float& acc, float& sq, float z) {
+  if (mode == PISA_SCORE_LSE) lse_add(m, acc, z);
+  else { const float dl = z - m; acc += dl; sq += dl * dl; }
+}
+__device__ __forceinline__ float score_finish(int mode, float m, float acc, float sq, int n) {
+  if (mode == PISA_SCORE_LSE) return m + __logf(acc);
+  const float mu = acc / (float)n;
+  return m + mu + ((mode == PISA_SCORE_MEAN_VAR) ? 0.5f * fmaxf(sq / (float)n - mu * mu, 0.f) : 0.f);
+}
+
 // The new token's path in the cached pyramid, by one whole CTA.  Nothing in the same step reads these
 // nodes (the path is forced, never scored), so this runs off the critical path, after the CTA's share
 // of the attention.  The current leaf's mean takes every loaded key in one round (eight warps, sixteen
@@ -122,8 +135,9 @@ __device__ void refresh_path(const Geometry& geo, const DecArgs& a, int b, int h
 
 // MINB = 1: all registers to one CTA per SM (lowest latency, small batches); MINB = 2: two CTAs per SM so
 // that the latency-bound phases of different clusters overlap once the grid exceeds the SM count.
-// CLU: CTAs per cluster.
-template <int D, int NT, int MINB, int CLU>
+// CLU: CTAs per cluster.  MOM: false = LSE score (the state of the other scores folds away), true = the
+// mean / mean + variance scores.
+template <int D, int NT, int MINB, int CLU, bool MOM>
 __global__ void __cluster_dims__(CLU, 1, 1) __launch_bounds__(kDecThreads, MINB)
 decode_step_kernel(Geometry geo, DecArgs a) {
   extern __shared__ float s_part[];                       // [kDecWarps][G*D + 2*G] attention partials
@@ -140,6 +154,7 @@ decode_step_kernel(Geometry geo, DecArgs a) {
   const int bh = blockIdx.y;
   const int b = bh / geo.Hkv, h = bh % geo.Hkv;
   const int K = geo.K, g = geo.g, G = geo.G, C = geo.C;
+  const int mode = MOM ? geo.score_mode : (int)PISA_SCORE_LSE;
   const int pos = a.pos;
   const int c = pos / C;
   const int f1 = (c >= 1) ? c - 1 : 0;
@@ -188,9 +203,12 @@ decode_step_kernel(Geometry geo, DecArgs a) {
         const int kap = k0 + gid;
         const bool has = kap < nV;
         const int node = has ? cand[kap] : 0;
-        float m[NT][2], ssum[NT][2];
+        float m[NT][2], ssum[NT][2], sq[NT][2];
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) { m[nt][0] = m[nt][1] = -CUDART_INF_F; ssum[nt][0] = ssum[nt][1] = 0.f; }
+        for (int nt = 0; nt < NT; ++nt) {
+          m[nt][0] = m[nt][1] = -CUDART_INF_F; ssum[nt][0] = ssum[nt][1] = 0.f; sq[nt][0] = sq[nt][1] = 0.f;
+        }
+        const int nch = has ? min(g, Mb - node * g) : 1;        // valid children of the candidate
         for (int r0 = 0; r0 < g; r0 += 2) {
           const int ch_lo = node * g + r0, ch_hi = ch_lo + 1;
           const bool ok_lo = has && ch_lo < Mb, ok_hi = has && (r0 + 1 < g) && ch_hi < Mb;
@@ -201,8 +219,9 @@ decode_step_kernel(Geometry geo, DecArgs a) {
           for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int jh = 0; jh < 2; ++jh) {
-              if (ok_lo) lse_add(m[nt][jh], ssum[nt][jh], z[nt][jh] * geo.scale);
-              if (ok_hi) lse_add(m[nt][jh], ssum[nt][jh], z[nt][2 + jh] * geo.scale);
+              if (mode != PISA_SCORE_LSE && r0 == 0) m[nt][jh] = z[nt][jh] * geo.scale;   // shift: the first child
+              if (ok_lo) score_add(mode, m[nt][jh], ssum[nt][jh], sq[nt][jh], z[nt][jh] * geo.scale);
+              if (ok_hi) score_add(mode, m[nt][jh], ssum[nt][jh], sq[nt][jh], z[nt][2 + jh] * geo.scale);
             }
         }
         float usum = 0.f;
@@ -210,7 +229,7 @@ decode_step_kernel(Geometry geo, DecArgs a) {
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
           for (int jh = 0; jh < 2; ++jh)
-            if (nt * 8 + 2 * tig + jh < G && has) usum += m[nt][jh] + __logf(ssum[nt][jh]);
+            if (nt * 8 + 2 * tig + jh < G && has) usum += score_finish(mode, m[nt][jh], ssum[nt][jh], sq[nt][jh], nch);
         usum += __shfl_xor_sync(0xffffffffu, usum, 1);
         usum += __shfl_xor_sync(0xffffffffu, usum, 2);
         if (has && tig == 0) s_u[kap] = (node == 0 || node == f1l || node == anc_c) ? forced_score(kap) : usum;
@@ -258,9 +277,11 @@ decode_step_kernel(Geometry geo, DecArgs a) {
       const int leaf = cand1[ci];
       if (leaf == 0 || leaf == f1 || leaf == c) continue;        // forced: never scored
       // a scored leaf lies strictly before the current one: all C keys exist and are visible
-      float m[NT][2], ssum[NT][2];
+      float m[NT][2], ssum[NT][2], sq[NT][2];
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt) { m[nt][0] = m[nt][1] = -CUDART_INF_F; ssum[nt][0] = ssum[nt][1] = 0.f; }
+      for (int nt = 0; nt < NT; ++nt) {
+        m[nt][0] = m[nt][1] = -CUDART_INF_F; ssum[nt][0] = ssum[nt][1] = 0.f; sq[nt][0] = sq[nt][1] = 0.f;
+      }
       for (int kt = 0; kt < C; kt += 32) {                       // two key tiles in flight per round
         const long long t_lo = (long long)leaf * C + kt + gid;
         RowPair<D> r0, r1;
@@ -268,20 +289,28 @@ decode_step_kernel(Geometry geo, DecArgs a) {
         r1.load(kbh + (t_lo + 16) * geo.ks[1], kbh + (t_lo + 24) * geo.ks[1], lane);
         float z[NT][4];
         rows2_dot<D, NT>(qf, r0, z);
+        if (mode != PISA_SCORE_LSE && kt == 0) {
+          // moment scores: every lane shifts by the logit of the block's first key, which the lanes with
+          // gid = 0 (lane = tig) hold for their two heads
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int jh = 0; jh < 2; ++jh) m[nt][jh] = __shfl_sync(0xffffffffu, z[nt][jh] * geo.scale, tig);
+        }
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
           for (int jh = 0; jh < 2; ++jh) {
-            lse_add(m[nt][jh], ssum[nt][jh], z[nt][jh] * geo.scale);
-            lse_add(m[nt][jh], ssum[nt][jh], z[nt][2 + jh] * geo.scale);
+            score_add(mode, m[nt][jh], ssum[nt][jh], sq[nt][jh], z[nt][jh] * geo.scale);
+            score_add(mode, m[nt][jh], ssum[nt][jh], sq[nt][jh], z[nt][2 + jh] * geo.scale);
           }
         rows2_dot<D, NT>(qf, r1, z);
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
           for (int jh = 0; jh < 2; ++jh) {
-            lse_add(m[nt][jh], ssum[nt][jh], z[nt][jh] * geo.scale);
-            lse_add(m[nt][jh], ssum[nt][jh], z[nt][2 + jh] * geo.scale);
+            score_add(mode, m[nt][jh], ssum[nt][jh], sq[nt][jh], z[nt][jh] * geo.scale);
+            score_add(mode, m[nt][jh], ssum[nt][jh], sq[nt][jh], z[nt][2 + jh] * geo.scale);
           }
       }
       float usum = 0.f;
@@ -294,9 +323,11 @@ decode_step_kernel(Geometry geo, DecArgs a) {
           for (int o = 4; o < 32; o <<= 1) {
             const float m2 = __shfl_xor_sync(0xffffffffu, m[nt][jh], o);
             const float s2 = __shfl_xor_sync(0xffffffffu, ssum[nt][jh], o);
-            lse_merge(m[nt][jh], ssum[nt][jh], m2, s2);
+            const float q2 = __shfl_xor_sync(0xffffffffu, sq[nt][jh], o);
+            if (mode == PISA_SCORE_LSE) lse_merge(m[nt][jh], ssum[nt][jh], m2, s2);
+            else { ssum[nt][jh] += s2; sq[nt][jh] += q2; }         // same shift in every lane
           }
-          if (nt * 8 + 2 * tig + jh < G) usum += m[nt][jh] + __logf(ssum[nt][jh]);
+          if (nt * 8 + 2 * tig + jh < G) usum += score_finish(mode, m[nt][jh], ssum[nt][jh], sq[nt][jh], C);
         }
       usum += __shfl_xor_sync(0xffffffffu, usum, 1);
       usum += __shfl_xor_sync(0xffffffffu, usum, 2);
@@ -483,14 +514,19 @@ decode_step_kernel(Geometry geo, DecArgs a) {
   }
 }
 
-template <int D, int NT, int MINB, int CLU>
-int launch_dnb(const Geometry& g, const DecArgs& a, cudaStream_t s) {
+template <int D, int NT, int MINB, int CLU, bool MOM>
+int launch_dnbm(const Geometry& g, const DecArgs& a, cudaStream_t s) {
   const size_t smem = (size_t)kDecWarps * (g.G * D + 2 * g.G) * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(decode_step_kernel<D, NT, MINB, CLU>,
+  cudaError_t e = cudaFuncSetAttribute(decode_step_kernel<D, NT, MINB, CLU, MOM>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("decode_step attr", e); return PISA_ERR_CUDA; }
-  decode_step_kernel<D, NT, MINB, CLU><<<dim3(CLU, (unsigned)(g.B * g.Hkv)), kDecThreads, smem, s>>>(g, a);
+  decode_step_kernel<D, NT, MINB, CLU, MOM><<<dim3(CLU, (unsigned)(g.B * g.Hkv)), kDecThreads, smem, s>>>(g, a);
   return check_launch("decode_step");
+}
+template <int D, int NT, int MINB, int CLU>
+int launch_dnb(const Geometry& g, const DecArgs& a, cudaStream_t s) {
+  return (g.score_mode == PISA_SCORE_LSE) ? launch_dnbm<D, NT, MINB, CLU, false>(g, a, s)
+                                          : launch_dnbm<D, NT, MINB, CLU, true>(g, a, s);
 }
 // Eight CTAs per (batch, KV head) while all clusters fit the GPU at once (one, then two CTAs per SM);
 // beyond that narrower clusters, so that a large batch still runs as a single wave.
@@ -512,7 +548,7 @@ int launch_dn(const Geometry& g, const DecArgs& a, cudaStream_t s) {
 }  // namespace
 
 bool decode_supported(const Geometry& g, int dtype) {
-  return dtype == PISA_BF16 && g.score_mode == PISA_SCORE_LSE && (g.d == 64 || g.d == 128) && g.G <= 16 &&
+  return dtype == PISA_BF16 && (g.d == 64 || g.d == 128) && g.G <= 16 &&
          (g.C == 64 || g.C == 128 || g.C == 32) && (long long)g.B * g.Hkv <= 65535;
 }
 

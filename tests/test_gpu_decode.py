@@ -27,9 +27,9 @@ class Cache:
     """KV caches of capacity `cap` filled as a decoder would: row pos is written just before its step;
     everything not yet written is NaN, so any read of the future shows up in the results."""
 
-    def __init__(self, w, t, cap, filled=0):
-        self.w, self.cap = w, cap
-        self.p = P.Params(w.B, cap, w.Hq, w.Hkv, w.d, w.C, w.g, w.K, dtype="bf16")
+    def __init__(self, w, t, cap, filled=0, score_mode="lse"):
+        self.w, self.cap, self.mode = w, cap, score_mode
+        self.p = P.Params(w.B, cap, w.Hq, w.Hkv, w.d, w.C, w.g, w.K, dtype="bf16", score_mode=score_mode)
         self.k_src, self.v_src = T.to_torch(t["k"], "bf16"), T.to_torch(t["v"], "bf16")
         self.k = torch.full((w.B, cap, w.Hkv, w.d), float("nan"), dtype=torch.bfloat16, device="cuda")
         self.v = torch.full_like(self.k, float("nan"))
@@ -60,7 +60,7 @@ def _check_step(cache, t, pos):
     torch.cuda.synchronize()
     assert P.read_status(cache.ws) == 0
     idx_ref, margin, out_ref, lse_ref = O.decode_step(t["q"][:, pos], t["k"], t["v"], pos, C=w.C, g=w.g, K=w.K,
-                                                      dtype="bf16")
+                                                      dtype="bf16", mode=cache.mode)
     got = cache.idx.cpu().numpy()
     c = pos // w.C
     for b in range(w.B):
@@ -164,3 +164,20 @@ def test_decode_large_batches_use_narrower_clusters(B, Hkv):
         if pos % 4 == 0 or pos == w.N - 1:
             in_band += _check_step(cache, t, pos)
     print(f"[batch {B}] rows inside the tie band: {in_band}")
+
+
+@pytest.mark.parametrize("mode", ["mean", "mean_var"])
+@pytest.mark.parametrize("name", ["gqa4_c64", "fan4_c32"])
+def test_decode_score_modes(name, mode):
+    """The mean and mean + variance / 2 scores (Sec. 4.3) in the decoding step, fan-in 2 and 4."""
+    w = CASES[name]
+    t = S.make_inputs(w)
+    n0 = w.N - 48
+    cache = Cache(w, t, cap=w.N, filled=n0, score_mode=mode)
+    P.pisa_build_pyramid(cache.p, cache.k, cache.pyr)
+    in_band = 0
+    for pos in range(n0, w.N):
+        cache.step(pos)
+        if pos % 3 == 0 or pos == w.N - 1:
+            in_band += _check_step(cache, t, pos)
+    print(f"[{name} {mode}] rows inside the tie band: {in_band}")
