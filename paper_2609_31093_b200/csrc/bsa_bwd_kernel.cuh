@@ -112,11 +112,17 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
   uint8_t* sdS = sP + P_BYTES;
   uint8_t* sK = sdS + P_BYTES;
   uint8_t* sV = sK + 2 * KV_SLAB;
+  // C = 64 leaves room for a second pair of Q / dO tiles: the next tile is then gathered under the whole
+  // of the current one instead of only under its dQ^T reduction
+  constexpr bool DB = (C == 64);
+  constexpr int NM = DB ? 3 : 2;                            // metadata buffers: tiles jt, jt+1 (and jt+2)
+  uint8_t* sQ1 = sV + 2 * KV_SLAB;
+  uint8_t* sdO1 = sQ1 + 2 * A_SLAB;
   __shared__ uint64_t bar_mma;
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_fail;
-  __shared__ int s_ent2[2][128];                            // per-tile metadata, two tiles (current, next)
-  __shared__ float s_nlse22[2][128], s_delta2[2][128];
+  __shared__ int s_ent2[NM][128];                           // per-tile metadata
+  __shared__ float s_nlse22[NM][128], s_delta2[NM][128];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
@@ -173,13 +179,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
         dl = a.delta[li];
       }
     };
-    auto gather_tile = [&](const int* ents) {
-      bwd_load_rows<CHV>(sQ, A_SLAB, 128, tid, [&](int r) {
+    auto gather_tile = [&](const int* ents, int buf) {
+      bwd_load_rows<CHV>((DB && buf) ? sQ1 : sQ, A_SLAB, 128, tid, [&](int r) {
         const int ent = ents[r];
         return (ent >= 0) ? qb + (long long)(ent & 0xFFFFFF) * geo.qs[1] + (long long)(r & (G - 1)) * geo.qs[2]
                           : (const __nv_bfloat16*)nullptr;
       });
-      bwd_load_rows<CHV>(sdO, A_SLAB, 128, tid, [&](int r) {
+      bwd_load_rows<CHV>((DB && buf) ? sdO1 : sdO, A_SLAB, 128, tid, [&](int r) {
         const int ent = ents[r];
         return (ent >= 0) ? dob + (long long)(ent & 0xFFFFFF) * geo.os[1] + (long long)(r & (G - 1)) * geo.os[2]
                           : (const __nv_bfloat16*)nullptr;
@@ -191,24 +197,34 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
       int ent; float nl, dl;
       load_meta(0, ent, nl, dl);
       s_ent2[0][tid] = ent; s_nlse22[0][tid] = nl; s_delta2[0][tid] = dl;
+      if (DB) {
+        load_meta(1, ent, nl, dl);
+        s_ent2[1][tid] = ent; s_nlse22[1][tid] = nl; s_delta2[1][tid] = dl;
+      }
     }
     __syncthreads();
-    gather_tile(s_ent2[0]);
+    gather_tile(s_ent2[0], 0);
     for (int jt = 0; jt < inf.ntiles && !dead; ++jt) {
-      const int cb = jt & 1;
+      const int cb = jt % NM;                                // this tile's metadata buffer
+      const int nb = (jt + NM - 1) % NM;                     // where the metadata fetched during this tile goes
+      const int qb_i = DB ? (jt & 1) : 0;                    // this tile's Q / dO pair
       const int* s_ent = s_ent2[cb];
       const float* s_nlse2 = s_nlse22[cb];
       const float* s_delta = s_delta2[cb];
-      // next tile's metadata: loads issued now, stored once this tile's products are under way
+      // metadata of the tile after the one already known: loads issued now, stored once this tile's
+      // products are under way
       int n_ent = -1; float n_nl = 0.f, n_dl = 0.f;
-      if (tid < 128) load_meta(jt + 1, n_ent, n_nl, n_dl);
+      if (tid < 128) load_meta(jt + NM - 1, n_ent, n_nl, n_dl);
       cp_async_wait_all();
       fence_proxy_async_smem();
       __syncthreads();
+      // the other Q / dO pair was last read by the previous tile's products, which have completed
+      if (DB && jt + 1 < inf.ntiles) gather_tile(s_ent2[(jt + 1) % NM], qb_i ^ 1);
       // ---- S = Q K^T, dP = dO V^T
       if (tid == 0) {
         tcgen05_fence_after_sync();
-        const uint32_t q0 = smem_u32(sQ), o0 = smem_u32(sdO), k0 = smem_u32(sK), v0 = smem_u32(sV);
+        const uint32_t q0 = smem_u32(qb_i ? sQ1 : sQ), o0 = smem_u32(qb_i ? sdO1 : sdO), k0 = smem_u32(sK),
+                       v0 = smem_u32(sV);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint64_t da = make_smem_desc(q0 + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
@@ -278,7 +294,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
       // ---- dV^T += dO^T P,  dK^T += Q^T dS,  dQ^T = K^T dS^T
       if (tid == 0) {
         tcgen05_fence_after_sync();
-        const uint32_t q0 = smem_u32(sQ), o0 = smem_u32(sdO), k0 = smem_u32(sK);
+        const uint32_t q0 = smem_u32(qb_i ? sQ1 : sQ), o0 = smem_u32(qb_i ? sdO1 : sdO), k0 = smem_u32(sK);
         const uint32_t p0 = smem_u32(sP), s0 = smem_u32(sdS);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {                       // contraction over the 128 tile rows
@@ -306,10 +322,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bsa_bwd_kernel(Geometry geo, B
         if (__syncthreads_or(!ok)) { s_fail = 1; dead = true; break; }
       }
       tcgen05_fence_after_sync();
-      // Q, dO, P, dS tiles are free: bring in the next tile while this one's dQ^T is reduced
-      if (tid < 128) { s_ent2[cb ^ 1][tid] = n_ent; s_nlse22[cb ^ 1][tid] = n_nl; s_delta2[cb ^ 1][tid] = n_dl; }
+      // Q, dO, P, dS tiles are free: (single pair) bring in the next tile while this one's dQ^T is reduced
+      if (tid < 128) { s_ent2[nb][tid] = n_ent; s_nlse22[nb][tid] = n_nl; s_delta2[nb][tid] = n_dl; }
       __syncthreads();
-      if (jt + 1 < inf.ntiles) gather_tile(s_ent2[cb ^ 1]);
+      if (!DB && jt + 1 < inf.ntiles) gather_tile(s_ent2[nb], 0);
       // ---- dQ^T out of TMEM: lane = column d, TMEM column = tile row (entry*G + head); this warp's 64 rows
       {
         float* acc_d = a.dq_acc + (((long long)b * geo.Hkv + h) * geo.N) * (long long)(DIN * G) + (long long)row * G;

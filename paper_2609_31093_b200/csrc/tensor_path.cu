@@ -1348,7 +1348,9 @@ BwdLayout bwd_layout(const Geometry& g) {
 
 template <int C, int DIN>
 int launch_bwd(const Geometry& g, const BwdArgs& a, cudaStream_t s) {
-  const size_t smem = 4 * (size_t)(128 * 128) + 2 * (size_t)(C / 64) * (128 * 128) + 4 * (size_t)(C * 128) + 1024;
+  // Q, dO (two pairs when C = 64), P, dS, K, V
+  const size_t smem = (C == 64 ? 8 : 4) * (size_t)(128 * 128) + 2 * (size_t)(C / 64) * (128 * 128) +
+                      4 * (size_t)(C * 128) + 1024;
   cudaError_t e = cudaFuncSetAttribute(bsa_bwd_kernel<C, DIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("bsa_bwd attr", e); return PISA_ERR_CUDA; }
   bsa_bwd_kernel<C, DIN><<<num_sms(), kBwdThreads, smem, s>>>(g, a);
