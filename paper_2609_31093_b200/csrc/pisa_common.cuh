@@ -149,4 +149,45 @@ __device__ __forceinline__ void warp_select_ranks(const float* u, int n, int lan
   }
 }
 
+// Select_K for at most 64 candidates (two per lane: s = lane and lane + 32) without ranks: a bitonic
+// network sorts the 64 scores across the warp (padding = -inf), the K-th largest is the threshold, and
+// a candidate is kept if its score is larger, or equal with few enough equal ones before it (ties go to
+// the smaller position, as the ranks do).  u0 / u1: the scores of this lane's candidates (-inf beyond n).
+// Needs n > K.  cut_k / cut_k1: the K-th and (K+1)-th largest scores (the cut margin is their gap).
+__device__ __forceinline__ void warp_select_sorted64(float u0, float u1, int K, int lane, bool& keep0, bool& keep1,
+                                                     float& cut_k, float& cut_k1) {
+  float v0 = u0, v1 = u1;                      // element e = lane + 32 * k; sorted ascending by e
+#pragma unroll
+  for (int size = 2; size <= 64; size <<= 1) {
+#pragma unroll
+    for (int j = size >> 1; j > 0; j >>= 1) {
+      if (j == 32) {                           // partner = the lane's other element; the last merge is ascending
+        const float lo = fminf(v0, v1), hi = fmaxf(v0, v1);
+        v0 = lo; v1 = hi;
+      } else {
+        const float o0 = __shfl_xor_sync(0xffffffffu, v0, j), o1 = __shfl_xor_sync(0xffffffffu, v1, j);
+        const bool lower = (lane & j) == 0;
+        // ascending block when bit `size` of e is clear: a lane bit below 32, the element bit at 32, none at 64
+        const bool asc0 = (size < 32) ? ((lane & size) == 0) : true;
+        const bool asc1 = (size < 32) ? ((lane & size) == 0) : (size == 64);
+        v0 = (lower == asc0) ? fminf(v0, o0) : fmaxf(v0, o0);
+        v1 = (lower == asc1) ? fminf(v1, o1) : fmaxf(v1, o1);
+      }
+    }
+  }
+  // position p of the sorted order sits in lane p & 31, element p >> 5; K-th largest = position 64 - K
+  const int pk = 64 - K, pk1 = pk - 1;
+  const float a0 = __shfl_sync(0xffffffffu, v0, pk & 31), a1 = __shfl_sync(0xffffffffu, v1, pk & 31);
+  const float b0 = __shfl_sync(0xffffffffu, v0, pk1 & 31), b1 = __shfl_sync(0xffffffffu, v1, pk1 & 31);
+  cut_k = (pk >> 5) ? a1 : a0;
+  cut_k1 = (pk1 >> 5) ? b1 : b0;
+  const float T = cut_k;
+  const unsigned gt0 = __ballot_sync(0xffffffffu, u0 > T), gt1 = __ballot_sync(0xffffffffu, u1 > T);
+  const unsigned eq0 = __ballot_sync(0xffffffffu, u0 == T), eq1 = __ballot_sync(0xffffffffu, u1 == T);
+  const int room = K - __popc(gt0) - __popc(gt1);                       // equal ones still to keep (>= 1)
+  const unsigned lt = (1u << lane) - 1u;
+  keep0 = (u0 > T) || ((u0 == T) && __popc(eq0 & lt) < room);
+  keep1 = (u1 > T) || ((u1 == T) && __popc(eq0) + __popc(eq1 & lt) < room);
+}
+
 }  // namespace pisa

@@ -179,7 +179,15 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
     }
     // Select_K: rank by (score desc, position asc); keep rank < K.  Without pruning keep all.
     int rank[kMaxCand / 32];
-    if (prune) warp_select_ranks(u, nV, lane, rank);
+    const bool sorted = prune && nV <= 64;       // the common case: a sorting network instead of ranks
+    bool keep_s[2] = {false, false};
+    float cut_a = 0.f, cut_b = 0.f;
+    if (sorted) {
+      const float u0 = (lane < nV) ? u[lane] : -CUDART_INF_F, u1 = (lane + 32 < nV) ? u[lane + 32] : -CUDART_INF_F;
+      warp_select_sorted64(u0, u1, K, lane, keep_s[0], keep_s[1], cut_a, cut_b);
+    } else if (prune) {
+      warp_select_ranks(u, nV, lane, rank);
+    }
     int base = 0;
 #pragma unroll
     for (int ch = 0; ch < kMaxCand / 32; ++ch) {
@@ -187,7 +195,9 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
       if (s0 >= nV) break;
       const int s = s0 + lane;
       bool keep = s < nV;
-      if (prune) {
+      if (sorted) {
+        keep = keep && keep_s[ch & 1];
+      } else if (prune) {
         keep = keep && (rank[ch] < K);
         if (s < nV && rank[ch] == K - 1) s_cut[warp][0] = u[s];
         if (s < nV && rank[ch] == K) s_cut[warp][1] = u[s];
@@ -206,7 +216,7 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
     }
     __syncwarp();
     if (prune) {
-      const float a = s_cut[warp][0], bb = s_cut[warp][1];
+      const float a = sorted ? cut_a : s_cut[warp][0], bb = sorted ? cut_b : s_cut[warp][1];
       if (a < kForcedFloor) min_gap = fminf(min_gap, (a - bb) / fmaxf(fabsf(a), 1.f));
     }
     if (l == 2) {

@@ -1029,7 +1029,15 @@ __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int
   __syncwarp();
   const bool prune = nV > K;
   int rank[kMaxCand / 32];
-  if (prune) warp_select_ranks(u, nV, lane, rank);
+  const bool sorted = prune && nV <= 64;         // the common case: a sorting network instead of ranks
+  bool keep_s[2] = {false, false};
+  float cut_a = 0.f, cut_b = 0.f;
+  if (sorted) {
+    const float u0 = (lane < nV) ? u[lane] : -CUDART_INF_F, u1 = (lane + 32 < nV) ? u[lane + 32] : -CUDART_INF_F;
+    warp_select_sorted64(u0, u1, K, lane, keep_s[0], keep_s[1], cut_a, cut_b);
+  } else if (prune) {
+    warp_select_ranks(u, nV, lane, rank);
+  }
   int base = 0;
   unsigned kept_mask[kMaxCand / 32];
 #pragma unroll
@@ -1037,7 +1045,9 @@ __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int
     const int s0 = ch * 32;
     const int s = s0 + lane;
     bool keep = s < nV;
-    if (prune && s0 < nV) {
+    if (sorted) {
+      keep = keep && (ch < 2) && keep_s[ch & 1];
+    } else if (prune && s0 < nV) {
       keep = keep && (rank[ch] < K);
       if (s < nV && rank[ch] == K - 1) s_cut[warp][0] = u[s];
       if (s < nV && rank[ch] == K) s_cut[warp][1] = u[s];
@@ -1054,7 +1064,7 @@ __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int
   if (margin != nullptr && lane == 0) {
     float mg = margin[w];
     if (prune) {
-      const float a = s_cut[warp][0], bb = s_cut[warp][1];
+      const float a = sorted ? cut_a : s_cut[warp][0], bb = sorted ? cut_b : s_cut[warp][1];
       if (a < kForcedFloor) mg = fminf(mg, (a - bb) / fmaxf(fabsf(a), 1.f));
     }
     margin[w] = mg;
