@@ -239,13 +239,22 @@ decode_step_kernel(Geometry geo, DecArgs a) {
     __syncthreads();
     if (warp == 0) {
       int rank_s[kMaxCand / 32];
-      if (prune) warp_select_ranks(s_u, nV, lane, rank_s);
+      const bool sorted = prune && nV <= 64;
+      bool keep_s[2] = {false, false};
+      if (sorted) {
+        float ca, cb;
+        warp_select_sorted64((lane < nV) ? s_u[lane] : -CUDART_INF_F, (lane + 32 < nV) ? s_u[lane + 32] : -CUDART_INF_F,
+                             K, lane, keep_s[0], keep_s[1], ca, cb);
+      } else if (prune) {
+        warp_select_ranks(s_u, nV, lane, rank_s);
+      }
       int base = 0;
 #pragma unroll
       for (int ch = 0; ch < kMaxCand / 32; ++ch) {
         const int s = ch * 32 + lane;
         bool keep = s < nV;
-        if (prune && ch * 32 < nV) keep = keep && (rank_s[ch] < K);
+        if (sorted) keep = keep && (ch < 2) && keep_s[ch & 1];
+        else if (prune && ch * 32 < nV) keep = keep && (rank_s[ch] < K);
         const unsigned bal = __ballot_sync(0xffffffffu, keep);
         const int p = base + __popc(bal & ((1u << lane) - 1u));
         if (keep) {
@@ -348,13 +357,21 @@ decode_step_kernel(Geometry geo, DecArgs a) {
     }
     __syncwarp();
     int rank_s[kMaxCand / 32];
-    if (prune1) warp_select_ranks(s_u, nV1, lane, rank_s);
+    const bool sorted = prune1 && nV1 <= 64;
+    bool keep_s[2] = {false, false};
+    if (sorted) {
+      float ca, cb;
+      warp_select_sorted64(s_u[lane], s_u[lane + 32], K, lane, keep_s[0], keep_s[1], ca, cb);   // -inf beyond nV1
+    } else if (prune1) {
+      warp_select_ranks(s_u, nV1, lane, rank_s);
+    }
     int base = 0;
 #pragma unroll
     for (int ch = 0; ch < kMaxCand / 32; ++ch) {
       const int s = ch * 32 + lane;
       bool keep = s < nV1;
-      if (prune1 && ch * 32 < nV1) keep = keep && (rank_s[ch] < K);
+      if (sorted) keep = keep && (ch < 2) && keep_s[ch & 1];
+      else if (prune1 && ch * 32 < nV1) keep = keep && (rank_s[ch] < K);
       const unsigned bal = __ballot_sync(0xffffffffu, keep);
       const int p = base + __popc(bal & ((1u << lane) - 1u));
       if (keep) s_sel[p] = cand1[s];
