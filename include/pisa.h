@@ -75,7 +75,9 @@ const char* pisa_last_cuda_error(void);
  * Hierarchy of Sec. 3.2 "Fine-to-coarse block aggregation".
  * Host-only.  Writes L, M[0..L] (M[0] = N; caller provides >= 34 entries) and level_off[0..L]
  * (element offset of level l inside the pyramid buffer; level_off[0] is unused), and the
- * buffer size in bytes.  Any output pointer may be NULL.
+ * buffer size in bytes.  Any output pointer may be NULL.  The pyramid buffer itself must start on
+ * a 32-byte boundary wherever it is passed (PISA_ERR_INVALID_ARG otherwise: the routing kernels read
+ * the summaries with 32-byte loads); tensor pointers need 16 bytes.
  */
 int pisa_pyramid_layout(const pisa_params_t* p, int32_t* L, int32_t* M, int64_t* level_off, size_t* bytes);
 

@@ -25,6 +25,18 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
 
 __device__ __forceinline__ uint4 ldg128(const void* p) { return *reinterpret_cast<const uint4*>(p); }
 
+// 32 bytes per lane in one load (sm_100): four lanes then cover a whole 128-byte line of a row, half the
+// L1 wavefronts per byte of the 16-byte form.  `p` must be 32-byte aligned.
+struct U32x8 { uint32_t r[8]; };
+__device__ __forceinline__ U32x8 ldg256(const void* p) {
+  U32x8 v;
+  asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(v.r[0]), "=r"(v.r[1]), "=r"(v.r[2]), "=r"(v.r[3]), "=r"(v.r[4]), "=r"(v.r[5]), "=r"(v.r[6]),
+                 "=r"(v.r[7])
+               : "l"(p));
+  return v;
+}
+
 // running (max, sum exp) of a stream of logits
 __device__ __forceinline__ void lse_add(float& m, float& s, float z) {
   const float mn = fmaxf(m, z);

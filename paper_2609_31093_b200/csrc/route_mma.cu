@@ -4,10 +4,11 @@
 // At one level a token scores at most g*K candidates, each from g child summaries, against its own G
 // query vectors: a gathered [g*K*g rows] x [d] by [d] x [G] product, far too small and too irregular
 // for a CTA-wide UMMA tile but a natural fit for m16n8k16 fragments held in registers.  The child
-// summaries are the A operand, loaded straight from global/L2 into fragment registers with 16-byte
+// summaries are the A operand, loaded straight from global/L2 into fragment registers with 32-byte
 // loads (the k index of both operands is permuted identically so that a lane's fragment pieces are
-// contiguous in memory); the G query vectors, padded to 8 columns, are the B operand and stay in
-// registers for all levels.  A candidate's g children occupy rows (r, r+8) of consecutive tiles, so
+// contiguous in memory: lane (gid, tig) owns 32-byte chunk c8*4 + tig of its row for every group c8 of
+// 64 elements, so the four lanes of a row read one whole 128-byte line per load); the G query vectors,
+// padded to 8 columns, are the B operand and stay in registers for all levels.  A candidate's g children occupy rows (r, r+8) of consecutive tiles, so
 // their logits meet in one lane and the child LSE needs no shuffles; the head sum takes two.
 // The selection logic (eligibility, forced nodes, Select_K, expansion) is the SIMT kernel's.
 #include <math_constants.h>
@@ -30,7 +31,7 @@ template <int D, int NT, bool G2, int MODE>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ pyr,
                         int32_t* __restrict__ par_out, float* __restrict__ margin) {
-  constexpr int C4 = D / 32;              // groups of four 16-byte chunks per row (one chunk per tig)
+  constexpr int C8 = D / 64;              // groups of four 32-byte chunks per row (one chunk per tig)
   __shared__ int s_cand[kWarpsPerCta][2][kMaxCand];
   __shared__ __align__(16) float s_u[kWarpsPerCta][kMaxCand];
   __shared__ float s_cut[kWarpsPerCta][2];
@@ -48,19 +49,21 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
   float* u = s_u[warp];
 
   // B fragments: column n = gid is query head nt*8 + gid (zero beyond G); k permuted as the A loads
-  uint32_t bq[NT][C4][4];
+  uint32_t bq[NT][C8][8];
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
     const int head = nt * 8 + gid;
     const __nv_bfloat16* row = q + (long long)b * geo.qs[0] + (long long)t * geo.qs[1] +
                                (long long)(h * G + head) * geo.qs[2];
 #pragma unroll
-    for (int c4 = 0; c4 < C4; ++c4) {
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (head < G) v = ldg128(row + (c4 * 4 + tig) * 8);
-      bq[nt][c4][0] = v.x; bq[nt][c4][1] = v.y; bq[nt][c4][2] = v.z; bq[nt][c4][3] = v.w;
+    for (int c8 = 0; c8 < C8; ++c8) {
+      uint4 v0 = make_uint4(0u, 0u, 0u, 0u), v1 = v0;             // query rows are only 16-byte aligned
+      if (head < G) { v0 = ldg128(row + (c8 * 4 + tig) * 16); v1 = ldg128(row + (c8 * 4 + tig) * 16 + 8); }
+      bq[nt][c8][0] = v0.x; bq[nt][c8][1] = v0.y; bq[nt][c8][2] = v0.z; bq[nt][c8][3] = v0.w;
+      bq[nt][c8][4] = v1.x; bq[nt][c8][5] = v1.y; bq[nt][c8][6] = v1.z; bq[nt][c8][7] = v1.w;
     }
   }
+  const U32x8 zero8 = {{0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u}};
 
   int cur = 0;
   int n = 1;
@@ -94,20 +97,21 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
           // fan-in 2: both children of a candidate meet in one lane; LSE(a, b) = max + log(1 + e^-|a-b|)
           const int ch_lo = node * 2, ch_hi = ch_lo + 1;
           const bool ok_hi = has && ch_hi < Mb;
-          uint4 lo[C4], hi[C4];
+          U32x8 lo[C8], hi[C8];
 #pragma unroll
-          for (int c4 = 0; c4 < C4; ++c4) {
-            lo[c4] = has ? ldg128(below + (long long)ch_lo * D + (c4 * 4 + tig) * 8) : make_uint4(0u, 0u, 0u, 0u);
-            hi[c4] = ok_hi ? ldg128(below + (long long)ch_hi * D + (c4 * 4 + tig) * 8) : make_uint4(0u, 0u, 0u, 0u);
+          for (int c8 = 0; c8 < C8; ++c8) {
+            lo[c8] = has ? ldg256(below + (long long)ch_lo * D + (c8 * 4 + tig) * 16) : zero8;
+            hi[c8] = ok_hi ? ldg256(below + (long long)ch_hi * D + (c8 * 4 + tig) * 16) : zero8;
           }
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) {
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c4 = 0; c4 < C4; ++c4) {
-              mma_bf16_16816(acc, lo[c4].x, hi[c4].x, lo[c4].y, hi[c4].y, bq[nt][c4][0], bq[nt][c4][1]);
-              mma_bf16_16816(acc, lo[c4].z, hi[c4].z, lo[c4].w, hi[c4].w, bq[nt][c4][2], bq[nt][c4][3]);
-            }
+            for (int c8 = 0; c8 < C8; ++c8)
+#pragma unroll
+              for (int i = 0; i < 8; i += 2)
+                mma_bf16_16816(acc, lo[c8].r[i], hi[c8].r[i], lo[c8].r[i + 1], hi[c8].r[i + 1], bq[nt][c8][i],
+                               bq[nt][c8][i + 1]);
 #pragma unroll
             for (int jh = 0; jh < 2; ++jh) {
               const float za = acc[jh] * geo.scale, zb = acc[2 + jh] * geo.scale;
@@ -128,20 +132,21 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
           for (int r0 = 0; r0 < g; r0 += 2) {
             const int ch_lo = node * g + r0, ch_hi = ch_lo + 1;
             const bool ok_lo = has && ch_lo < Mb, ok_hi = has && (r0 + 1 < g) && ch_hi < Mb;
-            uint4 lo[C4], hi[C4];
+            U32x8 lo[C8], hi[C8];
 #pragma unroll
-            for (int c4 = 0; c4 < C4; ++c4) {
-              lo[c4] = ok_lo ? ldg128(below + (long long)ch_lo * D + (c4 * 4 + tig) * 8) : make_uint4(0u, 0u, 0u, 0u);
-              hi[c4] = ok_hi ? ldg128(below + (long long)ch_hi * D + (c4 * 4 + tig) * 8) : make_uint4(0u, 0u, 0u, 0u);
+            for (int c8 = 0; c8 < C8; ++c8) {
+              lo[c8] = ok_lo ? ldg256(below + (long long)ch_lo * D + (c8 * 4 + tig) * 16) : zero8;
+              hi[c8] = ok_hi ? ldg256(below + (long long)ch_hi * D + (c8 * 4 + tig) * 16) : zero8;
             }
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
               float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-              for (int c4 = 0; c4 < C4; ++c4) {
-                mma_bf16_16816(acc, lo[c4].x, hi[c4].x, lo[c4].y, hi[c4].y, bq[nt][c4][0], bq[nt][c4][1]);
-                mma_bf16_16816(acc, lo[c4].z, hi[c4].z, lo[c4].w, hi[c4].w, bq[nt][c4][2], bq[nt][c4][3]);
-              }
+              for (int c8 = 0; c8 < C8; ++c8)
+#pragma unroll
+                for (int i = 0; i < 8; i += 2)
+                  mma_bf16_16816(acc, lo[c8].r[i], hi[c8].r[i], lo[c8].r[i + 1], hi[c8].r[i + 1], bq[nt][c8][i],
+                                 bq[nt][c8][i + 1]);
               // acc[0..1]: child lo, heads nt*8 + 2*tig + {0,1};  acc[2..3]: child hi, same heads
 #pragma unroll
               for (int jh = 0; jh < 2; ++jh) {
@@ -262,6 +267,9 @@ bool route_stage1_mma_supported(const Geometry& g, int dtype) {
 
 int launch_route_stage1_mma(const Geometry& g, const void* q, const void* pyramid, int32_t* par, float* margin,
                             cudaStream_t s) {
+  // the 32-byte loads of the summaries: rows are d*2 >= 128 bytes and the levels start on 256-byte
+  // boundaries, so the buffer's own alignment decides
+  if ((reinterpret_cast<uintptr_t>(pyramid) & 31u) != 0) return PISA_ERR_INVALID_ARG;
   const bool wide = g.G > 8;
   if (g.d == 128) return wide ? launch_dn<128, 2>(g, q, pyramid, par, margin, s) : launch_dn<128, 1>(g, q, pyramid, par, margin, s);
   if (g.d == 64) return wide ? launch_dn<64, 2>(g, q, pyramid, par, margin, s) : launch_dn<64, 1>(g, q, pyramid, par, margin, s);
