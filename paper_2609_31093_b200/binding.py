@@ -102,6 +102,15 @@ class Params:
         self.dtype = dtype
         self.B, self.N, self.Hq, self.Hkv, self.d, self.C, self.g, self.K = B, N, Hq, Hkv, d, C, g, K
 
+    def set_strides(self, q=None, k=None, v=None, o=None):
+        """Element strides (batch, token, head) of q, k, v and out; None keeps a tensor dense [B, N, H, d].
+        The last dimension is always contiguous."""
+        for name, val in (("q_stride", q), ("k_stride", k), ("v_stride", v), ("o_stride", o)):
+            arr = getattr(self.c, name)
+            for i in range(3):
+                arr[i] = 0 if val is None else int(val[i])
+        return self
+
     @classmethod
     def from_workload(cls, w, B=None, **kw):
         return cls(w.B if B is None else B, w.N, w.Hq, w.Hkv, w.d, w.C, w.g, w.K, dtype=w.dtype, **kw)
