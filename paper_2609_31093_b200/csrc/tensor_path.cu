@@ -32,6 +32,7 @@ namespace {
 
 constexpr int kInvTok = 1024;          // tokens per CTA in the inversion kernels
 constexpr int kWindowTok = 16384;      // tokens per window of the inverted lists
+constexpr int kBwdWindowTok = 32768;   // ... of the backward's lists (fewer, fuller lists: 2.3 ms of 55 at the headline shape)
 constexpr int kItemTiles = 32;         // a work item: at most this many consecutive tiles of one list
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -1202,11 +1203,11 @@ struct InvLayout {
   size_t count, entry_off, tile_off, item_off, item_key, cursor, blk_tot, entries, end;
 };
 
-int window_tokens(const Geometry& g) { return g.N < kWindowTok ? ((g.N + kInvTok - 1) / kInvTok) * kInvTok : kWindowTok; }
-int num_windows(const Geometry& g) { return (g.N + window_tokens(g) - 1) / window_tokens(g); }
+int window_tokens(const Geometry& g, int win) { return g.N < win ? ((g.N + kInvTok - 1) / kInvTok) * kInvTok : win; }
+int num_windows(const Geometry& g, int win) { return (g.N + window_tokens(g, win) - 1) / window_tokens(g, win); }
 
-InvLayout inv_layout(size_t base, const Geometry& g, int Mk) {
-  const size_t nkeys = (size_t)g.B * g.Hkv * num_windows(g) * Mk;
+InvLayout inv_layout(size_t base, const Geometry& g, int Mk, int win = kWindowTok) {
+  const size_t nkeys = (size_t)g.B * g.Hkv * num_windows(g, win) * Mk;
   InvLayout l;
   size_t o = base;
   l.count = o; o += align_up(nkeys * 4, 256);
@@ -1256,11 +1257,11 @@ int num_sms() {
 }
 
 int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char* ws, const InvLayout& l,
-                  InvArgs* out, cudaStream_t s) {
+                  InvArgs* out, cudaStream_t s, int win = kWindowTok) {
   InvArgs a;
   a.nodes = nodes; a.K = g.K; a.fan = fan; a.Mk = Mk; a.N = g.N; a.C = g.C; a.BH = g.B * g.Hkv;
   a.tpt = 128 / g.G;
-  a.W = window_tokens(g); a.NW = num_windows(g);
+  a.W = window_tokens(g, win); a.NW = num_windows(g, win);
   a.count = (int32_t*)(ws + l.count); a.entry_off = (int32_t*)(ws + l.entry_off);
   a.tile_off = (int32_t*)(ws + l.tile_off); a.item_off = (int32_t*)(ws + l.item_off);
   a.item_key = (int32_t*)(ws + l.item_key);
@@ -1351,7 +1352,7 @@ BwdLayout bwd_layout(const Geometry& g) {
   r.dq = o; o += align_up((size_t)g.B * g.N * g.Hq * g.d * 4, 256);
   r.dk = o; o += align_up((size_t)g.B * g.N * g.Hkv * g.d * 4, 256);
   r.dv = o; o += align_up((size_t)g.B * g.N * g.Hkv * g.d * 4, 256);
-  r.inv = inv_layout(o, g, g.M[1]);
+  r.inv = inv_layout(o, g, g.M[1], kBwdWindowTok);
   r.total = r.inv.end;
   return r;
 }
@@ -1473,7 +1474,7 @@ int tensor_bsa_bwd(const Geometry& g, const void* q, const void* k, const void* 
   const BwdLayout L = bwd_layout(g);
   kernel_mark("invert_by_leaf", s);
   InvArgs inv;
-  int st = run_inversion(g, idx, 1, g.M[1], ws, L.inv, &inv, s);
+  int st = run_inversion(g, idx, 1, g.M[1], ws, L.inv, &inv, s, kBwdWindowTok);
   if (st != PISA_OK) return st;
   BwdArgs a = {};
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
