@@ -545,20 +545,42 @@ int launch_dnb(const Geometry& g, const DecArgs& a, cudaStream_t s) {
   return (g.score_mode == PISA_SCORE_LSE) ? launch_dnbm<D, NT, MINB, CLU, false>(g, a, s)
                                           : launch_dnbm<D, NT, MINB, CLU, true>(g, a, s);
 }
-// Eight CTAs per (batch, KV head) while all clusters fit the GPU at once (one, then two CTAs per SM);
-// beyond that narrower clusters, so that a large batch still runs as a single wave.
+// How many clusters of this instantiation the GPU holds at once (clusters are placed inside one GPC, so
+// this is less than SMs * MINB / CLU); asked of the driver once per instantiation.
+template <int D, int NT, int MINB, int CLU>
+int max_resident_clusters(const Geometry& g) {
+  static int cached = -1;
+  if (cached >= 0) return cached;
+  const size_t smem = (size_t)kDecWarps * (g.G * D + 2 * g.G) * sizeof(float);
+  auto kern = decode_step_kernel<D, NT, MINB, CLU, false>;
+  cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(CLU, 1024);
+  cfg.blockDim = dim3(kDecThreads);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = CLU; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+  cached = n;
+  return n;
+}
+
+// The widest cluster whose clusters are all resident at once, at one CTA per SM (all registers) if
+// possible, else at two; beyond that the narrowest, in waves.  Measured at the headline shape, 128K
+// context: batch 3 / 4 / 6 / 8 take 82 / 86 / 127 / 130 us this way against 98 / 103 / 143 / 152 us with
+// clusters of eight at two CTAs per SM whenever those fit.
 template <int D, int NT>
 int launch_dn(const Geometry& g, const DecArgs& a, cudaStream_t s) {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  }
   const long long units = (long long)g.B * g.Hkv;
-  if (units * 8 <= sms) return launch_dnb<D, NT, 1, 8>(g, a, s);
-  if (units * 8 <= 2LL * sms) return launch_dnb<D, NT, 2, 8>(g, a, s);
-  if (units * 4 <= 2LL * sms) return launch_dnb<D, NT, 2, 4>(g, a, s);
+  if (units <= max_resident_clusters<D, NT, 1, 8>(g)) return launch_dnb<D, NT, 1, 8>(g, a, s);
+  if (units <= max_resident_clusters<D, NT, 1, 4>(g)) return launch_dnb<D, NT, 1, 4>(g, a, s);
+  if (units <= max_resident_clusters<D, NT, 1, 2>(g)) return launch_dnb<D, NT, 1, 2>(g, a, s);
+  if (units <= max_resident_clusters<D, NT, 2, 8>(g)) return launch_dnb<D, NT, 2, 8>(g, a, s);
+  if (units <= max_resident_clusters<D, NT, 2, 4>(g)) return launch_dnb<D, NT, 2, 4>(g, a, s);
   return launch_dnb<D, NT, 2, 2>(g, a, s);
 }
 
