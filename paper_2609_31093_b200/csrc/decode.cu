@@ -569,8 +569,8 @@ int max_resident_clusters(const Geometry& g) {
   return n;
 }
 
-// The widest cluster whose clusters are all resident at once, at one CTA per SM (all registers) if
-// possible, else at two; beyond that the narrowest, in waves.  Measured at the headline shape, 128K
+// The widest cluster whose clusters are all resident at once at one CTA per SM (all registers); beyond
+// that clusters of two at two CTAs per SM, in waves once even those do not fit.  Measured at the headline shape, 128K
 // context: batch 3 / 4 / 6 / 8 take 82 / 86 / 127 / 130 us this way against 98 / 103 / 143 / 152 us with
 // clusters of eight at two CTAs per SM whenever those fit.
 template <int D, int NT>
@@ -579,8 +579,7 @@ int launch_dn(const Geometry& g, const DecArgs& a, cudaStream_t s) {
   if (units <= max_resident_clusters<D, NT, 1, 8>(g)) return launch_dnb<D, NT, 1, 8>(g, a, s);
   if (units <= max_resident_clusters<D, NT, 1, 4>(g)) return launch_dnb<D, NT, 1, 4>(g, a, s);
   if (units <= max_resident_clusters<D, NT, 1, 2>(g)) return launch_dnb<D, NT, 1, 2>(g, a, s);
-  if (units <= max_resident_clusters<D, NT, 2, 8>(g)) return launch_dnb<D, NT, 2, 8>(g, a, s);
-  if (units <= max_resident_clusters<D, NT, 2, 4>(g)) return launch_dnb<D, NT, 2, 4>(g, a, s);
+  // two CTAs per SM: only the narrowest width holds more units than the options above
   return launch_dnb<D, NT, 2, 2>(g, a, s);
 }
 

@@ -151,8 +151,8 @@ def test_decode_long_context():
 
 @pytest.mark.parametrize("B,Hkv", [(5, 4), (10, 4), (20, 4)])
 def test_decode_large_batches_use_narrower_clusters(B, Hkv):
-    """20, 40 and 80 (batch, KV head) units: eight CTAs per unit at two per SM, then four, then two, where a
-    warp runs its online softmax across several half blocks (2 K = 40 of them per unit)."""
+    """20, 40 and 80 (batch, KV head) units: clusters of four and of two CTAs at one CTA per SM, then of two at
+    two per SM; a warp then runs its online softmax across several half blocks (2 K = 40 of them per unit)."""
     w = S.Workload(f"dec_batch{B}", B, 2000, 2 * Hkv, Hkv, 64, 32, 2, 20, "bf16", 406 + B, "iid")
     t = S.make_inputs(w)
     n0 = w.N - 12
