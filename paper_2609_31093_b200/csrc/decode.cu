@@ -28,7 +28,7 @@ using namespace frag;
 
 namespace {
 
-constexpr int kCluMax = 8;              // CTAs per cluster, at most (scratch is laid out for this many)
+constexpr int kCluMax = 16;             // CTAs per cluster, at most (scratch is laid out for this many)
 constexpr int kDecWarps = 8;
 constexpr int kDecThreads = kDecWarps * 32;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -398,11 +398,13 @@ decode_step_kernel(Geometry geo, DecArgs a) {
     for (int j = 0; j < DV; ++j) o_acc[hh][j] = 0.f;
   float m_run = -CUDART_INF_F, l_run = 0.f;                // lanes 0..G-1: running max (base 2) / sum of head `lane`
   const float sl2 = geo.scale * kLog2e;
-  for (int sh = gw; sh < 2 * nsel; sh += CLU * kDecWarps) {
-    const int slot = sh >> 1, half = sh & 1;
+  // clusters of sixteen (opt-in size) split a block in four, so that all 128 warps have a part
+  constexpr int SUB = (CLU == 16) ? 4 : 2;
+  for (int sh = gw; sh < SUB * nsel; sh += CLU * kDecWarps) {
+    const int slot = sh / SUB, half = sh % SUB;
     const int leaf = s_sel[slot];
-    const int key0 = leaf * C + half * (C / 2);
-    for (int kt = 0; kt < C / 2; kt += 16) {
+    const int key0 = leaf * C + half * (C / SUB);
+    for (int kt = 0; kt < C / SUB; kt += 16) {
       const int t_lo = key0 + kt + gid, t_hi = t_lo + 8;
       if (key0 + kt > pos) break;                          // the rest of the block lies in the future
       RowPair<D> kr;
@@ -536,6 +538,8 @@ int launch_dnbm(const Geometry& g, const DecArgs& a, cudaStream_t s) {
   const size_t smem = (size_t)kDecWarps * (g.G * D + 2 * g.G) * sizeof(float);
   cudaError_t e = cudaFuncSetAttribute(decode_step_kernel<D, NT, MINB, CLU, MOM>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e == cudaSuccess && CLU > 8)
+    e = cudaFuncSetAttribute(decode_step_kernel<D, NT, MINB, CLU, MOM>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   if (e != cudaSuccess) { record_cuda_error("decode_step attr", e); return PISA_ERR_CUDA; }
   decode_step_kernel<D, NT, MINB, CLU, MOM><<<dim3(CLU, (unsigned)(g.B * g.Hkv)), kDecThreads, smem, s>>>(g, a);
   return check_launch("decode_step");
@@ -554,6 +558,11 @@ int max_resident_clusters(const Geometry& g) {
   const size_t smem = (size_t)kDecWarps * (g.G * D + 2 * g.G) * sizeof(float);
   auto kern = decode_step_kernel<D, NT, MINB, CLU, false>;
   cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (CLU > 8 && cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+    cudaGetLastError();
+    cached = 0;
+    return 0;
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(CLU, 1024);
   cfg.blockDim = dim3(kDecThreads);
@@ -576,6 +585,10 @@ int max_resident_clusters(const Geometry& g) {
 template <int D, int NT>
 int launch_dn(const Geometry& g, const DecArgs& a, cudaStream_t s) {
   const long long units = (long long)g.B * g.Hkv;
+  // sixteen CTAs (a quarter block of at least one 16-key tile per warp) for very few units: measured at
+  // 128K context, 4 units 48.7 -> 45.4 us and 2 units 49.3 -> 47.3 us, but 8 units 55.6 -> 57.4 us
+  if (g.C >= 64 && units <= 4 && units <= max_resident_clusters<D, NT, 1, 16>(g))
+    return launch_dnb<D, NT, 1, 16>(g, a, s);
   if (units <= max_resident_clusters<D, NT, 1, 8>(g)) return launch_dnb<D, NT, 1, 8>(g, a, s);
   if (units <= max_resident_clusters<D, NT, 1, 4>(g)) return launch_dnb<D, NT, 1, 4>(g, a, s);
   if (units <= max_resident_clusters<D, NT, 1, 2>(g)) return launch_dnb<D, NT, 1, 2>(g, a, s);
