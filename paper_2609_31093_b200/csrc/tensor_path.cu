@@ -45,6 +45,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 struct InvArgs {
   const int32_t* nodes;   // [BH, N, K] node ids (ascending, -1 padded)
   int K, fan, Mk, N, C, BH, tpt;
+  int lgK, lgC;           // log2 of K and C when they are powers of two (shifts instead of divisions), else -1
   int W, NW;              // tokens per window (a multiple of kInvTok), windows per sequence
   int32_t* count;         // [BH*Mk]
   int32_t* entry_off;     // [BH*Mk + 1]
@@ -56,8 +57,11 @@ struct InvArgs {
   int32_t* entries;       // [<= BH*N*K]  token | slot << 24
 };
 
+__device__ __forceinline__ int inv_token(const InvArgs& a, int e) { return a.lgK >= 0 ? (e >> a.lgK) : e / a.K; }
+__device__ __forceinline__ int inv_slot(const InvArgs& a, int e) { return a.lgK >= 0 ? (e & (a.K - 1)) : e % a.K; }
 __device__ __forceinline__ bool inv_valid(const InvArgs& a, int node, int t) {
-  return node >= 0 && node < a.Mk && (long long)node * a.fan <= (long long)(t / a.C);
+  const int leaf = a.lgC >= 0 ? (t >> a.lgC) : t / a.C;
+  return node >= 0 && node < a.Mk && (long long)node * a.fan <= (long long)leaf;
 }
 
 __global__ void __launch_bounds__(256) inv_count_kernel(InvArgs a, int use_smem) {
@@ -71,7 +75,7 @@ __global__ void __launch_bounds__(256) inv_count_kernel(InvArgs a, int use_smem)
   }
   const int n = (t1 - t0) * a.K;
   for (int e = threadIdx.x; e < n; e += blockDim.x) {
-    const int t = t0 + e / a.K;
+    const int t = t0 + inv_token(a, e);
     const int node = a.nodes[((long long)bh * a.N + t0) * a.K + e];
     if (inv_valid(a, node, t)) {
       if (use_smem) atomicAdd(&s_hist[node], 1);
@@ -185,7 +189,7 @@ __global__ void __launch_bounds__(256) inv_fill_kernel(InvArgs a, int use_smem) 
   const int32_t* nodes = a.nodes + ((long long)bh * a.N + t0) * a.K;
   if (!use_smem) {
     for (int e = threadIdx.x; e < n; e += blockDim.x) {
-      const int t = t0 + e / a.K, slot = e % a.K, node = nodes[e];
+      const int t = t0 + inv_token(a, e), slot = inv_slot(a, e), node = nodes[e];
       if (inv_valid(a, node, t)) {
         const int pos = atomicAdd(&a.cursor[kbase + node], 1);
         a.entries[pos] = t | (slot << 24);
@@ -197,7 +201,7 @@ __global__ void __launch_bounds__(256) inv_fill_kernel(InvArgs a, int use_smem) 
   __syncthreads();
   for (int e = threadIdx.x; e < n; e += blockDim.x) {
     const int node = nodes[e];
-    if (inv_valid(a, node, t0 + e / a.K)) atomicAdd(&s_hist[node], 1);
+    if (inv_valid(a, node, t0 + inv_token(a, e))) atomicAdd(&s_hist[node], 1);
   }
   __syncthreads();
   for (int j = threadIdx.x; j < a.Mk; j += blockDim.x) {
@@ -207,7 +211,7 @@ __global__ void __launch_bounds__(256) inv_fill_kernel(InvArgs a, int use_smem) 
   }
   __syncthreads();
   for (int e = threadIdx.x; e < n; e += blockDim.x) {
-    const int t = t0 + e / a.K, slot = e % a.K, node = nodes[e];
+    const int t = t0 + inv_token(a, e), slot = inv_slot(a, e), node = nodes[e];
     if (inv_valid(a, node, t)) {
       const int r = atomicAdd(&s_hist[node], 1);
       a.entries[s_base[node] + r] = t | (slot << 24);
@@ -1261,6 +1265,8 @@ int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char
   InvArgs a;
   a.nodes = nodes; a.K = g.K; a.fan = fan; a.Mk = Mk; a.N = g.N; a.C = g.C; a.BH = g.B * g.Hkv;
   a.tpt = 128 / g.G;
+  a.lgK = (g.K & (g.K - 1)) == 0 ? 31 - __builtin_clz((unsigned)g.K) : -1;
+  a.lgC = (g.C & (g.C - 1)) == 0 ? 31 - __builtin_clz((unsigned)g.C) : -1;
   a.W = window_tokens(g, win); a.NW = num_windows(g, win);
   a.count = (int32_t*)(ws + l.count); a.entry_off = (int32_t*)(ws + l.entry_off);
   a.tile_off = (int32_t*)(ws + l.tile_off); a.item_off = (int32_t*)(ws + l.item_off);
