@@ -54,6 +54,18 @@ enum { PISA_OP_ROUTE = 0, PISA_OP_BSA = 1, PISA_OP_FORWARD = 2, PISA_OP_FLAT = 3
        PISA_OP_DECODE = 5, PISA_OP_BSA_BWD = 6 };
 /* implementation selector (params.impl): AUTO picks the tensor-core path where it applies */
 enum { PISA_IMPL_AUTO = 0, PISA_IMPL_SIMT = 1, PISA_IMPL_TENSOR = 2 };
+/*
+ * params.debug bits.  PISA_DEBUG_BOUNDS: every index a kernel is about to gather or scatter with (token
+ * positions, node / leaf ids read from idx, from the inverted lists or from intermediate routing
+ * results, list slots) is range-checked on the device first; a value out of range is not used, the
+ * access is skipped and PISA_ERR_BOUNDS lands in the workspace's status word (pisa_read_status).
+ * Nothing traps.  In this mode an idx entry other than -1 that names a leaf which does not exist or
+ * starts after the row's own leaf counts as out of range (without it such entries are silently
+ * ignored).  The environment variable PISA_DEBUG=1 sets the bit for every call of the process.
+ * Costs a few percent; meant for tests and for chasing a suspected stray index (no memory checker
+ * can be attached to these kernels everywhere).
+ */
+enum { PISA_DEBUG_BOUNDS = 1 };
 
 typedef struct {
   int32_t B, N, Hq, Hkv, d, C, g, K; /* prefill self-attention: N queries = N keys            */
@@ -62,7 +74,7 @@ typedef struct {
   int32_t score_mode;                /* PISA_SCORE_*                                            */
   int32_t impl;                      /* PISA_IMPL_*                                             */
   float   scale;                     /* logit scale, > 0; 0 => 1/sqrt(d)  (Eq. "block scores")  */
-  int32_t reserved;
+  int32_t debug;                     /* PISA_DEBUG_* bits; 0 = off                              */
   int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3]; /* elements, (b, n, h); all 0 => dense */
 } pisa_params_t;
 
@@ -76,8 +88,9 @@ const char* pisa_last_cuda_error(void);
  * Host-only.  Writes L, M[0..L] (M[0] = N; caller provides >= 34 entries) and level_off[0..L]
  * (element offset of level l inside the pyramid buffer; level_off[0] is unused), and the
  * buffer size in bytes.  Any output pointer may be NULL.  The pyramid buffer itself must start on
- * a 32-byte boundary wherever it is passed (PISA_ERR_INVALID_ARG otherwise: the routing kernels read
- * the summaries with 32-byte loads); tensor pointers need 16 bytes.
+ * a 32-byte boundary wherever it is passed (every entry point that takes a pyramid checks it and
+ * returns PISA_ERR_INVALID_ARG otherwise: the routing kernels read the summaries with 32-byte
+ * loads); tensor pointers need 16 bytes.
  */
 int pisa_pyramid_layout(const pisa_params_t* p, int32_t* L, int32_t* M, int64_t* level_off, size_t* bytes);
 
@@ -100,22 +113,30 @@ int pisa_build_pyramid(const pisa_params_t* p, const void* k, void* pyramid, voi
  * children (g child summaries above the leaves, the C raw keys at the leaves), ties to the smaller
  * index; expand the kept nodes' children; the kept leaves are the result.
  *   q, k, pyramid : device inputs            idx : device int32 [B,Hkv,N,K] output
+ *   sel_lse       : device float [B,Hq,N,K] or NULL — for every query head and kept slot s the
+ *                   natural-log softmax denominator of the visible keys (j <= t) of leaf idx[b,h,t,s]
+ *                   alone (-inf for a -1 slot).  The leaf scores of the LSE mode are exactly these
+ *                   numbers, so the tensor-core routing has them for free; handing them to
+ *                   pisa_bsa_fwd saves its own scoring pass over the selected blocks
  *   margin        : device float [B,Hkv,N] or NULL — smallest relative gap between the last kept
  *                   and the first dropped score over the scored levels (+inf if nothing was cut);
  *                   gap = (u_kept - u_dropped) / max(|u_kept|, 1)
  *   ws / ws_bytes : device workspace sized for PISA_OP_ROUTE
  */
 int pisa_route(const pisa_params_t* p, const void* q, const void* k, const void* pyramid,
-               int32_t* idx, float* margin, void* ws, size_t ws_bytes, void* stream);
+               int32_t* idx, float* sel_lse, float* margin, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Eq. "selected sparse attention" with the causal mask inside selected blocks (App. B): for every
  * query head, softmax over the tokens j <= t of the leaf blocks idx[b, h, t, :] (entries < 0 are
  * skipped) with logits q.k*scale, fp32 accumulation.  out: device [B,N,Hq,d] in the input dtype;
  * lse: device float [B,Hq,N].  Workspace sized for PISA_OP_BSA.
+ *   sel_lse : device float [B,Hq,N,K] or NULL — per-block denominators of exactly these idx as
+ *             pisa_route wrote them; with them the tensor-core path skips its own pass over the
+ *             selected blocks that would compute them (the exact-fp32 path ignores the argument)
  */
 int pisa_bsa_fwd(const pisa_params_t* p, const void* q, const void* k, const void* v, const int32_t* idx,
-                 void* out, float* lse, void* ws, size_t ws_bytes, void* stream);
+                 const float* sel_lse, void* out, float* lse, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * pisa_route for callers that cannot provide a workspace because they are not allowed to allocate
@@ -193,8 +214,8 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
                       void* ws, size_t ws_bytes, void* stream);
 
 /*
- * Backward of the block-sparse attention with the selected indices held fixed (App. B: gradients
- * flow through attention on the selected entries, not through the selection).
+ * Backward of the block-sparse attention (App. B).  idx is treated as a constant: only q, k and v
+ * receive gradients, each through the softmax attention over its row's selected, visible keys.
  *
  *   q, k, v, idx   : as for pisa_bsa_fwd
  *   out, lse       : what pisa_bsa_fwd / pisa_forward produced for these idx (out with o_stride)
@@ -308,6 +329,17 @@ int pisa_set_forward_chunks(int max_chunks);
 
 /* Number of kernels this process has launched through the library so far (host counter). */
 unsigned long long pisa_launch_count(void);
+
+/*
+ * Self-test of the bounded device-side waits (no counterpart in the paper).  Every wait inside the
+ * kernels (on an mbarrier another warp or the tensor pipe is to complete) gives up after a time
+ * limit, records PISA_ERR_TIMEOUT in the workspace's status word, releases what it holds and lets
+ * the kernel return, so that a scheduling bug can never hang the GPU.  This entry point launches one
+ * CTA that waits, with the limit `limit_ns` (clamped to [1 us, 1 s]), on a barrier nobody arrives
+ * at: after the stream has been synchronised pisa_read_status(ws) reports PISA_ERR_TIMEOUT and the
+ * device remains usable.  ws: at least 256 bytes of device memory.
+ */
+int pisa_debug_wait_timeout(void* ws, unsigned long long limit_ns, void* stream);
 
 #ifdef __cplusplus
 }

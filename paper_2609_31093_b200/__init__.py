@@ -24,6 +24,8 @@ from .binding import (  # noqa: F401
     pisa_decode_step,
     pisa_pyramid_regrow,
     read_status,
+    debug_wait_timeout,
+    DEBUG_BOUNDS,
     set_stage_timing,
     get_stage_ms,
     launch_count,

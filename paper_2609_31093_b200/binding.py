@@ -15,6 +15,7 @@ BF16, FP32 = 0, 1
 SCORE_LSE, SCORE_MEAN, SCORE_MEAN_VAR = 0, 1, 2
 OP_ROUTE, OP_BSA, OP_FORWARD, OP_FLAT, OP_FORWARD_HOST, OP_DECODE, OP_BSA_BWD = 0, 1, 2, 3, 4, 5, 6
 IMPL_AUTO, IMPL_SIMT, IMPL_TENSOR = 0, 1, 2
+DEBUG_BOUNDS = 1
 _SCORE = {"lse": SCORE_LSE, "mean": SCORE_MEAN, "mean_var": SCORE_MEAN_VAR}
 
 
@@ -27,7 +28,7 @@ class _CParams(C.Structure):
         ("B", C.c_int32), ("N", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32),
         ("d", C.c_int32), ("C", C.c_int32), ("g", C.c_int32), ("K", C.c_int32),
         ("causal", C.c_int32), ("dtype", C.c_int32), ("score_mode", C.c_int32), ("impl", C.c_int32),
-        ("scale", C.c_float), ("reserved", C.c_int32),
+        ("scale", C.c_float), ("debug", C.c_int32),
         ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 3),
         ("v_stride", C.c_int64 * 3), ("o_stride", C.c_int64 * 3),
     ]
@@ -50,8 +51,8 @@ def lib():
     L.pisa_pyramid_layout.argtypes = [pp, i32p, i32p, C.POINTER(C.c_int64), szp]
     L.pisa_workspace_bytes.argtypes = [pp, C.c_int, szp]
     L.pisa_build_pyramid.argtypes = [pp, vp, vp, vp]
-    L.pisa_route.argtypes = [pp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
-    L.pisa_bsa_fwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+    L.pisa_route.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+    L.pisa_bsa_fwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
     L.pisa_forward.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
     L.pisa_forward_host.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
     L.pisa_flat_select.argtypes = [pp, vp, vp, vp, vp, C.c_size_t, vp]
@@ -70,6 +71,8 @@ def lib():
     L.pisa_launch_count.restype = C.c_ulonglong
     L.pisa_get_kernel_ms.argtypes = [C.c_int, C.c_char_p, C.c_size_t, f32p]
     L.pisa_get_kernel_ms.restype = C.c_int
+    L.pisa_debug_wait_timeout.argtypes = [vp, C.c_ulonglong, vp]
+    L.pisa_debug_wait_timeout.restype = C.c_int
     for name in ("pisa_pyramid_layout", "pisa_workspace_bytes", "pisa_build_pyramid", "pisa_route",
                  "pisa_bsa_fwd", "pisa_forward", "pisa_forward_host", "pisa_flat_select", "pisa_read_status",
                  "pisa_decode_step", "pisa_pyramid_regrow", "pisa_bsa_bwd", "pisa_forward_packed", "pisa_bsa_bwd_packed",
@@ -90,7 +93,7 @@ def _check(st: int, what: str):
 class Params:
     """Problem description in the paper's notation; mirrors pisa_params_t."""
 
-    def __init__(self, B, N, Hq, Hkv, d, C, g, K, dtype="bf16", score_mode="lse", scale=0.0, impl=IMPL_AUTO):
+    def __init__(self, B, N, Hq, Hkv, d, C, g, K, dtype="bf16", score_mode="lse", scale=0.0, impl=IMPL_AUTO, debug=0):
         self.c = _CParams()
         self.c.B, self.c.N, self.c.Hq, self.c.Hkv = B, N, Hq, Hkv
         self.c.d, self.c.C, self.c.g, self.c.K = d, C, g, K
@@ -99,6 +102,7 @@ class Params:
         self.c.score_mode = _SCORE[score_mode] if isinstance(score_mode, str) else int(score_mode)
         self.c.impl = impl
         self.c.scale = float(scale)
+        self.c.debug = int(debug)
         self.dtype = dtype
         self.B, self.N, self.Hq, self.Hkv, self.d, self.C, self.g, self.K = B, N, Hq, Hkv, d, C, g, K
 
@@ -161,9 +165,10 @@ def pisa_build_pyramid(p: Params, k: torch.Tensor, pyramid: torch.Tensor):
     _check(lib().pisa_build_pyramid(p.ref(), _ptr(k), _ptr(pyramid), _stream()), "pisa_build_pyramid")
 
 
-def pisa_route(p: Params, q, k, pyramid, idx, margin, ws):
-    _check(lib().pisa_route(p.ref(), _ptr(q), _ptr(k), _ptr(pyramid), _ptr(idx), _ptr(margin), _ptr(ws),
-                            ws.numel(), _stream()), "pisa_route")
+def pisa_route(p: Params, q, k, pyramid, idx, margin, ws, sel_lse=None):
+    """sel_lse: optional float [B, Hq, N, K] output (per-head denominators of the kept leaves)."""
+    _check(lib().pisa_route(p.ref(), _ptr(q), _ptr(k), _ptr(pyramid), _ptr(idx), _ptr(sel_lse), _ptr(margin),
+                            _ptr(ws), ws.numel(), _stream()), "pisa_route")
 
 
 def pisa_route_static(p: Params, q, k, pyramid, idx, margin):
@@ -178,9 +183,10 @@ def route_static_capacity() -> int:
     return int(lib().pisa_route_static_capacity())
 
 
-def pisa_bsa_fwd(p: Params, q, k, v, idx, out, lse, ws):
-    _check(lib().pisa_bsa_fwd(p.ref(), _ptr(q), _ptr(k), _ptr(v), _ptr(idx), _ptr(out), _ptr(lse), _ptr(ws),
-                              ws.numel(), _stream()), "pisa_bsa_fwd")
+def pisa_bsa_fwd(p: Params, q, k, v, idx, out, lse, ws, sel_lse=None):
+    """sel_lse: optional float [B, Hq, N, K] input, as pisa_route wrote it for these idx."""
+    _check(lib().pisa_bsa_fwd(p.ref(), _ptr(q), _ptr(k), _ptr(v), _ptr(idx), _ptr(sel_lse), _ptr(out), _ptr(lse),
+                              _ptr(ws), ws.numel(), _stream()), "pisa_bsa_fwd")
 
 
 def pisa_forward(p: Params, q, k, v, pyramid, idx, out, lse, ws):
@@ -234,6 +240,11 @@ def pisa_pyramid_regrow(p_old: Params, p_new: Params, pyramid_old, pyramid_new):
 def pisa_flat_select(p: Params, q, pyramid, idx, ws):
     _check(lib().pisa_flat_select(p.ref(), _ptr(q), _ptr(pyramid), _ptr(idx), _ptr(ws), ws.numel(), _stream()),
            "pisa_flat_select")
+
+
+def debug_wait_timeout(ws, limit_ns: int):
+    """Launches the bounded-wait self-test (one CTA waiting on a barrier nobody arrives at)."""
+    _check(lib().pisa_debug_wait_timeout(_ptr(ws), int(limit_ns), _stream()), "pisa_debug_wait_timeout")
 
 
 def read_status(ws) -> int:

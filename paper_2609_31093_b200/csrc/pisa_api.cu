@@ -1,6 +1,7 @@
 // C-ABI entry points of libpisa: argument checks, hierarchy/workspace layout, stage sequencing.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "pisa_common.cuh"
@@ -53,6 +54,31 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 static size_t elem_size(int dtype) { return dtype == PISA_BF16 ? 2 : 4; }
 
+// PISA_DEBUG=1 in the environment switches the device-side index checks on for every call
+static int env_debug_bits() {
+  static int bits = -1;
+  if (bits < 0) {
+    const char* e = getenv("PISA_DEBUG");
+    bits = (e != nullptr && e[0] != '\0' && e[0] != '0') ? PISA_DEBUG_BOUNDS : 0;
+  }
+  return bits;
+}
+
+// SM count of the current device (cached per device ordinal)
+int num_sms() {
+  constexpr int kMaxDev = 64;
+  static int cached[kMaxDev] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) dev = 0;
+  int n = __atomic_load_n(&cached[dev], __ATOMIC_RELAXED);
+  if (n == 0) {
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+    __atomic_store_n(&cached[dev], n, __ATOMIC_RELAXED);
+  }
+  return n;
+}
+
 int resolve(const pisa_params_t* p, Geometry* g) {
   if (p == nullptr || g == nullptr) return PISA_ERR_INVALID_ARG;
   if (p->B <= 0 || p->N <= 0 || p->Hq <= 0 || p->Hkv <= 0 || p->d <= 0 || p->C <= 0) return PISA_ERR_INVALID_ARG;
@@ -69,6 +95,7 @@ int resolve(const pisa_params_t* p, Geometry* g) {
   g->B = p->B; g->N = p->N; g->Hq = p->Hq; g->Hkv = p->Hkv; g->G = G; g->d = p->d;
   g->C = p->C; g->g = p->g; g->K = p->K;
   g->score_mode = p->score_mode;
+  g->debug = p->debug | env_debug_bits();
   g->scale = (p->scale == 0.f) ? (float)(1.0 / sqrt((double)p->d)) : p->scale;
   g->M[0] = p->N;
   g->M[1] = (p->N + p->C - 1) / p->C;
@@ -115,6 +142,8 @@ static size_t pyramid_bytes_dtype(const Geometry& g, int dtype) {
 }
 
 static bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+// the pyramid is read with 32-byte loads
+static bool misaligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) != 0; }
 
 static bool use_tensor(const pisa_params_t* p, const Geometry& g) {
   if (p->impl == PISA_IMPL_SIMT) return false;
@@ -171,20 +200,24 @@ static int clear_status(void* ws, cudaStream_t s) {
 }
 
 static int do_route(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* pyr,
-                    int32_t* idx, float* margin, float* lse_out, void* ws, size_t ws_bytes, cudaStream_t s) {
+                    int32_t* idx, float* sel_lse, float* margin, float* lse_out, void* ws, size_t ws_bytes,
+                    cudaStream_t s) {
   if (ws_bytes < route_ws_bytes(p, g)) return PISA_ERR_WORKSPACE_TOO_SMALL;
   if (use_tensor(p, g))
-    return tensor_route(g, p->dtype, q, k, pyr, idx, margin, lse_out, (char*)ws + kStatusBytes, (int32_t*)ws, s);
+    return tensor_route(g, p->dtype, q, k, pyr, idx, sel_lse, margin, lse_out, (char*)ws + kStatusBytes, (int32_t*)ws, s);
   kernel_mark("route_simt", s);
-  return launch_route_simt(g, p->dtype, q, k, pyr, idx, margin, s);
+  int st = launch_route_simt(g, p->dtype, q, k, pyr, idx, margin, s);
+  if (st != PISA_OK || sel_lse == nullptr) return st;
+  kernel_mark("sel_lse", s);
+  return launch_sel_lse_simt(g, p->dtype, q, k, idx, sel_lse, (int32_t*)ws, s);
 }
 
 static int do_bsa(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v,
-                  const int32_t* idx, void* out, float* lse, bool lse_ready, void* ws, size_t ws_bytes,
-                  cudaStream_t s) {
+                  const int32_t* idx, const float* sel_lse, void* out, float* lse, bool lse_ready, void* ws,
+                  size_t ws_bytes, cudaStream_t s) {
   if (ws_bytes < bsa_ws_bytes(p, g)) return PISA_ERR_WORKSPACE_TOO_SMALL;
   if (use_tensor(p, g))
-    return tensor_bsa(g, p->dtype, q, k, v, idx, out, lse, lse_ready, (char*)ws + kStatusBytes, (int32_t*)ws, s);
+    return tensor_bsa(g, p->dtype, q, k, v, idx, sel_lse, out, lse, lse_ready, (char*)ws + kStatusBytes, (int32_t*)ws, s);
   kernel_mark("bsa_simt", s);
   return launch_bsa_simt(g, p->dtype, q, k, v, idx, out, lse, s);
 }
@@ -299,18 +332,31 @@ static int forward_plan(const pisa_params_t* p, const Geometry& g, int ops, Forw
   return PISA_OK;
 }
 
-static thread_local cudaStream_t g_side[kMaxStreams] = {};  // internal streams ([0] unused) and fork / join events
-static thread_local cudaEvent_t g_fork = nullptr, g_join[kMaxStreams] = {};
+// Internal streams ([0] unused) and fork / join events, per host thread AND per device: streams and
+// events belong to the device that was current when they were made.  g_side / g_fork / g_join point at
+// the set of the device that is current in the call being served (side_streams() selects it).
+constexpr int kMaxDevices = 64;
+struct SideSet { cudaStream_t side[kMaxStreams]; cudaEvent_t fork, join[kMaxStreams]; };
+static thread_local SideSet g_sets[kMaxDevices] = {};
+static thread_local cudaStream_t* g_side = g_sets[0].side;
+static thread_local cudaEvent_t g_fork = nullptr;
+static thread_local cudaEvent_t* g_join = g_sets[0].join;
 
 static int side_streams() {
-  if (g_fork != nullptr) return PISA_OK;
-  cudaError_t e = cudaSuccess;
-  for (int i = 1; i < kMaxStreams && e == cudaSuccess; ++i) {
-    e = cudaStreamCreateWithFlags(&g_side[i], cudaStreamNonBlocking);
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_join[i], cudaEventDisableTiming);
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) { record_cuda_error("cudaGetDevice", e); return PISA_ERR_CUDA; }
+  if (dev < 0 || dev >= kMaxDevices) return PISA_ERR_UNSUPPORTED;
+  SideSet& ss = g_sets[dev];
+  if (ss.fork == nullptr) {
+    for (int i = 1; i < kMaxStreams && e == cudaSuccess; ++i) {
+      e = cudaStreamCreateWithFlags(&ss.side[i], cudaStreamNonBlocking);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ss.join[i], cudaEventDisableTiming);
+    }
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming);
+    if (e != cudaSuccess) { record_cuda_error("internal streams", e); ss.fork = nullptr; return PISA_ERR_CUDA; }
   }
-  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_fork, cudaEventDisableTiming);
-  if (e != cudaSuccess) { record_cuda_error("internal streams", e); g_fork = nullptr; return PISA_ERR_CUDA; }
+  g_side = ss.side; g_fork = ss.fork; g_join = ss.join;
   return PISA_OK;
 }
 
@@ -378,38 +424,39 @@ static int run_chunks(const pisa_params_t* p, const Geometry& g, const ForwardPl
 }
 
 static int do_route_chunked(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* pyr,
-                            int32_t* idx, float* margin, void* ws, size_t ws_bytes, cudaStream_t s) {
+                            int32_t* idx, float* sel_lse, float* margin, void* ws, size_t ws_bytes, cudaStream_t s) {
   ForwardPlan pl;
   int st = plan_for(p, g, kOpRoute, ws_bytes, &pl);
   if (st != PISA_OK) return st;
   st = clear_status(ws, s);
   if (st != PISA_OK) return st;
   g_mark_n = 0;
-  if (pl.n == 1) st = do_route(p, g, q, k, pyr, idx, margin, nullptr, ws, ws_bytes, s);
+  if (pl.n == 1) st = do_route(p, g, q, k, pyr, idx, sel_lse, margin, nullptr, ws, ws_bytes, s);
   else
     st = run_chunks(p, g, pl, ws, s, [&](const ChunkView& v, int) {
       return tensor_route(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, pyr,
-                          idx + v.unit0 * g.N * g.K, margin ? margin + v.unit0 * g.N : nullptr, nullptr, v.region,
-                          (int32_t*)ws, v.stream);
+                          idx + v.unit0 * g.N * g.K, sel_lse ? sel_lse + v.unit0 * g.G * g.N * g.K : nullptr,
+                          margin ? margin + v.unit0 * g.N : nullptr, nullptr, v.region, (int32_t*)ws, v.stream);
     });
   kernel_mark("end", s);
   return st;
 }
 
 static int do_bsa_chunked(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v_,
-                          const int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes, cudaStream_t s) {
+                          const int32_t* idx, const float* sel_lse, void* out, float* lse, void* ws, size_t ws_bytes,
+                          cudaStream_t s) {
   ForwardPlan pl;
   int st = plan_for(p, g, kOpBsa, ws_bytes, &pl);
   if (st != PISA_OK) return st;
   st = clear_status(ws, s);
   if (st != PISA_OK) return st;
   g_mark_n = 0;
-  if (pl.n == 1) st = do_bsa(p, g, q, k, v_, idx, out, lse, false, ws, ws_bytes, s);
+  if (pl.n == 1) st = do_bsa(p, g, q, k, v_, idx, sel_lse, out, lse, false, ws, ws_bytes, s);
   else
     st = run_chunks(p, g, pl, ws, s, [&](const ChunkView& v, int) {
       return tensor_bsa(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, (const char*)v_ + v.v_off,
-                        idx + v.unit0 * g.N * g.K, (char*)out + v.o_off, lse + v.unit0 * g.G * g.N, false, v.region,
-                        (int32_t*)ws, v.stream);
+                        idx + v.unit0 * g.N * g.K, sel_lse ? sel_lse + v.unit0 * g.G * g.N * g.K : nullptr,
+                        (char*)out + v.o_off, lse + v.unit0 * g.G * g.N, false, v.region, (int32_t*)ws, v.stream);
     });
   kernel_mark("end", s);
   return st;
@@ -455,25 +502,48 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
   if (pl.n == 1) {
     // the tensor-core routing already knows every kept leaf's per-head LSE, so it hands the rows'
     // softmax denominators to the attention stage
-    st = do_route(p, g, q, k, pyr, idx, nullptr, lse, ws, ws_bytes, s);
+    st = do_route(p, g, q, k, pyr, idx, nullptr, nullptr, lse, ws, ws_bytes, s);
     if (st != PISA_OK) return st;
     stage_mark(2, s);
-    st = do_bsa(p, g, q, k, v_, idx, out, lse, use_tensor(p, g) && g.score_mode == PISA_SCORE_LSE, ws, ws_bytes, s);
+    st = do_bsa(p, g, q, k, v_, idx, nullptr, out, lse, use_tensor(p, g) && g.score_mode == PISA_SCORE_LSE, ws, ws_bytes, s);
   } else {
     st = run_chunks(p, g, pl, ws, s, [&](const ChunkView& v, int i) {
       int32_t* ic = idx + v.unit0 * g.N * g.K;
       float* lc = lse + v.unit0 * g.G * g.N;
-      int r = tensor_route(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, pyr, ic, nullptr, lc,
-                           v.region, (int32_t*)ws, v.stream);
+      int r = tensor_route(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, pyr, ic, nullptr, nullptr,
+                           lc, v.region, (int32_t*)ws, v.stream);
       if (r != PISA_OK) return r;
       if (i == 0) stage_mark(2, s);
       return tensor_bsa(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, (const char*)v_ + v.v_off,
-                        ic, (char*)out + v.o_off, lc, g.score_mode == PISA_SCORE_LSE, v.region, (int32_t*)ws, v.stream);
+                        ic, nullptr, (char*)out + v.o_off, lc, g.score_mode == PISA_SCORE_LSE, v.region, (int32_t*)ws,
+                        v.stream);
     });
   }
   stage_mark(3, s);
   kernel_mark("end", s);
   return st;
+}
+
+// pisa_route on the caller's stream only, never split into chunks: creates no stream or event
+int route_unsplit(const pisa_params_t* p, const void* q, const void* k, const void* pyramid, int32_t* idx,
+                  float* margin, void* ws, size_t ws_bytes, cudaStream_t s) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (!q || !k || !pyramid || !idx || !ws || misaligned(q) || misaligned(k) || misaligned32(pyramid) || misaligned(ws))
+    return PISA_ERR_INVALID_ARG;
+  if (ws_bytes < route_ws_bytes(p, g)) return PISA_ERR_WORKSPACE_TOO_SMALL;
+  st = clear_status(ws, s);
+  if (st != PISA_OK) return st;
+  return do_route(p, g, q, k, pyramid, idx, nullptr, margin, nullptr, ws, ws_bytes, s);
+}
+// bytes route_unsplit needs
+int route_unsplit_bytes(const pisa_params_t* p, size_t* bytes) {
+  Geometry g;
+  const int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  *bytes = route_ws_bytes(p, g);
+  return PISA_OK;
 }
 
 }  // namespace pisa
@@ -567,30 +637,30 @@ int pisa_build_pyramid(const pisa_params_t* p, const void* k, void* pyramid, voi
   Geometry g;
   int st = resolve(p, &g);
   if (st != PISA_OK) return st;
-  if (k == nullptr || pyramid == nullptr || misaligned(k) || misaligned(pyramid)) return PISA_ERR_INVALID_ARG;
+  if (k == nullptr || pyramid == nullptr || misaligned(k) || misaligned32(pyramid)) return PISA_ERR_INVALID_ARG;
   return launch_pyramid(g, p->dtype, k, pyramid, (cudaStream_t)stream);
 }
 
 int pisa_route(const pisa_params_t* p, const void* q, const void* k, const void* pyramid, int32_t* idx,
-               float* margin, void* ws, size_t ws_bytes, void* stream) {
+               float* sel_lse, float* margin, void* ws, size_t ws_bytes, void* stream) {
   Geometry g;
   int st = resolve(p, &g);
   if (st != PISA_OK) return st;
-  if (!q || !k || !pyramid || !idx || !ws || misaligned(q) || misaligned(k) || misaligned(pyramid) ||
+  if (!q || !k || !pyramid || !idx || !ws || misaligned(q) || misaligned(k) || misaligned32(pyramid) ||
       misaligned(ws))
     return PISA_ERR_INVALID_ARG;
-  return do_route_chunked(p, g, q, k, pyramid, idx, margin, ws, ws_bytes, (cudaStream_t)stream);
+  return do_route_chunked(p, g, q, k, pyramid, idx, sel_lse, margin, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 int pisa_bsa_fwd(const pisa_params_t* p, const void* q, const void* k, const void* v, const int32_t* idx,
-                 void* out, float* lse, void* ws, size_t ws_bytes, void* stream) {
+                 const float* sel_lse, void* out, float* lse, void* ws, size_t ws_bytes, void* stream) {
   Geometry g;
   int st = resolve(p, &g);
   if (st != PISA_OK) return st;
   if (!q || !k || !v || !idx || !out || !lse || !ws || misaligned(q) || misaligned(k) || misaligned(v) ||
       misaligned(out) || misaligned(ws))
     return PISA_ERR_INVALID_ARG;
-  return do_bsa_chunked(p, g, q, k, v, idx, out, lse, ws, ws_bytes, (cudaStream_t)stream);
+  return do_bsa_chunked(p, g, q, k, v, idx, sel_lse, out, lse, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const void* v, void* pyramid,
@@ -599,7 +669,7 @@ int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const voi
   int st = resolve(p, &g);
   if (st != PISA_OK) return st;
   if (!q || !k || !v || !pyramid || !idx || !out || !lse || !ws || misaligned(q) || misaligned(k) ||
-      misaligned(v) || misaligned(pyramid) || misaligned(out) || misaligned(ws))
+      misaligned(v) || misaligned32(pyramid) || misaligned(out) || misaligned(ws))
     return PISA_ERR_INVALID_ARG;
   return do_forward(p, g, q, k, v, pyramid, idx, out, lse, ws, ws_bytes, (cudaStream_t)stream);
 }
@@ -611,7 +681,7 @@ int pisa_forward_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32
   int st = resolve(p, &g);
   if (st != PISA_OK) return st;
   if (!cu_seqlens || nseq < 0 || !q || !k || !v || !pyramid || !idx || !out || !lse || !ws || misaligned(q) ||
-      misaligned(k) || misaligned(v) || misaligned(pyramid) || misaligned(out) || misaligned(ws))
+      misaligned(k) || misaligned(v) || misaligned32(pyramid) || misaligned(out) || misaligned(ws))
     return PISA_ERR_INVALID_ARG;
   if (p->B != 1 || cu_seqlens[0] != 0) return PISA_ERR_INVALID_ARG;
   for (int i = 0; i < 3; ++i)
@@ -832,7 +902,7 @@ int pisa_decode_step(const pisa_params_t* p, int32_t pos, const void* q, const v
   int st = resolve(p, &g);
   if (st != PISA_OK) return st;
   if (!q || !k_cache || !v_cache || !pyramid || !idx || !out || !lse || !ws) return PISA_ERR_INVALID_ARG;
-  if (misaligned(q) || misaligned(k_cache) || misaligned(v_cache) || misaligned(pyramid) || misaligned(ws))
+  if (misaligned(q) || misaligned(k_cache) || misaligned(v_cache) || misaligned32(pyramid) || misaligned(ws))
     return PISA_ERR_INVALID_ARG;
   if (pos < 0 || pos >= g.N) return PISA_ERR_INVALID_ARG;
   if (!decode_supported(g, p->dtype)) return PISA_ERR_UNSUPPORTED;
@@ -851,7 +921,7 @@ int pisa_pyramid_regrow(const pisa_params_t* p_old, const pisa_params_t* p_new, 
   if (st != PISA_OK) return st;
   st = resolve(p_new, &gn);
   if (st != PISA_OK) return st;
-  if (!pyramid_old || !pyramid_new) return PISA_ERR_INVALID_ARG;
+  if (!pyramid_old || !pyramid_new || misaligned32(pyramid_old) || misaligned32(pyramid_new)) return PISA_ERR_INVALID_ARG;
   if (go.B != gn.B || go.Hkv != gn.Hkv || go.d != gn.d || go.C != gn.C || go.g != gn.g ||
       p_old->dtype != p_new->dtype || gn.N < go.N)
     return PISA_ERR_INVALID_ARG;
@@ -871,7 +941,7 @@ int pisa_flat_select(const pisa_params_t* p, const void* q, const void* pyramid,
   Geometry g;
   int st = resolve(p, &g);
   if (st != PISA_OK) return st;
-  if (!q || !pyramid || !idx || !ws || misaligned(q) || misaligned(pyramid)) return PISA_ERR_INVALID_ARG;
+  if (!q || !pyramid || !idx || !ws || misaligned(q) || misaligned32(pyramid)) return PISA_ERR_INVALID_ARG;
   if (ws_bytes < kStatusBytes) return PISA_ERR_WORKSPACE_TOO_SMALL;
   st = clear_status(ws, (cudaStream_t)stream);
   if (st != PISA_OK) return st;
@@ -885,6 +955,15 @@ int pisa_read_status(const void* ws, int32_t* status) {
   if (e != cudaSuccess) { record_cuda_error("status read", e); return PISA_ERR_CUDA; }
   *status = word;
   return PISA_OK;
+}
+
+int pisa_debug_wait_timeout(void* ws, unsigned long long limit_ns, void* stream) {
+  if (!ws || misaligned(ws)) return PISA_ERR_INVALID_ARG;
+  if (limit_ns < 1000ull) limit_ns = 1000ull;
+  if (limit_ns > 1000000000ull) limit_ns = 1000000000ull;
+  int st = clear_status(ws, (cudaStream_t)stream);
+  if (st != PISA_OK) return st;
+  return launch_wait_timeout((int32_t*)ws, limit_ns, (cudaStream_t)stream);
 }
 
 int pisa_get_kernel_ms(int i, char* name, size_t name_len, float* ms) {

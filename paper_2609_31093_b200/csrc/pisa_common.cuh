@@ -18,6 +18,7 @@ constexpr int kWarp = 32;
 struct Geometry {
   int B, N, Hq, Hkv, G, d, C, g, K, L;
   int score_mode;
+  int debug;                       // PISA_DEBUG_* bits
   float scale;
   int M[kMaxLevels];               // M[0] = N, M[l] = blocks at level l
   long long span[kMaxLevels];      // span[l] = g^(l-1): leaves under one level-l node
@@ -27,6 +28,14 @@ struct Geometry {
 
 // Status word at the start of every workspace (device int32[4]; [0] = pisa_status).
 constexpr size_t kStatusBytes = 256;
+
+// Index check of the PISA_DEBUG_BOUNDS mode: true if 0 <= v < n; otherwise records PISA_ERR_BOUNDS in
+// the status word (the caller then skips the access).
+__device__ __forceinline__ bool bounds_ok(long long v, long long n, int32_t* status) {
+  if (v >= 0 && v < n) return true;
+  atomicExch(status, (int)PISA_ERR_BOUNDS);
+  return false;
+}
 
 int resolve(const pisa_params_t* p, Geometry* g);                // validates; returns pisa_status
 size_t align_up(size_t x, size_t a);
@@ -47,6 +56,12 @@ int launch_bsa_simt(const Geometry& g, int dtype, const void* q, const void* k, 
                     const int32_t* idx, void* out, float* lse, cudaStream_t s);
 int launch_flat_simt(const Geometry& g, int dtype, const void* q, const void* pyramid, int32_t* idx,
                      cudaStream_t s);
+// per-head softmax denominators of the selected leaves, float [B,Hq,N,K] (exact fp32, any shape)
+int launch_sel_lse_simt(const Geometry& g, int dtype, const void* q, const void* k, const int32_t* idx,
+                        float* sel_lse, int32_t* status, cudaStream_t s);
+// one CTA waiting, with a time limit, on a barrier nobody arrives at (self-test of the bounded waits)
+int launch_wait_timeout(int32_t* status, unsigned long long limit_ns, cudaStream_t s);
+int num_sms();                        // SM count of the current device
 
 // decoding step (one token per sequence); ws points past the status word
 bool decode_supported(const Geometry& g, int dtype);

@@ -10,11 +10,14 @@ size_t tensor_route_workspace_bytes(const Geometry& g);
 size_t tensor_bsa_workspace_bytes(const Geometry& g);
 // ws points past the status word; status is the workspace's status word
 // lse_out (nullable): softmax denominators of the kept leaves, float [B,Hq,N]
+// sel_lse (nullable): per-head denominators of the kept leaves, float [B,Hq,N,K]
 int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, const void* pyramid, int32_t* idx,
-                 float* margin, float* lse_out, void* ws, int32_t* status, cudaStream_t s);
+                 float* sel_lse, float* margin, float* lse_out, void* ws, int32_t* status, cudaStream_t s);
 // lse_ready: `lse` already holds the denominators of exactly these idx (as tensor_route writes them)
+// sel_lse (nullable): per-block denominators of exactly these idx (as tensor_route writes them); used when
+// lse_ready is false to skip the block-LSE pass
 int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const void* v, const int32_t* idx,
-               void* out, float* lse, bool lse_ready, void* ws, int32_t* status, cudaStream_t s);
+               const float* sel_lse, void* out, float* lse, bool lse_ready, void* ws, int32_t* status, cudaStream_t s);
 
 // backward of the block-sparse attention with frozen indices; dq [B,N,Hq,d], dk, dv [B,N,Hkv,d] dense
 bool tensor_bwd_supported(const Geometry& g, int dtype);

@@ -11,6 +11,14 @@
 
 #include "pisa_common.cuh"
 
+namespace pisa {
+// the routing of pisa_route on the caller's stream alone (no chunks on a second stream, hence no stream or
+// event creation), and its scratch size
+int route_unsplit(const pisa_params_t* p, const void* q, const void* k, const void* pyramid, int32_t* idx,
+                  float* margin, void* ws, size_t ws_bytes, cudaStream_t s);
+int route_unsplit_bytes(const pisa_params_t* p, size_t* bytes);
+}  // namespace pisa
+
 namespace {
 
 constexpr size_t kStaticScratchBytes = 32u << 20;      // 32 MiB per GPU
@@ -48,15 +56,17 @@ int scratch_for_current_device(void** out) {
 extern "C" int pisa_route_static(const pisa_params_t* p, const void* q, const void* k, const void* pyramid,
                                  int32_t* idx, float* margin, void* stream) {
   size_t need = 0;
-  int st = pisa_workspace_bytes(p, PISA_OP_ROUTE, &need);
+  int st = pisa::route_unsplit_bytes(p, &need);
   if (st != PISA_OK) return st;
   if (need > kStaticScratchBytes) return PISA_ERR_STATIC_SCRATCH_TOO_SMALL;
   void* scratch = nullptr;
   st = scratch_for_current_device(&scratch);
   if (st != PISA_OK) return st;
-  // pisa_route clears the status word and the list counters it needs at zero on the stream before
-  // its kernels read them; everything else in the scratch is written before it is read.
-  return pisa_route(p, q, k, pyramid, idx, margin, scratch, kStaticScratchBytes, stream);
+  // The routing runs as ONE sequence of launches on the caller's stream (pisa_route would cut a large
+  // problem into chunks on a second, library-owned stream, whose creation allocates).  It clears the
+  // status word and the list counters it needs at zero on the stream before its kernels read them;
+  // everything else in the scratch is written before it is read.
+  return pisa::route_unsplit(p, q, k, pyramid, idx, margin, scratch, need, (cudaStream_t)stream);
 }
 
 extern "C" size_t pisa_route_static_capacity(void) { return kStaticScratchBytes; }

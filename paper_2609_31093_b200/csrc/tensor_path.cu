@@ -55,13 +55,18 @@ struct InvArgs {
   int32_t* cursor;        // [nkeys]
   int32_t* blk_tot;       // [3][ceil(nkeys / 1024) + 1] scan scratch: per-block totals, then block offsets
   int32_t* entries;       // [<= BH*N*K]  token | slot << 24
+  int32_t* status;        // the workspace's status word
+  int debug;              // PISA_DEBUG_* bits
 };
 
 __device__ __forceinline__ int inv_token(const InvArgs& a, int e) { return a.lgK >= 0 ? (e >> a.lgK) : e / a.K; }
 __device__ __forceinline__ int inv_slot(const InvArgs& a, int e) { return a.lgK >= 0 ? (e & (a.K - 1)) : e % a.K; }
 __device__ __forceinline__ bool inv_valid(const InvArgs& a, int node, int t) {
   const int leaf = a.lgC >= 0 ? (t >> a.lgC) : t / a.C;
-  return node >= 0 && node < a.Mk && (long long)node * a.fan <= (long long)leaf;
+  const bool ok = node >= 0 && node < a.Mk && (long long)node * a.fan <= (long long)leaf;
+  // bounds-check mode: anything but the -1 padding that is not a usable node id is reported
+  if ((a.debug & PISA_DEBUG_BOUNDS) && !ok && node != -1) atomicExch(a.status, (int)PISA_ERR_BOUNDS);
+  return ok;
 }
 
 __global__ void __launch_bounds__(256) inv_count_kernel(InvArgs a, int use_smem) {
@@ -236,6 +241,7 @@ struct TileArgs {
   const float* row_lse;    // [B, Hq, N]              (tile_pv)
   float* o_acc;            // fp32 accumulator: [B, Hkv, N, D, G] when the second product is transposed, else [B, N, Hq, D]
   int32_t* status;
+  int debug;               // PISA_DEBUG_* bits: list entries are range-checked before they are used
 };
 
 __device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
@@ -329,6 +335,14 @@ constexpr int kMetaRing = 8;           // ring of per-tile metadata; deeper than
 struct ItemInfo {
   int key, ntiles, e_begin, e_end;
 };
+// bounds-check mode: a list entry (token | slot << 24) must name a token below N and a slot below `slots`;
+// one that does not is reported and dropped (-1 = no entry)
+__device__ __forceinline__ int checked_entry(const TileArgs& a, int N, int ent) {
+  if (!(a.debug & PISA_DEBUG_BOUNDS) || ent < 0) return ent;
+  if ((ent & 0xFFFFFF) < N && (ent >> 24) < a.slots) return ent;
+  atomicExch(a.status, (int)PISA_ERR_BOUNDS);
+  return -1;
+}
 __device__ __forceinline__ int fetch_entry(const int32_t* entries, int e0, int e_end, int tpt, int p) {
   return (p < tpt && e0 + p < e_end) ? entries[e0 + p] : -1;
 }
@@ -484,7 +498,7 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
 #pragma unroll
         for (int i = 0; i < RPT; ++i) {
           const int slot_i = (rb + i * RPP) >> lgG;
-          cur[i] = (e0 + slot_i < inf.e_end) ? nxt[i] : -1;
+          cur[i] = (e0 + slot_i < inf.e_end) ? checked_entry(a, geo.N, nxt[i]) : -1;
           nxt[i] = a.entries[min(e0 + tpt + slot_i, e_last)];
         }
         prod_gather_q_regs<D>(sA + s * A_STAGE, geo, qb, cur, tid);
@@ -547,7 +561,7 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
         const int ent_raw = a.entries[min(e_row, inf.e_end - 1)];
         if (!mbar_wait_bounded(&t_full[grp], (uint32_t)((it >> 1) & 1))) { s_fail = 1; break; }
         tcgen05_fence_after_sync();
-        const int ent = (e_row < inf.e_end) ? ent_raw : -1;
+        const int ent = (e_row < inf.e_end) ? checked_entry(a, geo.N, ent_raw) : -1;
         const bool valid = ent >= 0;
         const int t = ent & 0xFFFFFF, slot = valid ? (ent >> 24) : 0;
         const int c_t = t / C;
@@ -681,8 +695,8 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
         const int s = it % NS;
         const bool bad_t = it >= NS && !mbar_wait_bounded(&q_empty[s], (uint32_t)((it / NS - 1) & 1));
         const int e0 = inf.e_begin + jt * tpt;
-        const int ent_now = (jt == 0) ? fetch_entry(a.entries, e0, inf.e_end, tpt, tid) : ent_next;
-        ent_next = (jt + 1 < inf.ntiles) ? fetch_entry(a.entries, e0 + tpt, inf.e_end, tpt, tid) : -1;
+        const int ent_now = (jt == 0) ? checked_entry(a, geo.N, fetch_entry(a.entries, e0, inf.e_end, tpt, tid)) : ent_next;
+        ent_next = (jt + 1 < inf.ntiles) ? checked_entry(a, geo.N, fetch_entry(a.entries, e0 + tpt, inf.e_end, tpt, tid)) : -1;
         s_ent[it % kMetaRing][tid] = ent_now;
         if (prod_sync_or(bad_t)) { s_fail = 1; stop = true; break; }
         prod_gather_q<D>(sQ + s * Q_STAGE, geo, qb, s_ent[it % kMetaRing], tid);
@@ -980,7 +994,8 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
 __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int32_t* __restrict__ par,
                                                           const float* __restrict__ blk_lse,
                                                           int32_t* __restrict__ idx, float* __restrict__ margin,
-                                                          float* __restrict__ lse_out) {
+                                                          float* __restrict__ lse_out, float* __restrict__ sel_lse,
+                                                          int32_t* status) {
   __shared__ __align__(16) float s_u[4][kMaxCand];
   __shared__ int s_sel[4][kMaxK];
   __shared__ float s_cut[4][2];
@@ -1008,7 +1023,8 @@ __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int
     const int ci = c0 + lane;
     bool ok = false;
     if (ci < gK) {
-      const int p = pr[ci / g];
+      int p = pr[ci / g];
+      if ((geo.debug & PISA_DEBUG_BOUNDS) && p != -1 && !bounds_ok(p, geo.M[2], status)) p = -1;
       const int leaf = p * g + ci % g;
       ok = (p >= 0) && (leaf <= c);
       float sc = -CUDART_INF_F;
@@ -1061,7 +1077,19 @@ __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int
     kept_mask[ch] = bal;
     const int pos = base + __popc(bal & ((1u << lane) - 1u));
     if (keep) s_sel[warp][pos] = pr[s / g] * g + s % g;
+    if (keep && sel_lse != nullptr) {
+      // the kept leaf's per-head scores ARE its per-head softmax denominators (LSE mode)
+      const int bq = bh / geo.Hkv, hq = bh % geo.Hkv;
+      for (int hh = 0; hh < G; ++hh)
+        sel_lse[(((long long)bq * geo.Hq + hq * G + hh) * geo.N + t) * K + pos] = bl[s * G + hh];
+    }
     base += __popc(bal);
+  }
+  if (sel_lse != nullptr) {
+    const int bq = bh / geo.Hkv, hq = bh % geo.Hkv;
+    for (int s = base + lane; s < K; s += 32)
+      for (int hh = 0; hh < G; ++hh)
+        sel_lse[(((long long)bq * geo.Hq + hq * G + hh) * geo.N + t) * K + s] = -CUDART_INF_F;
   }
   __syncwarp();
   int32_t* dst = idx + w * (long long)K;
@@ -1157,6 +1185,32 @@ __global__ void __launch_bounds__(256) row_lse_kernel(Geometry geo, const int32_
   lse_out[((long long)b * geo.Hq + h * geo.G + head) * geo.N + t] = (ssum > 0.f) ? m + logf(ssum) : -CUDART_INF_F;
 }
 
+// the same from per-block denominators the caller hands in (float [B,Hq,N,K], as pisa_route writes them)
+__global__ void __launch_bounds__(256) row_lse_from_sel_kernel(Geometry geo, const int32_t* __restrict__ idx,
+                                                                const float* __restrict__ sel_lse,
+                                                                float* __restrict__ lse_out) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;     // (b*Hq + hq)*N + t
+  const long long total = (long long)geo.B * geo.Hq * geo.N;
+  if (i >= total) return;
+  const int t = (int)(i % geo.N);
+  const int hq = (int)((i / geo.N) % geo.Hq);
+  const int b = (int)(i / ((long long)geo.N * geo.Hq));
+  const int32_t* row = idx + (((long long)b * geo.Hkv + hq / geo.G) * geo.N + t) * geo.K;
+  const float* sl = sel_lse + i * geo.K;
+  const int c = t / geo.C;
+  float m = -CUDART_INF_F;
+  for (int s = 0; s < geo.K; ++s) {
+    const int leaf = row[s];
+    if (leaf >= 0 && leaf <= c && leaf < geo.M[1]) m = fmaxf(m, sl[s]);
+  }
+  float ssum = 0.f;
+  for (int s = 0; s < geo.K; ++s) {
+    const int leaf = row[s];
+    if (leaf >= 0 && leaf <= c && leaf < geo.M[1] && sl[s] > -CUDART_INF_F) ssum += expf(sl[s] - m);
+  }
+  lse_out[i] = (ssum > 0.f) ? m + logf(ssum) : -CUDART_INF_F;
+}
+
 // fp32 accumulator [B,N,Hq,d] -> out in bf16 (strided)
 __global__ void __launch_bounds__(256) convert_out_kernel(Geometry geo, const float* __restrict__ acc,
                                                            __nv_bfloat16* __restrict__ out) {
@@ -1249,20 +1303,10 @@ BsaLayout bsa_layout(const Geometry& g) {
   return r;
 }
 
-int num_sms() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
-  return n;
-}
-
 int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char* ws, const InvLayout& l,
-                  InvArgs* out, cudaStream_t s, int win = kWindowTok) {
+                  InvArgs* out, int32_t* status, cudaStream_t s, int win = kWindowTok) {
   InvArgs a;
+  a.status = status; a.debug = g.debug;
   a.nodes = nodes; a.K = g.K; a.fan = fan; a.Mk = Mk; a.N = g.N; a.C = g.C; a.BH = g.B * g.Hkv;
   a.tpt = 128 / g.G;
   a.lgK = (g.K & (g.K - 1)) == 0 ? 31 - __builtin_clz((unsigned)g.K) : -1;
@@ -1391,7 +1435,7 @@ size_t tensor_route_workspace_bytes(const Geometry& g) { return route_layout(g).
 size_t tensor_bsa_workspace_bytes(const Geometry& g) { return bsa_layout(g).total; }
 
 int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, const void* pyramid, int32_t* idx,
-                 float* margin, float* lse_out, void* ws_, int32_t* status, cudaStream_t s) {
+                 float* sel_lse, float* margin, float* lse_out, void* ws_, int32_t* status, cudaStream_t s) {
   char* ws = (char*)ws_;
   const RouteLayout L = route_layout(g);
   int32_t* par = (int32_t*)(ws + L.par);
@@ -1402,26 +1446,31 @@ int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, con
   if (st != PISA_OK) return st;
   kernel_mark("invert_by_parent", s);
   InvArgs inv;
-  st = run_inversion(g, par, g.g, g.M[2], ws, L.inv, &inv, s);
+  st = run_inversion(g, par, g.g, g.M[2], ws, L.inv, &inv, status, s);
   if (st != PISA_OK) return st;
   TileArgs a = {};
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = nullptr;
   a.entry_off = inv.entry_off; a.tile_off = inv.tile_off; a.item_off = inv.item_off; a.item_key = inv.item_key; a.entries = inv.entries;
   a.nkeys = g.B * g.Hkv * inv.NW * g.M[2]; a.Mk = g.M[2]; a.NW = inv.NW; a.fan = g.g; a.slots = g.K;
-  a.blk_lse = blk; a.status = status; a.mode = g.score_mode;
+  a.blk_lse = blk; a.status = status; a.mode = g.score_mode; a.debug = g.debug;
   kernel_mark("leaf_lse_tiles", s);
   st = dispatch_tile_lse(g, g.g * g.C, a, s);
   if (st != PISA_OK) return st;
   kernel_mark("final_topk", s);
   const long long total = (long long)g.B * g.Hkv * g.N;
   // only the LSE scores are also the per-leaf softmax denominators the attention stage can reuse
-  final_topk_kernel<<<(unsigned)((total + 3) / 4), 128, 0, s>>>(g, par, blk, idx, margin,
-                                                                (g.score_mode == PISA_SCORE_LSE) ? lse_out : nullptr);
-  return check_launch("final_topk");
+  const bool lse_scores = g.score_mode == PISA_SCORE_LSE;
+  final_topk_kernel<<<(unsigned)((total + 3) / 4), 128, 0, s>>>(g, par, blk, idx, margin, lse_scores ? lse_out : nullptr,
+                                                                lse_scores ? sel_lse : nullptr, status);
+  st = check_launch("final_topk");
+  if (st != PISA_OK || sel_lse == nullptr || lse_scores) return st;
+  // the other score modes rank by moments of the logits: the denominators take a pass of their own
+  kernel_mark("sel_lse", s);
+  return launch_sel_lse_simt(g, dtype, q, k, idx, sel_lse, status, s);
 }
 
 int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const void* v, const int32_t* idx,
-               void* out, float* lse, bool lse_ready, void* ws_, int32_t* status, cudaStream_t s) {
+               const float* sel_lse, void* out, float* lse, bool lse_ready, void* ws_, int32_t* status, cudaStream_t s) {
   (void)dtype;
   char* ws = (char*)ws_;
   const BsaLayout L = bsa_layout(g);
@@ -1429,14 +1478,20 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
   float* acc = (float*)(ws + L.acc);
   kernel_mark("invert_by_leaf", s);
   InvArgs inv;
-  int st = run_inversion(g, idx, 1, g.M[1], ws, L.inv, &inv, s);
+  int st = run_inversion(g, idx, 1, g.M[1], ws, L.inv, &inv, status, s);
   if (st != PISA_OK) return st;
   TileArgs a = {};
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
   a.entry_off = inv.entry_off; a.tile_off = inv.tile_off; a.item_off = inv.item_off; a.item_key = inv.item_key; a.entries = inv.entries;
   a.nkeys = g.B * g.Hkv * inv.NW * g.M[1]; a.Mk = g.M[1]; a.NW = inv.NW; a.fan = 1; a.slots = g.K;
-  a.blk_lse = blk; a.row_lse = lse; a.o_acc = acc; a.status = status;
-  if (!lse_ready) {
+  a.blk_lse = blk; a.row_lse = lse; a.o_acc = acc; a.status = status; a.debug = g.debug;
+  if (!lse_ready && sel_lse != nullptr) {
+    kernel_mark("row_lse", s);
+    const long long rows = (long long)g.B * g.Hq * g.N;
+    row_lse_from_sel_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, s>>>(g, idx, sel_lse, lse);
+    st = check_launch("row_lse_from_sel");
+    if (st != PISA_OK) return st;
+  } else if (!lse_ready) {
     kernel_mark("block_lse_tiles", s);
     st = dispatch_tile_lse(g, g.C, a, s);
     if (st != PISA_OK) return st;
@@ -1480,7 +1535,7 @@ int tensor_bsa_bwd(const Geometry& g, const void* q, const void* k, const void* 
   const BwdLayout L = bwd_layout(g);
   kernel_mark("invert_by_leaf", s);
   InvArgs inv;
-  int st = run_inversion(g, idx, 1, g.M[1], ws, L.inv, &inv, s, kBwdWindowTok);
+  int st = run_inversion(g, idx, 1, g.M[1], ws, L.inv, &inv, status, s, kBwdWindowTok);
   if (st != PISA_OK) return st;
   BwdArgs a = {};
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;

@@ -86,13 +86,92 @@ def gather_idx(idx_dev: torch.Tensor, triples: np.ndarray) -> np.ndarray:
     return idx_dev[t[:, 0], t[:, 1], t[:, 2]].cpu().numpy()
 
 
-def compare_index_sets(idx_gpu: np.ndarray, idx_ref: np.ndarray, margin_ref: np.ndarray, band=TIE_BAND):
-    """Rows must be equal (both ascending, -1 padded) except where the oracle's cut margin lies in
-    the tie band.  Returns (rows differing, of those outside the band, rows inside the band)."""
+def compare_index_sets(idx_gpu: np.ndarray, idx_ref: np.ndarray, margin_ref: np.ndarray, band=TIE_BAND,
+                       prob=None, triples=None):
+    """Rows must be equal (both ascending, -1 padded) except inside the tie band.  Returns (rows
+    differing, of those not explained by the band, rows whose oracle cut margin lies inside the band).
+
+    A differing row is accepted only if `admissible_under_band` finds the GPU's set among the results
+    the oracle's walk can reach when, at every scored level, a dropped node may replace a kept one whose
+    score exceeds its own by at most the band (`prob` and `triples` give the oracle problem and the
+    rows' (b, KV head, position); without them a differing row with margin <= band is accepted, which
+    is only used where no walk applies, e.g. the flat selector)."""
     diff = np.any(idx_gpu != idx_ref, axis=1)
     in_band = margin_ref <= band
-    bad = diff & ~in_band
+    if prob is None:
+        bad = diff & ~in_band
+    else:
+        bad = np.zeros_like(diff)
+        for s in np.nonzero(diff)[0]:
+            b, h, p = (int(x) for x in triples[s])
+            got = [int(x) for x in idx_gpu[s] if x >= 0]
+            bad[s] = (not in_band[s]) or (not admissible_under_band(prob, b, h, p, got, band))
     return int(diff.sum()), int(bad.sum()), int(in_band.sum())
+
+
+def admissible_under_band(prob: O.Problem, b: int, h: int, p: int, got_leaves, band=TIE_BAND, max_branches=4096):
+    """True if `got_leaves` is a result of the coarse-to-fine walk of Sec. 3.2 for this query when every
+    Select_K may resolve near-ties either way: a set S of the scored (non-forced) candidates is an
+    admissible choice at a level iff no dropped x and kept y have (u_x - u_y) / max(|u_x|, 1) > band, with
+    u the ORACLE's scores.  Every admissible choice is followed (depth first, restricted to choices that
+    contain the ancestors of `got_leaves`), so a set that differs from the oracle's anywhere but at a
+    near-tie, or in anything but the consequences of one, is rejected."""
+    import itertools
+    k_bh, _, lv = prob.head(b, h)
+    qg = prob.q_group(b, h, p)
+    C, g, K, M, L = prob.C, prob.g, prob.K, prob.M, prob.L
+    c = p // C
+    target = sorted(int(x) for x in got_leaves)
+    budget = [max_branches]
+
+    def walk(l, A):
+        if budget[0] <= 0:
+            return False
+        span = g ** (l - 1)
+        V = [i for i in A if i < M[l] and i <= c // span]
+        F = O.forced_nodes(l, c, g)
+        need = {x // span for x in target}                       # ancestors of the claimed leaves
+        if not need <= set(V):
+            return False
+        if len(V) <= K:
+            choices = [list(V)]
+        else:
+            rest = [i for i in V if i not in F]
+            u = {}
+            for i in rest:
+                ch = O.children(l, i, M, C, g)
+                x = k_bh[ch.start:ch.stop] if l == 1 else lv[l - 1][ch.start:ch.stop]
+                u[i] = O.lse_score(qg, x, prob.scale, prob.mode)
+            keep = K - len(F)
+            order = sorted(rest, key=lambda i: (-u[i], i))
+            rel = lambda ux, uy: (ux - uy) / max(abs(ux), 1.0)
+            top, below = order[:keep], order[keep:]
+            must = [x for x in top if rel(u[x], u[below[0]]) > band]
+            may = [x for x in top if x not in must] + [y for y in below if rel(u[top[-1]], u[y]) <= band]
+            want = [x for x in may if x in need]
+            if any(x in need for x in below if x not in may):
+                return False
+            free = [x for x in may if x not in want]
+            r = keep - len(must) - len(want)
+            if r < 0:
+                return False
+            choices = []
+            for extra in itertools.combinations(free, r):
+                S_ = set(must) | set(want) | set(extra)
+                dropped = [x for x in rest if x not in S_]
+                if all(rel(u[x], u[y]) <= band for x in dropped for y in S_):
+                    choices.append(sorted(set(F) | S_))
+        for I in choices:
+            budget[0] -= 1
+            if l == 1:
+                if sorted(I) == target:
+                    return True
+                continue
+            if walk(l - 1, [r_ for i in I for r_ in O.children(l, i, M, C, g)]):
+                return True
+        return False
+
+    return walk(L, [0])
 
 
 def check_index_rows_valid(idx_gpu: np.ndarray, triples: np.ndarray, w: S.Workload):
@@ -109,24 +188,70 @@ def check_index_rows_valid(idx_gpu: np.ndarray, triples: np.ndarray, w: S.Worklo
             assert f in sel, (p, row)
 
 
-def check_outputs(out_gpu: np.ndarray, lse_gpu: np.ndarray, out_ref: np.ndarray, lse_ref: np.ndarray, dtype: str):
+STRICT_RANGE = 2.56      # below this magnitude a bf16 ulp is at most 2e-2 / 1.28: the flat bounds apply as stated
+
+
+def check_outputs(out_gpu: np.ndarray, lse_gpu: np.ndarray, out_ref: np.ndarray, lse_ref: np.ndarray, dtype: str,
+                  report: dict = None):
     """out_* are fp64 arrays of stored values; tolerances per dtype as stated for the path.
 
-    bf16: max-abs 2e-2 and mean-abs 2e-3, stated for outputs of order one.  Both sides round their
-    result to bf16, so where |out| exceeds 2.56 a one-ulp disagreement (2^-7 |out| at most) already
-    exceeds 2e-2; the bound therefore grows by one output ulp, and the mean bound scales with the
-    mean output magnitude when that exceeds one."""
+    bf16: max-abs 2e-2 and mean-abs 2e-3.  These flat bounds are asserted as they stand whenever the
+    reference outputs stay below 2.56 in magnitude (every workload except the random-walk one).  Both
+    sides round their result to bf16, so where |out| exceeds 2.56 a one-ulp disagreement (2^-7 |out|
+    at most) already exceeds 2e-2; only for such outputs the per-element bound grows by one output
+    ulp and the mean bound scales with the mean output magnitude.  `report` (optional dict) receives
+    how many elements needed the ulp term."""
+    if out_ref.size == 0:
+        return 0.0, 0.0, 0.0
     err = np.abs(out_gpu - out_ref)
     lerr = np.abs(lse_gpu - lse_ref)
     if dtype == "bf16":
-        bound = BF16_MAX_ABS + 2.0 ** -7 * np.abs(out_ref)
-        assert np.all(err <= bound), f"max abs {err.max()} (worst excess {(err - bound).max()})"
-        assert err.mean() <= BF16_MEAN_ABS * max(1.0, np.abs(out_ref).mean()), f"mean abs {err.mean()}"
+        over_strict = int((err > BF16_MAX_ABS).sum())
+        if report is not None:
+            report["over_strict"] = report.get("over_strict", 0) + over_strict
+            report["elements"] = report.get("elements", 0) + int(err.size)
+        if np.abs(out_ref).max() <= STRICT_RANGE:
+            assert over_strict == 0, f"max abs {err.max()} > {BF16_MAX_ABS}"
+            assert err.mean() <= BF16_MEAN_ABS, f"mean abs {err.mean()}"
+        else:
+            bound = BF16_MAX_ABS + 2.0 ** -7 * np.abs(out_ref)
+            assert np.all(err <= bound), f"max abs {err.max()} (worst excess {(err - bound).max()})"
+            assert err.mean() <= BF16_MEAN_ABS * max(1.0, np.abs(out_ref).mean()), f"mean abs {err.mean()}"
         assert lerr.max() <= 1e-3 * max(1.0, np.abs(lse_ref).max()), f"lse {lerr.max()}"
     else:
         assert err.max() <= FP32_TOL, f"max abs {err.max()}"
         assert lerr.max() <= FP32_TOL * max(1.0, np.abs(lse_ref).max()), f"lse {lerr.max()}"
     return float(err.max()), float(err.mean()), float(lerr.max())
+
+
+def check_forward_rows(w, prob, tri: np.ndarray, got_idx: np.ndarray, out_gpu: np.ndarray, lse_gpu: np.ndarray,
+                       walk_prob=None, report: dict = None):
+    """The whole forward on sampled rows (b, KV head, position): index sets (exact outside the tie band,
+    admissible inside it), then outputs and denominators of EVERY sampled row -- rows whose set equals
+    the oracle's against the oracle's attention on that set, rows that differ inside the band against
+    the oracle's attention on the GPU's own set.  `prob` does the bulk work (either oracle),
+    `walk_prob` (the NumPy oracle; default `prob`) re-walks the differing rows.
+    got_idx [S, K]; out_gpu [S, G, d] stored values as fp64; lse_gpu [S, G].
+    Returns (rows differing, rows inside the band, (max abs, mean abs, lse) errors)."""
+    ref_idx, ref_margin = prob.route_all(tri)
+    check_index_rows_valid(got_idx, tri, w)
+    n_diff, n_bad, n_band = compare_index_sets(got_idx, ref_idx, ref_margin, prob=walk_prob or prob, triples=tri)
+    assert n_bad == 0, f"{n_bad} of {len(tri)} rows differ from the oracle beyond the tie band"
+    out_ref, lse_ref = prob.attend_all(tri, got_idx)     # the oracle's attention on the GPU's sets (its own where equal)
+    stats = check_outputs(out_gpu, lse_gpu, out_ref, lse_ref, w.dtype, report)
+    return n_diff, n_band, stats
+
+
+def check_forward_dev(dev: "Device", prob, tri: np.ndarray, walk_prob=None, report: dict = None):
+    """check_forward_rows on a Device's idx / out / lse."""
+    out_gpu, lse_gpu = gather_out(dev, tri)
+    return check_forward_rows(dev.w, prob, tri, gather_idx(dev.idx, tri), out_gpu, lse_gpu, walk_prob, report)
+
+
+def oracle_problem_c(w: S.Workload, tensors: dict, mode="lse"):
+    """The compiled oracle on the same tensors (bulk rows at full size; OpenMP over the sampled rows)."""
+    from oracle import pisa_oracle_c as OC
+    return OC.CProblem(tensors["q"], tensors["k"], tensors["v"], C=w.C, g=w.g, K=w.K, dtype=w.dtype, mode=mode)
 
 
 def gather_out(dev: Device, triples: np.ndarray):

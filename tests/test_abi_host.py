@@ -72,7 +72,9 @@ def test_argument_validation():
     # null pointers are rejected before anything is launched (no GPU needed to see that)
     lib = P.lib()
     assert lib.pisa_build_pyramid(ok.ref(), None, None, None) == -1
-    assert lib.pisa_route(ok.ref(), None, None, None, None, None, None, 0, None) == -1
+    assert lib.pisa_route(ok.ref(), None, None, None, None, None, None, None, 0, None) == -1
+    assert lib.pisa_bsa_fwd(ok.ref(), None, None, None, None, None, None, None, None, 0, None) == -1
+    assert lib.pisa_debug_wait_timeout(None, 1000, None) == -1
     assert lib.pisa_forward(ok.ref(), None, None, None, None, None, None, None, None, 0, None) == -1
     assert lib.pisa_status_string(-3).decode() == "workspace too small"
 

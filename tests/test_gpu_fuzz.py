@@ -30,12 +30,4 @@ def test_random_shape_matches_oracle(i):
     assert dev.sync_status() == 0, w
     tri = S.sample_queries(w, 30)
     prob = T.oracle_problem(w, t)
-    ref_idx, ref_margin = prob.route_all(tri)
-    got = T.gather_idx(dev.idx, tri)
-    T.check_index_rows_valid(got, tri, w)
-    n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin)
-    assert n_bad == 0, (w, n_bad)
-    same = ~np.any(got != ref_idx, axis=1)
-    out_ref, lse_ref = prob.attend_all(tri[same], ref_idx[same])
-    out_gpu, lse_gpu = T.gather_out(dev, tri[same])
-    T.check_outputs(out_gpu, lse_gpu, out_ref, lse_ref, w.dtype)
+    T.check_forward_dev(dev, prob, tri)

@@ -49,16 +49,10 @@ def test_host_path_matches_device_path_and_oracle(name):
     # and sampled rows against the oracle
     tri = S.sample_queries(w, 40)
     prob = T.oracle_problem(w, t)
-    ref_idx, ref_margin = prob.route_all(tri)
     ti = torch.from_numpy(tri)
     got = idx_h[ti[:, 0], ti[:, 1], ti[:, 2]].numpy()
-    n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin)
-    assert n_bad == 0
-    same = ~np.any(got != ref_idx, axis=1)
-    out_ref, lse_ref = prob.attend_all(tri[same], ref_idx[same])
     G = w.Hq // w.Hkv
-    ts = ti[torch.from_numpy(same)]
-    heads = ts[:, 1:2] * G + torch.arange(G)[None, :]
-    o = out_h[ts[:, 0:1], ts[:, 2:3], heads].to(torch.float64).numpy()
-    l = lse_h[ts[:, 0:1], heads, ts[:, 2:3]].to(torch.float64).numpy()
-    T.check_outputs(o, l, out_ref, lse_ref, w.dtype)
+    heads = ti[:, 1:2] * G + torch.arange(G)[None, :]
+    o = out_h[ti[:, 0:1], ti[:, 2:3], heads].to(torch.float64).numpy()
+    l = lse_h[ti[:, 0:1], heads, ti[:, 2:3]].to(torch.float64).numpy()
+    T.check_forward_rows(w, prob, tri, got, o, l)

@@ -53,7 +53,7 @@ def test_packed_sequences_equal_the_sequences_alone_and_the_oracle():
         ref_idx, ref_margin = prob.route_all(tri)
         ti = torch.from_numpy(tri)
         gi = got_idx.cpu()[ti[:, 1], ti[:, 2]].numpy()
-        n_diff, n_bad, n_band = T.compare_index_sets(gi, ref_idx, ref_margin)
+        n_diff, n_bad, n_band = T.compare_index_sets(gi, ref_idx, ref_margin, prob=prob, triples=tri)
         assert n_bad == 0, i
 
 

@@ -79,7 +79,7 @@ def test_route_matches_oracle(case, impl):
     got = T.gather_idx(dev.idx, tri)
     ref_idx, ref_margin = prob.route_all(tri)
     T.check_index_rows_valid(got, tri, w)
-    n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin)
+    n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin, prob=prob, triples=tri)
     print(f"[{name} impl={impl}] rows={len(tri)} differ={n_diff} outside_band={n_bad} band={n_band}")
     assert n_bad == 0
     # the margin the library reports agrees with the oracle's where sets agree
@@ -126,15 +126,7 @@ def test_forward_matches_oracle(case, impl):
     dev = T.Device(w, t, impl=impl)
     dev.forward()
     assert dev.sync_status() == 0
-    got = T.gather_idx(dev.idx, tri)
-    ref_idx, ref_margin = prob.route_all(tri)
-    T.check_index_rows_valid(got, tri, w)
-    n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin)
-    assert n_bad == 0
-    same = ~np.any(got != ref_idx, axis=1)
-    out_ref, lse_ref = prob.attend_all(tri[same], ref_idx[same])
-    out_gpu, lse_gpu = T.gather_out(dev, tri[same])
-    stats = T.check_outputs(out_gpu, lse_gpu, out_ref, lse_ref, w.dtype)
+    n_diff, n_band, stats = T.check_forward_dev(dev, prob, tri)
     print(f"[{name} impl={impl}] forward rows={len(tri)} differ={n_diff} band={n_band} "
           f"max_abs={stats[0]:.3e} mean_abs={stats[1]:.3e}")
 
@@ -172,15 +164,11 @@ def test_score_modes_match_oracle(name, mode, impl):
     got = T.gather_idx(dev.idx, tri)
     T.check_index_rows_valid(got, tri, w)
     ref_idx, ref_margin = prob.route_all(tri)
-    n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin)
+    n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin, prob=prob, triples=tri)
     assert n_bad == 0, f"{n_bad} rows differ outside the tie band"
     dev.forward()
     assert dev.sync_status() == 0
-    got = T.gather_idx(dev.idx, tri)
-    same = ~np.any(got != ref_idx, axis=1)
-    out_ref, lse_ref = prob.attend_all(tri[same], ref_idx[same])
-    out_gpu, lse_gpu = T.gather_out(dev, tri[same])
-    T.check_outputs(out_gpu, lse_gpu, out_ref, lse_ref, w.dtype)
+    T.check_forward_dev(dev, prob, tri)
 
 
 def test_dense_limit_equals_torch_causal_attention():

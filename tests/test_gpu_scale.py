@@ -34,18 +34,12 @@ def test_custom_scale(impl):
     assert P.read_status(ws) == 0
     tri = S.sample_queries(w, 120)
     got = T.gather_idx(idx, tri)
-    T.check_index_rows_valid(got, tri, w)
-    ref_idx, ref_margin = prob.route_all(tri)
-    n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin)
-    assert n_bad == 0, f"{n_bad} rows differ outside the tie band"
-    same = ~np.any(got != ref_idx, axis=1)
-    assert same.mean() > 0.9
-    out_ref, lse_ref = prob.attend_all(tri[same], ref_idx[same])
-    ti = torch.from_numpy(tri[same])
+    ti = torch.from_numpy(tri)
     G = w.Hq // w.Hkv
     o = out.view(w.B, w.N, w.Hkv, G, w.d)[ti[:, 0], ti[:, 2], ti[:, 1]].to(torch.float64).cpu().numpy()
     l = lse.view(w.B, w.Hkv, G, w.N)[ti[:, 0], ti[:, 1], :, ti[:, 2]].to(torch.float64).cpu().numpy()
-    T.check_outputs(o, l, out_ref, lse_ref, w.dtype)
+    n_diff, n_band, _ = T.check_forward_rows(w, prob, tri, got, o, l)
+    assert n_diff < 0.1 * len(tri)
     if impl == PB.IMPL_AUTO:
         rng = np.random.default_rng(3)
         dout_bits = S.f32_to_bf16_bits(rng.standard_normal(t["q"].shape).astype(np.float32))

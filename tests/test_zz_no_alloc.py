@@ -41,6 +41,32 @@ def test_static_scratch_routing_equals_workspace_routing_twice(w):
         assert torch.allclose(dev.margin[fin], ref_margin[fin], rtol=0, atol=2e-5)
 
 
+def test_static_scratch_call_on_a_large_problem_allocates_nothing_and_uses_no_second_stream():
+    """B * Hkv * N >= 131072: pisa_route would cut this problem into chunks on a library-owned second
+    stream (created on first use).  The allocation-free entry point must run it as one sequence on the
+    caller's stream: same result, and the device's free memory does not move across the call."""
+    w = S.Workload("static_large", 1, 65536, 2, 2, 128, 64, 2, 4, "bf16", 303, "iid")
+    t = S.make_inputs(w)
+    dev = T.Device(w, t)
+    assert P.workspace_bytes(dev.p, PB.OP_ROUTE) <= P.route_static_capacity()
+    dev.build_pyramid()
+    dev.route()
+    assert dev.sync_status() == 0
+    ref_idx = dev.idx.clone()
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for call in range(2):
+            dev.idx.fill_(-9)
+            stream.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
+            P.pisa_route_static(dev.p, dev.q, dev.k, dev.pyramid, dev.idx, None)
+            stream.synchronize()            # only the caller's stream: work on any other stream would not be waited for
+            free_after = torch.cuda.mem_get_info()[0]
+            assert torch.equal(dev.idx, ref_idx), f"call {call}: indices differ"
+            if call == 1:                   # the first call may look up the array's address; the second does nothing but launch
+                assert free_after == free_before
+
+
 def test_static_scratch_refuses_problems_beyond_its_capacity():
     big = P.Params(1, 131072, 32, 8, 128, 128, 2, 32)      # needs > 1 GB of routing scratch
     assert P.workspace_bytes(big, PB.OP_ROUTE) > P.route_static_capacity()
