@@ -289,7 +289,10 @@ __device__ __forceinline__ void lse_chunk(const uint32_t (&rr)[32], float sl2, f
   ssum = ssum * ex2_approx(m - mn) + ((a0 + a1) + (a2 + a3));
   m = mn;
 }
-// the same with only the first `nvalid` (>= 1) columns of the chunk taking part
+// the same with only the first `nvalid` (>= 1) columns of the chunk taking part.  The sums associate
+// exactly as in lse_chunk (four interleaved accumulators), so a full row gives bit-identical results on
+// either path: which path a row takes depends on the other rows of its tile, and the composition of a
+// tile (the order of a list's entries) varies from run to run.
 __device__ __forceinline__ void lse_chunk_masked(const uint32_t (&rr)[32], int nvalid, float sl2, float& m,
                                                  float& ssum) {
   float cm = -CUDART_INF_F;
@@ -298,11 +301,11 @@ __device__ __forceinline__ void lse_chunk_masked(const uint32_t (&rr)[32], int n
     if (j < nvalid) cm = fmaxf(cm, __uint_as_float(rr[j]));
   const float mn = fmaxf(m, cm * sl2);
   const float neg = -mn;
-  float acc = 0.f;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
   for (int j = 0; j < 32; ++j)
-    if (j < nvalid) acc += ex2_approx(fmaf(__uint_as_float(rr[j]), sl2, neg));
-  ssum = ssum * ex2_approx(m - mn) + acc;
+    if (j < nvalid) acc[j & 3] += ex2_approx(fmaf(__uint_as_float(rr[j]), sl2, neg));
+  ssum = ssum * ex2_approx(m - mn) + ((acc[0] + acc[1]) + (acc[2] + acc[3]));
   m = mn;
 }
 // first and second moments of the first `nvalid` of 32 logits about `shift` (score modes "mean" and
