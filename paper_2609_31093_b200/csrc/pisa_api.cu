@@ -496,7 +496,7 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
   g_mark_n = 0;
   stage_mark(0, s);
   kernel_mark("pyramid", s);
-  st = launch_pyramid(g, p->dtype, k, pyr, s);
+  st = launch_pyramid(g, p->dtype, k, pyr, (int32_t*)ws, s);
   if (st != PISA_OK) return st;
   stage_mark(1, s);
   if (pl.n == 1) {
@@ -638,7 +638,7 @@ int pisa_build_pyramid(const pisa_params_t* p, const void* k, void* pyramid, voi
   int st = resolve(p, &g);
   if (st != PISA_OK) return st;
   if (k == nullptr || pyramid == nullptr || misaligned(k) || misaligned32(pyramid)) return PISA_ERR_INVALID_ARG;
-  return launch_pyramid(g, p->dtype, k, pyramid, (cudaStream_t)stream);
+  return launch_pyramid(g, p->dtype, k, pyramid, nullptr, (cudaStream_t)stream);
 }
 
 int pisa_route(const pisa_params_t* p, const void* q, const void* k, const void* pyramid, int32_t* idx,

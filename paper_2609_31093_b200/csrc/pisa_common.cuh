@@ -41,7 +41,8 @@ int resolve(const pisa_params_t* p, Geometry* g);                // validates; r
 size_t align_up(size_t x, size_t a);
 
 // launchers (each returns a pisa_status; errors come from cudaGetLastError after the launch)
-int launch_pyramid(const Geometry& g, int dtype, const void* k, void* pyramid, cudaStream_t s);
+// status (nullable): the status word a bounded wait reports into
+int launch_pyramid(const Geometry& g, int dtype, const void* k, void* pyramid, int32_t* status, cudaStream_t s);
 int launch_route_simt(const Geometry& g, int dtype, const void* q, const void* k, const void* pyramid,
                       int32_t* idx, float* margin, cudaStream_t s);
 // stage 1 of the two-stage schedule (needs L >= 2): kept level-2 nodes [B,Hkv,N,K] (ascending,

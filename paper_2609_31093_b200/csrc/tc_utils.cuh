@@ -1,6 +1,6 @@
 // sm_100a primitives used by the tensor-core kernels: mbarrier with bounded waits, tcgen05
 // (TMEM allocation, UMMA issue/commit, TMEM loads), shared-memory matrix descriptors for the
-// 128-byte-swizzled canonical layouts, cp.async staging and bulk reductions.  Inline PTX only.
+// 128-byte-swizzled canonical layouts, cp.async staging and TMA tile loads.  Inline PTX only.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -194,34 +194,30 @@ __device__ __forceinline__ void st_shared_zero16(uint32_t saddr) {
 }
 
 // ---------------------------------------------------------------- TMA (tiled tensor copies)
-
-// 4-D tiled load global -> shared memory of this CTA; completes `bytes` of transaction on `bar`.
-// `tmap` points at a CUtensorMap (kernel parameter / constant / global memory, 64-byte aligned).
+//
+// Tile loads global -> shared memory of THIS CTA (no cluster multicast); the bytes complete as a
+// transaction on `bar`.  `tmap` points at a CUtensorMap (a __grid_constant__ kernel parameter).
+// The innermost coordinate times the element size must be a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_3d(uint32_t sdst, const void* tmap, uint64_t* bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(sdst), "l"(tmap), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
 __device__ __forceinline__ void tma_load_4d(uint32_t sdst, const void* tmap, uint64_t* bar, int c0, int c1, int c2,
                                             int c3) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      "cp.async.bulk.tensor.4d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(sdst), "l"(tmap), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
 }
-// announce `bytes` of pending transaction on `bar` without arriving
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+// one arrival on `bar` that also announces `bytes` of pending transaction
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-
-// ---------------------------------------------------------------- bulk reduction to global
-
-// global[dst .. dst+bytes) += shared[src .. src+bytes) as fp32 adds, performed by the copy engine
-// at the L2.  Both addresses 16-byte aligned, bytes a multiple of 16.
-__device__ __forceinline__ void bulk_reduce_add_f32(void* gdst, uint32_t ssrc, uint32_t bytes) {
-  asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(gdst), "r"(ssrc),
-               "r"(bytes)
-               : "memory");
+__device__ __forceinline__ void tma_prefetch_desc(const void* tmap) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// all of this thread's bulk groups have finished READING their shared-memory source
-__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 }  // namespace tc
 }  // namespace pisa
