@@ -945,6 +945,12 @@ int pisa_flat_select(const pisa_params_t* p, const void* q, const void* pyramid,
   if (ws_bytes < kStatusBytes) return PISA_ERR_WORKSPACE_TOO_SMALL;
   st = clear_status(ws, (cudaStream_t)stream);
   if (st != PISA_OK) return st;
+  if (p->impl != PISA_IMPL_SIMT && flat_tc_supported(g, p->dtype)) {
+    kernel_mark("flat_tc", (cudaStream_t)stream);
+    st = launch_flat_tc(g, q, pyramid, idx, (int32_t*)ws, (cudaStream_t)stream);
+    kernel_mark("end", (cudaStream_t)stream);
+    return st;
+  }
   return launch_flat_simt(g, p->dtype, q, pyramid, idx, (cudaStream_t)stream);
 }
 

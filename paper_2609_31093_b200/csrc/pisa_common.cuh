@@ -57,6 +57,10 @@ int launch_bsa_simt(const Geometry& g, int dtype, const void* q, const void* k, 
                     const int32_t* idx, void* out, float* lse, cudaStream_t s);
 int launch_flat_simt(const Geometry& g, int dtype, const void* q, const void* pyramid, int32_t* idx,
                      cudaStream_t s);
+// the same selection on tcgen05 (bf16, d in {64, 128}); status: the workspace's status word
+bool flat_tc_supported(const Geometry& g, int dtype);
+int launch_flat_tc(const Geometry& g, const void* q, const void* pyramid, int32_t* idx, int32_t* status,
+                   cudaStream_t s);
 // per-head softmax denominators of the selected leaves, float [B,Hq,N,K] (exact fp32, any shape)
 int launch_sel_lse_simt(const Geometry& g, int dtype, const void* q, const void* k, const int32_t* idx,
                         float* sel_lse, int32_t* status, cudaStream_t s);

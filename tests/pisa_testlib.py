@@ -188,6 +188,32 @@ def check_index_rows_valid(idx_gpu: np.ndarray, triples: np.ndarray, w: S.Worklo
             assert f in sel, (p, row)
 
 
+def flat_admissible(prob: O.Problem, b: int, h: int, p: int, got_leaves, band=TIE_BAND):
+    """Flat selection (Sec. 3.1): `got_leaves` may differ from the oracle's set only by swaps between leaves
+    whose oracle scores lie within `band` RELATIVE of each other across the cut (the scores are sums of
+    G probabilities, far below one, so the band is taken relative to the score itself)."""
+    C, K = prob.C, prob.K
+    c = p // C
+    got = sorted(int(x) for x in got_leaves)
+    if c + 1 <= K:
+        return got == list(range(c + 1))
+    F = O.forced_nodes(1, c, 2)
+    if len(got) != K or len(set(got)) != K or not set(F) <= set(got) or got[-1] > c or got[0] < 0:
+        return False
+    qg = prob.q_group(b, h, p)
+    lv1 = prob.head(b, h)[2][1]
+    s = (qg @ lv1[:c + 1].T) * prob.scale
+    s = s - s.max(axis=1, keepdims=True)
+    w = np.exp(s)
+    u = (w / w.sum(axis=1, keepdims=True)).sum(axis=0)
+    kept = [i for i in got if i not in F]
+    dropped = [i for i in range(c + 1) if i not in F and i not in got]
+    if not dropped:
+        return True
+    worst_kept, best_dropped = min(u[kept]), max(u[dropped])
+    return (best_dropped - worst_kept) / abs(best_dropped) <= band
+
+
 STRICT_RANGE = 2.56      # below this magnitude a bf16 ulp is at most 2e-2 / 1.28: the flat bounds apply as stated
 
 

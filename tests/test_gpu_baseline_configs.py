@@ -74,3 +74,24 @@ def test_full_size_forward_sampled_parity(name):
     dev.forward()
     torch.cuda.synchronize()
     assert torch.equal(first, dev.idx)
+
+
+@pytest.mark.parametrize("n", [8192, 32768, 131072])
+def test_flat_selector_at_sweep_sizes(n):
+    """The flat reference point (tcgen05 kernel) at the scaling sweep's sizes against the oracle's flat
+    selection on sampled rows; every row structurally valid."""
+    w = S.sweep_workload(n)
+    t = S.make_inputs(w)
+    dev = T.Device(w, t)
+    dev.build_pyramid()
+    dev.flat()
+    assert dev.sync_status() == 0
+    _all_rows_valid(dev, w)
+    tri = S.sample_queries(w, 256)
+    cprob, prob = T.oracle_problem_c(w, t), T.oracle_problem(w, t)
+    ref_idx, _ = cprob.flat_mean_all(tri)
+    got = T.gather_idx(dev.idx, tri)
+    differ = np.nonzero(np.any(got != ref_idx, axis=1))[0]
+    bad = [int(s_) for s_ in differ if not T.flat_admissible(prob, *(int(x) for x in tri[s_]), got[s_])]
+    print(f"[flat cfg5_{n}] rows={len(tri)} differ={len(differ)} not_explained_by_near_ties={len(bad)}")
+    assert not bad

@@ -131,20 +131,27 @@ def test_forward_matches_oracle(case, impl):
           f"max_abs={stats[0]:.3e} mean_abs={stats[1]:.3e}")
 
 
-def test_flat_select_matches_oracle(case):
+@pytest.mark.parametrize("impl", [PB.IMPL_SIMT, PB.IMPL_AUTO])
+def test_flat_select_matches_oracle(case, impl):
+    """Flat selection on the exact-fp32 kernel and (bf16, d in {64, 128}) on the tcgen05 kernel."""
     name, w, t, prob, tri = case
     if len(tri) > 1500:
         tri = tri[np.random.default_rng(2).choice(len(tri), 1500, replace=False)]
-    dev = T.Device(w, t)
+    dev = T.Device(w, t, impl=impl)
     dev.load_oracle_pyramid(prob.pyramid())
     dev.flat()
     assert dev.sync_status() == 0
     got = T.gather_idx(dev.idx, tri)
     ref_idx, ref_margin = prob.flat_mean_all(tri)
     T.check_index_rows_valid(got, tri, w)
-    n_diff, n_bad, n_band = T.compare_index_sets(got, ref_idx, ref_margin)
-    print(f"[{name}] flat rows={len(tri)} differ={n_diff} outside_band={n_bad} band={n_band}")
-    assert n_bad == 0
+    differ = np.nonzero(np.any(got != ref_idx, axis=1))[0]
+    bad = [int(s_) for s_ in differ if not T.flat_admissible(prob, *(int(x) for x in tri[s_]), got[s_])]
+    print(f"[{name} impl={impl}] flat rows={len(tri)} differ={len(differ)} not_explained_by_near_ties={len(bad)}")
+    assert not bad, (tri[bad[:4]], got[bad[:4]], ref_idx[bad[:4]])
+    first = dev.idx.clone()                      # deterministic
+    dev.flat()
+    torch.cuda.synchronize()
+    assert torch.equal(first, dev.idx)
 
 
 @pytest.mark.parametrize("impl", [PB.IMPL_SIMT, PB.IMPL_AUTO])
