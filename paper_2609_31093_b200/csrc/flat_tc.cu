@@ -63,7 +63,96 @@ __device__ __forceinline__ int flat_chunks(const Geometry& geo, int pair, int to
 
 }  // namespace
 
-template <int D>
+// One pass-1 update of a row's online (maximum, denominator), base 2, over the first nv of 32 logits.
+__device__ __forceinline__ void flat_pass1(const uint32_t (&x)[32], int nv, float sl2, float& m, float& l) {
+  float cm = -CUDART_INF_F;
+#pragma unroll
+  for (int j = 0; j < 32; ++j)
+    if (j < nv) cm = fmaxf(cm, __uint_as_float(x[j]));
+  const float mn = fmaxf(m, cm * sl2);
+  float acc4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int j = 0; j < 32; ++j)
+    if (j < nv) acc4[j & 3] += ex2f(fmaf(__uint_as_float(x[j]), sl2, -mn));
+  l = l * ex2f(m - mn) + ((acc4[0] + acc4[1]) + (acc4[2] + acc4[3]));
+  m = mn;
+}
+
+// Pass 2 on one 32-column group: normalised scores of this row, summed over the token's G = 2^LG heads by a
+// reduce-scatter among its lanes (lane `head` ends up owning 32 / G consecutive columns, starting at
+// col_off), then the owned scores that beat the token's current threshold go through its Top-K' list,
+// the token's lanes taking turns.  list_val / list_idx: the token's list; slot 32 holds the threshold /
+// (count | position of the minimum << 8).
+template <int LG>
+__device__ __forceinline__ void flat_pass2(const uint32_t (&x)[32], int nv, float sl2, float m2, int head, int leaf_first,
+                                           int leaf_last_cand, bool scored, int Kp, float* list_val, int* list_idx) {
+  constexpr int G = 1 << LG, OWN = 32 >> LG;
+  float v[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) v[j] = (j < nv) ? ex2f(fmaf(__uint_as_float(x[j]), sl2, -m2)) : 0.f;
+#pragma unroll
+  for (int s = 0; s < LG; ++s) {
+    const int half = 16 >> s;
+    const bool up = ((head >> s) & 1) != 0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      if (j < half) {
+        const float keep = up ? v[j + half] : v[j];
+        const float send = up ? v[j] : v[j + half];
+        v[j] = keep + __shfl_xor_sync(0xffffffffu, send, 1 << s);
+      }
+    }
+  }
+  // candidates among the owned columns: leaves 1 .. c - 2 that beat the threshold as it stands now (it only
+  // rises, so this is a superset of what will be inserted)
+  unsigned mask = 0;
+  if (scored) {
+    const int meta = list_idx[32];
+    const bool full = (meta & 0xFF) >= Kp;
+    const float tau = list_val[32];
+#pragma unroll
+    for (int j = 0; j < OWN; ++j) {
+      const int leaf = leaf_first + j;
+      if (leaf >= 1 && leaf <= leaf_last_cand && (!full || v[j] > tau)) mask |= 1u << j;
+    }
+  }
+  if (__all_sync(0xffffffffu, mask == 0)) return;
+#pragma unroll 1
+  for (int turn = 0; turn < G; ++turn) {
+    if (head == turn && mask != 0) {
+      const int meta = list_idx[32];
+      int cnt = meta & 0xFF, pos = meta >> 8;
+      float tau = list_val[32];
+      while (mask != 0) {
+        const int jj = __ffs(mask) - 1;
+        mask &= mask - 1;
+        float u = v[0];
+#pragma unroll
+        for (int j = 1; j < OWN; ++j) u = (j == jj) ? v[j] : u;
+        if (cnt < Kp || u > tau) {
+          const int at = (cnt < Kp) ? cnt : pos;
+          list_val[at] = u;
+          list_idx[at] = leaf_first + jj;
+          if (cnt < Kp) ++cnt;
+          if (cnt == Kp) {                       // the list is full: find what to replace next
+            tau = CUDART_INF_F;
+            int ileaf = -1;
+            for (int e = 0; e < Kp; ++e) {
+              const float ve = list_val[e];
+              const int ie = list_idx[e];
+              if (ve < tau || (ve == tau && ie > ileaf)) { tau = ve; pos = e; ileaf = ie; }
+            }
+          }
+        }
+      }
+      list_idx[32] = cnt | (pos << 8);
+      list_val[32] = tau;
+    }
+    __syncwarp();
+  }
+}
+
+template <int D, int LG>
 __global__ void __launch_bounds__(kFlatThreads, 1)
 flat_tc_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                FlatArgs a) {
@@ -74,7 +163,7 @@ flat_tc_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, const __g
   uint8_t* sQ = smem;                              // [2 tiles][TILE]
   uint8_t* sB = smem + 2 * TILE;                   // [stages][TILE]
   float* l_val = reinterpret_cast<float*>(sB + a.stages * TILE);       // [tokens per item][kListStride]
-  const int G = geo.G, lgG = 31 - __clz(G), tpt = 128 >> lgG, tok_per_item = 2 * tpt;
+  constexpr int G = 1 << LG, lgG = LG, tpt = 128 >> LG, tok_per_item = 2 * tpt;
   int* l_idx = reinterpret_cast<int*>(l_val + tok_per_item * kListStride);
   __shared__ uint64_t q_full, q_empty, b_full[4], b_empty[4], t_full[2], t_empty[2];
   __shared__ uint32_t tmem_slot;
@@ -197,88 +286,27 @@ flat_tc_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, const __g
         if (st == nch) m2 = m + log2f(l);            // pass 2: p = 2^(x - m) / l = 2^(x - m2)
         uint32_t ra[32], rb[32];
         tmem_ld_32x32(t_base + (uint32_t)(buf * 256), ra);
+#pragma unroll 1
+        for (int c0 = 0; c0 < kChunk; c0 += 64) {            // two 32-column groups per round (ra, then rb)
 #pragma unroll
-        for (int c0 = 0; c0 < kChunk; c0 += 32) {
-          uint32_t (&cur)[32] = ((c0 >> 5) & 1) ? rb : ra;
-          uint32_t (&nxt)[32] = ((c0 >> 5) & 1) ? ra : rb;
-          tmem_ld_wait();
-          if (c0 + 32 < kChunk) {
-            tmem_ld_32x32(t_base + (uint32_t)(buf * 256 + c0 + 32), nxt);
-          } else {
-            tcgen05_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&t_empty[buf]);       // the accumulator has been read out
-          }
-          const int leaf0 = ch * kChunk + c0;                // leaf of column 0 of this group
-          const int nv = scored ? max(0, min(32, c_row + 1 - leaf0)) : 0;   // eligible columns: leaves <= c_row
-          if (st < nch) {
-            // pass 1: online maximum and denominator (base 2) over the eligible leaves
-            if (nv > 0) {
-              float cm = -CUDART_INF_F;
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (j < nv) cm = fmaxf(cm, __uint_as_float(cur[j]));
-              const float mn = fmaxf(m, cm * sl2);
-              float acc4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (j < nv) acc4[j & 3] += ex2f(fmaf(__uint_as_float(cur[j]), sl2, -mn));
-              l = l * ex2f(m - mn) + ((acc4[0] + acc4[1]) + (acc4[2] + acc4[3]));
-              m = mn;
-            }
-          } else {
-            // pass 2: normalised scores, summed over the token's G heads by a reduce-scatter among its lanes
-            if (__all_sync(0xffffffffu, nv == 0)) continue;
-            float v[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = (j < nv) ? ex2f(fmaf(__uint_as_float(cur[j]), sl2, -m2)) : 0.f;
-#pragma unroll
-            for (int s = 0; s < 4; ++s) {
-              if (s < lgG) {
-                const int half = 16 >> s;
-                const bool up = ((head >> s) & 1) != 0;
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                  if (j < half) {
-                    const float keep = up ? v[j + half] : v[j];
-                    const float send = up ? v[j] : v[j + half];
-                    v[j] = keep + __shfl_xor_sync(0xffffffffu, send, 1 << s);
-                  }
-                }
-              }
-            }
-            // v[0 .. n_own) = grouped scores of leaves leaf0 + col_off + j; each of the token's lanes takes its turn
-            for (int turn = 0; turn < G; ++turn) {
-              if (scored && head == turn) {
-                int meta = my_idx[32];
-                int cnt = meta & 0xFF, pos = meta >> 8;
-                float tau = my_val[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                  if (j < n_own) {
-                    const int leaf = leaf0 + col_off + j;
-                    const float u = v[j];
-                    if (leaf >= 1 && leaf <= c_row - 2 && (cnt < Kp || u > tau)) {
-                      const int at = (cnt < Kp) ? cnt : pos;
-                      my_val[at] = u;
-                      my_idx[at] = leaf;
-                      if (cnt < Kp) ++cnt;
-                      if (cnt == Kp) {                       // the list is full: find what to replace next
-                        tau = CUDART_INF_F;
-                        int ileaf = -1;
-                        for (int e = 0; e < Kp; ++e) {
-                          const float ve = my_val[e];
-                          const int ie = my_idx[e];
-                          if (ve < tau || (ve == tau && ie > ileaf)) { tau = ve; pos = e; ileaf = ie; }
-                        }
-                      }
-                    }
-                  }
-                }
-                my_idx[32] = cnt | (pos << 8);
-                my_val[32] = tau;
-              }
+          for (int hh = 0; hh < 2; ++hh) {
+            uint32_t (&cur)[32] = hh ? rb : ra;
+            uint32_t (&nxt)[32] = hh ? ra : rb;
+            const int cc0 = c0 + hh * 32;
+            tmem_ld_wait();
+            if (cc0 + 32 < kChunk) {
+              tmem_ld_32x32(t_base + (uint32_t)(buf * 256 + cc0 + 32), nxt);
+            } else {
+              tcgen05_fence_before_sync();
               __syncwarp();
+              if (lane == 0) mbar_arrive(&t_empty[buf]);     // the accumulator has been read out
+            }
+            const int leaf0 = ch * kChunk + cc0;             // leaf of column 0 of this group
+            const int nv = scored ? max(0, min(32, c_row + 1 - leaf0)) : 0;   // eligible columns: leaves <= c_row
+            if (st < nch) {
+              if (nv > 0) flat_pass1(cur, nv, sl2, m, l);
+            } else if (!__all_sync(0xffffffffu, nv == 0)) {
+              flat_pass2<LG>(cur, nv, sl2, m2, head, leaf0 + col_off, c_row - 2, scored, Kp, my_val, my_idx);
             }
           }
         }
@@ -330,8 +358,8 @@ bool flat_tc_supported(const Geometry& g, int dtype) {
   return tma::encoder() != nullptr;
 }
 
-template <int D>
-static int launch_flat_tc_d(const Geometry& g, const void* q, const void* pyramid, int32_t* idx, int32_t* status,
+template <int D, int LG>
+static int launch_flat_tc_dg(const Geometry& g, const void* q, const void* pyramid, int32_t* idx, int32_t* status,
                             cudaStream_t s) {
   const int tpt = 128 / g.G, tok_per_item = 2 * tpt;
   constexpr int TILE = (D / 64) * 128 * 128;
@@ -360,11 +388,24 @@ static int launch_flat_tc_d(const Geometry& g, const void* q, const void* pyrami
     const uint32_t box[3] = {64u, (uint32_t)kChunk, 1u};
     if (!tma::make_map(&tm_k, 2, 3, lvl1, dims, str, box, true)) return PISA_ERR_UNSUPPORTED;
   }
-  cudaError_t e = cudaFuncSetAttribute(flat_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(flat_tc_kernel<D, LG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("flat_tc attr", e); return PISA_ERR_CUDA; }
   const int grid = a.n_items < num_sms() ? a.n_items : num_sms();
-  flat_tc_kernel<D><<<grid, kFlatThreads, smem, s>>>(g, tm_q, tm_k, a);
+  flat_tc_kernel<D, LG><<<grid, kFlatThreads, smem, s>>>(g, tm_q, tm_k, a);
   return check_launch("flat_tc");
+}
+
+template <int D>
+static int launch_flat_tc_d(const Geometry& g, const void* q, const void* pyramid, int32_t* idx, int32_t* status,
+                            cudaStream_t s) {
+  switch (g.G) {
+    case 1: return launch_flat_tc_dg<D, 0>(g, q, pyramid, idx, status, s);
+    case 2: return launch_flat_tc_dg<D, 1>(g, q, pyramid, idx, status, s);
+    case 4: return launch_flat_tc_dg<D, 2>(g, q, pyramid, idx, status, s);
+    case 8: return launch_flat_tc_dg<D, 3>(g, q, pyramid, idx, status, s);
+    case 16: return launch_flat_tc_dg<D, 4>(g, q, pyramid, idx, status, s);
+    default: return PISA_ERR_UNSUPPORTED;
+  }
 }
 
 int launch_flat_tc(const Geometry& g, const void* q, const void* pyramid, int32_t* idx, int32_t* status,
