@@ -32,10 +32,17 @@ import pisa_synth as S  # noqa: E402
 METRIC = "pisa_fwd_tokens_per_s_128k_ctx"
 UNIT = "tokens/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per selected (token, block) pair, from the ncu captures
-# summarised under profiles/ (B=1 Hq=8 Hkv=2 d=128 N=65536 C=128 g=2 K=32: 4.19 M pairs per launch)
-DRAM_BYTES_PER_PAIR = {"leaf_lse_tiles": (208.604928e6 + 106.822144e6) / 4194304.0,
-                       "attention_tiles": (1195.880e6 + 912.732416e6) / 4194304.0}
+
+
+def dram_bytes_per_pair() -> dict:
+    """dram__bytes_read.sum + dram__bytes_write.sum per selected (token, block) pair of the two tile
+    kernels, read from the file that is written with the ncu captures (profiles/)."""
+    try:
+        d = json.load(open(os.path.join(ROOT, "profiles", "dram_bytes_per_pair.json")))
+        n = float(d["pairs_per_launch"])
+        return {k_: (v_["dram_bytes_read"] + v_["dram_bytes_write"]) / n for k_, v_ in d.items() if isinstance(v_, dict)}
+    except Exception:
+        return {}
 
 
 def get_workload(name: str) -> S.Workload:
@@ -158,34 +165,63 @@ class ClockSampler:
 
 # ------------------------------------------------------------------ CPU oracle legs
 
-def oracle_sample_rate(w: S.Workload, tensors: dict, n_queries: int, seed: int = 0):
-    """Times the oracle (as it stands) on one KV head's pyramid plus `n_queries` sampled queries of
-    that head (routing + attention for the G heads of the group); returns the whole-workload
-    tokens/s this extrapolates to, the seconds spent and a description of the sample."""
-    from oracle import pisa_oracle as O
-    try:
-        from threadpoolctl import threadpool_limits
-        ctx = threadpool_limits(limits=1)
-    except Exception:  # pragma: no cover
-        import contextlib
-        ctx = contextlib.nullcontext()
+def oracle_sample_rate(w: S.Workload, tensors: dict, n_queries: int, seed: int = 0, threads: int = 0):
+    """Times the compiled oracle (oracle/pisa_oracle_c.c, as it stands) on one (batch, KV head) unit: its
+    pyramid in full plus `n_queries` sampled query positions of it (routing + attention of the group's
+    heads), on `threads` host threads (0 = all the box has).  Returns the whole-workload tokens/s this
+    extrapolates to, the seconds spent, the threads used and a description of the sample."""
+    from oracle import pisa_oracle_c as OC
     rng = np.random.default_rng(seed)
     h = int(rng.integers(0, w.Hkv))
     ps = np.sort(rng.integers(0, w.N, size=n_queries))
-    with ctx:
-        prob = O.Problem(tensors["q"], tensors["k"], tensors["v"], C=w.C, g=w.g, K=w.K, dtype=w.dtype)
-        t0 = time.perf_counter()
-        prob.head(0, h)                                   # converts the head's keys and pools its pyramid
-        t1 = time.perf_counter()
-        tri = np.stack([np.zeros_like(ps), np.full_like(ps, h), ps], axis=1)
-        idx, _ = prob.route_all(tri)
-        prob.attend_all(tri, idx)
-        t2 = time.perf_counter()
-    per_head = (t1 - t0) + (t2 - t1) / n_queries * w.N
-    total = per_head * w.B * w.Hkv
-    return (w.B * w.N) / total, (t2 - t0), (f"pyramid of 1 of {w.B * w.Hkv} (batch, KV head) units in full + {n_queries} "
-                                           f"uniformly sampled query positions of it (route + attention of its "
-                                           f"{w.Hq // w.Hkv} heads), scaled by N/{n_queries} and by the unit count")
+    prob = OC.CProblem(tensors["q"], tensors["k"], tensors["v"], C=w.C, g=w.g, K=w.K, dtype=w.dtype, threads=threads)
+    t0 = time.perf_counter()
+    prob.unit(0, h)                                   # widens the unit's keys and pools its pyramid
+    t1 = time.perf_counter()
+    tri = np.stack([np.zeros_like(ps), np.full_like(ps, h), ps], axis=1)
+    idx, _ = prob.route_all(tri)
+    prob.attend_all(tri, idx)
+    t2 = time.perf_counter()
+    per_unit = (t1 - t0) + (t2 - t1) / n_queries * w.N
+    total = per_unit * w.B * w.Hkv
+    return (w.B * w.N) / total, (t2 - t0), prob.threads, (
+        f"compiled oracle, {prob.threads} thread(s): pyramid of 1 of {w.B * w.Hkv} (batch, KV head) units in full + "
+        f"{n_queries} uniformly sampled query positions of it (route + attention of its {w.Hq // w.Hkv} heads), "
+        f"scaled by N/{n_queries} and by the unit count")
+
+
+def cpu_baseline_leg(w: S.Workload, tensors: dict, n_queries: int) -> dict:
+    """The oracle on the machine's host cores: all cores on `n_queries` sampled positions, one core on a quarter."""
+    val, secs, cores, sample = oracle_sample_rate(w, tensors, n_queries)
+    val1, secs1, _, _ = oracle_sample_rate(w, tensors, max(64, n_queries // 4), threads=1)
+    return {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample, "seconds": secs,
+            "host_cores": os.cpu_count(), "value_1_thread": val1, "seconds_1_thread": secs1}
+
+
+def parity_of_timed_buffers(w: S.Workload, tensors: dict, idx, out, lse, per_unit: int = 64) -> dict:
+    """Checks the buffers a timed run left behind against the oracle on sampled rows (at least 256 at the
+    headline shape): index sets (a differing row is excused only if the oracle's cut margin of that row is
+    inside the 1e-4 tie band), then outputs and denominators of every sampled row against the oracle's
+    attention on the sets the GPU selected.  idx / out / lse: torch tensors (device or host)."""
+    import torch
+    from oracle import pisa_oracle_c as OC
+    tri = S.sample_queries(w, per_unit)
+    prob = OC.CProblem(tensors["q"], tensors["k"], tensors["v"], C=w.C, g=w.g, K=w.K, dtype=w.dtype)
+    ref_idx, margin = prob.route_all(tri)
+    t = torch.from_numpy(tri).to(idx.device)
+    got = idx[t[:, 0], t[:, 1], t[:, 2]].cpu().numpy()
+    differ = np.any(got != ref_idx, axis=1)
+    out_ref, lse_ref = prob.attend_all(tri, got)
+    G = w.Hq // w.Hkv
+    heads = t[:, 1:2] * G + torch.arange(G, device=idx.device)[None, :]
+    o = out[t[:, 0:1], t[:, 2:3], heads].to(torch.float64).cpu().numpy()
+    l = lse[t[:, 0:1], heads, t[:, 2:3]].to(torch.float64).cpu().numpy()
+    err = np.abs(o - out_ref)
+    return {"rows": int(len(tri)), "rows_differ": int(differ.sum()), "rows_differ_outside_tie_band": int((differ & (margin > 1e-4)).sum()),
+            "rows_in_tie_band": int((margin <= 1e-4).sum()), "out_max_abs": float(err.max()), "out_mean_abs": float(err.mean()),
+            "lse_max_abs": float(np.abs(l - lse_ref).max()),
+            "ok": bool((differ & (margin > 1e-4)).sum() == 0 and err.max() <= (2e-2 if w.dtype == "bf16" else 1e-4)
+                       and err.mean() <= (2e-3 if w.dtype == "bf16" else 1e-4))}
 
 
 def run_reference(args):
@@ -199,8 +235,9 @@ def run_reference(args):
         oracle_sample_rate(w, tensors, max(4, nq // 8), seed=99)
     t0 = time.perf_counter()
     rates = []
+    cores = 1
     for s in range(args.steps):
-        r, _, sample = oracle_sample_rate(w, tensors, nq, seed=s)
+        r, _, cores, sample = oracle_sample_rate(w, tensors, nq, seed=s)
         rates.append(r)
     wall = time.perf_counter() - t0
     value = float(len(rates) / sum(1.0 / r for r in rates))
@@ -209,7 +246,7 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": wall / max(1, args.steps) * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": describe(w)},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
@@ -345,6 +382,7 @@ def run_ours(args):
     arena = PB.alloc_workspace(p, PB.OP_FORWARD_HOST)
     out_h = torch.empty(q.shape, dtype=tdt).pin_memory()
     lse_h = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
+    idx_h = torch.empty(idx.shape, dtype=torch.int32).pin_memory()
     e2e_steps = max(0, min(args.steps, args.e2e_steps))
     e2e_ms = float("nan")
     if e2e_steps > 0:
@@ -398,16 +436,22 @@ def run_ours(args):
     else:
         roof = {"kernel": dom, "bound": "tensor", "achieved": work / t_dom / 1e12, "peak": tens_peak,
                 "unit": "TFLOP/s"}
+    # `achieved` / `frac`: the kernel ALONE on the GPU (the whole problem as one launch, chunking off), which
+    # is what a per-kernel roofline means; the launch spans inside the timed region, where a launch shares
+    # the SMs with the other stream's kernels, are kept beside them as in_step_*
+    roof["in_step_achieved"] = roof["achieved"]
+    roof["in_step_frac"] = roof["achieved"] / roof["peak"]
+    roof["achieved"] = work / t_alone / (1e9 if bound == "hbm" else 1e12)
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["peak_source"] = peak_src + (" (sustained bf16, kernel timed inside a long step)" if bound == "tensor" else "")
     n_launch = max(1, launches_of.get(dom, 1))                    # one launch per chunk
     roof["launch_ms"] = t_dom * 1e3 / n_launch                    # average launch; achieved = (work / n) / this
     roof["launches_per_step"] = n_launch
     roof["alone_ms"] = t_alone * 1e3                               # the whole problem as one launch, GPU to itself
-    roof["alone_frac"] = work / t_alone / ((hbm_peak * 1e9) if bound == "hbm" else (tens_peak * 1e12))
+    roof["frac_of_burst_peak"] = (work / t_alone / 1e12 / peaks.get("bf16_tflops", 1590.0)) if bound == "tensor" else None
     # DRAM bytes per launch from the ncu capture of a smaller case of the same kernel (summary under
     # profiles/), scaled by the (token, block) pairs a launch processes: traffic grows with the pairs
-    per_pair = DRAM_BYTES_PER_PAIR.get(dom)
+    per_pair = dram_bytes_per_pair().get(dom)
     pairs = {"leaf_lse_tiles": wc["sel_pairs"], "attention_tiles": wc["sel_pairs"]}.get(dom)
     roof["traffic"] = (per_pair * pairs / n_launch) if (per_pair and pairs and w.dtype == "bf16") else None
     # The two tile kernels are limited by what L2 can gather and reduce, not by the tensor pipe: report
@@ -422,6 +466,11 @@ def run_ours(args):
         b_, w_ = algo[k_]
         roofs[k_] = {"ms": t_, ("gbs" if b_ == "hbm" else "tflops"): w_ / (t_ * 1e-3) / (1e9 if b_ == "hbm" else 1e12),
                      "frac": w_ / (t_ * 1e-3) / ((hbm_peak * 1e9) if b_ == "hbm" else (tens_peak * 1e12))}
+        if k_ == "route_stage1":
+            # gathered per-token products on warp-level MMAs: bound by instruction issue (ncu: about 70 % of the
+            # issue slots busy), not by the tensor pipe -- a fraction of the tensor peak would say nothing
+            roofs[k_]["bound"] = "instruction issue"
+            del roofs[k_]["frac"]
     # stage times from the kernels-alone pass (in the timed region the stages of different chunks overlap)
     t_pyr = kernels.get("pyramid", stage[0])
     t_route = sum(kernels.get(n_, 0.0) for n_ in ("route_stage1", "invert_by_parent", "leaf_lse_tiles", "final_topk",
@@ -436,9 +485,15 @@ def run_ours(args):
         "whole_step_hbm_min_gbs": wc["hbm_min_bytes"] / (ms / args.steps * 1e-3) / 1e9,
     }
     cpu = None
+    parity = None
     if world == 1 and not args.no_cpu_baseline:
-        val, secs, sample = oracle_sample_rate(w, tensors, args.ref_queries)
-        cpu = {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample, "seconds": secs}
+        cpu = cpu_baseline_leg(w, tensors, args.ref_queries)
+    if world == 1 and not args.no_parity:
+        # the buffers the timed region and the end-to-end region left behind, against the oracle
+        parity = {"device_buffers": parity_of_timed_buffers(w, tensors, idx, out, lse)}
+        if e2e_steps > 0:
+            P.pisa_forward_host(p, qh, kh, vh, out_h, lse_h, idx_h, arena)
+            parity["host_buffers"] = parity_of_timed_buffers(w, tensors, idx_h, out_h, lse_h)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
@@ -446,7 +501,7 @@ def run_ours(args):
         "config": {"workload": describe(w0), "path": args.path,
                    "l2": f"inputs larger than L2 (q {q.numel() * es / 1e6:.0f} MB, k+v {2 * k.numel() * es / 1e6:.0f} MB)",
                    "replicas": world},
-        "stages": stages, "kernels_ms": kernels, "kernels_ms_spans_in_timed_region": spans, "kernel_rooflines": roofs, "roofline": roof, "cpu_baseline": cpu,
+        "stages": stages, "kernels_ms": kernels, "kernels_ms_spans_in_timed_region": spans, "kernel_rooflines": roofs, "roofline": roof, "cpu_baseline": cpu, "parity": parity,
         "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps,
                 "h2d_bytes_per_step": int((q.numel() + 2 * k.numel()) * es),
                 "d2h_bytes_per_step": int(out.numel() * es + lse.numel() * 4)},
@@ -766,7 +821,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
-    ap.add_argument("--ref-queries", type=int, default=1024)
+    ap.add_argument("--ref-queries", type=int, default=4096,
+                    help="sampled query positions the CPU oracle is timed on (all cores; a quarter of them on one core)")
+    ap.add_argument("--no-parity", action="store_true", help="skip the oracle check of the timed buffers")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--forward-chunks", type=int, default=0,

@@ -109,17 +109,38 @@ def test_backward_at_the_headline_size_sampled_rows_and_identities():
     assert bool(((dv_sum - do_sum).abs() <= 2.0 ** -8 * scale_v).all())
     dk_sum = dk.double().sum(dim=1)
     assert bool((dk_sum.abs() <= 2.0 ** -8 * dk.double().abs().sum(dim=1)).all())
-    # sampled rows
-    tri = S.sample_queries(w, 10)
-    prob = T.oracle_problem(w, t)
+    # sampled dq rows (the compiled oracle: 256 positions per KV head)
+    tri = S.sample_queries(w, 256)
+    prob = T.oracle_problem_c(w, t)
     ti = torch.from_numpy(tri).cuda()
     idx_rows = dev.idx[ti[:, 0], ti[:, 1], ti[:, 2]].cpu().numpy()
     heads = ti[:, 1:2] * G + torch.arange(G, device="cuda")[None, :]
     do_rows = T.from_torch(dout[ti[:, 0:1], ti[:, 2:3], heads], "bf16")
-    ref = O.attend_backward_dq_rows(prob, tri, idx_rows, do_rows)               # [S, G, d]
+    ref = prob.backward_rows(tri, idx_rows, do_rows)                            # [S, G, d]
     got = dq[ti[:, 0:1], ti[:, 2:3], heads].double().cpu().numpy()
     o64 = dev.out[ti[:, 0:1], ti[:, 2:3], heads].double().cpu().numpy()
     do64 = O.load_storage(do_rows, "bf16")
     kmax = float(dev.k.abs().max())
     d_delta = 2.0 ** -9 * np.abs(o64 * do64).sum(axis=-1, keepdims=True) / np.sqrt(w.d) * kmax
     _close("dq rows", got, ref, d_delta)
+
+    # dk and dv of two whole key blocks of one KV head: the oracle's contributions of EVERY row that selected
+    # the block (found in the index tensor the backward was given), accumulated in fp64
+    for h, blk0 in ((1, 517), (6, 40)):
+        blk = blk0
+        while True:                                                             # a block a bounded number of rows selected
+            rows_sel = (dev.idx[0, h] == blk).any(dim=1).nonzero().flatten()    # positions that selected the block
+            if 0 < len(rows_sel) <= 8192:
+                break
+            blk += 1
+        tri_b = np.stack([np.zeros(len(rows_sel), dtype=np.int64), np.full(len(rows_sel), h, dtype=np.int64),
+                          rows_sel.cpu().numpy()], axis=1)
+        tb = torch.from_numpy(tri_b).cuda()
+        idx_b = dev.idx[0, h][rows_sel].cpu().numpy()
+        heads_b = tb[:, 1:2] * G + torch.arange(G, device="cuda")[None, :]
+        do_b = T.from_torch(dout[tb[:, 0:1], tb[:, 2:3], heads_b], "bf16")
+        lo, hi = blk * w.C, (blk + 1) * w.C
+        _, rdk, rdv = prob.backward_rows(tri_b, idx_b, do_b, key_range=(lo, hi))
+        T.check_gradient_rows(f"dk block {blk}", dk[0, lo:hi, h].double().cpu().numpy(), rdk)
+        T.check_gradient_rows(f"dv block {blk}", dv[0, lo:hi, h].double().cpu().numpy(), rdv)
+        print(f"[cfg4 backward] head {h} block {blk}: {len(rows_sel)} rows contribute")
