@@ -213,11 +213,12 @@ static int do_route(const pisa_params_t* p, const Geometry& g, const void* q, co
 }
 
 static int do_bsa(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v,
-                  const int32_t* idx, const float* sel_lse, void* out, float* lse, bool lse_ready, void* ws,
-                  size_t ws_bytes, cudaStream_t s) {
+                  const int32_t* idx, const float* sel_lse, void* out, float* lse, bool lse_ready, bool forced_present,
+                  void* ws, size_t ws_bytes, cudaStream_t s) {
   if (ws_bytes < bsa_ws_bytes(p, g)) return PISA_ERR_WORKSPACE_TOO_SMALL;
   if (use_tensor(p, g))
-    return tensor_bsa(g, p->dtype, q, k, v, idx, sel_lse, out, lse, lse_ready, (char*)ws + kStatusBytes, (int32_t*)ws, s);
+    return tensor_bsa(g, p->dtype, q, k, v, idx, sel_lse, out, lse, lse_ready, forced_present,
+                      (char*)ws + kStatusBytes, (int32_t*)ws, s);
   kernel_mark("bsa_simt", s);
   return launch_bsa_simt(g, p->dtype, q, k, v, idx, out, lse, s);
 }
@@ -451,12 +452,12 @@ static int do_bsa_chunked(const pisa_params_t* p, const Geometry& g, const void*
   st = clear_status(ws, s);
   if (st != PISA_OK) return st;
   g_mark_n = 0;
-  if (pl.n == 1) st = do_bsa(p, g, q, k, v_, idx, sel_lse, out, lse, false, ws, ws_bytes, s);
+  if (pl.n == 1) st = do_bsa(p, g, q, k, v_, idx, sel_lse, out, lse, false, false, ws, ws_bytes, s);
   else
     st = run_chunks(p, g, pl, ws, s, [&](const ChunkView& v, int) {
       return tensor_bsa(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, (const char*)v_ + v.v_off,
                         idx + v.unit0 * g.N * g.K, sel_lse ? sel_lse + v.unit0 * g.G * g.N * g.K : nullptr,
-                        (char*)out + v.o_off, lse + v.unit0 * g.G * g.N, false, v.region, (int32_t*)ws, v.stream);
+                        (char*)out + v.o_off, lse + v.unit0 * g.G * g.N, false, false, v.region, (int32_t*)ws, v.stream);
     });
   kernel_mark("end", s);
   return st;
@@ -505,7 +506,8 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
     st = do_route(p, g, q, k, pyr, idx, nullptr, nullptr, lse, ws, ws_bytes, s);
     if (st != PISA_OK) return st;
     stage_mark(2, s);
-    st = do_bsa(p, g, q, k, v_, idx, nullptr, out, lse, use_tensor(p, g) && g.score_mode == PISA_SCORE_LSE, ws, ws_bytes, s);
+    st = do_bsa(p, g, q, k, v_, idx, nullptr, out, lse, use_tensor(p, g) && g.score_mode == PISA_SCORE_LSE, true, ws,
+                ws_bytes, s);
   } else {
     st = run_chunks(p, g, pl, ws, s, [&](const ChunkView& v, int i) {
       int32_t* ic = idx + v.unit0 * g.N * g.K;
@@ -515,7 +517,7 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
       if (r != PISA_OK) return r;
       if (i == 0) stage_mark(2, s);
       return tensor_bsa(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, (const char*)v_ + v.v_off,
-                        ic, nullptr, (char*)out + v.o_off, lc, g.score_mode == PISA_SCORE_LSE, v.region, (int32_t*)ws,
+                        ic, nullptr, (char*)out + v.o_off, lc, g.score_mode == PISA_SCORE_LSE, true, v.region, (int32_t*)ws,
                         v.stream);
     });
   }

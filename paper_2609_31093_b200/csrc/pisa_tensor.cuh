@@ -16,8 +16,16 @@ int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, con
 // lse_ready: `lse` already holds the denominators of exactly these idx (as tensor_route writes them)
 // sel_lse (nullable): per-block denominators of exactly these idx (as tensor_route writes them); used when
 // lse_ready is false to skip the block-LSE pass
+// forced_present: idx comes from the routing, i.e. every row holds its forced leaves (0, c-1, c): they are then
+// served by the query-major local-window kernel instead of the lists
 int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const void* v, const int32_t* idx,
-               const float* sel_lse, void* out, float* lse, bool lse_ready, void* ws, int32_t* status, cudaStream_t s);
+               const float* sel_lse, void* out, float* lse, bool lse_ready, bool forced_present, void* ws,
+               int32_t* status, cudaStream_t s);
+
+// attention over the forced leaves, query-major (local_window.cu); stores the fp32 accumulator [B,Hkv,N,128,G]
+bool local_window_supported(const Geometry& g, int dtype);
+int launch_local_window(const Geometry& g, const void* q, const void* k, const void* v, const float* row_lse,
+                        float* o_acc, int32_t* status, cudaStream_t s);
 
 // backward of the block-sparse attention with frozen indices; dq [B,N,Hq,d], dk, dv [B,N,Hkv,d] dense
 bool tensor_bwd_supported(const Geometry& g, int dtype);

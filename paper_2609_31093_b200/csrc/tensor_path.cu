@@ -57,6 +57,7 @@ struct InvArgs {
   int32_t* entries;       // [<= BH*N*K]  token | slot << 24
   int32_t* status;        // the workspace's status word
   int debug;              // PISA_DEBUG_* bits
+  int skip_forced;        // leave the row's forced leaves (0, c-1, c) out of the lists: the local-window kernel serves them
 };
 
 __device__ __forceinline__ int inv_token(const InvArgs& a, int e) { return a.lgK >= 0 ? (e >> a.lgK) : e / a.K; }
@@ -66,6 +67,7 @@ __device__ __forceinline__ bool inv_valid(const InvArgs& a, int node, int t) {
   const bool ok = node >= 0 && node < a.Mk && (long long)node * a.fan <= (long long)leaf;
   // bounds-check mode: anything but the -1 padding that is not a usable node id is reported
   if ((a.debug & PISA_DEBUG_BOUNDS) && !ok && node != -1) atomicExch(a.status, (int)PISA_ERR_BOUNDS);
+  if (a.skip_forced && (node == 0 || node == leaf || node == leaf - 1)) return false;
   return ok;
 }
 
@@ -1307,9 +1309,9 @@ BsaLayout bsa_layout(const Geometry& g) {
 }
 
 int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char* ws, const InvLayout& l,
-                  InvArgs* out, int32_t* status, cudaStream_t s, int win = kWindowTok) {
+                  InvArgs* out, int32_t* status, cudaStream_t s, int win = kWindowTok, int skip_forced = 0) {
   InvArgs a;
-  a.status = status; a.debug = g.debug;
+  a.status = status; a.debug = g.debug; a.skip_forced = skip_forced;
   a.nodes = nodes; a.K = g.K; a.fan = fan; a.Mk = Mk; a.N = g.N; a.C = g.C; a.BH = g.B * g.Hkv;
   a.tpt = 128 / g.G;
   a.lgK = (g.K & (g.K - 1)) == 0 ? 31 - __builtin_clz((unsigned)g.K) : -1;
@@ -1473,7 +1475,8 @@ int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, con
 }
 
 int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const void* v, const int32_t* idx,
-               const float* sel_lse, void* out, float* lse, bool lse_ready, void* ws_, int32_t* status, cudaStream_t s) {
+               const float* sel_lse, void* out, float* lse, bool lse_ready, bool forced_present, void* ws_,
+               int32_t* status, cudaStream_t s) {
   (void)dtype;
   char* ws = (char*)ws_;
   const BsaLayout L = bsa_layout(g);
@@ -1481,7 +1484,11 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
   float* acc = (float*)(ws + L.acc);
   kernel_mark("invert_by_leaf", s);
   InvArgs inv;
-  int st = run_inversion(g, idx, 1, g.M[1], ws, L.inv, &inv, status, s);
+  // idx that came out of the routing holds every row's forced leaves: those go to the query-major
+  // local-window kernel, which also initialises the accumulator (it needs the rows' denominators, so only
+  // when the routing handed them over: the block-LSE pass below walks the very lists they are left out of)
+  const bool local = forced_present && lse_ready && local_window_supported(g, dtype);
+  int st = run_inversion(g, idx, 1, g.M[1], ws, L.inv, &inv, status, s, kWindowTok, local ? 1 : 0);
   if (st != PISA_OK) return st;
   TileArgs a = {};
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
@@ -1503,9 +1510,15 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
     st = check_launch("row_lse");
     if (st != PISA_OK) return st;
   }
-  kernel_mark("accumulator_memset", s);
-  cudaError_t e = cudaMemsetAsync(acc, 0, (size_t)g.B * g.N * g.Hq * g.d * 4, s);
-  if (e != cudaSuccess) { record_cuda_error("accumulator memset", e); return PISA_ERR_CUDA; }
+  if (local) {
+    kernel_mark("local_window", s);
+    st = launch_local_window(g, q, k, v, lse, acc, status, s);
+    if (st != PISA_OK) return st;
+  } else {
+    kernel_mark("accumulator_memset", s);
+    cudaError_t e = cudaMemsetAsync(acc, 0, (size_t)g.B * g.N * g.Hq * g.d * 4, s);
+    if (e != cudaSuccess) { record_cuda_error("accumulator memset", e); return PISA_ERR_CUDA; }
+  }
   kernel_mark("attention_tiles", s);
   st = dispatch_tile_pv(g, a, s);
   if (st != PISA_OK) return st;
