@@ -55,6 +55,7 @@ struct InvArgs {
   int32_t* cursor;        // [nkeys]
   int32_t* blk_tot;       // [3][ceil(nkeys / 1024) + 1] scan scratch: per-block totals, then block offsets
   int32_t* entries;       // [<= BH*N*K]  token | slot << 24
+  int32_t* work_ctr;      // next-work-item counter of the attention kernel that walks these lists (zeroed with count)
   int32_t* status;        // the workspace's status word
   int debug;              // PISA_DEBUG_* bits
   int skip_forced;        // leave the row's forced leaves (0, c-1, c) out of the lists: the local-window kernel serves them
@@ -260,6 +261,32 @@ __device__ __forceinline__ int find_key(const int32_t* tile_off, int nkeys, int 
   return lo;
 }
 
+// Work items of the attention kernel are handed out dynamically: lists differ in length, and a static
+// round-robin left the CTAs' tile counts 20 % apart (the leaf-scoring kernel keeps the static walk: its
+// epilogue warps sit at their register limit, and routing the item descriptions through shared memory
+// cost it more in spills than the balance gained).  Thread 0 of the CTA draws the next item from a global counter when the
+// producers start their k-th item and publishes it in a small shared-memory ring; every other role reads
+// the k-th entry when it gets there (it lags the producers by a few items at most: the producers cannot
+// start item k before the UMMAs of item k - 1 have completed).  An id >= the item count ends the walk.
+constexpr int kFeedRing = 16;
+struct ItemInfo {
+  int key, ntiles, e_begin, e_end;         // ntiles == 0: no more work
+};
+struct ItemFeed { volatile int4 info[kFeedRing]; volatile int seq[kFeedRing]; };
+// The wait is bounded by a poll count (about 2^27 shared-memory reads, seconds), not by the clock: the
+// readers are at their register limit and must not carry 64-bit time stamps through their loops.
+__device__ __noinline__ ItemInfo feed_get(ItemFeed& f, int k, volatile int* fail) {
+  ItemInfo r = {0, 0, 0, 0};
+  const int slot = k % kFeedRing;
+  for (uint32_t i = 0; f.seq[slot] != k + 1; ++i) {
+    if (*fail) return r;
+    if (i == (1u << 27)) { *fail = 1; return r; }
+  }
+  __threadfence_block();
+  r.key = f.info[slot].x; r.ntiles = f.info[slot].y; r.e_begin = f.info[slot].z; r.e_end = f.info[slot].w;
+  return r;
+}
+
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -337,9 +364,6 @@ constexpr int kLseThreads = 672;       // 4 producer warps, 1 MMA warp, 2 x 8 ep
 constexpr int kProdThreads = 128;
 constexpr int kMetaRing = 8;           // ring of per-tile metadata; deeper than any role can run ahead
 
-struct ItemInfo {
-  int key, ntiles, e_begin, e_end;
-};
 // bounds-check mode: a list entry (token | slot << 24) must name a token below N and a slot below `slots`;
 // one that does not is reported and dropped (-1 = no entry)
 __device__ __forceinline__ int checked_entry(const TileArgs& a, int N, int ent) {
@@ -361,6 +385,19 @@ __device__ __forceinline__ ItemInfo item_info(const TileArgs& a, int item, int t
   r.ntiles = min(kItemTiles, tiles - first);
   r.e_begin = list0 + first * tpt;
   r.e_end = list0 + cnt;
+  return r;
+}
+
+// thread 0 of the CTA: draw the k-th item of this CTA from the global counter and publish its description
+__device__ __forceinline__ ItemInfo feed_publish(ItemFeed& f, const TileArgs& a, int32_t* work_ctr, int n_items, int tpt,
+                                              int k) {
+  const int item = atomicAdd(work_ctr, 1);
+  ItemInfo r = {0, 0, 0, 0};
+  if (item < n_items) r = item_info(a, item, tpt);
+  f.info[k % kFeedRing].x = r.key; f.info[k % kFeedRing].y = r.ntiles;
+  f.info[k % kFeedRing].z = r.e_begin; f.info[k % kFeedRing].w = r.e_end;
+  __threadfence_block();
+  f.seq[k % kFeedRing] = k + 1;
   return r;
 }
 
@@ -634,7 +671,7 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
 constexpr int kPvThreads = 544;
 
 template <int D, int C>
-__global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, TileArgs a) {
+__global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int NS = 4;
   constexpr int KS = D / 64;
@@ -658,8 +695,10 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
   __shared__ volatile int s_fail;
   __shared__ int s_ent[kMetaRing][128];   // per-tile entries, written by the producers, read by all roles
   __shared__ float s_lse[kMetaRing][128]; // per-row softmax denominators
+  __shared__ ItemFeed feed;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid < kFeedRing) feed.seq[tid] = 0;
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) { mbar_init(&q_full[i], kProdThreads); mbar_init(&q_empty[i], kTransO ? 1 : 128); }
     mbar_init(&kv_empty, 1);
@@ -684,8 +723,11 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
     // ------------------------------------------------ producers
     int it = 0, kiter = 0, ent_next = -1;
     bool stop = false;
-    for (int item = blockIdx.x; item < n_items && !stop; item += gridDim.x, ++kiter) {
-      const ItemInfo inf = item_info(a, item, tpt);
+    for (;; ++kiter) {
+      if (tid == 0) feed_publish(feed, a, work_ctr, n_items, tpt, kiter);     // lane 0 draws the item; everybody reads it back
+      __syncwarp();
+      const ItemInfo inf = feed_get(feed, kiter, &s_fail);
+      if (inf.ntiles == 0 || stop) break;
       const int bh = inf.key / (a.NW * a.Mk), leaf = inf.key % a.Mk;
       const int b = bh / geo.Hkv, h = bh % geo.Hkv;
       bool bad = s_fail != 0;
@@ -726,14 +768,13 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
     const uint32_t idesc_ot = make_idesc_bf16(128, 128, 1, 0);   // O^T: M = d (V, MN-major), N = tile rows (P)
     int s_it = 0, pv_it = 0;              // next tile whose S / whose P V is to be issued
     unsigned last_bits = 0;               // bit (it & 31): tile `it` closes its work item
-    int item = blockIdx.x, jt = 0;
-    ItemInfo inf = {0, 0, 0, 0};
-    if (item < n_items) inf = item_info(a, item, tpt);
+    int kseq = 0, jt = 0;
+    ItemInfo inf = feed_get(feed, kseq, &s_fail);
     uint64_t t_idle = 0;
     uint32_t idle_polls = 0;
     bool ok = true;
     while (ok && !s_fail) {
-      const bool more_s = item < n_items;
+      const bool more_s = inf.ntiles > 0;
       if (!more_s && pv_it == s_it) break;
       int do_s = 0, do_pv = 0;
       if (lane == 0) {
@@ -786,9 +827,8 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
         last_bits = (last_bits & ~(1u << (s_it & 31))) | ((last ? 1u : 0u) << (s_it & 31));
         ++s_it;
         if (last) {
-          item += gridDim.x;
+          inf = feed_get(feed, ++kseq, &s_fail);
           jt = 0;
-          if (item < n_items) inf = item_info(a, item, tpt);
         } else {
           ++jt;
         }
@@ -810,8 +850,9 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
     const int row = (warp & 3) * 32 + lane;
     const uint32_t s_base = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(grp * 128);
     int it = 0;
-    for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x) {
-      const ItemInfo inf = item_info(a, item, tpt);
+    for (int kseq = 0; !s_fail; ++kseq) {
+      const ItemInfo inf = feed_get(feed, kseq, &s_fail);
+      if (inf.ntiles == 0) break;
       const int leaf = inf.key % a.Mk;
       for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
         if ((it & 1) != grp) continue;
@@ -878,8 +919,9 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
     const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
     const int sub = lane >> 4, ch = lane & 15;
     int it = 0;
-    for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x) {
-      const ItemInfo inf = item_info(a, item, tpt);
+    for (int kseq = 0; !s_fail; ++kseq) {
+      const ItemInfo inf = feed_get(feed, kseq, &s_fail);
+      if (inf.ntiles == 0) break;
       const int bh = inf.key / (a.NW * a.Mk);
       const int b = bh / geo.Hkv, h = bh % geo.Hkv;
       float* acc_bh = a.o_acc + ((long long)b * geo.N * geo.Hq + h * G) * D;
@@ -1263,7 +1305,7 @@ __global__ void __launch_bounds__(256) convert_out_heads_inner_kernel(Geometry g
 // ------------------------------------------------------------------ host side
 
 struct InvLayout {
-  size_t count, entry_off, tile_off, item_off, item_key, cursor, blk_tot, entries, end;
+  size_t count, work_ctr, entry_off, tile_off, item_off, item_key, cursor, blk_tot, entries, end;
 };
 
 int window_tokens(const Geometry& g, int win) { return g.N < win ? ((g.N + kInvTok - 1) / kInvTok) * kInvTok : win; }
@@ -1274,6 +1316,7 @@ InvLayout inv_layout(size_t base, const Geometry& g, int Mk, int win = kWindowTo
   InvLayout l;
   size_t o = base;
   l.count = o; o += align_up(nkeys * 4, 256);
+  l.work_ctr = o; o += 256;                 // right behind count: one memset clears both
   l.entry_off = o; o += align_up((nkeys + 1) * 4, 256);
   l.tile_off = o; o += align_up((nkeys + 1) * 4, 256);
   l.item_off = o; o += align_up((nkeys + 1) * 4, 256);
@@ -1323,8 +1366,9 @@ int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char
   a.cursor = (int32_t*)(ws + l.cursor);
   a.blk_tot = (int32_t*)(ws + l.blk_tot);
   a.entries = (int32_t*)(ws + l.entries);
+  a.work_ctr = (int32_t*)(ws + l.work_ctr);
   const size_t nkeys = (size_t)a.BH * a.NW * Mk;
-  cudaError_t e = cudaMemsetAsync(a.count, 0, nkeys * 4, s);
+  cudaError_t e = cudaMemsetAsync(a.count, 0, l.work_ctr + 256 - l.count, s);
   if (e != cudaSuccess) { record_cuda_error("inversion memset", e); return PISA_ERR_CUDA; }
   const int use_smem = (2 * (size_t)Mk * 4 <= 96 * 1024) ? 1 : 0;
   const size_t sm_count = use_smem ? (size_t)Mk * 4 : 0, sm_fill = use_smem ? 2 * (size_t)Mk * 4 : 0;
@@ -1353,47 +1397,50 @@ int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char
 }
 
 template <int D, int NB, bool MOM>
-int launch_tile_lse_m(const Geometry& g, const TileArgs& a, cudaStream_t s) {
+int launch_tile_lse_m(const Geometry& g, const TileArgs& a, int32_t* work_ctr, cudaStream_t s) {
   const size_t smem = (size_t)(D / 64) * (4 * 128 * 128 + NB * 128) + 1024;
   cudaError_t e = cudaFuncSetAttribute(lse_ws_kernel<D, NB, MOM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("lse_ws attr", e); return PISA_ERR_CUDA; }
+  (void)work_ctr;   // the leaf-scoring kernel walks its items statically (see ItemFeed)
   lse_ws_kernel<D, NB, MOM><<<num_sms(), kLseThreads, smem, s>>>(g, a);
   return check_launch("lse_ws");
 }
 template <int D, int NB>
-int launch_tile_lse(const Geometry& g, const TileArgs& a, cudaStream_t s) {
-  return (a.mode == PISA_SCORE_LSE) ? launch_tile_lse_m<D, NB, false>(g, a, s) : launch_tile_lse_m<D, NB, true>(g, a, s);
+int launch_tile_lse(const Geometry& g, const TileArgs& a, int32_t* work_ctr, cudaStream_t s) {
+  return (a.mode == PISA_SCORE_LSE) ? launch_tile_lse_m<D, NB, false>(g, a, work_ctr, s)
+                                    : launch_tile_lse_m<D, NB, true>(g, a, work_ctr, s);
 }
 
-int dispatch_tile_lse(const Geometry& g, int nb, const TileArgs& a, cudaStream_t s) {
+int dispatch_tile_lse(const Geometry& g, int nb, const TileArgs& a, int32_t* work_ctr, cudaStream_t s) {
   if (g.d == 128) {
-    if (nb == 64) return launch_tile_lse<128, 64>(g, a, s);
-    if (nb == 128) return launch_tile_lse<128, 128>(g, a, s);
-    if (nb == 256) return launch_tile_lse<128, 256>(g, a, s);
+    if (nb == 64) return launch_tile_lse<128, 64>(g, a, work_ctr, s);
+    if (nb == 128) return launch_tile_lse<128, 128>(g, a, work_ctr, s);
+    if (nb == 256) return launch_tile_lse<128, 256>(g, a, work_ctr, s);
   } else if (g.d == 64) {
-    if (nb == 64) return launch_tile_lse<64, 64>(g, a, s);
-    if (nb == 128) return launch_tile_lse<64, 128>(g, a, s);
-    if (nb == 256) return launch_tile_lse<64, 256>(g, a, s);
+    if (nb == 64) return launch_tile_lse<64, 64>(g, a, work_ctr, s);
+    if (nb == 128) return launch_tile_lse<64, 128>(g, a, work_ctr, s);
+    if (nb == 256) return launch_tile_lse<64, 256>(g, a, work_ctr, s);
   }
   return PISA_ERR_UNSUPPORTED;
 }
 
+// work_ctr: the launch's next-work-item counter (zero on entry)
 template <int D, int C>
-int launch_tile_pv(const Geometry& g, const TileArgs& a, cudaStream_t s) {
+int launch_tile_pv(const Geometry& g, const TileArgs& a, int32_t* work_ctr, cudaStream_t s) {
   constexpr int KS = D / 64;
   constexpr int QP = (KS * 128 * 128 > 128 * 272) ? KS * 128 * 128 : 128 * 272;
   const size_t smem = 4 * (size_t)((QP + 1023) / 1024 * 1024) + 2 * (size_t)KS * C * 128 + 1024;
   cudaError_t e = cudaFuncSetAttribute(pv_ws_kernel<D, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("pv_ws attr", e); return PISA_ERR_CUDA; }
-  pv_ws_kernel<D, C><<<num_sms(), kPvThreads, smem, s>>>(g, a);
+  pv_ws_kernel<D, C><<<num_sms(), kPvThreads, smem, s>>>(g, a, work_ctr);
   return check_launch("pv_ws");
 }
 
-int dispatch_tile_pv(const Geometry& g, const TileArgs& a, cudaStream_t s) {
-  if (g.d == 128 && g.C == 128) return launch_tile_pv<128, 128>(g, a, s);
-  if (g.d == 128 && g.C == 64) return launch_tile_pv<128, 64>(g, a, s);
-  if (g.d == 64 && g.C == 128) return launch_tile_pv<64, 128>(g, a, s);
-  if (g.d == 64 && g.C == 64) return launch_tile_pv<64, 64>(g, a, s);
+int dispatch_tile_pv(const Geometry& g, const TileArgs& a, int32_t* work_ctr, cudaStream_t s) {
+  if (g.d == 128 && g.C == 128) return launch_tile_pv<128, 128>(g, a, work_ctr, s);
+  if (g.d == 128 && g.C == 64) return launch_tile_pv<128, 64>(g, a, work_ctr, s);
+  if (g.d == 64 && g.C == 128) return launch_tile_pv<64, 128>(g, a, work_ctr, s);
+  if (g.d == 64 && g.C == 64) return launch_tile_pv<64, 64>(g, a, work_ctr, s);
   return PISA_ERR_UNSUPPORTED;
 }
 
@@ -1459,7 +1506,7 @@ int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, con
   a.nkeys = g.B * g.Hkv * inv.NW * g.M[2]; a.Mk = g.M[2]; a.NW = inv.NW; a.fan = g.g; a.slots = g.K;
   a.blk_lse = blk; a.status = status; a.mode = g.score_mode; a.debug = g.debug;
   kernel_mark("leaf_lse_tiles", s);
-  st = dispatch_tile_lse(g, g.g * g.C, a, s);
+  st = dispatch_tile_lse(g, g.g * g.C, a, inv.work_ctr, s);
   if (st != PISA_OK) return st;
   kernel_mark("final_topk", s);
   const long long total = (long long)g.B * g.Hkv * g.N;
@@ -1503,7 +1550,7 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
     if (st != PISA_OK) return st;
   } else if (!lse_ready) {
     kernel_mark("block_lse_tiles", s);
-    st = dispatch_tile_lse(g, g.C, a, s);
+    st = dispatch_tile_lse(g, g.C, a, inv.work_ctr, s);
     if (st != PISA_OK) return st;
     const long long rows = (long long)g.B * g.Hkv * g.N * g.G;
     row_lse_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, s>>>(g, idx, blk, lse);
@@ -1520,7 +1567,7 @@ int tensor_bsa(const Geometry& g, int dtype, const void* q, const void* k, const
     if (e != cudaSuccess) { record_cuda_error("accumulator memset", e); return PISA_ERR_CUDA; }
   }
   kernel_mark("attention_tiles", s);
-  st = dispatch_tile_pv(g, a, s);
+  st = dispatch_tile_pv(g, a, inv.work_ctr + 1, s);            // the block-LSE pass above, if it ran, used the first counter
   if (st != PISA_OK) return st;
   kernel_mark("convert_out", s);
   if (g.d == 128) {
