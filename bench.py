@@ -40,7 +40,8 @@ def dram_bytes_per_pair() -> dict:
     try:
         d = json.load(open(os.path.join(ROOT, "profiles", "dram_bytes_per_pair.json")))
         n = float(d["pairs_per_launch"])
-        return {k_: (v_["dram_bytes_read"] + v_["dram_bytes_write"]) / n for k_, v_ in d.items() if isinstance(v_, dict)}
+        return {k_: (v_["dram_bytes_read"] + v_["dram_bytes_write"]) / float(v_.get("pairs_per_launch", n))
+                for k_, v_ in d.items() if isinstance(v_, dict)}
     except Exception:
         return {}
 
@@ -73,6 +74,7 @@ def work_counts(w: S.Workload) -> dict:
     inter_pairs = 0      # (token, candidate) pairs scored from child summaries, summed over levels >= 2
     leaf_pairs = 0       # (token, leaf) pairs scored from raw keys
     sel_pairs = 0        # (token, selected leaf) pairs
+    forced_pairs = 0     # of those, the forced leaves (first / previous / current), served by the local-window kernel
     for c in range(M[1]):
         toks = min(w.C, w.N - c * w.C)
         n_kept = 1
@@ -97,6 +99,7 @@ def work_counts(w: S.Workload) -> dict:
             else:
                 n_kept = nV
         sel_pairs += toks * n_kept
+        forced_pairs += toks * min(3, c + 1)
     units = w.B * w.Hkv
     G = w.Hq // w.Hkv
     es = 2 if w.dtype == "bf16" else 4
@@ -107,6 +110,7 @@ def work_counts(w: S.Workload) -> dict:
         "pyramid_bytes": float(w.B * w.N * w.Hkv * w.d * es + w.B * w.Hkv * sum(M[1:]) * w.d * es),
         "hbm_min_bytes": float(w.B * w.N * ((2 * w.Hq + 2 * w.Hkv) * w.d * es + w.Hq * 4 + w.Hkv * w.K * 4)),
         "sel_pairs": sel_pairs * units, "leaf_pairs": leaf_pairs * units, "inter_pairs": inter_pairs * units,
+        "forced_pairs": forced_pairs * units, "forced_flops": 4.0 * forced_pairs * w.C * G * w.d * units,
     }
 
 
@@ -421,8 +425,13 @@ def run_ours(args):
     # Algorithmic work per launch: leaf scoring and attention are dense contractions (tensor bound,
     # 2*C*G*d flops per scored (token, leaf) pair, 4*C*G*d per selected pair), the intermediate levels
     # too (2*g*G*d per scored (token, node) pair); the pyramid is one streaming pass over k (HBM bound).
+    # with the local-window kernel in the launch list the list-driven attention kernel only sees the routed pairs
+    local = "local_window" in kernels
+    routed_flops = wc["attn_flops"] - (wc["forced_flops"] if local else 0.0)
+    routed_pairs = wc["sel_pairs"] - (wc["forced_pairs"] if local else 0)
     algo = {
-        "leaf_lse_tiles": ("tensor", wc["leaf_flops"]), "attention_tiles": ("tensor", wc["attn_flops"]),
+        "leaf_lse_tiles": ("tensor", wc["leaf_flops"]), "attention_tiles": ("tensor", routed_flops),
+        "local_window": ("tensor", wc["forced_flops"]),
         "route_stage1": ("tensor", wc["inter_flops"]), "route_simt": ("tensor", wc["leaf_flops"] + wc["inter_flops"]),
         "bsa_simt": ("tensor", wc["attn_flops"]), "pyramid": ("hbm", wc["pyramid_bytes"]),
     }
@@ -452,15 +461,16 @@ def run_ours(args):
     # DRAM bytes per launch from the ncu capture of a smaller case of the same kernel (summary under
     # profiles/), scaled by the (token, block) pairs a launch processes: traffic grows with the pairs
     per_pair = dram_bytes_per_pair().get(dom)
-    pairs = {"leaf_lse_tiles": wc["sel_pairs"], "attention_tiles": wc["sel_pairs"]}.get(dom)
+    pairs = {"leaf_lse_tiles": wc["sel_pairs"], "attention_tiles": routed_pairs}.get(dom)
     roof["traffic"] = (per_pair * pairs / n_launch) if (per_pair and pairs and w.dtype == "bf16") else None
     # The two tile kernels are limited by what L2 can gather and reduce, not by the tensor pipe: report
     # that stream too (per selected pair: G*d*2 bytes of query rows L2->SM, and in the attention
     # kernel G*d*4 bytes of fp32 reductions SM->L2).  Context for `frac`, not a substitute for it.
     if dom in ("leaf_lse_tiles", "attention_tiles") and w.dtype == "bf16":
         per_pair_l2 = w.G * w.d * 2 + (w.G * w.d * 4 if dom == "attention_tiles" else 0)
-        roof["l2_stream_bytes"] = per_pair_l2 * wc["sel_pairs"] / n_launch
-        roof["l2_stream_tbs"] = per_pair_l2 * wc["sel_pairs"] / t_dom / 1e12
+        l2_pairs = routed_pairs if dom == "attention_tiles" else wc["sel_pairs"]
+        roof["l2_stream_bytes"] = per_pair_l2 * l2_pairs / n_launch
+        roof["l2_stream_tbs"] = per_pair_l2 * l2_pairs / t_alone / 1e12
     roofs = {}
     for k_, t_ in cand.items():
         b_, w_ = algo[k_]
@@ -475,7 +485,7 @@ def run_ours(args):
     t_pyr = kernels.get("pyramid", stage[0])
     t_route = sum(kernels.get(n_, 0.0) for n_ in ("route_stage1", "invert_by_parent", "leaf_lse_tiles", "final_topk",
                                                    "route_simt")) or stage[1]
-    t_attn = sum(kernels.get(n_, 0.0) for n_ in ("invert_by_leaf", "accumulator_memset", "attention_tiles",
+    t_attn = sum(kernels.get(n_, 0.0) for n_ in ("invert_by_leaf", "accumulator_memset", "local_window", "attention_tiles",
                                                   "convert_out", "bsa_simt", "row_lse")) or stage[2]
     stages = {
         "pyramid_us": t_pyr * 1e3, "route_us": t_route * 1e3, "attn_us": t_attn * 1e3,
