@@ -493,7 +493,7 @@ def _visible_tokens(blocks, p: int, C: int, N: int) -> np.ndarray:
 
 def attend_backward(q, k, v, idx, dout, *, C: int, dtype: str, scale: Optional[float] = None):
     """Gradients of Eq. "selected sparse attention" with the selected block indices held fixed
-    (App. B: gradients flow through attention on the selected entries, not through the selection).
+    (App. B): idx is a constant, only q, k and v receive gradients.
 
     q, dout: [B, N, Hq, d]; k, v: [B, N, Hkv, d] storage form; idx: int [B, Hkv, N, K] (-1 padded).
     For one query row with probabilities p_j over its visible selected keys, o = sum_j p_j v_j:

@@ -292,8 +292,9 @@ static int forward_plan(const pisa_params_t* p, const Geometry& g, int ops, Forw
   long long parts = units * g.N / kMinChunkTokens;
   // The attention kernel draws its work items dynamically, so it no longer leaves a tail of idle SMs for
   // another chunk to fill: two chunks (measured 44.5 ms at B=1, Hkv=8, N=128K against 45.2 with four) keep
-  // the leaf-scoring kernel's tail covered.  The backward kernel walks its items statically: four chunks.
-  const int max_chunks = (ops == kOpBwd) ? kMaxChunks : 2;
+  // the leaf-scoring kernel's tail covered.  Routing alone (stage 1 and the statically walked leaf scoring
+  // fill each other's tails) and the backward kernel, which also walks its items statically, keep four.
+  const int max_chunks = (ops == kOpBwd || ops == kOpRoute) ? kMaxChunks : 2;
   if (parts > max_chunks) parts = max_chunks;
   if (g_chunk_limit > 0 && parts > g_chunk_limit) parts = g_chunk_limit;
   if (parts > units) parts = units;
