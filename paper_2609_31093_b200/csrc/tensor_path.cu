@@ -23,6 +23,7 @@
 
 #include "pisa_tensor.cuh"
 #include "tc_utils.cuh"
+#include "tma_map.cuh"
 
 namespace pisa {
 
@@ -671,7 +672,9 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
 constexpr int kPvThreads = 544;
 
 template <int D, int C>
-__global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr) {
+__global__ void __launch_bounds__(kPvThreads, 1)
+pv_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant__ CUtensorMap tm_k,
+             const __grid_constant__ CUtensorMap tm_v) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int NS = 4;
   constexpr int KS = D / 64;
@@ -689,7 +692,7 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
   uint8_t* sQ = smem;
   uint8_t* sK = smem + NS * Q_STAGE;
   uint8_t* sV = sK + KS * KV_SLAB;
-  __shared__ uint64_t q_full[NS], q_empty[NS], kv_empty, s_full[2], s_empty[2], p_ready[2], o_full[2], o_empty[2];
+  __shared__ uint64_t q_full[NS], q_empty[NS], kv_full, kv_empty, s_full[2], s_empty[2], p_ready[2], o_full[2], o_empty[2];
   __shared__ __align__(16) int s_rowidx[kMetaRing][128];  // accumulator row (t*Hq + head) of every tile row, -1 = none
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_fail;
@@ -702,6 +705,7 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) { mbar_init(&q_full[i], kProdThreads); mbar_init(&q_empty[i], kTransO ? 1 : 128); }
     mbar_init(&kv_empty, 1);
+    mbar_init(&kv_full, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 128); mbar_init(&p_ready[i], 128);
       mbar_init(&o_full[i], 1); mbar_init(&o_empty[i], 128);
@@ -733,10 +737,15 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
       bool bad = s_fail != 0;
       if (!bad && kiter > 0) bad = !mbar_wait_bounded(&kv_empty, (uint32_t)((kiter - 1) & 1));
       if (prod_sync_or(bad)) { s_fail = 1; stop = true; break; }
-      prod_load_rows<D>(sK, KV_SLAB, a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2], geo.ks[1], leaf * C,
-                        C, geo.N, tid);
-      prod_load_rows<D>(sV, KV_SLAB, a.v + (long long)b * geo.vs[0] + (long long)h * geo.vs[2], geo.vs[1], leaf * C,
-                        C, geo.N, tid);
+      if (tid == 0) {
+        // the block's keys and values: contiguous C x d slabs, one TMA tile load per 64-wide slab (this GPU's
+        // memory, no multicast; rows past N read as zero), so that the producer warps only gather queries
+        mbar_arrive_expect_tx(&kv_full, (uint32_t)(2 * KS * KV_SLAB));
+        for (int ks = 0; ks < KS; ++ks) {
+          tma_load_4d(smem_u32(sK + ks * KV_SLAB), &tm_k, &kv_full, ks * 64, h, leaf * C, b);
+          tma_load_4d(smem_u32(sV + ks * KV_SLAB), &tm_v, &kv_full, ks * 64, h, leaf * C, b);
+        }
+      }
       const __nv_bfloat16* qb = a.q + (long long)b * geo.qs[0] + (long long)(h * G) * geo.qs[2];
       for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
         const int s = it % NS;
@@ -780,7 +789,7 @@ __global__ void __launch_bounds__(kPvThreads, 1) pv_ws_kernel(Geometry geo, Tile
       if (lane == 0) {
         if (more_s && s_it - pv_it < 2) {
           const int s = s_it % NS, buf = s_it & 1;
-          do_s = mbar_test(&q_full[s], (uint32_t)((s_it / NS) & 1)) &&
+          do_s = mbar_test(&q_full[s], (uint32_t)((s_it / NS) & 1)) && mbar_test(&kv_full, (uint32_t)(kseq & 1)) &&
                  (s_it < 2 || mbar_test(&s_empty[buf], (uint32_t)(((s_it >> 1) - 1) & 1)));
         }
         if (pv_it < s_it) {
@@ -1428,11 +1437,22 @@ int dispatch_tile_lse(const Geometry& g, int nb, const TileArgs& a, int32_t* wor
 template <int D, int C>
 int launch_tile_pv(const Geometry& g, const TileArgs& a, int32_t* work_ctr, cudaStream_t s) {
   constexpr int KS = D / 64;
+  CUtensorMap tm_k, tm_v;
+  {
+    const uint64_t dims[4] = {(uint64_t)g.d, (uint64_t)g.Hkv, (uint64_t)g.N, (uint64_t)g.B};
+    const uint32_t box[4] = {64u, 1u, (uint32_t)C, 1u};
+    const uint64_t sk[4] = {2, (uint64_t)g.ks[2] * 2, (uint64_t)g.ks[1] * 2, (uint64_t)g.ks[0] * 2};
+    const uint64_t sv[4] = {2, (uint64_t)g.vs[2] * 2, (uint64_t)g.vs[1] * 2, (uint64_t)g.vs[0] * 2};
+    if (!tma::make_map(&tm_k, 2, 4, a.k, dims, sk, box, true) || !tma::make_map(&tm_v, 2, 4, a.v, dims, sv, box, true)) {
+      record_cuda_error("pv_ws tensor maps", cudaErrorInvalidValue);
+      return PISA_ERR_CUDA;
+    }
+  }
   constexpr int QP = (KS * 128 * 128 > 128 * 272) ? KS * 128 * 128 : 128 * 272;
   const size_t smem = 4 * (size_t)((QP + 1023) / 1024 * 1024) + 2 * (size_t)KS * C * 128 + 1024;
   cudaError_t e = cudaFuncSetAttribute(pv_ws_kernel<D, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("pv_ws attr", e); return PISA_ERR_CUDA; }
-  pv_ws_kernel<D, C><<<num_sms(), kPvThreads, smem, s>>>(g, a, work_ctr);
+  pv_ws_kernel<D, C><<<num_sms(), kPvThreads, smem, s>>>(g, a, work_ctr, tm_k, tm_v);
   return check_launch("pv_ws");
 }
 
