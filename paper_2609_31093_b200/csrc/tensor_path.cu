@@ -476,7 +476,7 @@ __device__ __forceinline__ bool prod_sync_or(bool flag) {
 // MOM: false = per-head LSE of every leaf; true = first / second moments of the logits (score modes
 // "mean" and "mean + variance/2"), a separate instantiation so that the LSE one keeps its registers.
 template <int D, int NB, bool MOM>
-__global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, TileArgs a) {
+__global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, TileArgs a, const __grid_constant__ CUtensorMap tm_k) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int NS = 4;
   constexpr int KS = D / 64;
@@ -486,7 +486,7 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
   uint8_t* smem = align1024(smem_raw);
   uint8_t* sA = smem;
   uint8_t* sB = smem + NS * A_STAGE;
-  __shared__ uint64_t a_full[NS], a_empty[NS], b_empty, t_full[2], t_empty[2];
+  __shared__ uint64_t a_full[NS], a_empty[NS], b_full, b_empty, t_full[2], t_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_fail;
 
@@ -494,6 +494,7 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) { mbar_init(&a_full[i], kProdThreads); mbar_init(&a_empty[i], 1); }
     mbar_init(&b_empty, 1);
+    mbar_init(&b_full, 1);
     for (int i = 0; i < 2; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 256); }
     s_fail = 0;
     mbar_fence_init();
@@ -529,8 +530,10 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
       bool ok = s_fail == 0;
       if (ok && kiter > 0) ok = mbar_wait_bounded(&b_empty, (uint32_t)((kiter - 1) & 1));
       if (!__all_sync(0xffffffffu, ok)) { s_fail = 1; stop = true; break; }
-      prod_load_rows<D>(sB, B_SLAB, a.k + (long long)b * geo.ks[0] + (long long)h * geo.ks[2], geo.ks[1], j * NB,
-                        NB, geo.N, tid);
+      if (tid == 0) {                             // the node's keys: one TMA tile load per 64-wide slab (own memory, no multicast)
+        mbar_arrive_expect_tx(&b_full, (uint32_t)(KS * B_SLAB));
+        for (int ks = 0; ks < KS; ++ks) tma_load_4d(smem_u32(sB + ks * B_SLAB), &tm_k, &b_full, ks * 64, h, j * NB, b);
+      }
       const __nv_bfloat16* qb = a.q + (long long)b * geo.qs[0] + (long long)(h * G) * geo.qs[2];
       for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
         const int s = it % NS;
@@ -553,10 +556,10 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
   } else if (warp == 4) {
     // ------------------------------------------------ MMA issuer (the warp walks the loop, lane 0 issues)
     const uint32_t idesc = make_idesc_bf16(128, NB, 0, 0);
-    int it = 0;
-    for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x) {
+    int it = 0, kit = 0;
+    for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x, ++kit) {
       const ItemInfo inf = item_info(a, item, tpt);
-      bool ok = true;
+      bool ok = mbar_wait_bounded(&b_full, (uint32_t)(kit & 1));      // the node's keys have landed
       for (int jt = 0; jt < inf.ntiles && ok; ++jt, ++it) {
         const int s = it % NS, buf = it & 1;
         ok = mbar_wait_bounded(&a_full[s], (uint32_t)((it / NS) & 1));
@@ -1407,11 +1410,21 @@ int run_inversion(const Geometry& g, const int32_t* nodes, int fan, int Mk, char
 
 template <int D, int NB, bool MOM>
 int launch_tile_lse_m(const Geometry& g, const TileArgs& a, int32_t* work_ctr, cudaStream_t s) {
+  CUtensorMap tm_k;
+  {
+    const uint64_t dims[4] = {(uint64_t)g.d, (uint64_t)g.Hkv, (uint64_t)g.N, (uint64_t)g.B};
+    const uint32_t box[4] = {64u, 1u, (uint32_t)NB, 1u};
+    const uint64_t sk[4] = {2, (uint64_t)g.ks[2] * 2, (uint64_t)g.ks[1] * 2, (uint64_t)g.ks[0] * 2};
+    if (!tma::make_map(&tm_k, 2, 4, a.k, dims, sk, box, true)) {
+      record_cuda_error("lse_ws tensor map", cudaErrorInvalidValue);
+      return PISA_ERR_CUDA;
+    }
+  }
   const size_t smem = (size_t)(D / 64) * (4 * 128 * 128 + NB * 128) + 1024;
   cudaError_t e = cudaFuncSetAttribute(lse_ws_kernel<D, NB, MOM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("lse_ws attr", e); return PISA_ERR_CUDA; }
   (void)work_ctr;   // the leaf-scoring kernel walks its items statically (see ItemFeed)
-  lse_ws_kernel<D, NB, MOM><<<num_sms(), kLseThreads, smem, s>>>(g, a);
+  lse_ws_kernel<D, NB, MOM><<<num_sms(), kLseThreads, smem, s>>>(g, a, tm_k);
   return check_launch("lse_ws");
 }
 template <int D, int NB>
