@@ -67,13 +67,23 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
   }
   const U32x8 zero8 = {{0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u}};
 
+  // Levels that hold at most K nodes cannot prune: every node that does not start after the query's leaf is
+  // kept and expanded.  The walk therefore starts at the highest level with more than K nodes (or at level
+  // 2), whose candidates are simply the nodes 0 .. anc(c) (at most g*K of them: the level above holds <= K).
+  int l_start = 2;
+  for (int l = geo.L; l > 2; --l)
+    if (geo.M[l] > K) { l_start = l; break; }
   int cur = 0;
-  int n = 1;
-  if (lane == 0) s_cand[warp][0][0] = 0;
+  int n;
+  {
+    const unsigned span0 = (unsigned)min(geo.span[l_start], (long long)0x7fffffff);
+    n = min((int)((unsigned)c / span0), geo.M[l_start] - 1) + 1;
+    for (int s = lane; s < n; s += 32) s_cand[warp][0][s] = s;
+  }
   float min_gap = CUDART_INF_F;
   __syncwarp();
 
-  for (int l = geo.L; l >= 2; --l) {
+  for (int l = l_start; l >= 2; --l) {
     int* cand = s_cand[warp][cur];
     int* next = s_cand[warp][cur ^ 1];
     // leaves under a level-l node; c < 2^31, so a span beyond that just means ancestor 0 (32-bit division)
