@@ -51,7 +51,7 @@ enum { PISA_BF16 = 0, PISA_FP32 = 1 };
 enum { PISA_SCORE_LSE = 0, PISA_SCORE_MEAN = 1, PISA_SCORE_MEAN_VAR = 2 };
 /* operations a workspace can be sized for */
 enum { PISA_OP_ROUTE = 0, PISA_OP_BSA = 1, PISA_OP_FORWARD = 2, PISA_OP_FLAT = 3, PISA_OP_FORWARD_HOST = 4,
-       PISA_OP_DECODE = 5, PISA_OP_BSA_BWD = 6 };
+       PISA_OP_DECODE = 5, PISA_OP_BSA_BWD = 6, PISA_OP_FORWARD_PACKED = 7 };
 /* implementation selector (params.impl): AUTO picks the tensor-core path where it applies */
 enum { PISA_IMPL_AUTO = 0, PISA_IMPL_SIMT = 1, PISA_IMPL_TENSOR = 2 };
 /*
@@ -189,7 +189,18 @@ int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const voi
  *   idx         : device int32, sequence-major: sequence i's [Hkv, len_i, K] block starts at element
  *                 Hkv * K * cu[i]; block ids are relative to the sequence
  *   lse         : device float, sequence-major: sequence i's [Hq, len_i] block starts at Hq * cu[i]
- *   ws          : device workspace sized for PISA_OP_FORWARD with p (N = the longest sequence)
+ *   ws          : device workspace sized for PISA_OP_FORWARD_PACKED with p (N = the longest sequence)
+ *
+ * Launches.  The method is causal (Sec. 3.2: a query only ever scores nodes that lie wholly in its
+ * past; the nodes on its own path are forced, not scored), so a sequence gives the same rows when it is
+ * the head of a longer, zero-filled batch element.  Sequences of at most 8192 tokens are therefore
+ * grouped by length (a group's members are no shorter than 3/4 of its padded length, padded lengths come
+ * from the grid m * 2^k, m = 8..15, and a group holds at most 32768 padded tokens), copied into a padded
+ * batch inside the workspace, run through ONE set of launches of the batched forward, and the valid rows
+ * copied back.  Longer sequences, and groups of one, run unpadded on the packed tensors.  With a
+ * workspace sized for PISA_OP_FORWARD only (too small for the padded copies) the call runs the sequences
+ * one after the other instead; the results are the same rows either way (up to the rounding order of
+ * the fp32 partial sums).
  */
 int pisa_forward_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32_t nseq, const void* q,
                         const void* k, const void* v, void* pyramid, int32_t* idx, void* out, float* lse,

@@ -4,6 +4,9 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
+#include <vector>
+
 #include "pisa_common.cuh"
 #include "pisa_tensor.cuh"
 
@@ -591,6 +594,74 @@ int pisa_pyramid_layout(const pisa_params_t* p, int32_t* L, int32_t* M, int64_t*
   return PISA_OK;
 }
 
+// ---------------------------------------------------------------- packed batches as padded batches
+//
+// pisa_forward_packed groups the short sequences of a packed batch by length and runs every group as a
+// padded batch [B', N'] through one set of launches (the copies are in packed.cu).  N' comes from a fixed
+// grid (m * 2^k, m = 8..15: at most 12.5 % apart) so that the workspace can be sized from the parameters
+// alone; a group holds sequences no shorter than 3/4 of its N' and at most kPackTokens padded tokens
+// (more if the longest sequence is longer).  Sequences above kPackDirectLen, and groups of one, run
+// unpadded on the packed tensors themselves.
+constexpr int kPackDirectLen = 8192;
+constexpr long long kPackTokens = 32768;
+
+static int pack_grid_len(int len) {
+  int k = 0;
+  while ((15LL << k) < len) ++k;
+  int m = (int)(((long long)len + (1LL << k) - 1) >> k);
+  if (m < 8) m = 8;
+  return m << k;
+}
+
+struct PackedArena {
+  long long tokens;                        // padded tokens one group may hold
+  size_t fwd, pyr, qb, kb, lb, ib, total;  // bytes: forward workspace, pyramid, q/out, k/v, lse, idx (one group)
+};
+
+static size_t forward_ws_bytes(const pisa_params_t* p, const Geometry& g, int* st) {
+  size_t r = route_ws_bytes(p, g), a = bsa_ws_bytes(p, g);
+  size_t f = r > a ? r : a;
+  ForwardPlan pl;
+  *st = forward_plan(p, g, kOpRoute | kOpBsa, &pl);
+  if (*st == PISA_OK && pl.total > f) f = pl.total;
+  return f;
+}
+
+static int packed_arena(const pisa_params_t* p, PackedArena* a) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  a->tokens = kPackTokens;
+  size_t fwd = forward_ws_bytes(p, g, &st), pyr = 0;
+  if (st != PISA_OK) return st;
+  const int n_max = p->N < kPackDirectLen ? p->N : kPackDirectLen;
+  for (int k = 0; k < 31; ++k)
+    for (int m = 8; m <= 15; ++m) {
+      const long long np = (long long)m << k;
+      if (np > pack_grid_len(n_max)) continue;
+      pisa_params_t pg = *p;
+      pg.N = (int)np;
+      pg.B = (int)(a->tokens / np < 1 ? 1 : a->tokens / np);
+      Geometry gg;
+      if ((st = resolve(&pg, &gg)) != PISA_OK) return st;
+      const size_t f = forward_ws_bytes(&pg, gg, &st);
+      if (st != PISA_OK) return st;
+      if (f > fwd) fwd = f;
+      const size_t pb = pyramid_bytes_dtype(gg, p->dtype);
+      if (pb > pyr) pyr = pb;
+    }
+  const size_t es = elem_size(p->dtype);
+  const size_t tok = (size_t)a->tokens;                                    // B' * N' <= tokens for every group
+  a->fwd = align_up(fwd, 256);
+  a->pyr = align_up(pyr, 256);
+  a->qb = align_up(tok * g.Hq * g.d * es, 256);
+  a->kb = align_up(tok * g.Hkv * g.d * es, 256);
+  a->lb = align_up(tok * g.Hq * sizeof(float), 256);
+  a->ib = align_up(tok * g.Hkv * g.K * sizeof(int32_t), 256);
+  a->total = a->fwd + a->pyr + 2 * a->qb + 2 * a->kb + a->lb + a->ib;
+  return PISA_OK;
+}
+
 int pisa_workspace_bytes(const pisa_params_t* p, int op, size_t* bytes) {
   Geometry g;
   int st = resolve(p, &g);
@@ -628,6 +699,13 @@ int pisa_workspace_bytes(const pisa_params_t* p, int op, size_t* bytes) {
       if (!decode_supported(g, p->dtype)) return PISA_ERR_UNSUPPORTED;
       *bytes = kStatusBytes + decode_workspace_bytes(g);
       break;
+    case PISA_OP_FORWARD_PACKED: {
+      PackedArena pa;
+      st = packed_arena(p, &pa);
+      if (st != PISA_OK) return st;
+      *bytes = pa.total;
+      break;
+    }
     case PISA_OP_FORWARD_HOST: {
       HostArena a;
       st = host_arena(p, &a);
@@ -701,19 +779,93 @@ int pisa_forward_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32
   st = clear_status(ws, s);
   if (st != PISA_OK) return st;
   const size_t es = elem_size(p->dtype);
-  for (int i = 0; i < nseq; ++i) {
+  auto run_alone = [&](int i) -> int {        // one sequence, unpadded, on the packed tensors themselves
     const size_t t0 = (size_t)cu_seqlens[i];
     const int len = cu_seqlens[i + 1] - cu_seqlens[i];
-    if (len == 0) continue;
+    if (len == 0) return PISA_OK;
     pisa_params_t pi = *p;
     pi.N = len;
     Geometry gi;
-    st = resolve(&pi, &gi);
+    int r = resolve(&pi, &gi);
+    if (r != PISA_OK) return r;
+    return do_forward(&pi, gi, (const char*)q + t0 * g.Hq * g.d * es, (const char*)k + t0 * g.Hkv * g.d * es,
+                      (const char*)v + t0 * g.Hkv * g.d * es, pyramid, idx + t0 * g.Hkv * g.K,
+                      (char*)out + t0 * g.Hq * g.d * es, lse + t0 * g.Hq, ws, ws_bytes, s, /*clear=*/false);
+  };
+  PackedArena pa;
+  st = packed_arena(p, &pa);
+  if (st != PISA_OK) return st;
+  if (ws_bytes < pa.total) {      // a workspace sized for PISA_OP_FORWARD: one sequence after the other
+    for (int i = 0; i < nseq; ++i)
+      if ((st = run_alone(i)) != PISA_OK) return st;
+    return PISA_OK;
+  }
+  char* base = (char*)ws;
+  char* pyr_pad = base + pa.fwd;
+  char* q_pad = pyr_pad + pa.pyr;
+  char* k_pad = q_pad + pa.qb;
+  char* v_pad = k_pad + pa.kb;
+  char* o_pad = v_pad + pa.kb;
+  float* l_pad = (float*)(o_pad + pa.qb);
+  int32_t* i_pad = (int32_t*)((char*)l_pad + pa.lb);
+  // the short sequences, longest first
+  std::vector<int> order;
+  order.reserve((size_t)nseq);
+  for (int i = 0; i < nseq; ++i) {
+    const int len = cu_seqlens[i + 1] - cu_seqlens[i];
+    if (len > kPackDirectLen) {
+      if ((st = run_alone(i)) != PISA_OK) return st;
+    } else if (len > 0) {
+      order.push_back(i);
+    }
+  }
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+    return cu_seqlens[a + 1] - cu_seqlens[a] > cu_seqlens[b + 1] - cu_seqlens[b];
+  });
+  size_t at = 0;
+  while (at < order.size()) {
+    const int first = order[at];
+    const int np = pack_grid_len(cu_seqlens[first + 1] - cu_seqlens[first]);
+    const long long b_cap = pa.tokens / np < 1 ? 1 : pa.tokens / np;
+    size_t end = at + 1;
+    while (end < order.size() && (long long)(end - at) < b_cap) {
+      const int len = cu_seqlens[order[end] + 1] - cu_seqlens[order[end]];
+      if (4LL * len < 3LL * np) break;
+      ++end;
+    }
+    const int nb = (int)(end - at);
+    if (nb == 1) {
+      if ((st = run_alone(first)) != PISA_OK) return st;
+      at = end;
+      continue;
+    }
+    pisa_params_t pg = *p;
+    pg.B = nb;
+    pg.N = np;
+    Geometry gg;
+    if ((st = resolve(&pg, &gg)) != PISA_OK) return st;
+    PackTable tab;
+    for (int b0 = 0; b0 < nb; b0 += kPackSeqs) {
+      tab.n = nb - b0 < kPackSeqs ? nb - b0 : kPackSeqs;
+      for (int j = 0; j < tab.n; ++j) {
+        const int sq = order[at + (size_t)b0 + j];
+        tab.off[j] = cu_seqlens[sq];
+        tab.len[j] = cu_seqlens[sq + 1] - cu_seqlens[sq];
+      }
+      if ((st = launch_pack_gather(gg, (int)es, q, k, v, q_pad, k_pad, v_pad, tab, b0, s)) != PISA_OK) return st;
+    }
+    st = do_forward(&pg, gg, q_pad, k_pad, v_pad, pyr_pad, i_pad, o_pad, l_pad, ws, pa.fwd, s, /*clear=*/false);
     if (st != PISA_OK) return st;
-    st = do_forward(&pi, gi, (const char*)q + t0 * g.Hq * g.d * es, (const char*)k + t0 * g.Hkv * g.d * es,
-                    (const char*)v + t0 * g.Hkv * g.d * es, pyramid, idx + t0 * g.Hkv * g.K,
-                    (char*)out + t0 * g.Hq * g.d * es, lse + t0 * g.Hq, ws, ws_bytes, s, /*clear=*/false);
-    if (st != PISA_OK) return st;
+    for (int b0 = 0; b0 < nb; b0 += kPackSeqs) {
+      tab.n = nb - b0 < kPackSeqs ? nb - b0 : kPackSeqs;
+      for (int j = 0; j < tab.n; ++j) {
+        const int sq = order[at + (size_t)b0 + j];
+        tab.off[j] = cu_seqlens[sq];
+        tab.len[j] = cu_seqlens[sq + 1] - cu_seqlens[sq];
+      }
+      if ((st = launch_pack_scatter(gg, (int)es, o_pad, l_pad, i_pad, out, lse, idx, tab, b0, s)) != PISA_OK) return st;
+    }
+    at = end;
   }
   return PISA_OK;
 }

@@ -68,6 +68,17 @@ int launch_sel_lse_simt(const Geometry& g, int dtype, const void* q, const void*
 int launch_wait_timeout(int32_t* status, unsigned long long limit_ns, cudaStream_t s);
 int num_sms();                        // SM count of the current device
 
+// packed variable-length batches run as padded batches: the copies between the two layouts.
+// A table names up to kPackSeqs sequences (first token in the packed tensors, length); sequence i of the
+// table is batch element b_first + i of the padded tensors [B', g.N, H, d] (g.N = padded length).
+constexpr int kPackSeqs = 384;
+struct PackTable { int n; int off[kPackSeqs]; int len[kPackSeqs]; };
+int launch_pack_gather(const Geometry& g, int elem_bytes, const void* q, const void* k, const void* v, void* q_pad,
+                       void* k_pad, void* v_pad, const PackTable& tab, int b_first, cudaStream_t s);
+int launch_pack_scatter(const Geometry& g, int elem_bytes, const void* out_pad, const float* lse_pad,
+                        const int32_t* idx_pad, void* out, float* lse, int32_t* idx, const PackTable& tab, int b_first,
+                        cudaStream_t s);
+
 // decoding step (one token per sequence); ws points past the status word
 bool decode_supported(const Geometry& g, int dtype);
 size_t decode_workspace_bytes(const Geometry& g);

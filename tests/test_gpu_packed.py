@@ -13,8 +13,15 @@ import paper_2609_31093_b200 as P  # noqa: E402
 from paper_2609_31093_b200 import binding as PB  # noqa: E402
 
 
-def test_packed_sequences_equal_the_sequences_alone_and_the_oracle():
-    lens = [700, 64, 1, 2085, 0, 130, 70000]          # the last one is long enough to run as two chunks
+launches = {}
+
+
+@pytest.mark.parametrize("op", ["forward", "packed"])
+def test_packed_sequences_equal_the_sequences_alone_and_the_oracle(op):
+    """op = "forward": a workspace sized for one sequence (the call then runs the sequences one after the
+    other); "packed": the padded groups (700/640/600 share one, 130/120/100 another, 64/60 a third; 2085, 1
+    and 70000 run alone)."""
+    lens = [700, 64, 1, 2085, 0, 130, 70000, 640, 600, 120, 100, 60]   # 70000: long enough to run as two chunks
     Hq, Hkv, d, C, g, K = 8, 2, 128, 64, 2, 4
     cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
     total = int(cu[-1])
@@ -25,13 +32,18 @@ def test_packed_sequences_equal_the_sequences_alone_and_the_oracle():
     q, k, v = (T.to_torch(cat(x), "bf16") for x in ("q", "k", "v"))          # [total, H, d]
     p = P.Params(1, max(lens), Hq, Hkv, d, C, g, K, dtype="bf16")
     pyramid = PB.alloc_pyramid(p)
-    ws = PB.alloc_workspace(p, PB.OP_FORWARD)
+    ws = PB.alloc_workspace(p, PB.OP_FORWARD_PACKED if op == "packed" else PB.OP_FORWARD)
+    assert P.workspace_bytes(p, PB.OP_FORWARD_PACKED) > P.workspace_bytes(p, PB.OP_FORWARD)
     idx = torch.full((Hkv * K * total,), -7, dtype=torch.int32, device="cuda")
     out = torch.zeros_like(q)
     lse = torch.zeros((Hq * total,), dtype=torch.float32, device="cuda")
+    n0 = P.launch_count()
     P.pisa_forward_packed(p, cu.tolist(), q, k, v, pyramid, idx, out, lse, ws)
     torch.cuda.synchronize()
     assert P.read_status(ws) == 0
+    launches[op] = P.launch_count() - n0
+    if len(launches) == 2:
+        assert launches["packed"] < launches["forward"]
     for i, n in enumerate(lens):
         if n == 0:
             continue
@@ -43,10 +55,17 @@ def test_packed_sequences_equal_the_sequences_alone_and_the_oracle():
         assert alone.sync_status() == 0
         got_idx = idx[Hkv * K * t0:Hkv * K * (t0 + n)].view(Hkv, n, K)
         got_lse = lse[Hq * t0:Hq * (t0 + n)].view(Hq, n)
-        assert torch.equal(got_idx, alone.idx[0]), i
-        assert torch.allclose(got_lse, alone.lse[0], rtol=1e-5, atol=1e-5), i
-        a, b = out[t0:t0 + n].double(), alone.out[0].double()
-        assert bool(((a - b).abs() <= 2.0 ** -7 * b.abs() + 1e-3).all()), i
+        if op == "forward":
+            assert torch.equal(got_idx, alone.idx[0]), i
+        else:                                   # other tile compositions: rows may differ only inside the tie band
+            differ = (got_idx != alone.idx[0]).any(dim=-1)
+            assert int(differ.sum()) <= max(1, got_idx.shape[0] * n // 200), (i, int(differ.sum()))
+        same = ~(got_idx != alone.idx[0]).any(dim=-1)                       # [Hkv, n] rows with equal index sets
+        same_q = same.repeat_interleave(Hq // Hkv, dim=0)                     # [Hq, n]
+        assert bool((((got_lse - alone.lse[0]).abs() <= 1e-5 * alone.lse[0].abs() + 1e-5) | ~same_q).all()), i
+        a, b = out[t0:t0 + n].double(), alone.out[0].double()                 # [n, Hq, d]
+        ok = ((a - b).abs() <= 2.0 ** -7 * b.abs() + 1e-3).all(dim=-1)
+        assert bool((ok | ~same_q.t()).all()), i
         # sampled rows of this sequence against the oracle
         tri = S.sample_queries(w, 12)
         prob = T.oracle_problem(w, t)
@@ -103,3 +122,60 @@ def test_packed_backward_matches_the_oracle_per_sequence():
             g64 = got[t0:t0 + n].to(torch.float64).cpu().numpy()[None]
             assert np.isfinite(g64).all(), (i, nm)
             T.check_gradient_rows(f"seq{i}.{nm}", g64, ref, extra)
+
+
+def test_many_short_sequences_run_as_a_few_launch_sets():
+    """256 sequences of at most 512 tokens: the padded groups against the one-after-the-other loop of the
+    same call (same rows up to tie-band differences, far fewer launches, less time), and sampled rows of
+    sampled sequences against the oracle run on each sequence alone."""
+    rng = np.random.default_rng(4242)
+    lens = rng.integers(1, 513, size=256).tolist()
+    Hq, Hkv, d, C, g, K = 8, 2, 128, 64, 2, 4
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    total = int(cu[-1])
+    w_all = S.Workload("pk_many", 1, total, Hq, Hkv, d, C, g, K, "bf16", 4243, "iid")
+    t_all = S.make_inputs(w_all)
+    q, k, v = (T.to_torch(t_all[x][0], "bf16") for x in ("q", "k", "v"))      # [total, H, d]
+    p = P.Params(1, max(lens), Hq, Hkv, d, C, g, K, dtype="bf16")
+    pyramid = PB.alloc_pyramid(p)
+    res = {}
+    for op in ("forward", "packed"):
+        ws = PB.alloc_workspace(p, PB.OP_FORWARD_PACKED if op == "packed" else PB.OP_FORWARD)
+        idx = torch.full((Hkv * K * total,), -7, dtype=torch.int32, device="cuda")
+        out = torch.zeros_like(q)
+        lse = torch.zeros((Hq * total,), dtype=torch.float32, device="cuda")
+        P.pisa_forward_packed(p, cu.tolist(), q, k, v, pyramid, idx, out, lse, ws)      # warm-up
+        torch.cuda.synchronize()
+        n0 = P.launch_count()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        P.pisa_forward_packed(p, cu.tolist(), q, k, v, pyramid, idx, out, lse, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        assert P.read_status(ws) == 0
+        res[op] = (idx, out, lse, P.launch_count() - n0, e0.elapsed_time(e1))
+    print(f"\n256 sequences <= 512 tokens ({total} tokens): loop {res['forward'][3]} launches {res['forward'][4]:.2f} ms, "
+          f"padded groups {res['packed'][3]} launches {res['packed'][4]:.2f} ms")
+    assert res["packed"][3] * 4 < res["forward"][3]
+    assert res["packed"][4] < res["forward"][4]
+    # the two modes against each other: index rows equal except inside the tie band
+    ia, ib = res["forward"][0].view(-1, K), res["packed"][0].view(-1, K)
+    differ = (ia != ib).any(dim=-1)
+    assert int(differ.sum()) <= ia.shape[0] // 200, int(differ.sum())
+    assert int((res["packed"][0] == -7).sum()) == 0                               # every row was written
+    # sampled sequences against the oracle on the sequence alone
+    idx, out, lse = res["packed"][:3]
+    for i in rng.choice(256, size=12, replace=False).tolist() + [int(np.argmax(lens)), int(np.argmin(lens))]:
+        n, t0 = lens[i], int(cu[i])
+        w = S.Workload(f"pk_many{i}", 1, n, Hq, Hkv, d, C, g, K, "bf16", 0, "iid")
+        t = {key: t_all[key][:, t0:t0 + n] for key in ("q", "k", "v")}
+        tri = S.sample_queries(w, 8)
+        prob = T.oracle_problem(w, t)
+        ti = torch.from_numpy(tri)
+        got_idx = idx[Hkv * K * t0:Hkv * K * (t0 + n)].view(Hkv, n, K)
+        gi = got_idx.cpu()[ti[:, 1], ti[:, 2]].numpy()
+        G = Hq // Hkv
+        heads = ti[:, 1:2] * G + torch.arange(G)[None, :]
+        o_g = out[t0:t0 + n].cpu()[ti[:, 2:3], heads].double().numpy()            # [S, G, d]
+        l_g = lse[Hq * t0:Hq * (t0 + n)].view(Hq, n).cpu()[heads, ti[:, 2:3]].double().numpy()
+        T.check_forward_rows(w, prob, tri, gi, o_g, l_g)
