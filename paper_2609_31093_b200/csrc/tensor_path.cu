@@ -262,10 +262,9 @@ __device__ __forceinline__ int find_key(const int32_t* tile_off, int nkeys, int 
   return lo;
 }
 
-// Work items of the attention kernel are handed out dynamically: lists differ in length, and a static
-// round-robin left the CTAs' tile counts 20 % apart (the leaf-scoring kernel keeps the static walk: its
-// epilogue warps sit at their register limit, and routing the item descriptions through shared memory
-// cost it more in spills than the balance gained).  Thread 0 of the CTA draws the next item from a global counter when the
+// Work items of both tile kernels are handed out dynamically: lists differ in length, and a static
+// round-robin left the CTAs' tile counts 20 % apart.  The leaf-scoring kernel has a scheduler warp of its own
+// (see there).  In the attention kernel thread 0 of the CTA draws the next item from a global counter when the
 // producers start their k-th item and publishes it in a small shared-memory ring; every other role reads
 // the k-th entry when it gets there (it lags the producers by a few items at most: the producers cannot
 // start item k before the UMMAs of item k - 1 have completed).  An id >= the item count ends the walk.
@@ -296,11 +295,12 @@ __device__ __forceinline__ float ex2_approx(float x) {
 
 // Online log-sum-exp (base 2) over one 32-column chunk of raw fp32 logits; (m, ssum) is the running
 // (max, sum of 2^(x - max)) with x = raw * sl2.  sl2 > 0, so the max commutes with the scaling.
-__device__ __forceinline__ void lse_chunk(const uint32_t (&rr)[32], float sl2, float& m, float& ssum) {
+template <int NW>
+__device__ __forceinline__ void lse_chunk(const uint32_t (&rr)[NW], float sl2, float& m, float& ssum) {
   float c0 = __uint_as_float(rr[0]), c1 = __uint_as_float(rr[1]);
   float c2 = __uint_as_float(rr[2]), c3 = __uint_as_float(rr[3]);
 #pragma unroll
-  for (int j = 4; j < 32; j += 4) {
+  for (int j = 4; j < NW; j += 4) {
     c0 = fmaxf(c0, __uint_as_float(rr[j]));
     c1 = fmaxf(c1, __uint_as_float(rr[j + 1]));
     c2 = fmaxf(c2, __uint_as_float(rr[j + 2]));
@@ -310,7 +310,7 @@ __device__ __forceinline__ void lse_chunk(const uint32_t (&rr)[32], float sl2, f
   const float neg = -mn;
   float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-  for (int j = 0; j < 32; j += 4) {
+  for (int j = 0; j < NW; j += 4) {
     a0 += ex2_approx(fmaf(__uint_as_float(rr[j]), sl2, neg));
     a1 += ex2_approx(fmaf(__uint_as_float(rr[j + 1]), sl2, neg));
     a2 += ex2_approx(fmaf(__uint_as_float(rr[j + 2]), sl2, neg));
@@ -323,27 +323,29 @@ __device__ __forceinline__ void lse_chunk(const uint32_t (&rr)[32], float sl2, f
 // exactly as in lse_chunk (four interleaved accumulators), so a full row gives bit-identical results on
 // either path: which path a row takes depends on the other rows of its tile, and the composition of a
 // tile (the order of a list's entries) varies from run to run.
-__device__ __forceinline__ void lse_chunk_masked(const uint32_t (&rr)[32], int nvalid, float sl2, float& m,
+template <int NW>
+__device__ __forceinline__ void lse_chunk_masked(const uint32_t (&rr)[NW], int nvalid, float sl2, float& m,
                                                  float& ssum) {
   float cm = -CUDART_INF_F;
 #pragma unroll
-  for (int j = 0; j < 32; ++j)
+  for (int j = 0; j < NW; ++j)
     if (j < nvalid) cm = fmaxf(cm, __uint_as_float(rr[j]));
   const float mn = fmaxf(m, cm * sl2);
   const float neg = -mn;
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-  for (int j = 0; j < 32; ++j)
+  for (int j = 0; j < NW; ++j)
     if (j < nvalid) acc[j & 3] += ex2_approx(fmaf(__uint_as_float(rr[j]), sl2, neg));
   ssum = ssum * ex2_approx(m - mn) + ((acc[0] + acc[1]) + (acc[2] + acc[3]));
   m = mn;
 }
 // first and second moments of the first `nvalid` of 32 logits about `shift` (score modes "mean" and
 // "mean + variance/2", Sec. 4.3)
-__device__ __forceinline__ void stat_chunk(const uint32_t (&rr)[32], int nvalid, float scale, float shift, float& s1,
+template <int NW>
+__device__ __forceinline__ void stat_chunk(const uint32_t (&rr)[NW], int nvalid, float scale, float shift, float& s1,
                                            float& s2) {
 #pragma unroll
-  for (int j = 0; j < 32; ++j)
+  for (int j = 0; j < NW; ++j)
     if (j < nvalid) {
       const float dlt = fmaf(__uint_as_float(rr[j]), scale, -shift);
       s1 += dlt;
@@ -353,15 +355,18 @@ __device__ __forceinline__ void stat_chunk(const uint32_t (&rr)[32], int nvalid,
 
 // ------------------------------------------------------------------ warp-specialised tile kernels
 //
-// One CTA per SM, thirteen warps: warps 0-3 stage operands (16-byte cp.async into the swizzled
-// layouts, a ring of NS query tiles; the block's keys/values ride with the first tile of a work item),
-// warp 4 issues the UMMA chains, warps 5-8 and 9-12 are two epilogue groups that take alternate tiles, each
-// on its own TMEM accumulator, so that the exponentials of one tile overlap the gathers and the MMAs
-// of the next.  Every role walks the same deterministic sequence of (work item, tile) and derives
-// ring slots and mbarrier parities from its own tile counter; all waits are time-bounded.
+// One persistent CTA per SM.  Producer warps stage the gathered query rows (16-byte cp.async into the
+// swizzled layouts, a ring of NS query tiles; the block's keys / values arrive by TMA tile loads with the
+// first tile of a work item), one warp issues the UMMA chains into two alternating TMEM accumulators, the
+// remaining warps read the accumulators out.  Every role derives ring slots and mbarrier parities from its
+// own tile counter; all waits are bounded.
 
-constexpr int kWsThreads = 416;        // 4 producer warps, 1 MMA warp, 2 x 4 epilogue warps
-constexpr int kLseThreads = 672;       // 4 producer warps, 1 MMA warp, 2 x 8 epilogue warps
+// leaf scoring: 4 producer warps, 1 UMMA warp, 1 scheduler warp, 16 epilogue warps.  22 warps put six on two of
+// the SM's sub-partitions, i.e. 80 registers per thread (as 21 warps did); more producer warps measured slower
+// (the gather is limited by the bytes the four ring slots keep in flight, not by the warps that issue it)
+constexpr int kLseProd = 128;
+constexpr int kLseThreads = kLseProd + 64 + 512;
+constexpr int kLseRing = 16;           // tiles the scheduler warp may run ahead of the epilogue
 constexpr int kProdThreads = 128;
 constexpr int kMetaRing = 8;           // ring of per-tile metadata; deeper than any role can run ahead
 
@@ -476,26 +481,37 @@ __device__ __forceinline__ bool prod_sync_or(bool flag) {
 // MOM: false = per-head LSE of every leaf; true = first / second moments of the logits (score modes
 // "mean" and "mean + variance/2"), a separate instantiation so that the LSE one keeps its registers.
 template <int D, int NB, bool MOM>
-__global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, TileArgs a, const __grid_constant__ CUtensorMap tm_k) {
+__global__ void __launch_bounds__(kLseThreads, 1)
+lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant__ CUtensorMap tm_k) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int NS = 4;
   constexpr int KS = D / 64;
   constexpr int A_SLAB = 128 * 128, B_SLAB = NB * 128;
   constexpr int A_STAGE = KS * A_SLAB;
   constexpr uint32_t TM_COLS = (2 * NB < 32) ? 32 : 2 * NB;
+  constexpr int R = kLseRing;
+  constexpr int W = NB / 4;                       // accumulator columns of one epilogue warp
+  constexpr int CW = (W < 32) ? W : 32;           // columns per TMEM load
   uint8_t* smem = align1024(smem_raw);
   uint8_t* sA = smem;
   uint8_t* sB = smem + NS * A_STAGE;
   __shared__ uint64_t a_full[NS], a_empty[NS], b_full, b_empty, t_full[2], t_empty[2];
+  __shared__ uint64_t m_full[R], m_empty[R];      // the tile ring: written by the scheduler warp, released by the epilogue
+  __shared__ int s_tent[R][128];                  // a tile's entries (token | slot << 24, -1 = none)
+  __shared__ int4 s_tkey[R];                      // its (unit, node, flags: 1 = first tile of a work item, 2 = last)
+  __shared__ float4 s_part[2][16][32];            // partial results of the warps that share a leaf (by tile parity)
+  __shared__ volatile int s_total;                // number of tiles of this CTA, known once the walk has ended
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_fail;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
-    for (int i = 0; i < NS; ++i) { mbar_init(&a_full[i], kProdThreads); mbar_init(&a_empty[i], 1); }
+    s_total = 0x7fffffff;
+    for (int i = 0; i < NS; ++i) { mbar_init(&a_full[i], kLseProd); mbar_init(&a_empty[i], 1); }
     mbar_init(&b_empty, 1);
     mbar_init(&b_full, 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 256); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 512); }
+    for (int i = 0; i < R; ++i) { mbar_init(&m_full[i], 1); mbar_init(&m_empty[i], 16); }
     s_fail = 0;
     mbar_fence_init();
   }
@@ -506,156 +522,229 @@ __global__ void __launch_bounds__(kLseThreads, 1) lse_ws_kernel(Geometry geo, Ti
   const uint32_t tmem = tmem_slot;
 
   const int G = geo.G, lgG = 31 - __clz(G), tpt = 128 >> lgG, C = geo.C;
-  const int n_items = a.item_off[a.nkeys];
   const float sl2 = geo.scale * kLog2e;
 
-  if (warp < 4) {
-    // ------------------------------------------------ producers
-    // The four producer warps run independently of one another: a thread reads the entries of the
-    // rows it copies straight from the list (one tile ahead, from a clamped -- always readable --
-    // address; validity is decided when the tile comes up, so nothing waits on the loads).
-    constexpr int CH = D / 8, RPP = kProdThreads / CH, RPT = 128 / RPP;
-    const int rb = tid / CH;
-    int it = 0, kiter = 0;
-    bool stop = false;
-    for (int item = blockIdx.x; item < n_items && !stop; item += gridDim.x, ++kiter) {
-      const ItemInfo inf = item_info(a, item, tpt);
-      const int bh = inf.key / (a.NW * a.Mk), j = inf.key % a.Mk;
-      const int b = bh / geo.Hkv, h = bh % geo.Hkv;
-      const int e_last = inf.e_end - 1;
-      int nxt[RPT];
-#pragma unroll
-      for (int i = 0; i < RPT; ++i) nxt[i] = a.entries[min(inf.e_begin + ((rb + i * RPP) >> lgG), e_last)];
-      // the previous item's MMAs must have released the key tile
-      bool ok = s_fail == 0;
-      if (ok && kiter > 0) ok = mbar_wait_bounded(&b_empty, (uint32_t)((kiter - 1) & 1));
-      if (!__all_sync(0xffffffffu, ok)) { s_fail = 1; stop = true; break; }
-      if (tid == 0) {                             // the node's keys: one TMA tile load per 64-wide slab (own memory, no multicast)
+  // Every role but the scheduler walks TILES: it waits for tile `it`'s ring entry (or its accumulator) and
+  // leaves when the scheduler has published the tile count and `it` has reached it.  A try_wait suspends the
+  // warp for a while, so the poll count bounds the wait to seconds.
+  auto wait_tile = [&](uint64_t* bar, uint32_t parity, int it) -> bool {
+    for (uint32_t i = 0; i < (1u << 24); ++i) {
+      if (mbar_try_wait(bar, parity)) return true;
+      if (it >= s_total || s_fail) return false;
+    }
+    s_fail = 1;
+    return false;
+  };
+
+  if (warp < kLseProd / 32) {
+    // ------------------------------------------------ producers: gather the tile's query rows
+    constexpr int CH = D / 8, RPP = kLseProd / CH;
+    const int ck = tid % CH, rb = tid / CH;
+    int n_item = 0;
+    for (int it = 0;; ++it) {
+      const int mr = it % R, s = it % NS;
+      if (!wait_tile(&m_full[mr], (uint32_t)((it / R) & 1), it)) break;
+      const int4 key = s_tkey[mr];
+      if (tid == 0 && (key.z & 1)) {
+        // first tile of a work item: the node's keys, one TMA tile load per 64-wide slab (own memory, no
+        // multicast), once the previous item's MMAs have released the buffer
+        if (n_item > 0 && !mbar_wait_bounded(&b_empty, (uint32_t)((n_item - 1) & 1))) { s_fail = 1; break; }
+        ++n_item;
+        const int b = key.x / geo.Hkv, h = key.x % geo.Hkv;
         mbar_arrive_expect_tx(&b_full, (uint32_t)(KS * B_SLAB));
-        for (int ks = 0; ks < KS; ++ks) tma_load_4d(smem_u32(sB + ks * B_SLAB), &tm_k, &b_full, ks * 64, h, j * NB, b);
+        for (int ks = 0; ks < KS; ++ks) tma_load_4d(smem_u32(sB + ks * B_SLAB), &tm_k, &b_full, ks * 64, h, key.y * NB, b);
       }
-      const __nv_bfloat16* qb = a.q + (long long)b * geo.qs[0] + (long long)(h * G) * geo.qs[2];
-      for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
-        const int s = it % NS;
-        ok = it < NS || mbar_wait_bounded(&a_empty[s], (uint32_t)((it / NS - 1) & 1));
-        if (!__all_sync(0xffffffffu, ok)) { s_fail = 1; stop = true; break; }
-        const int e0 = inf.e_begin + jt * tpt;
-        int cur[RPT];
-#pragma unroll
-        for (int i = 0; i < RPT; ++i) {
-          const int slot_i = (rb + i * RPP) >> lgG;
-          cur[i] = (e0 + slot_i < inf.e_end) ? checked_entry(a, geo.N, nxt[i]) : -1;
-          nxt[i] = a.entries[min(e0 + tpt + slot_i, e_last)];
-        }
-        prod_gather_q_regs<D>(sA + s * A_STAGE, geo, qb, cur, tid);
-        fence_proxy_async_smem();                 // zero-filled rows (plain stores) -> async proxy
-        cp_async_arrive_noinc(&a_full[s]);        // fires when this thread's copies have landed
+      if (it >= NS && !mbar_wait_bounded(&a_empty[s], (uint32_t)((it / NS - 1) & 1))) { s_fail = 1; break; }
+      const int b = key.x / geo.Hkv, h = key.x % geo.Hkv;
+      const __nv_bfloat16* src0 = a.q + (long long)b * geo.qs[0] + (long long)(h * G) * geo.qs[2] + ck * 8;
+      const long long s1 = geo.qs[1], s2 = geo.qs[2];
+      const uint32_t d0 = smem_u32(sA + s * A_STAGE + (ck >> 3) * A_SLAB);
+      const int* ents = s_tent[mr];
+#pragma unroll 4
+      for (int row = rb; row < 128; row += RPP) {       // RPP need not be a multiple of 8: the swizzle is per row
+        const int ent = ents[row >> lgG];
+        const uint32_t d = d0 + swz128(row, ck & 7);
+        if (ent >= 0) cp_async16(d, src0 + (long long)(ent & 0xFFFFFF) * s1 + (long long)(row & (G - 1)) * s2);
+        else st_shared_zero16(d);
       }
+      fence_proxy_async_smem();                 // zero-filled rows (plain stores) -> async proxy
+      cp_async_arrive_noinc(&a_full[s]);        // fires when this thread's copies have landed
     }
     cp_async_wait_all();
-  } else if (warp == 4) {
+  } else if (warp == kLseProd / 32) {
     // ------------------------------------------------ MMA issuer (the warp walks the loop, lane 0 issues)
     const uint32_t idesc = make_idesc_bf16(128, NB, 0, 0);
-    int it = 0, kit = 0;
-    for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x, ++kit) {
-      const ItemInfo inf = item_info(a, item, tpt);
-      bool ok = mbar_wait_bounded(&b_full, (uint32_t)(kit & 1));      // the node's keys have landed
-      for (int jt = 0; jt < inf.ntiles && ok; ++jt, ++it) {
-        const int s = it % NS, buf = it & 1;
-        ok = mbar_wait_bounded(&a_full[s], (uint32_t)((it / NS) & 1));
-        if (ok && it >= 2) ok = mbar_wait_bounded(&t_empty[buf], (uint32_t)(((it >> 1) - 1) & 1));
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        if (lane == 0) {
-          fence_proxy_async_smem();
-          tcgen05_fence_after_sync();
-          const uint32_t a0 = smem_u32(sA + s * A_STAGE), b0 = smem_u32(sB);
-#pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint64_t da = make_smem_desc(a0 + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
-            const uint64_t db = make_smem_desc(b0 + (kk >> 2) * B_SLAB + (kk & 3) * 32, 0, 1024);
-            umma_bf16(tmem + (uint32_t)(buf * NB), da, db, idesc, kk > 0);
-          }
-          umma_commit(&a_empty[s]);
-          umma_commit(&t_full[buf]);
-        }
-        __syncwarp();
-      }
+    int n_item = 0;
+    for (int it = 0;; ++it) {
+      const int mr = it % R, s = it % NS, buf = it & 1;
+      if (!wait_tile(&m_full[mr], (uint32_t)((it / R) & 1), it)) break;
+      const int flags = s_tkey[mr].z;
+      bool ok = true;
+      if (flags & 1) ok = mbar_wait_bounded(&b_full, (uint32_t)(n_item & 1));                // the node's keys have landed
+      if (ok) ok = mbar_wait_bounded(&a_full[s], (uint32_t)((it / NS) & 1));
+      if (ok && it >= 2) ok = mbar_wait_bounded(&t_empty[buf], (uint32_t)(((it >> 1) - 1) & 1));
+      ok = __all_sync(0xffffffffu, ok);
       if (!ok) { s_fail = 1; break; }
-      if (lane == 0) umma_commit(&b_empty);
+      if (lane == 0) {
+        fence_proxy_async_smem();
+        tcgen05_fence_after_sync();
+        const uint32_t a0 = smem_u32(sA + s * A_STAGE), b0 = smem_u32(sB);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint64_t da = make_smem_desc(a0 + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
+          const uint64_t db = make_smem_desc(b0 + (kk >> 2) * B_SLAB + (kk & 3) * 32, 0, 1024);
+          umma_bf16(tmem + (uint32_t)(buf * NB), da, db, idesc, kk > 0);
+        }
+        umma_commit(&a_empty[s]);
+        umma_commit(&t_full[buf]);
+        if (flags & 2) umma_commit(&b_empty);        // last tile of the item: its MMAs release the keys
+      }
+      if (flags & 2) ++n_item;
       __syncwarp();
     }
-  } else {
-    // ------------------------------------------------ epilogue groups
-    // eight warps per group: two warps share each TMEM lane quarter and split the tile's children
-    const int ew = warp - 5;
-    const int grp = ew >> 3;                            // 0: even tiles, 1: odd tiles
-    const int half = (ew >> 2) & 1;
-    const int row = (warp & 3) * 32 + lane;             // TMEM lane quarter of this warp = warp % 4
-    const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(grp * NB);
-    const int head = row & (G - 1);
-    const int r_lo = (a.fan >= 2) ? half * (a.fan / 2) : 0;
-    const int r_hi = (a.fan >= 2) ? ((half == 1) ? a.fan : a.fan / 2) : (half == 0 ? 1 : 0);
-    constexpr bool lse_mode = !MOM;
+  } else if (warp == kLseProd / 32 + 1) {
+    // ------------------------------------------------ scheduler: draws work items, lays out their tiles
+    // Lists differ in length, so the items are handed out dynamically from a global counter (zero on entry).
+    // The warp runs up to R tiles ahead of the epilogue: the latency of the draw, of the item's description
+    // and of the entries' loads stays off every other role's path.
+    const int n_items = a.item_off[a.nkeys];
     int it = 0;
-    for (int item = blockIdx.x; item < n_items && !s_fail; item += gridDim.x) {
+    bool ok = true;
+    while (ok) {
+      int item = 0;
+      if (lane == 0) item = atomicAdd(work_ctr, 1);
+      item = __shfl_sync(0xffffffffu, item, 0);
+      if (item >= n_items) break;
       const ItemInfo inf = item_info(a, item, tpt);
       const int bh = inf.key / (a.NW * a.Mk), j = inf.key % a.Mk;
-      for (int jt = 0; jt < inf.ntiles; ++jt, ++it) {
-        if ((it & 1) != grp) continue;
-        const int e_row = inf.e_begin + jt * tpt + (row >> lgG);
-        const int ent_raw = a.entries[min(e_row, inf.e_end - 1)];
-        if (!mbar_wait_bounded(&t_full[grp], (uint32_t)((it >> 1) & 1))) { s_fail = 1; break; }
-        tcgen05_fence_after_sync();
-        const int ent = (e_row < inf.e_end) ? checked_entry(a, geo.N, ent_raw) : -1;
-        const bool valid = ent >= 0;
-        const int t = ent & 0xFFFFFF, slot = valid ? (ent >> 24) : 0;
-        const int c_t = t / C;
-        for (int r = r_lo; r < r_hi; ++r) {
-          const int leaf = j * a.fan + r;
-          int ncols = 0;
-          if (valid && leaf <= c_t && leaf < geo.M[1])
-            ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
-          const bool fast = __all_sync(0xffffffffu, ncols == C || ncols == 0);
-          float m = -CUDART_INF_F, ssum = 0.f;
-          float shift = 0.f, s1 = 0.f, s2 = 0.f;          // moment modes: logits about the first one
-          uint32_t ra[32], rb[32];
-          const uint32_t col0 = lane_base + (uint32_t)(r * C);
-          tmem_ld_32x32(col0, ra);
-          for (int c0 = 0; c0 < C; c0 += 64) {
-            tmem_ld_wait();
-            tmem_ld_32x32(col0 + (uint32_t)(c0 + 32), rb);
-            if (!lse_mode) {
-              if (c0 == 0) shift = __uint_as_float(ra[0]) * geo.scale;
-              if (c0 < ncols) stat_chunk(ra, ncols - c0, geo.scale, shift, s1, s2);
-            } else if (fast) lse_chunk(ra, sl2, m, ssum);
-            else if (c0 < ncols) lse_chunk_masked(ra, ncols - c0, sl2, m, ssum);
-            tmem_ld_wait();
-            if (c0 + 64 < C) tmem_ld_32x32(col0 + (uint32_t)(c0 + 64), ra);
-            else if (r + 1 == r_hi) {
-              // the last chunk of this warp's share is in registers: the accumulator can be refilled
-              // while it is being reduced
-              tcgen05_fence_before_sync();
-              mbar_arrive(&t_empty[grp]);
-            }
-            if (!lse_mode) {
-              if (c0 + 32 < ncols) stat_chunk(rb, ncols - c0 - 32, geo.scale, shift, s1, s2);
-            } else if (fast) lse_chunk(rb, sl2, m, ssum);
-            else if (c0 + 32 < ncols) lse_chunk_masked(rb, ncols - c0 - 32, sl2, m, ssum);
+      // the entries of four tiles are fetched together: one round trip to L2 per four tiles, not per tile
+      constexpr int TB = 4, TPL = 4;                       // tiles per batch; entries per lane and tile (tpt <= 128)
+      for (int jt0 = 0; jt0 < inf.ntiles && ok; jt0 += TB) {
+        int ent[TB][TPL];
+#pragma unroll
+        for (int u = 0; u < TB; ++u)
+#pragma unroll
+          for (int x = 0; x < TPL; ++x) {
+            const int p = lane + 32 * x, e = inf.e_begin + (jt0 + u) * tpt + p;
+            ent[u][x] = (p < tpt && e < inf.e_end) ? a.entries[e] : -1;
           }
-          if (valid) {
-            float lse = (ncols > 0) ? (m + log2f(ssum)) * kLn2 : -CUDART_INF_F;
-            if (!lse_mode && ncols > 0) {
-              const float inv_n = 1.f / (float)ncols, mu = s1 * inv_n;
-              lse = shift + mu + ((a.mode == PISA_SCORE_MEAN_VAR) ? 0.5f * fmaxf(s2 * inv_n - mu * mu, 0.f) : 0.f);
+#pragma unroll
+        for (int u = 0; u < TB; ++u) {
+          const int jt = jt0 + u;
+          if (jt >= inf.ntiles) break;
+          const int mr = it % R;
+          if (it >= R) ok = mbar_wait_bounded(&m_empty[mr], (uint32_t)((it / R - 1) & 1));
+          ok = __all_sync(0xffffffffu, ok && !s_fail);
+          if (!ok) break;
+#pragma unroll
+          for (int x = 0; x < TPL; ++x)
+            if (lane + 32 * x < tpt) s_tent[mr][lane + 32 * x] = checked_entry(a, geo.N, ent[u][x]);
+          if (lane == 0) s_tkey[mr] = make_int4(bh, j, (jt == 0 ? 1 : 0) | (jt == inf.ntiles - 1 ? 2 : 0), 0);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&m_full[mr]);     // release: the ring entry is complete
+          ++it;
+        }
+      }
+    }
+    if (!ok) s_fail = 1;
+    if (lane == 0) s_total = it;
+  } else {
+    // ------------------------------------------------ epilogue: sixteen warps on every tile
+    // Four warps share each TMEM lane quarter and split the accumulator's NB columns, W = NB / 4 each -- few
+    // enough to hold in registers.  A warp therefore reads its columns out at once and releases the
+    // accumulator BEFORE it starts on the exponentials: the next-but-one tile's UMMAs never wait for
+    // arithmetic.  A leaf wider than W is shared by C / W warps of the quarter; they leave their partial
+    // (max, sum) in shared memory and the first of them combines (always in the same order).
+    const int ew = warp - (kLseProd / 32 + 2);
+    const int cq = ew >> 2;                             // column quarter; warp % 4 = TMEM lane quarter
+    const int row = (warp & 3) * 32 + lane;
+    const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(cq * W);
+    const int head = row & (G - 1);
+    const int wpl = C / W;                              // warps per leaf (C >= W: at most four children per node)
+    const int r = (cq * W) / C;                         // the child this warp's columns belong to
+    const int off = cq * W - r * C;                     // its first column inside that child
+    const bool owner = (cq % wpl) == 0;
+    const int bar_id = 1 + (warp & 3) * 2 + ((wpl == 2) ? (cq >> 1) : 0);
+    constexpr bool lse_mode = !MOM;
+    for (int it = 0;; ++it) {
+      const int buf = it & 1;
+      if (!wait_tile(&t_full[buf], (uint32_t)((it >> 1) & 1), it)) break;
+      tcgen05_fence_after_sync();
+      uint32_t ra[CW], rb[CW];
+      if constexpr (W == 16) {
+        tmem_ld_32x16(lane_base + (uint32_t)(buf * NB), ra);
+      } else {
+        tmem_ld_32x32(lane_base + (uint32_t)(buf * NB), ra);
+        if constexpr (W == 64) tmem_ld_32x32(lane_base + (uint32_t)(buf * NB + 32), rb);
+      }
+      tmem_ld_wait();
+      tcgen05_fence_before_sync();
+      mbar_arrive(&t_empty[buf]);                       // this thread's columns are in registers
+      const int mr = it % R;
+      const int ent = s_tent[mr][row >> lgG];
+      const int bh = s_tkey[mr].x, j = s_tkey[mr].y;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&m_empty[mr]);         // this warp has read the ring entry
+      const bool valid = ent >= 0;
+      const int t = ent & 0xFFFFFF, slot = valid ? (ent >> 24) : 0;
+      const int c_t = t / C;
+      const int leaf = j * a.fan + r;
+      int ncols = 0;                                    // causally visible columns of the child for this row
+      if (valid && leaf <= c_t && leaf < geo.M[1])
+        ncols = (leaf == c_t) ? (t - leaf * C + 1) : min(C, geo.N - leaf * C);
+      const int nv = max(0, min(W, ncols - off));       // ... of them inside this warp's columns
+      const bool fast = __all_sync(0xffffffffu, nv == W || nv == 0);
+      float m = -CUDART_INF_F, ssum = 0.f;
+      float shift = 0.f, s1 = 0.f, s2 = 0.f;            // moment modes: logits about the warp's first one
+      if (!lse_mode) {
+        shift = __uint_as_float(ra[0]) * geo.scale;
+        if (nv > 0) stat_chunk<CW>(ra, nv, geo.scale, shift, s1, s2);
+        if constexpr (W == 64) if (nv > 32) stat_chunk<CW>(rb, nv - 32, geo.scale, shift, s1, s2);
+      } else if (fast) {
+        lse_chunk<CW>(ra, sl2, m, ssum);
+        if constexpr (W == 64) lse_chunk<CW>(rb, sl2, m, ssum);
+      } else {
+        if (nv > 0) lse_chunk_masked<CW>(ra, nv, sl2, m, ssum);
+        if constexpr (W == 64) if (nv > 32) lse_chunk_masked<CW>(rb, nv - 32, sl2, m, ssum);
+      }
+      if (nv == 0) { m = -CUDART_INF_F; ssum = 0.f; }   // (the unmasked path ran on this row's columns all the same)
+      // partial of this warp: LSE mode (m, ssum); moment modes (count, mean, M2 = sum of squared deviations)
+      float4 part;
+      if (lse_mode) {
+        part = make_float4(m, ssum, 0.f, 0.f);
+      } else {
+        const float n = (float)nv, mu_d = (nv > 0) ? s1 / n : 0.f;
+        part = make_float4(n, shift + mu_d, fmaxf(s2 - s1 * mu_d, 0.f), 0.f);
+      }
+      if (wpl > 1) {
+        s_part[buf][ew][lane] = part;
+        asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(wpl * 32) : "memory");
+        if (owner) {
+          for (int i = 1; i < wpl; ++i) {
+            const float4 o = s_part[buf][ew + 4 * i][lane];
+            if (lse_mode) {
+              const float mn = fmaxf(part.x, o.x);
+              const float sa = (part.x == mn) ? part.y : part.y * ex2_approx(part.x - mn);
+              const float sb = (o.x == mn) ? o.y : o.y * ex2_approx(o.x - mn);
+              part.x = mn;
+              part.y = sa + sb;
+            } else if (o.x > 0.f) {
+              const float n = part.x + o.x, dl = o.y - part.y;
+              part.z = part.z + o.z + dl * dl * (part.x * o.x / n);
+              part.y = part.y + dl * (o.x / n);
+              part.x = n;
             }
-            a.blk_lse[(((long long)bh * geo.N + t) * (a.slots * a.fan) + slot * a.fan + r) * G + head] = lse;
           }
         }
-        if (r_lo >= r_hi) {              // a warp without a share of this tile still counts as an arrival
-          tcgen05_fence_before_sync();
-          mbar_arrive(&t_empty[grp]);
+      }
+      if (valid && owner) {
+        float lse;
+        if (lse_mode) {
+          lse = (ncols > 0) ? (part.x + log2f(part.y)) * kLn2 : -CUDART_INF_F;
+        } else {
+          lse = (ncols > 0) ? part.y + ((a.mode == PISA_SCORE_MEAN_VAR) ? 0.5f * part.z / part.x : 0.f) : -CUDART_INF_F;
         }
+        a.blk_lse[(((long long)bh * geo.N + t) * (a.slots * a.fan) + slot * a.fan + r) * G + head] = lse;
       }
     }
   }
@@ -1423,8 +1512,7 @@ int launch_tile_lse_m(const Geometry& g, const TileArgs& a, int32_t* work_ctr, c
   const size_t smem = (size_t)(D / 64) * (4 * 128 * 128 + NB * 128) + 1024;
   cudaError_t e = cudaFuncSetAttribute(lse_ws_kernel<D, NB, MOM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("lse_ws attr", e); return PISA_ERR_CUDA; }
-  (void)work_ctr;   // the leaf-scoring kernel walks its items statically (see ItemFeed)
-  lse_ws_kernel<D, NB, MOM><<<num_sms(), kLseThreads, smem, s>>>(g, a, tm_k);
+  lse_ws_kernel<D, NB, MOM><<<num_sms(), kLseThreads, smem, s>>>(g, a, work_ctr, tm_k);
   return check_launch("lse_ws");
 }
 template <int D, int NB>
