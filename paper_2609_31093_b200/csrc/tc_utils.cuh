@@ -71,6 +71,12 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// Asks for [p, p + bytes) (16-byte aligned, a multiple of 16 bytes, this GPU's memory) to be brought into L2;
+// nothing is written to shared memory and nothing waits for it.
+__device__ __forceinline__ void prefetch_l2_bulk(const void* p, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
 // ---------------------------------------------------------------- proxies / fences
 
 // generic-proxy writes to shared memory -> visible to the async proxy (UMMA, bulk copies)

@@ -608,7 +608,8 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
     // The warp runs up to R tiles ahead of the epilogue: the latency of the draw, of the item's description
     // and of the entries' loads stays off every other role's path.
     const int n_items = a.item_off[a.nkeys];
-    int it = 0;
+    const int win_tok = (geo.N < kWindowTok) ? ((geo.N + kInvTok - 1) / kInvTok) * kInvTok : kWindowTok;
+    int it = 0, last_win = -1;
     bool ok = true;
     while (ok) {
       int item = 0;
@@ -617,6 +618,22 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
       if (item >= n_items) break;
       const ItemInfo inf = item_info(a, item, tpt);
       const int bh = inf.key / (a.NW * a.Mk), j = inf.key % a.Mk;
+      // A gather completes when its last row has landed, and a tile that meets even one row for the first
+      // time waits for HBM.  So, on entering a window of the lists, the CTA asks for its share of the NEXT
+      // window's query rows to be brought into L2 (the CTAs walk the windows together).
+      if (inf.key / a.Mk != last_win) {
+        last_win = inf.key / a.Mk;
+        const int nw = last_win + 1;
+        if (nw < geo.B * geo.Hkv * a.NW) {
+          const int bh2 = nw / a.NW, w2 = nw % a.NW;
+          const int t0 = w2 * win_tok, t1 = min(geo.N, t0 + win_tok);
+          const int per = (t1 - t0 + (int)gridDim.x - 1) / (int)gridDim.x;
+          const int ta = t0 + (int)blockIdx.x * per, tb = min(t1, ta + per);
+          const __nv_bfloat16* qb2 = a.q + (long long)(bh2 / geo.Hkv) * geo.qs[0] + (long long)((bh2 % geo.Hkv) * G) * geo.qs[2];
+          for (int i = lane; i < (tb - ta) * G; i += 32)
+            prefetch_l2_bulk(qb2 + (long long)(ta + (i >> lgG)) * geo.qs[1] + (long long)(i & (G - 1)) * geo.qs[2], (uint32_t)(D * 2));
+        }
+      }
       // the entries of four tiles are fetched together: one round trip to L2 per four tiles, not per tile
       constexpr int TB = 4, TPL = 4;                       // tiles per batch; entries per lane and tile (tpt <= 128)
       for (int jt0 = 0; jt0 < inf.ntiles && ok; jt0 += TB) {
