@@ -14,7 +14,8 @@
 //   result    = the fp32 accumulator rows of these tokens are STORED (not added): this kernel initialises
 //               the accumulator the list-driven attention kernel then adds the routed blocks into, so
 //               no memset is needed and the routed kernel never sees a masked block.
-// Roles: warp 0 TMA producer, warp 1 UMMA issuer, warps 2-5 softmax and read-out.  Every wait is bounded.
+// Roles: warp 0 TMA producer, warps 1 and 2 UMMA issuers (first / second products), warps 4-7 and 8-11 two
+// softmax / read-out groups taking alternate blocks.  Every wait is bounded.
 #include <math_constants.h>
 
 #include "pisa_common.cuh"
@@ -27,7 +28,7 @@ using namespace tc;
 
 namespace {
 
-constexpr int kLocalThreads = 192;
+constexpr int kLocalThreads = 384;        // TMA warp, two UMMA issuers, (one idle), two softmax / read-out groups of four warps
 constexpr float kLog2eL = 1.4426950408889634f;
 
 struct LocalArgs {
@@ -72,25 +73,27 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
   constexpr int A_SLAB = 128 * 128, KV_SLAB = C * 128;
   constexpr int Q_BYTES = KS * A_SLAB, KV_BYTES = KS * KV_SLAB, P_BYTES = (C / 64) * A_SLAB;
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* sQ = smem;                      // [2][Q_BYTES]: this item's and the next item's query tile
-  uint8_t* sK = sQ + 2 * Q_BYTES;          // [2][KV_BYTES]
+  // One query tile (it is free once the item's last S has been computed, well before the item ends, so the next
+  // one loads under the remaining products) and TWO P tiles: the softmax of block j + 1 runs while P(j) V(j) does.
+  uint8_t* sQ = smem;                      // [Q_BYTES]
+  uint8_t* sK = sQ + Q_BYTES;              // [2][KV_BYTES]
   uint8_t* sV = sK + 2 * KV_BYTES;         // [2][KV_BYTES]
-  uint8_t* sP = sV + 2 * KV_BYTES;         // [P_BYTES]
-  __shared__ uint64_t q_full[2], q_empty[2], k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_empty[2],
-      p_full, p_empty, o_full, o_empty;
+  uint8_t* sP = sV + 2 * KV_BYTES;         // [2][P_BYTES]
+  __shared__ uint64_t q_full, q_empty, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_empty[2],
+      p_full[2], p_empty[2], o_full, o_empty;
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_fail;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&q_full[i], 1); mbar_init(&q_empty[i], 1);
       mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
       mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
       mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4);
+      mbar_init(&p_full[i], 4); mbar_init(&p_empty[i], 1);
     }
-    mbar_init(&p_full, 4); mbar_init(&p_empty, 1);
-    mbar_init(&o_full, 1); mbar_init(&o_empty, 4);
+    mbar_init(&q_full, 1); mbar_init(&q_empty, 1);
+    mbar_init(&o_full, 1); mbar_init(&o_empty, 8);
     s_fail = 0;
     mbar_fence_init();
   }
@@ -108,12 +111,10 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
       int it = 0, kv = 0;                  // items and (item, block) steps of this CTA
       for (int item = blockIdx.x; item < a.n_items && !s_fail; item += gridDim.x, ++it) {
         const LocalItem w = local_item(geo, a, item);
-        const int qs = it & 1;
-        if (it >= 2 && !mbar_wait_bounded(&q_empty[qs], (uint32_t)(((it >> 1) - 1) & 1))) { s_fail = 1; break; }
-        mbar_arrive_expect_tx(&q_full[qs], (uint32_t)Q_BYTES);
+        if (it >= 1 && !mbar_wait_bounded(&q_empty, (uint32_t)((it - 1) & 1))) { s_fail = 1; break; }
+        mbar_arrive_expect_tx(&q_full, (uint32_t)Q_BYTES);
         for (int ks = 0; ks < KS; ++ks)
-          tma_load_4d(smem_u32(sQ + qs * Q_BYTES + ks * A_SLAB), &tm_q, &q_full[qs], ks * 64, w.h * G,
-                      w.c * C + w.tile * tpt, w.b);
+          tma_load_4d(smem_u32(sQ + ks * A_SLAB), &tm_q, &q_full, ks * 64, w.h * G, w.c * C + w.tile * tpt, w.b);
         for (int j = 0; j < w.nb; ++j, ++kv) {
           const int s = kv & 1;
           if (kv >= 2 && !mbar_wait_bounded(&k_empty[s], (uint32_t)(((kv >> 1) - 1) & 1))) { s_fail = 1; break; }
@@ -128,24 +129,24 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------ UMMA issuer (the warp walks the loop, lane 0 issues)
+    // ------------------------------------------------ UMMA issuer of the first products, S = Q K^T
+    // (its own warp: an issue blocks while the tensor pipe works its queue off, and the two kinds of product
+    // wait for different things -- S for keys and a free S buffer, P V for the softmax)
     const uint32_t idesc_s = make_idesc_bf16(128, C, 0, 0);
-    const uint32_t idesc_ot = make_idesc_bf16(128, 128, 1, 0);     // O^T: M = d (V, MN-major), N = tile rows (P)
     int it = 0, kv = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < a.n_items && ok && !s_fail; item += gridDim.x, ++it) {
       const LocalItem w = local_item(geo, a, item);
-      const int qs = it & 1;
-      ok = mbar_wait_bounded(&q_full[qs], (uint32_t)((it >> 1) & 1));
-      // S of block j + 1 is issued before the second product of block j, so that it overlaps the softmax
-      auto issue_s = [&](int kvj) {
-        const int s = kvj & 1;
-        bool good = mbar_wait_bounded(&k_full[s], (uint32_t)((kvj >> 1) & 1));
-        if (good && kvj >= 2) good = mbar_wait_bounded(&s_empty[s], (uint32_t)(((kvj >> 1) - 1) & 1));
-        good = __all_sync(0xffffffffu, good);
-        if (good && lane == 0) {
+      ok = mbar_wait_bounded(&q_full, (uint32_t)(it & 1));
+      for (int j = 0; j < w.nb && ok; ++j) {
+        const int kvj = kv + j, s = kvj & 1;
+        ok = mbar_wait_bounded(&k_full[s], (uint32_t)((kvj >> 1) & 1));
+        if (ok && kvj >= 2) ok = mbar_wait_bounded(&s_empty[s], (uint32_t)(((kvj >> 1) - 1) & 1));
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (lane == 0) {
           tcgen05_fence_after_sync();
-          const uint32_t q0 = smem_u32(sQ + qs * Q_BYTES), k0 = smem_u32(sK + s * KV_BYTES);
+          const uint32_t q0 = smem_u32(sQ), k0 = smem_u32(sK + s * KV_BYTES);
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
             const uint64_t da = make_smem_desc(q0 + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
@@ -154,30 +155,37 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
           }
           umma_commit(&s_full[s]);
           umma_commit(&k_empty[s]);
+          if (j == w.nb - 1) umma_commit(&q_empty);          // every S of this item has been issued
         }
         __syncwarp();
-        return good;
-      };
-      if (ok) ok = issue_s(kv);
+      }
+      kv += w.nb;
+    }
+    if (!ok) s_fail = 1;
+  } else if (warp == 2) {
+    // ------------------------------------------------ UMMA issuer of the second products, O^T += V^T P^T
+    const uint32_t idesc_ot = make_idesc_bf16(128, 128, 1, 0);     // M = d (V, MN-major), N = tile rows (P)
+    int it = 0, kv = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < a.n_items && ok && !s_fail; item += gridDim.x, ++it) {
+      const LocalItem w = local_item(geo, a, item);
       for (int j = 0; j < w.nb && ok; ++j) {
         const int kvj = kv + j, s = kvj & 1;
-        if (j + 1 < w.nb) ok = issue_s(kvj + 1);
-        else if (lane == 0) umma_commit(&q_empty[qs]);       // every S of this item has been issued
-        if (ok) ok = mbar_wait_bounded(&p_full, (uint32_t)(kvj & 1));
+        ok = mbar_wait_bounded(&p_full[s], (uint32_t)((kvj >> 1) & 1));
         if (ok) ok = mbar_wait_bounded(&v_full[s], (uint32_t)((kvj >> 1) & 1));
         if (ok && j == 0 && it >= 1) ok = mbar_wait_bounded(&o_empty, (uint32_t)((it - 1) & 1));
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         if (lane == 0) {
           tcgen05_fence_after_sync();
-          const uint32_t p0 = smem_u32(sP), v0 = smem_u32(sV + s * KV_BYTES);
+          const uint32_t p0 = smem_u32(sP + s * P_BYTES), v0 = smem_u32(sV + s * KV_BYTES);
 #pragma unroll
           for (int kk = 0; kk < C / 16; ++kk) {
             const uint64_t dp = make_smem_desc(p0 + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
             const uint64_t dv = make_smem_desc(v0 + kk * (16 * 128), KV_SLAB, 1024);
             umma_bf16(tmem + 256u, dv, dp, idesc_ot, (j > 0 || kk > 0) ? 1u : 0u);
           }
-          umma_commit(&p_empty);
+          umma_commit(&p_empty[s]);
           umma_commit(&v_empty[s]);
           if (j == w.nb - 1) umma_commit(&o_full);
         }
@@ -186,8 +194,12 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
       kv += w.nb;
     }
     if (!ok) s_fail = 1;
-  } else {
+  } else if (warp >= 4) {
     // ------------------------------------------------ softmax and read-out warps (TMEM lane quarter = warp % 4)
+    // Two groups of four: a group takes every other (item, block) step -- S buffer, P buffer and barriers of
+    // its parity -- so that two warps per SM sub-partition overlap their exponentials and TMEM waits; both
+    // read the item's accumulator out, half of its columns each.
+    const int grp = (warp - 4) >> 2;
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;             // S: tile row = token * G + head;  O^T: output column d
     const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
@@ -203,13 +215,15 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
       if (live) neg_lse2 = -a.row_lse[((long long)w.b * geo.Hq + w.h * G + head) * geo.N + t] * kLog2eL;
       for (int j = 0; j < w.nb && ok; ++j, ++kv) {
         const int s = kv & 1;
+        if (s != grp) continue;
         // visible keys of this block for this row: all of an earlier leaf, keys <= t of the row's own leaf
         const int ncols = !live ? 0 : ((w.blk[j] == w.c) ? (t - w.c * C + 1) : C);
         ok = mbar_wait_bounded(&s_full[s], (uint32_t)((kv >> 1) & 1));
-        if (ok && kv >= 1) ok = mbar_wait_bounded(&p_empty, (uint32_t)((kv - 1) & 1));
+        if (ok && kv >= 2) ok = mbar_wait_bounded(&p_empty[s], (uint32_t)(((kv >> 1) - 1) & 1));
         if (!ok) break;
         tcgen05_fence_after_sync();
         const uint32_t s_base = tmem + lane_sel + (uint32_t)(s * 128);
+        const bool fast = __all_sync(0xffffffffu, ncols == C);     // no masked column in this warp's rows
         uint32_t ra[32], rb[32];
         tmem_ld_32x32(s_base, ra);
 #pragma unroll
@@ -229,15 +243,17 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
           for (int jx = 0; jx < 16; ++jx) {
             float p0 = ex2l(fmaf(__uint_as_float(cur[2 * jx]), sl2, neg_lse2));
             float p1 = ex2l(fmaf(__uint_as_float(cur[2 * jx + 1]), sl2, neg_lse2));
-            if (c0 + 2 * jx >= ncols) p0 = 0.f;
-            if (c0 + 2 * jx + 1 >= ncols) p1 = 0.f;
+            if (!fast) {
+              if (c0 + 2 * jx >= ncols) p0 = 0.f;
+              if (c0 + 2 * jx + 1 >= ncols) p1 = 0.f;
+            }
             const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
             pk[jx] = *reinterpret_cast<const uint32_t*>(&pp);
           }
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
             const int ck = c0 / 8 + q4;
-            const uint32_t dst = smem_u32(sP + (ck >> 3) * A_SLAB) + swz128(row, ck & 7);
+            const uint32_t dst = smem_u32(sP + s * P_BYTES + (ck >> 3) * A_SLAB) + swz128(row, ck & 7);
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * q4]), "r"(pk[4 * q4 + 1]),
                          "r"(pk[4 * q4 + 2]), "r"(pk[4 * q4 + 3])
                          : "memory");
@@ -245,7 +261,7 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
         }
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&p_full);
+        if (lane == 0) mbar_arrive(&p_full[s]);
       }
       if (!ok) break;
       // read-out: lane = output column d, TMEM column = tile row; the G heads of a token are G consecutive columns
@@ -256,13 +272,15 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
       float* acc_d = a.o_acc + (((long long)w.b * geo.Hkv + w.h) * geo.N) * (long long)(D * G) + (long long)row * G;
       const long long tok_stride = (long long)D * G;
       uint32_t ra[32], rb[32];
-      tmem_ld_32x32(o_base, ra);
+      const int cbeg = grp * 64;
+      tmem_ld_32x32(o_base + (uint32_t)cbeg, ra);
 #pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        uint32_t (&cur)[32] = ((c0 >> 5) & 1) ? rb : ra;
-        uint32_t (&nxt)[32] = ((c0 >> 5) & 1) ? ra : rb;
+      for (int cc = 0; cc < 64; cc += 32) {
+        const int c0 = cbeg + cc;
+        uint32_t (&cur)[32] = ((cc >> 5) & 1) ? rb : ra;
+        uint32_t (&nxt)[32] = ((cc >> 5) & 1) ? ra : rb;
         tmem_ld_wait();
-        if (c0 + 32 < 128) {
+        if (cc + 32 < 64) {
           tmem_ld_32x32(o_base + (uint32_t)(c0 + 32), nxt);
         } else {
           tcgen05_fence_before_sync();
@@ -332,7 +350,7 @@ static int launch_local_c(const Geometry& g, const void* q, const void* k, const
     if (!tma::make_map(&tm_k, 2, 4, k, dims, sk, box, true)) return PISA_ERR_UNSUPPORTED;
     if (!tma::make_map(&tm_v, 2, 4, v, dims, sv, box, true)) return PISA_ERR_UNSUPPORTED;
   }
-  const size_t smem = 2 * (size_t)(2 * 128 * 128) + 4 * (size_t)(2 * C * 128) + (size_t)(C / 64) * 128 * 128 + 1024;
+  const size_t smem = (size_t)(2 * 128 * 128) + 4 * (size_t)(2 * C * 128) + 2 * (size_t)(C / 64) * 128 * 128 + 1024;
   cudaError_t e = cudaFuncSetAttribute(local_window_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("local_window attr", e); return PISA_ERR_CUDA; }
   const int grid = a.n_items < num_sms() ? a.n_items : num_sms();
