@@ -206,13 +206,21 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
     const float sl2 = geo.scale * kLog2eL;
     int it = 0, kv = 0;
     bool ok = true;
+    // the row's softmax denominator is fetched one item ahead (the load would otherwise open every item)
+    auto row_lse_of = [&](int item) -> float {
+      if (item >= a.n_items) return 0.f;
+      const LocalItem x = local_item(geo, a, item);
+      const int tx = x.c * C + x.tile * tpt + (row >> lgG);
+      return (tx < geo.N) ? a.row_lse[((long long)x.b * geo.Hq + x.h * G + (row & (G - 1))) * geo.N + tx] : 0.f;
+    };
+    float lse_next = row_lse_of((int)blockIdx.x);
     for (int item = blockIdx.x; item < a.n_items && ok && !s_fail; item += gridDim.x, ++it) {
       const LocalItem w = local_item(geo, a, item);
       const int t0 = w.c * C + w.tile * tpt;         // first token of the tile
-      const int t = t0 + (row >> lgG), head = row & (G - 1);
+      const int t = t0 + (row >> lgG);
       const bool live = t < geo.N;
-      float neg_lse2 = 0.f;
-      if (live) neg_lse2 = -a.row_lse[((long long)w.b * geo.Hq + w.h * G + head) * geo.N + t] * kLog2eL;
+      const float neg_lse2 = -lse_next * kLog2eL;
+      lse_next = row_lse_of(item + (int)gridDim.x);
       for (int j = 0; j < w.nb && ok; ++j, ++kv) {
         const int s = kv & 1;
         if (s != grp) continue;
