@@ -490,7 +490,11 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
   constexpr int A_STAGE = KS * A_SLAB;
   constexpr uint32_t TM_COLS = (2 * NB < 32) ? 32 : 2 * NB;
   constexpr int R = kLseRing;
-  constexpr int W = NB / 4;                       // accumulator columns of one epilogue warp
+  // epilogue warps per tile: all sixteen on a 256-column accumulator; two groups of eight on alternate tiles
+  // for narrower ones (a small tile's fixed latencies then overlap with the other group's tile)
+  constexpr int GR = (NB <= 128) ? 2 : 1;
+  constexpr int WQ = 4 / GR;                      // warps of one tile that share a TMEM lane quarter
+  constexpr int W = NB / WQ;                      // accumulator columns of one epilogue warp
   constexpr int CW = (W < 32) ? W : 32;           // columns per TMEM load
   uint8_t* smem = align1024(smem_raw);
   uint8_t* sA = smem;
@@ -510,8 +514,8 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
     for (int i = 0; i < NS; ++i) { mbar_init(&a_full[i], kLseProd); mbar_init(&a_empty[i], 1); }
     mbar_init(&b_empty, 1);
     mbar_init(&b_full, 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 512); }
-    for (int i = 0; i < R; ++i) { mbar_init(&m_full[i], 1); mbar_init(&m_empty[i], 16); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 512 / GR); }
+    for (int i = 0; i < R; ++i) { mbar_init(&m_full[i], 1); mbar_init(&m_empty[i], 16 / GR); }
     s_fail = 0;
     mbar_fence_init();
   }
@@ -634,19 +638,24 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
             prefetch_l2_bulk(qb2 + (long long)(ta + (i >> lgG)) * geo.qs[1] + (long long)(i & (G - 1)) * geo.qs[2], (uint32_t)(D * 2));
         }
       }
-      // the entries of four tiles are fetched together: one round trip to L2 per four tiles, not per tile
-      constexpr int TB = 4, TPL = 4;                       // tiles per batch; entries per lane and tile (tpt <= 128)
-      for (int jt0 = 0; jt0 < inf.ntiles && ok; jt0 += TB) {
-        int ent[TB][TPL];
+      // 128 consecutive entries (128 / tpt tiles) are fetched per round trip to L2, and the next 128 are
+      // requested before the current ones are laid out
+      const int lg_tpt = 7 - lgG, tiles_per_batch = 128 >> lg_tpt;
+      auto fetch = [&](int jt0, int (&dst)[4]) {
 #pragma unroll
-        for (int u = 0; u < TB; ++u)
+        for (int x = 0; x < 4; ++x) {
+          const int e = inf.e_begin + (jt0 << lg_tpt) + lane + 32 * x;
+          dst[x] = (jt0 < inf.ntiles && e < inf.e_end) ? a.entries[e] : -1;
+        }
+      };
+      int nxt[4];
+      fetch(0, nxt);
+      for (int jt0 = 0; jt0 < inf.ntiles && ok; jt0 += tiles_per_batch) {
+        int ent[4];
 #pragma unroll
-          for (int x = 0; x < TPL; ++x) {
-            const int p = lane + 32 * x, e = inf.e_begin + (jt0 + u) * tpt + p;
-            ent[u][x] = (p < tpt && e < inf.e_end) ? a.entries[e] : -1;
-          }
-#pragma unroll
-        for (int u = 0; u < TB; ++u) {
+        for (int x = 0; x < 4; ++x) ent[x] = nxt[x];
+        fetch(jt0 + tiles_per_batch, nxt);
+        for (int u = 0; u < tiles_per_batch; ++u) {
           const int jt = jt0 + u;
           if (jt >= inf.ntiles) break;
           const int mr = it % R;
@@ -654,8 +663,10 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
           ok = __all_sync(0xffffffffu, ok && !s_fail);
           if (!ok) break;
 #pragma unroll
-          for (int x = 0; x < TPL; ++x)
-            if (lane + 32 * x < tpt) s_tent[mr][lane + 32 * x] = checked_entry(a, geo.N, ent[u][x]);
+          for (int x = 0; x < 4; ++x) {
+            const int f = lane + 32 * x;                  // position in the batch
+            if ((f >> lg_tpt) == u) s_tent[mr][f & (tpt - 1)] = checked_entry(a, geo.N, ent[x]);
+          }
           if (lane == 0) s_tkey[mr] = make_int4(bh, j, (jt == 0 ? 1 : 0) | (jt == inf.ntiles - 1 ? 2 : 0), 0);
           __syncwarp();
           if (lane == 0) mbar_arrive(&m_full[mr]);     // release: the ring entry is complete
@@ -666,14 +677,16 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
     if (!ok) s_fail = 1;
     if (lane == 0) s_total = it;
   } else {
-    // ------------------------------------------------ epilogue: sixteen warps on every tile
-    // Four warps share each TMEM lane quarter and split the accumulator's NB columns, W = NB / 4 each -- few
-    // enough to hold in registers.  A warp therefore reads its columns out at once and releases the
-    // accumulator BEFORE it starts on the exponentials: the next-but-one tile's UMMAs never wait for
-    // arithmetic.  A leaf wider than W is shared by C / W warps of the quarter; they leave their partial
+    // ------------------------------------------------ epilogue: sixteen warps
+    // The warps of a tile that share a TMEM lane quarter (four, all sixteen warps on one tile, for a 256-column
+    // accumulator; two, the warps in two groups on alternate tiles, for narrower ones) split the accumulator's
+    // columns, W each -- few enough to hold in registers.  A warp therefore reads its columns out at once and
+    // releases the accumulator BEFORE it starts on the exponentials: the next-but-one tile's UMMAs never wait
+    // for arithmetic.  A leaf wider than W is shared by C / W warps of the quarter; they leave their partial
     // (max, sum) in shared memory and the first of them combines (always in the same order).
     const int ew = warp - (kLseProd / 32 + 2);
-    const int cq = ew >> 2;                             // column quarter; warp % 4 = TMEM lane quarter
+    const int grp = (GR == 2) ? (ew >> 3) : 0;          // which tiles this warp works on (it % GR == grp)
+    const int cq = (ew >> 2) & (WQ - 1);                // column share inside the tile; warp % 4 = TMEM lane quarter
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(cq * W);
     const int head = row & (G - 1);
@@ -681,9 +694,9 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
     const int r = (cq * W) / C;                         // the child this warp's columns belong to
     const int off = cq * W - r * C;                     // its first column inside that child
     const bool owner = (cq % wpl) == 0;
-    const int bar_id = 1 + (warp & 3) * 2 + ((wpl == 2) ? (cq >> 1) : 0);
+    const int bar_id = 1 + grp * 8 + (warp & 3) * 2 + ((wpl == 2 && WQ == 4) ? (cq >> 1) : 0);
     constexpr bool lse_mode = !MOM;
-    for (int it = 0;; ++it) {
+    for (int it = grp;; it += GR) {
       const int buf = it & 1;
       if (!wait_tile(&t_full[buf], (uint32_t)((it >> 1) & 1), it)) break;
       tcgen05_fence_after_sync();
