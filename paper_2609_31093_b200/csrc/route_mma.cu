@@ -110,10 +110,10 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
           const int ch_lo = node * 2, ch_hi = ch_lo + 1;
           const bool ok_hi = has && ch_hi < Mb;
           U32x8 lo[C8], hi[C8];
-#pragma unroll
           // rows without a candidate (kap >= nV: node 0) or without a second child (ragged level: the first
           // child again) load valid summaries all the same; their logits are dropped below
           const long long off_hi = (long long)(ok_hi ? ch_hi : ch_lo) * D;
+#pragma unroll
           for (int c8 = 0; c8 < C8; ++c8) {
             lo[c8] = ldg256(below + (long long)ch_lo * D + (c8 * 4 + tig) * 16);
             hi[c8] = ldg256(below + off_hi + (c8 * 4 + tig) * 16);

@@ -252,16 +252,6 @@ __device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
   return reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~(uintptr_t)1023);
 }
 
-// last key whose first tile is <= tile (lists without tiles share their successor's offset)
-__device__ __forceinline__ int find_key(const int32_t* tile_off, int nkeys, int tile) {
-  int lo = 0, hi = nkeys;            // invariant: tile_off[lo] <= tile < tile_off[hi]
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (tile_off[mid] <= tile) lo = mid; else hi = mid;
-  }
-  return lo;
-}
-
 // Work items of both tile kernels are handed out dynamically: lists differ in length, and a static
 // round-robin left the CTAs' tile counts 20 % apart.  The leaf-scoring kernel has a scheduler warp of its own
 // (see there).  In the attention kernel thread 0 of the CTA draws the next item from a global counter when the
@@ -815,7 +805,6 @@ pv_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant_
   uint8_t* sK = smem + NS * Q_STAGE;
   uint8_t* sV = sK + KS * KV_SLAB;
   __shared__ uint64_t q_full[NS], q_empty[NS], kv_full, kv_empty, s_full[2], s_empty[2], p_ready[2], o_full[2], o_empty[2];
-  __shared__ __align__(16) int s_rowidx[kMetaRing][128];  // accumulator row (t*Hq + head) of every tile row, -1 = none
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_fail;
   __shared__ int s_ent[kMetaRing][128];   // per-tile entries, written by the producers, read by all roles
@@ -1064,7 +1053,7 @@ pv_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant_
         const uint32_t o_base = tmem + lane_sel + 256u + (uint32_t)(ob * 128);
         if (!mbar_wait_bounded(&o_full[ob], (uint32_t)((it >> 1) & 1))) { s_fail = 1; break; }
         tcgen05_fence_after_sync();
-        if (kTransO) {
+        if constexpr (kTransO) {
           // lane = output column d (= `row` of this thread), TMEM column = tile row = entry*G + head
           const int* ents = s_ent[it % kMetaRing];
           float* acc_d = a.o_acc + (((long long)b * geo.Hkv + h) * geo.N) * (long long)(D * G) + (long long)row * G;
@@ -1114,8 +1103,7 @@ pv_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant_
               }
             }
           }
-          continue;
-        }
+        } else {
 #pragma unroll
         for (int half = 0; half < KS; ++half) {
           uint32_t ra[32], rb[32];
@@ -1155,6 +1143,7 @@ pv_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant_
           __syncwarp();
         }
         mbar_arrive(&q_empty[s]);          // the ring slot is free again
+        }
       }
     }
   }
