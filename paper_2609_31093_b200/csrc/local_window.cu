@@ -10,7 +10,8 @@
 //   per forced block: K and V slabs by TMA tile loads (this GPU's memory, no multicast),
 //               S = Q K^T (tcgen05, TMEM) -> P = 2^(S * scale * log2e - lse_row) in bf16 (the row's
 //               denominator is known from the routing, so P is final: no running maximum), causal
-//               mask only inside the current leaf -> O^T += V^T P^T accumulated in TMEM over the blocks;
+//               mask only inside the current leaf -> O^T += V^T P^T (d = 128; O += P V with d = 64: a 64-row
+//               accumulator has another TMEM layout) accumulated in TMEM over the blocks;
 //   result    = the fp32 accumulator rows of these tokens are STORED (not added): this kernel initialises
 //               the accumulator the list-driven attention kernel then adds the routed blocks into, so
 //               no memset is needed and the routed kernel never sees a masked block.
@@ -33,7 +34,7 @@ constexpr float kLog2eL = 1.4426950408889634f;
 
 struct LocalArgs {
   const float* row_lse;    // [B, Hq, N] natural log
-  float* o_acc;            // [B, Hkv, N, 128, G] fp32
+  float* o_acc;            // fp32: [B, Hkv, N, 128, G] for d = 128, [B, N, Hq, 64] for d = 64 (the layouts of pv_ws)
   int32_t* status;
   int tiles_per_leaf;      // C / (128 / G)
   int n_items;             // B * Hkv * M1 * tiles_per_leaf
@@ -63,13 +64,14 @@ __device__ __forceinline__ LocalItem local_item(const Geometry& geo, const Local
 
 }  // namespace
 
-// D = 128.  C: leaf size (64 or 128).
-template <int C>
+// C: leaf size (64 or 128); D: head dimension (64 or 128).
+template <int C, int D>
 __global__ void __launch_bounds__(kLocalThreads, 1)
 local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, LocalArgs a) {
   extern __shared__ uint8_t smem_raw[];
-  constexpr int D = 128, KS = 2;
+  constexpr int KS = D / 64;
+  constexpr bool kTransO = (D == 128);
   constexpr int A_SLAB = 128 * 128, KV_SLAB = C * 128;
   constexpr int Q_BYTES = KS * A_SLAB, KV_BYTES = KS * KV_SLAB, P_BYTES = (C / 64) * A_SLAB;
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -164,7 +166,8 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
     if (!ok) s_fail = 1;
   } else if (warp == 2) {
     // ------------------------------------------------ UMMA issuer of the second products, O^T += V^T P^T
-    const uint32_t idesc_ot = make_idesc_bf16(128, 128, 1, 0);     // M = d (V, MN-major), N = tile rows (P)
+    const uint32_t idesc_ot = make_idesc_bf16(128, 128, 1, 0);     // O^T: M = d (V, MN-major), N = tile rows (P)
+    const uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);        // O: M = tile rows (P), N = d (V, MN-major)
     int it = 0, kv = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < a.n_items && ok && !s_fail; item += gridDim.x, ++it) {
@@ -183,7 +186,8 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
           for (int kk = 0; kk < C / 16; ++kk) {
             const uint64_t dp = make_smem_desc(p0 + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
             const uint64_t dv = make_smem_desc(v0 + kk * (16 * 128), KV_SLAB, 1024);
-            umma_bf16(tmem + 256u, dv, dp, idesc_ot, (j > 0 || kk > 0) ? 1u : 0u);
+            if (kTransO) umma_bf16(tmem + 256u, dv, dp, idesc_ot, (j > 0 || kk > 0) ? 1u : 0u);
+            else umma_bf16(tmem + 256u, dp, dv, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
           }
           umma_commit(&p_empty[s]);
           umma_commit(&v_empty[s]);
@@ -277,41 +281,63 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
       if (!ok) break;
       tcgen05_fence_after_sync();
       const uint32_t o_base = tmem + lane_sel + 256u;
-      float* acc_d = a.o_acc + (((long long)w.b * geo.Hkv + w.h) * geo.N) * (long long)(D * G) + (long long)row * G;
-      const long long tok_stride = (long long)D * G;
-      uint32_t ra[32], rb[32];
-      const int cbeg = grp * 64;
-      tmem_ld_32x32(o_base + (uint32_t)cbeg, ra);
+      if constexpr (kTransO) {
+        // lane = output column d, TMEM column = tile row; the G heads of a token are G consecutive columns of
+        // the heads-innermost accumulator [B, Hkv, N, d, G]; each group reads half of the columns
+        float* acc_d = a.o_acc + (((long long)w.b * geo.Hkv + w.h) * geo.N) * (long long)(D * G) + (long long)row * G;
+        const long long tok_stride = (long long)D * G;
+        uint32_t ra[32], rb[32];
+        const int cbeg = grp * 64;
+        tmem_ld_32x32(o_base + (uint32_t)cbeg, ra);
 #pragma unroll
-      for (int cc = 0; cc < 64; cc += 32) {
-        const int c0 = cbeg + cc;
-        uint32_t (&cur)[32] = ((cc >> 5) & 1) ? rb : ra;
-        uint32_t (&nxt)[32] = ((cc >> 5) & 1) ? ra : rb;
-        tmem_ld_wait();
-        if (cc + 32 < 64) {
-          tmem_ld_32x32(o_base + (uint32_t)(c0 + 32), nxt);
-        } else {
-          tcgen05_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&o_empty);          // O has been read out of TMEM
+        for (int cc = 0; cc < 64; cc += 32) {
+          const int c0 = cbeg + cc;
+          uint32_t (&cur)[32] = ((cc >> 5) & 1) ? rb : ra;
+          uint32_t (&nxt)[32] = ((cc >> 5) & 1) ? ra : rb;
+          tmem_ld_wait();
+          if (cc + 32 < 64) {
+            tmem_ld_32x32(o_base + (uint32_t)(c0 + 32), nxt);
+          } else {
+            tcgen05_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&o_empty);          // O has been read out of TMEM
+          }
+          if (G >= 4) {
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4) {
+              const int col = c0 + 4 * q4;
+              const int tt = t0 + (col >> lgG);
+              if (tt < geo.N)
+                *reinterpret_cast<float4*>(acc_d + (long long)tt * tok_stride + (col & (G - 1))) =
+                    make_float4(__uint_as_float(cur[4 * q4]), __uint_as_float(cur[4 * q4 + 1]),
+                                __uint_as_float(cur[4 * q4 + 2]), __uint_as_float(cur[4 * q4 + 3]));
+            }
+          } else {
+#pragma unroll
+            for (int q1 = 0; q1 < 32; ++q1) {
+              const int col = c0 + q1;
+              const int tt = t0 + (col >> lgG);
+              if (tt < geo.N) acc_d[(long long)tt * tok_stride + (col & (G - 1))] = __uint_as_float(cur[q1]);
+            }
+          }
         }
-        if (G >= 4) {
+      } else {
+        // lane = tile row (token, head), TMEM column = output column d; the token-major accumulator
+        // [B, N, Hq, d]; each group stores half of the row's columns (D / 2 = 32)
+        static_assert(D == 64, "the direct read-out is written for d = 64");
+        uint32_t ra[32];
+        tmem_ld_32x32(o_base + (uint32_t)(grp * 32), ra);
+        tmem_ld_wait();
+        tcgen05_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&o_empty);              // O has been read out of TMEM
+        if (live) {
+          float* dst = a.o_acc + (((long long)w.b * geo.N + t) * geo.Hq + w.h * G + (row & (G - 1))) * D + grp * 32;
 #pragma unroll
-          for (int q4 = 0; q4 < 8; ++q4) {
-            const int col = c0 + 4 * q4;
-            const int tt = t0 + (col >> lgG);
-            if (tt < geo.N)
-              *reinterpret_cast<float4*>(acc_d + (long long)tt * tok_stride + (col & (G - 1))) =
-                  make_float4(__uint_as_float(cur[4 * q4]), __uint_as_float(cur[4 * q4 + 1]),
-                              __uint_as_float(cur[4 * q4 + 2]), __uint_as_float(cur[4 * q4 + 3]));
-          }
-        } else {
-#pragma unroll
-          for (int q1 = 0; q1 < 32; ++q1) {
-            const int col = c0 + q1;
-            const int tt = t0 + (col >> lgG);
-            if (tt < geo.N) acc_d[(long long)tt * tok_stride + (col & (G - 1))] = __uint_as_float(cur[q1]);
-          }
+          for (int q4 = 0; q4 < 8; ++q4)
+            *reinterpret_cast<float4*>(dst + 4 * q4) =
+                make_float4(__uint_as_float(ra[4 * q4]), __uint_as_float(ra[4 * q4 + 1]), __uint_as_float(ra[4 * q4 + 2]),
+                            __uint_as_float(ra[4 * q4 + 3]));
         }
       }
     }
@@ -324,7 +350,7 @@ local_window_kernel(Geometry geo, const __grid_constant__ CUtensorMap tm_q, cons
 }
 
 bool local_window_supported(const Geometry& g, int dtype) {
-  if (dtype != PISA_BF16 || g.d != 128) return false;
+  if (dtype != PISA_BF16 || (g.d != 128 && g.d != 64)) return false;
   if (g.C != 64 && g.C != 128) return false;
   const int tpt = 128 / g.G;
   if (g.G > 16 || g.C % tpt != 0) return false;
@@ -333,7 +359,7 @@ bool local_window_supported(const Geometry& g, int dtype) {
   return tma::encoder() != nullptr;
 }
 
-template <int C>
+template <int C, int D>
 static int launch_local_c(const Geometry& g, const void* q, const void* k, const void* v, const float* row_lse,
                           float* o_acc, int32_t* status, cudaStream_t s) {
   const int tpt = 128 / g.G;
@@ -358,18 +384,22 @@ static int launch_local_c(const Geometry& g, const void* q, const void* k, const
     if (!tma::make_map(&tm_k, 2, 4, k, dims, sk, box, true)) return PISA_ERR_UNSUPPORTED;
     if (!tma::make_map(&tm_v, 2, 4, v, dims, sv, box, true)) return PISA_ERR_UNSUPPORTED;
   }
-  const size_t smem = (size_t)(2 * 128 * 128) + 4 * (size_t)(2 * C * 128) + 2 * (size_t)(C / 64) * 128 * 128 + 1024;
-  cudaError_t e = cudaFuncSetAttribute(local_window_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const size_t smem = (size_t)(D / 64) * ((size_t)(128 * 128) + 4 * (size_t)(C * 128)) + 2 * (size_t)(C / 64) * 128 * 128 + 1024;
+  cudaError_t e = cudaFuncSetAttribute(local_window_kernel<C, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("local_window attr", e); return PISA_ERR_CUDA; }
   const int grid = a.n_items < num_sms() ? a.n_items : num_sms();
-  local_window_kernel<C><<<grid, kLocalThreads, smem, s>>>(g, tm_q, tm_k, tm_v, a);
+  local_window_kernel<C, D><<<grid, kLocalThreads, smem, s>>>(g, tm_q, tm_k, tm_v, a);
   return check_launch("local_window");
 }
 
 int launch_local_window(const Geometry& g, const void* q, const void* k, const void* v, const float* row_lse,
                         float* o_acc, int32_t* status, cudaStream_t s) {
-  if (g.C == 128) return launch_local_c<128>(g, q, k, v, row_lse, o_acc, status, s);
-  return launch_local_c<64>(g, q, k, v, row_lse, o_acc, status, s);
+  if (g.d == 128) {
+    if (g.C == 128) return launch_local_c<128, 128>(g, q, k, v, row_lse, o_acc, status, s);
+    return launch_local_c<64, 128>(g, q, k, v, row_lse, o_acc, status, s);
+  }
+  if (g.C == 128) return launch_local_c<128, 64>(g, q, k, v, row_lse, o_acc, status, s);
+  return launch_local_c<64, 64>(g, q, k, v, row_lse, o_acc, status, s);
 }
 
 }  // namespace pisa
