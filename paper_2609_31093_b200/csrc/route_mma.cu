@@ -28,9 +28,10 @@ constexpr int kWarpsPerCta = 8;
 
 // MODE: PISA_SCORE_LSE, _MEAN (mean of the children's logits) or _MEAN_VAR (mean + variance / 2), Sec. 4.3
 template <int D, int NT, bool G2, int MODE>
-// three CTAs per SM (at most 85 registers) for the narrow fan-in-2 instantiations: measured 8.5 ms against
-// 8.7 (compiler's choice, 76 registers), 9.3 (64) and 9.7 (128) at the headline shape
-__global__ void __launch_bounds__(kWarpsPerCta * 32, (NT == 1 && G2) ? 3 : 1)
+// three CTAs per SM (at most 85 registers) for the narrow fan-in-2 instantiations at d = 128: measured 8.5 ms against
+// 8.7 (compiler's choice, 76 registers), 9.3 (64) and 9.7 (128) at the headline shape; four at d = 64 (64 registers:
+// 1.54 ms against 2.02 with two, B1 Hq32 Hkv2 d64 N131072 C64 K8)
+__global__ void __launch_bounds__(kWarpsPerCta * 32, (G2 && D == 64) ? 4 : (G2 && NT == 1) ? 3 : 1)
 route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ pyr,
                         int32_t* __restrict__ par_out, float* __restrict__ margin) {
   constexpr int C8 = D / 64;              // groups of four 32-byte chunks per row (one chunk per tig)
