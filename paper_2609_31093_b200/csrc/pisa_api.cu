@@ -494,9 +494,11 @@ static int do_bwd(const pisa_params_t* p, const Geometry& g, const void* q, cons
   });
 }
 
+// v_ready (optional): an event the attention stage must wait for (the values may still be on their way while
+// the routing runs); routed (optional): recorded when idx is final, before the attention stage
 static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, const void* k, const void* v_,
                       void* pyr, int32_t* idx, void* out, float* lse, void* ws, size_t ws_bytes,
-                      cudaStream_t s, bool clear = true) {
+                      cudaStream_t s, bool clear = true, cudaEvent_t v_ready = nullptr, cudaEvent_t routed = nullptr) {
   ForwardPlan pl;
   int st = plan_for(p, g, kOpRoute | kOpBsa, ws_bytes, &pl);
   if (st != PISA_OK) return st;
@@ -513,6 +515,8 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
     // softmax denominators to the attention stage
     st = do_route(p, g, q, k, pyr, idx, nullptr, nullptr, lse, ws, ws_bytes, s);
     if (st != PISA_OK) return st;
+    if (routed != nullptr) cudaEventRecord(routed, s);
+    if (v_ready != nullptr) cudaStreamWaitEvent(s, v_ready, 0);
     stage_mark(2, s);
     st = do_bsa(p, g, q, k, v_, idx, nullptr, out, lse, use_tensor(p, g) && g.score_mode == PISA_SCORE_LSE, true, ws,
                 ws_bytes, s);
@@ -523,11 +527,13 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
       int r = tensor_route(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, pyr, ic, nullptr, nullptr,
                            lc, v.region, (int32_t*)ws, v.stream);
       if (r != PISA_OK) return r;
+      if (v_ready != nullptr) cudaStreamWaitEvent(v.stream, v_ready, 0);
       if (i == 0) stage_mark(2, s);
       return tensor_bsa(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, (const char*)v_ + v.v_off,
                         ic, nullptr, (char*)out + v.o_off, lc, g.score_mode == PISA_SCORE_LSE, true, v.region, (int32_t*)ws,
                         v.stream);
     });
+    if (routed != nullptr) cudaEventRecord(routed, s);    // (chunks: the indices count as final when all chunks have ended)
   }
   stage_mark(3, s);
   kernel_mark("end", s);
@@ -898,7 +904,8 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
 
   // copy streams and the events that order the three stages of every unit
   cudaStream_t s_in = nullptr, s_out = nullptr;
-  cudaEvent_t ev_begin = nullptr, ev_in[kHostSlots] = {}, ev_done[kHostSlots] = {}, ev_out[kHostSlots] = {};
+  cudaEvent_t ev_begin = nullptr, ev_in[kHostSlots] = {}, ev_v[kHostSlots] = {}, ev_routed[kHostSlots] = {},
+              ev_done[kHostSlots] = {}, ev_out[kHostSlots] = {};
   cudaError_t e = cudaSuccess;
   const char* what = "copy streams";
   auto ok = [&](cudaError_t r, const char* w) { if (e == cudaSuccess && r != cudaSuccess) { e = r; what = w; } return e == cudaSuccess; };
@@ -908,6 +915,8 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
   cudaStream_t cs[2] = {s, g_side[1]};                             // compute streams
   for (int i = 0; i < kHostSlots; ++i) {
     ok(cudaEventCreateWithFlags(&ev_in[i], cudaEventDisableTiming), "event create");
+    ok(cudaEventCreateWithFlags(&ev_v[i], cudaEventDisableTiming), "event create");
+    ok(cudaEventCreateWithFlags(&ev_routed[i], cudaEventDisableTiming), "event create");
     ok(cudaEventCreateWithFlags(&ev_done[i], cudaEventDisableTiming), "event create");
     ok(cudaEventCreateWithFlags(&ev_out[i], cudaEventDisableTiming), "event create");
   }
@@ -933,25 +942,29 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
     char* di = dl + A.lb;
     // stage 1: inputs of unit u (its slot was last read by the kernels of the unit that had it before)
     if (u >= kHostSlots) ok(cudaStreamWaitEvent(s_in, ev_done[sl], 0), "stream wait");
-    ok(cudaMemcpy2DAsync(dq, q_w, (const char*)q_host + (size_t)u * q_w, q_pitch, q_w, rows, cudaMemcpyHostToDevice, s_in), "h2d copy");
+    // keys and queries first: the pyramid and the routing start on them while the values are still copied
     ok(cudaMemcpy2DAsync(dk, k_w, (const char*)k_host + (size_t)u * k_w, k_pitch, k_w, rows, cudaMemcpyHostToDevice, s_in), "h2d copy");
-    ok(cudaMemcpy2DAsync(dv, k_w, (const char*)v_host + (size_t)u * k_w, k_pitch, k_w, rows, cudaMemcpyHostToDevice, s_in), "h2d copy");
+    ok(cudaMemcpy2DAsync(dq, q_w, (const char*)q_host + (size_t)u * q_w, q_pitch, q_w, rows, cudaMemcpyHostToDevice, s_in), "h2d copy");
     ok(cudaEventRecord(ev_in[sl], s_in), "event record");
+    ok(cudaMemcpy2DAsync(dv, k_w, (const char*)v_host + (size_t)u * k_w, k_pitch, k_w, rows, cudaMemcpyHostToDevice, s_in), "h2d copy");
+    ok(cudaEventRecord(ev_v[sl], s_in), "event record");
     // stage 2: the kernels (the slot's outputs were last read by the copies of its previous unit); the
     // workspace and pyramid of this compute stream were last used by unit u-2, earlier on the same stream
     ok(cudaStreamWaitEvent(cs[ci], ev_in[sl], 0), "stream wait");
     if (u >= kHostSlots) ok(cudaStreamWaitEvent(cs[ci], ev_out[sl], 0), "stream wait");
     if (e != cudaSuccess) break;
     st = do_forward(&A.unit, A.ug, dq, dk, dv, dpyr + ci * A.pb, (int32_t*)di, dout, (float*)dl, base + ci * A.fwd,
-                    A.fwd, cs[ci], /*clear=*/false);
+                    A.fwd, cs[ci], /*clear=*/false, ev_v[sl], ev_routed[sl]);
     if (st != PISA_OK) break;
     ok(cudaEventRecord(ev_done[sl], cs[ci]), "event record");
-    // stage 3: results of unit u
+    // stage 3: results of unit u; the indices leave as soon as the routing has written them
+    if (idx_host) {
+      ok(cudaStreamWaitEvent(s_out, ev_routed[sl], 0), "stream wait");
+      ok(cudaMemcpy2DAsync((char*)idx_host + (size_t)u * i_w, i_pitch, di, i_w, i_w, (size_t)g.B, cudaMemcpyDeviceToHost, s_out), "d2h copy");
+    }
     ok(cudaStreamWaitEvent(s_out, ev_done[sl], 0), "stream wait");
     ok(cudaMemcpy2DAsync((char*)out_host + (size_t)u * q_w, q_pitch, dout, q_w, q_w, rows, cudaMemcpyDeviceToHost, s_out), "d2h copy");
     ok(cudaMemcpy2DAsync((char*)lse_host + (size_t)u * l_w, l_pitch, dl, l_w, l_w, (size_t)g.B, cudaMemcpyDeviceToHost, s_out), "d2h copy");
-    if (idx_host)
-      ok(cudaMemcpy2DAsync((char*)idx_host + (size_t)u * i_w, i_pitch, di, i_w, i_w, (size_t)g.B, cudaMemcpyDeviceToHost, s_out), "d2h copy");
     ok(cudaEventRecord(ev_out[sl], s_out), "event record");
   }
   // everything this call queued must be finished before its streams and events go away
@@ -968,6 +981,8 @@ int pisa_forward_host(const pisa_params_t* p, const void* q_host, const void* k_
   }
   for (int i = 0; i < kHostSlots; ++i) {
     if (ev_in[i]) cudaEventDestroy(ev_in[i]);
+    if (ev_v[i]) cudaEventDestroy(ev_v[i]);
+    if (ev_routed[i]) cudaEventDestroy(ev_routed[i]);
     if (ev_done[i]) cudaEventDestroy(ev_done[i]);
     if (ev_out[i]) cudaEventDestroy(ev_out[i]);
   }
