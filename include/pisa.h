@@ -215,7 +215,8 @@ int pisa_forward_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32
  * that head are copied back into their places in the host tensors.  The copies run on two internal
  * streams and the kernels of consecutive heads alternate between `stream` and a third internal
  * stream, so two heads' kernels are in flight while the next head is uploaded and the previous one
- * downloaded.
+ * downloaded.  A head's keys and queries are copied first: its pyramid and routing start on them while
+ * its values are still on the way, and its indices are copied back while its attention runs.
  * Host buffers should be pinned (pageable memory makes the copies synchronous); strides must be
  * dense.  Work already queued on `stream` is ordered before the call; the call returns after
  * everything it queued has finished.  This is the one entry point that synchronises.
