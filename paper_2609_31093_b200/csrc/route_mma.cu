@@ -110,24 +110,25 @@ route_stage1_mma_kernel(Geometry geo, const __nv_bfloat16* __restrict__ q, const
           // fan-in 2: both children of a candidate meet in one lane; LSE(a, b) = max + log(1 + e^-|a-b|)
           const int ch_lo = node * 2, ch_hi = ch_lo + 1;
           const bool ok_hi = has && ch_hi < Mb;
-          U32x8 lo[C8], hi[C8];
           // rows without a candidate (kap >= nV: node 0) or without a second child (ragged level: the first
           // child again) load valid summaries all the same; their logits are dropped below
           const long long off_hi = (long long)(ok_hi ? ch_hi : ch_lo) * D;
+          float accs[NT][4];
 #pragma unroll
-          for (int c8 = 0; c8 < C8; ++c8) {
-            lo[c8] = ldg256(below + (long long)ch_lo * D + (c8 * 4 + tig) * 16);
-            hi[c8] = ldg256(below + off_hi + (c8 * 4 + tig) * 16);
+          for (int nt = 0; nt < NT; ++nt) accs[nt][0] = accs[nt][1] = accs[nt][2] = accs[nt][3] = 0.f;
+#pragma unroll
+          for (int c8 = 0; c8 < C8; ++c8) {         // one 64-element group of the row at a time: 16 live data registers
+            const U32x8 lo = ldg256(below + (long long)ch_lo * D + (c8 * 4 + tig) * 16);
+            const U32x8 hi = ldg256(below + off_hi + (c8 * 4 + tig) * 16);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+              for (int i = 0; i < 8; i += 2)
+                mma_bf16_16816(accs[nt], lo.r[i], hi.r[i], lo.r[i + 1], hi.r[i + 1], bq[nt][c8][i], bq[nt][c8][i + 1]);
           }
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) {
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int c8 = 0; c8 < C8; ++c8)
-#pragma unroll
-              for (int i = 0; i < 8; i += 2)
-                mma_bf16_16816(acc, lo[c8].r[i], hi[c8].r[i], lo[c8].r[i + 1], hi[c8].r[i + 1], bq[nt][c8][i],
-                               bq[nt][c8][i + 1]);
+            const float (&acc)[4] = accs[nt];
 #pragma unroll
             for (int jh = 0; jh < 2; ++jh) {
               const float za = acc[jh] * geo.scale, zb = acc[2 + jh] * geo.scale;
