@@ -5,7 +5,8 @@
 #include <string.h>
 
 #include <algorithm>
-#include <vector>
+#include <memory>
+#include <new>
 
 #include "pisa_common.cuh"
 #include "pisa_tensor.cuh"
@@ -815,26 +816,28 @@ int pisa_forward_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32
   float* l_pad = (float*)(o_pad + pa.qb);
   int32_t* i_pad = (int32_t*)((char*)l_pad + pa.lb);
   // the short sequences, longest first
-  std::vector<int> order;
-  order.reserve((size_t)nseq);
+  // (no exception may cross the C boundary: a plain array, allocated without throwing)
+  std::unique_ptr<int[]> order(new (std::nothrow) int[(size_t)nseq + 1]);
+  if (!order) return PISA_ERR_INVALID_ARG;
+  size_t n_short = 0;
   for (int i = 0; i < nseq; ++i) {
     const int len = cu_seqlens[i + 1] - cu_seqlens[i];
     if (len > kPackDirectLen) {
       if ((st = run_alone(i)) != PISA_OK) return st;
     } else if (len > 0) {
-      order.push_back(i);
+      order[n_short++] = i;
     }
   }
-  std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+  std::stable_sort(order.get(), order.get() + n_short, [&](int a, int b) {
     return cu_seqlens[a + 1] - cu_seqlens[a] > cu_seqlens[b + 1] - cu_seqlens[b];
   });
   size_t at = 0;
-  while (at < order.size()) {
+  while (at < n_short) {
     const int first = order[at];
     const int np = pack_grid_len(cu_seqlens[first + 1] - cu_seqlens[first]);
     const long long b_cap = pa.tokens / np < 1 ? 1 : pa.tokens / np;
     size_t end = at + 1;
-    while (end < order.size() && (long long)(end - at) < b_cap) {
+    while (end < n_short && (long long)(end - at) < b_cap) {
       const int len = cu_seqlens[order[end] + 1] - cu_seqlens[order[end]];
       if (4LL * len < 3LL * np) break;
       ++end;
