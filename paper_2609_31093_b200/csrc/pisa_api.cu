@@ -516,8 +516,10 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
     // softmax denominators to the attention stage
     st = do_route(p, g, q, k, pyr, idx, nullptr, nullptr, lse, ws, ws_bytes, s);
     if (st != PISA_OK) return st;
-    if (routed != nullptr) cudaEventRecord(routed, s);
-    if (v_ready != nullptr) cudaStreamWaitEvent(s, v_ready, 0);
+    cudaError_t ee = cudaSuccess;
+    if (routed != nullptr) ee = cudaEventRecord(routed, s);
+    if (ee == cudaSuccess && v_ready != nullptr) ee = cudaStreamWaitEvent(s, v_ready, 0);
+    if (ee != cudaSuccess) { record_cuda_error("forward stage events", ee); return PISA_ERR_CUDA; }
     stage_mark(2, s);
     st = do_bsa(p, g, q, k, v_, idx, nullptr, out, lse, use_tensor(p, g) && g.score_mode == PISA_SCORE_LSE, true, ws,
                 ws_bytes, s);
@@ -528,13 +530,19 @@ static int do_forward(const pisa_params_t* p, const Geometry& g, const void* q, 
       int r = tensor_route(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, pyr, ic, nullptr, nullptr,
                            lc, v.region, (int32_t*)ws, v.stream);
       if (r != PISA_OK) return r;
-      if (v_ready != nullptr) cudaStreamWaitEvent(v.stream, v_ready, 0);
+      if (v_ready != nullptr) {
+        const cudaError_t ee = cudaStreamWaitEvent(v.stream, v_ready, 0);
+        if (ee != cudaSuccess) { record_cuda_error("forward stage events", ee); return (int)PISA_ERR_CUDA; }
+      }
       if (i == 0) stage_mark(2, s);
       return tensor_bsa(v.g, p->dtype, (const char*)q + v.q_off, (const char*)k + v.k_off, (const char*)v_ + v.v_off,
                         ic, nullptr, (char*)out + v.o_off, lc, g.score_mode == PISA_SCORE_LSE, true, v.region, (int32_t*)ws,
                         v.stream);
     });
-    if (routed != nullptr) cudaEventRecord(routed, s);    // (chunks: the indices count as final when all chunks have ended)
+    if (st == PISA_OK && routed != nullptr) {             // (chunks: the indices count as final when all chunks have ended)
+      const cudaError_t ee = cudaEventRecord(routed, s);
+      if (ee != cudaSuccess) { record_cuda_error("forward stage events", ee); return PISA_ERR_CUDA; }
+    }
   }
   stage_mark(3, s);
   kernel_mark("end", s);
