@@ -4,7 +4,10 @@
 //            warps of lse_ws / pv_ws do), 4 or 8 issuing warps per SM, several tiles in flight;
 //   reduce : 2 KB of fp32 per (token, block) pair added into an L2-resident accumulator window with
 //            red.global.add.v4.f32 (what the reducer warps of pv_ws do);
-//   mix    : both at once in the kernels' 1 : 2 byte ratio.
+//   mix    : both at once in the kernels' 1 : 2 byte ratio;
+//   half   : the reduce and the gather stream from half of the SMs (is the limit on the SM's path or in L2?);
+//   bulk   : the reduction stream through the copy engine (cp.reduce.async.bulk from shared memory, 2 KB per
+//            token), alone, from half of the SMs, and side by side with the vector reductions.
 // One CTA per SM.  Prints one line per case: name, milliseconds, TB/s, bytes per clock and SM at the SM
 // clock the run saw.  Build: nvcc -gencode arch=compute_100a,code=sm_100a -O3 l2_streams.cu -o l2_streams
 #include <cstdint>
@@ -49,6 +52,92 @@ __global__ void streams_kernel(const uint8_t* __restrict__ q, long long tok_stri
           asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %1, %1, %1};" ::"l"(dst), "f"(1.0f) : "memory");
         }
   }
+}
+
+// The reduction stream through the copy engine instead of the SM's load/store path: one warp, every lane adds one
+// token's 2 KB (shared memory -> accumulator row) with a bulk reduction, two tiles in flight.
+template <int DEPTH>
+__global__ void bulk_reduce_kernel(const int* __restrict__ tok, int tiles, float* acc, long long acc_tok_stride) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const int lane = threadIdx.x & 31;
+  const int* my = tok + (long long)blockIdx.x * tiles * 32;
+  for (int i = threadIdx.x; i < 2 * 65536 / 4; i += blockDim.x) reinterpret_cast<float*>(smem)[i] = 1.0f;
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    for (int t = 0; t < tiles; ++t) {
+      float* dst = acc + (long long)my[t * 32 + lane] * acc_tok_stride;
+      const uint32_t src = (uint32_t)__cvta_generic_to_shared(smem + (t & 1) * 65536 + lane * 2048);
+      asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(2048)
+                   : "memory");
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(DEPTH - 1) : "memory");
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+}
+
+// Both paths at once: warps 0-3 add the first 16 tokens of a tile with vector reductions, warp 4 the other 16 with
+// bulk reductions.
+__global__ void split_reduce_kernel(const int* __restrict__ tok, int tiles, float* acc, long long acc_tok_stride) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int* my = tok + (long long)blockIdx.x * tiles * 32;
+  for (int i = threadIdx.x; i < 65536 / 4; i += blockDim.x) reinterpret_cast<float*>(smem)[i] = 1.0f;
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
+  if (warp < 4) {
+    for (int t = 0; t < tiles; ++t)
+      for (int i = 0; i < 16; ++i) {
+        float* dst = acc + (long long)my[t * 32 + i] * acc_tok_stride + (warp * 32 + lane) * 4;
+        asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %1, %1, %1};" ::"l"(dst), "f"(1.0f) : "memory");
+      }
+  } else if (lane < 16) {
+    for (int t = 0; t < tiles; ++t) {
+      float* dst = acc + (long long)my[t * 32 + 16 + lane] * acc_tok_stride;
+      const uint32_t src = (uint32_t)__cvta_generic_to_shared(smem + (t & 1) * 32768 + lane * 2048);
+      asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(2048)
+                   : "memory");
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+}
+
+static int run_split(const char* name, const int* tok, int tiles, float* acc, int sms, double clk_hz) {
+  cudaEvent_t a, b;
+  CK(cudaEventCreate(&a)); CK(cudaEventCreate(&b));
+  CK(cudaFuncSetAttribute(split_reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536));
+  split_reduce_kernel<<<sms, 160, 65536>>>(tok, tiles, acc, 512);
+  CK(cudaDeviceSynchronize());
+  CK(cudaEventRecord(a));
+  split_reduce_kernel<<<sms, 160, 65536>>>(tok, tiles, acc, 512);
+  CK(cudaEventRecord(b));
+  CK(cudaDeviceSynchronize());
+  float ms = 0.f;
+  CK(cudaEventElapsedTime(&ms, a, b));
+  const double bytes = (double)sms * tiles * 65536.0;
+  printf("%-44s %8.3f ms %6.2f TB/s %6.1f B/clk/SM\n", name, ms, bytes / ms * 1e-9, bytes / sms / (ms * 1e-3 * clk_hz));
+  return 0;
+}
+
+template <int DEPTH>
+static int run_bulk(const char* name, const int* tok, int tiles, float* acc, int sms, double clk_hz) {
+  cudaEvent_t a, b;
+  CK(cudaEventCreate(&a)); CK(cudaEventCreate(&b));
+  CK(cudaFuncSetAttribute(bulk_reduce_kernel<DEPTH>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 65536));
+  bulk_reduce_kernel<DEPTH><<<sms, 128, 2 * 65536>>>(tok, tiles, acc, 512);
+  CK(cudaDeviceSynchronize());
+  CK(cudaEventRecord(a));
+  bulk_reduce_kernel<DEPTH><<<sms, 128, 2 * 65536>>>(tok, tiles, acc, 512);
+  CK(cudaEventRecord(b));
+  CK(cudaDeviceSynchronize());
+  float ms = 0.f;
+  CK(cudaEventElapsedTime(&ms, a, b));
+  const double bytes = (double)sms * tiles * 65536.0;
+  printf("%-44s %8.3f ms %6.2f TB/s %6.1f B/clk/SM\n", name, ms, bytes / ms * 1e-9, bytes / sms / (ms * 1e-3 * clk_hz));
+  return 0;
 }
 
 static int run(const char* name, const uint8_t* q, const int* tok, int tiles, int gw, int rw, float* acc, int sms,
@@ -101,5 +190,12 @@ int main() {
   if (run("mix: gather 4 warps + reduce 4 warps", q, tok, tiles, 4, 4, acc, sms, clk)) return 1;
   if (run("mix: gather 8 warps + reduce 4 warps", q, tok, tiles, 8, 4, acc, sms, clk)) return 1;
   if (run("mix: gather 8 warps + reduce 8 warps", q, tok, tiles, 8, 8, acc, sms, clk)) return 1;
+  // the same streams from half of the SMs: a limit that sits in L2 leaves the total where it was (twice the rate per
+  // active SM), a limit on the SM's own path halves the total
+  if (run("reduce fp32 v4, 4 warps, half of the SMs", q, tok, tiles, 0, 4, acc, sms / 2, clk)) return 1;
+  if (run("gather 1 KB pieces, 4 warps, half of the SMs", q, tok, tiles, 4, 0, acc, sms / 2, clk)) return 1;
+  if (run_bulk<2>("bulk reductions of 2 KB, 2 tiles in flight", tok, tiles, acc, sms, clk)) return 1;
+  if (run_bulk<2>("bulk reductions of 2 KB, half of the SMs", tok, tiles, acc, sms / 2, clk)) return 1;
+  if (run_split("half vector reductions, half bulk reductions", tok, tiles, acc, sms, clk)) return 1;
   return 0;
 }
