@@ -105,6 +105,50 @@ __global__ void split_reduce_kernel(const int* __restrict__ tok, int tiles, floa
   }
 }
 
+// Both paths from the same four warps, no barrier between them: every warp adds its 512-byte column share of 24 of a
+// tile's tokens with vector reductions and of the other 8 with one bulk reduction each (lanes 0-7 issue them).
+__global__ void warp_split_kernel(const int* __restrict__ tok, int tiles, float* acc, long long acc_tok_stride) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int* my = tok + (long long)blockIdx.x * tiles * 32;
+  for (int i = threadIdx.x; i < 32768 / 4; i += blockDim.x) reinterpret_cast<float*>(smem)[i] = 1.0f;
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
+  for (int t = 0; t < tiles; ++t) {
+    for (int i = 0; i < 24; ++i) {
+      float* dst = acc + (long long)my[t * 32 + i] * acc_tok_stride + (warp * 32 + lane) * 4;
+      asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %1, %1, %1};" ::"l"(dst), "f"(1.0f) : "memory");
+    }
+    if (lane < 8) {
+      float* dst = acc + (long long)my[t * 32 + 24 + lane] * acc_tok_stride + warp * 128;
+      const uint32_t src = (uint32_t)__cvta_generic_to_shared(smem + (t & 1) * 16384 + warp * 4096 + lane * 512);
+      asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(512)
+                   : "memory");
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+    }
+    __syncwarp();
+  }
+  if (lane < 8) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+static int run_warp_split(const char* name, const int* tok, int tiles, float* acc, int sms, double clk_hz) {
+  cudaEvent_t a, b;
+  CK(cudaEventCreate(&a)); CK(cudaEventCreate(&b));
+  CK(cudaFuncSetAttribute(warp_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768));
+  warp_split_kernel<<<sms, 128, 32768>>>(tok, tiles, acc, 512);
+  CK(cudaDeviceSynchronize());
+  CK(cudaEventRecord(a));
+  warp_split_kernel<<<sms, 128, 32768>>>(tok, tiles, acc, 512);
+  CK(cudaEventRecord(b));
+  CK(cudaDeviceSynchronize());
+  float ms = 0.f;
+  CK(cudaEventElapsedTime(&ms, a, b));
+  const double bytes = (double)sms * tiles * 65536.0;
+  printf("%-44s %8.3f ms %6.2f TB/s %6.1f B/clk/SM\n", name, ms, bytes / ms * 1e-9, bytes / sms / (ms * 1e-3 * clk_hz));
+  return 0;
+}
+
 static int run_split(const char* name, const int* tok, int tiles, float* acc, int sms, double clk_hz) {
   cudaEvent_t a, b;
   CK(cudaEventCreate(&a)); CK(cudaEventCreate(&b));
@@ -197,5 +241,6 @@ int main() {
   if (run_bulk<2>("bulk reductions of 2 KB, 2 tiles in flight", tok, tiles, acc, sms, clk)) return 1;
   if (run_bulk<2>("bulk reductions of 2 KB, half of the SMs", tok, tiles, acc, sms / 2, clk)) return 1;
   if (run_split("half vector reductions, half bulk reductions", tok, tiles, acc, sms, clk)) return 1;
+  if (run_warp_split("3/4 vector, 1/4 bulk (512 B), per warp", tok, tiles, acc, sms, clk)) return 1;
   return 0;
 }

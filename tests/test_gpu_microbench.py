@@ -25,4 +25,4 @@ def test_l2_stream_microbenchmark_runs_and_reports(tmp_path):
         if " TB/s" in line:
             name = line[:44].strip()
             rates[name] = float(line.split(" ms")[1].split("TB/s")[0])
-    assert len(rates) == 12 and all(0.5 < r < 20.0 for r in rates.values()), rates
+    assert len(rates) == 13 and all(0.5 < r < 20.0 for r in rates.values()), rates
