@@ -125,12 +125,17 @@ class ClockSampler:
         self.lines = []
         self.proc = None
         self.gpu_id = gpu_id
+        self.first = 0              # index of the first sample that belongs to the timed region
+
+    def mark(self):
+        """The timed region starts now: samples taken before this call are dropped."""
+        self.first = len(self.lines)
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "25"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -143,7 +148,7 @@ class ClockSampler:
     def stop(self) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        n_end = len(self.lines)       # samples that arrived while the timed region ran
         self.proc.terminate()
         try:
             self.proc.wait(timeout=2)
@@ -151,7 +156,7 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        for ln in self.lines[self.first:max(n_end, self.first + 1)]:
             parts = [x.strip() for x in ln.split(",")]
             if len(parts) < 7:
                 continue
@@ -330,6 +335,13 @@ def run_ours(args):
     def step():
         P.pisa_forward(p, q, k, v, pyramid, idx, out, lse, ws)
 
+    props = torch.cuda.get_device_properties(local)
+    gpu_id = str(local)
+    if hasattr(props, "uuid"):
+        u = str(props.uuid)
+        gpu_id = u if u.startswith("GPU-") else "GPU-" + u
+    sampler = ClockSampler(gpu_id)
+    sampler.start()                  # nvidia-smi takes a moment to come up: it runs through the warm-up
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
@@ -338,19 +350,13 @@ def run_ours(args):
         raise SystemExit(f"device status {st} after warm-up")
 
     P.set_stage_timing(True)
-    props = torch.cuda.get_device_properties(local)
-    gpu_id = str(local)
-    if hasattr(props, "uuid"):
-        u = str(props.uuid)
-        gpu_id = u if u.startswith("GPU-") else "GPU-" + u
-    sampler = ClockSampler(gpu_id)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     stage = np.zeros(3)
     kernels = {}
     launches_of = {}
     barrier()
     torch.cuda.synchronize()
-    sampler.start()
+    sampler.mark()
     l0 = P.launch_count()
     ev0.record()
     for _ in range(args.steps):
