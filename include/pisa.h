@@ -202,6 +202,19 @@ int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const voi
  * one after the other instead; the results are the same rows either way (up to the rounding order of
  * the fp32 partial sums).
  */
+/*
+ * The grouping pisa_forward_packed applies, as host arithmetic only (no GPU work, nothing allocated on the
+ * device): for sequence i, group[i] = the padded batch it runs in (0, 1, ... in launch order) and
+ * padded[i] = that batch's padded length; group[i] = -1 (padded[i] = its own length) for a sequence that
+ * runs alone -- longer than 8192 tokens, alone in its length class, or empty.
+ *   p, cu_seqlens, nseq : as for pisa_forward_packed
+ *   group, padded       : HOST int32 [nseq], written
+ *   n_groups            : HOST, nullable; receives the number of padded batches
+ * Returns PISA_ERR_INVALID_ARG for null pointers, cu_seqlens[0] != 0, or a length outside [0, p->N].
+ */
+int pisa_packed_plan(const pisa_params_t* p, const int32_t* cu_seqlens, int32_t nseq, int32_t* group,
+                     int32_t* padded, int32_t* n_groups);
+
 int pisa_forward_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32_t nseq, const void* q,
                         const void* k, const void* v, void* pyramid, int32_t* idx, void* out, float* lse,
                         void* ws, size_t ws_bytes, void* stream);

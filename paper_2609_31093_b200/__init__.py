@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     pisa_forward,
     pisa_forward_host,
     pisa_forward_packed,
+    packed_plan,
     pisa_flat_select,
     pisa_bsa_bwd,
     pisa_bsa_bwd_packed,

@@ -61,6 +61,7 @@ def lib():
     L.pisa_bsa_bwd.argtypes = [pp] + [vp] * 11 + [C.c_size_t, vp]
     L.pisa_forward_packed.argtypes = [pp, i32p, C.c_int32] + [vp] * 8 + [C.c_size_t, vp]
     L.pisa_bsa_bwd_packed.argtypes = [pp, i32p, C.c_int32] + [vp] * 11 + [C.c_size_t, vp]
+    L.pisa_packed_plan.argtypes = [pp, i32p, C.c_int32, i32p, i32p, i32p]
     L.pisa_read_status.argtypes = [vp, i32p]
     L.pisa_route_static.argtypes = [pp, vp, vp, vp, vp, vp, vp]
     L.pisa_route_static.restype = C.c_int
@@ -76,7 +77,7 @@ def lib():
     for name in ("pisa_pyramid_layout", "pisa_workspace_bytes", "pisa_build_pyramid", "pisa_route",
                  "pisa_bsa_fwd", "pisa_forward", "pisa_forward_host", "pisa_flat_select", "pisa_read_status",
                  "pisa_decode_step", "pisa_pyramid_regrow", "pisa_bsa_bwd", "pisa_forward_packed", "pisa_bsa_bwd_packed",
-                 "pisa_set_stage_timing", "pisa_get_stage_ms", "pisa_set_forward_chunks"):
+                 "pisa_set_stage_timing", "pisa_get_stage_ms", "pisa_set_forward_chunks", "pisa_packed_plan"):
         getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -200,6 +201,15 @@ def pisa_forward_packed(p: Params, cu_seqlens, q, k, v, pyramid, idx, out, lse, 
     _check(lib().pisa_forward_packed(p.ref(), cu, len(cu_seqlens) - 1, _ptr(q), _ptr(k), _ptr(v), _ptr(pyramid),
                                      _ptr(idx), _ptr(out), _ptr(lse), _ptr(ws), ws.numel(), _stream()),
            "pisa_forward_packed")
+
+
+def packed_plan(p: Params, cu_seqlens):
+    """Host-only: (group, padded, n_groups) of pisa_forward_packed's grouping; group -1 = the sequence runs alone."""
+    n = len(cu_seqlens) - 1
+    cu = (C.c_int32 * len(cu_seqlens))(*[int(x) for x in cu_seqlens])
+    group, padded, ng = (C.c_int32 * max(n, 1))(), (C.c_int32 * max(n, 1))(), C.c_int32(0)
+    _check(lib().pisa_packed_plan(p.ref(), cu, n, group, padded, C.byref(ng)), "pisa_packed_plan")
+    return list(group)[:n], list(padded)[:n], int(ng.value)
 
 
 def pisa_forward_host(p: Params, q_host, k_host, v_host, out_host, lse_host, idx_host, ws):

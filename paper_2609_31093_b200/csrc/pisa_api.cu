@@ -677,6 +677,60 @@ static int packed_arena(const pisa_params_t* p, PackedArena* a) {
   return PISA_OK;
 }
 
+// The grouping of pisa_forward_packed, host arithmetic only.  order: the sequences that take part in groups,
+// longest first (nseq + 1 ints of scratch); group[i] / padded[i] for sequence i: its group (0, 1, ... in launch
+// order) and the group's padded length, or group -1 for a sequence that runs alone (longer than kPackDirectLen, the
+// only one of its length class, or empty: padded = its own length).  Returns the number of groups.
+static int packed_plan(const pisa_params_t* p, const int32_t* cu, int nseq, long long tokens, int* order,
+                       int32_t* group, int32_t* padded) {
+  size_t n_short = 0;
+  for (int i = 0; i < nseq; ++i) {
+    const int len = cu[i + 1] - cu[i];
+    group[i] = -1;
+    padded[i] = len;
+    if (len > 0 && len <= kPackDirectLen) order[n_short++] = i;
+  }
+  std::stable_sort(order, order + n_short, [&](int a, int b) { return cu[a + 1] - cu[a] > cu[b + 1] - cu[b]; });
+  int n_groups = 0;
+  size_t at = 0;
+  while (at < n_short) {
+    const int np = pack_grid_len(cu[order[at] + 1] - cu[order[at]]);
+    const long long b_cap = tokens / np < 1 ? 1 : tokens / np;
+    size_t end = at + 1;
+    while (end < n_short && (long long)(end - at) < b_cap) {
+      const int len = cu[order[end] + 1] - cu[order[end]];
+      if (4LL * len < 3LL * np) break;
+      ++end;
+    }
+    if (end - at >= 2) {
+      for (size_t j = at; j < end; ++j) { group[order[j]] = n_groups; padded[order[j]] = np; }
+      ++n_groups;
+    }
+    at = end;
+  }
+  (void)p;
+  return n_groups;
+}
+
+int pisa_packed_plan(const pisa_params_t* p, const int32_t* cu_seqlens, int32_t nseq, int32_t* group, int32_t* padded,
+                     int32_t* n_groups) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  if (!cu_seqlens || nseq < 0 || !group || !padded || cu_seqlens[0] != 0) return PISA_ERR_INVALID_ARG;
+  for (int i = 0; i < nseq; ++i) {
+    const int len = cu_seqlens[i + 1] - cu_seqlens[i];
+    if (len < 0 || len > p->N) return PISA_ERR_INVALID_ARG;
+  }
+  PackedArena pa;
+  if ((st = packed_arena(p, &pa)) != PISA_OK) return st;
+  std::unique_ptr<int[]> order(new (std::nothrow) int[(size_t)nseq + 1]);
+  if (!order) return PISA_ERR_INVALID_ARG;
+  const int n = packed_plan(p, cu_seqlens, nseq, pa.tokens, order.get(), group, padded);
+  if (n_groups) *n_groups = n;
+  return PISA_OK;
+}
+
 int pisa_workspace_bytes(const pisa_params_t* p, int op, size_t* bytes) {
   Geometry g;
   int st = resolve(p, &g);
@@ -823,39 +877,28 @@ int pisa_forward_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32
   char* o_pad = v_pad + pa.kb;
   float* l_pad = (float*)(o_pad + pa.qb);
   int32_t* i_pad = (int32_t*)((char*)l_pad + pa.lb);
-  // the short sequences, longest first
-  // (no exception may cross the C boundary: a plain array, allocated without throwing)
+  // the plan: which sequences share a padded batch (host arithmetic, see packed_plan), then group by group
+  // (no exception may cross the C boundary: plain arrays, allocated without throwing)
   std::unique_ptr<int[]> order(new (std::nothrow) int[(size_t)nseq + 1]);
-  if (!order) return PISA_ERR_INVALID_ARG;
+  std::unique_ptr<int32_t[]> group(new (std::nothrow) int32_t[(size_t)nseq + 1]);
+  std::unique_ptr<int32_t[]> padded(new (std::nothrow) int32_t[(size_t)nseq + 1]);
+  if (!order || !group || !padded) return PISA_ERR_INVALID_ARG;
+  packed_plan(p, cu_seqlens, nseq, pa.tokens, order.get(), group.get(), padded.get());
+  for (int i = 0; i < nseq; ++i)
+    if (group[i] < 0 && (st = run_alone(i)) != PISA_OK) return st;
+  // `order` lists the grouped candidates longest first; the members of a group are consecutive in it
   size_t n_short = 0;
   for (int i = 0; i < nseq; ++i) {
     const int len = cu_seqlens[i + 1] - cu_seqlens[i];
-    if (len > kPackDirectLen) {
-      if ((st = run_alone(i)) != PISA_OK) return st;
-    } else if (len > 0) {
-      order[n_short++] = i;
-    }
+    if (len > 0 && len <= kPackDirectLen) ++n_short;
   }
-  std::stable_sort(order.get(), order.get() + n_short, [&](int a, int b) {
-    return cu_seqlens[a + 1] - cu_seqlens[a] > cu_seqlens[b + 1] - cu_seqlens[b];
-  });
   size_t at = 0;
   while (at < n_short) {
     const int first = order[at];
-    const int np = pack_grid_len(cu_seqlens[first + 1] - cu_seqlens[first]);
-    const long long b_cap = pa.tokens / np < 1 ? 1 : pa.tokens / np;
+    if (group[first] < 0) { ++at; continue; }
     size_t end = at + 1;
-    while (end < n_short && (long long)(end - at) < b_cap) {
-      const int len = cu_seqlens[order[end] + 1] - cu_seqlens[order[end]];
-      if (4LL * len < 3LL * np) break;
-      ++end;
-    }
-    const int nb = (int)(end - at);
-    if (nb == 1) {
-      if ((st = run_alone(first)) != PISA_OK) return st;
-      at = end;
-      continue;
-    }
+    while (end < n_short && group[order[end]] == group[first]) ++end;
+    const int nb = (int)(end - at), np = padded[first];
     pisa_params_t pg = *p;
     pg.B = nb;
     pg.N = np;
