@@ -179,3 +179,41 @@ def test_many_short_sequences_run_as_a_few_launch_sets():
         o_g = out[t0:t0 + n].cpu()[ti[:, 2:3], heads].double().numpy()            # [S, G, d]
         l_g = lse[Hq * t0:Hq * (t0 + n)].view(Hq, n).cpu()[heads, ti[:, 2:3]].double().numpy()
         T.check_forward_rows(w, prob, tri, gi, o_g, l_g)
+
+
+def test_packed_groups_on_the_exact_fp32_path():
+    """fp32 inputs (d = 32: the SIMT kernels) through the padded groups: batches of several sequences through the
+    exact-arithmetic path, sampled sequences against the oracle run on each sequence alone."""
+    rng = np.random.default_rng(99)
+    lens = rng.integers(1, 301, size=40).tolist()
+    Hq, Hkv, d, C, g, K = 4, 2, 32, 64, 2, 5
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    total = int(cu[-1])
+    w_all = S.Workload("pk_f32", 1, total, Hq, Hkv, d, C, g, K, "fp32", 4250, "iid")
+    t_all = S.make_inputs(w_all)
+    q, k, v = (T.to_torch(t_all[x][0], "fp32") for x in ("q", "k", "v"))
+    p = P.Params(1, max(lens), Hq, Hkv, d, C, g, K, dtype="fp32")
+    group, padded, n_groups = P.packed_plan(p, cu.tolist())
+    assert n_groups >= 3
+    pyramid = PB.alloc_pyramid(p)
+    ws = PB.alloc_workspace(p, PB.OP_FORWARD_PACKED)
+    idx = torch.full((Hkv * K * total,), -7, dtype=torch.int32, device="cuda")
+    out = torch.zeros_like(q)
+    lse = torch.zeros((Hq * total,), dtype=torch.float32, device="cuda")
+    P.pisa_forward_packed(p, cu.tolist(), q, k, v, pyramid, idx, out, lse, ws)
+    torch.cuda.synchronize()
+    assert P.read_status(ws) == 0
+    assert int((idx == -7).sum()) == 0
+    G = Hq // Hkv
+    for i in rng.choice(40, size=6, replace=False).tolist() + [int(np.argmax(lens))]:
+        n, t0 = lens[i], int(cu[i])
+        w = S.Workload(f"pk_f32_{i}", 1, n, Hq, Hkv, d, C, g, K, "fp32", 0, "iid")
+        t = {key: t_all[key][:, t0:t0 + n] for key in ("q", "k", "v")}
+        tri = S.sample_queries(w, 8)
+        prob = T.oracle_problem(w, t)
+        ti = torch.from_numpy(tri)
+        gi = idx[Hkv * K * t0:Hkv * K * (t0 + n)].view(Hkv, n, K).cpu()[ti[:, 1], ti[:, 2]].numpy()
+        heads = ti[:, 1:2] * G + torch.arange(G)[None, :]
+        o_g = out[t0:t0 + n].cpu()[ti[:, 2:3], heads].double().numpy()
+        l_g = lse[Hq * t0:Hq * (t0 + n)].view(Hq, n).cpu()[heads, ti[:, 2:3]].double().numpy()
+        T.check_forward_rows(w, prob, tri, gi, o_g, l_g)
