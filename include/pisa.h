@@ -51,7 +51,8 @@ enum { PISA_BF16 = 0, PISA_FP32 = 1 };
 enum { PISA_SCORE_LSE = 0, PISA_SCORE_MEAN = 1, PISA_SCORE_MEAN_VAR = 2 };
 /* operations a workspace can be sized for */
 enum { PISA_OP_ROUTE = 0, PISA_OP_BSA = 1, PISA_OP_FORWARD = 2, PISA_OP_FLAT = 3, PISA_OP_FORWARD_HOST = 4,
-       PISA_OP_DECODE = 5, PISA_OP_BSA_BWD = 6, PISA_OP_FORWARD_PACKED = 7 };
+       PISA_OP_DECODE = 5, PISA_OP_BSA_BWD = 6, PISA_OP_FORWARD_PACKED = 7,
+       PISA_OP_BSA_BWD_PACKED = 8 };
 /* implementation selector (params.impl): AUTO picks the tensor-core path where it applies */
 enum { PISA_IMPL_AUTO = 0, PISA_IMPL_SIMT = 1, PISA_IMPL_TENSOR = 2 };
 /*
@@ -265,7 +266,10 @@ int pisa_bsa_bwd(const pisa_params_t* p, const void* q, const void* k, const voi
  *   p, cu_seqlens, nseq : as for pisa_forward_packed (B = 1, dense strides, p->N the longest sequence)
  *   q, out, dout, dq    : device [total, Hq, d];  k, v, dk, dv : device [total, Hkv, d]
  *   idx, lse            : sequence-major, as pisa_forward_packed wrote them
- *   ws                  : device workspace sized for PISA_OP_BSA_BWD with p
+ *   ws                  : device workspace sized for PISA_OP_BSA_BWD_PACKED with p: the short sequences then run in
+ *                         the groups pisa_packed_plan reports, each group as one padded batch (a padded query row is
+ *                         given idx = -1 and so contributes to no gradient); a workspace sized for PISA_OP_BSA_BWD
+ *                         is accepted too and runs one backward per sequence
  *
  * All sequences are validated before anything is queued; one unsupported sequence fails the call.
  */

@@ -13,7 +13,7 @@ _lib = None
 
 BF16, FP32 = 0, 1
 SCORE_LSE, SCORE_MEAN, SCORE_MEAN_VAR = 0, 1, 2
-OP_ROUTE, OP_BSA, OP_FORWARD, OP_FLAT, OP_FORWARD_HOST, OP_DECODE, OP_BSA_BWD, OP_FORWARD_PACKED = 0, 1, 2, 3, 4, 5, 6, 7
+OP_ROUTE, OP_BSA, OP_FORWARD, OP_FLAT, OP_FORWARD_HOST, OP_DECODE, OP_BSA_BWD, OP_FORWARD_PACKED, OP_BSA_BWD_PACKED = 0, 1, 2, 3, 4, 5, 6, 7, 8
 IMPL_AUTO, IMPL_SIMT, IMPL_TENSOR = 0, 1, 2
 DEBUG_BOUNDS = 1
 _SCORE = {"lse": SCORE_LSE, "mean": SCORE_MEAN, "mean_var": SCORE_MEAN_VAR}

@@ -13,11 +13,11 @@ namespace pisa {
 
 namespace {
 
-// packed -> padded, q / k / v in one launch (blockIdx.z picks the tensor); 16-byte vectors
+// packed <-> padded rows of up to five tensors in one launch (blockIdx.z picks the tensor); 16-byte vectors
 struct PackSrc {
-  const uint4* src[3];
-  uint4* dst[3];
-  int row_vec[3];                 // 16-byte vectors per token row (H * d * elem / 16)
+  const uint4* src[5];
+  uint4* dst[5];
+  int row_vec[5];                 // 16-byte vectors per token row (H * d * elem / 16)
 };
 
 __global__ void __launch_bounds__(256) pack_gather_kernel(PackSrc a, PackTable tab, int b_first, int Np) {
@@ -74,6 +74,52 @@ __global__ void __launch_bounds__(256) pack_scatter_kernel(UnpackArgs a, PackTab
   }
 }
 
+// padded -> packed: the valid rows only (the gradients of a padded batch)
+__global__ void __launch_bounds__(256) pack_scatter_rows_kernel(PackSrc a, PackTable tab, int b_first, int Np) {
+  const int z = blockIdx.z, bl = blockIdx.y;
+  const int rv = a.row_vec[z];
+  const long long n_valid = (long long)tab.len[bl] * rv;
+  const uint4* src = a.src[z] + (long long)(b_first + bl) * Np * rv;
+  uint4* dst = a.dst[z] + (long long)tab.off[bl] * rv;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_valid; i += (long long)gridDim.x * blockDim.x)
+    dst[i] = src[i];
+}
+
+// packed -> padded for what the backward reads beside the rows: idx sequence-major [Hkv, len, K] -> [B', Hkv, Np, K]
+// with -1 past the end (a padded query row then has no blocks and adds nothing to any key's gradient), lse
+// sequence-major [Hq, len] -> [B', Hq, Np] with 0 past the end
+struct PackMeta {
+  const int32_t* idx;
+  int32_t* idx_pad;
+  const float* lse;
+  float* lse_pad;
+  int Hq, Hkv, K;
+};
+__global__ void __launch_bounds__(256) pack_gather_meta_kernel(PackMeta a, PackTable tab, int b_first, int Np) {
+  const int z = blockIdx.z, bl = blockIdx.y;
+  const long long off = tab.off[bl];
+  const int len = tab.len[bl];
+  const long long b = b_first + bl;
+  const long long tid0 = (long long)blockIdx.x * blockDim.x + threadIdx.x, step = (long long)gridDim.x * blockDim.x;
+  if (z == 0) {
+    const long long row = (long long)Np * a.K, n = (long long)a.Hkv * row;
+    const int32_t* src = a.idx + off * a.Hkv * a.K;
+    int32_t* dst = a.idx_pad + b * n;
+    for (long long i = tid0; i < n; i += step) {
+      const long long h = i / row, r = i - h * row;                 // r = t * K + slot
+      dst[i] = (r < (long long)len * a.K) ? src[h * (long long)len * a.K + r] : -1;
+    }
+  } else {
+    const long long n = (long long)a.Hq * Np;
+    const float* src = a.lse + off * a.Hq;
+    float* dst = a.lse_pad + b * n;
+    for (long long i = tid0; i < n; i += step) {
+      const long long h = i / Np, t = i - h * Np;
+      dst[i] = (t < len) ? src[h * len + t] : 0.f;
+    }
+  }
+}
+
 int grid_x(long long work) {
   long long gx = (work + 255) / 256;
   const long long cap = 8LL * num_sms();
@@ -85,7 +131,7 @@ int grid_x(long long work) {
 
 int launch_pack_gather(const Geometry& g, int elem_bytes, const void* q, const void* k, const void* v, void* q_pad,
                        void* k_pad, void* v_pad, const PackTable& tab, int b_first, cudaStream_t s) {
-  PackSrc a;
+  PackSrc a = {};
   a.src[0] = (const uint4*)q; a.src[1] = (const uint4*)k; a.src[2] = (const uint4*)v;
   a.dst[0] = (uint4*)q_pad; a.dst[1] = (uint4*)k_pad; a.dst[2] = (uint4*)v_pad;
   a.row_vec[0] = g.Hq * g.d * elem_bytes / 16;
@@ -107,6 +153,40 @@ int launch_pack_scatter(const Geometry& g, int elem_bytes, const void* out_pad, 
   dim3 grid(grid_x((long long)g.N * a.out_row_vec), tab.n, 3);
   pack_scatter_kernel<<<grid, 256, 0, s>>>(a, tab, b_first, g.N);
   return check_launch("pack_scatter");
+}
+
+// the backward's extra inputs: out and dout rows (zero past the end), idx and lse
+int launch_pack_gather_bwd(const Geometry& g, int elem_bytes, const void* out, const void* dout, const int32_t* idx,
+                           const float* lse, void* out_pad, void* dout_pad, int32_t* idx_pad, float* lse_pad,
+                           const PackTable& tab, int b_first, cudaStream_t s) {
+  PackSrc a = {};
+  a.src[0] = (const uint4*)out; a.src[1] = (const uint4*)dout;
+  a.dst[0] = (uint4*)out_pad; a.dst[1] = (uint4*)dout_pad;
+  a.row_vec[0] = a.row_vec[1] = g.Hq * g.d * elem_bytes / 16;
+  dim3 grid(grid_x((long long)g.N * a.row_vec[0]), tab.n, 2);
+  pack_gather_kernel<<<grid, 256, 0, s>>>(a, tab, b_first, g.N);
+  int st = check_launch("pack_gather_bwd");
+  if (st != PISA_OK) return st;
+  PackMeta m;
+  m.idx = idx; m.idx_pad = idx_pad; m.lse = lse; m.lse_pad = lse_pad;
+  m.Hq = g.Hq; m.Hkv = g.Hkv; m.K = g.K;
+  dim3 grid2(grid_x((long long)g.N * g.Hkv * g.K), tab.n, 2);
+  pack_gather_meta_kernel<<<grid2, 256, 0, s>>>(m, tab, b_first, g.N);
+  return check_launch("pack_gather_meta");
+}
+
+// the gradients of the valid rows back to the packed tensors
+int launch_pack_scatter_grads(const Geometry& g, int elem_bytes, const void* dq_pad, const void* dk_pad,
+                              const void* dv_pad, void* dq, void* dk, void* dv, const PackTable& tab, int b_first,
+                              cudaStream_t s) {
+  PackSrc a = {};
+  a.src[0] = (const uint4*)dq_pad; a.src[1] = (const uint4*)dk_pad; a.src[2] = (const uint4*)dv_pad;
+  a.dst[0] = (uint4*)dq; a.dst[1] = (uint4*)dk; a.dst[2] = (uint4*)dv;
+  a.row_vec[0] = g.Hq * g.d * elem_bytes / 16;
+  a.row_vec[1] = a.row_vec[2] = g.Hkv * g.d * elem_bytes / 16;
+  dim3 grid(grid_x((long long)g.N * a.row_vec[0]), tab.n, 3);
+  pack_scatter_rows_kernel<<<grid, 256, 0, s>>>(a, tab, b_first, g.N);
+  return check_launch("pack_scatter_grads");
 }
 
 }  // namespace pisa

@@ -677,6 +677,53 @@ static int packed_arena(const pisa_params_t* p, PackedArena* a) {
   return PISA_OK;
 }
 
+// ... and what pisa_bsa_bwd_packed needs to run the same groups: the backward's workspace for any group, padded q /
+// out / dout / dq, k / v / dk / dv, lse and idx
+struct PackedBwdArena {
+  long long tokens;
+  size_t bwd, qb, kb, lb, ib, total;
+};
+static int packed_bwd_arena(const pisa_params_t* p, PackedBwdArena* a) {
+  Geometry g;
+  int st = resolve(p, &g);
+  if (st != PISA_OK) return st;
+  a->tokens = kPackTokens;
+  auto need = [](const pisa_params_t* pp, const Geometry& gg, size_t* out) -> int {
+    if (!tensor_bwd_supported(gg, pp->dtype) || pp->impl == PISA_IMPL_SIMT) return PISA_ERR_UNSUPPORTED;
+    size_t b = kStatusBytes + tensor_bwd_workspace_bytes(gg);
+    ForwardPlan pl;
+    const int r = forward_plan(pp, gg, kOpBwd, &pl);
+    if (r != PISA_OK) return r;
+    if (pl.total > b) b = pl.total;
+    *out = b;
+    return PISA_OK;
+  };
+  size_t bwd = 0;
+  if ((st = need(p, g, &bwd)) != PISA_OK) return st;
+  const int n_max = p->N < kPackDirectLen ? p->N : kPackDirectLen;
+  for (int k = 0; k < 31; ++k)
+    for (int m = 8; m <= 15; ++m) {
+      const long long np = (long long)m << k;
+      if (np > pack_grid_len(n_max)) continue;
+      pisa_params_t pg = *p;
+      pg.N = (int)np;
+      pg.B = (int)(a->tokens / np < 1 ? 1 : a->tokens / np);
+      Geometry gg;
+      if ((st = resolve(&pg, &gg)) != PISA_OK) return st;
+      size_t b = 0;
+      if ((st = need(&pg, gg, &b)) != PISA_OK) return st;
+      if (b > bwd) bwd = b;
+    }
+  const size_t es = elem_size(p->dtype), tok = (size_t)a->tokens;
+  a->bwd = align_up(bwd, 256);
+  a->qb = align_up(tok * g.Hq * g.d * es, 256);
+  a->kb = align_up(tok * g.Hkv * g.d * es, 256);
+  a->lb = align_up(tok * g.Hq * sizeof(float), 256);
+  a->ib = align_up(tok * g.Hkv * g.K * sizeof(int32_t), 256);
+  a->total = a->bwd + 4 * a->qb + 4 * a->kb + a->lb + a->ib;
+  return PISA_OK;
+}
+
 // The grouping of pisa_forward_packed, host arithmetic only.  order: the sequences that take part in groups,
 // longest first (nseq + 1 ints of scratch); group[i] / padded[i] for sequence i: its group (0, 1, ... in launch
 // order) and the group's padded length, or group -1 for a sequence that runs alone (longer than kPackDirectLen, the
@@ -768,6 +815,13 @@ int pisa_workspace_bytes(const pisa_params_t* p, int op, size_t* bytes) {
       if (!decode_supported(g, p->dtype)) return PISA_ERR_UNSUPPORTED;
       *bytes = kStatusBytes + decode_workspace_bytes(g);
       break;
+    case PISA_OP_BSA_BWD_PACKED: {
+      PackedBwdArena pa;
+      st = packed_bwd_arena(p, &pa);
+      if (st != PISA_OK) return st;
+      *bytes = pa.total;
+      break;
+    }
     case PISA_OP_FORWARD_PACKED: {
       PackedArena pa;
       st = packed_arena(p, &pa);
@@ -1104,20 +1158,88 @@ int pisa_bsa_bwd_packed(const pisa_params_t* p, const int32_t* cu_seqlens, int32
   if (st != PISA_OK) return st;
   g_mark_n = 0;
   const size_t es = elem_size(p->dtype);
-  for (int i = 0; i < nseq; ++i) {
+  auto run_alone = [&](int i, size_t wsb) -> int {
     const size_t t0 = (size_t)cu_seqlens[i];
     const int len = cu_seqlens[i + 1] - cu_seqlens[i];
-    if (len == 0) continue;
+    if (len == 0) return PISA_OK;
     pisa_params_t pi = *p;
     pi.N = len;
     Geometry gi;
-    st = resolve(&pi, &gi);
-    if (st != PISA_OK) return st;
+    const int r = resolve(&pi, &gi);
+    if (r != PISA_OK) return r;
     const size_t oq = t0 * g.Hq * g.d * es, ok = t0 * g.Hkv * g.d * es;
-    st = do_bwd(&pi, gi, (const char*)q + oq, (const char*)k + ok, (const char*)v + ok, idx + t0 * g.Hkv * g.K,
-                (const char*)out + oq, lse + t0 * g.Hq, (const char*)dout + oq, (char*)dq + oq, (char*)dk + ok,
-                (char*)dv + ok, ws, ws_bytes, s);
+    return do_bwd(&pi, gi, (const char*)q + oq, (const char*)k + ok, (const char*)v + ok, idx + t0 * g.Hkv * g.K,
+                  (const char*)out + oq, lse + t0 * g.Hq, (const char*)dout + oq, (char*)dq + oq, (char*)dk + ok,
+                  (char*)dv + ok, ws, wsb, s);
+  };
+  // With a workspace sized for PISA_OP_BSA_BWD_PACKED the short sequences run in the forward's padded groups (a
+  // padded query row gets idx = -1: it has no blocks and adds nothing to any key's gradient); with the smaller
+  // PISA_OP_BSA_BWD one, one sequence after the other.
+  PackedBwdArena pa;
+  const bool grouped = packed_bwd_arena(p, &pa) == PISA_OK && ws_bytes >= pa.total;
+  if (!grouped) {
+    for (int i = 0; i < nseq; ++i)
+      if ((st = run_alone(i, ws_bytes)) != PISA_OK) return st;
+    kernel_mark("end", s);
+    return PISA_OK;
+  }
+  std::unique_ptr<int[]> order(new (std::nothrow) int[(size_t)nseq + 1]);
+  std::unique_ptr<int32_t[]> group(new (std::nothrow) int32_t[(size_t)nseq + 1]);
+  std::unique_ptr<int32_t[]> padded(new (std::nothrow) int32_t[(size_t)nseq + 1]);
+  if (!order || !group || !padded) return PISA_ERR_INVALID_ARG;
+  packed_plan(p, cu_seqlens, nseq, pa.tokens, order.get(), group.get(), padded.get());
+  for (int i = 0; i < nseq; ++i)
+    if (group[i] < 0 && (st = run_alone(i, pa.bwd)) != PISA_OK) return st;
+  char* q_pad = (char*)ws + pa.bwd;
+  char* o_pad = q_pad + pa.qb;
+  char* do_pad = o_pad + pa.qb;
+  char* dq_pad = do_pad + pa.qb;
+  char* k_pad = dq_pad + pa.qb;
+  char* v_pad = k_pad + pa.kb;
+  char* dk_pad = v_pad + pa.kb;
+  char* dv_pad = dk_pad + pa.kb;
+  float* l_pad = (float*)(dv_pad + pa.kb);
+  int32_t* i_pad = (int32_t*)((char*)l_pad + pa.lb);
+  size_t n_short = 0;
+  for (int i = 0; i < nseq; ++i) {
+    const int len = cu_seqlens[i + 1] - cu_seqlens[i];
+    if (len > 0 && len <= kPackDirectLen) ++n_short;
+  }
+  size_t at = 0;
+  while (at < n_short) {
+    const int first = order[at];
+    if (group[first] < 0) { ++at; continue; }
+    size_t end = at + 1;
+    while (end < n_short && group[order[end]] == group[first]) ++end;
+    const int nb = (int)(end - at), np = padded[first];
+    pisa_params_t pg = *p;
+    pg.B = nb;
+    pg.N = np;
+    Geometry gg;
+    if ((st = resolve(&pg, &gg)) != PISA_OK) return st;
+    PackTable tab;
+    auto fill = [&](int b0) {
+      tab.n = nb - b0 < kPackSeqs ? nb - b0 : kPackSeqs;
+      for (int j = 0; j < tab.n; ++j) {
+        const int sq = order[at + (size_t)b0 + j];
+        tab.off[j] = cu_seqlens[sq];
+        tab.len[j] = cu_seqlens[sq + 1] - cu_seqlens[sq];
+      }
+    };
+    for (int b0 = 0; b0 < nb; b0 += kPackSeqs) {
+      fill(b0);
+      if ((st = launch_pack_gather(gg, (int)es, q, k, v, q_pad, k_pad, v_pad, tab, b0, s)) != PISA_OK) return st;
+      st = launch_pack_gather_bwd(gg, (int)es, out, dout, idx, lse, o_pad, do_pad, i_pad, l_pad, tab, b0, s);
+      if (st != PISA_OK) return st;
+    }
+    st = do_bwd(&pg, gg, q_pad, k_pad, v_pad, i_pad, o_pad, l_pad, do_pad, dq_pad, dk_pad, dv_pad, ws, pa.bwd, s);
     if (st != PISA_OK) return st;
+    for (int b0 = 0; b0 < nb; b0 += kPackSeqs) {
+      fill(b0);
+      st = launch_pack_scatter_grads(gg, (int)es, dq_pad, dk_pad, dv_pad, dq, dk, dv, tab, b0, s);
+      if (st != PISA_OK) return st;
+    }
+    at = end;
   }
   kernel_mark("end", s);
   return PISA_OK;

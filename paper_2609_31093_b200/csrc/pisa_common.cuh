@@ -78,6 +78,12 @@ int launch_pack_gather(const Geometry& g, int elem_bytes, const void* q, const v
 int launch_pack_scatter(const Geometry& g, int elem_bytes, const void* out_pad, const float* lse_pad,
                         const int32_t* idx_pad, void* out, float* lse, int32_t* idx, const PackTable& tab, int b_first,
                         cudaStream_t s);
+int launch_pack_gather_bwd(const Geometry& g, int elem_bytes, const void* out, const void* dout, const int32_t* idx,
+                           const float* lse, void* out_pad, void* dout_pad, int32_t* idx_pad, float* lse_pad,
+                           const PackTable& tab, int b_first, cudaStream_t s);
+int launch_pack_scatter_grads(const Geometry& g, int elem_bytes, const void* dq_pad, const void* dk_pad,
+                              const void* dv_pad, void* dq, void* dk, void* dv, const PackTable& tab, int b_first,
+                              cudaStream_t s);
 
 // decoding step (one token per sequence); ws points past the status word
 bool decode_supported(const Geometry& g, int dtype);

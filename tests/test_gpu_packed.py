@@ -42,7 +42,7 @@ def test_packed_sequences_equal_the_sequences_alone_and_the_oracle(op):
     torch.cuda.synchronize()
     assert P.read_status(ws) == 0
     launches[op] = P.launch_count() - n0
-    if len(launches) == 2:
+    if "packed" in launches and "forward" in launches:
         assert launches["packed"] < launches["forward"]
     for i, n in enumerate(lens):
         if n == 0:
@@ -76,11 +76,14 @@ def test_packed_sequences_equal_the_sequences_alone_and_the_oracle(op):
         assert n_bad == 0, i
 
 
-def test_packed_backward_matches_the_oracle_per_sequence():
+@pytest.mark.parametrize("op", ["loop", "groups"])
+def test_packed_backward_matches_the_oracle_per_sequence(op):
     """Forward then backward over a pack; every sequence's gradients against the oracle run on that sequence
-    alone with the indices the forward selected (one sequence is a single partial block, one a single token)."""
+    alone with the indices the forward selected (one sequence is a single partial block, two a single token).
+    "loop": a workspace sized for one sequence, one backward per sequence; "groups": the larger workspace, the
+    short sequences of similar length as padded batches (five groups here, the rest alone)."""
     from oracle import pisa_oracle as O
-    lens = [700, 64, 1, 1500, 0, 130, 37]
+    lens = [700, 64, 1, 1500, 0, 130, 37, 690, 650, 60, 1400, 1, 125, 33]
     Hq, Hkv, d, C, g, K = 8, 2, 128, 64, 2, 4
     cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
     total = int(cu[-1])
@@ -99,10 +102,16 @@ def test_packed_backward_matches_the_oracle_per_sequence():
     dout_bits = S.f32_to_bf16_bits(rng.standard_normal((total, Hq, d)).astype(np.float32))
     dout = T.to_torch(dout_bits, "bf16")
     dq, dk, dv = (torch.full_like(x, float("nan")) for x in (q, k, v))
-    wsb = PB.alloc_workspace(p, PB.OP_BSA_BWD)
+    group, _, n_groups = P.packed_plan(p, cu.tolist())
+    assert n_groups == 5 and sum(1 for x in group if x < 0) == 3
+    wsb = PB.alloc_workspace(p, PB.OP_BSA_BWD_PACKED if op == "groups" else PB.OP_BSA_BWD)
+    n0 = P.launch_count()
     P.pisa_bsa_bwd_packed(p, cu.tolist(), q, k, v, idx, out, lse, dout, dq, dk, dv, wsb)
     torch.cuda.synchronize()
+    launches["bwd_" + op] = P.launch_count() - n0
     assert P.read_status(ws) == 0 and P.read_status(wsb) == 0
+    if "bwd_loop" in launches and "bwd_groups" in launches:   # 13 backwards against 2 alone + 5 groups
+        assert launches["bwd_groups"] < launches["bwd_loop"], launches
     for i, n in enumerate(lens):
         if n == 0:
             continue
