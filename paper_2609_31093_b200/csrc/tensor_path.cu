@@ -1167,13 +1167,17 @@ __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int
   __shared__ int s_sel[4][kMaxK];
   __shared__ float s_cut[4][2];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long w = (long long)blockIdx.x * 4 + warp;
-  const long long total = (long long)geo.B * geo.Hkv * geo.N;
-  if (w >= total) return;
-  const int t = (int)(w % geo.N);
-  const int bh = (int)(w / geo.N);
+  // one warp per (b, KV head, token): blockIdx.y = the (b, KV head) unit, so no 64-bit division; the divisions
+  // by g and C are shifts where those are powers of two (the usual case)
+  const int t = blockIdx.x * 4 + warp;
+  if (t >= geo.N) return;
+  const int bh = blockIdx.y;
+  const long long w = (long long)bh * geo.N + t;
   const int K = geo.K, g = geo.g, gK = g * K, G = geo.G;
-  const int c = t / geo.C;
+  const int lgg = (g & (g - 1)) == 0 ? __ffs(g) - 1 : -1, lgC = (geo.C & (geo.C - 1)) == 0 ? __ffs(geo.C) - 1 : -1;
+  auto div_g = [&](int x) { return lgg >= 0 ? x >> lgg : x / g; };
+  auto mod_g = [&](int x) { return lgg >= 0 ? x & (g - 1) : x % g; };
+  const int c = lgC >= 0 ? t >> lgC : t / geo.C;
   const int f1 = (c >= 1) ? c - 1 : 0;
   const int32_t* pr = par + w * (long long)K;
   const float* bl = blk_lse + w * (long long)gK * G;
@@ -1190,9 +1194,9 @@ __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int
     const int ci = c0 + lane;
     bool ok = false;
     if (ci < gK) {
-      int p = pr[ci / g];
+      int p = pr[div_g(ci)];
       if ((geo.debug & PISA_DEBUG_BOUNDS) && p != -1 && !bounds_ok(p, geo.M[2], status)) p = -1;
-      const int leaf = p * g + ci % g;
+      const int leaf = p * g + mod_g(ci);
       ok = (p >= 0) && (leaf <= c);
       float sc = -CUDART_INF_F;
       if (ok) {
@@ -1243,7 +1247,7 @@ __global__ void __launch_bounds__(128) final_topk_kernel(Geometry geo, const int
     const unsigned bal = __ballot_sync(0xffffffffu, keep);
     kept_mask[ch] = bal;
     const int pos = base + __popc(bal & ((1u << lane) - 1u));
-    if (keep) s_sel[warp][pos] = pr[s / g] * g + s % g;
+    if (keep) s_sel[warp][pos] = pr[div_g(s)] * g + mod_g(s);
     if (keep && sel_lse != nullptr) {
       // the kept leaf's per-head scores ARE its per-head softmax denominators (LSE mode)
       const int bq = bh / geo.Hkv, hq = bh % geo.Hkv;
@@ -1620,6 +1624,7 @@ bool tensor_path_supported(const Geometry& g, int dtype) {
   if (nb != 128 && nb != 256) return false;
   if (g.L < 2 || g.N >= (1 << 24)) return false;
   if ((long long)g.B * g.Hkv * g.N * g.K >= (1LL << 31)) return false;   // entry offsets are int32
+  if ((long long)g.B * g.Hkv > 65535) return false;                      // the (b, KV head) unit is a grid's y index
   return true;
 }
 
@@ -1649,11 +1654,10 @@ int tensor_route(const Geometry& g, int dtype, const void* q, const void* k, con
   st = dispatch_tile_lse(g, g.g * g.C, a, inv.work_ctr, s);
   if (st != PISA_OK) return st;
   kernel_mark("final_topk", s);
-  const long long total = (long long)g.B * g.Hkv * g.N;
   // only the LSE scores are also the per-leaf softmax denominators the attention stage can reuse
   const bool lse_scores = g.score_mode == PISA_SCORE_LSE;
-  final_topk_kernel<<<(unsigned)((total + 3) / 4), 128, 0, s>>>(g, par, blk, idx, margin, lse_scores ? lse_out : nullptr,
-                                                                lse_scores ? sel_lse : nullptr, status);
+  final_topk_kernel<<<dim3((unsigned)((g.N + 3) / 4), (unsigned)(g.B * g.Hkv)), 128, 0, s>>>(
+      g, par, blk, idx, margin, lse_scores ? lse_out : nullptr, lse_scores ? sel_lse : nullptr, status);
   st = check_launch("final_topk");
   if (st != PISA_OK || sel_lse == nullptr || lse_scores) return st;
   // the other score modes rank by moments of the logits: the denominators take a pass of their own
@@ -1727,6 +1731,7 @@ bool tensor_bwd_supported(const Geometry& g, int dtype) {
   if (g.C != 64 && g.C != 128) return false;
   if (g.N >= (1 << 24)) return false;
   if ((long long)g.B * g.Hkv * g.N * g.K >= (1LL << 31)) return false;   // entry offsets are int32
+  if ((long long)g.B * g.Hkv > 65535) return false;                      // the (b, KV head) unit is a grid's y index
   return true;
 }
 size_t tensor_bwd_workspace_bytes(const Geometry& g) { return bwd_layout(g).total; }
