@@ -468,16 +468,24 @@ __device__ __forceinline__ bool prod_sync_or(bool flag) {
   return any != 0;
 }
 
+// query-ring stages of lse_ws_kernel: what 227 KB leave beside two key buffers and ~26 KB of static shared memory
+__host__ __device__ constexpr int lse_ws_stages(int D, int NB) {
+  return ((D / 64) * 128 * 128 * 4 + 2 * (D / 64) * NB * 128 + 27 * 1024 <= 227 * 1024) ? 4 : 2;
+}
+
 // MOM: false = per-head LSE of every leaf; true = first / second moments of the logits (score modes
 // "mean" and "mean + variance/2"), a separate instantiation so that the LSE one keeps its registers.
 template <int D, int NB, bool MOM>
 __global__ void __launch_bounds__(kLseThreads, 1)
 lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant__ CUtensorMap tm_k) {
   extern __shared__ uint8_t smem_raw[];
-  constexpr int NS = 4;
   constexpr int KS = D / 64;
   constexpr int A_SLAB = 128 * 128, B_SLAB = NB * 128;
   constexpr int A_STAGE = KS * A_SLAB;
+  // the node's keys are double-buffered (the next work item's keys load while this one's tiles run); the query
+  // ring gets what is left: four stages, two when the keys take 2 x 64 KB
+  constexpr int B_BUF = KS * B_SLAB;
+  constexpr int NS = lse_ws_stages(D, NB);
   constexpr uint32_t TM_COLS = (2 * NB < 32) ? 32 : 2 * NB;
   constexpr int R = kLseRing;
   // epilogue warps per tile: all sixteen on a 256-column accumulator; two groups of eight on alternate tiles
@@ -489,7 +497,7 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
   uint8_t* smem = align1024(smem_raw);
   uint8_t* sA = smem;
   uint8_t* sB = smem + NS * A_STAGE;
-  __shared__ uint64_t a_full[NS], a_empty[NS], b_full, b_empty, t_full[2], t_empty[2];
+  __shared__ uint64_t a_full[NS], a_empty[NS], b_full[2], b_empty[2], t_full[2], t_empty[2];
   __shared__ uint64_t m_full[R], m_empty[R];      // the tile ring: written by the scheduler warp, released by the epilogue
   __shared__ int s_tent[R][128];                  // a tile's entries (token | slot << 24, -1 = none)
   __shared__ int4 s_tkey[R];                      // its (unit, node, flags: 1 = first tile of a work item, 2 = last)
@@ -502,8 +510,7 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
   if (tid == 0) {
     s_total = 0x7fffffff;
     for (int i = 0; i < NS; ++i) { mbar_init(&a_full[i], kLseProd); mbar_init(&a_empty[i], 1); }
-    mbar_init(&b_empty, 1);
-    mbar_init(&b_full, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&b_empty[i], 1); mbar_init(&b_full[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 512 / GR); }
     for (int i = 0; i < R; ++i) { mbar_init(&m_full[i], 1); mbar_init(&m_empty[i], 16 / GR); }
     s_fail = 0;
@@ -541,12 +548,14 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
       const int4 key = s_tkey[mr];
       if (tid == 0 && (key.z & 1)) {
         // first tile of a work item: the node's keys, one TMA tile load per 64-wide slab (own memory, no
-        // multicast), once the previous item's MMAs have released the buffer
-        if (n_item > 0 && !mbar_wait_bounded(&b_empty, (uint32_t)((n_item - 1) & 1))) { s_fail = 1; break; }
+        // multicast), into the buffer the item before the previous one used, once its MMAs have released it
+        const int pb = n_item & 1;
+        if (n_item >= 2 && !mbar_wait_bounded(&b_empty[pb], (uint32_t)((n_item / 2 - 1) & 1))) { s_fail = 1; break; }
         ++n_item;
         const int b = key.x / geo.Hkv, h = key.x % geo.Hkv;
-        mbar_arrive_expect_tx(&b_full, (uint32_t)(KS * B_SLAB));
-        for (int ks = 0; ks < KS; ++ks) tma_load_4d(smem_u32(sB + ks * B_SLAB), &tm_k, &b_full, ks * 64, h, key.y * NB, b);
+        mbar_arrive_expect_tx(&b_full[pb], (uint32_t)B_BUF);
+        for (int ks = 0; ks < KS; ++ks)
+          tma_load_4d(smem_u32(sB + pb * B_BUF + ks * B_SLAB), &tm_k, &b_full[pb], ks * 64, h, key.y * NB, b);
       }
       if (it >= NS && !mbar_wait_bounded(&a_empty[s], (uint32_t)((it / NS - 1) & 1))) { s_fail = 1; break; }
       const int b = key.x / geo.Hkv, h = key.x % geo.Hkv;
@@ -574,7 +583,8 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
       if (!wait_tile(&m_full[mr], (uint32_t)((it / R) & 1), it)) break;
       const int flags = s_tkey[mr].z;
       bool ok = true;
-      if (flags & 1) ok = mbar_wait_bounded(&b_full, (uint32_t)(n_item & 1));                // the node's keys have landed
+      const int pb = n_item & 1;
+      if (flags & 1) ok = mbar_wait_bounded(&b_full[pb], (uint32_t)((n_item / 2) & 1));      // the node's keys have landed
       if (ok) ok = mbar_wait_bounded(&a_full[s], (uint32_t)((it / NS) & 1));
       if (ok && it >= 2) ok = mbar_wait_bounded(&t_empty[buf], (uint32_t)(((it >> 1) - 1) & 1));
       ok = __all_sync(0xffffffffu, ok);
@@ -582,7 +592,7 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
       if (lane == 0) {
         fence_proxy_async_smem();
         tcgen05_fence_after_sync();
-        const uint32_t a0 = smem_u32(sA + s * A_STAGE), b0 = smem_u32(sB);
+        const uint32_t a0 = smem_u32(sA + s * A_STAGE), b0 = smem_u32(sB + pb * B_BUF);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint64_t da = make_smem_desc(a0 + (kk >> 2) * A_SLAB + (kk & 3) * 32, 0, 1024);
@@ -591,7 +601,7 @@ lse_ws_kernel(Geometry geo, TileArgs a, int32_t* work_ctr, const __grid_constant
         }
         umma_commit(&a_empty[s]);
         umma_commit(&t_full[buf]);
-        if (flags & 2) umma_commit(&b_empty);        // last tile of the item: its MMAs release the keys
+        if (flags & 2) umma_commit(&b_empty[pb]);    // last tile of the item: its MMAs release the keys
       }
       if (flags & 2) ++n_item;
       __syncwarp();
@@ -1532,7 +1542,7 @@ int launch_tile_lse_m(const Geometry& g, const TileArgs& a, int32_t* work_ctr, c
       return PISA_ERR_CUDA;
     }
   }
-  const size_t smem = (size_t)(D / 64) * (4 * 128 * 128 + NB * 128) + 1024;
+  const size_t smem = (size_t)(D / 64) * (lse_ws_stages(D, NB) * 128 * 128 + 2 * NB * 128) + 1024;
   cudaError_t e = cudaFuncSetAttribute(lse_ws_kernel<D, NB, MOM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { record_cuda_error("lse_ws attr", e); return PISA_ERR_CUDA; }
   lse_ws_kernel<D, NB, MOM><<<num_sms(), kLseThreads, smem, s>>>(g, a, work_ctr, tm_k);
