@@ -88,3 +88,20 @@ def test_host_arena_size_covers_its_slots():
     slot = 2 * 8192 * G * 128 * es + 2 * 8192 * 128 * es + G * 8192 * 4 + 8192 * 16 * 4
     need = 4 * slot + 2 * P.pyramid_layout(unit)[3] + 2 * P.workspace_bytes(unit, PB.OP_FORWARD)
     assert P.workspace_bytes(p, PB.OP_FORWARD_HOST) >= need
+
+
+def test_packed_arena_sizes_cover_their_padded_tensors():
+    """The packed entry points run a group of short sequences as a padded batch of at most 32768 tokens held in the
+    workspace: the forward needs padded q, out, k, v, lse and idx beside a forward workspace and a pyramid, the
+    backward padded q, out, dout, dq, k, v, dk, dv, lse and idx beside a backward workspace.  The backward's arena
+    is refused (unsupported) where the backward itself is: fp32 inputs."""
+    p = P.Params(1, 4096, 8, 2, 128, 64, 2, 4)
+    es, tok = 2, 32768
+    qb, kb = tok * 8 * 128 * es, tok * 2 * 128 * es
+    lb, ib = tok * 8 * 4, tok * 2 * 4 * 4
+    fwd = P.workspace_bytes(p, PB.OP_FORWARD_PACKED)
+    assert fwd >= P.workspace_bytes(p, PB.OP_FORWARD) + 2 * qb + 2 * kb + lb + ib
+    bwd = P.workspace_bytes(p, PB.OP_BSA_BWD_PACKED)
+    assert bwd >= P.workspace_bytes(p, PB.OP_BSA_BWD) + 4 * qb + 4 * kb + lb + ib
+    with pytest.raises(P.PisaError):
+        P.workspace_bytes(P.Params(1, 4096, 8, 2, 32, 64, 2, 4, dtype="fp32"), PB.OP_BSA_BWD_PACKED)
