@@ -196,7 +196,7 @@ int pisa_forward(const pisa_params_t* p, const void* q, const void* k, const voi
  * past; the nodes on its own path are forced, not scored), so a sequence gives the same rows when it is
  * the head of a longer, zero-filled batch element.  Sequences of at most 8192 tokens are therefore
  * grouped by length (a group's members are no shorter than 3/4 of its padded length, padded lengths come
- * from the grid m * 2^k, m = 8..15, and a group holds at most 32768 padded tokens), copied into a padded
+ * from the grid 1, 2, .., 15, then m * 2^k with m = 8..15, and a group holds at most 32768 padded tokens and at most 65535 / Hkv sequences), copied into a padded
  * batch inside the workspace, run through ONE set of launches of the batched forward, and the valid rows
  * copied back.  Longer sequences, and groups of one, run unpadded on the packed tensors.  With a
  * workspace sized for PISA_OP_FORWARD only (too small for the padded copies) the call runs the sequences

@@ -613,7 +613,7 @@ int pisa_pyramid_layout(const pisa_params_t* p, int32_t* L, int32_t* M, int64_t*
 //
 // pisa_forward_packed groups the short sequences of a packed batch by length and runs every group as a
 // padded batch [B', N'] through one set of launches (the copies are in packed.cu).  N' comes from a fixed
-// grid (m * 2^k, m = 8..15: at most 12.5 % apart) so that the workspace can be sized from the parameters
+// grid (every length up to 15, then m * 2^k, m = 8..15: at most 12.5 % apart) so that the workspace can be sized from the parameters
 // alone; a group holds sequences no shorter than 3/4 of its N' and at most kPackTokens padded tokens
 // (more if the longest sequence is longer).  Sequences above kPackDirectLen, and groups of one, run
 // unpadded on the packed tensors themselves.
@@ -623,9 +623,16 @@ constexpr long long kPackTokens = 32768;
 static int pack_grid_len(int len) {
   int k = 0;
   while ((15LL << k) < len) ++k;
-  int m = (int)(((long long)len + (1LL << k) - 1) >> k);
-  if (m < 8) m = 8;
+  const int m = (int)(((long long)len + (1LL << k) - 1) >> k);      // 8..15 for k > 0; the length itself up to 15
   return m << k;
+}
+
+// sequences one group of padded length np may hold: kPackTokens padded tokens, and (batch, KV head) units that
+// still index a grid's y dimension
+static long long pack_group_cap(const pisa_params_t* p, long long tokens, long long np) {
+  long long b = tokens / np < 1 ? 1 : tokens / np;
+  if (b * p->Hkv > 65535) b = 65535 / p->Hkv;
+  return b < 1 ? 1 : b;
 }
 
 struct PackedArena {
@@ -651,12 +658,12 @@ static int packed_arena(const pisa_params_t* p, PackedArena* a) {
   if (st != PISA_OK) return st;
   const int n_max = p->N < kPackDirectLen ? p->N : kPackDirectLen;
   for (int k = 0; k < 31; ++k)
-    for (int m = 8; m <= 15; ++m) {
+    for (int m = (k == 0) ? 1 : 8; m <= 15; ++m) {
       const long long np = (long long)m << k;
       if (np > pack_grid_len(n_max)) continue;
       pisa_params_t pg = *p;
       pg.N = (int)np;
-      pg.B = (int)(a->tokens / np < 1 ? 1 : a->tokens / np);
+      pg.B = (int)pack_group_cap(p, a->tokens, np);
       Geometry gg;
       if ((st = resolve(&pg, &gg)) != PISA_OK) return st;
       const size_t f = forward_ws_bytes(&pg, gg, &st);
@@ -702,12 +709,12 @@ static int packed_bwd_arena(const pisa_params_t* p, PackedBwdArena* a) {
   if ((st = need(p, g, &bwd)) != PISA_OK) return st;
   const int n_max = p->N < kPackDirectLen ? p->N : kPackDirectLen;
   for (int k = 0; k < 31; ++k)
-    for (int m = 8; m <= 15; ++m) {
+    for (int m = (k == 0) ? 1 : 8; m <= 15; ++m) {
       const long long np = (long long)m << k;
       if (np > pack_grid_len(n_max)) continue;
       pisa_params_t pg = *p;
       pg.N = (int)np;
-      pg.B = (int)(a->tokens / np < 1 ? 1 : a->tokens / np);
+      pg.B = (int)pack_group_cap(p, a->tokens, np);
       Geometry gg;
       if ((st = resolve(&pg, &gg)) != PISA_OK) return st;
       size_t b = 0;
@@ -742,7 +749,7 @@ static int packed_plan(const pisa_params_t* p, const int32_t* cu, int nseq, long
   size_t at = 0;
   while (at < n_short) {
     const int np = pack_grid_len(cu[order[at] + 1] - cu[order[at]]);
-    const long long b_cap = tokens / np < 1 ? 1 : tokens / np;
+    const long long b_cap = pack_group_cap(p, tokens, np);
     size_t end = at + 1;
     while (end < n_short && (long long)(end - at) < b_cap) {
       const int len = cu[order[end] + 1] - cu[order[end]];
@@ -755,7 +762,6 @@ static int packed_plan(const pisa_params_t* p, const int32_t* cu, int nseq, long
     }
     at = end;
   }
-  (void)p;
   return n_groups;
 }
 

@@ -1,6 +1,6 @@
 """Host logic of pisa_forward_packed's grouping (no GPU): which sequences share a padded batch.  The rules,
 from the header: only sequences of 1 .. 8192 tokens are grouped; a group's padded length is the smallest
-m * 2^k (m = 8..15) that holds its longest member; every member is at least 3/4 of it; a group holds at
+m * 2^k (m = 8..15; below 16 every length is on the grid) that holds its longest member; every member is at least 3/4 of it; a group holds at
 most 32768 padded tokens (at least one sequence); a group of one runs alone."""
 import numpy as np
 import pytest
@@ -12,7 +12,7 @@ def _grid(n):
     k = 0
     while (15 << k) < n:
         k += 1
-    return max(8, -(-n // (1 << k))) << k
+    return -(-n // (1 << k)) << k
 
 
 def _plan(lens, N=None):
@@ -76,3 +76,15 @@ def test_argument_errors():
         P.packed_plan(p, [1, 5])                                            # cu[0] != 0
     with pytest.raises(Exception):
         P.packed_plan(p, [0, 10, 5])                                        # negative length
+
+
+def test_group_size_is_capped_by_the_kv_head_count():
+    """A group's (sequence, KV head) units index a grid dimension: at most 65535 / Hkv sequences per group."""
+    lens = [8] * 5000
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64).tolist()
+    for Hkv, cap in ((2, 4096), (16, 4095), (32, 2047)):          # 32768 / 8 = 4096 sequences by the token rule
+        p = P.Params(1, 8, 2 * Hkv, Hkv, 128, 64, 2, 4, dtype="bf16")
+        group, padded, n_groups = P.packed_plan(p, cu)
+        sizes = np.bincount(np.asarray(group))
+        assert sizes.max() == cap and n_groups == -(-5000 // cap), (Hkv, sizes.max(), n_groups)
+        assert set(padded) == {8}
